@@ -1,0 +1,202 @@
+"""CPU oracle for the SPICE MoE-layer forward -- TEST INFRASTRUCTURE, not product code.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
+It wraps `spice_oracle.c` (plain fp64 loops, see that file's header for the passages it
+follows and the readings taken) through ctypes.  It imports nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "spice_oracle.c")
+_LIB = os.path.join(_HERE, "libspice_oracle.so")
+
+HIT, MISS_EXACT, LOWCONF = 0, 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (-O2, OpenMP).  Returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Cfg(C.Structure):
+    _fields_ = [("d", C.c_int32), ("n_experts", C.c_int32), ("top_k", C.c_int32), ("inter", C.c_int32),
+                ("inter_shared", C.c_int32), ("lore_rank", C.c_int32), ("norm_topk", C.c_int32),
+                ("conf_stride", C.c_int32), ("tau", C.c_float)]
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.oracle_layer.restype = C.c_int
+        _lib.oracle_swiglu_ffn.restype = C.c_int
+        _lib.oracle_lore_delta.restype = C.c_int
+        _lib.oracle_num_threads.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+@dataclass
+class LayerResult:
+    logits: np.ndarray        # [T,N] f64
+    idx: np.ndarray           # [T,K] i32, decreasing logit
+    gate: np.ndarray          # [T,K] f64
+    cls: np.ndarray           # [T,K] u8  (0 HIT, 1 MISS_EXACT, 2 LOWCONF)
+    counts: np.ndarray        # [3] i32
+    resid_tok: np.ndarray     # [n_resid] i32, (t,k) order
+    resid_k: np.ndarray
+    resid_expert: np.ndarray
+    resid_gate: np.ndarray    # f64
+    y: Optional[np.ndarray]        # [rows,d] f64 (GPU part of the layer output)
+    y_full: Optional[np.ndarray]   # [rows,d] f64 (with the exact-recovery terms added)
+    rows: np.ndarray          # token index of every row of y
+
+
+def router_logits(h, w_router) -> np.ndarray:
+    h, w = _f32(h), _f32(w_router)
+    T, d = h.shape
+    N = w.shape[0]
+    out = np.empty((T, N), dtype=np.float64)
+    _load().oracle_router_logits(C.c_int(T), C.c_int(d), C.c_int(N), _p(h), _p(w), _p(out))
+    return out
+
+
+def topk_gates(logits, K: int, norm_topk: int = 1):
+    l = np.ascontiguousarray(logits, dtype=np.float64)
+    T, N = l.shape
+    idx = np.empty((T, K), dtype=np.int32)
+    gate = np.empty((T, K), dtype=np.float64)
+    _load().oracle_topk_gates(C.c_int(T), C.c_int(N), C.c_int(K), C.c_int(norm_topk), _p(l), _p(idx), _p(gate))
+    return idx, gate
+
+
+def classify(idx, resident, conf, tau: float, conf_stride: Optional[int] = None):
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    T, K = idx.shape
+    res = np.ascontiguousarray(resident, dtype=np.uint8)
+    N = res.shape[0]
+    conf = _f32(conf)
+    if conf_stride is None:
+        conf_stride = 0 if conf.ndim == 1 else N
+    cls = np.empty((T, K), dtype=np.uint8)
+    counts = np.zeros(3, dtype=np.int32)
+    _load().oracle_classify(C.c_int(T), C.c_int(N), C.c_int(K), _p(idx), _p(res), _p(conf),
+                            C.c_int(conf_stride), C.c_float(tau), _p(cls), _p(counts))
+    return cls, counts
+
+
+def swiglu_ffn(w_gate, w_up, w_down, x) -> np.ndarray:
+    wg, wu, wd, x = _f32(w_gate), _f32(w_up), _f32(w_down), _f32(x)
+    I, d = wg.shape
+    assert wu.shape == (I, d) and wd.shape == (d, I) and x.shape == (d,)
+    out = np.empty(d, dtype=np.float64)
+    rc = _load().oracle_swiglu_ffn(C.c_int(d), C.c_int(I), _p(wg), _p(wu), _p(wd), _p(x), _p(out))
+    assert rc == 0
+    return out
+
+
+def lore_delta(A, B, x) -> np.ndarray:
+    A, B, x = _f32(A), _f32(B), _f32(x)
+    r, d = A.shape
+    assert B.shape == (d, r) and x.shape == (d,)
+    out = np.empty(d, dtype=np.float64)
+    rc = _load().oracle_lore_delta(C.c_int(d), C.c_int(r), _p(A), _p(B), _p(x), _p(out))
+    assert rc == 0
+    return out
+
+
+def layer(*, h, w_router, experts, shared, lore_A, lore_B, resident, conf, top_k: int, tau: float,
+          norm_topk: int = 1, conf_stride: Optional[int] = None, tokens: Optional[Sequence[int]] = None,
+          want_full: bool = True, skip_ffn: bool = False) -> LayerResult:
+    """Evaluate one layer.
+
+    experts: dict {e: (w_gate [I,d], w_up [I,d], w_down [d,I])} or a list of N such tuples;
+             experts that are never evaluated may be absent.
+    shared:  (s_gate [I_s,d], s_up [I_s,d], s_down [d,I_s]).
+    tokens:  evaluate y / y_full only for these token indices (routing is always done for all).
+    skip_ffn: routing + classification only (y, y_full are None).
+    """
+    h, w_router = _f32(h), _f32(w_router)
+    T, d = h.shape
+    N = w_router.shape[0]
+    K = top_k
+    resident = np.ascontiguousarray(resident, dtype=np.uint8)
+    conf = _f32(conf)
+    if conf_stride is None:
+        conf_stride = 0 if conf.ndim == 1 else N
+    sg, su, sd = (_f32(a) for a in shared)
+    Is = sg.shape[0]
+    lore_A, lore_B = _f32(lore_A), _f32(lore_B)
+    r = lore_A.shape[1]
+    if isinstance(experts, dict):
+        items = experts
+    else:
+        items = {e: w for e, w in enumerate(experts) if w is not None}
+    keep = []
+    PA = C.c_void_p * N
+    pg, pu, pd = PA(), PA(), PA()
+    I = None
+    for e, (g, u, w) in items.items():
+        g, u, w = _f32(g), _f32(u), _f32(w)
+        keep.append((g, u, w))
+        I = g.shape[0]
+        assert g.shape == (I, d) and u.shape == (I, d) and w.shape == (d, I)
+        pg[e], pu[e], pd[e] = g.ctypes.data, u.ctypes.data, w.ctypes.data
+    if I is None:
+        I = 1
+    cfg = _Cfg(d, N, K, I, Is, r, norm_topk, conf_stride, tau)
+    if skip_ffn:
+        sel = np.zeros(1, dtype=np.int32)   # non-NULL pointer, zero rows
+    elif tokens is None:
+        sel = np.arange(T, dtype=np.int32)
+    else:
+        sel = np.ascontiguousarray(tokens, dtype=np.int32)
+    rows = 0 if skip_ffn else sel.shape[0]
+    logits = np.empty((T, N), dtype=np.float64)
+    idx = np.empty((T, K), dtype=np.int32)
+    gate = np.empty((T, K), dtype=np.float64)
+    cls = np.empty((T, K), dtype=np.uint8)
+    counts = np.zeros(3, dtype=np.int32)
+    n_resid = C.c_int32(0)
+    rt = np.empty(T * K, dtype=np.int32)
+    rk = np.empty(T * K, dtype=np.int32)
+    re_ = np.empty(T * K, dtype=np.int32)
+    rg = np.empty(T * K, dtype=np.float64)
+    y = np.zeros((rows, d), dtype=np.float64)
+    yf = np.zeros((rows, d), dtype=np.float64) if want_full else None
+    rc = _load().oracle_layer(
+        C.byref(cfg), C.c_int(T), _p(h), _p(w_router), pg, pu, pd, _p(sg), _p(su), _p(sd),
+        _p(lore_A), _p(lore_B), _p(resident), _p(conf), C.c_int(rows), _p(sel),
+        _p(logits), _p(idx), _p(gate), _p(cls), _p(counts), C.byref(n_resid),
+        _p(rt), _p(rk), _p(re_), _p(rg), _p(y), _p(yf) if yf is not None else None)
+    if rc != 0:
+        raise RuntimeError(f"oracle_layer failed with code {rc} (-(e+1): weights of expert e missing)")
+    n = n_resid.value
+    return LayerResult(logits, idx, gate, cls, counts, rt[:n].copy(), rk[:n].copy(), re_[:n].copy(),
+                       rg[:n].copy(), None if skip_ffn else y, None if (skip_ffn or yf is None) else yf, sel[:rows])

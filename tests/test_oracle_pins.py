@@ -1,0 +1,320 @@
+"""Pins for the CPU oracle: it is checked against things other than itself -- brute-force
+dense evaluation through an independent numpy path, invariants, closed forms, special
+cases that reduce to the textbook MoE layer, and a hand-computed example."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_21240_b200 import workloads as W
+from tests._cases import enforce_margins
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ independent numpy path
+def np_silu(v):
+    return v / (1.0 + np.exp(-v))
+
+
+def np_ffn(wg, wu, wd, X):
+    """SwiGLU FFN for a batch, all in fp64 numpy matmuls.  X: [T,d] -> [T,d]."""
+    X = X.astype(np.float64)
+    a = np_silu(X @ wg.astype(np.float64).T) * (X @ wu.astype(np.float64).T)
+    return a @ wd.astype(np.float64).T
+
+
+def np_dense_gates(h, w_router, K, norm_topk=1):
+    """Dense [T,N] gate matrix built by sorting full-softmax probabilities."""
+    logits = h.astype(np.float64) @ w_router.astype(np.float64).T
+    z = logits - logits.max(axis=1, keepdims=True)
+    p = np.exp(z)
+    p /= p.sum(axis=1, keepdims=True)
+    order = np.argsort(-p, axis=1, kind="stable")[:, :K]
+    G = np.zeros_like(p)
+    for t in range(h.shape[0]):
+        sel = order[t]
+        G[t, sel] = p[t, sel] / p[t, sel].sum() if norm_topk else p[t, sel]
+    return G, order
+
+
+def tiny(T=4, variant=0, **kw):
+    s = W.scaled_shape(W.SHAPES["tiny"], **kw) if kw else W.SHAPES["tiny"]
+    wl = W.make_layer(s, T, variant=variant)
+    enforce_margins(wl)
+    return wl
+
+
+def run(wl, resident=None, conf=None, lore=None, tau=None, norm_topk=1, tokens=None):
+    s = wl.shape
+    A, B = wl.lore() if lore is None else lore
+    return oracle.layer(h=wl.h, w_router=wl.w_router, experts=[wl.expert(e) for e in range(s.n_experts)],
+                        shared=wl.shared(), lore_A=A, lore_B=B,
+                        resident=wl.resident if resident is None else resident,
+                        conf=wl.conf if conf is None else conf, top_k=s.top_k,
+                        tau=s.tau if tau is None else tau, norm_topk=norm_topk, tokens=tokens)
+
+
+def dense_layer(wl, norm_topk=1):
+    s = wl.shape
+    G, order = np_dense_gates(wl.h, wl.w_router, s.top_k, norm_topk)
+    y = np_ffn(*wl.shared(), wl.h)
+    for e in range(s.n_experts):
+        y = y + G[:, [e]] * np_ffn(*wl.expert(e), wl.h)
+    return y, G, order
+
+
+def rel(a, b):
+    return np.abs(a - b).max() / max(np.abs(b).max(), 1e-30)
+
+
+# ------------------------------------------------------------------ P1 brute force
+@pytest.mark.parametrize("variant,norm_topk", [(0, 1), (1, 1), (2, 0)])
+def test_p1_all_resident_equals_bruteforce_dense(variant, norm_topk):
+    wl = tiny(T=5, variant=variant)
+    res = run(wl, resident=np.ones(wl.shape.n_experts, np.uint8), norm_topk=norm_topk)
+    y, G, order = dense_layer(wl, norm_topk)
+    assert rel(res.y, y) < 1e-9
+    assert rel(res.y_full, y) < 1e-9
+    assert (res.idx == order).all()
+    assert res.counts.tolist() == [wl.T * wl.shape.top_k, 0, 0] and res.resid_tok.size == 0
+
+
+def test_router_logits_match_numpy_matmul():
+    wl = tiny(T=7)
+    ref = wl.h.astype(np.float64) @ wl.w_router.astype(np.float64).T
+    assert np.abs(oracle.router_logits(wl.h, wl.w_router) - ref).max() < 1e-12
+
+
+def test_ffn_and_lore_match_numpy():
+    wl = tiny(T=3)
+    for e in (0, 3):
+        ref = np_ffn(*wl.expert(e), wl.h[1:2])[0]
+        assert rel(oracle.swiglu_ffn(*wl.expert(e), wl.h[1]), ref) < 1e-10
+    A, B = wl.lore()
+    ref = B[2].astype(np.float64) @ (A[2].astype(np.float64) @ wl.h[0].astype(np.float64))
+    assert rel(oracle.lore_delta(A[2], B[2], wl.h[0]), ref) < 1e-10
+    # a transposed operand would give the wrong shape/values: asymmetric check
+    wg, wu, wd = wl.expert(1)
+    assert rel(oracle.swiglu_ffn(wg, wu, wd, wl.h[0]), np_ffn(wu, wg, wd, wl.h[0:1])[0]) > 1e-3
+
+
+# ------------------------------------------------------------------ P2 gate invariants
+@pytest.mark.parametrize("K", [1, 2, 3, 8])
+def test_p2_gate_invariants(K):
+    rng = np.random.default_rng(5)
+    logits = rng.normal(size=(9, 8)) * 2.0
+    idx, gate = oracle.topk_gates(logits, K, 1)
+    assert np.allclose(gate.sum(axis=1), 1.0, atol=1e-12)
+    assert (gate > 0).all() and (np.diff(gate, axis=1) <= 1e-15).all()
+    for t in range(9):
+        assert len(set(idx[t])) == K and idx[t].min() >= 0 and idx[t].max() < 8
+        assert (np.sort(logits[t])[::-1][:K] == logits[t, idx[t]]).all()
+    if K == 8:   # K = N: gates are the full softmax
+        p = np.exp(logits - logits.max(1, keepdims=True))
+        p /= p.sum(1, keepdims=True)
+        assert np.allclose(np.take_along_axis(p, idx, 1), gate, atol=1e-13)
+    if K == 1:
+        assert (gate == 1.0).all()
+    # shift invariance
+    idx2, gate2 = oracle.topk_gates(logits + 3.25, K, 1)
+    assert (idx2 == idx).all() and np.allclose(gate2, gate, atol=1e-13)
+    # un-normalised variant = full softmax probabilities of the winners
+    idx3, gate3 = oracle.topk_gates(logits, K, 0)
+    p = np.exp(logits - logits.max(1, keepdims=True))
+    p /= p.sum(1, keepdims=True)
+    assert (idx3 == idx).all() and np.allclose(np.take_along_axis(p, idx, 1), gate3, atol=1e-13)
+
+
+def test_topk_ties_prefer_lower_index():
+    logits = np.array([[1.0, 3.0, 3.0, 0.5, 3.0, 2.0]])
+    idx, gate = oracle.topk_gates(logits, 4, 1)
+    assert idx.tolist() == [[1, 2, 4, 5]]
+
+
+# ------------------------------------------------------------------ P3 all-hit = textbook MoE
+def test_p3_all_hit_ignores_conf_tau_lore():
+    wl = tiny(T=4)
+    ones = np.ones(wl.shape.n_experts, np.uint8)
+    base = run(wl, resident=ones)
+    A, B = wl.lore()
+    other = run(wl, resident=ones, conf=np.zeros_like(wl.conf), tau=2.0, lore=(A * 3, B * -2))
+    assert np.array_equal(base.y, other.y) and other.counts[2] == 0
+
+
+# ------------------------------------------------------------------ P4 rank-sufficient LoRE
+def test_p4_rank_sufficient_lore_reproduces_exact_expert():
+    wl = tiny(T=4)
+    s = wl.shape
+    H = wl.h.astype(np.float64).T                      # [d,T]
+    Hp = np.linalg.pinv(H)                             # [T,d], Hp @ H = I_T
+    SH = np_ffn(*wl.shared(), wl.h).T                  # [d,T]
+    A = np.zeros((s.n_experts, s.lore_rank, s.d))
+    B = np.zeros((s.n_experts, s.d, s.lore_rank))
+    for e in range(s.n_experts):
+        A[e, : wl.T] = Hp
+        B[e, :, : wl.T] = np_ffn(*wl.expert(e), wl.h).T - SH
+    # fp32 storage of A,B costs ~1e-7 relative; keep fp64 by calling with float32 copies and loose bound
+    all_hit = run(wl, resident=np.ones(s.n_experts, np.uint8))
+    for mask_seed in range(3):
+        rng = np.random.default_rng(mask_seed)
+        resident = (rng.random(s.n_experts) < 0.4).astype(np.uint8)
+        res = run(wl, resident=resident, conf=np.zeros_like(wl.conf), tau=0.5, lore=(A, B))
+        assert res.counts[1] == 0 and res.counts[2] > 0
+        assert rel(res.y, all_hit.y) < 2e-5
+    none = run(wl, resident=np.zeros(s.n_experts, np.uint8), conf=np.zeros_like(wl.conf), tau=0.5, lore=(A, B))
+    assert none.counts.tolist() == [0, 0, wl.T * s.top_k]
+    assert rel(none.y, all_hit.y) < 2e-5
+
+
+def test_p4b_identity_lore_full_rank():
+    """r = d, A = I: B A h = B h, so a linear 'expert minus shared' map is reproduced exactly."""
+    s = W.scaled_shape(W.SHAPES["tiny"], d=32, inter=16, inter_shared=16, lore_rank=32)
+    wl = W.make_layer(s, 3)
+    enforce_margins(wl)
+    rng = np.random.default_rng(0)
+    Bm = rng.normal(size=(s.n_experts, s.d, s.d)).astype(np.float32)
+    A = np.broadcast_to(np.eye(s.d, dtype=np.float32), (s.n_experts, s.d, s.d)).copy()
+    res = run(wl, resident=np.zeros(s.n_experts, np.uint8), conf=np.zeros_like(wl.conf), tau=0.5, lore=(A, Bm))
+    S = np_ffn(*wl.shared(), wl.h)
+    exp = np.zeros_like(S)
+    for t in range(wl.T):
+        exp[t] = S[t]
+        for k in range(s.top_k):
+            e = res.idx[t, k]
+            exp[t] += res.gate[t, k] * (S[t] + Bm[e].astype(np.float64) @ wl.h[t].astype(np.float64))
+    assert rel(res.y, exp) < 1e-10
+
+
+# ------------------------------------------------------------------ P5 / P6 closed forms
+def test_p5_all_miss_high_conf_gives_shared_only():
+    wl = tiny(T=4)
+    s = wl.shape
+    res = run(wl, resident=np.zeros(s.n_experts, np.uint8), conf=np.ones_like(wl.conf), tau=0.5)
+    S = np_ffn(*wl.shared(), wl.h)
+    assert rel(res.y, S) < 1e-10
+    assert res.resid_tok.size == wl.T * s.top_k and res.counts.tolist() == [0, wl.T * s.top_k, 0]
+    dense, _, _ = dense_layer(wl)
+    assert rel(res.y_full, dense) < 1e-9
+    # residual list is in (t,k) order and carries the routing
+    assert (res.resid_tok == np.repeat(np.arange(wl.T), s.top_k)).all()
+    assert (res.resid_k == np.tile(np.arange(s.top_k), wl.T)).all()
+    assert (res.resid_expert == res.idx.ravel()).all() and np.array_equal(res.resid_gate, res.gate.ravel())
+
+
+def test_p6_all_miss_low_conf_zero_lore_gives_twice_shared():
+    wl = tiny(T=4)
+    s = wl.shape
+    A, B = wl.lore()
+    res = run(wl, resident=np.zeros(s.n_experts, np.uint8), conf=np.zeros_like(wl.conf), tau=0.5,
+              lore=(A * 0, B * 0))
+    S = np_ffn(*wl.shared(), wl.h)
+    assert rel(res.y, 2 * S) < 1e-10
+    assert res.resid_tok.size == 0
+
+
+# ------------------------------------------------------------------ P7 threshold edges
+def test_p7_threshold_edges():
+    idx = np.array([[0, 1, 2, 3]], dtype=np.int32)
+    resident = np.array([1, 0, 0, 0], np.uint8)
+    tau = np.float32(0.6)
+    conf = np.array([[0.0, tau, np.nextafter(tau, np.float32(0)), np.nan]], dtype=np.float32)
+    cls, counts = oracle.classify(idx, resident, conf, float(tau))
+    assert cls.tolist() == [[oracle.HIT, oracle.MISS_EXACT, oracle.LOWCONF, oracle.MISS_EXACT]]
+    assert counts.tolist() == [1, 2, 1]
+    cls0, _ = oracle.classify(idx, resident, np.abs(np.nan_to_num(conf)), 0.0)
+    assert (cls0[0, 1:] == oracle.MISS_EXACT).all()           # tau = 0: nothing is low-confidence
+    cls2, _ = oracle.classify(idx, resident, np.nan_to_num(conf), 1.5)
+    assert (cls2[0, 1:] == oracle.LOWCONF).all()              # tau > 1: every miss is
+    # one scalar confidence per token (conf_stride = 0)
+    cls3, _ = oracle.classify(np.array([[1, 2], [1, 2]], np.int32), resident, np.array([0.1, 0.9], np.float32), 0.6)
+    assert cls3.tolist() == [[oracle.LOWCONF] * 2, [oracle.MISS_EXACT] * 2]
+
+
+# ------------------------------------------------------------------ P8 linearity
+def test_p8_lore_term_is_linear_and_residual_is_exact_sum():
+    wl = tiny(T=4, variant=3)
+    s = wl.shape
+    A, B = wl.lore()
+    r1 = run(wl)
+    r0 = run(wl, lore=(A, B * 0))
+    r3 = run(wl, lore=(A, B * 3))
+    assert r1.counts[2] > 0 and r1.counts[1] > 0 and r1.counts[0] > 0
+    assert rel(r3.y - r0.y, 3 * (r1.y - r0.y)) < 1e-9
+    extra = np.zeros_like(r1.y)
+    for t, k, e, g in zip(r1.resid_tok, r1.resid_k, r1.resid_expert, r1.resid_gate):
+        assert r1.idx[t, k] == e and r1.cls[t, k] == oracle.MISS_EXACT
+        extra[t] += g * np_ffn(*wl.expert(e), wl.h[t:t + 1])[0]
+    assert rel(r1.y_full - r1.y, extra) < 1e-9
+
+
+# ------------------------------------------------------------------ P9 symmetries
+def test_p9_token_permutation_and_batch_independence():
+    wl = tiny(T=5, variant=1)
+    full = run(wl)
+    for t in range(wl.T):
+        one = oracle.layer(h=wl.h[t:t + 1], w_router=wl.w_router,
+                           experts=[wl.expert(e) for e in range(wl.shape.n_experts)], shared=wl.shared(),
+                           lore_A=wl.lore()[0], lore_B=wl.lore()[1], resident=wl.resident,
+                           conf=wl.conf[t:t + 1], top_k=wl.shape.top_k, tau=wl.shape.tau)
+        assert np.array_equal(one.y[0], full.y[t]) and (one.idx[0] == full.idx[t]).all()
+    sub = run(wl, tokens=[3, 1])
+    assert np.array_equal(sub.y, full.y[[3, 1]]) and np.array_equal(sub.y_full, full.y_full[[3, 1]])
+
+
+def test_p9_expert_relabelling():
+    wl = tiny(T=4, variant=2)
+    s = wl.shape
+    base = run(wl)
+    perm = np.random.default_rng(1).permutation(s.n_experts)      # new expert j = old expert perm[j]
+    A, B = wl.lore()
+    res = oracle.layer(h=wl.h, w_router=wl.w_router[perm], experts=[wl.expert(int(perm[j])) for j in range(s.n_experts)],
+                       shared=wl.shared(), lore_A=A[perm], lore_B=B[perm], resident=wl.resident[perm],
+                       conf=wl.conf[:, perm], top_k=s.top_k, tau=s.tau)
+    assert (perm[res.idx] == base.idx).all() and (res.cls == base.cls).all()
+    assert rel(res.y, base.y) < 1e-12
+
+
+# ------------------------------------------------------------------ P10 closed forms
+def test_p10_zero_input_gives_zero_output():
+    wl = tiny(T=2)
+    wl.h[:] = 0
+    res = run(wl)
+    assert np.abs(res.y).max() == 0.0
+
+
+def test_p10_hand_computed_example():
+    rows = []
+    with open(os.path.join(GOLD, "swiglu_hand_example.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].split()
+            if len(line) == 4:
+                rows.append((line[0], int(line[1]), float(line[2]), float(line[3])))
+    assert len(rows) == 5
+    h = np.array([[1.0, 2.0]], np.float32)
+    wr = np.eye(2, dtype=np.float32)
+    e1 = (np.array([[1, 0.5]], np.float32), np.array([[0.5, 0.25]], np.float32), np.array([[2], [-1]], np.float32))
+    e0 = (np.array([[-1, 0.5]], np.float32), np.array([[1, 1]], np.float32), np.array([[1], [3]], np.float32))
+    sh = (np.array([[1, 0]], np.float32), np.array([[0, 1]], np.float32), np.array([[1], [1]], np.float32))
+    A = np.array([[[9, 9]], [[1, 1]]], np.float32)
+    B = np.array([[[9], [9]], [[0.5], [-0.5]]], np.float32)
+    for case, norm, y0, y1 in rows:
+        resident = np.array([0, 1 if case == "hit" else 0], np.uint8)
+        conf = np.array([[0.9, 0.1 if case == "lowconf" else 0.9]], np.float32)
+        res = oracle.layer(h=h, w_router=wr, experts=[e0, e1], shared=sh, lore_A=A, lore_B=B, resident=resident,
+                           conf=conf, top_k=1, tau=0.5, norm_topk=norm)
+        assert res.idx.tolist() == [[1]]
+        assert np.allclose(res.y[0], [y0, y1], rtol=0, atol=1e-14), (case, norm, res.y)
+        assert res.resid_tok.size == (1 if case == "exact" else 0)
+
+
+# ------------------------------------------------------------------ P12 y_full vs dense
+@pytest.mark.parametrize("seed", [0, 1])
+def test_p12_y_full_equals_dense_when_nothing_is_substituted(seed):
+    wl = tiny(T=4, variant=seed)
+    resident = (np.random.default_rng(seed).random(wl.shape.n_experts) < 0.5).astype(np.uint8)
+    res = run(wl, resident=resident, tau=0.0)
+    assert res.counts[2] == 0 and res.counts[1] > 0
+    dense, _, _ = dense_layer(wl)
+    assert rel(res.y_full, dense) < 1e-9
