@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE-layer decode step (spice_moe_layer_fwd) on B200.
+
+One step = one pass of the whole hot path (route, classify, grouped expert FFN over the
+resident slots, shared expert + LoRE surrogate, combine) over one decode batch of a
+DeepSeek-V2-Lite-shaped layer.  Successive steps rotate through several independent
+layer weight sets so that the bytes touched between two uses of the same weights are
+several times the L2 capacity (cold-L2 timing without a flush inside the timed region).
+
+Prints ONE JSON line (see README for the keys).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moe_layer_decode_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as f:
+                d = json.load(f)
+            return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]), "source": "measured"}
+        except Exception:
+            pass
+    return {**FALLBACK_PEAKS, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks sampler
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                try:
+                    self.samples.append((time.time(), float(parts[0]), float(parts[1]), parts[2:6]))
+                except ValueError:
+                    pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        win = [s for s in self.samples if t0 <= s[0] <= t1]
+        where = "timed region"
+        if not win:
+            win = self.samples[-5:]
+            where = "nearest samples (timed region shorter than the sampling period)"
+        if not win:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "none"}
+        reasons = sorted({n for s in win for n, v in zip(names, s[3]) if v.lower().startswith("active")})
+        return {"sm_mhz": float(np.median([s[1] for s in win])), "sm_max_mhz": float(max(s[2] for s in win)),
+                "reasons": reasons, "samples": len(win), "window": where}
+
+
+# ----------------------------------------------------------------------------- workload
+def algorithmic_bytes(shape, T, idx, cls):
+    """Bytes the method must move for one layer call (bf16 weights read once per distinct expert)."""
+    s = shape
+    hit = {int(e) for e, c in zip(idx.ravel(), cls.ravel()) if c == 0}
+    low = {int(e) for e, c in zip(idx.ravel(), cls.ravel()) if c == 2}
+    w = 2 * (s.n_experts * s.d + 3 * s.d * s.inter_shared + len(hit) * 3 * s.d * s.inter
+             + len(low) * 2 * s.lore_rank * s.d)
+    act = 2 * T * s.d + 2 * T * s.d + 4 * T * s.top_k
+    return w + act, len(hit), len(low)
+
+
+def device_replica(torch, B, shape, gen, dev):
+    """A layer weight set drawn on the device: N(0, 0.02) bf16, random residency of S experts."""
+    s = shape
+
+    def rn(*sz):
+        return (torch.randn(*sz, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+
+    gu = torch.empty(s.n_slots, 2 * s.inter, s.d, dtype=torch.bfloat16, device=dev)
+    dn = torch.empty(s.n_slots, s.d, s.inter, dtype=torch.bfloat16, device=dev)
+    for i in range(s.n_slots):
+        gu[i] = rn(2 * s.inter, s.d)
+        dn[i] = rn(s.d, s.inter)
+    perm = torch.randperm(s.n_experts, generator=gen, device=dev)
+    soe = torch.full((s.n_experts,), -1, dtype=torch.int32, device=dev)
+    soe[perm[: s.n_slots]] = torch.arange(s.n_slots, dtype=torch.int32, device=dev)
+    return B.LayerWeights(w_router=rn(s.n_experts, s.d), slot_w_gate_up=gu, slot_w_down=dn, slot_of_expert=soe,
+                          shared_w_gate_up=rn(2 * s.inter_shared, s.d), shared_w_down=rn(s.d, s.inter_shared),
+                          lore_A=rn(s.n_experts, s.lore_rank, s.d), lore_B=rn(s.n_experts, s.d, s.lore_rank))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_21240_b200 import binding as B
+    from paper_2608_21240_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()   # fail loudly when the extension is missing
+
+    shape = W.SHAPES[args.shape]
+    T, R = args.tokens, args.replicas
+    peaks = load_peaks()
+
+    # replica 0 comes from the numpy generator (the CPU baseline needs the same numbers);
+    # the others are drawn on the device with the same distributions
+    wl0 = W.make_layer(shape, T, variant=100 + rank)
+    upload, bf16_tensor, cfg_of = B.upload, B.bf16_tensor, B.cfg_of
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(W.BASE_SEED + 1000 * rank)
+    reps = [upload(wl0, dev)] + [device_replica(torch, B, shape, gen, dev) for _ in range(R - 1)]
+    structs = [r.c_struct() for r in reps]
+    h = bf16_tensor(wl0.h, dev)
+    conf = torch.from_numpy(wl0.conf).to(dev)
+    layer = B.SpiceLayer(cfg_of(shape), T, device=local)
+    y = torch.empty(T, shape.d, dtype=torch.bfloat16, device=dev)
+    idx = torch.empty(T, shape.top_k, dtype=torch.int32, device=dev)
+    gate = torch.empty(T, shape.top_k, dtype=torch.float32, device=dev)
+    cls = torch.empty(T, shape.top_k, dtype=torch.uint8, device=dev)
+    counts = torch.zeros(3, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h, conf, T, y, idx=idx, gate=gate, cls=cls, counts=counts,
+                              stream=stream)
+
+    # algorithmic bytes of every replica's call (from the routing the library itself produced)
+    rep_bytes, rep_hit, rep_low = [], [], []
+    for i in range(R):
+        step(i)
+        torch.cuda.synchronize()
+        b, nh, nl = algorithmic_bytes(shape, T, idx.cpu().numpy(), cls.cpu().numpy())
+        rep_bytes.append(b)
+        rep_hit.append(nh)
+        rep_low.append(nl)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    l0 = layer.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    w0 = time.time()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    w1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    launches = layer.launch_count() - l0
+    total_bytes = sum(rep_bytes[i % R] for i in range(args.steps))
+
+    # end to end: inputs start in pinned host memory, the result is read back to the host every step
+    h_host = h.cpu().pin_memory()
+    conf_host = conf.cpu().pin_memory()
+    y_host = torch.empty(T, shape.d, dtype=torch.bfloat16).pin_memory()
+    cnt_host = torch.empty(3, dtype=torch.int32).pin_memory()
+    h_dev, conf_dev = torch.empty_like(h), torch.empty_like(conf)
+
+    def e2e_step(i):
+        h_dev.copy_(h_host, non_blocking=True)
+        conf_dev.copy_(conf_host, non_blocking=True)
+        B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h_dev, conf_dev, T, y, idx=idx, gate=gate, cls=cls,
+                              counts=counts, stream=stream)
+        y_host.copy_(y, non_blocking=True)
+        cnt_host.copy_(counts, non_blocking=True)
+        stream.synchronize()     # the caller consumes y before the next step
+
+    for i in range(min(args.warmup, 5)):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    n_e2e = args.steps
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for i in range(n_e2e):
+        e2e_step(i)
+    f1.record(stream)
+    torch.cuda.synchronize()
+    w2 = time.time()
+    ms_e2e = f0.elapsed_time(f1)
+    if sampler:
+        sampler.stop()
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    status = layer.device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status} after the timed region")
+
+    if rank == 0:
+        tok_s = world * T * args.steps / (ms * 1e-3)
+        achieved = total_bytes / (ms * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": tok_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{shape.name} decode layer, batch {T} tokens "
+                                   f"(d={shape.d}, N={shape.n_experts}, K={shape.top_k}, I={shape.inter}, "
+                                   f"I_s={shape.inter_shared}, r={shape.lore_rank}, {shape.n_slots} resident slots, "
+                                   f"tau={shape.tau}, Beta(2,2) confidences)",
+                       "tokens_per_step": T, "cold_l2": f"steps rotate through {R} independent weight sets "
+                       f"({sum(rep_bytes) / 1e6:.0f} MB between reuses, L2 is 126 MB); no flush in the timed region",
+                       "distinct_hit_experts_mean": float(np.mean(rep_hit)),
+                       "distinct_lowconf_experts_mean": float(np.mean(rep_low)),
+                       "multi_gpu": "replicas only (no collective on the data path)"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                         "kernel": "all launches of spice_moe_layer_fwd (algorithmic bytes of the call / time per call)",
+                         "algorithmic_bytes_per_step": total_bytes / args.steps, "peak_source": peaks["source"],
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "e2e": {"value": world * T * n_e2e / (ms_e2e * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": int(h_host.numel() * 2 + conf_host.numel() * 4),
+                    "d2h_bytes_per_step": int(y_host.numel() * 2 + 12), "ms_per_step": ms_e2e / n_e2e},
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(w0, w1) if sampler else None,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            out["cpu_baseline"] = cpu_baseline(wl0, budget_s=args.cpu_budget)
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_call(wl, tokens):
+    """One oracle evaluation of the GPU part of the layer for the given tokens."""
+    import oracle
+    from tests._cases import run_oracle
+    return run_oracle(wl, tokens=tokens, want_full=False)
+
+
+def cpu_baseline(wl, budget_s=15.0):
+    """The oracle, as it stands, timed on this machine's host cores on a bounded sample of the same batch."""
+    import oracle
+    T = wl.T
+    oracle_call(wl, list(range(T)))          # draws the needed expert weights, warms caches
+    t0 = time.time()
+    reps = 0
+    while True:
+        oracle_call(wl, list(range(T)))
+        reps += 1
+        if time.time() - t0 > budget_s or reps >= 20:
+            break
+    dt = (time.time() - t0) / reps
+    return {"value": T / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"the full batch of {T} tokens of weight set 0, {reps} repetitions, mean", "s_per_step": dt}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores (there is no reference implementation)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2608_21240_b200 import workloads as W
+    shape = W.SHAPES[args.shape]
+    T = args.tokens
+    wl = W.make_layer(shape, T, variant=100)
+    t0 = time.time()
+    oracle_call(wl, [0])
+    oracle_call(wl, list(range(T)))          # draw all needed experts once
+    t0 = time.time()
+    oracle_call(wl, [0])
+    t_one = time.time() - t0
+    budget = 150.0
+    n_tok = int(max(1, min(T, budget / max(1e-3, (args.steps + args.warmup) * t_one))))
+    toks = list(range(n_tok))
+    for _ in range(args.warmup):
+        oracle_call(wl, toks)
+    t0 = time.time()
+    for _ in range(args.steps):
+        oracle_call(wl, toks)
+    dt = time.time() - t0
+    val = n_tok * args.steps / dt
+    sample = f"{n_tok} of the batch's {T} tokens per step (weight set 0)"
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"{shape.name} decode layer, batch {T} tokens (CPU oracle, {sample})"},
+           "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--shape", default="dsv2lite")
+    ap.add_argument("--tokens", type=int, default=16)
+    ap.add_argument("--replicas", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,157 @@
+/*
+ * spice.h -- C ABI of the B200 (sm_100a) MoE-layer forward for SPICE-style offloaded decoding.
+ *
+ * One call of spice_moe_layer_fwd computes the GPU part of one offloaded-MoE layer as the
+ * paper states it:
+ *     S_t = TopK(Router(h_t), K)                                   (Eq. 1, Sec. 2.2)
+ *     shared experts always on, routed outputs gate-weighted        (Sec. 2.1)
+ *     resident (prefetched) expert      -> executed exactly         (Sec. 4.2, runtime policy)
+ *     missing, confidence < tau         -> S(h) + B_e A_e h         (Sec. 4.2, LoRE surrogate)
+ *     missing, otherwise                -> listed for exact recovery (Sec. 4.3, set M)
+ *     y_t = s_t + sum_{HIT} g_k E_{e_k}(h_t) + sum_{LOWCONF} g_k ( s_t + B_{e_k} A_{e_k} h_t )
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless it says "host".
+ *   - bf16 tensors are passed as spice_bf16* (raw 16-bit patterns), row-major, 16-byte aligned,
+ *     weights in [out, in] order.  Expert FFNs are SwiGLU: E(x) = W_d ( silu(W_g x) * (W_u x) ).
+ *   - All calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and return without synchronising.  The library allocates device memory only in
+ *     spice_create; per call it allocates nothing.  A ctx must not be used by two streams at once.
+ *   - Errors found on the host return a code and launch nothing.  Conditions found on the device
+ *     (expert id out of range, slot index >= n_slots, an expired bounded wait) never trap: the
+ *     entry is treated as an exact-recovery miss or skipped, a status word is set, and
+ *     spice_get_device_status reports it.
+ *   - T = 0 is SPICE_OK and launches nothing.
+ *   - Class codes: 0 = HIT, 1 = MISS_EXACT, 2 = LOWCONF.  LOWCONF iff the expert is not resident
+ *     and confidence < tau (strict; NaN compares false, i.e. exact recovery).
+ *   - Top-k order: decreasing logit, equal logits towards the smaller expert index.
+ */
+#ifndef SPICE_H_
+#define SPICE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint16_t spice_bf16;
+typedef struct spice_ctx spice_ctx;
+
+typedef enum {
+    SPICE_OK = 0,
+    SPICE_ERR_INVALID_ARG = 1,       /* NULL / misaligned pointer, T < 0, T > max_tokens            */
+    SPICE_ERR_UNSUPPORTED_SHAPE = 2, /* a dimension the kernels do not cover (see spice_create)      */
+    SPICE_ERR_WORKSPACE = 3,         /* workspace allocation failed                                  */
+    SPICE_ERR_CUDA = 4,              /* a CUDA runtime call failed                                   */
+    SPICE_ERR_BAD_TABLE = 5,         /* device: slot_of_expert entry >= n_slots, or expert id bad    */
+    SPICE_ERR_TIMEOUT = 6            /* device: a bounded wait expired                               */
+} spice_status;
+
+enum { SPICE_HIT = 0, SPICE_MISS_EXACT = 1, SPICE_LOWCONF = 2 };
+
+/* Static shape of one layer (notation of the paper: K of Eq. 1, r and d of the LoRE factors,
+ * tau of Sec. 4.1/4.2). */
+typedef struct {
+    int32_t d;            /* hidden width; multiple of 8                                  */
+    int32_t n_experts;    /* N routed experts, 1..1024                                    */
+    int32_t top_k;        /* K, 1..min(N,32)                                              */
+    int32_t inter;        /* I, routed SwiGLU intermediate width; multiple of 8           */
+    int32_t inter_shared; /* I_s, width of the fused shared expert; multiple of 8         */
+    int32_t lore_rank;    /* r; multiple of 8                                             */
+    int32_t n_slots;      /* S, resident expert slots, 1..1024                            */
+    int32_t norm_topk;    /* 1: gates = softmax over the K winners; 0: full-softmax probs */
+    int32_t conf_stride;  /* N: conf is [T,N] per (token, expert); 0: conf is [T]         */
+    float tau;            /* confidence threshold                                         */
+} spice_layer_cfg;
+
+/* Weights of one layer.  The slot pool holds the resident experts; LoRE factors and the shared
+ * expert are resident for every expert (Sec. 3, scenario 2). */
+typedef struct {
+    const spice_bf16 *w_router;         /* [N, d]                                          */
+    const spice_bf16 *slot_w_gate_up;   /* [S, 2I, d]: I gate rows, then I up rows         */
+    const spice_bf16 *slot_w_down;      /* [S, d, I]                                       */
+    const int32_t *slot_of_expert;      /* [N]; slot index, or -1 when not resident        */
+    const spice_bf16 *shared_w_gate_up; /* [2 I_s, d]: I_s gate rows, then I_s up rows     */
+    const spice_bf16 *shared_w_down;    /* [d, I_s]                                        */
+    const spice_bf16 *lore_A;           /* [N, r, d]   A_e of Delta_e(h) = B_e A_e h       */
+    const spice_bf16 *lore_B;           /* [N, d, r]   B_e                                 */
+} spice_layer_weights;
+
+/* Library version (major*10000 + minor*100 + patch).  Host only. */
+int32_t spice_version(void);
+
+/* Create a context for layers of shape *cfg on CUDA device `device`, able to process up to
+ * max_tokens tokens per call.  Allocates the workspace (its size is reported by
+ * spice_workspace_bytes).  Returns SPICE_ERR_UNSUPPORTED_SHAPE when a dimension breaks the
+ * limits stated in spice_layer_cfg, SPICE_ERR_WORKSPACE / SPICE_ERR_CUDA on allocation failure.
+ * The ctx is owned by the caller and released with spice_destroy. */
+spice_status spice_create(spice_ctx **ctx, int32_t device, const spice_layer_cfg *cfg, int32_t max_tokens);
+spice_status spice_destroy(spice_ctx *ctx);
+spice_status spice_workspace_bytes(const spice_ctx *ctx, size_t *bytes /* host */);
+
+/* Router + TopK + gate scores (Eq. 1; "selected experts and their gate scores", Sec. 4.2).
+ *   h [T,d] bf16, w_router [N,d] bf16  ->  idx [T,K] int32, gate [T,K] fp32,
+ *   logits [T,N] fp32 (optional, may be NULL).
+ * Logits are accumulated in fp32; selection is done on logits, never on exponentials. */
+spice_status spice_route_topk(spice_ctx *ctx, const spice_bf16 *h, const spice_bf16 *w_router, int32_t T,
+                              int32_t *idx, float *gate, float *logits, void *stream);
+
+/* Hit / miss / low-confidence classification of every selected expert against the slot table and
+ * the draft model's confidences (runtime policy of Sec. 4.2), and the residual-miss list
+ * (set M of Sec. 4.3) in ascending (t*K + k) order.
+ *   idx [T,K], gate [T,K], slot_of_expert [N], conf [T,N] fp32 (or [T] when conf_stride == 0)
+ *   -> cls [T,K] uint8, slot [T,K] int32 (slot index for HIT, else -1),
+ *      counts [3] int32 (entries per class code),
+ *      resid_tok / resid_k / resid_expert [T*K] int32 and resid_gate [T*K] fp32: the first
+ *      counts[1] entries are valid.  Any of the four resid arrays may be NULL (then none is written). */
+spice_status spice_classify_misses(spice_ctx *ctx, const int32_t *idx, const float *gate,
+                                   const int32_t *slot_of_expert, const float *conf, int32_t T,
+                                   uint8_t *cls, int32_t *slot, int32_t *counts,
+                                   int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
+                                   float *resid_gate, void *stream);
+
+/* Exact execution of the resident experts (Sec. 4.2: "executes it exactly"):
+ *   y[t,:] += sum over k with cls[t,k] == HIT of gate[t,k] * E_{slot[t,k]}(h[t,:]),   y [T,d] fp32.
+ * Tokens are grouped by slot so that each resident expert's weights are read once. */
+spice_status spice_grouped_expert_ffn(spice_ctx *ctx, const spice_layer_weights *w /* host struct */,
+                                      const spice_bf16 *h, const int32_t *idx, const float *gate,
+                                      const uint8_t *cls, const int32_t *slot, int32_t T, float *y,
+                                      void *stream);
+
+/* Shared expert plus LoRE substitution for low-confidence misses (Sec. 4.2, y~_e = S(h) + B_e A_e h):
+ *   y[t,:] += (1 + sum_{LOWCONF} gate[t,k]) * S(h[t,:]) + sum_{LOWCONF} gate[t,k] * B_e A_e h[t,:],  y fp32. */
+spice_status spice_lore_surrogate(spice_ctx *ctx, const spice_layer_weights *w /* host struct */,
+                                  const spice_bf16 *h, const int32_t *idx, const float *gate,
+                                  const uint8_t *cls, int32_t T, float *y, void *stream);
+
+/* The whole layer: route -> classify -> resident experts + shared/LoRE -> combine.
+ *   h [T,d] bf16, conf as in spice_classify_misses.
+ *   y_cpu_residual [T,d] fp32, optional: outputs of exactly recovered experts computed elsewhere
+ *       (Sec. 4.3, "merges their outputs with the CPU expert outputs"); added before rounding.
+ *   x_resid [T,d] bf16, optional, in/out: residual stream, x_resid <- x_resid + y.
+ *   y [T,d] bf16 out.  idx, gate, cls, counts, resid_*: as above; each may be NULL when not wanted.
+ * Equals spice_route_topk, spice_classify_misses, y = 0, spice_grouped_expert_ffn,
+ * spice_lore_surrogate applied in turn, up to fp32 summation order and the final bf16 rounding. */
+spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w /* host struct */,
+                                 const spice_bf16 *h, const float *conf, int32_t T,
+                                 const float *y_cpu_residual, spice_bf16 *x_resid, spice_bf16 *y,
+                                 int32_t *idx, float *gate, uint8_t *cls, int32_t *counts,
+                                 int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
+                                 float *resid_gate, void *stream);
+
+/* Synchronises the device work issued through ctx so far and returns the sticky device status
+ * (SPICE_OK, SPICE_ERR_BAD_TABLE or SPICE_ERR_TIMEOUT) in *code (host), then clears it. */
+spice_status spice_get_device_status(spice_ctx *ctx, int32_t *code /* host */);
+
+/* Number of kernels the library has launched through ctx since it was created (host counter). */
+spice_status spice_launch_count(const spice_ctx *ctx, int64_t *launches /* host */);
+
+/* Text for a status code (static storage, never NULL). */
+const char *spice_status_string(spice_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPICE_H_ */

@@ -1,0 +1,291 @@
+// C ABI of libspice: argument checking, workspace ownership and kernel dispatch.
+#include <new>
+
+#include "spice_internal.cuh"
+
+using namespace spice;
+
+struct spice_ctx {
+    int device;
+    spice_layer_cfg cfg;
+    int32_t max_tokens;
+    void *ws;          // one device allocation, carved below
+    size_t ws_bytes;
+    Tables tb;
+    // call-private copies of routing results when the caller does not want them
+    int32_t *ws_idx, *ws_slot, *ws_counts;
+    float *ws_gate;
+    uint8_t *ws_cls;
+    float *y32;        // [Tm, d] fp32 accumulator of the fused call
+    int64_t launches;
+};
+
+namespace {
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Carver {
+    char *base;
+    size_t off = 0;
+    template <typename T>
+    T *take(size_t n) {
+        off = (off + 255) & ~size_t(255);
+        T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+void carve(spice_ctx *c, char *base, size_t *total) {
+    const spice_layer_cfg &g = c->cfg;
+    const size_t Tm = (size_t)c->max_tokens, K = g.top_k, n = Tm * K;
+    Carver cv{base};
+    c->tb.groups = cv.take<GroupDesc>(1 + (size_t)g.n_slots + g.n_experts);
+    c->tb.hdr = cv.take<int32_t>(HDR_WORDS);
+    c->tb.status = cv.take<int32_t>(4);
+    c->tb.perm_hit = cv.take<int32_t>(n);
+    c->tb.perm_low = cv.take<int32_t>(n);
+    c->tb.pos_of_entry = cv.take<int32_t>(n);
+    c->tb.coef_shared = cv.take<float>(Tm);
+    c->tb.act_hit = cv.take<float>(n * g.inter);
+    c->tb.act_shared = cv.take<float>(Tm * g.inter_shared);
+    c->tb.z_low = cv.take<float>(n * g.lore_rank);
+    c->tb.part = cv.take<float>(n * g.d);
+    c->tb.part_shared = cv.take<float>(Tm * g.d);
+    c->ws_idx = cv.take<int32_t>(n);
+    c->ws_slot = cv.take<int32_t>(n);
+    c->ws_counts = cv.take<int32_t>(4);
+    c->ws_gate = cv.take<float>(n);
+    c->ws_cls = cv.take<uint8_t>(n);
+    c->y32 = cv.take<float>(Tm * g.d);
+    *total = (cv.off + 255) & ~size_t(255);
+}
+
+spice_status check_cfg(const spice_layer_cfg *g, int32_t max_tokens) {
+    if (!g) return SPICE_ERR_INVALID_ARG;
+    if (max_tokens < 1 || max_tokens > 65535) return SPICE_ERR_INVALID_ARG;
+    if (g->d < 8 || g->d % 8 || g->inter < 8 || g->inter % 8 || g->inter_shared < 8 || g->inter_shared % 8 ||
+        g->lore_rank < 8 || g->lore_rank % 8)
+        return SPICE_ERR_UNSUPPORTED_SHAPE;
+    if (g->n_experts < 1 || g->n_experts > 1024 || g->n_slots < 1 || g->n_slots > 1024)
+        return SPICE_ERR_UNSUPPORTED_SHAPE;
+    if (g->top_k < 1 || g->top_k > 32 || g->top_k > g->n_experts) return SPICE_ERR_UNSUPPORTED_SHAPE;
+    if (g->conf_stride != 0 && g->conf_stride != g->n_experts) return SPICE_ERR_INVALID_ARG;
+    if ((size_t)g->d * 4 + (size_t)g->n_experts * 4 > 200 * 1024) return SPICE_ERR_UNSUPPORTED_SHAPE;
+    return SPICE_OK;
+}
+
+Dims dims_of(const spice_ctx *c, int T) {
+    const spice_layer_cfg &g = c->cfg;
+    return Dims{T, g.d, g.n_experts, g.top_k, g.inter, g.inter_shared, g.lore_rank, g.n_slots};
+}
+
+spice_status check_call(const spice_ctx *c, int32_t T) {
+    if (!c) return SPICE_ERR_INVALID_ARG;
+    if (T < 0 || T > c->max_tokens) return SPICE_ERR_INVALID_ARG;
+    return SPICE_OK;
+}
+
+bool weights_ok(const spice_layer_weights *w, bool routed, bool shared_lore) {
+    if (!w) return false;
+    if (routed && !(w->slot_w_gate_up && w->slot_w_down && aligned16(w->slot_w_gate_up) && aligned16(w->slot_w_down)))
+        return false;
+    if (shared_lore && !(w->shared_w_gate_up && w->shared_w_down && w->lore_A && w->lore_B &&
+                         aligned16(w->shared_w_gate_up) && aligned16(w->shared_w_down) && aligned16(w->lore_A) &&
+                         aligned16(w->lore_B)))
+        return false;
+    return true;
+}
+
+// adds n launches or turns a launch failure into SPICE_ERR_CUDA
+#define SPICE_LAUNCH(expr)                       \
+    do {                                         \
+        int n_ = (expr);                         \
+        if (n_ < 0) return SPICE_ERR_CUDA;       \
+        ctx->launches += n_;                     \
+    } while (0)
+
+}  // namespace
+
+extern "C" {
+
+int32_t spice_version(void) { return 100; }
+
+const char *spice_status_string(spice_status s) {
+    switch (s) {
+        case SPICE_OK: return "ok";
+        case SPICE_ERR_INVALID_ARG: return "invalid argument";
+        case SPICE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case SPICE_ERR_WORKSPACE: return "workspace allocation failed";
+        case SPICE_ERR_CUDA: return "CUDA runtime error";
+        case SPICE_ERR_BAD_TABLE: return "bad slot table or expert index (device)";
+        case SPICE_ERR_TIMEOUT: return "bounded device wait expired";
+    }
+    return "unknown status";
+}
+
+spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg *cfg, int32_t max_tokens) {
+    if (!out) return SPICE_ERR_INVALID_ARG;
+    *out = nullptr;
+    spice_status s = check_cfg(cfg, max_tokens);
+    if (s != SPICE_OK) return s;
+    if (cudaSetDevice(device) != cudaSuccess) return SPICE_ERR_CUDA;
+    spice_ctx *c = new (std::nothrow) spice_ctx();
+    if (!c) return SPICE_ERR_WORKSPACE;
+    c->device = device;
+    c->cfg = *cfg;
+    c->max_tokens = max_tokens;
+    c->launches = 0;
+    carve(c, nullptr, &c->ws_bytes);
+    if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return SPICE_ERR_WORKSPACE;
+    }
+    size_t total;
+    carve(c, static_cast<char *>(c->ws), &total);
+    if (cudaMemset(c->ws, 0, c->ws_bytes) != cudaSuccess) {
+        cudaFree(c->ws);
+        delete c;
+        return SPICE_ERR_CUDA;
+    }
+    *out = c;
+    return SPICE_OK;
+}
+
+spice_status spice_destroy(spice_ctx *ctx) {
+    if (!ctx) return SPICE_OK;
+    cudaSetDevice(ctx->device);
+    cudaError_t e = cudaFree(ctx->ws);
+    delete ctx;
+    return e == cudaSuccess ? SPICE_OK : SPICE_ERR_CUDA;
+}
+
+spice_status spice_workspace_bytes(const spice_ctx *ctx, size_t *bytes) {
+    if (!ctx || !bytes) return SPICE_ERR_INVALID_ARG;
+    *bytes = ctx->ws_bytes;
+    return SPICE_OK;
+}
+
+spice_status spice_launch_count(const spice_ctx *ctx, int64_t *launches) {
+    if (!ctx || !launches) return SPICE_ERR_INVALID_ARG;
+    *launches = ctx->launches;
+    return SPICE_OK;
+}
+
+spice_status spice_get_device_status(spice_ctx *ctx, int32_t *code) {
+    if (!ctx || !code) return SPICE_ERR_INVALID_ARG;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return SPICE_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return SPICE_ERR_CUDA;
+    int32_t v = 0;
+    if (cudaMemcpy(&v, ctx->tb.status, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return SPICE_ERR_CUDA;
+    if (cudaMemset(ctx->tb.status, 0, sizeof(int32_t)) != cudaSuccess) return SPICE_ERR_CUDA;
+    *code = v;
+    return SPICE_OK;
+}
+
+spice_status spice_route_topk(spice_ctx *ctx, const spice_bf16 *h, const spice_bf16 *w_router, int32_t T,
+                              int32_t *idx, float *gate, float *logits, void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    if (T == 0) return SPICE_OK;
+    if (!h || !w_router || !idx || !gate || !aligned16(h) || !aligned16(w_router)) return SPICE_ERR_INVALID_ARG;
+    SPICE_LAUNCH(launch_route_topk(dims_of(ctx, T), ctx->cfg.norm_topk, reinterpret_cast<const __nv_bfloat16 *>(h),
+                                   reinterpret_cast<const __nv_bfloat16 *>(w_router), idx, gate, logits,
+                                   static_cast<cudaStream_t>(stream)));
+    return SPICE_OK;
+}
+
+spice_status spice_classify_misses(spice_ctx *ctx, const int32_t *idx, const float *gate,
+                                   const int32_t *slot_of_expert, const float *conf, int32_t T, uint8_t *cls,
+                                   int32_t *slot, int32_t *counts, int32_t *resid_tok, int32_t *resid_k,
+                                   int32_t *resid_expert, float *resid_gate, void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (T == 0) {
+        if (!counts) return SPICE_OK;
+        return cudaMemsetAsync(counts, 0, 3 * sizeof(int32_t), st) == cudaSuccess ? SPICE_OK : SPICE_ERR_CUDA;
+    }
+    if (!idx || !gate || !slot_of_expert || !conf || !cls || !slot || !counts) return SPICE_ERR_INVALID_ARG;
+    if (!(resid_tok && resid_k && resid_expert && resid_gate)) resid_tok = resid_k = resid_expert = nullptr, resid_gate = nullptr;
+    SPICE_LAUNCH(launch_classify(dims_of(ctx, T), ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, slot_of_expert, conf,
+                                 cls, slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
+    return SPICE_OK;
+}
+
+spice_status spice_grouped_expert_ffn(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *h,
+                                      const int32_t *idx, const float *gate, const uint8_t *cls,
+                                      const int32_t *slot, int32_t T, float *y, void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    if (T == 0) return SPICE_OK;
+    if (!weights_ok(w, true, false) || !h || !idx || !gate || !cls || !slot || !y || !aligned16(h) || !aligned16(y))
+        return SPICE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Dims dm = dims_of(ctx, T);
+    const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
+    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, slot, ctx->tb, st));
+    SPICE_LAUNCH(launch_gateup(dm, KIND_HIT, *w, hb, ctx->tb, st));
+    SPICE_LAUNCH(launch_down(dm, KIND_HIT, *w, ctx->tb, st));
+    CombineArgs ca{KIND_HIT, 1, gate, cls, y, nullptr, nullptr, nullptr};
+    SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));
+    return SPICE_OK;
+}
+
+spice_status spice_lore_surrogate(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *h,
+                                  const int32_t *idx, const float *gate, const uint8_t *cls, int32_t T, float *y,
+                                  void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    if (T == 0) return SPICE_OK;
+    if (!weights_ok(w, false, true) || !h || !idx || !gate || !cls || !y || !aligned16(h) || !aligned16(y))
+        return SPICE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Dims dm = dims_of(ctx, T);
+    const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
+    // no slot array: HIT entries are left out of the grouping
+    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, nullptr, ctx->tb, st));
+    SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED, *w, hb, ctx->tb, st));
+    SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
+    SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_LOW, *w, ctx->tb, st));
+    CombineArgs ca{KIND_SHARED | KIND_LOW, 1, gate, cls, y, nullptr, nullptr, nullptr};
+    SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));
+    return SPICE_OK;
+}
+
+spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *h,
+                                 const float *conf, int32_t T, const float *y_cpu_residual, spice_bf16 *x_resid,
+                                 spice_bf16 *y, int32_t *idx, float *gate, uint8_t *cls, int32_t *counts,
+                                 int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert, float *resid_gate,
+                                 void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!counts) counts = ctx->ws_counts;
+    if (T == 0) return cudaMemsetAsync(counts, 0, 3 * sizeof(int32_t), st) == cudaSuccess ? SPICE_OK : SPICE_ERR_CUDA;
+    if (!weights_ok(w, true, true) || !w->w_router || !w->slot_of_expert || !aligned16(w->w_router) || !h || !conf ||
+        !y || !aligned16(h) || !aligned16(y))
+        return SPICE_ERR_INVALID_ARG;
+    if ((y_cpu_residual && !aligned16(y_cpu_residual)) || (x_resid && !aligned16(x_resid))) return SPICE_ERR_INVALID_ARG;
+    if (!idx) idx = ctx->ws_idx;
+    if (!gate) gate = ctx->ws_gate;
+    if (!cls) cls = ctx->ws_cls;
+    if (!(resid_tok && resid_k && resid_expert && resid_gate)) resid_tok = resid_k = resid_expert = nullptr, resid_gate = nullptr;
+    const Dims dm = dims_of(ctx, T);
+    const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
+    SPICE_LAUNCH(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
+                                   gate, nullptr, st));
+    SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
+                                 ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
+    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st));
+    SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED | KIND_HIT, *w, hb, ctx->tb, st));
+    SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
+    SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_HIT | KIND_LOW, *w, ctx->tb, st));
+    CombineArgs ca{KIND_SHARED | KIND_HIT | KIND_LOW, 0, gate, cls, nullptr, reinterpret_cast<__nv_bfloat16 *>(y),
+                   y_cpu_residual, reinterpret_cast<__nv_bfloat16 *>(x_resid)};
+    SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));
+    return SPICE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,206 @@
+// Hit / miss / low-confidence classification (runtime policy of Sec. 4.2 of the paper), the
+// residual-miss list (set M of Sec. 4.3) and the token-to-expert grouping that the expert kernels
+// consume.  Both kernels run as ONE CTA: the tables are a few thousand entries at most and every
+// step is a histogram, a scan or an ordered compaction.
+#include "spice_internal.cuh"
+
+namespace spice {
+
+constexpr int CT = 1024;  // threads of the single CTA
+
+// exclusive scan of one value per thread across the CTA; returns the exclusive prefix and the total
+__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_tot /* [33] smem */, int &total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    __syncthreads();   // protect warp_tot from the previous use
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_tot[lane];
+        int winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += n;
+        }
+        warp_tot[lane] = winc - w;
+        if (lane == 31) warp_tot[32] = winc;
+    }
+    __syncthreads();
+    total = warp_tot[32];
+    return warp_tot[warp] + inc - v;
+}
+
+__global__ void __launch_bounds__(CT) classify_kernel(int T, int N, int K, int S, int conf_stride, float tau,
+                                                      const int32_t *__restrict__ idx, const float *__restrict__ gate,
+                                                      const int32_t *__restrict__ slot_of_expert,
+                                                      const float *__restrict__ conf, uint8_t *__restrict__ cls,
+                                                      int32_t *__restrict__ slot, int32_t *__restrict__ counts,
+                                                      int32_t *__restrict__ resid_tok, int32_t *__restrict__ resid_k,
+                                                      int32_t *__restrict__ resid_expert,
+                                                      float *__restrict__ resid_gate, int32_t *__restrict__ status) {
+    __shared__ int warp_tot[33];
+    __shared__ int s_cnt[3];
+    if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0;
+    __syncthreads();
+    const int n = T * K;
+    int base = 0;   // residual entries emitted by earlier chunks
+    for (int i0 = 0; i0 < n; i0 += CT) {
+        const int i = i0 + threadIdx.x;
+        int c = -1, e = 0, sl = -1;
+        if (i < n) {
+            e = idx[i];
+            if (e < 0 || e >= N) {                 // cannot happen after spice_route_topk
+                atomicMax(status, (int)SPICE_ERR_BAD_TABLE);
+                c = SPICE_MISS_EXACT;
+            } else {
+                sl = slot_of_expert[e];
+                if (sl >= S) {                     // corrupt table entry: do not touch the pool
+                    atomicMax(status, (int)SPICE_ERR_BAD_TABLE);
+                    sl = -1;
+                    c = SPICE_MISS_EXACT;
+                } else if (sl >= 0) {
+                    c = SPICE_HIT;
+                } else {
+                    sl = -1;
+                    const int t = i / K;
+                    const float cf = conf_stride ? conf[(size_t)t * conf_stride + e] : conf[t];
+                    c = (cf < tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
+                }
+            }
+            cls[i] = (uint8_t)c;
+            slot[i] = sl;
+            atomicAdd(&s_cnt[c], 1);
+        }
+        int total;
+        const int pos = block_exclusive_scan(c == SPICE_MISS_EXACT ? 1 : 0, warp_tot, total);
+        if (c == SPICE_MISS_EXACT && resid_tok) {
+            const int o = base + pos;
+            resid_tok[o] = i / K;
+            resid_k[o] = i % K;
+            resid_expert[o] = e;
+            resid_gate[o] = gate[i];
+        }
+        base += total;
+    }
+    __syncthreads();
+    if (threadIdx.x < 3) counts[threadIdx.x] = s_cnt[threadIdx.x];
+}
+
+// Builds, from cls / slot / idx / gate:
+//   groups[0] = shared expert (m = T); then one group per slot with >= 1 HIT entry (slot order);
+//   then one group per expert with >= 1 LOWCONF entry (expert order);
+//   perm_hit / perm_low: entry ids grouped accordingly; pos_of_entry; coef_shared[t] = 1 + sum of
+//   LOWCONF gates in k order.
+// Positions inside a group are handed out by warp-aggregated shared-memory atomics; the order of
+// entries inside a group is therefore not fixed, which no result depends on (every entry's row is
+// computed independently and the combine step gathers by entry id).
+__global__ void __launch_bounds__(CT) group_kernel(int T, int N, int K, int S, const int32_t *__restrict__ idx,
+                                                   const float *__restrict__ gate, const uint8_t *__restrict__ cls,
+                                                   const int32_t *__restrict__ slot, Tables tb) {
+    __shared__ int warp_tot[33];
+    __shared__ int cnt_hit[1024], cnt_low[1024];   // later reused as cursors
+    __shared__ int off_hit[1024], off_low[1024];
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int n = T * K;
+    cnt_hit[tid] = 0;
+    cnt_low[tid] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += CT) {
+        const int c = cls[i];
+        if (c == SPICE_HIT) {
+            if (!slot) continue;   // caller only wants the shared / low-confidence groups
+            const int s = slot[i];
+            if (s >= 0 && s < S) atomicAdd(&cnt_hit[s], 1);
+            else atomicMax(tb.status, (int)SPICE_ERR_BAD_TABLE);
+        } else if (c == SPICE_LOWCONF) {
+            const int e = idx[i];
+            if (e >= 0 && e < N) atomicAdd(&cnt_low[e], 1);
+            else atomicMax(tb.status, (int)SPICE_ERR_BAD_TABLE);
+        }
+    }
+    __syncthreads();
+    const int ch = cnt_hit[tid], cl = cnt_low[tid];
+    int n_hit, n_low, n_hg, n_lg;
+    const int oh = block_exclusive_scan(ch, warp_tot, n_hit);
+    const int ol = block_exclusive_scan(cl, warp_tot, n_low);
+    const int gh = block_exclusive_scan(ch > 0 ? 1 : 0, warp_tot, n_hg);
+    const int gl = block_exclusive_scan(cl > 0 ? 1 : 0, warp_tot, n_lg);
+    off_hit[tid] = oh;
+    off_low[tid] = ol;
+    if (ch > 0) tb.groups[1 + gh] = GroupDesc{KIND_HIT, tid, oh, ch};
+    if (cl > 0) tb.groups[1 + n_hg + gl] = GroupDesc{KIND_LOW, tid, ol, cl};
+    if (tid == 0) {
+        tb.groups[0] = GroupDesc{KIND_SHARED, 0, 0, T};
+        tb.hdr[HDR_N_GROUPS] = 1 + n_hg + n_lg;
+        tb.hdr[HDR_N_HIT_GROUPS] = n_hg;
+        tb.hdr[HDR_N_LOW_GROUPS] = n_lg;
+        tb.hdr[HDR_N_HIT] = n_hit;
+        tb.hdr[HDR_N_LOW] = n_low;
+    }
+    __syncthreads();
+    cnt_hit[tid] = 0;   // cursors
+    cnt_low[tid] = 0;
+    __syncthreads();
+    for (int i0 = 0; i0 < n; i0 += CT) {   // warp-uniform trip count
+        const int i = i0 + tid;
+        int key = -1;                        // 0..1023 hit slot, 1024..2047 low expert
+        if (i < n) {
+            const int c = cls[i];
+            if (c == SPICE_HIT) {
+                const int s = slot ? slot[i] : -1;
+                if (s >= 0 && s < S) key = s;
+            } else if (c == SPICE_LOWCONF) {
+                const int e = idx[i];
+                if (e >= 0 && e < N) key = 1024 + e;
+            }
+        }
+        const unsigned peers = __match_any_sync(0xffffffffu, key);
+        int pos = -1;
+        if (key >= 0) {
+            const int leader = __ffs(peers) - 1;
+            int basep = 0;
+            if (lane == leader)
+                basep = (key < 1024) ? atomicAdd(&cnt_hit[key], __popc(peers))
+                                     : atomicAdd(&cnt_low[key - 1024], __popc(peers));
+            basep = __shfl_sync(peers, basep, leader);
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            if (key < 1024) {
+                pos = off_hit[key] + basep + rank;
+                tb.perm_hit[pos] = i;
+            } else {
+                pos = off_low[key - 1024] + basep + rank;
+                tb.perm_low[pos] = i;
+            }
+        }
+        if (i < n) tb.pos_of_entry[i] = pos;
+    }
+    for (int t = tid; t < T; t += CT) {
+        float c = 1.0f;
+        for (int k = 0; k < K; ++k)
+            if (cls[t * K + k] == SPICE_LOWCONF) c += gate[t * K + k];
+        tb.coef_shared[t] = c;
+    }
+}
+
+int launch_classify(const Dims &dm, int conf_stride, float tau, const int32_t *idx, const float *gate,
+                    const int32_t *slot_of_expert, const float *conf, uint8_t *cls, int32_t *slot,
+                    int32_t *counts, int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
+                    float *resid_gate, int32_t *status, cudaStream_t st) {
+    classify_kernel<<<1, CT, 0, st>>>(dm.T, dm.N, dm.K, dm.S, conf_stride, tau, idx, gate, slot_of_expert, conf, cls,
+                                      slot, counts, resid_tok, resid_k, resid_expert, resid_gate, status);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_group(const Dims &dm, const int32_t *idx, const float *gate, const uint8_t *cls, const int32_t *slot,
+                 const Tables &tb, cudaStream_t st) {
+    group_kernel<<<1, CT, 0, st>>>(dm.T, dm.N, dm.K, dm.S, idx, gate, cls, slot, tb);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace spice

@@ -1,0 +1,132 @@
+// Router logits, Top-K and gate scores (Eq. 1 of the paper; "selected experts and their gate
+// scores", Sec. 4.2).  One CTA owns TPC tokens: its warps share the router rows (each warp takes
+// experts e = warp, warp+nwarps, ...), logits are accumulated in fp32 and parked in shared memory,
+// then one warp per token does K rounds of a shuffle arg-max (ties -> smaller expert index).
+#include "spice_internal.cuh"
+
+namespace spice {
+
+template <int TPC>
+__global__ void route_topk_kernel(const __nv_bfloat16 *__restrict__ h, const __nv_bfloat16 *__restrict__ wr,
+                                  int T, int d, int N, int K, int norm_topk, int32_t *__restrict__ idx,
+                                  float *__restrict__ gate, float *__restrict__ logits_out) {
+    extern __shared__ __align__(16) float smem[];
+    float *hs = smem;                   // [TPC][d] fp32 copy of the tokens
+    float *lg = smem + (size_t)TPC * d; // [TPC][N]
+    const int t0 = blockIdx.x * TPC;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+
+    // stage the tokens (8 bf16 per thread-step), zero rows past T
+    for (int v = threadIdx.x; v < TPC * (d >> 3); v += blockDim.x) {
+        int tt = v / (d >> 3), c = v - tt * (d >> 3);
+        uint4 u = make_uint4(0, 0, 0, 0);
+        if (t0 + tt < T) u = *reinterpret_cast<const uint4 *>(h + (size_t)(t0 + tt) * d + c * 8);
+        float *dst = hs + (size_t)tt * d + c * 8;
+        reinterpret_cast<float4 *>(dst)[0] = make_float4(bf_lo(u.x), bf_hi(u.x), bf_lo(u.y), bf_hi(u.y));
+        reinterpret_cast<float4 *>(dst)[1] = make_float4(bf_lo(u.z), bf_hi(u.z), bf_lo(u.w), bf_hi(u.w));
+    }
+    __syncthreads();
+
+    for (int e = warp; e < N; e += nwarps) {
+        float acc[TPC];
+#pragma unroll
+        for (int tt = 0; tt < TPC; ++tt) acc[tt] = 0.f;
+        const __nv_bfloat16 *row = wr + (size_t)e * d;
+        for (int k = lane * 8; k < d; k += 256) {
+            uint4 u = *reinterpret_cast<const uint4 *>(row + k);
+            float w0 = bf_lo(u.x), w1 = bf_hi(u.x), w2 = bf_lo(u.y), w3 = bf_hi(u.y);
+            float w4 = bf_lo(u.z), w5 = bf_hi(u.z), w6 = bf_lo(u.w), w7 = bf_hi(u.w);
+#pragma unroll
+            for (int tt = 0; tt < TPC; ++tt) {
+                const float4 a = *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k);
+                const float4 b = *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k + 4);
+                float s = acc[tt];
+                s = fmaf(w0, a.x, s); s = fmaf(w1, a.y, s); s = fmaf(w2, a.z, s); s = fmaf(w3, a.w, s);
+                s = fmaf(w4, b.x, s); s = fmaf(w5, b.y, s); s = fmaf(w6, b.z, s); s = fmaf(w7, b.w, s);
+                acc[tt] = s;
+            }
+        }
+#pragma unroll
+        for (int tt = 0; tt < TPC; ++tt) {
+            float s = warp_sum(acc[tt]);
+            if (lane == 0) lg[tt * N + e] = s;
+        }
+    }
+    __syncthreads();
+
+    for (int tt = warp; tt < TPC; tt += nwarps) {
+        const int t = t0 + tt;
+        if (t >= T) continue;   // warp-uniform
+        const float *l = lg + tt * N;
+        if (logits_out)
+            for (int e = lane; e < N; e += 32) logits_out[(size_t)t * N + e] = l[e];
+        uint32_t taken = 0;     // bit i: expert lane + 32*i already selected (N <= 1024)
+        float m = 0.f, denom = 0.f, my_val = 0.f;
+        int my_idx = 0;
+        for (int k = 0; k < K; ++k) {
+            float bv = -INFINITY;
+            int be = 0x7fffffff;
+            for (int i = 0, e = lane; e < N; ++i, e += 32) {
+                if ((taken >> i) & 1u) continue;
+                float v = l[e];
+                if (!(v == v)) v = -INFINITY;   // NaN never wins
+                if (be == 0x7fffffff || v > bv) { bv = v; be = e; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                int oe = __shfl_xor_sync(0xffffffffu, be, o);
+                if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
+            }
+            if ((be & 31) == lane) taken |= 1u << (be >> 5);
+            if (k == 0) {
+                m = bv;
+                if (!norm_topk) {   // full-softmax denominator
+                    float s = 0.f;
+                    for (int e = lane; e < N; e += 32) s += expf(l[e] - m);
+                    denom = warp_sum(s);
+                }
+            }
+            if (lane == k) { my_val = bv; my_idx = be; }
+        }
+        float p = (lane < K) ? expf(my_val - m) : 0.f;
+        if (norm_topk) {
+            // sum the K numerators in k order on every lane (deterministic, matches the definition)
+            float s = 0.f;
+            for (int k = 0; k < K; ++k) s += __shfl_sync(0xffffffffu, p, k);
+            denom = s;
+        }
+        if (lane < K) {
+            idx[(size_t)t * K + lane] = my_idx;
+            gate[(size_t)t * K + lane] = p / denom;
+        }
+    }
+}
+
+template <int TPC>
+static int launch_tpc(const Dims &dm, int norm_topk, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router,
+                      int32_t *idx, float *gate, float *logits, int threads, cudaStream_t st) {
+    size_t smem = ((size_t)TPC * dm.d + (size_t)TPC * dm.N) * sizeof(float);
+    if (smem > 220 * 1024) return -1;
+    if (cudaFuncSetAttribute(route_topk_kernel<TPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+        return -1;
+    int grid = (dm.T + TPC - 1) / TPC;
+    route_topk_kernel<TPC><<<grid, threads, smem, st>>>(h, w_router, dm.T, dm.d, dm.N, dm.K, norm_topk, idx, gate,
+                                                        logits);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_route_topk(const Dims &dm, int norm_topk, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router,
+                      int32_t *idx, float *gate, float *logits, cudaStream_t st) {
+    // few tokens: one token per CTA with many warps across the experts;
+    // many tokens: several tokens per CTA share each router row read.
+    if (dm.T <= 64) return launch_tpc<1>(dm, norm_topk, h, w_router, idx, gate, logits, dm.N >= 32 ? 1024 : 256, st);
+    if ((size_t)8 * (dm.d + dm.N) * sizeof(float) <= 160 * 1024)
+        return launch_tpc<8>(dm, norm_topk, h, w_router, idx, gate, logits, 256, st);
+    if ((size_t)2 * (dm.d + dm.N) * sizeof(float) <= 200 * 1024)
+        return launch_tpc<2>(dm, norm_topk, h, w_router, idx, gate, logits, 256, st);
+    return launch_tpc<1>(dm, norm_topk, h, w_router, idx, gate, logits, 256, st);
+}
+
+}  // namespace spice

@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of libspice (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "spice.h"
+
+namespace spice {
+
+constexpr int KIND_SHARED = 1;  // the fused shared expert, all T tokens
+constexpr int KIND_HIT = 2;     // one resident slot and the (t,k) entries routed to it
+constexpr int KIND_LOW = 4;     // one non-resident expert and its low-confidence entries
+
+// One unit of grouped work: m rows that all use the same weight matrices.
+struct GroupDesc {
+    int32_t kind;  // KIND_*
+    int32_t id;    // slot index (HIT), expert index (LOW), 0 (SHARED)
+    int32_t off;   // first position in perm_hit / perm_low (0 for SHARED)
+    int32_t m;     // number of rows
+};
+
+// Header words written by the grouping kernel.
+enum { HDR_N_GROUPS = 0, HDR_N_HIT_GROUPS, HDR_N_LOW_GROUPS, HDR_N_HIT, HDR_N_LOW, HDR_WORDS = 8 };
+
+// Device-side view of the per-call tables that live in the ctx workspace.
+struct Tables {
+    GroupDesc *groups;     // [1 + S + N]  group 0 is always the shared expert
+    int32_t *hdr;          // [HDR_WORDS]
+    int32_t *perm_hit;     // [Tm*K] entry ids (t*K+k) grouped by slot
+    int32_t *perm_low;     // [Tm*K] entry ids grouped by expert
+    int32_t *pos_of_entry; // [Tm*K] position of the entry in perm_hit / perm_low, -1 if none
+    float *coef_shared;    // [Tm] 1 + sum of LOWCONF gates
+    float *act_hit;        // [Tm*K, I]   silu(gate)*up of HIT entries, perm_hit order
+    float *act_shared;     // [Tm, I_s]
+    float *z_low;          // [Tm*K, r]   A_e h of LOWCONF entries, perm_low order
+    float *part;           // [Tm*K, d]   down-projected row of entry t*K+k (un-gated)
+    float *part_shared;    // [Tm, d]
+    int32_t *status;       // sticky device status word
+};
+
+struct Dims {
+    int32_t T, d, N, K, I, Is, r, S;
+};
+
+// ---- kernels launchers (each returns the number of kernels it launched, or -1 on launch error)
+int launch_route_topk(const Dims &dm, int norm_topk, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router,
+                      int32_t *idx, float *gate, float *logits, cudaStream_t st);
+
+int launch_classify(const Dims &dm, int conf_stride, float tau, const int32_t *idx, const float *gate,
+                    const int32_t *slot_of_expert, const float *conf, uint8_t *cls, int32_t *slot,
+                    int32_t *counts, int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
+                    float *resid_gate, int32_t *status, cudaStream_t st);
+
+int launch_group(const Dims &dm, const int32_t *idx, const float *gate, const uint8_t *cls,
+                 const int32_t *slot, const Tables &tb, cudaStream_t st);
+
+// Reference ("v1") expert path: warp-per-row GEMV kernels for any shape.
+int launch_gateup(const Dims &dm, int kind_mask, const spice_layer_weights &w, const __nv_bfloat16 *h,
+                  const Tables &tb, cudaStream_t st);
+int launch_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
+                  cudaStream_t st);
+int launch_down(const Dims &dm, int kind_mask, const spice_layer_weights &w, const Tables &tb, cudaStream_t st);
+
+struct CombineArgs {
+    int kind_mask;              // which terms enter
+    int accumulate;             // 1: y32 += ..., 0: y = ...
+    const float *gate;          // [T,K]
+    const uint8_t *cls;         // [T,K]
+    float *y32;                 // fp32 output / accumulator or NULL
+    __nv_bfloat16 *y16;         // bf16 output or NULL
+    const float *y_cpu;         // optional fp32 addend
+    __nv_bfloat16 *x_resid;     // optional bf16 in/out residual stream
+};
+int launch_combine(const Dims &dm, const CombineArgs &a, const Tables &tb, cudaStream_t st);
+
+// ---- small device helpers
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// bf16 pair packed in a 32-bit word -> two fp32 (exact)
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+__device__ __forceinline__ uint4 ldg_stream(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
+
+}  // namespace spice

@@ -1,0 +1,37 @@
+"""GPU-side test helpers: upload a synthetic workload, run the library, compare with the oracle."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from paper_2608_21240_b200 import binding as B
+from paper_2608_21240_b200 import workloads as W
+
+Y_RTOL, Y_ATOL = 1e-2, 1e-3      # max|gpu - oracle| <= 1e-2 * max|oracle| + 1e-3
+GATE_ATOL = 2e-6
+LOGIT_ATOL = 2e-4
+
+
+from paper_2608_21240_b200.binding import bf16_tensor, bits_tensor, cfg_of, upload  # noqa: E402,F401
+
+
+def y_close(y_gpu: np.ndarray, y_ref: np.ndarray):
+    err = np.abs(y_gpu.astype(np.float64) - y_ref).max() if y_ref.size else 0.0
+    bound = Y_RTOL * (np.abs(y_ref).max() if y_ref.size else 0.0) + Y_ATOL
+    return err, bound
+
+
+def check_routing(out, ref, T, K):
+    """Bit-exact idx / cls / counts / residual list; gates within fp32 rounding."""
+    idx = out.idx.cpu().numpy()
+    assert np.array_equal(idx, ref.idx), "top-k indices differ"
+    assert np.abs(out.gate.cpu().numpy().astype(np.float64) - ref.gate).max() <= GATE_ATOL
+    assert np.array_equal(out.cls.cpu().numpy(), ref.cls), "classification differs"
+    counts = out.counts.cpu().numpy()
+    assert counts.tolist() == ref.counts.tolist()
+    n = int(counts[1])
+    assert np.array_equal(out.resid_tok.cpu().numpy()[:n], ref.resid_tok)
+    assert np.array_equal(out.resid_k.cpu().numpy()[:n], ref.resid_k)
+    assert np.array_equal(out.resid_expert.cpu().numpy()[:n], ref.resid_expert)
+    if n:
+        assert np.abs(out.resid_gate.cpu().numpy()[:n].astype(np.float64) - ref.resid_gate).max() <= GATE_ATOL

@@ -1,0 +1,282 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Routing and classification must be bit-exact; outputs must satisfy
+max|gpu - oracle| <= 1e-2 * max|oracle| + 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_21240_b200 import binding as B
+from paper_2608_21240_b200 import workloads as W
+from tests._cases import enforce_margins, run_oracle
+from tests._gpu import (GATE_ATOL, LOGIT_ATOL, bf16_tensor, cfg_of, check_routing, upload, y_close)
+
+pytestmark = pytest.mark.gpu
+
+DECODE_CASES = [("tiny", 4), ("dsv2lite", 1), ("dsv2lite", 4), ("dsv2lite", 16),
+                ("qwen2_57b", 1), ("qwen2_57b", 8), ("qwen2_57b", 32)]
+
+
+def _layer_case(name, T, variant=0, margin=1e-3, **mk):
+    wl = W.make_layer(name, T, variant=variant, **mk)
+    enforce_margins(wl, margin)
+    return wl
+
+
+@pytest.mark.parametrize("name,T", DECODE_CASES + [("dsv2lite_prefill", 4096)])
+def test_route_topk_bit_exact(name, T):
+    wl = _layer_case(name, T, zipf=(name == "dsv2lite_prefill"))
+    s = wl.shape
+    ref_logits = oracle.router_logits(wl.h, wl.w_router)
+    ref_idx, ref_gate = oracle.topk_gates(ref_logits, s.top_k, 1)
+    L = B.SpiceLayer(cfg_of(s), T)
+    idx, gate, logits = L.route_topk(bf16_tensor(wl.h), bf16_tensor(wl.w_router), want_logits=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    assert np.abs(gate.cpu().numpy() - ref_gate).max() <= GATE_ATOL
+    assert np.abs(logits.cpu().numpy() - ref_logits).max() <= LOGIT_ATOL
+    assert L.device_status() == 0
+    L.close()
+
+
+@pytest.mark.parametrize("N,K,d,T,norm", [(10, 3, 264, 5, 0), (64, 1, 512, 3, 1), (7, 7, 128, 2, 1),
+                                           (160, 6, 1024, 70, 1), (1024, 32, 64, 3, 0)])
+def test_route_topk_odd_shapes(N, K, d, T, norm):
+    s = W.scaled_shape(W.SHAPES["tiny"], d=d, n_experts=N, top_k=K, n_slots=min(5, N), norm_topk=norm)
+    wl = _layer_case(s, T, variant=3, margin=1e-3 if N < 1024 else 1e-5)   # 33 of 1024 logits cannot be 1e-3 apart
+    ref_idx, ref_gate = oracle.topk_gates(oracle.router_logits(wl.h, wl.w_router), K, norm)
+    L = B.SpiceLayer(cfg_of(s), T)
+    idx, gate = L.route_topk(bf16_tensor(wl.h), bf16_tensor(wl.w_router))
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    assert np.abs(gate.cpu().numpy() - ref_gate).max() <= GATE_ATOL
+    L.close()
+
+
+def test_route_topk_ties_go_to_lower_index():
+    s = W.scaled_shape(W.SHAPES["tiny"], d=64, n_experts=12, top_k=4)
+    wr = np.zeros((12, 64), np.float32)
+    wr[[1, 2, 4], 0] = 3.0       # three equal winners
+    wr[5, 0] = 2.0
+    h = np.zeros((2, 64), np.float32)
+    h[:, 0] = 1.0
+    L = B.SpiceLayer(cfg_of(s), 2)
+    idx, gate = L.route_topk(bf16_tensor(h), bf16_tensor(wr))
+    ref_idx, ref_gate = oracle.topk_gates(oracle.router_logits(h, wr), 4, 1)
+    assert idx.cpu().numpy().tolist() == [[1, 2, 4, 5]] * 2 == ref_idx.tolist()
+    assert np.abs(gate.cpu().numpy() - ref_gate).max() <= GATE_ATOL
+    L.close()
+
+
+@pytest.mark.parametrize("name,T", DECODE_CASES)
+def test_classify_bit_exact(name, T):
+    wl = _layer_case(name, T, variant=1)
+    s = wl.shape
+    ref = run_oracle(wl, skip_ffn=True)
+    L = B.SpiceLayer(cfg_of(s), T)
+    idx = torch.from_numpy(ref.idx).cuda()
+    gate = torch.from_numpy(ref.gate.astype(np.float32)).cuda()
+    cls, slot, counts, (rt, rk, re_, rg) = L.classify_misses(idx, gate, torch.from_numpy(wl.slot_of_expert).cuda(),
+                                                             torch.from_numpy(wl.conf).cuda())
+    assert np.array_equal(cls.cpu().numpy(), ref.cls)
+    exp_slot = np.where(ref.cls == oracle.HIT, wl.slot_of_expert[ref.idx], -1)
+    assert np.array_equal(slot.cpu().numpy(), exp_slot)
+    assert counts.cpu().numpy().tolist() == ref.counts.tolist()
+    n = int(ref.counts[1])
+    assert np.array_equal(rt.cpu().numpy()[:n], ref.resid_tok) and np.array_equal(rk.cpu().numpy()[:n], ref.resid_k)
+    assert np.array_equal(re_.cpu().numpy()[:n], ref.resid_expert)
+    assert np.array_equal(rg.cpu().numpy()[:n], ref.resid_gate.astype(np.float32))
+    assert L.device_status() == 0
+    L.close()
+
+
+def test_classify_threshold_edges_and_scalar_conf():
+    s = W.scaled_shape(W.SHAPES["tiny"], n_experts=8, top_k=4, tau=0.6)
+    tau = np.float32(0.6)
+    idx = np.array([[0, 1, 2, 3], [4, 5, 6, 7]], np.int32)
+    soe = np.array([2, -1, -1, -1, -1, 0, -1, -1], np.int32)
+    conf = np.full((2, 8), 0.9, np.float32)
+    conf[0, 1] = tau
+    conf[0, 2] = np.nextafter(tau, np.float32(0))
+    conf[0, 3] = np.nan
+    conf[1, 4] = 0.0
+    gate = np.full((2, 4), 0.25, np.float32)
+    ref_cls, ref_counts = oracle.classify(idx, (soe >= 0).astype(np.uint8), conf, float(tau))
+    L = B.SpiceLayer(cfg_of(s, tau=float(tau)), 2)
+    cls, slot, counts, _ = L.classify_misses(*(torch.from_numpy(a).cuda() for a in (idx, gate, soe, conf)))
+    assert cls.cpu().numpy().tolist() == ref_cls.tolist() == [[0, 1, 2, 1], [2, 0, 1, 1]]
+    assert counts.cpu().numpy().tolist() == ref_counts.tolist()
+    L.close()
+    # one confidence per token
+    L = B.SpiceLayer(cfg_of(s, tau=float(tau), conf_per_expert=False), 2)
+    c1 = np.array([0.1, 0.9], np.float32)
+    cls, _, _, _ = L.classify_misses(*(torch.from_numpy(a).cuda() for a in (idx, gate, soe, c1)))
+    ref_cls, _ = oracle.classify(idx, (soe >= 0).astype(np.uint8), c1, float(tau))
+    assert np.array_equal(cls.cpu().numpy(), ref_cls)
+    L.close()
+
+
+def _fwd_and_check(wl, tokens=None, y_cpu=None, **ora):
+    s = wl.shape
+    ref = run_oracle(wl, tokens=tokens, **ora)
+    L = B.SpiceLayer(cfg_of(s, tau=ora.get("tau"), norm_topk=ora.get("norm_topk")), wl.T)
+    w = upload(wl)
+    if "resident" in ora:
+        raise AssertionError("change residency through wl.set_residency so the pool matches")
+    conf = torch.from_numpy(np.ascontiguousarray(ora.get("conf", wl.conf))).cuda()
+    out = L.moe_layer_fwd(w, bf16_tensor(wl.h), conf, y_cpu_residual=y_cpu)
+    torch.cuda.synchronize()
+    check_routing(out, ref, wl.T, s.top_k)
+    y = out.y.float().cpu().numpy()
+    if tokens is not None:
+        y = y[np.asarray(tokens)]
+    assert np.isfinite(y).all()
+    err, bound = y_close(y, ref.y if y_cpu is None else ref.y + y_cpu.cpu().numpy()[ref.rows])
+    assert err <= bound, f"max err {err:.3e} > bound {bound:.3e}"
+    assert L.device_status() == 0
+    return L, w, out, ref
+
+
+@pytest.mark.parametrize("name,T", DECODE_CASES)
+def test_moe_layer_fwd_matches_oracle(name, T):
+    wl = _layer_case(name, T)
+    L, w, out, ref = _fwd_and_check(wl, want_full=False)
+    assert ref.counts[0] > 0
+    L.close()
+
+
+@pytest.mark.parametrize("T", [3, 5, 13, 37])
+def test_moe_layer_fwd_ragged_token_counts_and_dims(T):
+    s = W.scaled_shape(W.SHAPES["tiny"], d=264, n_experts=10, top_k=3, inter=200, inter_shared=328, lore_rank=24,
+                       n_slots=4)
+    wl = _layer_case(s, T, variant=T)
+    L, *_ = _fwd_and_check(wl, want_full=False)
+    L.close()
+
+
+def test_moe_layer_fwd_degenerate_residency():
+    s = W.SHAPES["tiny"]
+    # all hit
+    wl = _layer_case(W.scaled_shape(s, n_slots=8), 4, variant=5)
+    L, w, out, ref = _fwd_and_check(wl, want_full=False)
+    assert ref.counts.tolist() == [8, 0, 0]
+    L.close()
+    # nothing resident: all misses, mixed low-confidence / exact
+    wl = _layer_case(s, 4, variant=6, n_resident=0)
+    L, w, out, ref = _fwd_and_check(wl, want_full=False)
+    assert ref.counts[0] == 0 and ref.counts[1] > 0 and ref.counts[2] > 0
+    L.close()
+    # all misses low-confidence (tau > 1) and all exact (tau = 0)
+    for tau in (1.5, 0.0):
+        wl = _layer_case(s, 4, variant=7, n_resident=0)
+        L, w, out, ref = _fwd_and_check(wl, want_full=False, tau=tau)
+        assert ref.counts[2 if tau > 1 else 1] == 8
+        L.close()
+
+
+def test_moe_layer_fwd_unnormalised_gates_and_cpu_residual_and_resid_stream():
+    wl = _layer_case("tiny", 4, variant=8)
+    s = wl.shape
+    ref = run_oracle(wl, want_full=True, norm_topk=0)
+    # exact-recovery outputs computed elsewhere are merged by the layer call
+    y_cpu = torch.from_numpy((ref.y_full - ref.y).astype(np.float32)).cuda()
+    L = B.SpiceLayer(cfg_of(s, norm_topk=0), wl.T)
+    w = upload(wl)
+    x0 = torch.randn(wl.T, s.d, device="cuda").bfloat16()
+    x = x0.clone()
+    out = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda(), y_cpu_residual=y_cpu, x_resid=x)
+    check_routing(out, ref, wl.T, s.top_k)
+    err, bound = y_close(out.y.float().cpu().numpy(), ref.y_full)
+    assert err <= bound
+    errx, boundx = y_close(x.float().cpu().numpy(), x0.float().cpu().numpy().astype(np.float64) + ref.y_full)
+    assert errx <= boundx + 2e-2    # bf16 rounding of the O(1) residual stream
+    L.close()
+
+
+def test_split_exports_compose_to_the_fused_call():
+    wl = _layer_case("dsv2lite", 4, variant=2)
+    s = wl.shape
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    w = upload(wl)
+    h = bf16_tensor(wl.h)
+    conf = torch.from_numpy(wl.conf).cuda()
+    fused = L.moe_layer_fwd(w, h, conf)
+    idx, gate = L.route_topk(h, w.w_router)
+    cls, slot, counts, resid = L.classify_misses(idx, gate, w.slot_of_expert, conf)
+    assert torch.equal(idx, fused.idx) and torch.equal(gate, fused.gate) and torch.equal(cls, fused.cls)
+    assert torch.equal(counts, fused.counts)
+    y = torch.zeros(wl.T, s.d, device="cuda")
+    L.grouped_expert_ffn(w, h, idx, gate, cls, slot, y)
+    y_hit = y.clone()
+    L.lore_surrogate(w, h, idx, gate, cls, y)
+    torch.cuda.synchronize()
+    ref = run_oracle(wl, want_full=False)
+    err, bound = y_close(y.cpu().numpy(), ref.y)
+    assert err <= bound
+    assert (y.bfloat16().float() - fused.y.float()).abs().max().item() <= 2e-2 * fused.y.float().abs().max().item()
+    # the routed part alone: oracle with the shared/LoRE part removed = hits only
+    hits_only = np.zeros_like(ref.y)
+    for t in range(wl.T):
+        for k in range(s.top_k):
+            if ref.cls[t, k] == oracle.HIT:
+                e = int(ref.idx[t, k])
+                hits_only[t] += ref.gate[t, k] * oracle.swiglu_ffn(*wl.expert(e), wl.h[t])
+    err, bound = y_close(y_hit.cpu().numpy(), hits_only)
+    assert err <= bound
+    L.close()
+
+
+def test_batch_independence_and_repeatability():
+    wl = _layer_case("dsv2lite", 16, variant=4)
+    s = wl.shape
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    w = upload(wl)
+    h = bf16_tensor(wl.h)
+    conf = torch.from_numpy(wl.conf).cuda()
+    a = L.moe_layer_fwd(w, h, conf)
+    b = L.moe_layer_fwd(w, h, conf)
+    assert torch.equal(a.y, b.y), "two runs on the same inputs must be bit-identical"
+    for t in (0, 7, 15):
+        one = L.moe_layer_fwd(w, h[t:t + 1].contiguous(), conf[t:t + 1].contiguous())
+        assert torch.equal(one.idx[0], a.idx[t]) and torch.equal(one.cls[0], a.cls[t])
+        diff = (one.y[0].float() - a.y[t].float()).abs().max().item()
+        assert diff <= 1e-2 * a.y[t].float().abs().max().item() + 1e-3
+    L.close()
+
+
+def test_zero_tokens_and_argument_errors():
+    s = W.SHAPES["tiny"]
+    wl = W.make_layer(s, 4)
+    L = B.SpiceLayer(cfg_of(s), 4)
+    w = upload(wl)
+    h0 = torch.empty(0, s.d, dtype=torch.bfloat16, device="cuda")
+    c0 = torch.empty(0, s.n_experts, device="cuda")
+    out = L.moe_layer_fwd(w, h0, c0)
+    assert out.counts.cpu().tolist() == [0, 0, 0] and L.launch_count() == 0
+    with pytest.raises(B.SpiceError):   # more tokens than the ctx was created for
+        L.moe_layer_fwd(w, bf16_tensor(np.zeros((5, s.d), np.float32)), torch.zeros(5, s.n_experts, device="cuda"))
+    with pytest.raises(B.SpiceError):   # misaligned activation pointer
+        buf = torch.zeros(4 * s.d + 8, dtype=torch.bfloat16, device="cuda")
+        L.moe_layer_fwd(w, buf[1:1 + 4 * s.d].view(4, s.d), torch.zeros(4, s.n_experts, device="cuda"))
+    with pytest.raises(B.SpiceError):
+        B.SpiceLayer(cfg_of(W.scaled_shape(s, d=100)), 4)      # d not a multiple of 8
+    with pytest.raises(B.SpiceError):
+        B.SpiceLayer(cfg_of(W.scaled_shape(s, top_k=9)), 4)    # K > N
+    L.close()
+
+
+def test_corrupt_slot_table_sets_status_without_faulting():
+    wl = _layer_case("tiny", 4, variant=9)
+    s = wl.shape
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    w = upload(wl)
+    ref = run_oracle(wl, skip_ffn=True)
+    e_bad = int(ref.idx[0, 0])
+    w.slot_of_expert[e_bad] = s.n_slots + 3          # points outside the pool
+    out = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
+    torch.cuda.synchronize()
+    assert L.device_status() == 5                    # SPICE_ERR_BAD_TABLE, sticky until read
+    assert L.device_status() == 0
+    cls = out.cls.cpu().numpy()
+    assert (cls[ref.idx == e_bad] == B.MISS_EXACT).all()
+    assert torch.isfinite(out.y.float()).all()
+    L.close()
