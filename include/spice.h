@@ -148,6 +148,13 @@ spice_status spice_get_device_status(spice_ctx *ctx, int32_t *code /* host */);
 /* Number of kernels the library has launched through ctx since it was created (host counter). */
 spice_status spice_launch_count(const spice_ctx *ctx, int64_t *launches /* host */);
 
+/* Knobs (host only).  SPICE_OPT_PATH: 0 = choose the kernel path by batch size (default),
+ * 1 = always use the general-shape kernels.  SPICE_OPT_SPIN_LIMIT: number of polls after which a
+ * dependency wait inside the fused decode kernel gives up and reports SPICE_ERR_TIMEOUT
+ * (default 2^20; a poll takes 0.1 to 1 us). */
+enum { SPICE_OPT_PATH = 0, SPICE_OPT_SPIN_LIMIT = 1 };
+spice_status spice_set_option(spice_ctx *ctx, int32_t option, int64_t value);
+
 /* Text for a status code (static storage, never NULL). */
 const char *spice_status_string(spice_status s);
 

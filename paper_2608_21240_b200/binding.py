@@ -54,7 +54,7 @@ def lib() -> C.CDLL:
         L.spice_version.restype = C.c_int32
         for name in ("spice_create", "spice_destroy", "spice_workspace_bytes", "spice_route_topk",
                      "spice_classify_misses", "spice_grouped_expert_ffn", "spice_lore_surrogate",
-                     "spice_moe_layer_fwd", "spice_get_device_status", "spice_launch_count"):
+                     "spice_moe_layer_fwd", "spice_get_device_status", "spice_launch_count", "spice_set_option"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -102,6 +102,13 @@ def spice_launch_count(ctx) -> int:
     n = C.c_int64()
     _check(lib().spice_launch_count(ctx, C.byref(n)), "spice_launch_count")
     return n.value
+
+
+OPT_PATH, OPT_SPIN_LIMIT = 0, 1
+
+
+def spice_set_option(ctx, option: int, value: int) -> None:
+    _check(lib().spice_set_option(ctx, C.c_int32(option), C.c_int64(value)), "spice_set_option")
 
 
 def spice_get_device_status(ctx) -> int:
@@ -248,6 +255,9 @@ class SpiceLayer:
         spice_moe_layer_fwd(self.ctx, w.c_struct(), h, conf, T, o.y, y_cpu_residual, x_resid, o.idx, o.gate, o.cls,
                             o.counts, o.resid_tok, o.resid_k, o.resid_expert, o.resid_gate, stream)
         return o
+
+    def set_option(self, option: int, value: int) -> None:
+        spice_set_option(self.ctx, option, value)
 
     def device_status(self) -> int:
         return spice_get_device_status(self.ctx)

@@ -17,6 +17,15 @@ struct spice_ctx {
     float *ws_gate;
     uint8_t *ws_cls;
     float *y32;        // [Tm, d] fp32 accumulator of the fused call
+    // fused decode kernel
+    float *logits;                  // [Td, N]
+    __nv_bfloat16 *act_hit16, *act_shared16, *z16;
+    int32_t *sync;
+    int32_t sync_words;
+    int32_t decode_tokens;          // largest T the decode buffers were sized for (0: path unavailable)
+    int n_sms, max_smem_optin;
+    int64_t opt_path;               // 0 auto, 1 general kernels only
+    int64_t opt_spin_limit;
     int64_t launches;
 };
 
@@ -58,6 +67,13 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->ws_gate = cv.take<float>(n);
     c->ws_cls = cv.take<uint8_t>(n);
     c->y32 = cv.take<float>(Tm * g.d);
+    const size_t Td = Tm < 32 ? Tm : 32, nd = Td * K;
+    c->logits = cv.take<float>(Td * g.n_experts);
+    c->act_hit16 = cv.take<__nv_bfloat16>(nd * g.inter);
+    c->act_shared16 = cv.take<__nv_bfloat16>(Td * g.inter_shared);
+    c->z16 = cv.take<__nv_bfloat16>(nd * g.lore_rank);
+    c->sync_words = SY_GROUP0 + 1 + g.n_slots + g.n_experts;
+    c->sync = cv.take<int32_t>(c->sync_words);
     *total = (cv.off + 255) & ~size_t(255);
 }
 
@@ -136,6 +152,16 @@ spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg
     c->cfg = *cfg;
     c->max_tokens = max_tokens;
     c->launches = 0;
+    c->opt_path = 0;
+    c->opt_spin_limit = 1 << 20;
+    int coop = 0;
+    if (cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&c->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device) != cudaSuccess) {
+        delete c;
+        return SPICE_ERR_CUDA;
+    }
+    c->decode_tokens = (coop && decode_prepare(c->max_smem_optin) == 0) ? (max_tokens < 32 ? max_tokens : 32) : 0;
     carve(c, nullptr, &c->ws_bytes);
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -180,8 +206,25 @@ spice_status spice_get_device_status(spice_ctx *ctx, int32_t *code) {
     int32_t v = 0;
     if (cudaMemcpy(&v, ctx->tb.status, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return SPICE_ERR_CUDA;
     if (cudaMemset(ctx->tb.status, 0, sizeof(int32_t)) != cudaSuccess) return SPICE_ERR_CUDA;
+    // a kernel that gave up may have left dependency counters behind
+    if (v != 0 && cudaMemset(ctx->sync, 0, sizeof(int32_t) * ctx->sync_words) != cudaSuccess) return SPICE_ERR_CUDA;
     *code = v;
     return SPICE_OK;
+}
+
+spice_status spice_set_option(spice_ctx *ctx, int32_t option, int64_t value) {
+    if (!ctx) return SPICE_ERR_INVALID_ARG;
+    switch (option) {
+        case SPICE_OPT_PATH:
+            if (value != 0 && value != 1) return SPICE_ERR_INVALID_ARG;
+            ctx->opt_path = value;
+            return SPICE_OK;
+        case SPICE_OPT_SPIN_LIMIT:
+            if (value < 1 || value > (1ll << 30)) return SPICE_ERR_INVALID_ARG;
+            ctx->opt_spin_limit = value;
+            return SPICE_OK;
+    }
+    return SPICE_ERR_INVALID_ARG;
 }
 
 spice_status spice_route_topk(spice_ctx *ctx, const spice_bf16 *h, const spice_bf16 *w_router, int32_t T,
@@ -274,6 +317,43 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     if (!(resid_tok && resid_k && resid_expert && resid_gate)) resid_tok = resid_k = resid_expert = nullptr, resid_gate = nullptr;
     const Dims dm = dims_of(ctx, T);
     const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
+    if (ctx->opt_path == 0 && T <= ctx->decode_tokens && decode_supported(dm, (size_t)ctx->max_smem_optin)) {
+        // small batch: one persistent kernel for the whole layer
+        DecodeParams p;
+        p.dm = dm;
+        p.norm_topk = ctx->cfg.norm_topk;
+        p.conf_stride = ctx->cfg.conf_stride;
+        p.tau = ctx->cfg.tau;
+        p.n_r1 = dm.N >= 64 ? 8 : (dm.N + 7) / 8;
+        p.spin_limit = (int32_t)ctx->opt_spin_limit;
+        p.sync_words = ctx->sync_words;
+        p.h = hb;
+        p.conf = conf;
+        p.w = *w;
+        p.idx = idx;
+        p.gate = gate;
+        p.cls = cls;
+        p.counts = counts;
+        p.resid_tok = resid_tok;
+        p.resid_k = resid_k;
+        p.resid_expert = resid_expert;
+        p.resid_gate = resid_gate;
+        p.y16 = reinterpret_cast<__nv_bfloat16 *>(y);
+        p.y_cpu = y_cpu_residual;
+        p.x_resid = reinterpret_cast<__nv_bfloat16 *>(x_resid);
+        p.tb = ctx->tb;
+        p.logits = ctx->logits;
+        p.act_hit16 = ctx->act_hit16;
+        p.act_shared16 = ctx->act_shared16;
+        p.z16 = ctx->z16;
+        p.sync = ctx->sync;
+        int n = launch_decode(p, ctx->n_sms, st);
+        if (n > 0) {
+            ctx->launches += n;
+            return SPICE_OK;
+        }
+        // cooperative launch refused (e.g. device shared with another context): use the general path
+    }
     SPICE_LAUNCH(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
                                    gate, nullptr, st));
     SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,

@@ -2,6 +2,7 @@
 // scores", Sec. 4.2).  One CTA owns TPC tokens: its warps share the router rows (each warp takes
 // experts e = warp, warp+nwarps, ...), logits are accumulated in fp32 and parked in shared memory,
 // then one warp per token does K rounds of a shuffle arg-max (ties -> smaller expert index).
+#include "route_device.cuh"
 #include "spice_internal.cuh"
 
 namespace spice {
@@ -57,49 +58,8 @@ __global__ void route_topk_kernel(const __nv_bfloat16 *__restrict__ h, const __n
     for (int tt = warp; tt < TPC; tt += nwarps) {
         const int t = t0 + tt;
         if (t >= T) continue;   // warp-uniform
-        const float *l = lg + tt * N;
-        if (logits_out)
-            for (int e = lane; e < N; e += 32) logits_out[(size_t)t * N + e] = l[e];
-        uint32_t taken = 0;     // bit i: expert lane + 32*i already selected (N <= 1024)
-        float m = 0.f, denom = 0.f, my_val = 0.f;
-        int my_idx = 0;
-        for (int k = 0; k < K; ++k) {
-            float bv = -INFINITY;
-            int be = 0x7fffffff;
-            for (int i = 0, e = lane; e < N; ++i, e += 32) {
-                if ((taken >> i) & 1u) continue;
-                float v = l[e];
-                if (!(v == v)) v = -INFINITY;   // NaN never wins
-                if (be == 0x7fffffff || v > bv) { bv = v; be = e; }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-                int oe = __shfl_xor_sync(0xffffffffu, be, o);
-                if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
-            }
-            if ((be & 31) == lane) taken |= 1u << (be >> 5);
-            if (k == 0) {
-                m = bv;
-                if (!norm_topk) {   // full-softmax denominator
-                    float s = 0.f;
-                    for (int e = lane; e < N; e += 32) s += expf(l[e] - m);
-                    denom = warp_sum(s);
-                }
-            }
-            if (lane == k) { my_val = bv; my_idx = be; }
-        }
-        float p = (lane < K) ? expf(my_val - m) : 0.f;
-        if (norm_topk) {
-            // sum the K numerators in k order on every lane (deterministic, matches the definition)
-            float s = 0.f;
-            for (int k = 0; k < K; ++k) s += __shfl_sync(0xffffffffu, p, k);
-            denom = s;
-        }
-        if (lane < K) {
-            idx[(size_t)t * K + lane] = my_idx;
-            gate[(size_t)t * K + lane] = p / denom;
-        }
+        warp_topk_gates(lg + tt * N, N, K, norm_topk, lane, idx + (size_t)t * K, gate + (size_t)t * K,
+                        logits_out ? logits_out + (size_t)t * N : nullptr);
     }
 }
 

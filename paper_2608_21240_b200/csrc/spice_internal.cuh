@@ -75,6 +75,41 @@ struct CombineArgs {
 };
 int launch_combine(const Dims &dm, const CombineArgs &a, const Tables &tb, cudaStream_t st);
 
+// ---- fused decode kernel (decode.cu)
+// words of the dependency-counter array
+enum { SY_ABORT = 0, SY_TEAMS_DONE, SY_R1_DONE, SY_ROUTE_DONE, SY_P2_DONE, SY_GROUP0 = 8 };
+
+struct DecodeParams {
+    Dims dm;
+    int32_t norm_topk, conf_stride;
+    float tau;
+    int32_t n_r1;         // router tasks
+    int32_t spin_limit;   // iterations after which a dependency wait gives up
+    int32_t sync_words;   // length of sync[]
+    const __nv_bfloat16 *h;
+    const float *conf;
+    spice_layer_weights w;
+    int32_t *idx;
+    float *gate;
+    uint8_t *cls;
+    int32_t *counts;
+    int32_t *resid_tok, *resid_k, *resid_expert;
+    float *resid_gate;
+    __nv_bfloat16 *y16;
+    const float *y_cpu;
+    __nv_bfloat16 *x_resid;
+    Tables tb;
+    float *logits;                 // [T,N]
+    __nv_bfloat16 *act_hit16;      // [Tm*K, I]  perm_hit order
+    __nv_bfloat16 *act_shared16;   // [Tm, I_s]
+    __nv_bfloat16 *z16;            // [Tm*K, r]  perm_low order
+    int32_t *sync;                 // [sync_words] zero between launches
+};
+size_t decode_smem_bytes(const Dims &dm);
+bool decode_supported(const Dims &dm, size_t max_smem);
+int decode_prepare(int max_smem_optin);
+int launch_decode(const DecodeParams &p, int n_ctas, cudaStream_t st);
+
 // ---- small device helpers
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

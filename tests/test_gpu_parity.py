@@ -115,10 +115,12 @@ def test_classify_threshold_edges_and_scalar_conf():
     L.close()
 
 
-def _fwd_and_check(wl, tokens=None, y_cpu=None, **ora):
+def _fwd_and_check(wl, tokens=None, y_cpu=None, general_path=False, **ora):
     s = wl.shape
     ref = run_oracle(wl, tokens=tokens, **ora)
     L = B.SpiceLayer(cfg_of(s, tau=ora.get("tau"), norm_topk=ora.get("norm_topk")), wl.T)
+    if general_path:
+        L.set_option(B.OPT_PATH, 1)
     w = upload(wl)
     if "resident" in ora:
         raise AssertionError("change residency through wl.set_residency so the pool matches")
@@ -144,12 +146,48 @@ def test_moe_layer_fwd_matches_oracle(name, T):
     L.close()
 
 
-@pytest.mark.parametrize("T", [3, 5, 13, 37])
+@pytest.mark.parametrize("name,T", [("tiny", 4), ("dsv2lite", 4), ("dsv2lite", 16)])
+def test_moe_layer_fwd_general_kernels_match_oracle(name, T):
+    """The any-shape kernels (forced) against the oracle, and against the fused decode kernel."""
+    wl = _layer_case(name, T)
+    L, w, out, ref = _fwd_and_check(wl, want_full=False, general_path=True)
+    n_general = L.launch_count()
+    L.set_option(B.OPT_PATH, 0)
+    fused = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
+    assert L.launch_count() - n_general == 1 and n_general > 1
+    assert torch.equal(fused.idx, out.idx) and torch.equal(fused.gate, out.gate) and torch.equal(fused.cls, out.cls)
+    diff = (fused.y.float() - out.y.float()).abs().max().item()
+    assert diff <= 1e-2 * out.y.float().abs().max().item() + 1e-3
+    L.close()
+
+
+@pytest.mark.parametrize("T", [3, 5, 13, 32, 37])
 def test_moe_layer_fwd_ragged_token_counts_and_dims(T):
     s = W.scaled_shape(W.SHAPES["tiny"], d=264, n_experts=10, top_k=3, inter=200, inter_shared=328, lore_rank=24,
                        n_slots=4)
     wl = _layer_case(s, T, variant=T)
     L, *_ = _fwd_and_check(wl, want_full=False)
+    L.close()
+
+
+def test_expired_dependency_wait_reports_timeout_and_recovers():
+    """A wait that cannot be satisfied within its poll limit ends the kernel with a status, not a hang."""
+    wl = _layer_case("dsv2lite", 16, variant=11)
+    s = wl.shape
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    w = upload(wl)
+    h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+    good = L.moe_layer_fwd(w, h, conf)
+    assert L.device_status() == 0
+    L.set_option(B.OPT_SPIN_LIMIT, 1)          # one poll: the router cannot be done by then
+    L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert L.device_status() == 6               # SPICE_ERR_TIMEOUT
+    L.set_option(B.OPT_SPIN_LIMIT, 1 << 20)
+    again = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    assert torch.equal(again.y, good.y) and torch.equal(again.idx, good.idx)
     L.close()
 
 
