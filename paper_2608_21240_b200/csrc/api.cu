@@ -324,7 +324,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         p.norm_topk = ctx->cfg.norm_topk;
         p.conf_stride = ctx->cfg.conf_stride;
         p.tau = ctx->cfg.tau;
-        p.n_r1 = dm.N >= 64 ? 8 : (dm.N + 7) / 8;
+        p.n_r1 = dm.N;   // one router task per expert
         p.spin_limit = (int32_t)ctx->opt_spin_limit;
         p.sync_words = ctx->sync_words;
         p.h = hb;

@@ -8,24 +8,25 @@
 // tasks, dealt round-robin to the teams; dependencies between tasks are counters in global memory
 // (release add by the producer, acquire poll by the consumer, every poll bounded):
 //
-//   A  R1   router logits for a slice of experts              (no dependency)
+//   A  R1   router logits of one expert for all tokens         (no dependency)
 //      R2   top-k, gates, classification, residual list,
 //           grouping of (t,k) entries by slot / expert         (all R1 done)
 //      P1s  16 rows of the shared expert's gate/up + SwiGLU    (no dependency)
 //   B  P1   16 rows of gate/up of one hit slot, or 16 rows of
 //           LoRE A_e of one low-confidence expert              (R2 done)
 //   C  P2   16 rows of a down projection (shared / hit slot),
-//           or 128 rows of LoRE B_e                            (that group's P1 rows done)
+//           or 128 rows of LoRE B_e                            (all P1 rows done)
 //   D  P3   combine: y_t = c_t S(h_t) + sum_k g_k part_{t,k}   (all P2 done)
 //
 // A task streams its weight rows with 128-bit loads straight into mma.sync.m16n8k16 A fragments
 // (the reduction index is permuted identically for both operands, so no shuffle is needed); the
 // tokens (B fragments, 8 per n-tile) come from shared memory (P1) or L2 (P2).  The 8 warps of a
 // team split the reduction dimension and add their partial tiles in shared memory in a fixed
-// order, so results are bit-reproducible.  Tensor cores are used only because they make the
-// per-byte instruction cost negligible; the kernel is bandwidth-bound by construction.
-#include <cooperative_groups.h>
-
+// order, so results are bit-reproducible.  A release costs a fence of about one memory round trip,
+// so a warp counts its finished P1 / P2 tiles in a register and publishes the count once, when it
+// first has to wait for the next phase (or leaves).
+// Tensor cores are used only because they make the per-byte instruction cost negligible; the
+// kernel is bandwidth-bound by construction.
 #include "route_device.cuh"
 #include "spice_internal.cuh"
 
@@ -55,6 +56,16 @@ __device__ __forceinline__ void red_release_add(int *p, int v) {
 __device__ __forceinline__ void team_sync(int team) {
     asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(TEAM) : "memory");
 }
+// team barrier that also ORs a flag over the team (uniform result)
+__device__ __forceinline__ bool team_sync_or(int team, bool flag) {
+    int out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.or.pred q, %2, %3, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out)
+        : "r"((int)flag), "r"(team + 1), "r"(TEAM)
+        : "memory");
+    return out != 0;
+}
 __device__ __forceinline__ uint4 ldcg128(const void *p) {
     uint4 v;
     asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
@@ -73,43 +84,90 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Optional timeline recorder (compiled in only with -DSPICE_PROF; used while tuning).
+#ifdef SPICE_PROF
+constexpr int PROF_TEAMS = 296, PROF_EVENTS = 512;
+__device__ unsigned long long g_prof[PROF_TEAMS * PROF_EVENTS * 2];
+__device__ __forceinline__ unsigned long long prof_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+#define PROF(tc, tag)                                                                        \
+    do {                                                                                     \
+        if ((tc).ttid == 0 && (tc).gteam < PROF_TEAMS && (tc).nprof < PROF_EVENTS) {         \
+            g_prof[((tc).gteam * PROF_EVENTS + (tc).nprof) * 2] = (unsigned long long)(tag); \
+            g_prof[((tc).gteam * PROF_EVENTS + (tc).nprof) * 2 + 1] = prof_now();            \
+            (tc).nprof++;                                                                    \
+        }                                                                                    \
+    } while (0)
+#else
+#define PROF(tc, tag) \
+    do {              \
+    } while (0)
+#endif
+
 struct TeamCtx {
+#ifdef SPICE_PROF
+    int gteam, nprof;
+#endif
     int team, ttid, twarp, lane;
-    float *red;        // [TW][2][NT][128] partial tiles of this team
-    int *tok;          // [32] token of every B row; orow = tok + 32: output row (position, entry id
-                       // or token) of every B row; flag = tok + 64: broadcast slot
-    __device__ __forceinline__ int *orow() const { return tok + 32; }
-    __device__ __forceinline__ int *flag() const { return tok + 64; }
+    int n_p1, n_p2;      // P1 / P2 tiles this warp has finished but not yet published
+    bool p1_all;         // this warp has seen every P1 tile of the layer published
+    float *red;          // [TW][2][NT][128] partial tiles of this team
+    int *flag;           // [2] broadcast slots
+    GroupDesc *gtab;     // [1 + S + N] team-private copy of the group table
+    int *perm_h;         // [T*K] copy of perm_hit
+    int *perm_l;         // [T*K] copy of perm_low
 };
 
-// Bounded wait (leader thread only): true when *ctr >= target, false on abort or when the limit
-// expires, in which case the sticky status and the abort flag are set.
-__device__ bool wait_ge(const int *ctr, int target, int *sync, int *status, int spin_limit) {
+// this warp's global stores are done -> publish one unit of progress (counters count warps)
+__device__ __forceinline__ void warp_signal(const TeamCtx &tc, int *ctr) {
+    __syncwarp();
+    if (tc.lane == 0) red_release_add(ctr, 1);
+}
+// Publish this warp's finished-tile counts (one release each); called before the warp waits for
+// a later phase and when it leaves the task loop.
+__device__ __forceinline__ void flush_counts(TeamCtx &tc, int *sync) {
+    if (tc.n_p1 | tc.n_p2) {   // warp-uniform
+        __syncwarp();
+        if (tc.lane == 0) {
+            if (tc.n_p1) red_release_add(sync + SY_P1_ALL, tc.n_p1);
+            if (tc.n_p2) red_release_add(sync + SY_P2_DONE, tc.n_p2);
+        }
+        tc.n_p1 = 0;
+        tc.n_p2 = 0;
+    }
+}
+
+// Bounded wait (one thread): true when *ctr >= target, false on abort or when the limit expires,
+// in which case the sticky status and the abort flag are set.
+__device__ __noinline__ bool wait_ge(const int *ctr, int target, int *sync, int *status, int spin_limit) {
     for (int it = 0; it < spin_limit; ++it) {
         if (ld_acquire(ctr) >= target) return true;
-        if (ld_relaxed(sync + SY_ABORT)) return false;
-        if (it > 64) __nanosleep(64);
+        if ((it & 15) == 15 && ld_relaxed(sync + SY_ABORT)) return false;
+        if (it > 32) __nanosleep(32);
     }
     atomicMax(status, (int)SPICE_ERR_TIMEOUT);
     atomicExch(sync + SY_ABORT, 1);
     return false;
 }
 
-__device__ __forceinline__ bool team_wait_ge(const TeamCtx &tc, const int *ctr, int target, const DecodeParams &p) {
-    if (tc.ttid == 0) *tc.flag() = wait_ge(ctr, target, p.sync, p.tb.status, p.spin_limit) ? 1 : 0;
-    team_sync(tc.team);
-    const bool ok = *tc.flag() != 0;
-    team_sync(tc.team);
-    return ok;
+// lane 0 polls, the warp learns the result
+__device__ __forceinline__ bool warp_wait_ge(const TeamCtx &tc, const int *ctr, int target, const DecodeParams &p) {
+    int ok = 1;
+    if (tc.lane == 0) ok = wait_ge(ctr, target, p.sync, p.tb.status, p.spin_limit) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
-// all global stores of the team are done -> publish one unit of progress
-__device__ __forceinline__ void team_signal(const TeamCtx &tc, int *ctr) {
+// leader polls, result is broadcast through a slot: team-uniform result
+__device__ __forceinline__ bool team_wait_ge(TeamCtx &tc, const int *ctr, int target, const DecodeParams &p) {
+    flush_counts(tc, p.sync);
+    if (tc.ttid == 0) tc.flag[0] = wait_ge(ctr, target, p.sync, p.tb.status, p.spin_limit) ? 1 : 0;
     team_sync(tc.team);
-    if (tc.ttid == 0) {
-        __threadfence();
-        red_release_add(ctr, 1);
-    }
+    const bool ok = tc.flag[0] != 0;
+    team_sync(tc.team);
+    return ok;
 }
 
 // exclusive scan over the 256 threads of a team
@@ -137,45 +195,74 @@ __device__ __forceinline__ int team_excl_scan(const TeamCtx &tc, int v, int *wt 
     return wt[tc.twarp] + inc - v;
 }
 
+__device__ __forceinline__ GroupDesc load_group(const GroupDesc *g) {
+    const int4 v = __ldcg(reinterpret_cast<const int4 *>(g));
+    return GroupDesc{v.x, v.y, v.z, v.w};
+}
+
 // ------------------------------------------------------------------------------------------
-// One warp: C[16 x 8*NT] += W[row0 + {g, g+8}][k] * X[token][k] over k-steps [ks0, ks1).
+// The weight rows of one task as this lane sees them.
+struct WRows {
+    const __nv_bfloat16 *p0lo, *p0hi;   // rows g and g+8 of the first matrix
+    const __nv_bfloat16 *p1lo, *p1hi;   // same rows of the second matrix (gate/up pair) or unused
+    int K;                              // reduction length
+    int ks0, ks1;                       // this warp's k-steps
+    bool ok_lo, ok_hi;
+};
+
+// One warp: C[16 x 8*NT] += W[rows g, g+8][k] * X[token][k] over this warp's k-steps.
 // A k-step covers 32 reduction indices; lane (g = lane/4, c = lane%4) owns indices
 // ks*32 + c*8 .. +7 of rows g and g+8 (one 128-bit load each) and of token g of every n-tile.
-template <int NT, bool DUAL, bool B_SMEM, int U>
-__device__ __forceinline__ void warp_mma_range(const __nv_bfloat16 *__restrict__ W0,
-                                               const __nv_bfloat16 *__restrict__ W1, int K, int row_lo, int row_hi,
-                                               bool ok_lo, bool ok_hi, int ks0, int ks1,
-                                               const unsigned long long (&bptr)[NT], const bool (&bok)[NT],
-                                               float (&acc0)[NT][4], float (&acc1)[NT][4], int lane) {
+// The U k-steps of a batch are all loaded before the first mma, so their latencies overlap.
+// `gate` (P2 only): called once, after the first batch of weight loads is in flight and before the
+// first activation load, to wait for the activations to exist.
+template <int NT, bool DUAL, bool B_SMEM, int U, typename Gate>
+__device__ __forceinline__ void warp_mma_range(const WRows &w, const unsigned long long (&bptr)[NT],
+                                               const bool (&bok)[NT], float (&acc0)[NT][4], float (&acc1)[NT][4],
+                                               int lane, Gate gate) {
     const int c = lane & 3;
-    const __nv_bfloat16 *p0lo = W0 + (size_t)row_lo * K, *p0hi = W0 + (size_t)row_hi * K;
-    const __nv_bfloat16 *p1lo = DUAL ? W1 + (size_t)row_lo * K : nullptr, *p1hi = DUAL ? W1 + (size_t)row_hi * K : nullptr;
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    for (int ks = ks0; ks < ks1; ks += U) {
+    bool first = true;
+    for (int ks = w.ks0; ks < w.ks1 || first; ks += U) {
         uint4 a0lo[U], a0hi[U], a1lo[U], a1hi[U];
+        uint4 bg[B_SMEM ? 1 : U][NT];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int kb = (ks + u) * 32 + c * 8;
-            const bool in = (ks + u < ks1) && (kb < K);
-            a0lo[u] = (in && ok_lo) ? ldg_stream(p0lo + kb) : zero;
-            a0hi[u] = (in && ok_hi) ? ldg_stream(p0hi + kb) : zero;
+            const bool in = (ks + u < w.ks1) && (kb < w.K);
+            a0lo[u] = (in && w.ok_lo) ? ldg_stream(w.p0lo + kb) : zero;
+            a0hi[u] = (in && w.ok_hi) ? ldg_stream(w.p0hi + kb) : zero;
             if (DUAL) {
-                a1lo[u] = (in && ok_lo) ? ldg_stream(p1lo + kb) : zero;
-                a1hi[u] = (in && ok_hi) ? ldg_stream(p1hi + kb) : zero;
+                a1lo[u] = (in && w.ok_lo) ? ldg_stream(w.p1lo + kb) : zero;
+                a1hi[u] = (in && w.ok_hi) ? ldg_stream(w.p1hi + kb) : zero;
+            }
+        }
+        if (first) {
+            gate();
+            first = false;
+        }
+        if (!B_SMEM) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int kb = (ks + u) * 32 + c * 8;
+                const bool in = (ks + u < w.ks1) && (kb < w.K);
+#pragma unroll
+                for (int nn = 0; nn < NT; ++nn)
+                    bg[u][nn] = (in && bok[nn])
+                                    ? ldcg128(reinterpret_cast<const unsigned char *>(bptr[nn]) + (size_t)kb * 2)
+                                    : zero;
             }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int kb = (ks + u) * 32 + c * 8;
-            const bool in = (ks + u < ks1) && (kb < K);
-            if (ks + u < ks1) {   // warp-uniform
+            const bool in = (ks + u < w.ks1) && (kb < w.K);
+            if (ks + u < w.ks1) {   // warp-uniform
 #pragma unroll
                 for (int nn = 0; nn < NT; ++nn) {
-                    uint4 b = zero;
-                    if (in && bok[nn]) {
-                        if (B_SMEM) b = lds128((uint32_t)bptr[nn] + kb * 2);
-                        else b = ldcg128(reinterpret_cast<const unsigned char *>(bptr[nn]) + (size_t)kb * 2);
-                    }
+                    uint4 b;
+                    if (B_SMEM) b = (in && bok[nn]) ? lds128((uint32_t)bptr[nn] + kb * 2) : zero;
+                    else b = bg[u][nn];
                     mma_bf16(acc0[nn], a0lo[u].x, a0hi[u].x, a0lo[u].y, a0hi[u].y, b.x, b.y);
                     mma_bf16(acc0[nn], a0lo[u].z, a0hi[u].z, a0lo[u].w, a0hi[u].w, b.z, b.w);
                     if (DUAL) {
@@ -188,39 +275,57 @@ __device__ __forceinline__ void warp_mma_range(const __nv_bfloat16 *__restrict__
     }
 }
 
-__device__ __forceinline__ GroupDesc load_group(const GroupDesc *g) {
-    const int4 v = __ldcg(reinterpret_cast<const int4 *>(g));
-    return GroupDesc{v.x, v.y, v.z, v.w};
-}
-
 enum { EPI_ACT = 0, EPI_Z = 1, EPI_PART = 2 };
 
-// One team, one 16-row tile, reduction split over the 8 warps.
-//   EPI_ACT : rows of W0 = gate, W1 = up; out16[(orow)*ld_out + row] = silu(g)*u          (P1 shared/hit)
-//   EPI_Z   : out16[(orow)*ld_out + row] = sum                                            (P1 LoRE A)
-//   EPI_PART: out32[(orow)*ld_out + row] = sum                                            (P2 down)
-template <int NT, int EPI, bool B_SMEM>
-__device__ __forceinline__ void team_tile_ksplit(const TeamCtx &tc, const __nv_bfloat16 *W0, const __nv_bfloat16 *W1,
-                                                 int row0, int n_rows, int K, int m,
+// where row n of a group lands: the token (shared expert), the position in the group's buffer
+// (P1 of a hit / low group) or the entry id t*K+k (P2 of a hit / low group)
+__device__ __forceinline__ int out_row(const TeamCtx &tc, const GroupDesc &grp, bool by_pos, int n) {
+    if (grp.kind == KIND_SHARED) return n;
+    if (by_pos) return grp.off + n;
+    return (grp.kind == KIND_HIT ? tc.perm_h : tc.perm_l)[grp.off + n];
+}
+
+// One team, one 16-row tile, reduction split over the 8 warps.  Returns false (team-uniform) when
+// some warp's wait failed; nothing is stored then.
+//   EPI_ACT : rows of W0 = gate, W1 = up; out16[orow*ld_out + row] = silu(g)*u          (P1 shared/hit)
+//   EPI_Z   : out16[orow*ld_out + row] = sum                                            (P1 LoRE A)
+//   EPI_PART: out32[orow*ld_out + row] = sum                                            (P2 down)
+template <int NT, int EPI, bool B_SMEM, typename Gate>
+__device__ __forceinline__ bool team_tile_ksplit(TeamCtx &tc, const GroupDesc &grp, const __nv_bfloat16 *W0,
+                                                 const __nv_bfloat16 *W1, int row0, int n_rows, int K,
                                                  const unsigned long long (&bptr)[NT], const bool (&bok)[NT],
-                                                 __nv_bfloat16 *out16, float *out32, int ld_out) {
+                                                 __nv_bfloat16 *out16, float *out32, int ld_out, Gate gate) {
     constexpr bool DUAL = (EPI == EPI_ACT);
     constexpr int MATS = DUAL ? 2 : 1;
-    constexpr int U = DUAL ? (NT == 4 ? 2 : 4) : (NT == 4 ? 4 : 8);
+#ifdef SPICE_U
+    constexpr int U = SPICE_U;
+#else
+    constexpr int U = (NT == 4) ? 2 : 4;
+#endif
     const int g = tc.lane >> 2;
     const int KS = (K + 31) >> 5;
     const int base = KS / TW, rem = KS % TW;
-    const int ks0 = tc.twarp * base + min(tc.twarp, rem);
-    const int ks1 = ks0 + base + (tc.twarp < rem ? 1 : 0);
+    WRows w;
+    w.K = K;
+    w.ks0 = tc.twarp * base + min(tc.twarp, rem);
+    w.ks1 = w.ks0 + base + (tc.twarp < rem ? 1 : 0);
+    const int rlo = row0 + g, rhi = row0 + g + 8;
+    w.ok_lo = rlo < n_rows;
+    w.ok_hi = rhi < n_rows;
+    w.p0lo = W0 + (size_t)(w.ok_lo ? rlo : 0) * K;
+    w.p0hi = W0 + (size_t)(w.ok_hi ? rhi : 0) * K;
+    w.p1lo = DUAL ? W1 + (size_t)(w.ok_lo ? rlo : 0) * K : nullptr;
+    w.p1hi = DUAL ? W1 + (size_t)(w.ok_hi ? rhi : 0) * K : nullptr;
     float acc0[NT][4], acc1[NT][4];
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
         for (int r = 0; r < 4; ++r) acc0[nn][r] = acc1[nn][r] = 0.f;
-    const int rlo = row0 + g, rhi = row0 + g + 8;
-    const bool ok_lo = rlo < n_rows, ok_hi = rhi < n_rows;
-    warp_mma_range<NT, DUAL, B_SMEM, U>(W0, W1, K, ok_lo ? rlo : 0, ok_hi ? rhi : 0, ok_lo, ok_hi, ks0, ks1, bptr, bok,
-                                       acc0, acc1, tc.lane);
+    bool failed = false;
+    warp_mma_range<NT, DUAL, B_SMEM, U>(w, bptr, bok, acc0, acc1, tc.lane, [&]() { failed = !gate(); });
+    PROF(tc, 20);
+    // every warp is past the previous tile's epilogue once it arrives here
+    if (team_sync_or(tc.team, failed)) return false;
     float *red = tc.red;
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn)
@@ -230,31 +335,36 @@ __device__ __forceinline__ void team_tile_ksplit(const TeamCtx &tc, const __nv_b
             if (DUAL) red[((tc.twarp * MATS + 1) * NT + nn) * 128 + r * 32 + tc.lane] = acc1[nn][r];
         }
     team_sync(tc.team);
+    PROF(tc, 21);
     for (int e = tc.ttid; e < NT * 128; e += TEAM) {
         const int nn = e >> 7, r = (e >> 5) & 3, ln = e & 31;
         const int row = row0 + (ln >> 2) + ((r & 2) ? 8 : 0);
         const int n = nn * 8 + 2 * (ln & 3) + (r & 1);
         float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-        for (int w = 0; w < TW; ++w) {
-            s0 += red[((w * MATS + 0) * NT + nn) * 128 + r * 32 + ln];
-            if (DUAL) s1 += red[((w * MATS + 1) * NT + nn) * 128 + r * 32 + ln];
+        for (int wi = 0; wi < TW; ++wi) {
+            s0 += red[((wi * MATS + 0) * NT + nn) * 128 + r * 32 + ln];
+            if (DUAL) s1 += red[((wi * MATS + 1) * NT + nn) * 128 + r * 32 + ln];
         }
-        if (n < m && row < n_rows) {
-            const size_t o = (size_t)tc.orow()[n] * ld_out + row;
+        if (n < grp.m && row < n_rows) {
+            const size_t o = (size_t)out_row(tc, grp, EPI != EPI_PART, n) * ld_out + row;
             if (EPI == EPI_ACT) out16[o] = __float2bfloat16(silu_f(s0) * s1);
             else if (EPI == EPI_Z) out16[o] = __float2bfloat16(s0);
             else out32[o] = s0;
         }
     }
+    PROF(tc, 22);
+    if (EPI == EPI_PART) tc.n_p2++;
+    else tc.n_p1++;
+    return true;
 }
 
 // P2 of a LoRE group: part[entry, j] = sum_q B_e[j,q] z[q]; the reduction (r) is short, so each warp
 // takes its own 16 rows and nothing is exchanged.
-template <int NT>
-__device__ __forceinline__ void team_block_rows(const TeamCtx &tc, const __nv_bfloat16 *W, int row0, int n_rows,
-                                                int K, int m, const unsigned long long (&bptr)[NT],
-                                                const bool (&bok)[NT], float *out32, int ld_out) {
+template <int NT, typename Gate>
+__device__ __forceinline__ bool team_block_rows(TeamCtx &tc, const GroupDesc &grp, const __nv_bfloat16 *W, int row0,
+                                                int n_rows, int K, const unsigned long long (&bptr)[NT],
+                                                const bool (&bok)[NT], float *out32, int ld_out, Gate gate) {
     const int g = tc.lane >> 2, c = tc.lane & 3;
     float acc0[NT][4], acc1[NT][4];
 #pragma unroll
@@ -263,17 +373,28 @@ __device__ __forceinline__ void team_block_rows(const TeamCtx &tc, const __nv_bf
         for (int r = 0; r < 4; ++r) acc0[nn][r] = acc1[nn][r] = 0.f;
     const int r0 = row0 + tc.twarp * 16;
     const int rlo = r0 + g, rhi = r0 + g + 8;
-    const bool ok_lo = rlo < n_rows, ok_hi = rhi < n_rows;
-    warp_mma_range<NT, false, false, 4>(W, nullptr, K, ok_lo ? rlo : 0, ok_hi ? rhi : 0, ok_lo, ok_hi, 0, (K + 31) >> 5,
-                                        bptr, bok, acc0, acc1, tc.lane);
+    WRows w;
+    w.K = K;
+    w.ks0 = 0;
+    w.ks1 = (K + 31) >> 5;
+    w.ok_lo = rlo < n_rows;
+    w.ok_hi = rhi < n_rows;
+    w.p0lo = W + (size_t)(w.ok_lo ? rlo : 0) * K;
+    w.p0hi = W + (size_t)(w.ok_hi ? rhi : 0) * K;
+    w.p1lo = w.p1hi = nullptr;
+    bool failed = false;
+    warp_mma_range<NT, false, false, 2>(w, bptr, bok, acc0, acc1, tc.lane, [&]() { failed = !gate(); });
+    if (team_sync_or(tc.team, failed)) return false;
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             const int row = (r & 2) ? rhi : rlo;
             const int n = nn * 8 + 2 * c + (r & 1);
-            if (n < m && row < n_rows) out32[(size_t)tc.orow()[n] * ld_out + row] = acc0[nn][r];
+            if (n < grp.m && row < n_rows) out32[(size_t)out_row(tc, grp, false, n) * ld_out + row] = acc0[nn][r];
         }
+    tc.n_p2++;
+    return true;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -281,9 +402,13 @@ struct Smem {
     unsigned char *xs;   // [T][d*2 + XPAD] tokens, bf16
     int xstride;
     float *red[2];
-    int *tok[2];         // per team: tok[32], orow[32], flag[4]
+    int *flag[2];        // per team: 2 broadcast slots
+    GroupDesc *gtab[2];  // per team: copy of the group table
+    int *perm_h[2], *perm_l[2];
     // R2 scratch
     float *lg;           // [T][N]
+    float *s_conf;       // [T][N] or [T]
+    int *s_soe;          // [N]
     int *s_idx;          // [T*K]
     float *s_gate;       // [T*K]
     int *s_slot;         // [T*K]
@@ -307,8 +432,13 @@ __host__ __device__ inline size_t smem_layout(const Dims &dm, int nt, Smem *s, u
     const size_t xstride = (size_t)dm.d * 2 + XPAD;
     size_t o_xs = take((size_t)dm.T * xstride);
     size_t o_red0 = take((size_t)TW * 2 * nt * 128 * 4), o_red1 = take((size_t)TW * 2 * nt * 128 * 4);
-    size_t o_small = take(2 * (32 + 32 + 4) * 4);
+    size_t o_small = take(2 * 4 * 4);
+    const size_t ng = 1 + (size_t)dm.S + dm.N;
+    size_t o_gt0 = take(ng * sizeof(GroupDesc)), o_gt1 = take(ng * sizeof(GroupDesc));
+    size_t o_ph0 = take((size_t)n * 4), o_ph1 = take((size_t)n * 4), o_pl0 = take((size_t)n * 4), o_pl1 = take((size_t)n * 4);
     size_t o_lg = take((size_t)dm.T * dm.N * 4);
+    size_t o_conf = take((size_t)dm.T * dm.N * 4);
+    size_t o_soe = take((size_t)dm.N * 4);
     size_t o_idx = take((size_t)n * 4), o_gate = take((size_t)n * 4), o_slot = take((size_t)n * 4), o_cls = take(n);
     size_t o_hist = take(4 * 256 * 4);
     size_t o_wt = take((TW + 1 + 4) * 4);
@@ -318,8 +448,16 @@ __host__ __device__ inline size_t smem_layout(const Dims &dm, int nt, Smem *s, u
         s->red[0] = reinterpret_cast<float *>(base + o_red0);
         s->red[1] = reinterpret_cast<float *>(base + o_red1);
         int *sm = reinterpret_cast<int *>(base + o_small);
-        for (int t = 0; t < 2; ++t) s->tok[t] = sm + t * 68;
+        for (int t = 0; t < 2; ++t) s->flag[t] = sm + t * 4;
+        s->gtab[0] = reinterpret_cast<GroupDesc *>(base + o_gt0);
+        s->gtab[1] = reinterpret_cast<GroupDesc *>(base + o_gt1);
+        s->perm_h[0] = reinterpret_cast<int *>(base + o_ph0);
+        s->perm_h[1] = reinterpret_cast<int *>(base + o_ph1);
+        s->perm_l[0] = reinterpret_cast<int *>(base + o_pl0);
+        s->perm_l[1] = reinterpret_cast<int *>(base + o_pl1);
         s->lg = reinterpret_cast<float *>(base + o_lg);
+        s->s_conf = reinterpret_cast<float *>(base + o_conf);
+        s->s_soe = reinterpret_cast<int *>(base + o_soe);
         s->s_idx = reinterpret_cast<int *>(base + o_idx);
         s->s_gate = reinterpret_cast<float *>(base + o_gate);
         s->s_slot = reinterpret_cast<int *>(base + o_slot);
@@ -336,53 +474,39 @@ __host__ __device__ inline size_t smem_layout(const Dims &dm, int nt, Smem *s, u
 }
 
 // ------------------------------------------------------------------------------------------
-// R1: logits of experts [e0, e1) for all tokens; one warp per expert, router row kept in registers
-__device__ __noinline__ void task_r1(const DecodeParams &p, unsigned char *smem_raw, int nt, TeamCtx tc, int task) {
+// R1: logits of ONE expert for all tokens; the router row sits in registers, the warps share the
+// tokens.  Same arithmetic order as lane_dot_bf16 (see route_device.cuh).
+__device__ __noinline__ void task_r1(const DecodeParams &p, unsigned char *smem_raw, TeamCtx tc, int e) {
     const Dims &dm = p.dm;
-    Smem sm;
-    smem_layout(dm, nt, &sm, smem_raw);
-    const int per = (dm.N + p.n_r1 - 1) / p.n_r1;
-    const int e0 = task * per, e1 = min(dm.N, e0 + per);
-    const __nv_bfloat16 *wr = reinterpret_cast<const __nv_bfloat16 *>(p.w.w_router);
-    const int nsl = (dm.d + 255) >> 8;   // 8-element slices per lane
-    for (int e = e0 + tc.twarp; e < e1; e += TW) {
-        const __nv_bfloat16 *row = wr + (size_t)e * dm.d;
-        if (nsl <= 16) {
-            // keep this lane's slices of the router row in registers; same fmaf order as lane_dot_bf16
-            uint4 wreg[16];
+    const int xstride = dm.d * 2 + XPAD;
+    const __nv_bfloat16 *row = reinterpret_cast<const __nv_bfloat16 *>(p.w.w_router) + (size_t)e * dm.d;
+    if (dm.d <= 4096) {
+        uint4 wreg[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int k = i * 256 + tc.lane * 8;
+            wreg[i] = (k < dm.d) ? *reinterpret_cast<const uint4 *>(row + k) : make_uint4(0, 0, 0, 0);
+        }
+        for (int t = tc.twarp; t < dm.T; t += TW) {
+            const __nv_bfloat16 *x = reinterpret_cast<const __nv_bfloat16 *>(smem_raw + (size_t)t * xstride);
+            float s = 0.f;
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const int k = i * 256 + tc.lane * 8;
-                wreg[i] = (k < dm.d) ? *reinterpret_cast<const uint4 *>(row + k) : make_uint4(0, 0, 0, 0);
+                if (k < dm.d) s += slice_dot(wreg[i], *reinterpret_cast<const uint4 *>(x + k));
             }
-            for (int t = 0; t < dm.T; ++t) {
-                const __nv_bfloat16 *x = reinterpret_cast<const __nv_bfloat16 *>(sm.xs + (size_t)t * sm.xstride);
-                float s = 0.f;
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int k = i * 256 + tc.lane * 8;
-                    if (k < dm.d) {
-                        const uint4 u = wreg[i];
-                        const uint4 v = *reinterpret_cast<const uint4 *>(x + k);
-                        s = fmaf(bf_lo(u.x), bf_lo(v.x), s); s = fmaf(bf_hi(u.x), bf_hi(v.x), s);
-                        s = fmaf(bf_lo(u.y), bf_lo(v.y), s); s = fmaf(bf_hi(u.y), bf_hi(v.y), s);
-                        s = fmaf(bf_lo(u.z), bf_lo(v.z), s); s = fmaf(bf_hi(u.z), bf_hi(v.z), s);
-                        s = fmaf(bf_lo(u.w), bf_lo(v.w), s); s = fmaf(bf_hi(u.w), bf_hi(v.w), s);
-                    }
-                }
-                const float tot = warp_sum(s);
-                if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
-            }
-        } else {
-            for (int t = 0; t < dm.T; ++t) {
-                const float s = lane_dot_bf16(row, reinterpret_cast<const __nv_bfloat16 *>(sm.xs + (size_t)t * sm.xstride),
-                                              dm.d, tc.lane);
-                const float tot = warp_sum(s);
-                if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
-            }
+            const float tot = warp_sum(s);
+            if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
+        }
+    } else {
+        for (int t = tc.twarp; t < dm.T; t += TW) {
+            const float s = lane_dot_bf16(row, reinterpret_cast<const __nv_bfloat16 *>(smem_raw + (size_t)t * xstride),
+                                          dm.d, tc.lane);
+            const float tot = warp_sum(s);
+            if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
         }
     }
-    team_signal(tc, p.sync + SY_R1_DONE);
+    warp_signal(tc, p.sync + SY_R1_DONE);
 }
 
 // R2: top-k + gates, classification, residual list, grouping (one team)
@@ -391,11 +515,15 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
     Smem sm;
     smem_layout(dm, nt, &sm, smem_raw);
     const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
-    if (!team_wait_ge(tc, p.sync + SY_R1_DONE, p.n_r1, p)) return;
-    for (int i = tc.ttid; i < T * N; i += TEAM) sm.lg[i] = __ldcg(p.logits + i);
+    // while the logits are being produced: fetch what classification will need
+    for (int i = tc.ttid; i < N; i += TEAM) sm.s_soe[i] = p.w.slot_of_expert[i];
+    const int n_conf = p.conf_stride ? T * N : T;
+    for (int i = tc.ttid; i < n_conf; i += TEAM) sm.s_conf[i] = p.conf[i];
     if (tc.ttid < 4) sm.s_cnt[tc.ttid] = 0;
     sm.cnt_hit[tc.ttid] = 0;
     sm.cnt_low[tc.ttid] = 0;
+    if (!team_wait_ge(tc, p.sync + SY_R1_DONE, N * TW, p)) return;
+    for (int i = tc.ttid; i < T * N; i += TEAM) sm.lg[i] = __ldcg(p.logits + i);
     team_sync(tc.team);
     for (int t = tc.twarp; t < T; t += TW)
         warp_topk_gates(sm.lg + t * N, N, K, p.norm_topk, tc.lane, sm.s_idx + t * K, sm.s_gate + t * K, nullptr);
@@ -407,7 +535,7 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
         int c = -1, e = 0, sl = -1;
         if (i < n) {
             e = sm.s_idx[i];
-            sl = p.w.slot_of_expert[e];
+            sl = sm.s_soe[e];
             if (sl >= S) {
                 atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
                 sl = -1;
@@ -418,7 +546,7 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
             } else {
                 sl = -1;
                 const int t = i / K;
-                const float cf = p.conf_stride ? p.conf[(size_t)t * p.conf_stride + e] : p.conf[t];
+                const float cf = p.conf_stride ? sm.s_conf[t * N + e] : sm.s_conf[t];
                 c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
                 if (c == SPICE_LOWCONF) atomicAdd(&sm.cnt_low[e], 1);
             }
@@ -499,38 +627,68 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
             if (sm.s_cls[t * K + k] == SPICE_LOWCONF) c += sm.s_gate[t * K + k];
         p.tb.coef_shared[t] = c;
     }
-    team_signal(tc, p.sync + SY_ROUTE_DONE);
+    team_sync(tc.team);
+    if (tc.ttid == 0) {
+        __threadfence();
+        red_release_add(p.sync + SY_ROUTE_DONE, 1);
+    }
 }
 
-// fill the per-team token / output-row tables of a group and the per-lane B pointers
+// ------------------------------------------------------------------------------------------
+// Task list.  ids [0, nA) are known at launch; the rest once the router has published the groups.
+struct Plan {
+    int n_r1, nA;                       // phase A: R1 tasks, R2, shared gate/up tiles
+    int tIs, tI, tr, td, tb128, nb;     // tiles per matrix
+    int n_hg, n_lg, nB_hit, endB;       // phase B: hit gate/up tiles, LoRE A tiles
+    int nC_sh, nC_hit, endC, endD;      // phase C: down tiles; phase D: combine blocks
+    bool routed;                        // phases B..D resolvable
+};
+enum { TK_NONE = 0, TK_R1, TK_R2, TK_P1, TK_P2, TK_P3 };
+struct TaskRef {
+    int kind, gi, tile;
+};
+
+__device__ __forceinline__ TaskRef resolve(const Plan &pl, int id) {
+    if (id < pl.nA) {
+        if (id < pl.n_r1) return TaskRef{TK_R1, 0, id};
+        if (id == pl.n_r1) return TaskRef{TK_R2, 0, 0};
+        return TaskRef{TK_P1, 0, id - pl.n_r1 - 1};
+    }
+    if (!pl.routed || id >= pl.endD) return TaskRef{TK_NONE, 0, 0};
+    if (id < pl.endB) {
+        const int l = id - pl.nA;
+        if (l < pl.nB_hit) return TaskRef{TK_P1, 1 + l / pl.tI, l % pl.tI};
+        return TaskRef{TK_P1, 1 + pl.n_hg + (l - pl.nB_hit) / pl.tr, (l - pl.nB_hit) % pl.tr};
+    }
+    if (id < pl.endC) {
+        const int l = id - pl.endB;
+        if (l < pl.nC_sh) return TaskRef{TK_P2, 0, l};
+        if (l < pl.nC_sh + pl.nC_hit) return TaskRef{TK_P2, 1 + (l - pl.nC_sh) / pl.td, (l - pl.nC_sh) % pl.td};
+        const int q = l - pl.nC_sh - pl.nC_hit;
+        return TaskRef{TK_P2, 1 + pl.n_hg + q / pl.tb128, q % pl.tb128};
+    }
+    return TaskRef{TK_P3, 0, id - pl.endC};
+}
+
+__device__ __forceinline__ GroupDesc group_of(const DecodeParams &p, const TeamCtx &tc, int gi) {
+    if (gi == 0) return GroupDesc{KIND_SHARED, 0, 0, p.dm.T};
+    return tc.gtab[gi];
+}
+
+// per-lane B rows (token g of every n-tile) of a group
 template <int NT, bool B_SMEM>
 __device__ __forceinline__ void setup_rows(const DecodeParams &p, uint32_t xs_s, int xstride, const TeamCtx &tc,
-                                           const GroupDesc &grp, bool orow_is_pos, const unsigned char *b_base,
-                                           size_t b_row_bytes, unsigned long long (&bptr)[NT], bool (&bok)[NT]) {
-    // tok[n]: token of row n; orow[n]: output row of row n (position in the group's buffer, or entry id)
-    if (tc.ttid < 32) {
-        int tk = -1, orow = 0;
-        if (tc.ttid < grp.m) {
-            if (grp.kind == KIND_SHARED) {
-                tk = tc.ttid;
-                orow = tc.ttid;
-            } else {
-                const int entry = __ldcg((grp.kind == KIND_HIT ? p.tb.perm_hit : p.tb.perm_low) + grp.off + tc.ttid);
-                tk = entry / p.dm.K;
-                orow = orow_is_pos ? grp.off + tc.ttid : entry;
-            }
-        }
-        tc.tok[tc.ttid] = tk;
-        tc.orow()[tc.ttid] = orow;
-    }
-    team_sync(tc.team);
+                                           const GroupDesc &grp, const unsigned char *b_base, size_t b_row_bytes,
+                                           unsigned long long (&bptr)[NT], bool (&bok)[NT]) {
     const int g = tc.lane >> 2;
 #pragma unroll
     for (int nn = 0; nn < NT; ++nn) {
         const int n = nn * 8 + g;
         bok[nn] = n < grp.m;
         if (B_SMEM) {
-            const int tk = bok[nn] ? tc.tok[n] : 0;
+            int tk = 0;
+            if (bok[nn])
+                tk = (grp.kind == KIND_SHARED) ? n : (grp.kind == KIND_HIT ? tc.perm_h : tc.perm_l)[grp.off + n] / p.dm.K;
             bptr[nn] = (unsigned long long)(xs_s + (uint32_t)(tk * xstride));
         } else {
             bptr[nn] = (unsigned long long)(b_base + (size_t)(bok[nn] ? n : 0) * b_row_bytes);
@@ -538,57 +696,66 @@ __device__ __forceinline__ void setup_rows(const DecodeParams &p, uint32_t xs_s,
     }
 }
 
+struct NoGate {
+    __device__ __forceinline__ bool operator()() const { return true; }
+};
+
 // P1 task: gate/up + SwiGLU rows of the shared expert or of a hit slot, or LoRE A rows
 template <int NT>
-__device__ __forceinline__ void task_p1(const DecodeParams &p, uint32_t xs_s, int xstride, const TeamCtx &tc, int gi, int tile) {
+__device__ __forceinline__ bool task_p1(const DecodeParams &p, uint32_t xs_s, int xstride, TeamCtx &tc, int gi,
+                                        int tile) {
     const Dims &dm = p.dm;
-    const GroupDesc grp = (gi == 0) ? GroupDesc{KIND_SHARED, 0, 0, dm.T} : load_group(p.tb.groups + gi);
+    const GroupDesc grp = group_of(p, tc, gi);
     unsigned long long bptr[NT];
     bool bok[NT];
-    setup_rows<NT, true>(p, xs_s, xstride, tc, grp, true, nullptr, 0, bptr, bok);
+    setup_rows<NT, true>(p, xs_s, xstride, tc, grp, nullptr, 0, bptr, bok);
     if (grp.kind == KIND_LOW) {
         const __nv_bfloat16 *A = reinterpret_cast<const __nv_bfloat16 *>(p.w.lore_A) + (size_t)grp.id * dm.r * dm.d;
-        team_tile_ksplit<NT, EPI_Z, true>(tc, A, nullptr, tile * 16, dm.r, dm.d, grp.m, bptr, bok, p.z16, nullptr, dm.r);
+        return team_tile_ksplit<NT, EPI_Z, true>(tc, grp, A, nullptr, tile * 16, dm.r, dm.d, bptr, bok, p.z16, nullptr,
+                                                 dm.r, NoGate());
     } else if (grp.kind == KIND_HIT) {
         const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.slot_w_gate_up) + (size_t)grp.id * 2 * dm.I * dm.d;
-        team_tile_ksplit<NT, EPI_ACT, true>(tc, W, W + (size_t)dm.I * dm.d, tile * 16, dm.I, dm.d, grp.m, bptr, bok,
-                                            p.act_hit16, nullptr, dm.I);
-    } else {
-        const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_gate_up);
-        team_tile_ksplit<NT, EPI_ACT, true>(tc, W, W + (size_t)dm.Is * dm.d, tile * 16, dm.Is, dm.d, grp.m, bptr, bok,
-                                            p.act_shared16, nullptr, dm.Is);
+        return team_tile_ksplit<NT, EPI_ACT, true>(tc, grp, W, W + (size_t)dm.I * dm.d, tile * 16, dm.I, dm.d, bptr, bok,
+                                                   p.act_hit16, nullptr, dm.I, NoGate());
     }
-    team_signal(tc, p.sync + SY_GROUP0 + gi);
+    const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_gate_up);
+    return team_tile_ksplit<NT, EPI_ACT, true>(tc, grp, W, W + (size_t)dm.Is * dm.d, tile * 16, dm.Is, dm.d, bptr, bok,
+                                               p.act_shared16, nullptr, dm.Is, NoGate());
 }
 
-// P2 task: down-projection rows of one group
+// P2 task: down-projection rows of one group.  The first P2 tile of a warp publishes the warp's P1
+// count and waits (after its first weight loads are in flight) until every P1 tile of the layer is
+// published; later tiles do not wait.
 template <int NT>
-__device__ __forceinline__ bool task_p2(const DecodeParams &p, const TeamCtx &tc, int gi, int tile, int need) {
+__device__ __forceinline__ bool task_p2(const DecodeParams &p, TeamCtx &tc, int gi, int tile, int p1_total) {
     const Dims &dm = p.dm;
-    if (!team_wait_ge(tc, p.sync + SY_GROUP0 + gi, need, p)) return false;
-    const GroupDesc grp = (gi == 0) ? GroupDesc{KIND_SHARED, 0, 0, dm.T} : load_group(p.tb.groups + gi);
+    const GroupDesc grp = group_of(p, tc, gi);
     unsigned long long bptr[NT];
     bool bok[NT];
+    auto gate = [&]() {
+        if (tc.p1_all) return true;
+        flush_counts(tc, p.sync);
+        tc.p1_all = warp_wait_ge(tc, p.sync + SY_P1_ALL, p1_total, p);
+        return tc.p1_all;
+    };
     if (grp.kind == KIND_SHARED) {
-        setup_rows<NT, false>(p, 0u, 0, tc, grp, false, reinterpret_cast<const unsigned char *>(p.act_shared16), (size_t)dm.Is * 2,
-                              bptr, bok);
-        team_tile_ksplit<NT, EPI_PART, false>(tc, reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_down), nullptr,
-                                              tile * 16, dm.d, dm.Is, grp.m, bptr, bok, nullptr, p.tb.part_shared, dm.d);
+        setup_rows<NT, false>(p, 0u, 0, tc, grp, reinterpret_cast<const unsigned char *>(p.act_shared16),
+                              (size_t)dm.Is * 2, bptr, bok);
+        return team_tile_ksplit<NT, EPI_PART, false>(tc, grp, reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_down),
+                                                     nullptr, tile * 16, dm.d, dm.Is, bptr, bok, nullptr,
+                                                     p.tb.part_shared, dm.d, gate);
     } else if (grp.kind == KIND_HIT) {
-        setup_rows<NT, false>(p, 0u, 0, tc, grp, false,
+        setup_rows<NT, false>(p, 0u, 0, tc, grp,
                               reinterpret_cast<const unsigned char *>(p.act_hit16 + (size_t)grp.off * dm.I),
                               (size_t)dm.I * 2, bptr, bok);
         const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.slot_w_down) + (size_t)grp.id * dm.d * dm.I;
-        team_tile_ksplit<NT, EPI_PART, false>(tc, W, nullptr, tile * 16, dm.d, dm.I, grp.m, bptr, bok, nullptr, p.tb.part,
-                                              dm.d);
-    } else {
-        setup_rows<NT, false>(p, 0u, 0, tc, grp, false, reinterpret_cast<const unsigned char *>(p.z16 + (size_t)grp.off * dm.r),
-                              (size_t)dm.r * 2, bptr, bok);
-        const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.lore_B) + (size_t)grp.id * dm.d * dm.r;
-        team_block_rows<NT>(tc, W, tile * 128, dm.d, dm.r, grp.m, bptr, bok, p.tb.part, dm.d);
+        return team_tile_ksplit<NT, EPI_PART, false>(tc, grp, W, nullptr, tile * 16, dm.d, dm.I, bptr, bok, nullptr,
+                                                     p.tb.part, dm.d, gate);
     }
-    team_signal(tc, p.sync + SY_P2_DONE);
-    return true;
+    setup_rows<NT, false>(p, 0u, 0, tc, grp, reinterpret_cast<const unsigned char *>(p.z16 + (size_t)grp.off * dm.r),
+                          (size_t)dm.r * 2, bptr, bok);
+    const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.lore_B) + (size_t)grp.id * dm.d * dm.r;
+    return team_block_rows<NT>(tc, grp, W, tile * 128, dm.d, dm.r, bptr, bok, p.tb.part, dm.d, gate);
 }
 
 // P3 task: 1024 columns of one token
@@ -633,77 +800,124 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
     tc.ttid = threadIdx.x & (TEAM - 1);
     tc.twarp = tc.ttid >> 5;
     tc.lane = threadIdx.x & 31;
+    tc.n_p1 = tc.n_p2 = 0;
+    tc.p1_all = false;
+#ifdef SPICE_PROF
+    tc.gteam = blockIdx.x * 2 + tc.team;
+    tc.nprof = 0;
+#endif
+    PROF(tc, 1);
     {
         Smem sm;
         smem_layout(dm, NT, &sm, smem_raw);
         tc.red = sm.red[tc.team];
-        tc.tok = sm.tok[tc.team];
+        tc.flag = sm.flag[tc.team];
+        tc.gtab = sm.gtab[tc.team];
+        tc.perm_h = sm.perm_h[tc.team];
+        tc.perm_l = sm.perm_l[tc.team];
     }
     const int xstride = dm.d * 2 + XPAD;
     const uint32_t xs_s = (uint32_t)__cvta_generic_to_shared(smem_raw);   // the token tile sits first
 
-    // tokens -> shared memory (bf16, padded rows)
-    const int vec = dm.d >> 3;
-    for (int v = threadIdx.x; v < dm.T * vec; v += DT) {
-        const int t = v / vec, cidx = v - t * vec;
-        *reinterpret_cast<uint4 *>(smem_raw + (size_t)t * xstride + cidx * 16) =
-            *reinterpret_cast<const uint4 *>(p.h + (size_t)t * dm.d + cidx * 8);
-    }
-    __syncthreads();
+    Plan pl;
+    pl.n_r1 = p.n_r1;
+    pl.tIs = (dm.Is + 15) >> 4;
+    pl.tI = (dm.I + 15) >> 4;
+    pl.tr = (dm.r + 15) >> 4;
+    pl.td = (dm.d + 15) >> 4;
+    pl.tb128 = (dm.d + 127) >> 7;
+    pl.nb = (dm.d + 1023) >> 10;
+    pl.nA = p.n_r1 + 1 + pl.tIs;
+    pl.routed = false;
+    pl.n_hg = pl.n_lg = pl.nB_hit = pl.endB = pl.nC_sh = pl.nC_hit = pl.endC = pl.endD = 0;
 
     const int n_teams = gridDim.x * 2;
-    const int me = blockIdx.x * 2 + tc.team;
-    const int tIs = (dm.Is + 15) >> 4, tI = (dm.I + 15) >> 4, tr = (dm.r + 15) >> 4, td = (dm.d + 15) >> 4;
-    const int tb128 = (dm.d + 127) >> 7;
-    const int nA = p.n_r1 + 1 + tIs;
-    int id = me;
-    for (; id < nA; id += n_teams) {
-        if (id < p.n_r1) task_r1(p, smem_raw, NT, tc, id);
-        else if (id == p.n_r1) task_r2(p, smem_raw, NT, tc);
-        else task_p1<NT>(p, xs_s, xstride, tc, 0, id - p.n_r1 - 1);
-    }
-    // every quantity below is uniform across the team (it comes from broadcast wait results)
-    bool alive = team_wait_ge(tc, p.sync + SY_ROUTE_DONE, 1, p);
-    if (alive) {
-        const int n_hg = __ldcg(p.tb.hdr + HDR_N_HIT_GROUPS), n_lg = __ldcg(p.tb.hdr + HDR_N_LOW_GROUPS);
-        const int nB_hit = n_hg * tI, nB = nB_hit + n_lg * tr;
-        const int nC_sh = td, nC_hit = n_hg * td, nC = nC_sh + nC_hit + n_lg * tb128;
-        const int nb = (dm.d + 1023) >> 10;
-        const int nD = dm.T * nb;
-        const int endB = nA + nB, endC = endB + nC, endD = endC + nD;
-        bool p2_ready = false;
-        for (; id < endD && alive; id += n_teams) {
-            if (id < endB) {
-                const int l = id - nA;
-                if (l < nB_hit) task_p1<NT>(p, xs_s, xstride, tc, 1 + l / tI, l % tI);
-                else task_p1<NT>(p, xs_s, xstride, tc, 1 + n_hg + (l - nB_hit) / tr, (l - nB_hit) % tr);
-            } else if (id < endC) {
-                const int l = id - endB;
-                if (l < nC_sh) alive = task_p2<NT>(p, tc, 0, l, tIs);
-                else if (l < nC_sh + nC_hit) alive = task_p2<NT>(p, tc, 1 + (l - nC_sh) / td, (l - nC_sh) % td, tI);
-                else {
-                    const int q = l - nC_sh - nC_hit;
-                    alive = task_p2<NT>(p, tc, 1 + n_hg + q / tb128, q % tb128, tr);
+    int id = blockIdx.x * 2 + tc.team;
+
+    // tokens -> shared memory (bf16, padded rows); 8 loads in flight per thread
+    {
+        const int vec = dm.d >> 3, total = dm.T * vec;
+        for (int v0 = threadIdx.x; v0 < total; v0 += DT * 8) {
+            uint4 tmp[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int v = v0 + i * DT;
+                if (v < total) {
+                    const int t = v / vec, cidx = v - t * vec;
+                    tmp[i] = __ldg(reinterpret_cast<const uint4 *>(p.h + (size_t)t * dm.d + cidx * 8));
                 }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int v = v0 + i * DT;
+                if (v < total) {
+                    const int t = v / vec, cidx = v - t * vec;
+                    *reinterpret_cast<uint4 *>(smem_raw + (size_t)t * xstride + cidx * 16) = tmp[i];
+                }
+            }
+        }
+    }
+    __syncthreads();
+    PROF(tc, 2);
+
+    bool alive = true;
+    for (; id < pl.nA && alive; id += n_teams) {
+        PROF(tc, 100 + resolve(pl, id).kind);
+        if (id < p.n_r1) task_r1(p, smem_raw, tc, id);
+        else if (id == p.n_r1) task_r2(p, smem_raw, NT, tc);
+        else alive = task_p1<NT>(p, xs_s, xstride, tc, 0, id - p.n_r1 - 1);
+    }
+    // every quantity below is uniform across the team (it comes from team-wide reductions)
+    PROF(tc, 30);
+    alive = alive && team_wait_ge(tc, p.sync + SY_ROUTE_DONE, 1, p);
+    PROF(tc, 31);
+    if (alive) {
+        // team-private copy of the group table and the permutations: task set-up never goes to L2 again
+        pl.n_hg = __ldcg(p.tb.hdr + HDR_N_HIT_GROUPS);
+        pl.n_lg = __ldcg(p.tb.hdr + HDR_N_LOW_GROUPS);
+        const int n_hit = __ldcg(p.tb.hdr + HDR_N_HIT), n_low = __ldcg(p.tb.hdr + HDR_N_LOW);
+        for (int i = tc.ttid; i < 1 + pl.n_hg + pl.n_lg; i += TEAM) tc.gtab[i] = load_group(p.tb.groups + i);
+        for (int i = tc.ttid; i < n_hit; i += TEAM) tc.perm_h[i] = __ldcg(p.tb.perm_hit + i);
+        for (int i = tc.ttid; i < n_low; i += TEAM) tc.perm_l[i] = __ldcg(p.tb.perm_low + i);
+        pl.nB_hit = pl.n_hg * pl.tI;
+        pl.endB = pl.nA + pl.nB_hit + pl.n_lg * pl.tr;
+        pl.nC_sh = pl.td;
+        pl.nC_hit = pl.n_hg * pl.td;
+        const int nC = pl.nC_sh + pl.nC_hit + pl.n_lg * pl.tb128;
+        pl.endC = pl.endB + nC;
+        pl.endD = pl.endC + dm.T * pl.nb;
+        pl.routed = true;
+        const int p1_total = (pl.tIs + pl.nB_hit + pl.n_lg * pl.tr) * TW;
+        team_sync(tc.team);
+        bool p2_ready = false;
+        for (; id < pl.endD && alive; id += n_teams) {
+            const TaskRef t = resolve(pl, id);
+            PROF(tc, 100 + t.kind);
+                PROF(tc, 10);
+            if (t.kind == TK_P1) {
+                alive = task_p1<NT>(p, xs_s, xstride, tc, t.gi, t.tile);
+            } else if (t.kind == TK_P2) {
+                alive = task_p2<NT>(p, tc, t.gi, t.tile, p1_total);
             } else {
-                if (!p2_ready) {   // combine needs every down-projected row
-                    alive = team_wait_ge(tc, p.sync + SY_P2_DONE, nC, p);
+                if (!p2_ready) {   // combine needs every down-projected row (counted per warp)
+                    alive = team_wait_ge(tc, p.sync + SY_P2_DONE, nC * TW, p);
                     if (!alive) break;
                     p2_ready = true;
                 }
-                const int l = id - endC;
-                task_p3(p, tc.ttid, l / nb, l % nb);
+                task_p3(p, tc.ttid, t.tile / pl.nb, t.tile % pl.nb);
             }
         }
     }
     // the last team to finish clears the counters for the next launch
+    PROF(tc, 40);
+    flush_counts(tc, p.sync);
     team_sync(tc.team);
     if (tc.ttid == 0) {
         __threadfence();
-        *tc.flag() = atomicAdd(p.sync + SY_TEAMS_DONE, 1);
+        tc.flag[1] = atomicAdd(p.sync + SY_TEAMS_DONE, 1);
     }
     team_sync(tc.team);
-    if (*tc.flag() == n_teams - 1) {
+    if (tc.flag[1] == n_teams - 1) {
         __threadfence();
         for (int i = tc.ttid; i < p.sync_words; i += TEAM) p.sync[i] = 0;
     }
@@ -746,5 +960,19 @@ int launch_decode(const DecodeParams &p, int n_ctas, cudaStream_t st) {
     }
     return 1;
 }
+
+#ifdef SPICE_PROF
+extern "C" int spice_debug_prof_read(unsigned long long *host, size_t n_words) {
+    size_t total = sizeof(unsigned long long) * (size_t)PROF_TEAMS * PROF_EVENTS * 2;
+    if (n_words * 8 < total) return -1;
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(host, g_prof, total) == cudaSuccess ? 0 : -2;
+}
+extern "C" int spice_debug_prof_clear(void) {
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_prof) != cudaSuccess) return -1;
+    return cudaMemset(ptr, 0, sizeof(unsigned long long) * (size_t)PROF_TEAMS * PROF_EVENTS * 2) == cudaSuccess ? 0 : -2;
+}
+#endif
 
 }  // namespace spice

@@ -34,18 +34,11 @@ __global__ void route_topk_kernel(const __nv_bfloat16 *__restrict__ h, const __n
         for (int tt = 0; tt < TPC; ++tt) acc[tt] = 0.f;
         const __nv_bfloat16 *row = wr + (size_t)e * d;
         for (int k = lane * 8; k < d; k += 256) {
-            uint4 u = *reinterpret_cast<const uint4 *>(row + k);
-            float w0 = bf_lo(u.x), w1 = bf_hi(u.x), w2 = bf_lo(u.y), w3 = bf_hi(u.y);
-            float w4 = bf_lo(u.z), w5 = bf_hi(u.z), w6 = bf_lo(u.w), w7 = bf_hi(u.w);
+            const uint4 u = *reinterpret_cast<const uint4 *>(row + k);
 #pragma unroll
-            for (int tt = 0; tt < TPC; ++tt) {
-                const float4 a = *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k);
-                const float4 b = *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k + 4);
-                float s = acc[tt];
-                s = fmaf(w0, a.x, s); s = fmaf(w1, a.y, s); s = fmaf(w2, a.z, s); s = fmaf(w3, a.w, s);
-                s = fmaf(w4, b.x, s); s = fmaf(w5, b.y, s); s = fmaf(w6, b.z, s); s = fmaf(w7, b.w, s);
-                acc[tt] = s;
-            }
+            for (int tt = 0; tt < TPC; ++tt)
+                acc[tt] += slice_dot(u, *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k),
+                                     *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k + 4));
         }
 #pragma unroll
         for (int tt = 0; tt < TPC; ++tt) {

@@ -1,39 +1,46 @@
 // Device routines shared by the stand-alone router kernel and the fused decode kernel, so that
 // both produce bit-identical logits, selections and gates (Eq. 1 of the paper; gate scores of
-// Sec. 4.2).  The arithmetic order is fixed: each lane accumulates its 8-element slices of the
-// row in increasing k with fmaf, then the 32 lane sums are combined by an xor-shuffle tree.
+// Sec. 4.2).  The arithmetic order is fixed: each lane reduces every 8-element slice it owns with
+// an fmaf chain from zero, adds the slice sums in increasing k, then the 32 lane sums are
+// combined by an xor-shuffle tree.
 #pragma once
 #include "spice_internal.cuh"
 
 namespace spice {
 
-// acc += sum over this lane's slices of w_row[k] * x[k];  x is an fp32 row in shared memory
+// 8 products of one 128-bit slice, accumulated in index order starting from zero
+__device__ __forceinline__ float slice_dot(const uint4 u, const float4 a, const float4 b) {
+    float q = 0.f;
+    q = fmaf(bf_lo(u.x), a.x, q); q = fmaf(bf_hi(u.x), a.y, q);
+    q = fmaf(bf_lo(u.y), a.z, q); q = fmaf(bf_hi(u.y), a.w, q);
+    q = fmaf(bf_lo(u.z), b.x, q); q = fmaf(bf_hi(u.z), b.y, q);
+    q = fmaf(bf_lo(u.w), b.z, q); q = fmaf(bf_hi(u.w), b.w, q);
+    return q;
+}
+__device__ __forceinline__ float slice_dot(const uint4 u, const uint4 v) {
+    return slice_dot(u, make_float4(bf_lo(v.x), bf_hi(v.x), bf_lo(v.y), bf_hi(v.y)),
+                     make_float4(bf_lo(v.z), bf_hi(v.z), bf_lo(v.w), bf_hi(v.w)));
+}
+
+// This lane's share of dot(w_row, x): slices k = lane*8 + 256*i, each reduced by slice_dot, the
+// slice sums added in increasing i.  x is an fp32 row in shared memory.
 __device__ __forceinline__ float lane_dot_f32(const __nv_bfloat16 *__restrict__ w_row, const float *x, int d, int lane) {
     float s = 0.f;
     for (int k = lane * 8; k < d; k += 256) {
         const uint4 u = *reinterpret_cast<const uint4 *>(w_row + k);
-        const float4 a = *reinterpret_cast<const float4 *>(x + k);
-        const float4 b = *reinterpret_cast<const float4 *>(x + k + 4);
-        s = fmaf(bf_lo(u.x), a.x, s); s = fmaf(bf_hi(u.x), a.y, s);
-        s = fmaf(bf_lo(u.y), a.z, s); s = fmaf(bf_hi(u.y), a.w, s);
-        s = fmaf(bf_lo(u.z), b.x, s); s = fmaf(bf_hi(u.z), b.y, s);
-        s = fmaf(bf_lo(u.w), b.z, s); s = fmaf(bf_hi(u.w), b.w, s);
+        s += slice_dot(u, *reinterpret_cast<const float4 *>(x + k), *reinterpret_cast<const float4 *>(x + k + 4));
     }
     return s;
 }
 
-// same sum with the activation row held as bf16 in shared memory (values are identical after
-// the exact bf16 -> fp32 widening, so the result equals lane_dot_f32 bit for bit)
+// same sum with the activation row held as bf16 (the bf16 -> fp32 widening is exact, so the
+// result equals lane_dot_f32 bit for bit)
 __device__ __forceinline__ float lane_dot_bf16(const __nv_bfloat16 *__restrict__ w_row, const __nv_bfloat16 *x, int d,
                                                int lane) {
     float s = 0.f;
     for (int k = lane * 8; k < d; k += 256) {
         const uint4 u = *reinterpret_cast<const uint4 *>(w_row + k);
-        const uint4 v = *reinterpret_cast<const uint4 *>(x + k);
-        s = fmaf(bf_lo(u.x), bf_lo(v.x), s); s = fmaf(bf_hi(u.x), bf_hi(v.x), s);
-        s = fmaf(bf_lo(u.y), bf_lo(v.y), s); s = fmaf(bf_hi(u.y), bf_hi(v.y), s);
-        s = fmaf(bf_lo(u.z), bf_lo(v.z), s); s = fmaf(bf_hi(u.z), bf_hi(v.z), s);
-        s = fmaf(bf_lo(u.w), bf_lo(v.w), s); s = fmaf(bf_hi(u.w), bf_hi(v.w), s);
+        s += slice_dot(u, *reinterpret_cast<const uint4 *>(x + k));
     }
     return s;
 }
