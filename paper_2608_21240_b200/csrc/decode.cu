@@ -34,6 +34,10 @@ namespace spice {
 
 namespace {
 
+#ifndef SPICE_RUN_INLINE
+#define SPICE_RUN_INLINE __forceinline__
+#endif
+
 constexpr int DT = 512;     // threads per CTA
 constexpr int TEAM = 256;   // threads per team
 constexpr int TW = 8;       // warps per team
@@ -106,6 +110,11 @@ __device__ __forceinline__ unsigned long long prof_now() {
     do {              \
     } while (0)
 #endif
+#ifdef SPICE_PROF
+#define TC_ARG TeamCtx &
+#else
+#define TC_ARG TeamCtx
+#endif
 
 struct TeamCtx {
 #ifdef SPICE_PROF
@@ -170,31 +179,6 @@ __device__ __forceinline__ bool team_wait_ge(TeamCtx &tc, const int *ctr, int ta
     return ok;
 }
 
-// exclusive scan over the 256 threads of a team
-__device__ __forceinline__ int team_excl_scan(const TeamCtx &tc, int v, int *wt /* [TW+1] */, int &total) {
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, inc, o);
-        if (tc.lane >= o) inc += n;
-    }
-    team_sync(tc.team);
-    if (tc.lane == 31) wt[tc.twarp] = inc;
-    team_sync(tc.team);
-    if (tc.ttid == 0) {
-        int run = 0;
-        for (int w = 0; w < TW; ++w) {
-            int x = wt[w];
-            wt[w] = run;
-            run += x;
-        }
-        wt[TW] = run;
-    }
-    team_sync(tc.team);
-    total = wt[TW];
-    return wt[tc.twarp] + inc - v;
-}
-
 __device__ __forceinline__ GroupDesc load_group(const GroupDesc *g) {
     const int4 v = __ldcg(reinterpret_cast<const int4 *>(g));
     return GroupDesc{v.x, v.y, v.z, v.w};
@@ -207,7 +191,8 @@ struct WRows {
     const __nv_bfloat16 *p1lo, *p1hi;   // same rows of the second matrix (gate/up pair) or unused
     int K;                              // reduction length
     int ks0, ks1;                       // this warp's k-steps
-    bool ok_lo, ok_hi;
+    bool ok_lo, ok_hi;                  // rows g / g+8 of the first matrix exist
+    bool ok1_lo, ok1_hi;                // same for the second matrix
 };
 
 // One warp: C[16 x 8*NT] += W[rows g, g+8][k] * X[token][k] over this warp's k-steps.
@@ -233,8 +218,8 @@ __device__ __forceinline__ void warp_mma_range(const WRows &w, const unsigned lo
             a0lo[u] = (in && w.ok_lo) ? ldg_stream(w.p0lo + kb) : zero;
             a0hi[u] = (in && w.ok_hi) ? ldg_stream(w.p0hi + kb) : zero;
             if (DUAL) {
-                a1lo[u] = (in && w.ok_lo) ? ldg_stream(w.p1lo + kb) : zero;
-                a1hi[u] = (in && w.ok_hi) ? ldg_stream(w.p1hi + kb) : zero;
+                a1lo[u] = (in && w.ok1_lo) ? ldg_stream(w.p1lo + kb) : zero;
+                a1hi[u] = (in && w.ok1_hi) ? ldg_stream(w.p1hi + kb) : zero;
             }
         }
         if (first) {
@@ -275,7 +260,7 @@ __device__ __forceinline__ void warp_mma_range(const WRows &w, const unsigned lo
     }
 }
 
-enum { EPI_ACT = 0, EPI_Z = 1, EPI_PART = 2 };
+enum { EPI_ACT = 0, EPI_Z = 1, EPI_PART = 2, EPI_PART2 = 3 };
 
 // where row n of a group lands: the token (shared expert), the position in the group's buffer
 // (P1 of a hit / low group) or the entry id t*K+k (P2 of a hit / low group)
@@ -283,80 +268,6 @@ __device__ __forceinline__ int out_row(const TeamCtx &tc, const GroupDesc &grp, 
     if (grp.kind == KIND_SHARED) return n;
     if (by_pos) return grp.off + n;
     return (grp.kind == KIND_HIT ? tc.perm_h : tc.perm_l)[grp.off + n];
-}
-
-// One team, one 16-row tile, reduction split over the 8 warps.  Returns false (team-uniform) when
-// some warp's wait failed; nothing is stored then.
-//   EPI_ACT : rows of W0 = gate, W1 = up; out16[orow*ld_out + row] = silu(g)*u          (P1 shared/hit)
-//   EPI_Z   : out16[orow*ld_out + row] = sum                                            (P1 LoRE A)
-//   EPI_PART: out32[orow*ld_out + row] = sum                                            (P2 down)
-template <int NT, int EPI, bool B_SMEM, typename Gate>
-__device__ __forceinline__ bool team_tile_ksplit(TeamCtx &tc, const GroupDesc &grp, const __nv_bfloat16 *W0,
-                                                 const __nv_bfloat16 *W1, int row0, int n_rows, int K,
-                                                 const unsigned long long (&bptr)[NT], const bool (&bok)[NT],
-                                                 __nv_bfloat16 *out16, float *out32, int ld_out, Gate gate) {
-    constexpr bool DUAL = (EPI == EPI_ACT);
-    constexpr int MATS = DUAL ? 2 : 1;
-#ifdef SPICE_U
-    constexpr int U = SPICE_U;
-#else
-    constexpr int U = (NT == 4) ? 2 : 4;
-#endif
-    const int g = tc.lane >> 2;
-    const int KS = (K + 31) >> 5;
-    const int base = KS / TW, rem = KS % TW;
-    WRows w;
-    w.K = K;
-    w.ks0 = tc.twarp * base + min(tc.twarp, rem);
-    w.ks1 = w.ks0 + base + (tc.twarp < rem ? 1 : 0);
-    const int rlo = row0 + g, rhi = row0 + g + 8;
-    w.ok_lo = rlo < n_rows;
-    w.ok_hi = rhi < n_rows;
-    w.p0lo = W0 + (size_t)(w.ok_lo ? rlo : 0) * K;
-    w.p0hi = W0 + (size_t)(w.ok_hi ? rhi : 0) * K;
-    w.p1lo = DUAL ? W1 + (size_t)(w.ok_lo ? rlo : 0) * K : nullptr;
-    w.p1hi = DUAL ? W1 + (size_t)(w.ok_hi ? rhi : 0) * K : nullptr;
-    float acc0[NT][4], acc1[NT][4];
-#pragma unroll
-    for (int nn = 0; nn < NT; ++nn)
-#pragma unroll
-        for (int r = 0; r < 4; ++r) acc0[nn][r] = acc1[nn][r] = 0.f;
-    bool failed = false;
-    warp_mma_range<NT, DUAL, B_SMEM, U>(w, bptr, bok, acc0, acc1, tc.lane, [&]() { failed = !gate(); });
-    PROF(tc, 20);
-    // every warp is past the previous tile's epilogue once it arrives here
-    if (team_sync_or(tc.team, failed)) return false;
-    float *red = tc.red;
-#pragma unroll
-    for (int nn = 0; nn < NT; ++nn)
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            red[((tc.twarp * MATS + 0) * NT + nn) * 128 + r * 32 + tc.lane] = acc0[nn][r];
-            if (DUAL) red[((tc.twarp * MATS + 1) * NT + nn) * 128 + r * 32 + tc.lane] = acc1[nn][r];
-        }
-    team_sync(tc.team);
-    PROF(tc, 21);
-    for (int e = tc.ttid; e < NT * 128; e += TEAM) {
-        const int nn = e >> 7, r = (e >> 5) & 3, ln = e & 31;
-        const int row = row0 + (ln >> 2) + ((r & 2) ? 8 : 0);
-        const int n = nn * 8 + 2 * (ln & 3) + (r & 1);
-        float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-        for (int wi = 0; wi < TW; ++wi) {
-            s0 += red[((wi * MATS + 0) * NT + nn) * 128 + r * 32 + ln];
-            if (DUAL) s1 += red[((wi * MATS + 1) * NT + nn) * 128 + r * 32 + ln];
-        }
-        if (n < grp.m && row < n_rows) {
-            const size_t o = (size_t)out_row(tc, grp, EPI != EPI_PART, n) * ld_out + row;
-            if (EPI == EPI_ACT) out16[o] = __float2bfloat16(silu_f(s0) * s1);
-            else if (EPI == EPI_Z) out16[o] = __float2bfloat16(s0);
-            else out32[o] = s0;
-        }
-    }
-    PROF(tc, 22);
-    if (EPI == EPI_PART) tc.n_p2++;
-    else tc.n_p1++;
-    return true;
 }
 
 // P2 of a LoRE group: part[entry, j] = sum_q B_e[j,q] z[q]; the reduction (r) is short, so each warp
@@ -382,6 +293,7 @@ __device__ __forceinline__ bool team_block_rows(TeamCtx &tc, const GroupDesc &gr
     w.p0lo = W + (size_t)(w.ok_lo ? rlo : 0) * K;
     w.p0hi = W + (size_t)(w.ok_hi ? rhi : 0) * K;
     w.p1lo = w.p1hi = nullptr;
+    w.ok1_lo = w.ok1_hi = false;
     bool failed = false;
     warp_mma_range<NT, false, false, 2>(w, bptr, bok, acc0, acc1, tc.lane, [&]() { failed = !gate(); });
     if (team_sync_or(tc.team, failed)) return false;
@@ -476,131 +388,176 @@ __host__ __device__ inline size_t smem_layout(const Dims &dm, int nt, Smem *s, u
 // ------------------------------------------------------------------------------------------
 // R1: logits of ONE expert for all tokens; the router row sits in registers, the warps share the
 // tokens.  Same arithmetic order as lane_dot_bf16 (see route_device.cuh).
-__device__ __noinline__ void task_r1(const DecodeParams &p, unsigned char *smem_raw, TeamCtx tc, int e) {
+__device__ __noinline__ void task_r1(const DecodeParams &p, unsigned char *smem_raw, TC_ARG tc, int e) {
     const Dims &dm = p.dm;
     const int xstride = dm.d * 2 + XPAD;
     const __nv_bfloat16 *row = reinterpret_cast<const __nv_bfloat16 *>(p.w.w_router) + (size_t)e * dm.d;
-    if (dm.d <= 4096) {
-        uint4 wreg[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const int k = i * 256 + tc.lane * 8;
-            wreg[i] = (k < dm.d) ? *reinterpret_cast<const uint4 *>(row + k) : make_uint4(0, 0, 0, 0);
-        }
-        for (int t = tc.twarp; t < dm.T; t += TW) {
-            const __nv_bfloat16 *x = reinterpret_cast<const __nv_bfloat16 *>(smem_raw + (size_t)t * xstride);
-            float s = 0.f;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const int k = i * 256 + tc.lane * 8;
-                if (k < dm.d) s += slice_dot(wreg[i], *reinterpret_cast<const uint4 *>(x + k));
-            }
-            const float tot = warp_sum(s);
-            if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
-        }
-    } else {
-        for (int t = tc.twarp; t < dm.T; t += TW) {
-            const float s = lane_dot_bf16(row, reinterpret_cast<const __nv_bfloat16 *>(smem_raw + (size_t)t * xstride),
-                                          dm.d, tc.lane);
-            const float tot = warp_sum(s);
-            if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
-        }
+    PROF(tc, 60);
+    for (int t = tc.twarp; t < dm.T; t += TW) {
+        const float sdot = lane_dot_bf16(row, reinterpret_cast<const __nv_bfloat16 *>(smem_raw + (size_t)t * xstride), dm.d,
+                                         tc.lane);
+        const float tot = warp_sum(sdot);
+        if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
     }
+    PROF(tc, 61);
     warp_signal(tc, p.sync + SY_R1_DONE);
+    PROF(tc, 62);
 }
 
-// R2: top-k + gates, classification, residual list, grouping (one team)
-__device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_raw, int nt, TeamCtx tc) {
+// exclusive scan across the lanes of a warp; returns the prefix of this lane and the warp total
+__device__ __forceinline__ int warp_excl_scan(int v, int lane, int &total) {
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    total = __shfl_sync(0xffffffffu, inc, 31);
+    return inc - v;
+}
+
+// R2: top-k + gates, classification, residual list, grouping (one team).  Everything between the
+// arrival of the logits and the published tables works out of shared memory; the ordered parts
+// (residual list, offsets of slots and experts) are done by single warps with shuffle scans.
+__device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_raw, int nt, TC_ARG tc) {
     const Dims &dm = p.dm;
     Smem sm;
     smem_layout(dm, nt, &sm, smem_raw);
     const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
     // while the logits are being produced: fetch what classification will need
+#pragma unroll 1
     for (int i = tc.ttid; i < N; i += TEAM) sm.s_soe[i] = p.w.slot_of_expert[i];
     const int n_conf = p.conf_stride ? T * N : T;
+#pragma unroll 1
     for (int i = tc.ttid; i < n_conf; i += TEAM) sm.s_conf[i] = p.conf[i];
     if (tc.ttid < 4) sm.s_cnt[tc.ttid] = 0;
     sm.cnt_hit[tc.ttid] = 0;
     sm.cnt_low[tc.ttid] = 0;
+    PROF(tc, 50);
     if (!team_wait_ge(tc, p.sync + SY_R1_DONE, N * TW, p)) return;
+    PROF(tc, 51);
+#pragma unroll 1
     for (int i = tc.ttid; i < T * N; i += TEAM) sm.lg[i] = __ldcg(p.logits + i);
     team_sync(tc.team);
+    PROF(tc, 52);
+#pragma unroll 1
     for (int t = tc.twarp; t < T; t += TW)
         warp_topk_gates(sm.lg + t * N, N, K, p.norm_topk, tc.lane, sm.s_idx + t * K, sm.s_gate + t * K, nullptr);
     team_sync(tc.team);
-    // classification (Sec. 4.2 policy) + ordered residual list (set M of Sec. 4.3)
-    int base = 0;
-    for (int i0 = 0; i0 < n; i0 += TEAM) {
-        const int i = i0 + tc.ttid;
-        int c = -1, e = 0, sl = -1;
-        if (i < n) {
-            e = sm.s_idx[i];
-            sl = sm.s_soe[e];
-            if (sl >= S) {
-                atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
-                sl = -1;
-                c = SPICE_MISS_EXACT;
-            } else if (sl >= 0) {
-                c = SPICE_HIT;
-                atomicAdd(&sm.cnt_hit[sl], 1);
-            } else {
-                sl = -1;
-                const int t = i / K;
-                const float cf = p.conf_stride ? sm.s_conf[t * N + e] : sm.s_conf[t];
-                c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
-                if (c == SPICE_LOWCONF) atomicAdd(&sm.cnt_low[e], 1);
+    PROF(tc, 53);
+    // classification (Sec. 4.2 policy); s_slot holds the grouping key: slot (HIT), 1024 + e (LOWCONF), -1
+#pragma unroll 1
+    for (int i = tc.ttid; i < n; i += TEAM) {
+        const int e = sm.s_idx[i];
+        int sl = sm.s_soe[e], c, key = -1;
+        if (sl >= S) {
+            atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
+            c = SPICE_MISS_EXACT;
+        } else if (sl >= 0) {
+            c = SPICE_HIT;
+            key = sl;
+            atomicAdd(&sm.cnt_hit[sl], 1);
+        } else {
+            const int t = i / K;
+            const float cf = p.conf_stride ? sm.s_conf[t * N + e] : sm.s_conf[t];
+            c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
+            if (c == SPICE_LOWCONF) {
+                key = 1024 + e;
+                atomicAdd(&sm.cnt_low[e], 1);
             }
-            sm.s_cls[i] = (unsigned char)c;
-            sm.s_slot[i] = sl;
-            p.idx[i] = e;
-            p.gate[i] = sm.s_gate[i];
-            p.cls[i] = (uint8_t)c;
-            atomicAdd(&sm.s_cnt[c], 1);
         }
+        sm.s_cls[i] = (unsigned char)c;
+        sm.s_slot[i] = key;
+        p.idx[i] = e;
+        p.gate[i] = sm.s_gate[i];
+        p.cls[i] = (uint8_t)c;
+        atomicAdd(&sm.s_cnt[c], 1);
+    }
+    team_sync(tc.team);
+    PROF(tc, 54);
+    if (tc.twarp == 0) {
+        // residual-miss list (set M of Sec. 4.3) in (t,k) order: each lane owns a contiguous run
+        const int per = (n + 31) / 32, i0 = min(n, tc.lane * per), i1 = min(n, i0 + per);
+        int mine = 0;
+#pragma unroll 1
+        for (int i = i0; i < i1; ++i) mine += sm.s_cls[i] == SPICE_MISS_EXACT;
         int total;
-        const int pos = team_excl_scan(tc, c == SPICE_MISS_EXACT ? 1 : 0, sm.wt, total);
-        if (c == SPICE_MISS_EXACT && p.resid_tok) {
-            const int o = base + pos;
-            p.resid_tok[o] = i / K;
-            p.resid_k[o] = i % K;
-            p.resid_expert[o] = e;
-            p.resid_gate[o] = sm.s_gate[i];
+        int o = warp_excl_scan(mine, tc.lane, total);
+        if (p.resid_tok)
+#pragma unroll 1
+            for (int i = i0; i < i1; ++i)
+                if (sm.s_cls[i] == SPICE_MISS_EXACT) {
+                    p.resid_tok[o] = i / K;
+                    p.resid_k[o] = i % K;
+                    p.resid_expert[o] = sm.s_idx[i];
+                    p.resid_gate[o] = sm.s_gate[i];
+                    ++o;
+                }
+        if (tc.lane < 3) p.counts[tc.lane] = sm.s_cnt[tc.lane];
+    } else if (tc.twarp == 1) {
+        // hit groups in slot order, then low-confidence groups in expert order (8 ids per lane)
+        int cnt[8], n_here = 0, g_here = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            cnt[j] = sm.cnt_hit[tc.lane * 8 + j];
+            n_here += cnt[j];
+            g_here += cnt[j] > 0;
         }
-        base += total;
+        int n_hit, n_hg;
+        int off = warp_excl_scan(n_here, tc.lane, n_hit);
+        int gi = warp_excl_scan(g_here, tc.lane, n_hg);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int id = tc.lane * 8 + j;
+            sm.off_hit[id] = off;
+            if (cnt[j] > 0) p.tb.groups[1 + gi++] = GroupDesc{KIND_HIT, id, off, cnt[j]};
+            off += cnt[j];
+        }
+        n_here = g_here = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            cnt[j] = sm.cnt_low[tc.lane * 8 + j];
+            n_here += cnt[j];
+            g_here += cnt[j] > 0;
+        }
+        int n_low, n_lg;
+        off = warp_excl_scan(n_here, tc.lane, n_low);
+        gi = warp_excl_scan(g_here, tc.lane, n_lg);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int id = tc.lane * 8 + j;
+            sm.off_low[id] = off;
+            if (cnt[j] > 0) p.tb.groups[1 + n_hg + gi++] = GroupDesc{KIND_LOW, id, off, cnt[j]};
+            off += cnt[j];
+        }
+        if (tc.lane == 0) {
+            p.tb.groups[0] = GroupDesc{KIND_SHARED, 0, 0, T};
+            p.tb.hdr[HDR_N_GROUPS] = 1 + n_hg + n_lg;
+            p.tb.hdr[HDR_N_HIT_GROUPS] = n_hg;
+            p.tb.hdr[HDR_N_LOW_GROUPS] = n_lg;
+            p.tb.hdr[HDR_N_HIT] = n_hit;
+            p.tb.hdr[HDR_N_LOW] = n_low;
+        }
+    } else {
+        // coefficient of the shared expert's output: 1 + sum of LOWCONF gates, in k order
+#pragma unroll 1
+        for (int t = tc.ttid - 64; t < T; t += TEAM - 64) {
+            float c = 1.0f;
+#pragma unroll 1
+            for (int k = 0; k < K; ++k)
+                if (sm.s_cls[t * K + k] == SPICE_LOWCONF) c += sm.s_gate[t * K + k];
+            p.tb.coef_shared[t] = c;
+        }
     }
     team_sync(tc.team);
-    if (tc.ttid < 3) p.counts[tc.ttid] = sm.s_cnt[tc.ttid];
-    // grouping
-    const int ch = sm.cnt_hit[tc.ttid], cl = sm.cnt_low[tc.ttid];
-    int n_hit, n_low, n_hg, n_lg;
-    const int oh = team_excl_scan(tc, ch, sm.wt, n_hit);
-    const int ol = team_excl_scan(tc, cl, sm.wt, n_low);
-    const int gh = team_excl_scan(tc, ch > 0 ? 1 : 0, sm.wt, n_hg);
-    const int gl = team_excl_scan(tc, cl > 0 ? 1 : 0, sm.wt, n_lg);
-    sm.off_hit[tc.ttid] = oh;
-    sm.off_low[tc.ttid] = ol;
-    if (ch > 0) p.tb.groups[1 + gh] = GroupDesc{KIND_HIT, tc.ttid, oh, ch};
-    if (cl > 0) p.tb.groups[1 + n_hg + gl] = GroupDesc{KIND_LOW, tc.ttid, ol, cl};
-    if (tc.ttid == 0) {
-        p.tb.groups[0] = GroupDesc{KIND_SHARED, 0, 0, T};
-        p.tb.hdr[HDR_N_GROUPS] = 1 + n_hg + n_lg;
-        p.tb.hdr[HDR_N_HIT_GROUPS] = n_hg;
-        p.tb.hdr[HDR_N_LOW_GROUPS] = n_lg;
-        p.tb.hdr[HDR_N_HIT] = n_hit;
-        p.tb.hdr[HDR_N_LOW] = n_low;
-    }
-    team_sync(tc.team);
+    PROF(tc, 55);
     sm.cnt_hit[tc.ttid] = 0;   // now cursors
     sm.cnt_low[tc.ttid] = 0;
     team_sync(tc.team);
+#pragma unroll 1
     for (int i0 = 0; i0 < n; i0 += TEAM) {
         const int i = i0 + tc.ttid;
-        int key = -1;
-        if (i < n) {
-            const int c = sm.s_cls[i];
-            if (c == SPICE_HIT) key = sm.s_slot[i];
-            else if (c == SPICE_LOWCONF) key = 1024 + sm.s_idx[i];
-        }
+        const int key = i < n ? sm.s_slot[i] : -1;
         const unsigned peers = __match_any_sync(0xffffffffu, key);
         int pos = -1;
         if (key >= 0) {
@@ -621,24 +578,18 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
         }
         if (i < n) p.tb.pos_of_entry[i] = pos;
     }
-    for (int t = tc.ttid; t < T; t += TEAM) {
-        float c = 1.0f;
-        for (int k = 0; k < K; ++k)
-            if (sm.s_cls[t * K + k] == SPICE_LOWCONF) c += sm.s_gate[t * K + k];
-        p.tb.coef_shared[t] = c;
-    }
     team_sync(tc.team);
-    if (tc.ttid == 0) {
-        __threadfence();
-        red_release_add(p.sync + SY_ROUTE_DONE, 1);
-    }
+    PROF(tc, 56);
+    if (tc.ttid == 0) red_release_add(p.sync + SY_ROUTE_DONE, 1);
+    PROF(tc, 57);
 }
 
 // ------------------------------------------------------------------------------------------
 // Task list.  ids [0, nA) are known at launch; the rest once the router has published the groups.
 struct Plan {
     int n_r1, nA;                       // phase A: R1 tasks, R2, shared gate/up tiles
-    int tIs, tI, tr, td, tb128, nb;     // tiles per matrix
+    int tIs, tI, tr, td_sh, td_hit, tb128, nb;   // tiles per matrix
+    int rt_sh, rt_hit;                  // 16-row tiles per P2 task (shared / hit groups)
     int n_hg, n_lg, nB_hit, endB;       // phase B: hit gate/up tiles, LoRE A tiles
     int nC_sh, nC_hit, endC, endD;      // phase C: down tiles; phase D: combine blocks
     bool routed;                        // phases B..D resolvable
@@ -663,7 +614,7 @@ __device__ __forceinline__ TaskRef resolve(const Plan &pl, int id) {
     if (id < pl.endC) {
         const int l = id - pl.endB;
         if (l < pl.nC_sh) return TaskRef{TK_P2, 0, l};
-        if (l < pl.nC_sh + pl.nC_hit) return TaskRef{TK_P2, 1 + (l - pl.nC_sh) / pl.td, (l - pl.nC_sh) % pl.td};
+        if (l < pl.nC_sh + pl.nC_hit) return TaskRef{TK_P2, 1 + (l - pl.nC_sh) / pl.td_hit, (l - pl.nC_sh) % pl.td_hit};
         const int q = l - pl.nC_sh - pl.nC_hit;
         return TaskRef{TK_P2, 1 + pl.n_hg + q / pl.tb128, q % pl.tb128};
     }
@@ -696,66 +647,277 @@ __device__ __forceinline__ void setup_rows(const DecodeParams &p, uint32_t xs_s,
     }
 }
 
-struct NoGate {
-    __device__ __forceinline__ bool operator()() const { return true; }
-};
-
-// P1 task: gate/up + SwiGLU rows of the shared expert or of a hit slot, or LoRE A rows
-template <int NT>
-__device__ __forceinline__ bool task_p1(const DecodeParams &p, uint32_t xs_s, int xstride, TeamCtx &tc, int gi,
-                                        int tile) {
-    const Dims &dm = p.dm;
-    const GroupDesc grp = group_of(p, tc, gi);
-    unsigned long long bptr[NT];
-    bool bok[NT];
-    setup_rows<NT, true>(p, xs_s, xstride, tc, grp, nullptr, 0, bptr, bok);
-    if (grp.kind == KIND_LOW) {
-        const __nv_bfloat16 *A = reinterpret_cast<const __nv_bfloat16 *>(p.w.lore_A) + (size_t)grp.id * dm.r * dm.d;
-        return team_tile_ksplit<NT, EPI_Z, true>(tc, grp, A, nullptr, tile * 16, dm.r, dm.d, bptr, bok, p.z16, nullptr,
-                                                 dm.r, NoGate());
-    } else if (grp.kind == KIND_HIT) {
-        const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.slot_w_gate_up) + (size_t)grp.id * 2 * dm.I * dm.d;
-        return team_tile_ksplit<NT, EPI_ACT, true>(tc, grp, W, W + (size_t)dm.I * dm.d, tile * 16, dm.I, dm.d, bptr, bok,
-                                                   p.act_hit16, nullptr, dm.I, NoGate());
-    }
-    const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_gate_up);
-    return team_tile_ksplit<NT, EPI_ACT, true>(tc, grp, W, W + (size_t)dm.Is * dm.d, tile * 16, dm.Is, dm.d, bptr, bok,
-                                               p.act_shared16, nullptr, dm.Is, NoGate());
-}
-
-// P2 task: down-projection rows of one group.  The first P2 tile of a warp publishes the warp's P1
-// count and waits (after its first weight loads are in flight) until every P1 tile of the layer is
-// published; later tiles do not wait.
-template <int NT>
-__device__ __forceinline__ bool task_p2(const DecodeParams &p, TeamCtx &tc, int gi, int tile, int p1_total) {
-    const Dims &dm = p.dm;
-    const GroupDesc grp = group_of(p, tc, gi);
-    unsigned long long bptr[NT];
-    bool bok[NT];
-    auto gate = [&]() {
+// The first P2 tile of a warp publishes the warp's P1 count and waits (after its first weight loads
+// are in flight) until every P1 tile of the layer is published; later tiles do not wait.
+struct P1DoneGate {
+    const DecodeParams &p;
+    TeamCtx &tc;
+    int p1_total;
+    __device__ __forceinline__ bool operator()() const {
         if (tc.p1_all) return true;
         flush_counts(tc, p.sync);
         tc.p1_all = warp_wait_ge(tc, p.sync + SY_P1_ALL, p1_total, p);
         return tc.p1_all;
-    };
-    if (grp.kind == KIND_SHARED) {
-        setup_rows<NT, false>(p, 0u, 0, tc, grp, reinterpret_cast<const unsigned char *>(p.act_shared16),
-                              (size_t)dm.Is * 2, bptr, bok);
-        return team_tile_ksplit<NT, EPI_PART, false>(tc, grp, reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_down),
-                                                     nullptr, tile * 16, dm.d, dm.Is, bptr, bok, nullptr,
-                                                     p.tb.part_shared, dm.d, gate);
-    } else if (grp.kind == KIND_HIT) {
-        setup_rows<NT, false>(p, 0u, 0, tc, grp,
-                              reinterpret_cast<const unsigned char *>(p.act_hit16 + (size_t)grp.off * dm.I),
-                              (size_t)dm.I * 2, bptr, bok);
-        const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.slot_w_down) + (size_t)grp.id * dm.d * dm.I;
-        return team_tile_ksplit<NT, EPI_PART, false>(tc, grp, W, nullptr, tile * 16, dm.d, dm.I, bptr, bok, nullptr,
-                                                     p.tb.part, dm.d, gate);
     }
+};
+
+// What a task runs as.  Consecutive tasks of one team with the same flavour are executed as one
+// software-pipelined run (team_run).
+enum { FL_NONE = 0, FL_R1, FL_R2, FL_ACT, FL_Z, FL_PART, FL_PART2, FL_LOREB, FL_P3 };
+
+__device__ __forceinline__ int flavour_of(const Plan &pl, const TeamCtx &tc, const TaskRef &t) {
+    if (t.kind == TK_NONE) return FL_NONE;
+    if (t.kind == TK_R1) return FL_R1;
+    if (t.kind == TK_R2) return FL_R2;
+    if (t.kind == TK_P3) return FL_P3;
+    const int kind = t.gi == 0 ? KIND_SHARED : tc.gtab[t.gi].kind;
+    if (t.kind == TK_P1) return kind == KIND_LOW ? FL_Z : FL_ACT;
+    if (kind == KIND_LOW) return FL_LOREB;
+    return (kind == KIND_HIT ? pl.rt_hit : pl.rt_sh) == 2 ? FL_PART2 : FL_PART;
+}
+
+// Everything one tile needs, resolved from its task.
+struct TileArgs {
+    GroupDesc grp;
+    const __nv_bfloat16 *W0, *W1;   // first rows of the matrix (pair)
+    int row0, n_rows, K;
+    __nv_bfloat16 *out16;
+    float *out32;
+    int ld_out;
+    const unsigned char *b_base;    // P2: first activation row of the group
+};
+
+template <int EPI>
+__device__ __forceinline__ TileArgs tile_args(const DecodeParams &p, const TeamCtx &tc, const TaskRef &t) {
+    const Dims &dm = p.dm;
+    TileArgs a;
+    a.grp = group_of(p, tc, t.gi);
+    const bool hit = a.grp.kind == KIND_HIT;
+    a.out16 = nullptr;
+    a.out32 = nullptr;
+    a.b_base = nullptr;
+    a.W1 = nullptr;
+    if (EPI == EPI_ACT) {
+        a.n_rows = hit ? dm.I : dm.Is;
+        a.K = dm.d;
+        a.W0 = hit ? reinterpret_cast<const __nv_bfloat16 *>(p.w.slot_w_gate_up) + (size_t)a.grp.id * 2 * dm.I * dm.d
+                   : reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_gate_up);
+        a.W1 = a.W0 + (size_t)a.n_rows * dm.d;
+        a.row0 = t.tile * 16;
+        a.out16 = hit ? p.act_hit16 : p.act_shared16;
+        a.ld_out = a.n_rows;
+    } else if (EPI == EPI_Z) {
+        a.n_rows = dm.r;
+        a.K = dm.d;
+        a.W0 = reinterpret_cast<const __nv_bfloat16 *>(p.w.lore_A) + (size_t)a.grp.id * dm.r * dm.d;
+        a.row0 = t.tile * 16;
+        a.out16 = p.z16;
+        a.ld_out = dm.r;
+    } else {
+        a.n_rows = dm.d;
+        a.K = hit ? dm.I : dm.Is;
+        a.W0 = hit ? reinterpret_cast<const __nv_bfloat16 *>(p.w.slot_w_down) + (size_t)a.grp.id * dm.d * dm.I
+                   : reinterpret_cast<const __nv_bfloat16 *>(p.w.shared_w_down);
+        a.row0 = t.tile * (EPI == EPI_PART2 ? 32 : 16);
+        a.out32 = hit ? p.tb.part : p.tb.part_shared;
+        a.ld_out = dm.d;
+        a.b_base = hit ? reinterpret_cast<const unsigned char *>(p.act_hit16 + (size_t)a.grp.off * dm.I)
+                       : reinterpret_cast<const unsigned char *>(p.act_shared16);
+    }
+    return a;
+}
+
+// this lane's weight rows and this warp's share of the reduction
+template <int EPI>
+__device__ __forceinline__ WRows make_rows(const TileArgs &a, const TeamCtx &tc) {
+    constexpr bool DUAL = (EPI == EPI_ACT || EPI == EPI_PART2);
+    const int g = tc.lane >> 2;
+    const int KS = (a.K + 31) >> 5;
+    const int base = KS / TW, rem = KS % TW;
+    WRows w;
+    w.K = a.K;
+    w.ks0 = tc.twarp * base + min(tc.twarp, rem);
+    w.ks1 = w.ks0 + base + (tc.twarp < rem ? 1 : 0);
+    const int rlo = a.row0 + g, rhi = a.row0 + g + 8;
+    // second matrix: the up rows of the same indices, or (EPI_PART2) rows +16 of the same matrix
+    const int r1lo = (EPI == EPI_PART2) ? rlo + 16 : rlo, r1hi = (EPI == EPI_PART2) ? rhi + 16 : rhi;
+    const __nv_bfloat16 *W1 = (EPI == EPI_PART2) ? a.W0 : a.W1;
+    w.ok_lo = rlo < a.n_rows;
+    w.ok_hi = rhi < a.n_rows;
+    w.ok1_lo = DUAL && r1lo < a.n_rows;
+    w.ok1_hi = DUAL && r1hi < a.n_rows;
+    w.p0lo = a.W0 + (size_t)(w.ok_lo ? rlo : 0) * a.K;
+    w.p0hi = a.W0 + (size_t)(w.ok_hi ? rhi : 0) * a.K;
+    w.p1lo = DUAL ? W1 + (size_t)(w.ok1_lo ? r1lo : 0) * a.K : nullptr;
+    w.p1hi = DUAL ? W1 + (size_t)(w.ok1_hi ? r1hi : 0) * a.K : nullptr;
+    return w;
+}
+
+// issue the 128-bit loads of U k-steps starting at ks (rows / k-steps that do not exist give zeros)
+template <bool DUAL, int U>
+__device__ __forceinline__ void load_batch(const WRows &w, int ks, uint4 (&a0lo)[U], uint4 (&a0hi)[U], uint4 (&a1lo)[U],
+                                           uint4 (&a1hi)[U], int c) {
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int kb = (ks + u) * 32 + c * 8;
+        const bool in = (ks + u < w.ks1) && (kb < w.K);
+        a0lo[u] = (in && w.ok_lo) ? ldg_stream(w.p0lo + kb) : zero;
+        a0hi[u] = (in && w.ok_hi) ? ldg_stream(w.p0hi + kb) : zero;
+        if (DUAL) {
+            a1lo[u] = (in && w.ok1_lo) ? ldg_stream(w.p1lo + kb) : zero;
+            a1hi[u] = (in && w.ok1_hi) ? ldg_stream(w.p1hi + kb) : zero;
+        }
+    }
+}
+
+// A run of consecutive tiles of one flavour for one team, reduction split over the 8 warps.
+//   EPI_ACT  : W0 = gate rows, W1 = up rows; act[orow][row] = silu(g)*u            (P1 shared / hit)
+//   EPI_Z    : z[orow][row] = sum                                                 (P1 LoRE A)
+//   EPI_PART : part[orow][row] = sum                                              (P2 down, 16 rows)
+//   EPI_PART2: the same for 32 rows: rows +16 share the activation loads          (P2 down, short K)
+// The weight loads of a tile's next batch -- or of the NEXT tile's first batch -- are issued before
+// the partial sums are exchanged, so the memory pipe stays busy through barriers and epilogue.
+// Returns the id of the first task not executed; *alive = 0 (team-uniform) when a wait failed.
+template <int NT, int EPI>
+__device__ SPICE_RUN_INLINE int team_run(const DecodeParams &p, const Plan &pl, TeamCtx &tc, uint32_t xs_s, int xstride, int id,
+                                     int n_teams, int p1_total, int *alive) {
+    constexpr bool DUAL = (EPI == EPI_ACT || EPI == EPI_PART2);
+    constexpr bool B_SMEM = (EPI == EPI_ACT || EPI == EPI_Z);
+    constexpr int MATS = DUAL ? 2 : 1;
+    constexpr int U = (NT == 4 || EPI == EPI_PART2) ? 2 : 4;
+    constexpr int MYFL = EPI == EPI_ACT ? FL_ACT : (EPI == EPI_Z ? FL_Z : (EPI == EPI_PART ? FL_PART : FL_PART2));
+    const int c = tc.lane & 3;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    uint4 a0lo[U], a0hi[U], a1lo[U], a1hi[U];
+    TileArgs a = tile_args<EPI>(p, tc, resolve(pl, id));
+    WRows w = make_rows<EPI>(a, tc);
+    load_batch<DUAL, U>(w, w.ks0, a0lo, a0hi, a1lo, a1hi, c);
+    bool failed = false;
+    if (!B_SMEM && !tc.p1_all) {   // first P2 tile of this warp: every P1 tile must be published
+        flush_counts(tc, p.sync);
+        tc.p1_all = warp_wait_ge(tc, p.sync + SY_P1_ALL, p1_total, p);
+        failed = !tc.p1_all;
+    }
+    *alive = 1;
+    for (;;) {
+        PROF(tc, 100 + (B_SMEM ? TK_P1 : TK_P2));
+        const int nid = id + n_teams;
+        const TaskRef nt = resolve(pl, nid);
+        const bool same = flavour_of(pl, tc, nt) == MYFL;
+        unsigned long long bptr[NT];
+        bool bok[NT];
+        setup_rows<NT, B_SMEM>(p, xs_s, xstride, tc, a.grp, a.b_base, (size_t)a.K * 2, bptr, bok);
+        float acc0[NT][4], acc1[NT][4];
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc0[nn][r] = acc1[nn][r] = 0.f;
+        for (int ks = w.ks0;; ks += U) {
+            uint4 bg[B_SMEM ? 1 : U][NT];
+            if (!B_SMEM) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int kb = (ks + u) * 32 + c * 8;
+                    const bool in = (ks + u < w.ks1) && (kb < w.K);
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn)
+                        bg[u][nn] = (in && bok[nn])
+                                        ? ldcg128(reinterpret_cast<const unsigned char *>(bptr[nn]) + (size_t)kb * 2)
+                                        : zero;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int kb = (ks + u) * 32 + c * 8;
+                const bool in = (ks + u < w.ks1) && (kb < w.K);
+                if (ks + u < w.ks1) {   // warp-uniform
+#pragma unroll
+                    for (int nn = 0; nn < NT; ++nn) {
+                        uint4 b;
+                        if (B_SMEM) b = (in && bok[nn]) ? lds128((uint32_t)bptr[nn] + kb * 2) : zero;
+                        else b = bg[u][nn];
+                        mma_bf16(acc0[nn], a0lo[u].x, a0hi[u].x, a0lo[u].y, a0hi[u].y, b.x, b.y);
+                        mma_bf16(acc0[nn], a0lo[u].z, a0hi[u].z, a0lo[u].w, a0hi[u].w, b.z, b.w);
+                        if (DUAL) {
+                            mma_bf16(acc1[nn], a1lo[u].x, a1hi[u].x, a1lo[u].y, a1hi[u].y, b.x, b.y);
+                            mma_bf16(acc1[nn], a1lo[u].z, a1hi[u].z, a1lo[u].w, a1hi[u].w, b.z, b.w);
+                        }
+                    }
+                }
+            }
+            if (ks + U < w.ks1) {
+                load_batch<DUAL, U>(w, ks + U, a0lo, a0hi, a1lo, a1hi, c);
+            } else {
+#ifndef SPICE_NO_PRELOAD
+                if (same) {   // first batch of the next tile rides through this tile's exchange and epilogue
+                    const TileArgs an = tile_args<EPI>(p, tc, nt);
+                    const WRows wn = make_rows<EPI>(an, tc);
+                    load_batch<DUAL, U>(wn, wn.ks0, a0lo, a0hi, a1lo, a1hi, c);
+                }
+#endif
+                break;
+            }
+        }
+        PROF(tc, 20);
+        // every warp is past the previous tile's epilogue once it arrives here
+        if (team_sync_or(tc.team, failed)) {
+            *alive = 0;
+            return nid;
+        }
+        float *red = tc.red;
+#pragma unroll
+        for (int nn = 0; nn < NT; ++nn)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                red[((tc.twarp * MATS + 0) * NT + nn) * 128 + r * 32 + tc.lane] = acc0[nn][r];
+                if (DUAL) red[((tc.twarp * MATS + 1) * NT + nn) * 128 + r * 32 + tc.lane] = acc1[nn][r];
+            }
+        team_sync(tc.team);
+        PROF(tc, 21);
+        for (int e = tc.ttid; e < NT * 128; e += TEAM) {
+            const int nn = e >> 7, r = (e >> 5) & 3, ln = e & 31;
+            const int row = a.row0 + (ln >> 2) + ((r & 2) ? 8 : 0);
+            const int n = nn * 8 + 2 * (ln & 3) + (r & 1);
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int wi = 0; wi < TW; ++wi) {
+                s0 += red[((wi * MATS + 0) * NT + nn) * 128 + r * 32 + ln];
+                if (DUAL) s1 += red[((wi * MATS + 1) * NT + nn) * 128 + r * 32 + ln];
+            }
+            if (n < a.grp.m && row < a.n_rows) {
+                const size_t o = (size_t)out_row(tc, a.grp, B_SMEM, n) * a.ld_out + row;
+                if (EPI == EPI_ACT) a.out16[o] = __float2bfloat16(silu_f(s0) * s1);
+                else if (EPI == EPI_Z) a.out16[o] = __float2bfloat16(s0);
+                else a.out32[o] = s0;
+                if (EPI == EPI_PART2 && row + 16 < a.n_rows) a.out32[o + 16] = s1;
+            }
+        }
+        PROF(tc, 22);
+        if (B_SMEM) tc.n_p1++;
+        else tc.n_p2++;
+        id = nid;
+        if (!same) break;
+        a = tile_args<EPI>(p, tc, nt);
+        w = make_rows<EPI>(a, tc);
+#ifdef SPICE_NO_PRELOAD
+        load_batch<DUAL, U>(w, w.ks0, a0lo, a0hi, a1lo, a1hi, c);
+#endif
+    }
+    return id;
+}
+
+// P2 of a LoRE group (short reduction, 128 rows per task); not pipelined, the tasks are tiny
+template <int NT>
+__device__ __noinline__ bool task_lore_b(const DecodeParams &p, TeamCtx &tc, int gi, int tile, int p1_total) {
+    const Dims &dm = p.dm;
+    const GroupDesc grp = group_of(p, tc, gi);
+    unsigned long long bptr[NT];
+    bool bok[NT];
     setup_rows<NT, false>(p, 0u, 0, tc, grp, reinterpret_cast<const unsigned char *>(p.z16 + (size_t)grp.off * dm.r),
                           (size_t)dm.r * 2, bptr, bok);
     const __nv_bfloat16 *W = reinterpret_cast<const __nv_bfloat16 *>(p.w.lore_B) + (size_t)grp.id * dm.d * dm.r;
-    return team_block_rows<NT>(tc, grp, W, tile * 128, dm.d, dm.r, bptr, bok, p.tb.part, dm.d, gate);
+    return team_block_rows<NT>(tc, grp, W, tile * 128, dm.d, dm.r, bptr, bok, p.tb.part, dm.d, P1DoneGate{p, tc, p1_total});
 }
 
 // P3 task: 1024 columns of one token
@@ -824,7 +986,10 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
     pl.tIs = (dm.Is + 15) >> 4;
     pl.tI = (dm.I + 15) >> 4;
     pl.tr = (dm.r + 15) >> 4;
-    pl.td = (dm.d + 15) >> 4;
+    pl.rt_sh = (NT <= 2 && dm.Is <= 4096) ? 2 : 1;
+    pl.rt_hit = (NT <= 2 && dm.I <= 4096) ? 2 : 1;
+    pl.td_sh = (dm.d + 16 * pl.rt_sh - 1) / (16 * pl.rt_sh);
+    pl.td_hit = (dm.d + 16 * pl.rt_hit - 1) / (16 * pl.rt_hit);
     pl.tb128 = (dm.d + 127) >> 7;
     pl.nb = (dm.d + 1023) >> 10;
     pl.nA = p.n_r1 + 1 + pl.tIs;
@@ -860,16 +1025,24 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
     __syncthreads();
     PROF(tc, 2);
 
-    bool alive = true;
-    for (; id < pl.nA && alive; id += n_teams) {
-        PROF(tc, 100 + resolve(pl, id).kind);
-        if (id < p.n_r1) task_r1(p, smem_raw, tc, id);
-        else if (id == p.n_r1) task_r2(p, smem_raw, NT, tc);
-        else alive = task_p1<NT>(p, xs_s, xstride, tc, 0, id - p.n_r1 - 1);
+    int alive = 1;
+    while (id < pl.nA && alive) {
+        const int fl = flavour_of(pl, tc, resolve(pl, id));
+        if (fl == FL_R1) {
+            PROF(tc, 100 + TK_R1);
+            task_r1(p, smem_raw, tc, id);
+            id += n_teams;
+        } else if (fl == FL_R2) {
+            PROF(tc, 100 + TK_R2);
+            task_r2(p, smem_raw, NT, tc);
+            id += n_teams;
+        } else {
+            id = team_run<NT, EPI_ACT>(p, pl, tc, xs_s, xstride, id, n_teams, 0, &alive);   // shared gate/up tiles
+        }
     }
     // every quantity below is uniform across the team (it comes from team-wide reductions)
     PROF(tc, 30);
-    alive = alive && team_wait_ge(tc, p.sync + SY_ROUTE_DONE, 1, p);
+    if (alive) alive = team_wait_ge(tc, p.sync + SY_ROUTE_DONE, 1, p) ? 1 : 0;
     PROF(tc, 31);
     if (alive) {
         // team-private copy of the group table and the permutations: task set-up never goes to L2 again
@@ -881,8 +1054,8 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
         for (int i = tc.ttid; i < n_low; i += TEAM) tc.perm_l[i] = __ldcg(p.tb.perm_low + i);
         pl.nB_hit = pl.n_hg * pl.tI;
         pl.endB = pl.nA + pl.nB_hit + pl.n_lg * pl.tr;
-        pl.nC_sh = pl.td;
-        pl.nC_hit = pl.n_hg * pl.td;
+        pl.nC_sh = pl.td_sh;
+        pl.nC_hit = pl.n_hg * pl.td_hit;
         const int nC = pl.nC_sh + pl.nC_hit + pl.n_lg * pl.tb128;
         pl.endC = pl.endB + nC;
         pl.endD = pl.endC + dm.T * pl.nb;
@@ -890,21 +1063,24 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
         const int p1_total = (pl.tIs + pl.nB_hit + pl.n_lg * pl.tr) * TW;
         team_sync(tc.team);
         bool p2_ready = false;
-        for (; id < pl.endD && alive; id += n_teams) {
+        while (id < pl.endD && alive) {
             const TaskRef t = resolve(pl, id);
-            PROF(tc, 100 + t.kind);
-                PROF(tc, 10);
-            if (t.kind == TK_P1) {
-                alive = task_p1<NT>(p, xs_s, xstride, tc, t.gi, t.tile);
-            } else if (t.kind == TK_P2) {
-                alive = task_p2<NT>(p, tc, t.gi, t.tile, p1_total);
+            const int fl = flavour_of(pl, tc, t);
+            if (fl == FL_ACT) id = team_run<NT, EPI_ACT>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+            else if (fl == FL_Z) id = team_run<NT, EPI_Z>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+            else if (fl == FL_PART2) id = team_run<(NT <= 2 ? NT : 1), EPI_PART2>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+            else if (fl == FL_PART) id = team_run<NT, EPI_PART>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+            else if (fl == FL_LOREB) {
+                alive = task_lore_b<NT>(p, tc, t.gi, t.tile, p1_total) ? 1 : 0;
+                id += n_teams;
             } else {
                 if (!p2_ready) {   // combine needs every down-projected row (counted per warp)
-                    alive = team_wait_ge(tc, p.sync + SY_P2_DONE, nC * TW, p);
+                    alive = team_wait_ge(tc, p.sync + SY_P2_DONE, nC * TW, p) ? 1 : 0;
                     if (!alive) break;
                     p2_ready = true;
                 }
                 task_p3(p, tc.ttid, t.tile / pl.nb, t.tile % pl.nb);
+                id += n_teams;
             }
         }
     }

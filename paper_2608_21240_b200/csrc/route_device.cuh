@@ -51,13 +51,16 @@ __device__ __forceinline__ float lane_dot_bf16(const __nv_bfloat16 *__restrict__
 __device__ __forceinline__ void warp_topk_gates(const float *l, int N, int K, int norm_topk, int lane,
                                                 int32_t *idx_out, float *gate_out, float *logits_out) {
     if (logits_out)
+#pragma unroll 1
         for (int e = lane; e < N; e += 32) logits_out[e] = l[e];
     uint32_t taken = 0;     // bit i: expert lane + 32*i already selected (N <= 1024)
     float m = 0.f, denom = 0.f, my_val = 0.f;
     int my_idx = 0;
+#pragma unroll 1
     for (int k = 0; k < K; ++k) {
         float bv = -INFINITY;
         int be = 0x7fffffff;
+#pragma unroll 1
         for (int i = 0, e = lane; e < N; ++i, e += 32) {
             if ((taken >> i) & 1u) continue;
             float v = l[e];
@@ -75,6 +78,7 @@ __device__ __forceinline__ void warp_topk_gates(const float *l, int N, int K, in
             m = bv;
             if (!norm_topk) {   // full-softmax denominator
                 float s = 0.f;
+#pragma unroll 1
                 for (int e = lane; e < N; e += 32) s += expf(l[e] - m);
                 denom = warp_sum(s);
             }
@@ -85,6 +89,7 @@ __device__ __forceinline__ void warp_topk_gates(const float *l, int N, int K, in
     if (norm_topk) {
         // sum the K numerators in k order on every lane (deterministic, matches the definition)
         float s = 0.f;
+#pragma unroll 1
         for (int k = 0; k < K; ++k) s += __shfl_sync(0xffffffffu, p, k);
         denom = s;
     }
