@@ -34,10 +34,6 @@ namespace spice {
 
 namespace {
 
-#ifndef SPICE_RUN_INLINE
-#define SPICE_RUN_INLINE __forceinline__
-#endif
-
 constexpr int DT = 512;     // threads per CTA
 constexpr int TEAM = 256;   // threads per team
 constexpr int TW = 8;       // warps per team
@@ -328,6 +324,8 @@ struct Smem {
     int *cnt_hit, *cnt_low, *off_hit, *off_low;   // [256] each
     int *wt;             // [TW+1]
     int *s_cnt;          // [4]
+    int *sel_idx;        // [TW][32] top-k scratch
+    float *sel_val;      // [TW][32]
 };
 
 __host__ __device__ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -354,6 +352,7 @@ __host__ __device__ inline size_t smem_layout(const Dims &dm, int nt, Smem *s, u
     size_t o_idx = take((size_t)n * 4), o_gate = take((size_t)n * 4), o_slot = take((size_t)n * 4), o_cls = take(n);
     size_t o_hist = take(4 * 256 * 4);
     size_t o_wt = take((TW + 1 + 4) * 4);
+    size_t o_sel = take(2 * TW * 32 * 4);
     if (s) {
         s->xs = base + o_xs;
         s->xstride = (int)xstride;
@@ -381,6 +380,8 @@ __host__ __device__ inline size_t smem_layout(const Dims &dm, int nt, Smem *s, u
         s->off_low = hist + 768;
         s->wt = reinterpret_cast<int *>(base + o_wt);
         s->s_cnt = s->wt + TW + 1;
+        s->sel_idx = reinterpret_cast<int *>(base + o_sel);
+        s->sel_val = reinterpret_cast<float *>(base + o_sel) + TW * 32;
     }
     return align_up(off, 128);
 }
@@ -442,7 +443,8 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
     PROF(tc, 52);
 #pragma unroll 1
     for (int t = tc.twarp; t < T; t += TW)
-        warp_topk_gates(sm.lg + t * N, N, K, p.norm_topk, tc.lane, sm.s_idx + t * K, sm.s_gate + t * K, nullptr);
+        warp_topk_gates(sm.lg + t * N, N, K, p.norm_topk, tc.lane, sm.s_idx + t * K, sm.s_gate + t * K, nullptr,
+                        sm.sel_idx + tc.twarp * 32, sm.sel_val + tc.twarp * 32);
     team_sync(tc.team);
     PROF(tc, 53);
     // classification (Sec. 4.2 policy); s_slot holds the grouping key: slot (HIT), 1024 + e (LOWCONF), -1
@@ -780,7 +782,7 @@ __device__ __forceinline__ void load_batch(const WRows &w, int ks, uint4 (&a0lo)
 // the partial sums are exchanged, so the memory pipe stays busy through barriers and epilogue.
 // Returns the id of the first task not executed; *alive = 0 (team-uniform) when a wait failed.
 template <int NT, int EPI>
-__device__ SPICE_RUN_INLINE int team_run(const DecodeParams &p, const Plan &pl, TeamCtx &tc, uint32_t xs_s, int xstride, int id,
+__device__ __forceinline__ int team_run(const DecodeParams &p, const Plan &pl, TeamCtx &tc, uint32_t xs_s, int xstride, int id,
                                      int n_teams, int p1_total, int *alive) {
     constexpr bool DUAL = (EPI == EPI_ACT || EPI == EPI_PART2);
     constexpr bool B_SMEM = (EPI == EPI_ACT || EPI == EPI_Z);
@@ -813,20 +815,20 @@ __device__ SPICE_RUN_INLINE int team_run(const DecodeParams &p, const Plan &pl, 
         for (int nn = 0; nn < NT; ++nn)
 #pragma unroll
             for (int r = 0; r < 4; ++r) acc0[nn][r] = acc1[nn][r] = 0.f;
-        for (int ks = w.ks0;; ks += U) {
-            uint4 bg[B_SMEM ? 1 : U][NT];
-            if (!B_SMEM) {
+        uint4 bg[B_SMEM ? 1 : U][NT];   // activations (P2): fetched one batch ahead, like the weights
+        auto load_acts = [&](int ks) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int kb = (ks + u) * 32 + c * 8;
-                    const bool in = (ks + u < w.ks1) && (kb < w.K);
+            for (int u = 0; u < U; ++u) {
+                const int kb = (ks + u) * 32 + c * 8;
+                const bool in = (ks + u < w.ks1) && (kb < w.K);
 #pragma unroll
-                    for (int nn = 0; nn < NT; ++nn)
-                        bg[u][nn] = (in && bok[nn])
-                                        ? ldcg128(reinterpret_cast<const unsigned char *>(bptr[nn]) + (size_t)kb * 2)
-                                        : zero;
-                }
+                for (int nn = 0; nn < NT; ++nn)
+                    bg[B_SMEM ? 0 : u][nn] =
+                        (in && bok[nn]) ? ldcg128(reinterpret_cast<const unsigned char *>(bptr[nn]) + (size_t)kb * 2) : zero;
             }
+        };
+        if (!B_SMEM) load_acts(w.ks0);
+        for (int ks = w.ks0;; ks += U) {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int kb = (ks + u) * 32 + c * 8;
@@ -836,7 +838,7 @@ __device__ SPICE_RUN_INLINE int team_run(const DecodeParams &p, const Plan &pl, 
                     for (int nn = 0; nn < NT; ++nn) {
                         uint4 b;
                         if (B_SMEM) b = (in && bok[nn]) ? lds128((uint32_t)bptr[nn] + kb * 2) : zero;
-                        else b = bg[u][nn];
+                        else b = bg[B_SMEM ? 0 : u][nn];
                         mma_bf16(acc0[nn], a0lo[u].x, a0hi[u].x, a0lo[u].y, a0hi[u].y, b.x, b.y);
                         mma_bf16(acc0[nn], a0lo[u].z, a0hi[u].z, a0lo[u].w, a0hi[u].w, b.z, b.w);
                         if (DUAL) {
@@ -848,14 +850,13 @@ __device__ SPICE_RUN_INLINE int team_run(const DecodeParams &p, const Plan &pl, 
             }
             if (ks + U < w.ks1) {
                 load_batch<DUAL, U>(w, ks + U, a0lo, a0hi, a1lo, a1hi, c);
+                if (!B_SMEM) load_acts(ks + U);
             } else {
-#ifndef SPICE_NO_PRELOAD
                 if (same) {   // first batch of the next tile rides through this tile's exchange and epilogue
                     const TileArgs an = tile_args<EPI>(p, tc, nt);
                     const WRows wn = make_rows<EPI>(an, tc);
                     load_batch<DUAL, U>(wn, wn.ks0, a0lo, a0hi, a1lo, a1hi, c);
                 }
-#endif
                 break;
             }
         }
@@ -900,9 +901,6 @@ __device__ SPICE_RUN_INLINE int team_run(const DecodeParams &p, const Plan &pl, 
         if (!same) break;
         a = tile_args<EPI>(p, tc, nt);
         w = make_rows<EPI>(a, tc);
-#ifdef SPICE_NO_PRELOAD
-        load_batch<DUAL, U>(w, w.ks0, a0lo, a0hi, a1lo, a1hi, c);
-#endif
     }
     return id;
 }
@@ -1025,54 +1023,54 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
     __syncthreads();
     PROF(tc, 2);
 
-    int alive = 1;
-    while (id < pl.nA && alive) {
-        const int fl = flavour_of(pl, tc, resolve(pl, id));
-        if (fl == FL_R1) {
-            PROF(tc, 100 + TK_R1);
-            task_r1(p, smem_raw, tc, id);
-            id += n_teams;
-        } else if (fl == FL_R2) {
-            PROF(tc, 100 + TK_R2);
-            task_r2(p, smem_raw, NT, tc);
-            id += n_teams;
-        } else {
-            id = team_run<NT, EPI_ACT>(p, pl, tc, xs_s, xstride, id, n_teams, 0, &alive);   // shared gate/up tiles
+    // One dispatch loop: a single call site per tile flavour keeps the code small.  Everything that
+    // steers it is uniform across the team (ids, and results of team-wide reductions).
+    int alive = 1, p1_total = 0, nC = 0;
+    bool p2_ready = false;
+    int end = pl.nA;
+    while (alive) {
+        if (id >= end) {
+            if (pl.routed) break;
+            // first task beyond phase A: the router's tables are needed from here on
+            PROF(tc, 30);
+            alive = team_wait_ge(tc, p.sync + SY_ROUTE_DONE, 1, p) ? 1 : 0;
+            PROF(tc, 31);
+            if (!alive) break;
+            // team-private copy of the group table and the permutations: task set-up never goes to L2 again
+            pl.n_hg = __ldcg(p.tb.hdr + HDR_N_HIT_GROUPS);
+            pl.n_lg = __ldcg(p.tb.hdr + HDR_N_LOW_GROUPS);
+            const int n_hit = __ldcg(p.tb.hdr + HDR_N_HIT), n_low = __ldcg(p.tb.hdr + HDR_N_LOW);
+            for (int i = tc.ttid; i < 1 + pl.n_hg + pl.n_lg; i += TEAM) tc.gtab[i] = load_group(p.tb.groups + i);
+            for (int i = tc.ttid; i < n_hit; i += TEAM) tc.perm_h[i] = __ldcg(p.tb.perm_hit + i);
+            for (int i = tc.ttid; i < n_low; i += TEAM) tc.perm_l[i] = __ldcg(p.tb.perm_low + i);
+            pl.nB_hit = pl.n_hg * pl.tI;
+            pl.endB = pl.nA + pl.nB_hit + pl.n_lg * pl.tr;
+            pl.nC_sh = pl.td_sh;
+            pl.nC_hit = pl.n_hg * pl.td_hit;
+            nC = pl.nC_sh + pl.nC_hit + pl.n_lg * pl.tb128;
+            pl.endC = pl.endB + nC;
+            pl.endD = pl.endC + dm.T * pl.nb;
+            pl.routed = true;
+            p1_total = (pl.tIs + pl.nB_hit + pl.n_lg * pl.tr) * TW;
+            end = pl.endD;
+            team_sync(tc.team);
+            continue;
         }
-    }
-    // every quantity below is uniform across the team (it comes from team-wide reductions)
-    PROF(tc, 30);
-    if (alive) alive = team_wait_ge(tc, p.sync + SY_ROUTE_DONE, 1, p) ? 1 : 0;
-    PROF(tc, 31);
-    if (alive) {
-        // team-private copy of the group table and the permutations: task set-up never goes to L2 again
-        pl.n_hg = __ldcg(p.tb.hdr + HDR_N_HIT_GROUPS);
-        pl.n_lg = __ldcg(p.tb.hdr + HDR_N_LOW_GROUPS);
-        const int n_hit = __ldcg(p.tb.hdr + HDR_N_HIT), n_low = __ldcg(p.tb.hdr + HDR_N_LOW);
-        for (int i = tc.ttid; i < 1 + pl.n_hg + pl.n_lg; i += TEAM) tc.gtab[i] = load_group(p.tb.groups + i);
-        for (int i = tc.ttid; i < n_hit; i += TEAM) tc.perm_h[i] = __ldcg(p.tb.perm_hit + i);
-        for (int i = tc.ttid; i < n_low; i += TEAM) tc.perm_l[i] = __ldcg(p.tb.perm_low + i);
-        pl.nB_hit = pl.n_hg * pl.tI;
-        pl.endB = pl.nA + pl.nB_hit + pl.n_lg * pl.tr;
-        pl.nC_sh = pl.td_sh;
-        pl.nC_hit = pl.n_hg * pl.td_hit;
-        const int nC = pl.nC_sh + pl.nC_hit + pl.n_lg * pl.tb128;
-        pl.endC = pl.endB + nC;
-        pl.endD = pl.endC + dm.T * pl.nb;
-        pl.routed = true;
-        const int p1_total = (pl.tIs + pl.nB_hit + pl.n_lg * pl.tr) * TW;
-        team_sync(tc.team);
-        bool p2_ready = false;
-        while (id < pl.endD && alive) {
-            const TaskRef t = resolve(pl, id);
-            const int fl = flavour_of(pl, tc, t);
-            if (fl == FL_ACT) id = team_run<NT, EPI_ACT>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
-            else if (fl == FL_Z) id = team_run<NT, EPI_Z>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
-            else if (fl == FL_PART2) id = team_run<(NT <= 2 ? NT : 1), EPI_PART2>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
-            else if (fl == FL_PART) id = team_run<NT, EPI_PART>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
-            else if (fl == FL_LOREB) {
+        const TaskRef t = resolve(pl, id);
+        const int fl = flavour_of(pl, tc, t);
+        if (fl == FL_ACT) id = team_run<NT, EPI_ACT>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        else if (fl == FL_Z) id = team_run<NT, EPI_Z>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        else if (fl == FL_PART2) id = team_run<(NT <= 2 ? NT : 1), EPI_PART2>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        else if (fl == FL_PART) id = team_run<NT, EPI_PART>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        else {
+            if (fl == FL_R1) {
+                PROF(tc, 100 + TK_R1);
+                task_r1(p, smem_raw, tc, id);
+            } else if (fl == FL_R2) {
+                PROF(tc, 100 + TK_R2);
+                task_r2(p, smem_raw, NT, tc);
+            } else if (fl == FL_LOREB) {
                 alive = task_lore_b<NT>(p, tc, t.gi, t.tile, p1_total) ? 1 : 0;
-                id += n_teams;
             } else {
                 if (!p2_ready) {   // combine needs every down-projected row (counted per warp)
                     alive = team_wait_ge(tc, p.sync + SY_P2_DONE, nC * TW, p) ? 1 : 0;
@@ -1080,8 +1078,8 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
                     p2_ready = true;
                 }
                 task_p3(p, tc.ttid, t.tile / pl.nb, t.tile % pl.nb);
-                id += n_teams;
             }
+            id += n_teams;
         }
     }
     // the last team to finish clears the counters for the next launch

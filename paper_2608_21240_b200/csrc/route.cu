@@ -14,6 +14,8 @@ __global__ void route_topk_kernel(const __nv_bfloat16 *__restrict__ h, const __n
     extern __shared__ __align__(16) float smem[];
     float *hs = smem;                   // [TPC][d] fp32 copy of the tokens
     float *lg = smem + (size_t)TPC * d; // [TPC][N]
+    float *sel_val = lg + (size_t)TPC * N;                       // [nwarps][32]
+    int *sel_idx = reinterpret_cast<int *>(sel_val + 32 * 32);   // [nwarps][32]
     const int t0 = blockIdx.x * TPC;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
 
@@ -51,15 +53,19 @@ __global__ void route_topk_kernel(const __nv_bfloat16 *__restrict__ h, const __n
     for (int tt = warp; tt < TPC; tt += nwarps) {
         const int t = t0 + tt;
         if (t >= T) continue;   // warp-uniform
-        warp_topk_gates(lg + tt * N, N, K, norm_topk, lane, idx + (size_t)t * K, gate + (size_t)t * K,
-                        logits_out ? logits_out + (size_t)t * N : nullptr);
+        if (N <= 256)
+            warp_topk_gates(lg + tt * N, N, K, norm_topk, lane, idx + (size_t)t * K, gate + (size_t)t * K,
+                            logits_out ? logits_out + (size_t)t * N : nullptr, sel_idx + warp * 32, sel_val + warp * 32);
+        else
+            warp_topk_gates_rounds(lg + tt * N, N, K, norm_topk, lane, idx + (size_t)t * K, gate + (size_t)t * K,
+                                   logits_out ? logits_out + (size_t)t * N : nullptr);
     }
 }
 
 template <int TPC>
 static int launch_tpc(const Dims &dm, int norm_topk, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router,
                       int32_t *idx, float *gate, float *logits, int threads, cudaStream_t st) {
-    size_t smem = ((size_t)TPC * dm.d + (size_t)TPC * dm.N) * sizeof(float);
+    size_t smem = ((size_t)TPC * dm.d + (size_t)TPC * dm.N + 2 * 32 * 32) * sizeof(float);
     if (smem > 220 * 1024) return -1;
     if (cudaFuncSetAttribute(route_topk_kernel<TPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)

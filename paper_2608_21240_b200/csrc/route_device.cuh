@@ -38,6 +38,7 @@ __device__ __forceinline__ float lane_dot_f32(const __nv_bfloat16 *__restrict__ 
 __device__ __forceinline__ float lane_dot_bf16(const __nv_bfloat16 *__restrict__ w_row, const __nv_bfloat16 *x, int d,
                                                int lane) {
     float s = 0.f;
+#pragma unroll 8
     for (int k = lane * 8; k < d; k += 256) {
         const uint4 u = *reinterpret_cast<const uint4 *>(w_row + k);
         s += slice_dot(u, *reinterpret_cast<const uint4 *>(x + k));
@@ -47,8 +48,60 @@ __device__ __forceinline__ float lane_dot_bf16(const __nv_bfloat16 *__restrict__
 
 // One warp selects the K largest of l[0..N) (ties -> smaller index), writes idx_out[0..K) in
 // decreasing order and the gates: softmax over the winners (norm_topk) or full-softmax values.
-// N <= 1024, K <= 32.  l may live in shared memory; it is not modified.
+// N <= 1024, K <= 32.  l may live in shared memory; it is not modified.  sel_idx / sel_val:
+// K-entry scratch rows in shared memory owned by this warp.
+// The winners are found by ranking: element e has rank #{j : l[j] > l[e] or (l[j] == l[e] and j < e)}
+// and is the rank-th winner when rank < K.  Ranks are a permutation, so every output slot is written
+// exactly once; the result is the same as K rounds of arg-max with ties to the smaller index.
 __device__ __forceinline__ void warp_topk_gates(const float *l, int N, int K, int norm_topk, int lane,
+                                                int32_t *idx_out, float *gate_out, float *logits_out,
+                                                int *sel_idx, float *sel_val) {
+    if (logits_out) {
+#pragma unroll 1
+        for (int e = lane; e < N; e += 32) logits_out[e] = l[e];
+    }
+#pragma unroll 1
+    for (int e = lane; e < N; e += 32) {
+        float v = l[e];
+        if (!(v == v)) v = -INFINITY;   // NaN never wins
+        int rank = 0;
+#pragma unroll 4
+        for (int j = 0; j < N; ++j) {
+            float u = l[j];
+            if (!(u == u)) u = -INFINITY;
+            rank += (u > v) || (u == v && j < e);
+        }
+        if (rank < K) {
+            sel_idx[rank] = e;
+            sel_val[rank] = v;
+        }
+    }
+    __syncwarp();
+    const float m = sel_val[0];
+    float denom = 0.f;
+    if (!norm_topk) {   // full-softmax denominator
+        float s = 0.f;
+#pragma unroll 1
+        for (int e = lane; e < N; e += 32) s += expf(l[e] - m);
+        denom = warp_sum(s);
+    }
+    const float p = (lane < K) ? expf(sel_val[lane] - m) : 0.f;
+    if (norm_topk) {
+        // sum the K numerators in k order on every lane (deterministic, matches the definition)
+        float s = 0.f;
+#pragma unroll 1
+        for (int k = 0; k < K; ++k) s += __shfl_sync(0xffffffffu, p, k);
+        denom = s;
+    }
+    if (lane < K) {
+        idx_out[lane] = sel_idx[lane];
+        gate_out[lane] = p / denom;
+    }
+    __syncwarp();
+}
+
+// The same selection by K rounds of a shuffle arg-max; used when N is large (ranking is O(N^2)).
+__device__ __forceinline__ void warp_topk_gates_rounds(const float *l, int N, int K, int norm_topk, int lane,
                                                 int32_t *idx_out, float *gate_out, float *logits_out) {
     if (logits_out)
 #pragma unroll 1
