@@ -141,6 +141,38 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w /*
                                  int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
                                  float *resid_gate, void *stream);
 
+/* The resident-expert FFN for callers that cannot allocate (the paper has no counterpart: this is
+ * a packaging variant of spice_grouped_expert_ffn, not a step of the method).
+ *
+ * Every other call needs a spice_ctx, and spice_create obtains the workspace with cudaMalloc.  A
+ * host that is not allowed to do that -- a server that gives each component a fixed arena and
+ * forbids driver allocations after start-up, a process whose memory cap works by failing cudaMalloc
+ * -- can use this entry point instead.  It needs no ctx and allocates nothing, on the host or on
+ * the device: the scratch of the kernels (group table, permutation, activations, un-gated rows)
+ * lives in one fixed device array of spice_static_scratch_bytes() = 8 MiB that every GPU loading
+ * the library holds until the process exits.
+ *
+ *   y[t,:] += sum over k with cls[t,k] == HIT of gate[t,k] * E_{slot[t,k]}(h[t,:]),   y [T,d] fp32
+ *
+ * with the arguments of spice_grouped_expert_ffn; cfg is a host struct (only d, n_experts, top_k,
+ * inter, n_slots are used), the GPU used is the calling thread's current device.
+ *   device_status: optional device int32; receives SPICE_OK or SPICE_ERR_BAD_TABLE for this call.
+ * Limits and behaviour:
+ *   - A call needs about T*K*(inter + d)*4 bytes of the array (e.g. 96 (t,k) entries of a
+ *     DeepSeek-V2-Lite-shaped layer: 1.3 MB).  A call that does not fit returns
+ *     SPICE_ERR_WORKSPACE and launches nothing.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, no
+ *     allocation).  Make that first call before any stream capture is begun on the device.
+ *   - All calls on a device share the array and it keeps the previous call's contents; what must
+ *     start from zero is cleared by the call itself.  Two calls that overlap on the GPU (different
+ *     streams, or different threads without ordering) race on it: keep them ordered. */
+spice_status spice_grouped_expert_ffn_static(const spice_layer_cfg *cfg /* host */,
+                                             const spice_layer_weights *w /* host struct */, const spice_bf16 *h,
+                                             const int32_t *idx, const float *gate, const uint8_t *cls,
+                                             const int32_t *slot, int32_t T, float *y, int32_t *device_status,
+                                             void *stream);
+size_t spice_static_scratch_bytes(void);
+
 /* Synchronises the device work issued through ctx so far and returns the sticky device status
  * (SPICE_OK, SPICE_ERR_BAD_TABLE or SPICE_ERR_TIMEOUT) in *code (host), then clears it. */
 spice_status spice_get_device_status(spice_ctx *ctx, int32_t *code /* host */);

@@ -54,8 +54,10 @@ def lib() -> C.CDLL:
         L.spice_version.restype = C.c_int32
         for name in ("spice_create", "spice_destroy", "spice_workspace_bytes", "spice_route_topk",
                      "spice_classify_misses", "spice_grouped_expert_ffn", "spice_lore_surrogate",
-                     "spice_moe_layer_fwd", "spice_get_device_status", "spice_launch_count", "spice_set_option"):
+                     "spice_moe_layer_fwd", "spice_get_device_status", "spice_launch_count", "spice_set_option",
+                     "spice_grouped_expert_ffn_static"):
             getattr(L, name).restype = C.c_int
+        L.spice_static_scratch_bytes.restype = C.c_size_t
         _lib = L
     return _lib
 
@@ -138,6 +140,22 @@ def spice_grouped_expert_ffn(ctx, weights: LayerWeightsC, h, idx, gate, cls, slo
                                           _ptr(gate, torch.float32), _ptr(cls, torch.uint8), _ptr(slot, torch.int32),
                                           C.c_int32(T), _ptr(y, torch.float32), _stream(stream)),
            "spice_grouped_expert_ffn")
+
+
+def spice_grouped_expert_ffn_static(cfg: LayerCfg, weights: LayerWeightsC, h, idx, gate, cls, slot, T, y,
+                                    device_status=None, stream=None) -> None:
+    """The resident-expert FFN without a ctx and without any allocation (for hosts that may not call
+    cudaMalloc): scratch lives in a fixed 8 MiB device array inside the library.  Calls on one GPU must
+    not overlap; the first call on a GPU should precede any stream capture."""
+    _check(lib().spice_grouped_expert_ffn_static(C.byref(cfg), C.byref(weights), _ptr(h, torch.bfloat16),
+                                                 _ptr(idx, torch.int32), _ptr(gate, torch.float32),
+                                                 _ptr(cls, torch.uint8), _ptr(slot, torch.int32), C.c_int32(T),
+                                                 _ptr(y, torch.float32), _ptr(device_status, torch.int32),
+                                                 _stream(stream)), "spice_grouped_expert_ffn_static")
+
+
+def spice_static_scratch_bytes() -> int:
+    return int(lib().spice_static_scratch_bytes())
 
 
 def spice_lore_surrogate(ctx, weights: LayerWeightsC, h, idx, gate, cls, T, y, stream=None) -> None:

@@ -42,6 +42,10 @@ def test_host_side_checks_need_no_device():
     assert lib.spice_route_topk(None, None, None, 1, None, None, None, None) == 1
     assert lib.spice_moe_layer_fwd(None, None, None, None, 1, None, None, None, None, None, None, None, None, None,
                                    None, None, None) == 1
+    assert lib.spice_static_scratch_bytes() == 8 << 20
+    # the entry point without a ctx refuses a call that does not fit its fixed array before anything else
+    assert lib.spice_grouped_expert_ffn_static(C.byref(B.make_cfg(2048, 64, 6, 1408, 2816, 64, 32, 0.6)), None, None,
+                                               None, None, None, None, 4096, None, None, None) == 3
 
 
 def test_binding_refuses_host_tensors():
