@@ -90,6 +90,23 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(win), "window": where}
 
 
+# ----------------------------------------------------------------------------- multi-rank plumbing
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of per-rank timings (the slowest rank defines a step); identity for one rank."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_throughput(units_per_rank_per_step, steps, world, ms_max):
+    """Replicas only: every rank runs the same number of units; the job's rate is all ranks' units over the slowest rank's time."""
+    return world * units_per_rank_per_step * steps / (ms_max * 1e-3)
+
+
 # ----------------------------------------------------------------------------- workload
 def algorithmic_bytes(shape, T, idx, cls):
     """Bytes the method must move for one layer call (bf16 weights read once per distinct expert)."""
@@ -231,16 +248,13 @@ def run_ours(args):
     if sampler:
         sampler.stop()
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev)
     status = layer.device_status()
     if status != 0:
         raise SystemExit(f"device status {status} after the timed region")
 
     if rank == 0:
-        tok_s = world * T * args.steps / (ms * 1e-3)
+        tok_s = whole_job_throughput(T, args.steps, world, ms)
         achieved = total_bytes / (ms * 1e-3) / 1e9
         out = {
             "metric": METRIC, "value": tok_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -260,7 +274,7 @@ def run_ours(args):
                          "kernel": "all launches of spice_moe_layer_fwd (algorithmic bytes of the call / time per call)",
                          "algorithmic_bytes_per_step": total_bytes / args.steps, "peak_source": peaks["source"],
                          "frac_of_nominal_8TBs": achieved / 8000.0},
-            "e2e": {"value": world * T * n_e2e / (ms_e2e * 1e-3), "unit": UNIT,
+            "e2e": {"value": whole_job_throughput(T, n_e2e, world, ms_e2e), "unit": UNIT,
                     "h2d_bytes_per_step": int(h_host.numel() * 2 + conf_host.numel() * 4),
                     "d2h_bytes_per_step": int(y_host.numel() * 2 + 12), "ms_per_step": ms_e2e / n_e2e},
             "gpu_launches": int(launches),

@@ -304,9 +304,11 @@ def cfg_of(s, tau=None, norm_topk=None, conf_per_expert=True) -> LayerCfg:
                     s.tau if tau is None else tau, s.norm_topk if norm_topk is None else norm_topk, conf_per_expert)
 
 
-def upload(wl, dev="cuda") -> LayerWeights:
-    """Copy a workloads.LayerWorkload's weights to the device in the library's layout."""
-    gu, dn = wl.slot_pool_bits()
+def upload(wl, dev="cuda", only=None) -> LayerWeights:
+    """Copy a workloads.LayerWorkload's weights to the device in the library's layout.
+
+    only: experts whose slot contents matter (see LayerWorkload.slot_pool_bits)."""
+    gu, dn = wl.slot_pool_bits(only)
     sg, su, sd = wl.shared()
     A, Bm = wl.lore()
     return LayerWeights(

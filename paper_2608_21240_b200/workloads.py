@@ -190,13 +190,16 @@ class LayerWorkload:
         self.slot_of_expert = a
 
     # ---- slot pool in the device layout: gate rows then up rows; down
-    def slot_pool_bits(self):
-        """bf16 bit patterns: slot_w_gate_up [S,2I,d], slot_w_down [S,d,I] (empty slots zero)."""
+    def slot_pool_bits(self, only=None):
+        """bf16 bit patterns: slot_w_gate_up [S,2I,d], slot_w_down [S,d,I] (empty slots zero).
+
+        only: if given, a set of expert ids; slots of other experts are left zero (they model stale
+        prefetches that no token of the batch uses, so their contents are never read)."""
         s = self.shape
         gu = np.zeros((s.n_slots, 2 * s.inter, s.d), dtype=np.uint16)
         dn = np.zeros((s.n_slots, s.d, s.inter), dtype=np.uint16)
         for sl, e in enumerate(self.expert_of_slot()):
-            if e < 0:
+            if e < 0 or (only is not None and int(e) not in only):
                 continue
             keep = ("expert", int(e)) in self._cache
             g, u, w = self.expert(int(e))

@@ -69,3 +69,53 @@ def run_oracle(wl: W.LayerWorkload, tokens=None, want_full: bool = True, conf=No
 
 def _tiny_shared(s):
     return (np.zeros((1, s.d), np.float32), np.zeros((1, s.d), np.float32), np.zeros((s.d, 1), np.float32))
+
+
+# ------------------------------------------------------------------ config 5: the 26-layer decode stack
+STACK_LAYERS = 26
+STACK_HIT_RATE = 0.7
+
+
+def rms_normalise(x: np.ndarray) -> np.ndarray:
+    """Weight-less RMSNorm (eps 1e-6) between layers: harness glue, not part of the layer call.
+    Needed because 26 un-normalised SwiGLU layers with N(0, 0.02) weights would not keep O(1) inputs."""
+    x = x.astype(np.float64)
+    return x / np.sqrt((x * x).mean(axis=1, keepdims=True) + 1e-6)
+
+
+def stack_layer(l: int, x: np.ndarray, T: int = 8, variant: int = 0):
+    """Inputs and oracle result of layer l of the stack, given the residual stream x [T,d] (fp64).
+
+    Residency is chosen GIVEN the routing: the distinct selected experts are shuffled and made resident until
+    >= 70 % of the T*K picks hit; the other slots hold unselected experts (stale prefetches).  Every miss is
+    low-confidence with probability 1/2 (conf ~ U(0,tau)) else exact (conf ~ U(tau,1)).
+    Returns (workload, oracle result with y and y_full for all tokens, number of redrawn tokens)."""
+    s = W.SHAPES["dsv2lite_stack"]
+    wl = W.make_layer(s, T, variant=variant, layer=l, n_resident=0)
+    wl.h = W.bf16_round(rms_normalise(x).astype(np.float32))
+    redrawn = enforce_margins(wl)
+    pre = oracle.layer(h=wl.h, w_router=wl.w_router, experts={}, shared=_tiny_shared(s),
+                       lore_A=np.zeros((s.n_experts, 1, s.d), np.float32), lore_B=np.zeros((s.n_experts, s.d, 1), np.float32),
+                       resident=np.zeros(s.n_experts, np.uint8), conf=wl.conf, top_k=s.top_k, tau=s.tau, skip_ffn=True)
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([W.BASE_SEED, 5, variant, l, 99])))
+    picks = pre.idx.ravel()
+    selected = rng.permutation(np.unique(picks))
+    resident, hits = [], 0
+    for e in selected:
+        if hits >= STACK_HIT_RATE * picks.size or len(resident) >= s.n_slots:
+            break
+        resident.append(int(e))
+        hits += int((picks == e).sum())
+    others = [int(e) for e in rng.permutation(s.n_experts) if e not in set(selected.tolist())]
+    resident += others[: s.n_slots - len(resident)]
+    soe = np.full(s.n_experts, -1, np.int32)
+    soe[np.array(resident)] = rng.permutation(len(resident)).astype(np.int32)
+    wl.set_residency(soe)
+    tau = np.float32(s.tau)
+    for t in range(T):
+        for e in pre.idx[t]:
+            if soe[e] < 0:
+                lo = rng.random() < 0.5
+                wl.conf[t, e] = np.float32(rng.uniform(0.0, tau * 0.999) if lo else rng.uniform(tau * 1.001, 1.0))
+    ref = run_oracle(wl, want_full=True)
+    return wl, ref, redrawn

@@ -318,3 +318,59 @@ def test_corrupt_slot_table_sets_status_without_faulting():
     assert (cls[ref.idx == e_bad] == B.MISS_EXACT).all()
     assert torch.isfinite(out.y.float()).all()
     L.close()
+
+
+def test_config4_prefill_4096_tokens_skewed_loads_sampled_against_oracle():
+    """DeepSeek-V2-Lite-shaped layer, 4096 tokens, Zipf-skewed router, every expert resident.
+    Routing / classification are compared for all tokens, outputs for a sample the oracle can afford."""
+    wl = _layer_case("dsv2lite_prefill", 4096, zipf=True)
+    s = wl.shape
+    tokens = sorted(np.random.default_rng(4).choice(4096, size=24, replace=False).tolist())
+    ref = run_oracle(wl, tokens=tokens, want_full=False)
+    load = np.bincount(ref.idx.ravel(), minlength=s.n_experts)
+    assert load.max() > 8 * max(1, load.min())            # loads really are imbalanced
+    assert ref.counts.tolist() == [4096 * s.top_k, 0, 0]
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    w = upload(wl)
+    out = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
+    torch.cuda.synchronize()
+    check_routing(out, ref, wl.T, s.top_k)
+    y = out.y.float().cpu().numpy()
+    assert np.isfinite(y).all()
+    err, bound = y_close(y[np.asarray(tokens)], ref.y)
+    assert err <= bound, (err, bound)
+    assert L.device_status() == 0
+    L.close()
+
+
+def test_config5_decode_stack_teacher_forced_per_layer():
+    """26 layers of DeepSeek-V2-Lite shape, batch 8, slot cache of 26 experts with ~70 % hits.  Each GPU layer
+    call gets the oracle chain's input for that layer (bf16-level output error must not be allowed to flip later
+    routing decisions), the exact-recovery outputs as y_cpu_residual, and the residual stream to update."""
+    from tests._cases import STACK_LAYERS, stack_layer
+    s = W.SHAPES["dsv2lite_stack"]
+    T = 8
+    x = W.make_layer(s, T, variant=55).h.astype(np.float64)          # embedding-like start of the stream
+    L = B.SpiceLayer(cfg_of(s), T)
+    tot = np.zeros(3, np.int64)
+    for l in range(STACK_LAYERS):
+        wl, ref, _ = stack_layer(l, x, T)
+        need = {int(e) for e, c in zip(ref.idx.ravel(), ref.cls.ravel()) if c == oracle.HIT}
+        w = upload(wl, only=need)
+        y_cpu = torch.from_numpy((ref.y_full - ref.y).astype(np.float32)).cuda()
+        xr = bf16_tensor(W.bf16_round(x.astype(np.float32)))
+        out = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda(), y_cpu_residual=y_cpu, x_resid=xr)
+        torch.cuda.synchronize()
+        check_routing(out, ref, T, s.top_k)
+        err, bound = y_close(out.y.float().cpu().numpy(), ref.y_full)
+        assert err <= bound, (l, err, bound)
+        x_next = x + ref.y_full
+        errx = np.abs(xr.float().cpu().numpy() - x_next).max()
+        assert errx <= 1e-2 * np.abs(x_next).max() + 1e-3 + 2.0 ** -8 * np.abs(x_next).max()   # + bf16 rounding of x
+        tot += ref.counts
+        x = x_next
+        del w
+    hit_rate = tot[0] / tot.sum()
+    assert 0.6 <= hit_rate <= 0.85 and tot[1] > 0 and tot[2] > 0
+    assert L.device_status() == 0
+    L.close()
