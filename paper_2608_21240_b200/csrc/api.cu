@@ -24,6 +24,8 @@ struct spice_ctx {
     int32_t sync_words;
     int32_t decode_tokens;          // largest T the decode buffers were sized for (0: path unavailable)
     int n_sms, max_smem_optin;
+    TcBuffers tcb;                  // tensor-core path buffers (large batches)
+    bool tc_ok;
     int64_t opt_path;               // 0 auto, 1 general kernels only
     int64_t opt_spin_limit;
     int64_t launches;
@@ -74,6 +76,15 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->z16 = cv.take<__nv_bfloat16>(nd * g.lore_rank);
     c->sync_words = SY_GROUP0 + 1 + g.n_slots + g.n_experts;
     c->sync = cv.take<int32_t>(c->sync_words);
+    if (Tm > 32) {   // large batches: buffers of the tensor-core path
+        c->tcb.x_perm = cv.take<__nv_bfloat16>(n * g.d);
+        c->tcb.act16 = cv.take<__nv_bfloat16>(n * g.inter);
+        c->tcb.act_shared16 = cv.take<__nv_bfloat16>(Tm * g.inter_shared);
+        c->tcb.mtiles = cv.take<MTile>(n / 128 + g.n_slots + 1);
+        c->tcb.mtiles_shared = cv.take<MTile>(Tm / 128 + 1);
+        c->tcb.n_mtiles = cv.take<int32_t>(4);
+        c->tcb.n_mtiles_shared = cv.take<int32_t>(4);
+    }
     *total = (cv.off + 255) & ~size_t(255);
 }
 
@@ -162,6 +173,8 @@ spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg
         return SPICE_ERR_CUDA;
     }
     c->decode_tokens = (coop && decode_prepare(c->max_smem_optin) == 0) ? (max_tokens < 32 ? max_tokens : 32) : 0;
+    c->tcb = TcBuffers{};
+    c->tc_ok = max_tokens > 32 && tc_available() && tc_prepare() == 0;
     carve(c, nullptr, &c->ws_bytes);
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -359,9 +372,16 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
                                  ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st));
-    SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED | KIND_HIT, *w, hb, ctx->tb, st));
-    SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
-    SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_HIT | KIND_LOW, *w, ctx->tb, st));
+    if (ctx->opt_path == 0 && ctx->tc_ok && T > 32 && tc_shape_ok(dm)) {
+        // large batch: exact experts and shared expert on the tensor cores, LoRE on the general kernels
+        SPICE_LAUNCH(launch_tc_expert_path(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
+        SPICE_LAUNCH(launch_down(dm, KIND_LOW, *w, ctx->tb, st));
+    } else {
+        SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED | KIND_HIT, *w, hb, ctx->tb, st));
+        SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
+        SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_HIT | KIND_LOW, *w, ctx->tb, st));
+    }
     CombineArgs ca{KIND_SHARED | KIND_HIT | KIND_LOW, 0, gate, cls, nullptr, reinterpret_cast<__nv_bfloat16 *>(y),
                    y_cpu_residual, reinterpret_cast<__nv_bfloat16 *>(x_resid)};
     SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));

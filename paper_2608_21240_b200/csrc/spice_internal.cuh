@@ -110,6 +110,25 @@ bool decode_supported(const Dims &dm, size_t max_smem);
 int decode_prepare(int max_smem_optin);
 int launch_decode(const DecodeParams &p, int n_ctas, cudaStream_t st);
 
+// ---- tensor-core path for large batches (tc_gemm.cu)
+// One m-tile of the grouped problem: rows [row0, row0+rows) of the gathered activation buffer, all of
+// which use the weights of slot `slot`.
+struct MTile {
+    int32_t slot, row0, rows, pad;
+};
+struct TcBuffers {
+    __nv_bfloat16 *x_perm;        // [Tm*K, d]   tokens gathered in perm_hit order
+    __nv_bfloat16 *act16;         // [Tm*K, I]   silu(gate)*up of HIT entries
+    __nv_bfloat16 *act_shared16;  // [Tm, I_s]
+    MTile *mtiles, *mtiles_shared;
+    int32_t *n_mtiles, *n_mtiles_shared;
+};
+bool tc_available();
+int tc_prepare();
+bool tc_shape_ok(const Dims &dm);
+int launch_tc_expert_path(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
+                          const TcBuffers &b, int n_sms, cudaStream_t st);
+
 // ---- small device helpers
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

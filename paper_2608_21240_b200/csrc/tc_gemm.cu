@@ -1,0 +1,457 @@
+// Grouped expert GEMMs for large batches on the 5th-generation tensor cores (tcgen05 + TMEM), fed
+// by TMA.  This is the compute-bound regime of the exact resident experts E_e of Sec. 4.2 and of
+// the shared expert S of Sec. 2.1: once an expert sees hundreds of tokens the contraction is a
+// dense GEMM (arithmetic intensity ~330 FLOP/B at 4096 tokens of a DeepSeek-V2-Lite-shaped layer).
+//
+//   MODE_ACT : act[row, i]        = silu(X W_g^T)[row,i] * (X W_u^T)[row,i]      (bf16 out)
+//   MODE_OUT : out[orow(row), j]  = (act W_d^T)[row, j]                          (fp32 out)
+//
+// C[M,N] = A[M,K] B[N,K]^T with both operands K-major.  A rows are tokens (gathered so that every
+// group is a contiguous row range), B rows are weight rows.  One persistent CTA per SM:
+//   warp 0   TMA producer: 128 x 64 A box + 256 rows of B (gate box + up box, or one 256-row box)
+//            per k-block into a 4-stage shared-memory ring (128-byte swizzle), mbarrier complete_tx
+//   warp 1   issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) on the staged tiles; the
+//            accumulator (256 TMEM columns) is double-buffered so the epilogue of tile i overlaps
+//            the main loop of tile i+1; tcgen05.commit releases ring stages / publishes accumulators
+//   warps 2-5 epilogue: tcgen05.ld 32 lanes x 32 columns at a time, SwiGLU or plain, masked stores
+// Every wait is bounded: on expiry the CTA records SPICE_ERR_TIMEOUT, stops, drains its own copies
+// in flight (again bounded), frees its TMEM and returns.  No load uses cluster multicast.
+#include <cuda.h>
+
+#include "spice_internal.cuh"
+
+namespace spice {
+
+namespace {
+
+constexpr int BM = 128, BK = 64, BN2 = 256;          // CTA tile: 128 rows x 256 accumulator columns
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN2 * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int TC_THREADS = 192;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;   // polls per wait before the CTA gives up
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t a, int n) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a), "r"(n));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t a, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(a), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t a) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t a, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok)
+                 : "r"(a), "r"(parity)
+                 : "memory");
+    return ok != 0;
+}
+// bounded wait; false when the limit expired or another role already gave up
+__device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try(a, parity)) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t mbar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(mbar)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t mbar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(mbar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,"
+        "%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 B, 8-row groups 1024 B apart
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);        // start address
+    d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major) = 1
+    d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset: 8 rows x 128 B
+    d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                         // SWIZZLE_128B
+    return d;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN2 >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+struct TcShared {
+    alignas(8) unsigned long long full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+}  // namespace
+
+struct TcGemmArgs {
+    const MTile *mtiles;        // device
+    const int32_t *n_mtiles;    // device scalar
+    int32_t n_ntiles;           // column tiles per m-tile
+    int32_t K;                  // reduction length
+    int32_t b_rows_per_slot;    // rows of B per slot (2I for gate/up, d for down)
+    int32_t b_second_off;       // MODE_ACT: row offset of the second (up) block inside a slot, = I
+    int32_t n_cols;             // valid output columns (I or d)
+    // epilogue
+    __nv_bfloat16 *out16;       // MODE_ACT: [rows, ld]
+    float *out32;               // MODE_OUT: [orows, ld]
+    const int32_t *row_map;     // MODE_OUT: output row of A row r (entry id), or null for identity
+    int32_t ld;
+    int32_t *status;
+};
+
+template <int MODE>   // 0 = gate/up + SwiGLU, 1 = plain
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                        const __grid_constant__ CUtensorMap map_b,
+                                                                        const TcGemmArgs g) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    // ring first (1024-byte aligned tiles), control block after it
+    unsigned char *ring = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    TcShared *sh = reinterpret_cast<TcShared *>(ring + STAGES * STAGE_BYTES);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &sh->abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh->tmem_full[b]), 1);
+            mbar_init(smem_u32(&sh->tmem_empty[b]), 4);
+        }
+        sh->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // TMEM: all 512 columns (two 256-column accumulators)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    const int n_mt = *g.n_mtiles;
+    const int n_tiles = n_mt * g.n_ntiles;
+    const int kblocks = (g.K + BK - 1) / BK;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (one lane)
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const MTile mt = g.mtiles[tile / g.n_ntiles];
+                const int nt = tile % g.n_ntiles;
+                const int b_row = mt.slot * g.b_rows_per_slot + nt * (MODE == 0 ? 128 : BN2);
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(smem_u32(&sh->empty[s]), ((it / STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t full = smem_u32(&sh->full[s]);
+                    const uint32_t dst = smem_u32(ring + s * STAGE_BYTES);
+                    mbar_expect_tx(full, STAGE_BYTES);
+                    tma_load_2d(dst, &map_a, kb * BK, mt.row0, full);
+                    if (MODE == 0) {
+                        tma_load_2d(dst + A_BYTES, &map_b, kb * BK, b_row, full);                              // gate rows
+                        tma_load_2d(dst + A_BYTES + B_BYTES / 2, &map_b, kb * BK, b_row + g.b_second_off, full);  // up rows
+                    } else {
+                        tma_load_2d(dst + A_BYTES, &map_b, kb * BK, b_row, full);
+                        tma_load_2d(dst + A_BYTES + B_BYTES / 2, &map_b, kb * BK, b_row + 128, full);
+                    }
+                }
+            }
+            // drain: every stage that was armed must have landed before the CTA may end
+            for (uint32_t j = (it > STAGES ? it - STAGES : 0); j < it; ++j)
+                mbar_wait(smem_u32(&sh->full[j % STAGES]), (j / STAGES) & 1, abort_flag);
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (one lane)
+        if (lane == 0) {
+            uint32_t it = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
+                const int buf = tcount & 1;
+                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN2;
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    if (!mbar_wait(smem_u32(&sh->full[s]), (it / STAGES) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a0 = smem_u32(ring + s * STAGE_BYTES), b0 = a0 + A_BYTES;
+                    const uint64_t da = make_desc(a0), db = make_desc(b0);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
+                        tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | k) ? 1u : 0u);
+                    tc_commit(smem_u32(&sh->empty[s]));   // stage free once these MMAs have read it
+                }
+                if (ok) tc_commit(smem_u32(&sh->tmem_full[buf]));
+            }
+        }
+    } else {
+        // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 = rows of the tile
+        const int q = warp & 3;
+        uint32_t tcount = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tcount) {
+            const int buf = tcount & 1;
+            const MTile mt = g.mtiles[tile / g.n_ntiles];
+            const int nt = tile % g.n_ntiles;
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait(smem_u32(&sh->tmem_full[buf]), (tcount >> 1) & 1, abort_flag);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            tc_fence_after();
+            const int r = q * 32 + lane;                       // row inside the tile
+            const bool row_ok = r < mt.rows;
+            const uint32_t t0 = tmem_base + buf * BN2 + ((uint32_t)(q * 32) << 16);
+            if (MODE == 0) {
+                const int col0 = nt * 128;
+                __nv_bfloat16 *orow = g.out16 + (size_t)(mt.row0 + r) * g.ld;
+#pragma unroll 1
+                for (int c = 0; c < 128; c += 32) {
+                    uint32_t gv[32], uv[32];
+                    tc_ld32(t0 + c, gv);
+                    tc_ld32(t0 + 128 + c, uv);
+                    tc_wait_ld();
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            const int col = col0 + c + j;
+                            const float a0 = silu_f(__uint_as_float(gv[j])) * __uint_as_float(uv[j]);
+                            const float a1 = silu_f(__uint_as_float(gv[j + 1])) * __uint_as_float(uv[j + 1]);
+                            if (col + 1 < g.n_cols) {
+                                __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
+                                *reinterpret_cast<__nv_bfloat162 *>(orow + col) = pk;
+                            } else if (col < g.n_cols) {
+                                orow[col] = __float2bfloat16(a0);
+                            }
+                        }
+                    }
+                }
+            } else {
+                const int col0 = nt * BN2;
+                const int out_r = row_ok ? (g.row_map ? g.row_map[mt.row0 + r] : mt.row0 + r) : 0;
+                float *orow = g.out32 + (size_t)out_r * g.ld;
+#pragma unroll 1
+                for (int c = 0; c < BN2; c += 32) {
+                    uint32_t v[32];
+                    tc_ld32(t0 + c, v);
+                    tc_wait_ld();
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const int col = col0 + c + j;
+                            if (col + 3 < g.n_cols) {
+                                *reinterpret_cast<float4 *>(orow + col) =
+                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                                                __uint_as_float(v[j + 3]));
+                            } else {
+                                for (int e = 0; e < 4; ++e)
+                                    if (col + e < g.n_cols) orow[col + e] = __uint_as_float(v[j + e]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh->abort_flag) atomicMax(g.status, (int)SPICE_ERR_TIMEOUT);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// helpers around the GEMMs
+
+// x_perm[p, :] = h[perm_hit[p] / K, :]  (rows of one slot become contiguous)
+__global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16 *__restrict__ h, const int32_t *__restrict__ perm,
+                                                          const int32_t *__restrict__ hdr, int K, int d,
+                                                          __nv_bfloat16 *__restrict__ out) {
+    const int n_hit = hdr[HDR_N_HIT];
+    const int vec = d >> 3;
+    for (int p = blockIdx.x; p < n_hit; p += gridDim.x) {
+        const int t = perm[p] / K;
+        const uint4 *src = reinterpret_cast<const uint4 *>(h + (size_t)t * d);
+        uint4 *dst = reinterpret_cast<uint4 *>(out + (size_t)p * d);
+        for (int v = threadIdx.x; v < vec; v += blockDim.x) dst[v] = src[v];
+    }
+}
+
+// m-tiles of the hit groups (group list order), 128 rows each
+__global__ void build_mtiles_kernel(const GroupDesc *__restrict__ groups, const int32_t *__restrict__ hdr, MTile *mtiles,
+                                    int32_t *n_mtiles) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const int n_hg = hdr[HDR_N_HIT_GROUPS];
+    int n = 0;
+    for (int gi = 1; gi <= n_hg; ++gi) {
+        const GroupDesc grp = groups[gi];
+        for (int r = 0; r < grp.m; r += BM) mtiles[n++] = MTile{grp.id, grp.off + r, min(BM, grp.m - r), 0};
+    }
+    *n_mtiles = n;
+}
+
+// m-tiles of the shared expert: all T rows, "slot" 0
+__global__ void build_shared_mtiles_kernel(int T, MTile *mtiles, int32_t *n_mtiles) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int n = 0;
+    for (int r = 0; r < T; r += BM) mtiles[n++] = MTile{0, r, min(BM, T - r), 0};
+    *n_mtiles = n;
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows, cols] (cols contiguous), box = box_rows x 64 columns, 128-byte swizzle, zero fill
+bool make_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t TC_SMEM = STAGES * STAGE_BYTES + sizeof(TcShared) + 1024;
+
+}  // namespace
+
+bool tc_available() { return encode_fn() != nullptr; }
+
+int tc_prepare() {
+    if (cudaFuncSetAttribute(tc_grouped_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM) != cudaSuccess)
+        return -1;
+    if (cudaFuncSetAttribute(tc_grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM) != cudaSuccess)
+        return -1;
+    return 0;
+}
+
+bool tc_shape_ok(const Dims &dm) {
+    // TMA: row pitches must be multiples of 16 bytes (dims are multiples of 8: yes); nothing else is required,
+    // partial tiles are zero-filled on load and masked on store
+    return dm.d % 8 == 0 && dm.I % 8 == 0 && dm.Is % 8 == 0;
+}
+
+// The exact-expert part of a large batch: gather, grouped gate/up + SwiGLU, grouped down, for the hit groups and
+// for the shared expert.  Results land in tb.part (by entry id) and tb.part_shared (by token) as fp32, exactly
+// where the general kernels put them, so the LoRE path and the combine kernel are shared with the general path.
+int launch_tc_expert_path(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
+                          const TcBuffers &b, int n_sms, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    int launches = 0;
+    const size_t cap = (size_t)dm.T * dm.K;
+    TcGemmArgs g{};
+    g.status = tb.status;
+    // ---- routed experts
+    build_mtiles_kernel<<<1, 32, 0, st>>>(tb.groups, tb.hdr, b.mtiles, b.n_mtiles);
+    gather_rows_kernel<<<n_sms * 4, 256, 0, st>>>(h, tb.perm_hit, tb.hdr, dm.K, dm.d, b.x_perm);
+    launches += 2;
+    if (!make_map(&ma, b.x_perm, cap, dm.d, BM) || !make_map(&mb, w.slot_w_gate_up, (uint64_t)dm.S * 2 * dm.I, dm.d, 128))
+        return -1;
+    g.mtiles = b.mtiles;
+    g.n_mtiles = b.n_mtiles;
+    g.n_ntiles = (dm.I + 127) / 128;
+    g.K = dm.d;
+    g.b_rows_per_slot = 2 * dm.I;
+    g.b_second_off = dm.I;
+    g.n_cols = dm.I;
+    g.out16 = b.act16;
+    g.ld = dm.I;
+    tc_grouped_gemm_kernel<0><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    ++launches;
+    if (!make_map(&ma, b.act16, cap, dm.I, BM) || !make_map(&mb, w.slot_w_down, (uint64_t)dm.S * dm.d, dm.I, 128)) return -1;
+    g.n_ntiles = (dm.d + BN2 - 1) / BN2;
+    g.K = dm.I;
+    g.b_rows_per_slot = dm.d;
+    g.b_second_off = 0;
+    g.n_cols = dm.d;
+    g.out16 = nullptr;
+    g.out32 = tb.part;
+    g.row_map = tb.perm_hit;
+    g.ld = dm.d;
+    tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    ++launches;
+    // ---- shared expert: one group of all T tokens, A is h itself
+    build_shared_mtiles_kernel<<<1, 32, 0, st>>>(dm.T, b.mtiles_shared, b.n_mtiles_shared);
+    ++launches;
+    if (!make_map(&ma, h, dm.T, dm.d, BM) || !make_map(&mb, w.shared_w_gate_up, (uint64_t)2 * dm.Is, dm.d, 128)) return -1;
+    g.mtiles = b.mtiles_shared;
+    g.n_mtiles = b.n_mtiles_shared;
+    g.n_ntiles = (dm.Is + 127) / 128;
+    g.K = dm.d;
+    g.b_rows_per_slot = 2 * dm.Is;
+    g.b_second_off = dm.Is;
+    g.n_cols = dm.Is;
+    g.out16 = b.act_shared16;
+    g.out32 = nullptr;
+    g.row_map = nullptr;
+    g.ld = dm.Is;
+    tc_grouped_gemm_kernel<0><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    ++launches;
+    if (!make_map(&ma, b.act_shared16, dm.T, dm.Is, BM) || !make_map(&mb, w.shared_w_down, dm.d, dm.Is, 128)) return -1;
+    g.n_ntiles = (dm.d + BN2 - 1) / BN2;
+    g.K = dm.Is;
+    g.b_rows_per_slot = dm.d;
+    g.b_second_off = 0;
+    g.n_cols = dm.d;
+    g.out16 = nullptr;
+    g.out32 = tb.part_shared;
+    g.ld = dm.d;
+    tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    ++launches;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+}  // namespace spice

@@ -374,3 +374,27 @@ def test_config5_decode_stack_teacher_forced_per_layer():
     assert 0.6 <= hit_rate <= 0.85 and tot[1] > 0 and tot[2] > 0
     assert L.device_status() == 0
     L.close()
+
+
+@pytest.mark.parametrize("T,dims", [
+    (300, {}),                                                                   # tiny shape, several tokens per expert
+    (200, dict(d=264, n_experts=10, top_k=3, inter=200, inter_shared=328, lore_rank=24, n_slots=4)),   # ragged tiles
+    (1000, dict(d=512, n_experts=16, top_k=4, inter=384, inter_shared=768, lore_rank=32, n_slots=9)),
+])
+def test_tensor_core_path_matches_oracle_and_general_path(T, dims):
+    """Batches beyond the decode kernel run the exact experts on the tcgen05 grouped GEMM; same answers as
+    the oracle (sampled tokens) and as the general-shape kernels (all tokens)."""
+    s = W.scaled_shape(W.SHAPES["tiny"], **dims) if dims else W.SHAPES["tiny"]
+    wl = _layer_case(s, T, variant=31)
+    tokens = sorted(np.random.default_rng(T).choice(T, size=16, replace=False).tolist())
+    L, w, out, ref = _fwd_and_check(wl, tokens=tokens, want_full=False)
+    assert ref.counts[0] > 0 and ref.counts[2] > 0
+    n_tc = L.launch_count()
+    L.set_option(B.OPT_PATH, 1)
+    gen = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
+    torch.cuda.synchronize()
+    assert torch.equal(gen.idx, out.idx) and torch.equal(gen.cls, out.cls)
+    diff = (gen.y.float() - out.y.float()).abs().max().item()
+    assert diff <= 1e-2 * gen.y.float().abs().max().item() + 1e-3, diff
+    assert L.device_status() == 0 and n_tc > 0
+    L.close()
