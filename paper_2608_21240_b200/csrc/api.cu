@@ -76,7 +76,7 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->z16 = cv.take<__nv_bfloat16>(nd * g.lore_rank);
     c->sync_words = SY_GROUP0 + 1 + g.n_slots + g.n_experts;
     c->sync = cv.take<int32_t>(c->sync_words);
-    if (Tm > 32) {   // large batches: buffers of the tensor-core path
+    {   // buffers of the tensor-core path
         c->tcb.x_perm = cv.take<__nv_bfloat16>(n * g.d);
         c->tcb.act16 = cv.take<__nv_bfloat16>(n * g.inter);
         c->tcb.act_shared16 = cv.take<__nv_bfloat16>(Tm * g.inter_shared);
@@ -174,7 +174,7 @@ spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg
     }
     c->decode_tokens = (coop && decode_prepare(c->max_smem_optin) == 0) ? (max_tokens < 32 ? max_tokens : 32) : 0;
     c->tcb = TcBuffers{};
-    c->tc_ok = max_tokens > 32 && tc_available() && tc_prepare() == 0;
+    c->tc_ok = tc_available() && tc_prepare() == 0;
     carve(c, nullptr, &c->ws_bytes);
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -372,8 +372,9 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
                                  ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st));
-    if (ctx->opt_path == 0 && ctx->tc_ok && T > 32 && tc_shape_ok(dm)) {
-        // large batch: exact experts and shared expert on the tensor cores, LoRE on the general kernels
+    if (ctx->opt_path == 0 && ctx->tc_ok && tc_shape_ok(dm)) {
+        // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
+        // LoRE on the general kernels
         SPICE_LAUNCH(launch_tc_expert_path(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
         SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
         SPICE_LAUNCH(launch_down(dm, KIND_LOW, *w, ctx->tb, st));

@@ -58,7 +58,8 @@ __global__ void __launch_bounds__(GT) rows_from_h_kernel(Dims dm, int kind_mask,
                                                          const __nv_bfloat16 *__restrict__ h, Tables tb) {
     __shared__ __align__(16) float xs[MT * KC];
     __shared__ const void *rows[MT];
-    const int g = blockIdx.y;
+    // when only the low-confidence groups are wanted they are addressed directly (they follow the hit groups)
+    const int g = blockIdx.y + (kind_mask == KIND_LOW ? 1 + tb.hdr[HDR_N_HIT_GROUPS] : 0);
     if (g >= tb.hdr[HDR_N_GROUPS]) return;
     const GroupDesc grp = tb.groups[g];
     if (!(grp.kind & kind_mask)) return;
@@ -141,7 +142,7 @@ __global__ void __launch_bounds__(GT) down_kernel(Dims dm, int kind_mask, spice_
     __shared__ __align__(16) float xs[MT * KC];
     __shared__ const void *rows[MT];
     __shared__ float *outs[MT];
-    const int g = blockIdx.y;
+    const int g = blockIdx.y + (kind_mask == KIND_LOW ? 1 + tb.hdr[HDR_N_HIT_GROUPS] : 0);
     if (g >= tb.hdr[HDR_N_GROUPS]) return;
     const GroupDesc grp = tb.groups[g];
     if (!(grp.kind & kind_mask)) return;
@@ -261,13 +262,13 @@ int launch_gateup(const Dims &dm, int kind_mask, const spice_layer_weights &w, c
 
 int launch_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
                   cudaStream_t st) {
-    dim3 grid((dm.r + GW - 1) / GW, max_groups(dm));
+    dim3 grid((dm.r + GW - 1) / GW, min(dm.N, dm.T * dm.K));
     rows_from_h_kernel<1><<<grid, GT, 0, st>>>(dm, KIND_LOW, w, h, tb);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 int launch_down(const Dims &dm, int kind_mask, const spice_layer_weights &w, const Tables &tb, cudaStream_t st) {
-    dim3 grid((dm.d + GW - 1) / GW, max_groups(dm));
+    dim3 grid((dm.d + GW - 1) / GW, kind_mask == KIND_LOW ? min(dm.N, dm.T * dm.K) : max_groups(dm));
     down_kernel<<<grid, GT, 0, st>>>(dm, kind_mask, w, tb);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

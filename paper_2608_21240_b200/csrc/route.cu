@@ -1,7 +1,7 @@
 // Router logits, Top-K and gate scores (Eq. 1 of the paper; "selected experts and their gate
-// scores", Sec. 4.2).  One CTA owns TPC tokens: its warps share the router rows (each warp takes
-// experts e = warp, warp+nwarps, ...), logits are accumulated in fp32 and parked in shared memory,
-// then one warp per token does K rounds of a shuffle arg-max (ties -> smaller expert index).
+// scores", Sec. 4.2).  One CTA owns TPC tokens: its warps share the router rows (each warp takes a
+// few experts at a time), logits are accumulated in fp32 in a fixed order and parked in shared
+// memory, then one warp per token selects the K winners (ties -> smaller expert index).
 #include "route_device.cuh"
 #include "spice_internal.cuh"
 
@@ -30,23 +30,35 @@ __global__ void route_topk_kernel(const __nv_bfloat16 *__restrict__ h, const __n
     }
     __syncthreads();
 
-    for (int e = warp; e < N; e += nwarps) {
-        float acc[TPC];
+    // Each warp takes EPW experts at a time so that every token slice read from shared memory feeds
+    // EPW fmaf chains; per (expert, token) the arithmetic is exactly lane_dot_f32's.
+    constexpr int EPW = (TPC >= 4) ? 4 : 1;
+    for (int e0 = warp * EPW; e0 < N; e0 += nwarps * EPW) {
+        float acc[EPW][TPC];
 #pragma unroll
-        for (int tt = 0; tt < TPC; ++tt) acc[tt] = 0.f;
-        const __nv_bfloat16 *row = wr + (size_t)e * d;
+        for (int ee = 0; ee < EPW; ++ee)
+#pragma unroll
+            for (int tt = 0; tt < TPC; ++tt) acc[ee][tt] = 0.f;
         for (int k = lane * 8; k < d; k += 256) {
-            const uint4 u = *reinterpret_cast<const uint4 *>(row + k);
+            uint4 u[EPW];
 #pragma unroll
-            for (int tt = 0; tt < TPC; ++tt)
-                acc[tt] += slice_dot(u, *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k),
-                                     *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k + 4));
+            for (int ee = 0; ee < EPW; ++ee)
+                u[ee] = (e0 + ee < N) ? *reinterpret_cast<const uint4 *>(wr + (size_t)(e0 + ee) * d + k) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int tt = 0; tt < TPC; ++tt) {
+                const float4 a = *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k);
+                const float4 b = *reinterpret_cast<const float4 *>(hs + (size_t)tt * d + k + 4);
+#pragma unroll
+                for (int ee = 0; ee < EPW; ++ee) acc[ee][tt] += slice_dot(u[ee], a, b);
+            }
         }
 #pragma unroll
-        for (int tt = 0; tt < TPC; ++tt) {
-            float s = warp_sum(acc[tt]);
-            if (lane == 0) lg[tt * N + e] = s;
-        }
+        for (int ee = 0; ee < EPW; ++ee)
+#pragma unroll
+            for (int tt = 0; tt < TPC; ++tt) {
+                const float s = warp_sum(acc[ee][tt]);
+                if (lane == 0 && e0 + ee < N) lg[tt * N + e0 + ee] = s;
+            }
     }
     __syncthreads();
 

@@ -308,17 +308,29 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16 *_
     }
 }
 
-// m-tiles of the hit groups (group list order), 128 rows each
+// m-tiles of the hit groups (group list order), 128 rows each; one warp, a group per lane
 __global__ void build_mtiles_kernel(const GroupDesc *__restrict__ groups, const int32_t *__restrict__ hdr, MTile *mtiles,
                                     int32_t *n_mtiles) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    if (blockIdx.x != 0 || threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
     const int n_hg = hdr[HDR_N_HIT_GROUPS];
-    int n = 0;
-    for (int gi = 1; gi <= n_hg; ++gi) {
-        const GroupDesc grp = groups[gi];
-        for (int r = 0; r < grp.m; r += BM) mtiles[n++] = MTile{grp.id, grp.off + r, min(BM, grp.m - r), 0};
+    int base = 0;
+    for (int g0 = 0; g0 < n_hg; g0 += 32) {
+        const int gi = 1 + g0 + lane;
+        GroupDesc grp{0, 0, 0, 0};
+        if (g0 + lane < n_hg) grp = groups[gi];
+        const int nt = (grp.m + BM - 1) / BM;
+        int inc = nt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        const int first = base + inc - nt;
+        for (int j = 0; j < nt; ++j) mtiles[first + j] = MTile{grp.id, grp.off + j * BM, min(BM, grp.m - j * BM), 0};
+        base += __shfl_sync(0xffffffffu, inc, 31);
     }
-    *n_mtiles = n;
+    if (lane == 0) *n_mtiles = base;
 }
 
 // m-tiles of the shared expert: all T rows, "slot" 0
