@@ -26,7 +26,7 @@ struct spice_ctx {
     int n_sms, max_smem_optin;
     TcBuffers tcb;                  // tensor-core path buffers (large batches)
     bool tc_ok;
-    int64_t opt_path;               // 0 auto, 1 general kernels only
+    int64_t opt_path;               // 0 auto, 1 general kernels only, 2 never the fused decode kernel
     int64_t opt_spin_limit;
     int64_t launches;
 };
@@ -69,7 +69,7 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->ws_gate = cv.take<float>(n);
     c->ws_cls = cv.take<uint8_t>(n);
     c->y32 = cv.take<float>(Tm * g.d);
-    const size_t Td = Tm < 32 ? Tm : 32, nd = Td * K;
+    const size_t Td = Tm < 16 ? Tm : 16, nd = Td * K;
     c->logits = cv.take<float>(Td * g.n_experts);
     c->act_hit16 = cv.take<__nv_bfloat16>(nd * g.inter);
     c->act_shared16 = cv.take<__nv_bfloat16>(Td * g.inter_shared);
@@ -172,7 +172,7 @@ spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg
         delete c;
         return SPICE_ERR_CUDA;
     }
-    c->decode_tokens = (coop && decode_prepare(c->max_smem_optin) == 0) ? (max_tokens < 32 ? max_tokens : 32) : 0;
+    c->decode_tokens = (coop && decode_prepare(c->max_smem_optin) == 0) ? (max_tokens < 16 ? max_tokens : 16) : 0;
     c->tcb = TcBuffers{};
     c->tc_ok = tc_available() && tc_prepare() == 0;
     carve(c, nullptr, &c->ws_bytes);
@@ -229,7 +229,7 @@ spice_status spice_set_option(spice_ctx *ctx, int32_t option, int64_t value) {
     if (!ctx) return SPICE_ERR_INVALID_ARG;
     switch (option) {
         case SPICE_OPT_PATH:
-            if (value != 0 && value != 1) return SPICE_ERR_INVALID_ARG;
+            if (value < 0 || value > 2) return SPICE_ERR_INVALID_ARG;
             ctx->opt_path = value;
             return SPICE_OK;
         case SPICE_OPT_SPIN_LIMIT:
@@ -372,7 +372,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
                                  ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st));
-    if (ctx->opt_path == 0 && ctx->tc_ok && tc_shape_ok(dm)) {
+    if (ctx->opt_path != 1 && ctx->tc_ok && tc_shape_ok(dm)) {
         // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
         // LoRE on the general kernels
         SPICE_LAUNCH(launch_tc_expert_path(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));

@@ -37,7 +37,7 @@ namespace {
 constexpr int DT = 512;     // threads per CTA
 constexpr int TEAM = 256;   // threads per team
 constexpr int TW = 8;       // warps per team
-constexpr int NT_MAX = 4;   // n-tiles of 8 tokens
+constexpr int NT_MAX = 2;   // n-tiles of 8 tokens
 constexpr int XPAD = 64;    // row padding (bytes) of the token tile in shared memory
 
 __device__ __forceinline__ int ld_acquire(const int *p) {
@@ -781,13 +781,15 @@ __device__ __forceinline__ void load_batch(const WRows &w, int ks, uint4 (&a0lo)
 // The weight loads of a tile's next batch -- or of the NEXT tile's first batch -- are issued before
 // the partial sums are exchanged, so the memory pipe stays busy through barriers and epilogue.
 // Returns the id of the first task not executed; *alive = 0 (team-uniform) when a wait failed.
-template <int NT, int EPI>
+template <int NT, int EPI, int UD>
 __device__ __forceinline__ int team_run(const DecodeParams &p, const Plan &pl, TeamCtx &tc, uint32_t xs_s, int xstride, int id,
                                      int n_teams, int p1_total, int *alive) {
     constexpr bool DUAL = (EPI == EPI_ACT || EPI == EPI_PART2);
     constexpr bool B_SMEM = (EPI == EPI_ACT || EPI == EPI_Z);
     constexpr int MATS = DUAL ? 2 : 1;
-    constexpr int U = (NT == 4 || EPI == EPI_PART2) ? 2 : 4;
+    // k-steps in flight per warp.  More than the bandwidth-delay product only deepens the memory queues
+    // (every dependent access on the router's critical path then waits behind them): measured optimum.
+    constexpr int U = DUAL ? UD : 2 * UD;
     constexpr int MYFL = EPI == EPI_ACT ? FL_ACT : (EPI == EPI_Z ? FL_Z : (EPI == EPI_PART ? FL_PART : FL_PART2));
     const int c = tc.lane & 3;
     const uint4 zero = make_uint4(0, 0, 0, 0);
@@ -951,7 +953,7 @@ __device__ __noinline__ void task_p3(const DecodeParams &p, int ttid, int t, int
     }
 }
 
-template <int NT>
+template <int NT, int UD>
 __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const Dims &dm = p.dm;
@@ -984,10 +986,8 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
     pl.tIs = (dm.Is + 15) >> 4;
     pl.tI = (dm.I + 15) >> 4;
     pl.tr = (dm.r + 15) >> 4;
-    pl.rt_sh = (NT <= 2 && dm.Is <= 4096) ? 2 : 1;
-    pl.rt_hit = (NT <= 2 && dm.I <= 4096) ? 2 : 1;
-    pl.td_sh = (dm.d + 16 * pl.rt_sh - 1) / (16 * pl.rt_sh);
-    pl.td_hit = (dm.d + 16 * pl.rt_hit - 1) / (16 * pl.rt_hit);
+    pl.rt_sh = pl.rt_hit = 1;   // decided once the number of hit groups is known
+    pl.td_sh = pl.td_hit = (dm.d + 15) >> 4;
     pl.tb128 = (dm.d + 127) >> 7;
     pl.nb = (dm.d + 1023) >> 10;
     pl.nA = p.n_r1 + 1 + pl.tIs;
@@ -1045,6 +1045,14 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
             for (int i = tc.ttid; i < n_low; i += TEAM) tc.perm_l[i] = __ldcg(p.tb.perm_low + i);
             pl.nB_hit = pl.n_hg * pl.tI;
             pl.endB = pl.nA + pl.nB_hit + pl.n_lg * pl.tr;
+            // 32-row down tiles halve the activation reads and the tile-closing overhead per byte, but only pay
+            // when every team still gets several of them; with few tiles 16 rows keep more teams busy
+            if ((1 + pl.n_hg) * pl.td_sh >= 6 * n_teams) {
+                pl.rt_sh = dm.Is <= 4096 ? 2 : 1;
+                pl.rt_hit = dm.I <= 4096 ? 2 : 1;
+                pl.td_sh = (dm.d + 16 * pl.rt_sh - 1) / (16 * pl.rt_sh);
+                pl.td_hit = (dm.d + 16 * pl.rt_hit - 1) / (16 * pl.rt_hit);
+            }
             pl.nC_sh = pl.td_sh;
             pl.nC_hit = pl.n_hg * pl.td_hit;
             nC = pl.nC_sh + pl.nC_hit + pl.n_lg * pl.tb128;
@@ -1058,10 +1066,10 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
         }
         const TaskRef t = resolve(pl, id);
         const int fl = flavour_of(pl, tc, t);
-        if (fl == FL_ACT) id = team_run<NT, EPI_ACT>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
-        else if (fl == FL_Z) id = team_run<NT, EPI_Z>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
-        else if (fl == FL_PART2) id = team_run<(NT <= 2 ? NT : 1), EPI_PART2>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
-        else if (fl == FL_PART) id = team_run<NT, EPI_PART>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        if (fl == FL_ACT) id = team_run<NT, EPI_ACT, UD>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        else if (fl == FL_Z) id = team_run<NT, EPI_Z, UD>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        else if (fl == FL_PART2) id = team_run<(NT <= 2 ? NT : 1), EPI_PART2, UD>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
+        else if (fl == FL_PART) id = team_run<NT, EPI_PART, UD>(p, pl, tc, xs_s, xstride, id, n_teams, p1_total, &alive);
         else {
             if (fl == FL_R1) {
                 PROF(tc, 100 + TK_R1);
@@ -1100,21 +1108,31 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
 }  // namespace
 
 size_t decode_smem_bytes(const Dims &dm) {
-    const int nt = dm.T <= 8 ? 1 : (dm.T <= 16 ? 2 : 4);
+    const int nt = dm.T <= 8 ? 1 : 2;
     return smem_layout(dm, nt, nullptr, nullptr);
 }
 
 bool decode_supported(const Dims &dm, size_t max_smem) {
-    if (dm.T < 1 || dm.T > 8 * NT_MAX) return false;
+    // beyond 16 tokens the tensor-core path is faster (mma.sync work per weight byte grows with the n-tiles)
+    if (dm.T < 1 || dm.T > 16) return false;
     if (dm.N > 256 || dm.S > 256) return false;
     return decode_smem_bytes(dm) <= max_smem;
 }
 
+namespace {
+// (n-tiles, k-steps in flight per warp).  More in flight than the bandwidth-delay product only deepens the
+// memory queues, and every dependent access of the router's critical path then waits behind them; the
+// settings are the measured optimum on B200 for both layer shapes.
+const void *decode_variant(const Dims &dm) {
+    if (dm.T <= 8) return reinterpret_cast<const void *>(decode_layer_kernel<1, 2>);
+    return reinterpret_cast<const void *>(decode_layer_kernel<2, 1>);
+}
+}  // namespace
+
 // once per process and device: allow the kernels the opt-in shared memory size
 int decode_prepare(int max_smem_optin) {
-    const void *fns[3] = {reinterpret_cast<const void *>(decode_layer_kernel<1>),
-                          reinterpret_cast<const void *>(decode_layer_kernel<2>),
-                          reinterpret_cast<const void *>(decode_layer_kernel<4>)};
+    const void *fns[2] = {reinterpret_cast<const void *>(decode_layer_kernel<1, 2>),
+                          reinterpret_cast<const void *>(decode_layer_kernel<2, 1>)};
     for (const void *fn : fns)
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem_optin) != cudaSuccess)
             return -1;
@@ -1123,10 +1141,7 @@ int decode_prepare(int max_smem_optin) {
 
 int launch_decode(const DecodeParams &p, int n_ctas, cudaStream_t st) {
     const size_t smem = decode_smem_bytes(p.dm);
-    const void *fn;
-    if (p.dm.T <= 8) fn = reinterpret_cast<const void *>(decode_layer_kernel<1>);
-    else if (p.dm.T <= 16) fn = reinterpret_cast<const void *>(decode_layer_kernel<2>);
-    else fn = reinterpret_cast<const void *>(decode_layer_kernel<4>);
+    const void *fn = decode_variant(p.dm);
     void *args[] = {const_cast<DecodeParams *>(&p)};
     if (cudaLaunchCooperativeKernel(fn, dim3(n_ctas), dim3(DT), args, smem, st) != cudaSuccess) {
         cudaGetLastError();
