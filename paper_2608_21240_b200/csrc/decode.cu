@@ -117,8 +117,8 @@ struct TeamCtx {
     int gteam, nprof;
 #endif
     int team, ttid, twarp, lane;
-    int n_p1, n_p2;      // P1 / P2 tiles this warp has finished but not yet published
-    bool p1_all;         // this warp has seen every P1 tile of the layer published
+    int n_p1, n_p2;      // P1 / P2 tiles this team has finished but not yet published
+    bool p1_all;         // this team has seen every P1 tile of the layer published
     float *red;          // [TW][2][NT][128] partial tiles of this team
     int *flag;           // [2] broadcast slots
     GroupDesc *gtab;     // [1 + S + N] team-private copy of the group table
@@ -126,17 +126,19 @@ struct TeamCtx {
     int *perm_l;         // [T*K] copy of perm_low
 };
 
-// this warp's global stores are done -> publish one unit of progress (counters count warps)
-__device__ __forceinline__ void warp_signal(const TeamCtx &tc, int *ctr) {
-    __syncwarp();
-    if (tc.lane == 0) red_release_add(ctr, 1);
+// the team's global stores are done -> publish one unit of progress
+__device__ __forceinline__ void team_signal(const TeamCtx &tc, int *ctr) {
+    team_sync(tc.team);
+    if (tc.ttid == 0) red_release_add(ctr, 1);
 }
-// Publish this warp's finished-tile counts (one release each); called before the warp waits for
-// a later phase and when it leaves the task loop.
+// Publish the team's finished-tile counts (every warp of a team holds the same counts): one barrier so
+// that all stores of the team are issued, then one release by the leader.  Called before the team waits
+// for a later phase and when it leaves the task loop.  One atomic per team and phase: thousands of
+// atomics on one address would serialise in L2 and delay the phase change by microseconds.
 __device__ __forceinline__ void flush_counts(TeamCtx &tc, int *sync) {
-    if (tc.n_p1 | tc.n_p2) {   // warp-uniform
-        __syncwarp();
-        if (tc.lane == 0) {
+    if (tc.n_p1 | tc.n_p2) {   // team-uniform
+        team_sync(tc.team);
+        if (tc.ttid == 0) {
             if (tc.n_p1) red_release_add(sync + SY_P1_ALL, tc.n_p1);
             if (tc.n_p2) red_release_add(sync + SY_P2_DONE, tc.n_p2);
         }
@@ -156,13 +158,6 @@ __device__ __noinline__ bool wait_ge(const int *ctr, int target, int *sync, int 
     atomicMax(status, (int)SPICE_ERR_TIMEOUT);
     atomicExch(sync + SY_ABORT, 1);
     return false;
-}
-
-// lane 0 polls, the warp learns the result
-__device__ __forceinline__ bool warp_wait_ge(const TeamCtx &tc, const int *ctr, int target, const DecodeParams &p) {
-    int ok = 1;
-    if (tc.lane == 0) ok = wait_ge(ctr, target, p.sync, p.tb.status, p.spin_limit) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 // leader polls, result is broadcast through a slot: team-uniform result
@@ -401,7 +396,7 @@ __device__ __noinline__ void task_r1(const DecodeParams &p, unsigned char *smem_
         if (tc.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
     }
     PROF(tc, 61);
-    warp_signal(tc, p.sync + SY_R1_DONE);
+    team_signal(tc, p.sync + SY_R1_DONE);
     PROF(tc, 62);
 }
 
@@ -418,8 +413,10 @@ __device__ __forceinline__ int warp_excl_scan(int v, int lane, int &total) {
 }
 
 // R2: top-k + gates, classification, residual list, grouping (one team).  Everything between the
-// arrival of the logits and the published tables works out of shared memory; the ordered parts
-// (residual list, offsets of slots and experts) are done by single warps with shuffle scans.
+// arrival of the logits and the published tables works out of shared memory and is spread over the
+// 256 threads: this task is the serial section of the layer, every microsecond of it is paid by all SMs.
+// The arithmetic of the gates is that of warp_topk_gates (route_device.cuh), so the fused call and the
+// stand-alone router agree bit for bit; the winners are found by the same ranking rule.
 __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_raw, int nt, TC_ARG tc) {
     const Dims &dm = p.dm;
     Smem sm;
@@ -435,16 +432,54 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
     sm.cnt_hit[tc.ttid] = 0;
     sm.cnt_low[tc.ttid] = 0;
     PROF(tc, 50);
-    if (!team_wait_ge(tc, p.sync + SY_R1_DONE, N * TW, p)) return;
+    if (!team_wait_ge(tc, p.sync + SY_R1_DONE, N, p)) return;
     PROF(tc, 51);
 #pragma unroll 1
-    for (int i = tc.ttid; i < T * N; i += TEAM) sm.lg[i] = __ldcg(p.logits + i);
+    for (int i = tc.ttid; i < T * N; i += TEAM) {
+        float v = __ldcg(p.logits + i);
+        sm.lg[i] = (v == v) ? v : -INFINITY;   // NaN never wins
+    }
     team_sync(tc.team);
     PROF(tc, 52);
+    // winners by ranking, one (token, expert) pair per thread-step: rank = #{j : l_j > l_e or (l_j == l_e and j < e)}
 #pragma unroll 1
-    for (int t = tc.twarp; t < T; t += TW)
-        warp_topk_gates(sm.lg + t * N, N, K, p.norm_topk, tc.lane, sm.s_idx + t * K, sm.s_gate + t * K, nullptr,
-                        sm.sel_idx + tc.twarp * 32, sm.sel_val + tc.twarp * 32);
+    for (int i = tc.ttid; i < T * N; i += TEAM) {
+        const int t = i / N, e = i - t * N;
+        const float *l = sm.lg + t * N;
+        const float v = l[e];
+        int rank = 0;
+#pragma unroll 4
+        for (int j = 0; j < N; ++j) {
+            const float u = l[j];
+            rank += (u > v) || (u == v && j < e);
+        }
+        if (rank < K) {
+            sm.s_idx[t * K + rank] = e;
+            sm.s_gate[t * K + rank] = v;   // the logit for now
+        }
+    }
+    team_sync(tc.team);
+    // gates: p_k = exp(l_k - l_0); denominator = sum over the winners in k order, or the full softmax sum
+#pragma unroll 1
+    for (int t = tc.twarp; t < T; t += TW) {
+        const float m = sm.s_gate[t * K];
+        float denom = 0.f;
+        if (!p.norm_topk) {
+            float sacc = 0.f;
+#pragma unroll 1
+            for (int e = tc.lane; e < N; e += 32) sacc += expf(sm.lg[t * N + e] - m);
+            denom = warp_sum(sacc);
+        }
+        const float pk = (tc.lane < K) ? expf(sm.s_gate[t * K + tc.lane] - m) : 0.f;
+        if (p.norm_topk) {
+            float sacc = 0.f;
+#pragma unroll 1
+            for (int k = 0; k < K; ++k) sacc += __shfl_sync(0xffffffffu, pk, k);
+            denom = sacc;
+        }
+        __syncwarp();
+        if (tc.lane < K) sm.s_gate[t * K + tc.lane] = pk / denom;
+    }
     team_sync(tc.team);
     PROF(tc, 53);
     // classification (Sec. 4.2 policy); s_slot holds the grouping key: slot (HIT), 1024 + e (LOWCONF), -1
@@ -478,72 +513,64 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
     team_sync(tc.team);
     PROF(tc, 54);
     if (tc.twarp == 0) {
-        // residual-miss list (set M of Sec. 4.3) in (t,k) order: each lane owns a contiguous run
-        const int per = (n + 31) / 32, i0 = min(n, tc.lane * per), i1 = min(n, i0 + per);
-        int mine = 0;
+        // residual-miss list (set M of Sec. 4.3) in (t,k) order: 32 entries per step, ballot + popc
+        int base = 0;
 #pragma unroll 1
-        for (int i = i0; i < i1; ++i) mine += sm.s_cls[i] == SPICE_MISS_EXACT;
-        int total;
-        int o = warp_excl_scan(mine, tc.lane, total);
-        if (p.resid_tok)
-#pragma unroll 1
-            for (int i = i0; i < i1; ++i)
-                if (sm.s_cls[i] == SPICE_MISS_EXACT) {
-                    p.resid_tok[o] = i / K;
-                    p.resid_k[o] = i % K;
-                    p.resid_expert[o] = sm.s_idx[i];
-                    p.resid_gate[o] = sm.s_gate[i];
-                    ++o;
-                }
+        for (int i0 = 0; i0 < n; i0 += 32) {
+            const int i = i0 + tc.lane;
+            const bool miss = i < n && sm.s_cls[i] == SPICE_MISS_EXACT;
+            const unsigned m = __ballot_sync(0xffffffffu, miss);
+            if (miss && p.resid_tok) {
+                const int o = base + __popc(m & ((1u << tc.lane) - 1u));
+                p.resid_tok[o] = i / K;
+                p.resid_k[o] = i % K;
+                p.resid_expert[o] = sm.s_idx[i];
+                p.resid_gate[o] = sm.s_gate[i];
+            }
+            base += __popc(m);
+        }
         if (tc.lane < 3) p.counts[tc.lane] = sm.s_cnt[tc.lane];
-    } else if (tc.twarp == 1) {
-        // hit groups in slot order, then low-confidence groups in expert order (8 ids per lane)
-        int cnt[8], n_here = 0, g_here = 0;
-#pragma unroll
+    } else if (tc.twarp <= 2) {
+        // warp 1: hit groups in slot order; warp 2: low-confidence groups in expert order (8 ids per lane).
+        // Both need the number of hit groups, so both count them.
+        const bool low = tc.twarp == 2;
+        const int *cnt = low ? sm.cnt_low : sm.cnt_hit;
+        int *off_out = low ? sm.off_low : sm.off_hit;
+        int n_here = 0, g_here = 0, gh_here = 0;
+#pragma unroll 1
         for (int j = 0; j < 8; ++j) {
-            cnt[j] = sm.cnt_hit[tc.lane * 8 + j];
-            n_here += cnt[j];
-            g_here += cnt[j] > 0;
+            const int cj = cnt[tc.lane * 8 + j];
+            n_here += cj;
+            g_here += cj > 0;
+            gh_here += sm.cnt_hit[tc.lane * 8 + j] > 0;
         }
-        int n_hit, n_hg;
-        int off = warp_excl_scan(n_here, tc.lane, n_hit);
-        int gi = warp_excl_scan(g_here, tc.lane, n_hg);
-#pragma unroll
+        int n_tot, n_g, n_hg;
+        int off = warp_excl_scan(n_here, tc.lane, n_tot);
+        int gi = warp_excl_scan(g_here, tc.lane, n_g);
+        warp_excl_scan(gh_here, tc.lane, n_hg);
+        const int gbase = low ? 1 + n_hg : 1;
+#pragma unroll 1
         for (int j = 0; j < 8; ++j) {
             const int id = tc.lane * 8 + j;
-            sm.off_hit[id] = off;
-            if (cnt[j] > 0) p.tb.groups[1 + gi++] = GroupDesc{KIND_HIT, id, off, cnt[j]};
-            off += cnt[j];
-        }
-        n_here = g_here = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            cnt[j] = sm.cnt_low[tc.lane * 8 + j];
-            n_here += cnt[j];
-            g_here += cnt[j] > 0;
-        }
-        int n_low, n_lg;
-        off = warp_excl_scan(n_here, tc.lane, n_low);
-        gi = warp_excl_scan(g_here, tc.lane, n_lg);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int id = tc.lane * 8 + j;
-            sm.off_low[id] = off;
-            if (cnt[j] > 0) p.tb.groups[1 + n_hg + gi++] = GroupDesc{KIND_LOW, id, off, cnt[j]};
-            off += cnt[j];
+            const int cj = cnt[id];
+            off_out[id] = off;
+            if (cj > 0) p.tb.groups[gbase + gi++] = GroupDesc{low ? KIND_LOW : KIND_HIT, id, off, cj};
+            off += cj;
         }
         if (tc.lane == 0) {
-            p.tb.groups[0] = GroupDesc{KIND_SHARED, 0, 0, T};
-            p.tb.hdr[HDR_N_GROUPS] = 1 + n_hg + n_lg;
-            p.tb.hdr[HDR_N_HIT_GROUPS] = n_hg;
-            p.tb.hdr[HDR_N_LOW_GROUPS] = n_lg;
-            p.tb.hdr[HDR_N_HIT] = n_hit;
-            p.tb.hdr[HDR_N_LOW] = n_low;
+            if (low) {
+                p.tb.hdr[HDR_N_LOW_GROUPS] = n_g;
+                p.tb.hdr[HDR_N_LOW] = n_tot;
+            } else {
+                p.tb.groups[0] = GroupDesc{KIND_SHARED, 0, 0, T};
+                p.tb.hdr[HDR_N_HIT_GROUPS] = n_g;
+                p.tb.hdr[HDR_N_HIT] = n_tot;
+            }
         }
     } else {
         // coefficient of the shared expert's output: 1 + sum of LOWCONF gates, in k order
 #pragma unroll 1
-        for (int t = tc.ttid - 64; t < T; t += TEAM - 64) {
+        for (int t = tc.ttid - 96; t < T; t += TEAM - 96) {
             float c = 1.0f;
 #pragma unroll 1
             for (int k = 0; k < K; ++k)
@@ -553,36 +580,31 @@ __device__ __noinline__ void task_r2(const DecodeParams &p, unsigned char *smem_
     }
     team_sync(tc.team);
     PROF(tc, 55);
-    sm.cnt_hit[tc.ttid] = 0;   // now cursors
-    sm.cnt_low[tc.ttid] = 0;
-    team_sync(tc.team);
+    // position of every entry inside its group = offset of the group + number of earlier entries of the group
 #pragma unroll 1
-    for (int i0 = 0; i0 < n; i0 += TEAM) {
-        const int i = i0 + tc.ttid;
-        const int key = i < n ? sm.s_slot[i] : -1;
-        const unsigned peers = __match_any_sync(0xffffffffu, key);
+    for (int i = tc.ttid; i < n; i += TEAM) {
+        const int key = sm.s_slot[i];
         int pos = -1;
         if (key >= 0) {
-            const int leader = __ffs(peers) - 1;
-            int basep = 0;
-            if (tc.lane == leader)
-                basep = (key < 1024) ? atomicAdd(&sm.cnt_hit[key], __popc(peers))
-                                     : atomicAdd(&sm.cnt_low[key - 1024], __popc(peers));
-            basep = __shfl_sync(peers, basep, leader);
-            const int rank = __popc(peers & ((1u << tc.lane) - 1u));
+            int rank = 0;
+#pragma unroll 4
+            for (int j = 0; j < i; ++j) rank += sm.s_slot[j] == key;
             if (key < 1024) {
-                pos = sm.off_hit[key] + basep + rank;
+                pos = sm.off_hit[key] + rank;
                 p.tb.perm_hit[pos] = i;
             } else {
-                pos = sm.off_low[key - 1024] + basep + rank;
+                pos = sm.off_low[key - 1024] + rank;
                 p.tb.perm_low[pos] = i;
             }
         }
-        if (i < n) p.tb.pos_of_entry[i] = pos;
+        p.tb.pos_of_entry[i] = pos;
     }
     team_sync(tc.team);
     PROF(tc, 56);
-    if (tc.ttid == 0) red_release_add(p.sync + SY_ROUTE_DONE, 1);
+    if (tc.ttid == 0) {
+        p.tb.hdr[HDR_N_GROUPS] = 0;   // (not used by this kernel)
+        red_release_add(p.sync + SY_ROUTE_DONE, 1);
+    }
     PROF(tc, 57);
 }
 
@@ -657,8 +679,7 @@ struct P1DoneGate {
     int p1_total;
     __device__ __forceinline__ bool operator()() const {
         if (tc.p1_all) return true;
-        flush_counts(tc, p.sync);
-        tc.p1_all = warp_wait_ge(tc, p.sync + SY_P1_ALL, p1_total, p);
+        tc.p1_all = team_wait_ge(tc, p.sync + SY_P1_ALL, p1_total, p);
         return tc.p1_all;
     }
 };
@@ -789,7 +810,11 @@ __device__ __forceinline__ int team_run(const DecodeParams &p, const Plan &pl, T
     constexpr int MATS = DUAL ? 2 : 1;
     // k-steps in flight per warp.  More than the bandwidth-delay product only deepens the memory queues
     // (every dependent access on the router's critical path then waits behind them): measured optimum.
+#ifdef SPICE_U_P2
+    constexpr int U = (EPI == EPI_PART2) ? SPICE_U_P2 : (DUAL ? UD : 2 * UD);
+#else
     constexpr int U = DUAL ? UD : 2 * UD;
+#endif
     constexpr int MYFL = EPI == EPI_ACT ? FL_ACT : (EPI == EPI_Z ? FL_Z : (EPI == EPI_PART ? FL_PART : FL_PART2));
     const int c = tc.lane & 3;
     const uint4 zero = make_uint4(0, 0, 0, 0);
@@ -798,9 +823,8 @@ __device__ __forceinline__ int team_run(const DecodeParams &p, const Plan &pl, T
     WRows w = make_rows<EPI>(a, tc);
     load_batch<DUAL, U>(w, w.ks0, a0lo, a0hi, a1lo, a1hi, c);
     bool failed = false;
-    if (!B_SMEM && !tc.p1_all) {   // first P2 tile of this warp: every P1 tile must be published
-        flush_counts(tc, p.sync);
-        tc.p1_all = warp_wait_ge(tc, p.sync + SY_P1_ALL, p1_total, p);
+    if (!B_SMEM && !tc.p1_all) {   // first P2 tile of this team: every P1 tile must be published
+        tc.p1_all = team_wait_ge(tc, p.sync + SY_P1_ALL, p1_total, p);   // (publishes the team's own count first)
         failed = !tc.p1_all;
     }
     *alive = 1;
@@ -1037,12 +1061,17 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
             PROF(tc, 31);
             if (!alive) break;
             // team-private copy of the group table and the permutations: task set-up never goes to L2 again
+            // (everything is requested at once, at its maximum size, so this costs one memory round trip)
             pl.n_hg = __ldcg(p.tb.hdr + HDR_N_HIT_GROUPS);
             pl.n_lg = __ldcg(p.tb.hdr + HDR_N_LOW_GROUPS);
-            const int n_hit = __ldcg(p.tb.hdr + HDR_N_HIT), n_low = __ldcg(p.tb.hdr + HDR_N_LOW);
-            for (int i = tc.ttid; i < 1 + pl.n_hg + pl.n_lg; i += TEAM) tc.gtab[i] = load_group(p.tb.groups + i);
-            for (int i = tc.ttid; i < n_hit; i += TEAM) tc.perm_h[i] = __ldcg(p.tb.perm_hit + i);
-            for (int i = tc.ttid; i < n_low; i += TEAM) tc.perm_l[i] = __ldcg(p.tb.perm_low + i);
+            {
+                const int ng_max = 1 + min(dm.S, dm.T * dm.K) + min(dm.N, dm.T * dm.K), ne = dm.T * dm.K;
+                for (int i = tc.ttid; i < ng_max; i += TEAM) tc.gtab[i] = load_group(p.tb.groups + i);
+                for (int i = tc.ttid; i < ne; i += TEAM) {
+                    tc.perm_h[i] = __ldcg(p.tb.perm_hit + i);
+                    tc.perm_l[i] = __ldcg(p.tb.perm_low + i);
+                }
+            }
             pl.nB_hit = pl.n_hg * pl.tI;
             pl.endB = pl.nA + pl.nB_hit + pl.n_lg * pl.tr;
             // 32-row down tiles halve the activation reads and the tile-closing overhead per byte, but only pay
@@ -1059,7 +1088,7 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
             pl.endC = pl.endB + nC;
             pl.endD = pl.endC + dm.T * pl.nb;
             pl.routed = true;
-            p1_total = (pl.tIs + pl.nB_hit + pl.n_lg * pl.tr) * TW;
+            p1_total = pl.tIs + pl.nB_hit + pl.n_lg * pl.tr;
             end = pl.endD;
             team_sync(tc.team);
             continue;
@@ -1081,7 +1110,7 @@ __global__ void __launch_bounds__(DT, 1) decode_layer_kernel(const __grid_consta
                 alive = task_lore_b<NT>(p, tc, t.gi, t.tile, p1_total) ? 1 : 0;
             } else {
                 if (!p2_ready) {   // combine needs every down-projected row (counted per warp)
-                    alive = team_wait_ge(tc, p.sync + SY_P2_DONE, nC * TW, p) ? 1 : 0;
+                    alive = team_wait_ge(tc, p.sync + SY_P2_DONE, nC, p) ? 1 : 0;
                     if (!alive) break;
                     p2_ready = true;
                 }
