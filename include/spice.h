@@ -181,8 +181,9 @@ spice_status spice_get_device_status(spice_ctx *ctx, int32_t *code /* host */);
 spice_status spice_launch_count(const spice_ctx *ctx, int64_t *launches /* host */);
 
 /* Knobs (host only).  SPICE_OPT_PATH: 0 = choose the kernel path by batch size (default),
- * 1 = always use the general-shape kernels, 2 = never use the fused decode kernel (tensor-core
- * grouped GEMM for the experts at any batch size).  SPICE_OPT_SPIN_LIMIT: number of polls after which a
+ * 1 = always use the general-shape kernels, 2 = never use a fused decode kernel (tensor-core
+ * grouped GEMM for the experts at any batch size), 3 = for small batches use the fused decode
+ * kernel built on mma.sync instead of the tcgen05 one.  SPICE_OPT_SPIN_LIMIT: number of polls after which a
  * dependency wait inside the fused decode kernel gives up and reports SPICE_ERR_TIMEOUT
  * (default 2^20; a poll takes 0.1 to 1 us). */
 enum { SPICE_OPT_PATH = 0, SPICE_OPT_SPIN_LIMIT = 1 };

@@ -22,11 +22,13 @@ struct spice_ctx {
     __nv_bfloat16 *act_hit16, *act_shared16, *z16;
     int32_t *sync;
     int32_t sync_words;
-    int32_t decode_tokens;          // largest T the decode buffers were sized for (0: path unavailable)
+    int32_t decode_tokens;          // largest T of the mma.sync decode kernel (0: path unavailable)
+    int32_t dtc_tokens;             // largest T of the tcgen05 decode kernel (0: path unavailable)
+    float *part_split;              // [splits][Td, d] partial shared-expert outputs of the tcgen05 decode kernel
     int n_sms, max_smem_optin;
     TcBuffers tcb;                  // tensor-core path buffers (large batches)
     bool tc_ok;
-    int64_t opt_path;               // 0 auto, 1 general kernels only, 2 never the fused decode kernel
+    int64_t opt_path;               // 0 auto, 1 general kernels only, 2 no fused decode kernel, 3 mma.sync decode kernel
     int64_t opt_spin_limit;
     int64_t launches;
 };
@@ -46,6 +48,10 @@ struct Carver {
         return p;
     }
 };
+
+Dims dims_of_cfg(const spice_layer_cfg &g, int T) {
+    return Dims{T, g.d, g.n_experts, g.top_k, g.inter, g.inter_shared, g.lore_rank, g.n_slots};
+}
 
 void carve(spice_ctx *c, char *base, size_t *total) {
     const spice_layer_cfg &g = c->cfg;
@@ -69,11 +75,14 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->ws_gate = cv.take<float>(n);
     c->ws_cls = cv.take<uint8_t>(n);
     c->y32 = cv.take<float>(Tm * g.d);
-    const size_t Td = Tm < 16 ? Tm : 16, nd = Td * K;
+    // decode kernels: activations of a group are kept for every token of the batch ([group][T][width])
+    const size_t Td = Tm < 64 ? Tm : 64, nd = Td * K;
+    const size_t g_hit = (size_t)g.n_slots < nd ? g.n_slots : nd, g_low = (size_t)g.n_experts < nd ? g.n_experts : nd;
     c->logits = cv.take<float>(Td * g.n_experts);
-    c->act_hit16 = cv.take<__nv_bfloat16>(nd * g.inter);
+    c->act_hit16 = cv.take<__nv_bfloat16>((g_hit * Td > nd ? g_hit * Td : nd) * g.inter);
     c->act_shared16 = cv.take<__nv_bfloat16>(Td * g.inter_shared);
-    c->z16 = cv.take<__nv_bfloat16>(nd * g.lore_rank);
+    c->z16 = cv.take<__nv_bfloat16>((g_low * Td > nd ? g_low * Td : nd) * g.lore_rank);
+    c->part_split = cv.take<float>((size_t)decode_tc_nsplit(dims_of_cfg(g, 1)) * Td * g.d);
     c->sync_words = SY_GROUP0 + 1 + g.n_slots + g.n_experts;
     c->sync = cv.take<int32_t>(c->sync_words);
     {   // buffers of the tensor-core path
@@ -175,6 +184,7 @@ spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg
     c->decode_tokens = (coop && decode_prepare(c->max_smem_optin) == 0) ? (max_tokens < 16 ? max_tokens : 16) : 0;
     c->tcb = TcBuffers{};
     c->tc_ok = tc_available() && tc_prepare() == 0;
+    c->dtc_tokens = (coop && c->tc_ok && decode_tc_prepare(c->max_smem_optin) == 0) ? (max_tokens < 64 ? max_tokens : 64) : 0;
     carve(c, nullptr, &c->ws_bytes);
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -229,7 +239,7 @@ spice_status spice_set_option(spice_ctx *ctx, int32_t option, int64_t value) {
     if (!ctx) return SPICE_ERR_INVALID_ARG;
     switch (option) {
         case SPICE_OPT_PATH:
-            if (value < 0 || value > 2) return SPICE_ERR_INVALID_ARG;
+            if (value < 0 || value > 3) return SPICE_ERR_INVALID_ARG;
             ctx->opt_path = value;
             return SPICE_OK;
         case SPICE_OPT_SPIN_LIMIT:
@@ -330,7 +340,11 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     if (!(resid_tok && resid_k && resid_expert && resid_gate)) resid_tok = resid_k = resid_expert = nullptr, resid_gate = nullptr;
     const Dims dm = dims_of(ctx, T);
     const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
-    if (ctx->opt_path == 0 && T <= ctx->decode_tokens && decode_supported(dm, (size_t)ctx->max_smem_optin)) {
+    const bool use_dtc = ctx->opt_path == 0 && T <= ctx->dtc_tokens &&
+                         decode_tc_supported(dm, ctx->cfg.conf_stride, (size_t)ctx->max_smem_optin);
+    const bool use_dec = !use_dtc && (ctx->opt_path == 0 || ctx->opt_path == 3) && T <= ctx->decode_tokens &&
+                         decode_supported(dm, (size_t)ctx->max_smem_optin);
+    if (use_dtc || use_dec) {
         // small batch: one persistent kernel for the whole layer
         DecodeParams p;
         p.dm = dm;
@@ -360,7 +374,8 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         p.act_shared16 = ctx->act_shared16;
         p.z16 = ctx->z16;
         p.sync = ctx->sync;
-        int n = launch_decode(p, ctx->n_sms, st);
+        int n = use_dtc ? launch_decode_tc(p, ctx->part_split, ctx->n_sms, ctx->max_smem_optin, st)
+                        : launch_decode(p, ctx->n_sms, st);
         if (n > 0) {
             ctx->launches += n;
             return SPICE_OK;
@@ -372,7 +387,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
                                  ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st));
-    if (ctx->opt_path != 1 && ctx->tc_ok && tc_shape_ok(dm)) {
+    if (ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm)) {
         // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
         // LoRE on the general kernels
         SPICE_LAUNCH(launch_tc_expert_path(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));

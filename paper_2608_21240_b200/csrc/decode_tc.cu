@@ -1,0 +1,964 @@
+// Fused decode kernel on the Blackwell tensor-core pipeline: the whole MoE layer (Eq. 1 routing;
+// Sec. 4.2 hit / low-confidence / exact-recovery policy; exact resident experts; shared expert +
+// LoRE surrogate; gate-weighted aggregation of Sec. 2.1) in ONE persistent cooperative launch for
+// small batches (T <= 64).
+//
+// At these batch sizes the layer is HBM-bound: every weight byte is needed once.  The kernel is a
+// weight streamer built like a GEMM with the operands swapped: the WEIGHT rows are the M side of
+// the MMA (128 rows per tile), the tokens are the N side (16, 32 or 64 columns), so one
+// tcgen05.mma consumes 128 x 16 weight elements per token column and the per-byte instruction
+// cost vanishes.  Every group (shared expert, resident slot, low-confidence expert) is computed
+// for ALL tokens of the batch -- the tensor core is idle anyway -- and the epilogue keeps only the
+// columns of tokens routed to the group; nothing is gathered.
+//
+// One CTA per SM, 14 warps:
+//   warp 0      TMA producer: walks the task list, waits (bounded) for a task's dependency counter,
+//               queues the task for the other roles and streams its operands k-chunk by k-chunk
+//               (128 weight rows x 64 k + NB token rows x 64 k, 128-byte swizzle) into a
+//               shared-memory ring of up to 12 stages; mbarrier complete_tx
+//   warp 1      issues tcgen05.mma (M = 128, N = NB, K = 16, bf16 -> fp32 in TMEM); accumulators are
+//               double-buffered; tcgen05.commit frees ring stages and publishes accumulators
+//   warps 2-5   epilogue: tcgen05.ld, SwiGLU (gate rows in TMEM lanes 0-63, up rows in lanes 64-127,
+//               paired through shared memory) or plain; stores; release of the task's counter
+//   warps 6-13  auxiliary team: router logits (its share), then the routing decisions computed
+//               REDUNDANTLY by every CTA from the logits (top-k, gates, classification, grouping):
+//               the tables land in shared memory without a second grid-wide hop; finally the combine
+//
+// Tasks (ids dealt round-robin to the CTAs; a task depends only on tasks with smaller ids):
+//   A  gate/up tile of the shared expert: 64 gate + 64 up rows, K = d              (no dependency)
+//   B  gate/up tile of a resident slot; A_e tile of a low-confidence expert        (routing)
+//   C  down tile, 128 rows: shared expert (K split into ranges), slot, B_e         (that group's B tiles)
+//   D  combine y_t = c_t S(h_t) + sum_k g_k part_{t,k}  (auxiliary teams)          (all C tiles)
+// Dependencies are counters in global memory: red.release by the finishing warp, bounded
+// ld.acquire polls by the waiting one.  Data written by plain stores and later fetched by TMA is
+// ordered with fence.proxy.async on both sides.  Every wait in the kernel is bounded; on expiry
+// the CTA records SPICE_ERR_TIMEOUT, raises the abort flag, drains its copies in flight, frees
+// its TMEM and returns.  No load uses cluster multicast.
+#include <cuda.h>
+
+#include "route_device.cuh"
+#include "spice_internal.cuh"
+#include "tc_device.cuh"
+
+namespace spice {
+
+namespace {
+
+using namespace tcdev;
+
+constexpr int DTC_THREADS = 448;
+constexpr int AUX_T0 = 192, AUX_T = 256, AUX_W = 8;
+constexpr int MAX_STAGES = 12, TQ = 4;
+constexpr int A_BYTES = 128 * 64 * 2;
+constexpr int MAX_SPLIT = 16, CHUNKS_PER_SPLIT = 32;
+
+enum { TASK_EXIT = 0, TASK_ACT = 1, TASK_Z = 2, TASK_DOWN = 3 };
+enum { MAP_H = 0, MAP_SLOT_GU, MAP_SH_GU, MAP_LORE_A, MAP_SLOT_D, MAP_SH_D, MAP_LORE_B, MAP_ACT_HIT, MAP_ACT_SH, MAP_Z, N_MAPS };
+
+struct TaskDesc {
+    int32_t kind, gi, tile, split, nk, pad0, pad1, pad2;
+};
+
+struct DtcParams {
+    DecodeParams p;
+    float *part_split;   // [nsplit_sh][T][d] partial sums of the shared expert's down projection
+    int32_t stages;      // ring depth
+    int32_t nsplit_sh;   // K ranges of the shared down projection
+    int32_t cps_sh;      // k-chunks per range
+    int32_t r1_sub;      // token subsets per expert in the router-logit units
+};
+struct DtcMaps {
+    CUtensorMap m[N_MAPS];
+};
+
+struct Ctl {
+    alignas(8) unsigned long long full[MAX_STAGES], empty[MAX_STAGES];
+    unsigned long long tmem_full[2], tmem_empty[2];
+    unsigned long long tq_full[TQ], tq_empty[TQ];
+    unsigned long long xch_full[2], xch_empty[2];
+    unsigned long long plan_ready, mma_drain;
+    TaskDesc tq[TQ];
+    uint32_t tmem_base;
+    int abort_flag;
+    int n_hg, n_lg;
+    int aux_flag;
+    int last_flag;
+    int wsum[2][AUX_W];
+    int s_cnt[4];
+};
+
+// auxiliary team's shared memory (routing scratch and the tables every role reads)
+struct AuxSmem {
+    float *lg, *conf, *gate, *coef, *xch;
+    int *soe, *idx, *key, *pos, *perm_h, *perm_l, *cnt_hit, *cnt_low, *off_hit, *off_low, *ent;
+    unsigned char *cls;
+    GroupDesc *gtab;
+};
+
+__host__ __device__ inline size_t up16(size_t v) { return (v + 15) & ~size_t(15); }
+
+__host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, int nb, AuxSmem *s, unsigned char *base) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off += up16(bytes);
+        return o;
+    };
+    const size_t n = (size_t)dm.T * dm.K, TN = (size_t)dm.T * dm.N;
+    const size_t o_lg = take(TN * 4), o_conf = take((conf_stride ? TN : (size_t)dm.T) * 4), o_gate = take(n * 4);
+    const size_t o_coef = take((size_t)dm.T * 4), o_xch = take((size_t)2 * nb * 64 * 4);
+    const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_key = take(n * 4), o_pos = take(n * 4);
+    const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take(4 * 256 * 4), o_ent = take((size_t)4 * nb * 4);
+    const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
+    if (s) {
+        s->lg = reinterpret_cast<float *>(base + o_lg);
+        s->conf = reinterpret_cast<float *>(base + o_conf);
+        s->gate = reinterpret_cast<float *>(base + o_gate);
+        s->coef = reinterpret_cast<float *>(base + o_coef);
+        s->xch = reinterpret_cast<float *>(base + o_xch);
+        s->soe = reinterpret_cast<int *>(base + o_soe);
+        s->idx = reinterpret_cast<int *>(base + o_idx);
+        s->key = reinterpret_cast<int *>(base + o_key);
+        s->pos = reinterpret_cast<int *>(base + o_pos);
+        s->perm_h = reinterpret_cast<int *>(base + o_ph);
+        s->perm_l = reinterpret_cast<int *>(base + o_pl);
+        int *hist = reinterpret_cast<int *>(base + o_hist);
+        s->cnt_hit = hist;
+        s->cnt_low = hist + 256;
+        s->off_hit = hist + 512;
+        s->off_low = hist + 768;
+        s->ent = reinterpret_cast<int *>(base + o_ent);
+        s->cls = base + o_cls;
+        s->gtab = reinterpret_cast<GroupDesc *>(base + o_gt);
+    }
+    return off;
+}
+
+__host__ __device__ inline int nb_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
+__host__ __device__ inline int stage_bytes_of(int nb) { return A_BYTES + nb * 128; }
+
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int ld_acquire(const int *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ int ld_relaxed(const int *p) {
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_add(int *p, int v) {
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void aux_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// Bounded wait of ONE thread on a dependency counter: true when *ctr >= target; false on abort or when
+// the limit expires, in which case the sticky status and both abort flags are set.
+__device__ __noinline__ bool wait_ge(const int *ctr, int target, int *sync, int *status, int spin_limit, volatile int *cta_abort) {
+    for (int it = 0; it < spin_limit; ++it) {
+        if (ld_acquire(ctr) >= target) return true;
+        if ((it & 15) == 15 && (ld_relaxed(sync + SY_ABORT) || *cta_abort)) {
+            *cta_abort = 1;
+            return false;
+        }
+        if (it > 32) __nanosleep(32);
+    }
+    atomicMax(status, (int)SPICE_ERR_TIMEOUT);
+    atomicExch(sync + SY_ABORT, 1);
+    *cta_abort = 1;
+    return false;
+}
+
+__device__ __forceinline__ unsigned long long now_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+constexpr unsigned long long ROLE_WAIT_NS = 1000000000ull;   // a role gives up after a second without progress
+constexpr unsigned long long DRAIN_WAIT_NS = 200000000ull;
+
+// mbarrier wait bounded by time (a try_wait may itself suspend the thread for a while, so polls are not a
+// measure); false when the limit expired or another role already gave up
+__device__ __forceinline__ bool mb_wait(uint32_t a, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try(a, parity)) return true;
+    const unsigned long long t0 = now_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try(a, parity)) return true;
+        if ((i & 31u) == 0u) {
+            if (*abort_flag) return false;
+            if (now_ns() - t0 > ROLE_WAIT_NS) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+// the same without the abort check, for waits that must outlast an abort (copies / MMAs in flight)
+__device__ __forceinline__ void mb_drain(uint32_t a, uint32_t parity) {
+    const unsigned long long t0 = now_ns();
+    for (uint32_t i = 1;; ++i) {
+        if (mbar_try(a, parity)) return;
+        if ((i & 31u) == 0u && now_ns() - t0 > DRAIN_WAIT_NS) return;
+    }
+}
+
+// whole warp: lane 0 polls (bounded), the outcome is warp-uniform; every lane then observes the completed phase itself
+__device__ __forceinline__ bool warp_mb_wait(uint32_t a, uint32_t parity, volatile int *abort_flag, int lane) {
+    bool ok = true;
+    if (lane == 0) ok = mb_wait(a, parity, abort_flag);
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    if (ok) (void)mbar_try(a, parity);
+    return ok;
+}
+
+// ------------------------------------------------------------------------------------------
+// Task list.  ids [0, nA) are known at launch; the rest once the routing tables exist.
+struct Plan {
+    int tIs, tI, tz, td;            // tiles per matrix
+    int kcd, kcI, kcr;              // k-chunks (64 elements) of d, I, r
+    int nsplit, cps, kcIs;          // shared down projection: K ranges, chunks per range, chunks in all
+    int nA, nBh, endB, nCs, nCh, endC;
+    int n_hg, n_lg;
+};
+
+__device__ __forceinline__ void plan_static(Plan &pl, const DtcParams &q) {
+    const Dims &dm = q.p.dm;
+    pl.tIs = (dm.Is + 63) >> 6;
+    pl.tI = (dm.I + 63) >> 6;
+    pl.tz = (dm.r + 127) >> 7;
+    pl.td = (dm.d + 127) >> 7;
+    pl.kcd = (dm.d + 63) >> 6;
+    pl.kcI = (dm.I + 63) >> 6;
+    pl.kcr = (dm.r + 63) >> 6;
+    pl.kcIs = (dm.Is + 63) >> 6;
+    pl.nsplit = q.nsplit_sh;
+    pl.cps = q.cps_sh;
+    pl.nA = pl.tIs;
+    pl.n_hg = pl.n_lg = pl.nBh = pl.nCs = pl.nCh = 0;
+    pl.endB = pl.endC = pl.nA;
+}
+__device__ __forceinline__ void plan_routed(Plan &pl, int n_hg, int n_lg) {
+    pl.n_hg = n_hg;
+    pl.n_lg = n_lg;
+    pl.nBh = n_hg * pl.tI;
+    pl.endB = pl.nA + pl.nBh + n_lg * pl.tz;
+    pl.nCs = pl.td * pl.nsplit;
+    pl.nCh = n_hg * pl.td;
+    pl.endC = pl.endB + pl.nCs + pl.nCh + n_lg * pl.td;
+}
+
+// ------------------------------------------------------------------------------------------
+// Auxiliary team
+struct AuxCtx {
+    int atid, lane, aw;
+};
+
+// leader polls, result broadcast through shared memory: team-uniform
+__device__ __forceinline__ bool aux_wait_ge(const DtcParams &q, Ctl *sh, const AuxCtx &a, const int *ctr, int target) {
+    if (a.atid == 0)
+        sh->aux_flag = wait_ge(ctr, target, q.p.sync, q.p.tb.status, q.p.spin_limit, &sh->abort_flag) ? 1 : 0;
+    aux_sync();
+    const bool ok = sh->aux_flag != 0;
+    aux_sync();
+    return ok;
+}
+
+// router logits: unit u = (expert e, token subset s); each warp takes the tokens s*8 + warp (+ 8*r1_sub ...).
+// Same arithmetic order as the stand-alone router (route_device.cuh): logits agree bit for bit.
+__device__ __noinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) {
+    const DecodeParams &p = q.p;
+    const Dims &dm = p.dm;
+    const int n_units = dm.N * q.r1_sub;
+    int done = 0;
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++done) {
+        const int e = u % dm.N, s = u / dm.N;
+        const __nv_bfloat16 *row = reinterpret_cast<const __nv_bfloat16 *>(p.w.w_router) + (size_t)e * dm.d;
+        for (int t = s * AUX_W + a.aw; t < dm.T; t += AUX_W * q.r1_sub) {
+            const float sdot = lane_dot_bf16(row, p.h + (size_t)t * dm.d, dm.d, a.lane);
+            const float tot = warp_sum(sdot);
+            if (a.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
+        }
+    }
+    if (done) {   // CTA-uniform
+        aux_sync();
+        if (a.atid == 0) red_release_add(p.sync + SY_R1_DONE, done);
+    }
+}
+
+// Routing decisions from the logits, entirely in shared memory.  Every CTA computes the same tables
+// (the code is deterministic: counts by atomics, positions by ranking); CTA 0 also writes the outputs.
+// The arithmetic of the gates is that of warp_topk_gates (route_device.cuh).
+__device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, const AuxCtx &a) {
+    const DecodeParams &p = q.p;
+    const Dims &dm = p.dm;
+    const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
+#pragma unroll 1
+    for (int i = a.atid; i < T * N; i += AUX_T) {
+        const float v = __ldcg(p.logits + i);
+        ax.lg[i] = (v == v) ? v : -INFINITY;   // NaN never wins
+    }
+    aux_sync();
+    // winners by ranking: rank = #{j : l_j > l_e or (l_j == l_e and j < e)}
+#pragma unroll 1
+    for (int i = a.atid; i < T * N; i += AUX_T) {
+        const int t = i / N, e = i - t * N;
+        const float *l = ax.lg + t * N;
+        const float v = l[e];
+        int rank = 0;
+#pragma unroll 8
+        for (int j = 0; j < N; ++j) {
+            const float u = l[j];
+            rank += (u > v) || (u == v && j < e);
+        }
+        if (rank < K) {
+            ax.idx[t * K + rank] = e;
+            ax.gate[t * K + rank] = v;   // the logit for now
+        }
+    }
+    aux_sync();
+    // gates: p_k = exp(l_k - l_0); denominator = sum over the winners in k order, or the full softmax sum
+#pragma unroll 1
+    for (int t = a.aw; t < T; t += AUX_W) {
+        const float m = ax.gate[t * K];
+        float denom = 0.f;
+        if (!p.norm_topk) {
+            float sacc = 0.f;
+#pragma unroll 1
+            for (int e = a.lane; e < N; e += 32) sacc += expf(ax.lg[t * N + e] - m);
+            denom = warp_sum(sacc);
+        }
+        const float pk = (a.lane < K) ? expf(ax.gate[t * K + a.lane] - m) : 0.f;
+        if (p.norm_topk) {
+            float sacc = 0.f;
+#pragma unroll 1
+            for (int k = 0; k < K; ++k) sacc += __shfl_sync(0xffffffffu, pk, k);
+            denom = sacc;
+        }
+        __syncwarp();
+        if (a.lane < K) ax.gate[t * K + a.lane] = pk / denom;
+    }
+    aux_sync();
+    // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
+#pragma unroll 1
+    for (int i = a.atid; i < n; i += AUX_T) {
+        const int e = ax.idx[i];
+        const int sl = ax.soe[e];
+        int c, key = -1;
+        if (sl >= S) {
+            atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
+            c = SPICE_MISS_EXACT;
+        } else if (sl >= 0) {
+            c = SPICE_HIT;
+            key = sl;
+            atomicAdd(&ax.cnt_hit[sl], 1);
+        } else {
+            const int t = i / K;
+            const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
+            c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
+            if (c == SPICE_LOWCONF) {
+                key = 1024 + e;
+                atomicAdd(&ax.cnt_low[e], 1);
+            }
+        }
+        ax.cls[i] = (unsigned char)c;
+        ax.key[i] = key;
+        atomicAdd(&sh->s_cnt[c], 1);
+    }
+    aux_sync();
+    // groups: thread i owns slot i and expert i; packed scan of (entries, non-empty flag << 16)
+    {
+        const int ch = a.atid < S ? ax.cnt_hit[a.atid] : 0, cl = a.atid < N ? ax.cnt_low[a.atid] : 0;
+        const int va = ch | ((ch > 0) << 16), vb = cl | ((cl > 0) << 16);
+        int ia = va, ib = vb;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int na = __shfl_up_sync(0xffffffffu, ia, o), nbv = __shfl_up_sync(0xffffffffu, ib, o);
+            if (a.lane >= o) {
+                ia += na;
+                ib += nbv;
+            }
+        }
+        if (a.lane == 31) {
+            sh->wsum[0][a.aw] = ia;
+            sh->wsum[1][a.aw] = ib;
+        }
+        aux_sync();
+        int ba = 0, bb = 0, ta = 0;
+#pragma unroll
+        for (int w = 0; w < AUX_W; ++w) {
+            const int sa = sh->wsum[0][w], sb = sh->wsum[1][w];
+            if (w < a.aw) {
+                ba += sa;
+                bb += sb;
+            }
+            ta += sa;
+        }
+        const int ea = ba + ia - va, eb = bb + ib - vb;   // exclusive
+        const int n_hg = ta >> 16;
+        ax.off_hit[a.atid] = ea & 0xffff;
+        ax.off_low[a.atid] = eb & 0xffff;
+        if (ch > 0) ax.gtab[1 + (ea >> 16)] = GroupDesc{KIND_HIT, a.atid, ea & 0xffff, ch};
+        if (cl > 0) ax.gtab[1 + n_hg + (eb >> 16)] = GroupDesc{KIND_LOW, a.atid, eb & 0xffff, cl};
+        if (a.atid == AUX_T - 1) {   // this thread's inclusive sums are the totals
+            sh->n_hg = n_hg;
+            sh->n_lg = (bb + ib) >> 16;
+            ax.gtab[0] = GroupDesc{KIND_SHARED, 0, 0, T};
+        }
+    }
+    // coefficient of the shared expert's output: 1 + sum of LOWCONF gates, in k order
+#pragma unroll 1
+    for (int t = a.atid; t < T; t += AUX_T) {
+        float c = 1.0f;
+#pragma unroll 1
+        for (int k = 0; k < K; ++k)
+            if (ax.cls[t * K + k] == SPICE_LOWCONF) c += ax.gate[t * K + k];
+        ax.coef[t] = c;
+    }
+    aux_sync();
+    // position of every entry inside its group = offset of the group + number of earlier entries of the group
+#pragma unroll 1
+    for (int i = a.atid; i < n; i += AUX_T) {
+        const int key = ax.key[i];
+        int pos = -1;
+        if (key >= 0) {
+            int rank = 0;
+#pragma unroll 4
+            for (int j = 0; j < i; ++j) rank += ax.key[j] == key;
+            if (key < 1024) {
+                pos = ax.off_hit[key] + rank;
+                ax.perm_h[pos] = i;
+            } else {
+                pos = ax.off_low[key - 1024] + rank;
+                ax.perm_l[pos] = i;
+            }
+        }
+        ax.pos[i] = pos;
+    }
+    aux_sync();
+}
+
+// CTA 0: routing results for the caller (top-k, gates, classes, counts, residual-miss list in (t,k) order)
+__device__ __noinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, const AuxSmem &ax, const AuxCtx &a) {
+    const DecodeParams &p = q.p;
+    const int K = p.dm.K, n = p.dm.T * K;
+#pragma unroll 1
+    for (int i = a.atid; i < n; i += AUX_T) {
+        p.idx[i] = ax.idx[i];
+        p.gate[i] = ax.gate[i];
+        p.cls[i] = ax.cls[i];
+    }
+    if (a.aw == 0) {
+        int base = 0;
+#pragma unroll 1
+        for (int i0 = 0; i0 < n; i0 += 32) {
+            const int i = i0 + a.lane;
+            const bool miss = i < n && ax.cls[i] == SPICE_MISS_EXACT;
+            const unsigned m = __ballot_sync(0xffffffffu, miss);
+            if (miss && p.resid_tok) {
+                const int o = base + __popc(m & ((1u << a.lane) - 1u));
+                p.resid_tok[o] = i / K;
+                p.resid_k[o] = i % K;
+                p.resid_expert[o] = ax.idx[i];
+                p.resid_gate[o] = ax.gate[i];
+            }
+            base += __popc(m);
+        }
+        if (a.lane < 3) p.counts[a.lane] = sh->s_cnt[a.lane];
+    }
+}
+
+// combine: 1024 columns of one token
+__device__ __forceinline__ void aux_combine(const DtcParams &q, const AuxSmem &ax, const AuxCtx &a, int t, int blk) {
+    const DecodeParams &p = q.p;
+    const Dims &dm = p.dm;
+    const int j = blk * 1024 + a.atid * 4;
+    if (j >= dm.d) return;
+    const int d = dm.d, K = dm.K;
+    float4 sh4 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+    for (int s = 0; s < q.nsplit_sh; ++s) {
+        const float4 v = __ldcg(reinterpret_cast<const float4 *>(q.part_split + ((size_t)s * dm.T + t) * d + j));
+        sh4.x += v.x; sh4.y += v.y; sh4.z += v.z; sh4.w += v.w;
+    }
+    const float c = ax.coef[t];
+    float4 acc = make_float4(c * sh4.x, c * sh4.y, c * sh4.z, c * sh4.w);
+#pragma unroll 1
+    for (int k = 0; k < K; ++k) {
+        const int i = t * K + k;
+        if (ax.pos[i] < 0) continue;
+        const float g = ax.gate[i];
+        const float4 s = __ldcg(reinterpret_cast<const float4 *>(p.tb.part + (size_t)i * d + j));
+        acc.x = fmaf(g, s.x, acc.x); acc.y = fmaf(g, s.y, acc.y);
+        acc.z = fmaf(g, s.z, acc.z); acc.w = fmaf(g, s.w, acc.w);
+    }
+    if (p.y_cpu) {
+        const float4 s = *reinterpret_cast<const float4 *>(p.y_cpu + (size_t)t * d + j);
+        acc.x += s.x; acc.y += s.y; acc.z += s.z; acc.w += s.w;
+    }
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+    *reinterpret_cast<uint2 *>(p.y16 + (size_t)t * d + j) =
+        make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+    if (p.x_resid) {
+        const uint2 xr = *reinterpret_cast<const uint2 *>(p.x_resid + (size_t)t * d + j);
+        lo = __floats2bfloat162_rn(bf_lo(xr.x) + acc.x, bf_hi(xr.x) + acc.y);
+        hi = __floats2bfloat162_rn(bf_lo(xr.y) + acc.z, bf_hi(xr.y) + acc.w);
+        *reinterpret_cast<uint2 *>(p.x_resid + (size_t)t * d + j) =
+            make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+template <int NB>
+__global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_constant__ DtcParams q,
+                                                                   const __grid_constant__ DtcMaps maps) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr int STAGE_BYTES = A_BYTES + NB * 128;
+    constexpr int TMEM_COLS = 2 * NB < 32 ? 32 : 2 * NB;
+    const DecodeParams &p = q.p;
+    const Dims &dm = p.dm;
+    unsigned char *ring = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Ctl *sh = reinterpret_cast<Ctl *>(ring + (size_t)q.stages * STAGE_BYTES);
+    AuxSmem ax;
+    aux_layout(dm, p.conf_stride, NB, &ax, reinterpret_cast<unsigned char *>(sh) + ((sizeof(Ctl) + 15) & ~size_t(15)));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &sh->abort_flag;
+    const int stages = q.stages;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh->tmem_full[b]), 1);
+            mbar_init(smem_u32(&sh->tmem_empty[b]), 4);
+            mbar_init(smem_u32(&sh->xch_full[b]), 2);
+            mbar_init(smem_u32(&sh->xch_empty[b]), 2);
+        }
+        for (int s = 0; s < TQ; ++s) {
+            mbar_init(smem_u32(&sh->tq_full[s]), 1);
+            mbar_init(smem_u32(&sh->tq_empty[s]), 5);
+        }
+        mbar_init(smem_u32(&sh->plan_ready), 1);
+        mbar_init(smem_u32(&sh->mma_drain), 1);
+        sh->abort_flag = 0;
+        sh->aux_flag = 0;
+        sh->last_flag = 0;
+        sh->n_hg = sh->n_lg = 0;
+        for (int i = 0; i < 4; ++i) sh->s_cnt[i] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (one lane)
+        if (lane == 0) {
+            Plan pl;
+            plan_static(pl, q);
+            bool routed = false;
+            uint32_t it = 0, tcount = 0;
+            int s = 0;
+            uint32_t ring_phase = 0;   // parity of the current pass over the ring
+            int end = pl.nA;
+            bool ok = true;
+            for (int id = blockIdx.x; ok; id += gridDim.x) {
+                if (id >= end) {
+                    if (routed) break;
+                    if (!mb_wait(smem_u32(&sh->plan_ready), 0, abort_flag)) { ok = false; break; }
+                    routed = true;
+                    plan_routed(pl, sh->n_hg, sh->n_lg);
+                    end = pl.endC;
+                    if (id >= end) break;
+                }
+                // resolve the task: operands, k range, dependency
+                TaskDesc t{};
+                const CUtensorMap *ma, *mb;
+                int a_row0, a_row1 = -1, a_z = 0, b_z = 0, k0 = 0, dep = -1, dep_target = 0;
+                if (id < pl.endB) {
+                    t.nk = pl.kcd;
+                    mb = &maps.m[MAP_H];
+                    if (id < pl.nA + pl.nBh) {
+                        t.kind = TASK_ACT;
+                        if (id < pl.nA) {
+                            t.gi = 0;
+                            t.tile = id;
+                            ma = &maps.m[MAP_SH_GU];
+                            a_row0 = t.tile * 64;
+                            a_row1 = dm.Is + t.tile * 64;
+                        } else {
+                            const int l = id - pl.nA;
+                            t.gi = 1 + l / pl.tI;
+                            t.tile = l % pl.tI;
+                            ma = &maps.m[MAP_SLOT_GU];
+                            a_row0 = t.tile * 64;
+                            a_row1 = dm.I + t.tile * 64;
+                            a_z = ax.gtab[t.gi].id;
+                        }
+                    } else {
+                        const int l = id - pl.nA - pl.nBh;
+                        t.kind = TASK_Z;
+                        t.gi = 1 + pl.n_hg + l / pl.tz;
+                        t.tile = l % pl.tz;
+                        ma = &maps.m[MAP_LORE_A];
+                        a_row0 = t.tile * 128;
+                        a_z = ax.gtab[t.gi].id;
+                    }
+                } else {
+                    t.kind = TASK_DOWN;
+                    const int l = id - pl.endB;
+                    if (l < pl.nCs) {
+                        t.gi = 0;
+                        t.tile = l % pl.td;
+                        t.split = l / pl.td;
+                        k0 = t.split * pl.cps;
+                        t.nk = min(pl.cps, pl.kcIs - k0);
+                        ma = &maps.m[MAP_SH_D];
+                        mb = &maps.m[MAP_ACT_SH];
+                        dep = SY_GROUP0;
+                        dep_target = 4 * pl.tIs;
+                    } else if (l < pl.nCs + pl.nCh) {
+                        const int l2 = l - pl.nCs;
+                        t.gi = 1 + l2 / pl.td;
+                        t.tile = l2 % pl.td;
+                        t.nk = pl.kcI;
+                        ma = &maps.m[MAP_SLOT_D];
+                        mb = &maps.m[MAP_ACT_HIT];
+                        a_z = ax.gtab[t.gi].id;
+                        b_z = t.gi - 1;
+                        dep = SY_GROUP0 + t.gi;
+                        dep_target = 4 * pl.tI;
+                    } else {
+                        const int l2 = l - pl.nCs - pl.nCh;
+                        t.gi = 1 + pl.n_hg + l2 / pl.td;
+                        t.tile = l2 % pl.td;
+                        t.nk = pl.kcr;
+                        ma = &maps.m[MAP_LORE_B];
+                        mb = &maps.m[MAP_Z];
+                        a_z = ax.gtab[t.gi].id;
+                        b_z = t.gi - 1 - pl.n_hg;
+                        dep = SY_GROUP0 + t.gi;
+                        dep_target = 4 * pl.tz;
+                    }
+                    a_row0 = t.tile * 128;
+                }
+                if (dep >= 0) {
+                    if (!wait_ge(p.sync + dep, dep_target, p.sync, p.tb.status, p.spin_limit, abort_flag)) { ok = false; break; }
+                    fence_proxy_async();
+                }
+                {   // hand the task to the MMA and epilogue roles
+                    const int slot = tcount % TQ;
+                    if (!mb_wait(smem_u32(&sh->tq_empty[slot]), ((tcount / TQ) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    sh->tq[slot] = t;
+                    mbar_arrive(smem_u32(&sh->tq_full[slot]));
+                    ++tcount;
+                }
+                for (int kb = 0; kb < t.nk; ++kb, ++it) {
+                    if (!mb_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t full = smem_u32(&sh->full[s]);
+                    const uint32_t dst = smem_u32(ring + (size_t)s * STAGE_BYTES);
+                    const int kx = (k0 + kb) * 64;
+                    mbar_expect_tx(full, STAGE_BYTES);
+                    if (a_row1 >= 0) {
+                        tma_load_3d(dst, ma, kx, a_row0, a_z, full);
+                        tma_load_3d(dst + A_BYTES / 2, ma, kx, a_row1, a_z, full);
+                    } else {
+                        tma_load_3d(dst, ma, kx, a_row0, a_z, full);
+                    }
+                    tma_load_3d(dst + A_BYTES, mb, kx, 0, b_z, full);
+                    if (++s == stages) {
+                        s = 0;
+                        ring_phase ^= 1;
+                    }
+                }
+            }
+            if (ok) {   // tell the other roles that the list is exhausted
+                const int slot = tcount % TQ;
+                if (mb_wait(smem_u32(&sh->tq_empty[slot]), ((tcount / TQ) & 1) ^ 1, abort_flag)) {
+                    sh->tq[slot].kind = TASK_EXIT;
+                    mbar_arrive(smem_u32(&sh->tq_full[slot]));
+                }
+            }
+            // drain: every stage that was armed must have landed before the CTA may end
+            {
+                const uint32_t n_back = it < (uint32_t)stages ? it : (uint32_t)stages;
+                int ds = s;
+                uint32_t dph = ring_phase;
+                for (uint32_t j = 0; j < n_back; ++j) {
+                    if (--ds < 0) {
+                        ds = stages - 1;
+                        dph ^= 1;
+                    }
+                    mb_drain(smem_u32(&sh->full[ds]), dph);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (one lane)
+        if (lane == 0) {
+            constexpr uint32_t IDESC = make_idesc(128, NB);
+            int s = 0;
+            uint32_t ring_phase = 0;
+            for (uint32_t tcount = 0;; ++tcount) {
+                const int slot = tcount % TQ;
+                if (!mb_wait(smem_u32(&sh->tq_full[slot]), (tcount / TQ) & 1, abort_flag)) break;
+                const int kind = sh->tq[slot].kind, nk = sh->tq[slot].nk;
+                if (kind == TASK_EXIT) break;
+                const int buf = tcount & 1;
+                if (!mb_wait(smem_u32(&sh->tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * NB;
+                bool ok = true;
+                for (int kb = 0; kb < nk; ++kb) {
+                    if (!mb_wait(smem_u32(&sh->full[s]), ring_phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a0 = smem_u32(ring + (size_t)s * STAGE_BYTES), b0 = a0 + A_BYTES;
+                    const uint64_t da = make_desc(a0), db = make_desc(b0);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | k) ? 1u : 0u);
+                    tc_commit(smem_u32(&sh->empty[s]));
+                    if (++s == stages) {
+                        s = 0;
+                        ring_phase ^= 1;
+                    }
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&sh->tmem_full[buf]));
+                mbar_arrive(smem_u32(&sh->tq_empty[slot]));
+            }
+            // every MMA issued by this thread must have completed before the TMEM columns are given back
+            tc_commit(smem_u32(&sh->mma_drain));
+            mb_drain(smem_u32(&sh->mma_drain), 0);
+        }
+    } else if (warp < 6) {
+        // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 = weight rows of the tile
+        const int qd = warp & 3;
+        const int L = qd * 32 + lane;
+        uint32_t xc = 0;   // gate/up tiles seen (exchange buffer use count)
+        const int T = dm.T;
+        for (uint32_t tcount = 0;; ++tcount) {
+            const int slot = tcount % TQ;
+            if (!warp_mb_wait(smem_u32(&sh->tq_full[slot]), (tcount / TQ) & 1, abort_flag, lane)) break;
+            const TaskDesc t = sh->tq[slot];
+            if (t.kind == TASK_EXIT) break;
+            const int buf = tcount & 1;
+            if (!warp_mb_wait(smem_u32(&sh->tmem_full[buf]), (tcount >> 1) & 1, abort_flag, lane)) break;
+            tc_fence_after();
+            uint32_t v[NB];
+            const uint32_t t0 = tmem_base + buf * NB + ((uint32_t)(qd * 32) << 16);
+#pragma unroll
+            for (int c = 0; c < NB; c += 16) tc_ld16(t0 + c, &v[c]);
+            tc_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));   // accumulator is in registers now
+            const GroupDesc grp = t.gi == 0 ? GroupDesc{KIND_SHARED, 0, 0, T} : ax.gtab[t.gi];
+            int *ctr = p.sync + SY_GROUP0 + t.gi;
+            if (t.kind == TASK_ACT) {
+                const bool hit = grp.kind == KIND_HIT;
+                const int n_cols = hit ? dm.I : dm.Is;
+                __nv_bfloat16 *out = hit ? p.act_hit16 + (size_t)(t.gi - 1) * T * dm.I : p.act_shared16;
+                const int xb = xc & 1;
+                float *xch = ax.xch + xb * NB * 64;
+                if (qd >= 2) {   // up rows: park them for the warps that hold the gate rows
+                    if (!warp_mb_wait(smem_u32(&sh->xch_empty[xb]), ((xc >> 1) & 1) ^ 1, abort_flag, lane)) break;
+#pragma unroll
+                    for (int nn = 0; nn < NB; ++nn) xch[nn * 64 + (L - 64)] = __uint_as_float(v[nn]);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->xch_full[xb]));
+                } else {
+                    if (!warp_mb_wait(smem_u32(&sh->xch_full[xb]), (xc >> 1) & 1, abort_flag, lane)) break;
+                    const int col = t.tile * 64 + L;
+#pragma unroll
+                    for (int nn = 0; nn < NB; ++nn) {
+                        if (nn < T && col < n_cols) {
+                            const float u = xch[nn * 64 + L];
+                            out[(size_t)nn * n_cols + col] = __float2bfloat16(silu_f(__uint_as_float(v[nn])) * u);
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->xch_empty[xb]));
+                }
+                ++xc;
+            } else if (t.kind == TASK_Z) {
+                const int row = t.tile * 128 + L;
+                __nv_bfloat16 *out = p.z16 + (size_t)(t.gi - 1 - sh->n_hg) * T * dm.r;
+#pragma unroll
+                for (int nn = 0; nn < NB; ++nn)
+                    if (nn < T && row < dm.r) out[(size_t)nn * dm.r + row] = __float2bfloat16(__uint_as_float(v[nn]));
+            } else {
+                // down tile: column n belongs to entry ent[n] (the token's (t,k) entry routed to this group) or to nobody
+                int *ent = ax.ent + qd * NB;
+                for (int nn = lane; nn < NB; nn += 32) ent[nn] = -1;
+                __syncwarp();
+                if (grp.kind == KIND_SHARED) {
+                    for (int nn = lane; nn < T; nn += 32) ent[nn] = nn;
+                } else {
+                    const int *perm = grp.kind == KIND_HIT ? ax.perm_h : ax.perm_l;
+                    for (int qq = lane; qq < grp.m; qq += 32) {
+                        const int i = perm[grp.off + qq];
+                        ent[i / dm.K] = i;
+                    }
+                }
+                __syncwarp();
+                const int row = t.tile * 128 + L;
+                float *out = grp.kind == KIND_SHARED ? q.part_split + (size_t)t.split * T * dm.d : p.tb.part;
+#pragma unroll
+                for (int nn = 0; nn < NB; ++nn) {
+                    const int e = ent[nn];
+                    if (e >= 0 && row < dm.d) out[(size_t)e * dm.d + row] = __uint_as_float(v[nn]);
+                }
+                __syncwarp();   // ent[] is rewritten by the next down tile
+                ctr = p.sync + SY_P2_DONE;
+            }
+            fence_proxy_async();   // act / z rows are fetched by TMA in the tasks that depend on this one
+            __syncwarp();
+            if (lane == 0) {
+                red_release_add(ctr, 1);
+                mbar_arrive(smem_u32(&sh->tq_empty[slot]));
+            }
+        }
+    } else {
+        // ---------------- auxiliary team
+        AuxCtx a;
+        a.atid = threadIdx.x - AUX_T0;
+        a.lane = lane;
+        a.aw = a.atid >> 5;
+        const int T = dm.T, N = dm.N;
+        // while the logits are being produced: fetch what classification will need
+#pragma unroll 1
+        for (int i = a.atid; i < N; i += AUX_T) ax.soe[i] = p.w.slot_of_expert[i];
+        const int n_conf = p.conf_stride ? T * N : T;
+#pragma unroll 1
+        for (int i = a.atid; i < n_conf; i += AUX_T) ax.conf[i] = p.conf[i];
+        ax.cnt_hit[a.atid] = 0;
+        ax.cnt_low[a.atid] = 0;
+        aux_logits(q, a);
+        bool ok = aux_wait_ge(q, sh, a, p.sync + SY_R1_DONE, N * q.r1_sub);
+        if (ok) {
+            aux_route(q, sh, ax, a);
+            if (a.atid == 0) mbar_arrive(smem_u32(&sh->plan_ready));
+            if (blockIdx.x == 0) aux_write_outputs(q, sh, ax, a);
+            Plan pl;
+            plan_static(pl, q);
+            plan_routed(pl, sh->n_hg, sh->n_lg);
+            const int nb = (dm.d + 1023) >> 10, n_tasks = T * nb;
+            if ((int)blockIdx.x < n_tasks) {   // CTA-uniform
+                ok = aux_wait_ge(q, sh, a, p.sync + SY_P2_DONE, 4 * (pl.endC - pl.endB));
+                if (ok)
+                    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x) aux_combine(q, ax, a, task / nb, task % nb);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS));
+    }
+    // the last CTA to finish clears the counters for the next launch (after an abort the host does it)
+    if (threadIdx.x == 0) {
+        if (sh->abort_flag) atomicMax(p.tb.status, (int)SPICE_ERR_TIMEOUT);
+        __threadfence();
+        sh->last_flag = atomicAdd(p.sync + SY_TEAMS_DONE, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (sh->last_flag && !sh->abort_flag) {
+        __threadfence();
+        for (int i = threadIdx.x; i < p.sync_words; i += DTC_THREADS) p.sync[i] = 0;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+bool make_map3(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t mats, uint64_t mat_stride_elems,
+               uint32_t box_rows) {
+    return tc_encode_map3(m, base, cols, rows, mats, mat_stride_elems, box_rows);
+}
+
+size_t dtc_smem_bytes(const Dims &dm, int conf_stride, int stages) {
+    const int nb = nb_of(dm.T);
+    return 1024 + (size_t)stages * stage_bytes_of(nb) + ((sizeof(Ctl) + 15) & ~size_t(15)) + aux_layout(dm, conf_stride, nb, nullptr, nullptr);
+}
+
+int dtc_stages(const Dims &dm, int conf_stride, size_t max_smem) {
+    for (int s = MAX_STAGES; s >= 4; --s)
+        if (dtc_smem_bytes(dm, conf_stride, s) <= max_smem) return s;
+    return 0;
+}
+
+}  // namespace
+
+bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem) {
+    if (dm.T < 1 || dm.T > 64) return false;
+    if (dm.N > 256 || dm.S > 256) return false;
+    if ((size_t)dm.T * dm.K > 1024 || (size_t)dm.T * dm.N > 8192) return false;
+    if (dm.d % 8 || dm.I % 8 || dm.Is % 8 || dm.r % 8) return false;
+    const int kcIs = (dm.Is + 63) / 64;
+    if ((kcIs + CHUNKS_PER_SPLIT - 1) / CHUNKS_PER_SPLIT > MAX_SPLIT) return false;
+    return dtc_stages(dm, conf_stride, max_smem) >= 4;
+}
+
+int decode_tc_nsplit(const Dims &dm) {
+    const int kcIs = (dm.Is + 63) / 64;
+    return (kcIs + CHUNKS_PER_SPLIT - 1) / CHUNKS_PER_SPLIT;
+}
+
+int decode_tc_prepare(int max_smem_optin) {
+    const void *fns[3] = {reinterpret_cast<const void *>(decode_tc_kernel<16>), reinterpret_cast<const void *>(decode_tc_kernel<32>),
+                          reinterpret_cast<const void *>(decode_tc_kernel<64>)};
+    for (const void *fn : fns)
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem_optin) != cudaSuccess) return -1;
+    return 0;
+}
+
+int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int max_smem_optin, cudaStream_t st) {
+    const Dims &dm = p.dm;
+    DtcParams q;
+    q.p = p;
+    q.part_split = part_split;
+    q.stages = dtc_stages(dm, p.conf_stride, (size_t)max_smem_optin);
+    if (q.stages < 4) return -1;
+    const int kcIs = (dm.Is + 63) / 64;
+    q.nsplit_sh = decode_tc_nsplit(dm);
+    q.cps_sh = (kcIs + q.nsplit_sh - 1) / q.nsplit_sh;
+    {
+        const int per = (dm.T + AUX_W - 1) / AUX_W, fit = n_ctas / dm.N;
+        q.r1_sub = per < 1 ? 1 : per;
+        if (q.r1_sub > fit) q.r1_sub = fit < 1 ? 1 : fit;
+    }
+    const int nb = nb_of(dm.T);
+    const uint64_t T = dm.T, d = dm.d, I = dm.I, Is = dm.Is, r = dm.r;
+    const uint64_t n = T * dm.K, g_hit = (uint64_t)dm.S < n ? dm.S : n, g_low = (uint64_t)dm.N < n ? dm.N : n;
+    DtcMaps maps;
+    bool ok = true;
+    ok = ok && make_map3(&maps.m[MAP_H], p.h, d, T, 1, T * d, nb);
+    ok = ok && make_map3(&maps.m[MAP_SLOT_GU], p.w.slot_w_gate_up, d, 2 * I, dm.S, 2 * I * d, 64);
+    ok = ok && make_map3(&maps.m[MAP_SH_GU], p.w.shared_w_gate_up, d, 2 * Is, 1, 2 * Is * d, 64);
+    ok = ok && make_map3(&maps.m[MAP_LORE_A], p.w.lore_A, d, r, dm.N, r * d, 128);
+    ok = ok && make_map3(&maps.m[MAP_SLOT_D], p.w.slot_w_down, I, d, dm.S, d * I, 128);
+    ok = ok && make_map3(&maps.m[MAP_SH_D], p.w.shared_w_down, Is, d, 1, d * Is, 128);
+    ok = ok && make_map3(&maps.m[MAP_LORE_B], p.w.lore_B, r, d, dm.N, d * r, 128);
+    ok = ok && make_map3(&maps.m[MAP_ACT_HIT], p.act_hit16, I, T, g_hit, T * I, nb);
+    ok = ok && make_map3(&maps.m[MAP_ACT_SH], p.act_shared16, Is, T, 1, T * Is, nb);
+    ok = ok && make_map3(&maps.m[MAP_Z], p.z16, r, T, g_low, T * r, nb);
+    if (!ok) return -1;
+    const size_t smem = dtc_smem_bytes(dm, p.conf_stride, q.stages);
+    const void *fn = nb == 16 ? reinterpret_cast<const void *>(decode_tc_kernel<16>)
+                              : (nb == 32 ? reinterpret_cast<const void *>(decode_tc_kernel<32>)
+                                          : reinterpret_cast<const void *>(decode_tc_kernel<64>));
+    void *args[] = {&q, &maps};
+    if (cudaLaunchCooperativeKernel(fn, dim3(n_ctas), dim3(DTC_THREADS), args, smem, st) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
+    return 1;
+}
+
+}  // namespace spice

@@ -110,6 +110,12 @@ bool decode_supported(const Dims &dm, size_t max_smem);
 int decode_prepare(int max_smem_optin);
 int launch_decode(const DecodeParams &p, int n_ctas, cudaStream_t st);
 
+// ---- fused decode kernel on tcgen05 / TMA (decode_tc.cu); shares DecodeParams and the counter words
+bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem);
+int decode_tc_nsplit(const Dims &dm);   // K ranges of the shared expert's down projection (rows of part_split)
+int decode_tc_prepare(int max_smem_optin);
+int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int max_smem_optin, cudaStream_t st);
+
 // ---- tensor-core path for large batches (tc_gemm.cu)
 // One m-tile of the grouped problem: rows [row0, row0+rows) of the gathered activation buffer, all of
 // which use the weights of slot `slot`.
