@@ -14,8 +14,8 @@
 // One CTA per SM, 14 warps:
 //   warp 0      TMA producer: walks the task list, waits (bounded) for a task's dependency counter,
 //               queues the task for the other roles and streams its operands k-chunk by k-chunk
-//               (128 weight rows x 64 k + NB token rows x 64 k, 128-byte swizzle) into a
-//               shared-memory ring of up to 12 stages; mbarrier complete_tx
+//               (128 weight rows x 128 k + NB token rows x 128 k, as 64-k boxes with 128-byte swizzle) into a
+//               shared-memory ring of up to 5 stages of 128 k each; mbarrier complete_tx
 //   warp 1      issues tcgen05.mma (M = 128, N = NB, K = 16, bf16 -> fp32 in TMEM); accumulators are
 //               double-buffered; tcgen05.commit frees ring stages and publishes accumulators
 //   warps 2-5   epilogue: tcgen05.ld, SwiGLU (gate rows in TMEM lanes 0-63, up rows in lanes 64-127,
@@ -24,10 +24,12 @@
 //               REDUNDANTLY by every CTA from the logits (top-k, gates, classification, grouping):
 //               the tables land in shared memory without a second grid-wide hop; finally the combine
 //
-// Tasks (ids dealt round-robin to the CTAs; a task depends only on tasks with smaller ids):
+// Tasks (a CTA starts with the id of its index and draws every further id from a global counter; a task
+// depends only on tasks with smaller ids, and every CTA issues its tasks in increasing order):
 //   A  gate/up tile of the shared expert: 64 gate + 64 up rows, K = d              (no dependency)
+//      down tile of the shared expert: 128 rows, one K range                       (the A gate/up tiles)
 //   B  gate/up tile of a resident slot; A_e tile of a low-confidence expert        (routing)
-//   C  down tile, 128 rows: shared expert (K split into ranges), slot, B_e         (that group's B tiles)
+//   C  down tile, 128 rows, of a slot; B_e tile                                    (that group's B tiles)
 //   D  combine y_t = c_t S(h_t) + sum_k g_k part_{t,k}  (auxiliary teams)          (all C tiles)
 // Dependencies are counters in global memory: red.release by the finishing warp, bounded
 // ld.acquire polls by the waiting one.  Data written by plain stores and later fetched by TMA is
@@ -35,6 +37,7 @@
 // the CTA records SPICE_ERR_TIMEOUT, raises the abort flag, drains its copies in flight, frees
 // its TMEM and returns.  No load uses cluster multicast.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "route_device.cuh"
 #include "spice_internal.cuh"
@@ -48,9 +51,11 @@ using namespace tcdev;
 
 constexpr int DTC_THREADS = 448;
 constexpr int AUX_T0 = 192, AUX_T = 256, AUX_W = 8;
-constexpr int MAX_STAGES = 12, TQ = 4;
-constexpr int A_BYTES = 128 * 64 * 2;
-constexpr int MAX_SPLIT = 16, CHUNKS_PER_SPLIT = 32;
+constexpr int MAX_STAGES = 5, TQ = 4;   // deeper rings only lengthen the memory queues (every fence waits behind them)
+constexpr int KSTAGE = 128;                 // reduction elements per ring stage: two 64-element sub-chunks
+constexpr int SUB_A = 128 * 64 * 2;         // weight bytes of one sub-chunk
+constexpr int A_BYTES = 2 * SUB_A;
+constexpr int MAX_SPLIT = 16, CHUNKS_PER_SPLIT = 16;
 
 enum { TASK_EXIT = 0, TASK_ACT = 1, TASK_Z = 2, TASK_DOWN = 3 };
 enum { MAP_H = 0, MAP_SLOT_GU, MAP_SH_GU, MAP_LORE_A, MAP_SLOT_D, MAP_SH_D, MAP_LORE_B, MAP_ACT_HIT, MAP_ACT_SH, MAP_Z, N_MAPS };
@@ -135,7 +140,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
 }
 
 __host__ __device__ inline int nb_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
-__host__ __device__ inline int stage_bytes_of(int nb) { return A_BYTES + nb * 128; }
+__host__ __device__ inline int stage_bytes_of(int nb) { return A_BYTES + 2 * nb * 128; }
 
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ int ld_acquire(const int *p) {
@@ -150,6 +155,9 @@ __device__ __forceinline__ int ld_relaxed(const int *p) {
 }
 __device__ __forceinline__ void red_release_add(int *p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void aux_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
@@ -175,19 +183,44 @@ __device__ __forceinline__ unsigned long long now_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-constexpr unsigned long long ROLE_WAIT_NS = 1000000000ull;   // a role gives up after a second without progress
-constexpr unsigned long long DRAIN_WAIT_NS = 200000000ull;
+// Optional timeline recorder (compiled in only with -DSPICE_PROF; used while tuning).
+#ifdef SPICE_PROF
+constexpr int PR_CTAS = 148, PR_ROLES = 4, PR_EVENTS = 512;
+__device__ unsigned long long g_dtc_prof[PR_CTAS * PR_ROLES * PR_EVENTS * 2];
+#define DPROF(role, cnt, tag)                                                                 \
+    do {                                                                                      \
+        if (blockIdx.x < PR_CTAS && (cnt) < PR_EVENTS) {                                      \
+            const size_t o_ = (((size_t)blockIdx.x * PR_ROLES + (role)) * PR_EVENTS + (cnt)) * 2; \
+            g_dtc_prof[o_] = (unsigned long long)(tag);                                       \
+            g_dtc_prof[o_ + 1] = now_ns();                                                    \
+            ++(cnt);                                                                          \
+        }                                                                                     \
+    } while (0)
+#else
+#define DPROF(role, cnt, tag) \
+    do {                      \
+    } while (0)
+#endif
+#define APROF(a, tag)                                \
+    do {                                             \
+        if ((a).atid == 0) DPROF(2, (a).npf, tag);   \
+    } while (0)
 
-// mbarrier wait bounded by time (a try_wait may itself suspend the thread for a while, so polls are not a
-// measure); false when the limit expired or another role already gave up
+// limits in SM clock cycles (clock64 is a cheap local counter; the global timer costs about a microsecond to read)
+constexpr long long ROLE_WAIT_CYCLES = 2000000000ll;   // a role gives up after about a second without progress
+constexpr long long DRAIN_WAIT_CYCLES = 400000000ll;
+
+// mbarrier wait bounded by elapsed cycles (a try_wait may itself suspend the thread for a while, so polls are
+// not a measure); false when the limit expired or another role already gave up
 __device__ __forceinline__ bool mb_wait(uint32_t a, uint32_t parity, volatile int *abort_flag) {
     if (mbar_try(a, parity)) return true;
-    const unsigned long long t0 = now_ns();
+    const long long t0 = clock64();
     for (uint32_t i = 1;; ++i) {
         if (mbar_try(a, parity)) return true;
+        if (i > 16u) __nanosleep(20);   // leave the issue slots to the warps that have work
         if ((i & 31u) == 0u) {
             if (*abort_flag) return false;
-            if (now_ns() - t0 > ROLE_WAIT_NS) break;
+            if (clock64() - t0 > ROLE_WAIT_CYCLES) break;
         }
     }
     *abort_flag = 1;
@@ -195,10 +228,10 @@ __device__ __forceinline__ bool mb_wait(uint32_t a, uint32_t parity, volatile in
 }
 // the same without the abort check, for waits that must outlast an abort (copies / MMAs in flight)
 __device__ __forceinline__ void mb_drain(uint32_t a, uint32_t parity) {
-    const unsigned long long t0 = now_ns();
+    const long long t0 = clock64();
     for (uint32_t i = 1;; ++i) {
         if (mbar_try(a, parity)) return;
-        if ((i & 31u) == 0u && now_ns() - t0 > DRAIN_WAIT_NS) return;
+        if ((i & 31u) == 0u && clock64() - t0 > DRAIN_WAIT_CYCLES) return;
     }
 }
 
@@ -215,10 +248,11 @@ __device__ __forceinline__ bool warp_mb_wait(uint32_t a, uint32_t parity, volati
 // Task list.  ids [0, nA) are known at launch; the rest once the routing tables exist.
 struct Plan {
     int tIs, tI, tz, td;            // tiles per matrix
-    int kcd, kcI, kcr;              // k-chunks (64 elements) of d, I, r
+    int kcd, kcI, kcr;              // k-chunks (one ring stage = 128 elements) of d, I, r
     int nsplit, cps, kcIs;          // shared down projection: K ranges, chunks per range, chunks in all
     int nA, nBh, endB, nCs, nCh, endC;
     int n_hg, n_lg;
+    int sh_early;                   // the shared down tiles are part of phase A (else they follow phase B)
 };
 
 __device__ __forceinline__ void plan_static(Plan &pl, const DtcParams &q) {
@@ -227,14 +261,18 @@ __device__ __forceinline__ void plan_static(Plan &pl, const DtcParams &q) {
     pl.tI = (dm.I + 63) >> 6;
     pl.tz = (dm.r + 127) >> 7;
     pl.td = (dm.d + 127) >> 7;
-    pl.kcd = (dm.d + 63) >> 6;
-    pl.kcI = (dm.I + 63) >> 6;
-    pl.kcr = (dm.r + 63) >> 6;
-    pl.kcIs = (dm.Is + 63) >> 6;
+    pl.kcd = (dm.d + KSTAGE - 1) / KSTAGE;
+    pl.kcI = (dm.I + KSTAGE - 1) / KSTAGE;
+    pl.kcr = (dm.r + KSTAGE - 1) / KSTAGE;
+    pl.kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
     pl.nsplit = q.nsplit_sh;
     pl.cps = q.cps_sh;
-    pl.nA = pl.tIs;
-    pl.n_hg = pl.n_lg = pl.nBh = pl.nCs = pl.nCh = 0;
+    pl.nCs = pl.td * pl.nsplit;
+    // Before the routing is known only the shared expert can be worked on.  Its down tiles wait for ALL its
+    // gate/up tiles, so they go first only when the CTAs that take them would have nothing else to do.
+    pl.sh_early = (pl.tIs + pl.nCs <= (int)gridDim.x) ? 1 : 0;
+    pl.nA = pl.tIs + (pl.sh_early ? pl.nCs : 0);
+    pl.n_hg = pl.n_lg = pl.nBh = pl.nCh = 0;
     pl.endB = pl.endC = pl.nA;
 }
 __device__ __forceinline__ void plan_routed(Plan &pl, int n_hg, int n_lg) {
@@ -242,15 +280,15 @@ __device__ __forceinline__ void plan_routed(Plan &pl, int n_hg, int n_lg) {
     pl.n_lg = n_lg;
     pl.nBh = n_hg * pl.tI;
     pl.endB = pl.nA + pl.nBh + n_lg * pl.tz;
-    pl.nCs = pl.td * pl.nsplit;
     pl.nCh = n_hg * pl.td;
-    pl.endC = pl.endB + pl.nCs + pl.nCh + n_lg * pl.td;
+    pl.endC = pl.endB + (pl.sh_early ? 0 : pl.nCs) + pl.nCh + n_lg * pl.td;
 }
 
 // ------------------------------------------------------------------------------------------
 // Auxiliary team
 struct AuxCtx {
     int atid, lane, aw;
+    int npf;   // timeline events recorded (tuning builds only)
 };
 
 // leader polls, result broadcast through shared memory: team-uniform
@@ -288,27 +326,45 @@ __device__ __noinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) {
 // Routing decisions from the logits, entirely in shared memory.  Every CTA computes the same tables
 // (the code is deterministic: counts by atomics, positions by ranking); CTA 0 also writes the outputs.
 // The arithmetic of the gates is that of warp_topk_gates (route_device.cuh).
-__device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, const AuxCtx &a) {
+__device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
     const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
+    // all of this thread's logits are requested before the first one is parked
 #pragma unroll 1
-    for (int i = a.atid; i < T * N; i += AUX_T) {
-        const float v = __ldcg(p.logits + i);
-        ax.lg[i] = (v == v) ? v : -INFINITY;   // NaN never wins
+    for (int i0 = a.atid; i0 < T * N; i0 += AUX_T * 4) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = (i0 + u * AUX_T < T * N) ? __ldcg(p.logits + i0 + u * AUX_T) : 0.f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (i0 + u * AUX_T < T * N) ax.lg[i0 + u * AUX_T] = (v[u] == v[u]) ? v[u] : -INFINITY;   // NaN never wins
     }
     aux_sync();
-    // winners by ranking: rank = #{j : l_j > l_e or (l_j == l_e and j < e)}
+    APROF(a, 70);
+    // winners by ranking: rank = #{j : l_j > l_e or (l_j == l_e and j < e)}; 16 candidates are read per step
+    // (four 128-bit reads issued together) so the compare chain never waits for shared memory
 #pragma unroll 1
     for (int i = a.atid; i < T * N; i += AUX_T) {
         const int t = i / N, e = i - t * N;
         const float *l = ax.lg + t * N;
         const float v = l[e];
         int rank = 0;
-#pragma unroll 8
-        for (int j = 0; j < N; ++j) {
+        int j = 0;
+        if ((N & 3) == 0) {
+            const float4 *l4 = reinterpret_cast<const float4 *>(l);
+#pragma unroll 1
+            for (; j + 16 <= N; j += 16) {
+                const float4 q0 = l4[(j >> 2)], q1 = l4[(j >> 2) + 1], q2 = l4[(j >> 2) + 2], q3 = l4[(j >> 2) + 3];
+                const float u[16] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w, q2.x, q2.y, q2.z, q2.w, q3.x, q3.y, q3.z, q3.w};
+#pragma unroll
+                for (int c = 0; c < 16; ++c) rank += (int)(u[c] > v) | ((int)(u[c] == v) & (int)(j + c < e));
+            }
+        }
+#pragma unroll 1
+        for (; j < N; ++j) {
             const float u = l[j];
-            rank += (u > v) || (u == v && j < e);
+            rank += (int)(u > v) | ((int)(u == v) & (int)(j < e));
         }
         if (rank < K) {
             ax.idx[t * K + rank] = e;
@@ -316,6 +372,7 @@ __device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSme
         }
     }
     aux_sync();
+    APROF(a, 71);
     // gates: p_k = exp(l_k - l_0); denominator = sum over the winners in k order, or the full softmax sum
 #pragma unroll 1
     for (int t = a.aw; t < T; t += AUX_W) {
@@ -338,6 +395,7 @@ __device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSme
         if (a.lane < K) ax.gate[t * K + a.lane] = pk / denom;
     }
     aux_sync();
+    APROF(a, 72);
     // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
 #pragma unroll 1
     for (int i = a.atid; i < n; i += AUX_T) {
@@ -365,6 +423,7 @@ __device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSme
         atomicAdd(&sh->s_cnt[c], 1);
     }
     aux_sync();
+    APROF(a, 73);
     // groups: thread i owns slot i and expert i; packed scan of (entries, non-empty flag << 16)
     {
         const int ch = a.atid < S ? ax.cnt_hit[a.atid] : 0, cl = a.atid < N ? ax.cnt_low[a.atid] : 0;
@@ -415,15 +474,24 @@ __device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSme
         ax.coef[t] = c;
     }
     aux_sync();
+    APROF(a, 74);
     // position of every entry inside its group = offset of the group + number of earlier entries of the group
 #pragma unroll 1
     for (int i = a.atid; i < n; i += AUX_T) {
         const int key = ax.key[i];
         int pos = -1;
         if (key >= 0) {
-            int rank = 0;
-#pragma unroll 4
-            for (int j = 0; j < i; ++j) rank += ax.key[j] == key;
+            int rank = 0, j = 0;
+            const int4 *k4 = reinterpret_cast<const int4 *>(ax.key);
+#pragma unroll 1
+            for (; j + 16 <= i; j += 16) {
+                const int4 q0 = k4[(j >> 2)], q1 = k4[(j >> 2) + 1], q2 = k4[(j >> 2) + 2], q3 = k4[(j >> 2) + 3];
+                rank += (q0.x == key) + (q0.y == key) + (q0.z == key) + (q0.w == key) + (q1.x == key) + (q1.y == key) +
+                        (q1.z == key) + (q1.w == key) + (q2.x == key) + (q2.y == key) + (q2.z == key) + (q2.w == key) +
+                        (q3.x == key) + (q3.y == key) + (q3.z == key) + (q3.w == key);
+            }
+#pragma unroll 1
+            for (; j < i; ++j) rank += ax.key[j] == key;
             if (key < 1024) {
                 pos = ax.off_hit[key] + rank;
                 ax.perm_h[pos] = i;
@@ -467,29 +535,45 @@ __device__ __noinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, cons
     }
 }
 
-// combine: 1024 columns of one token
-__device__ __forceinline__ void aux_combine(const DtcParams &q, const AuxSmem &ax, const AuxCtx &a, int t, int blk) {
+// combine: 256 columns of one token per 64-thread unit; the reads of up to 8 entries are in flight together
+__device__ __forceinline__ void aux_combine(const DtcParams &q, const AuxSmem &ax, int t, int j) {
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
-    const int j = blk * 1024 + a.atid * 4;
     if (j >= dm.d) return;
     const int d = dm.d, K = dm.K;
     float4 sh4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-    for (int s = 0; s < q.nsplit_sh; ++s) {
-        const float4 v = __ldcg(reinterpret_cast<const float4 *>(q.part_split + ((size_t)s * dm.T + t) * d + j));
-        sh4.x += v.x; sh4.y += v.y; sh4.z += v.z; sh4.w += v.w;
+    for (int s0 = 0; s0 < q.nsplit_sh; s0 += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (s0 + u < q.nsplit_sh)
+                v[u] = __ldcg(reinterpret_cast<const float4 *>(q.part_split + ((size_t)(s0 + u) * dm.T + t) * d + j));
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (s0 + u < q.nsplit_sh) {
+                sh4.x += v[u].x; sh4.y += v[u].y; sh4.z += v[u].z; sh4.w += v[u].w;
+            }
     }
     const float c = ax.coef[t];
     float4 acc = make_float4(c * sh4.x, c * sh4.y, c * sh4.z, c * sh4.w);
 #pragma unroll 1
-    for (int k = 0; k < K; ++k) {
-        const int i = t * K + k;
-        if (ax.pos[i] < 0) continue;
-        const float g = ax.gate[i];
-        const float4 s = __ldcg(reinterpret_cast<const float4 *>(p.tb.part + (size_t)i * d + j));
-        acc.x = fmaf(g, s.x, acc.x); acc.y = fmaf(g, s.y, acc.y);
-        acc.z = fmaf(g, s.z, acc.z); acc.w = fmaf(g, s.w, acc.w);
+    for (int k0 = 0; k0 < K; k0 += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = t * K + k0 + u;
+            if (k0 + u < K && ax.pos[i] >= 0) v[u] = __ldcg(reinterpret_cast<const float4 *>(p.tb.part + (size_t)i * d + j));
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = t * K + k0 + u;
+            if (k0 + u < K && ax.pos[i] >= 0) {
+                const float g = ax.gate[i];
+                acc.x = fmaf(g, v[u].x, acc.x); acc.y = fmaf(g, v[u].y, acc.y);
+                acc.z = fmaf(g, v[u].z, acc.z); acc.w = fmaf(g, v[u].w, acc.w);
+            }
+        }
     }
     if (p.y_cpu) {
         const float4 s = *reinterpret_cast<const float4 *>(p.y_cpu + (size_t)t * d + j);
@@ -512,7 +596,7 @@ template <int NB>
 __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_constant__ DtcParams q,
                                                                    const __grid_constant__ DtcMaps maps) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    constexpr int STAGE_BYTES = A_BYTES + NB * 128;
+    constexpr int STAGE_BYTES = A_BYTES + 2 * NB * 128;
     constexpr int TMEM_COLS = 2 * NB < 32 ? 32 : 2 * NB;
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
@@ -558,20 +642,37 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
     const uint32_t tmem_base = sh->tmem_base;
 
     if (warp == 0) {
-        // ---------------- TMA producer (one lane)
-        if (lane == 0) {
+        // ---------------- TMA producer: lane 0 drives, lanes 0-5 each issue one of a stage's copies.  A stage holds
+        // two 64-element sub-chunks: waiting for a free stage, arming it and issuing a copy cost a thread a few hundred
+        // cycles whatever the size, so the stage is made large and its copies are issued side by side.
+        constexpr unsigned PM = 0x3Fu;
+        if (lane < 6) {
             Plan pl;
             plan_static(pl, q);
             bool routed = false;
+            int npf = 0;
+            if (lane == 0) DPROF(0, npf, 1);
             uint32_t it = 0, tcount = 0;
             int s = 0;
             uint32_t ring_phase = 0;   // parity of the current pass over the ring
             int end = pl.nA;
             bool ok = true;
-            for (int id = blockIdx.x; ok; id += gridDim.x) {
+            // ids: the first one is the CTA's index, every later one is drawn from a global counter.  The draw is
+            // issued a whole task ahead of its use, so its latency hides behind the task's copies.
+            int id = blockIdx.x;
+            auto lead_wait = [&](uint32_t bar, uint32_t parity) {   // lane 0 waits, the outcome is uniform
+                int r = 1;
+                if (lane == 0) r = mb_wait(bar, parity, abort_flag) ? 1 : 0;
+                return __shfl_sync(PM, r, 0) != 0;
+            };
+            while (ok) {
+                int drawn = 0;
+                if (lane == 0) drawn = (int)gridDim.x + atomicAdd(p.sync + SY_NEXT_TASK, 1);
                 if (id >= end) {
                     if (routed) break;
-                    if (!mb_wait(smem_u32(&sh->plan_ready), 0, abort_flag)) { ok = false; break; }
+                    if (lane == 0) DPROF(0, npf, 30);
+                    if (!lead_wait(smem_u32(&sh->plan_ready), 0)) { ok = false; break; }
+                    if (lane == 0) DPROF(0, npf, 31);
                     routed = true;
                     plan_routed(pl, sh->n_hg, sh->n_lg);
                     end = pl.endC;
@@ -581,104 +682,122 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 TaskDesc t{};
                 const CUtensorMap *ma, *mb;
                 int a_row0, a_row1 = -1, a_z = 0, b_z = 0, k0 = 0, dep = -1, dep_target = 0;
-                if (id < pl.endB) {
+                const int c0 = pl.endB + (pl.sh_early ? 0 : pl.nCs);   // first down tile of a slot
+                const bool sh_down = pl.sh_early ? (id >= pl.tIs && id < pl.nA) : (id >= pl.endB && id < c0);
+                if (id < pl.tIs) {                       // gate/up tile of the shared expert
+                    t.kind = TASK_ACT;
+                    t.tile = id;
                     t.nk = pl.kcd;
+                    ma = &maps.m[MAP_SH_GU];
                     mb = &maps.m[MAP_H];
-                    if (id < pl.nA + pl.nBh) {
-                        t.kind = TASK_ACT;
-                        if (id < pl.nA) {
-                            t.gi = 0;
-                            t.tile = id;
-                            ma = &maps.m[MAP_SH_GU];
-                            a_row0 = t.tile * 64;
-                            a_row1 = dm.Is + t.tile * 64;
-                        } else {
-                            const int l = id - pl.nA;
-                            t.gi = 1 + l / pl.tI;
-                            t.tile = l % pl.tI;
-                            ma = &maps.m[MAP_SLOT_GU];
-                            a_row0 = t.tile * 64;
-                            a_row1 = dm.I + t.tile * 64;
-                            a_z = ax.gtab[t.gi].id;
-                        }
-                    } else {
-                        const int l = id - pl.nA - pl.nBh;
-                        t.kind = TASK_Z;
-                        t.gi = 1 + pl.n_hg + l / pl.tz;
-                        t.tile = l % pl.tz;
-                        ma = &maps.m[MAP_LORE_A];
-                        a_row0 = t.tile * 128;
-                        a_z = ax.gtab[t.gi].id;
-                    }
-                } else {
+                    a_row0 = t.tile * 64;
+                    a_row1 = dm.Is + t.tile * 64;
+                } else if (sh_down) {                    // down tile of the shared expert, one K range
+                    const int l = id - (pl.sh_early ? pl.tIs : pl.endB);
                     t.kind = TASK_DOWN;
-                    const int l = id - pl.endB;
-                    if (l < pl.nCs) {
-                        t.gi = 0;
-                        t.tile = l % pl.td;
-                        t.split = l / pl.td;
-                        k0 = t.split * pl.cps;
-                        t.nk = min(pl.cps, pl.kcIs - k0);
-                        ma = &maps.m[MAP_SH_D];
-                        mb = &maps.m[MAP_ACT_SH];
-                        dep = SY_GROUP0;
-                        dep_target = 4 * pl.tIs;
-                    } else if (l < pl.nCs + pl.nCh) {
-                        const int l2 = l - pl.nCs;
-                        t.gi = 1 + l2 / pl.td;
-                        t.tile = l2 % pl.td;
-                        t.nk = pl.kcI;
-                        ma = &maps.m[MAP_SLOT_D];
-                        mb = &maps.m[MAP_ACT_HIT];
-                        a_z = ax.gtab[t.gi].id;
-                        b_z = t.gi - 1;
-                        dep = SY_GROUP0 + t.gi;
-                        dep_target = 4 * pl.tI;
-                    } else {
-                        const int l2 = l - pl.nCs - pl.nCh;
-                        t.gi = 1 + pl.n_hg + l2 / pl.td;
-                        t.tile = l2 % pl.td;
-                        t.nk = pl.kcr;
-                        ma = &maps.m[MAP_LORE_B];
-                        mb = &maps.m[MAP_Z];
-                        a_z = ax.gtab[t.gi].id;
-                        b_z = t.gi - 1 - pl.n_hg;
-                        dep = SY_GROUP0 + t.gi;
-                        dep_target = 4 * pl.tz;
-                    }
+                    t.tile = l % pl.td;
+                    t.split = l / pl.td;
+                    k0 = t.split * pl.cps;
+                    t.nk = min(pl.cps, pl.kcIs - k0);
+                    ma = &maps.m[MAP_SH_D];
+                    mb = &maps.m[MAP_ACT_SH];
                     a_row0 = t.tile * 128;
+                    dep = SY_GROUP0;
+                    dep_target = 4 * pl.tIs;
+                } else if (id < pl.nA + pl.nBh) {        // gate/up tile of a resident slot
+                    const int l = id - pl.nA;
+                    t.kind = TASK_ACT;
+                    t.gi = 1 + l / pl.tI;
+                    t.tile = l % pl.tI;
+                    t.nk = pl.kcd;
+                    ma = &maps.m[MAP_SLOT_GU];
+                    mb = &maps.m[MAP_H];
+                    a_row0 = t.tile * 64;
+                    a_row1 = dm.I + t.tile * 64;
+                    a_z = ax.gtab[t.gi].id;
+                } else if (id < pl.endB) {               // A_e tile of a low-confidence expert
+                    const int l = id - pl.nA - pl.nBh;
+                    t.kind = TASK_Z;
+                    t.gi = 1 + pl.n_hg + l / pl.tz;
+                    t.tile = l % pl.tz;
+                    t.nk = pl.kcd;
+                    ma = &maps.m[MAP_LORE_A];
+                    mb = &maps.m[MAP_H];
+                    a_row0 = t.tile * 128;
+                    a_z = ax.gtab[t.gi].id;
+                } else if (id < c0 + pl.nCh) {           // down tile of a resident slot
+                    const int l = id - c0;
+                    t.kind = TASK_DOWN;
+                    t.gi = 1 + l / pl.td;
+                    t.tile = l % pl.td;
+                    t.nk = pl.kcI;
+                    ma = &maps.m[MAP_SLOT_D];
+                    mb = &maps.m[MAP_ACT_HIT];
+                    a_row0 = t.tile * 128;
+                    a_z = ax.gtab[t.gi].id;
+                    b_z = t.gi - 1;
+                    dep = SY_GROUP0 + t.gi;
+                    dep_target = 4 * pl.tI;
+                } else {                                 // B_e tile of a low-confidence expert
+                    const int l = id - c0 - pl.nCh;
+                    t.kind = TASK_DOWN;
+                    t.gi = 1 + pl.n_hg + l / pl.td;
+                    t.tile = l % pl.td;
+                    t.nk = pl.kcr;
+                    ma = &maps.m[MAP_LORE_B];
+                    mb = &maps.m[MAP_Z];
+                    a_row0 = t.tile * 128;
+                    a_z = ax.gtab[t.gi].id;
+                    b_z = t.gi - 1 - pl.n_hg;
+                    dep = SY_GROUP0 + t.gi;
+                    dep_target = 4 * pl.tz;
                 }
+                if (lane == 0) DPROF(0, npf, 10 + t.kind);
                 if (dep >= 0) {
-                    if (!wait_ge(p.sync + dep, dep_target, p.sync, p.tb.status, p.spin_limit, abort_flag)) { ok = false; break; }
+                    int r = 1;
+                    if (lane == 0) r = wait_ge(p.sync + dep, dep_target, p.sync, p.tb.status, p.spin_limit, abort_flag) ? 1 : 0;
+                    __syncwarp(PM);
+                    if (__shfl_sync(PM, r, 0) == 0) { ok = false; break; }
+                    if (lane == 0) DPROF(0, npf, 22);
                     fence_proxy_async();
+                    if (lane == 0) DPROF(0, npf, 23);
                 }
                 {   // hand the task to the MMA and epilogue roles
                     const int slot = tcount % TQ;
-                    if (!mb_wait(smem_u32(&sh->tq_empty[slot]), ((tcount / TQ) & 1) ^ 1, abort_flag)) { ok = false; break; }
-                    sh->tq[slot] = t;
-                    mbar_arrive(smem_u32(&sh->tq_full[slot]));
+                    if (!lead_wait(smem_u32(&sh->tq_empty[slot]), ((tcount / TQ) & 1) ^ 1)) { ok = false; break; }
+                    if (lane == 0) {
+                        sh->tq[slot] = t;
+                        mbar_arrive(smem_u32(&sh->tq_full[slot]));
+                    }
                     ++tcount;
                 }
+                if (lane == 0) DPROF(0, npf, 21);
+                // this lane's copy of every stage: lanes 0,1 the (first) weight box of sub-chunk 0,1; lanes 2,3 the
+                // second weight box (up rows); lanes 4,5 the tokens
+                const int sub = lane & 1, what = lane >> 1;
+                const CUtensorMap *my_map = what == 2 ? mb : ma;
+                const uint32_t my_off = what == 2 ? (uint32_t)(A_BYTES + sub * NB * 128)
+                                                  : (uint32_t)(sub * SUB_A + (what == 1 ? SUB_A / 2 : 0));
+                const int my_y = what == 0 ? a_row0 : (what == 1 ? a_row1 : 0);
+                const int my_z = what == 2 ? b_z : a_z;
+                const bool my_on = what != 1 || a_row1 >= 0;
                 for (int kb = 0; kb < t.nk; ++kb, ++it) {
-                    if (!mb_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1, abort_flag)) { ok = false; break; }
+                    if (!lead_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1)) { ok = false; break; }
                     const uint32_t full = smem_u32(&sh->full[s]);
                     const uint32_t dst = smem_u32(ring + (size_t)s * STAGE_BYTES);
-                    const int kx = (k0 + kb) * 64;
-                    mbar_expect_tx(full, STAGE_BYTES);
-                    if (a_row1 >= 0) {
-                        tma_load_3d(dst, ma, kx, a_row0, a_z, full);
-                        tma_load_3d(dst + A_BYTES / 2, ma, kx, a_row1, a_z, full);
-                    } else {
-                        tma_load_3d(dst, ma, kx, a_row0, a_z, full);
-                    }
-                    tma_load_3d(dst + A_BYTES, mb, kx, 0, b_z, full);
+                    const int kx = (k0 + kb) * KSTAGE + sub * 64;
+                    if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
+                    __syncwarp(PM);
+                    if (my_on) tma_load_3d(dst + my_off, my_map, kx, my_y, my_z, full);
                     if (++s == stages) {
                         s = 0;
                         ring_phase ^= 1;
                     }
                 }
+                id = __shfl_sync(PM, drawn, 0);
             }
-            if (ok) {   // tell the other roles that the list is exhausted
+            if (lane == 0) DPROF(0, npf, 40);
+            if (ok && lane == 0) {   // tell the other roles that the list is exhausted
                 const int slot = tcount % TQ;
                 if (mb_wait(smem_u32(&sh->tq_empty[slot]), ((tcount / TQ) & 1) ^ 1, abort_flag)) {
                     sh->tq[slot].kind = TASK_EXIT;
@@ -686,7 +805,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 }
             }
             // drain: every stage that was armed must have landed before the CTA may end
-            {
+            if (lane == 0) {
                 const uint32_t n_back = it < (uint32_t)stages ? it : (uint32_t)stages;
                 int ds = s;
                 uint32_t dph = ring_phase;
@@ -703,6 +822,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         // ---------------- MMA issuer (one lane)
         if (lane == 0) {
             constexpr uint32_t IDESC = make_idesc(128, NB);
+#ifdef SPICE_PROF_STAGES
+            int npf_m = 0;
+#endif
             int s = 0;
             uint32_t ring_phase = 0;
             for (uint32_t tcount = 0;; ++tcount) {
@@ -717,11 +839,17 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 bool ok = true;
                 for (int kb = 0; kb < nk; ++kb) {
                     if (!mb_wait(smem_u32(&sh->full[s]), ring_phase, abort_flag)) { ok = false; break; }
+#ifdef SPICE_PROF_STAGES
+                    if (npf_m < 48) DPROF(3, npf_m, 91);
+#endif
                     tc_fence_after();
                     const uint32_t a0 = smem_u32(ring + (size_t)s * STAGE_BYTES), b0 = a0 + A_BYTES;
-                    const uint64_t da = make_desc(a0), db = make_desc(b0);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | k) ? 1u : 0u);
+                    for (int c = 0; c < 2; ++c) {
+                        const uint64_t da = make_desc(a0 + c * SUB_A), db = make_desc(b0 + c * NB * 128);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | c | k) ? 1u : 0u);
+                    }
                     tc_commit(smem_u32(&sh->empty[s]));
                     if (++s == stages) {
                         s = 0;
@@ -741,14 +869,18 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         const int qd = warp & 3;
         const int L = qd * 32 + lane;
         uint32_t xc = 0;   // gate/up tiles seen (exchange buffer use count)
+        int n_down = 0;    // down tiles finished by this warp, published once: only the combine waits for them
         const int T = dm.T;
+        int npf = 0;
         for (uint32_t tcount = 0;; ++tcount) {
             const int slot = tcount % TQ;
             if (!warp_mb_wait(smem_u32(&sh->tq_full[slot]), (tcount / TQ) & 1, abort_flag, lane)) break;
             const TaskDesc t = sh->tq[slot];
             if (t.kind == TASK_EXIT) break;
             const int buf = tcount & 1;
+            if (warp == 2 && lane == 0) DPROF(1, npf, 50 + t.kind);
             if (!warp_mb_wait(smem_u32(&sh->tmem_full[buf]), (tcount >> 1) & 1, abort_flag, lane)) break;
+            if (warp == 2 && lane == 0) DPROF(1, npf, 54);
             tc_fence_after();
             uint32_t v[NB];
             const uint32_t t0 = tmem_base + buf * NB + ((uint32_t)(qd * 32) << 16);
@@ -758,6 +890,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));   // accumulator is in registers now
+            if (warp == 2 && lane == 0) DPROF(1, npf, 56);
             const GroupDesc grp = t.gi == 0 ? GroupDesc{KIND_SHARED, 0, 0, T} : ax.gtab[t.gi];
             int *ctr = p.sync + SY_GROUP0 + t.gi;
             if (t.kind == TASK_ACT) {
@@ -815,44 +948,74 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     if (e >= 0 && row < dm.d) out[(size_t)e * dm.d + row] = __uint_as_float(v[nn]);
                 }
                 __syncwarp();   // ent[] is rewritten by the next down tile
-                ctr = p.sync + SY_P2_DONE;
             }
-            fence_proxy_async();   // act / z rows are fetched by TMA in the tasks that depend on this one
-            __syncwarp();
-            if (lane == 0) {
-                red_release_add(ctr, 1);
-                mbar_arrive(smem_u32(&sh->tq_empty[slot]));
+            if (warp == 2 && lane == 0) DPROF(1, npf, 57);
+            if (t.kind == TASK_DOWN) {
+                ++n_down;
+                if (lane == 0) mbar_arrive(smem_u32(&sh->tq_empty[slot]));
+            } else {
+                fence_proxy_async();   // act / z rows are fetched by TMA in the tasks that depend on this one
+                __syncwarp();
+                if (warp == 2 && lane == 0) DPROF(1, npf, 58);
+                if (lane == 0) {
+                    red_release_add(ctr, 1);
+                    mbar_arrive(smem_u32(&sh->tq_empty[slot]));
+                }
             }
+            if (warp == 2 && lane == 0) DPROF(1, npf, 55);
         }
+        __syncwarp();
+        if (lane == 0 && n_down) red_release_add(p.sync + SY_P2_DONE, n_down);
     } else {
         // ---------------- auxiliary team
         AuxCtx a;
         a.atid = threadIdx.x - AUX_T0;
         a.lane = lane;
         a.aw = a.atid >> 5;
+        a.npf = 0;
+        APROF(a, 60);
         const int T = dm.T, N = dm.N;
-        // while the logits are being produced: fetch what classification will need
-#pragma unroll 1
-        for (int i = a.atid; i < N; i += AUX_T) ax.soe[i] = p.w.slot_of_expert[i];
+        // what classification will need is copied asynchronously (global -> shared) while the logits are produced
         const int n_conf = p.conf_stride ? T * N : T;
 #pragma unroll 1
-        for (int i = a.atid; i < n_conf; i += AUX_T) ax.conf[i] = p.conf[i];
+        for (int i = a.atid; i < N; i += AUX_T) cp_async4(smem_u32(ax.soe + i), p.w.slot_of_expert + i);
+#pragma unroll 1
+        for (int i = a.atid; i < n_conf; i += AUX_T) cp_async4(smem_u32(ax.conf + i), p.conf + i);
+        asm volatile("cp.async.commit_group;" ::: "memory");
         ax.cnt_hit[a.atid] = 0;
         ax.cnt_low[a.atid] = 0;
+        APROF(a, 61);
         aux_logits(q, a);
+        APROF(a, 62);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");   // (made visible to the team by the barriers of the wait below)
         bool ok = aux_wait_ge(q, sh, a, p.sync + SY_R1_DONE, N * q.r1_sub);
+        APROF(a, 63);
         if (ok) {
+#ifdef SPICE_ROUTE_TWICE
+            aux_route(q, sh, ax, a);
+            ax.cnt_hit[a.atid] = 0;
+            ax.cnt_low[a.atid] = 0;
+            if (a.atid < 4) sh->s_cnt[a.atid] = 0;
+            aux_sync();
+            APROF(a, 79);
+#endif
             aux_route(q, sh, ax, a);
             if (a.atid == 0) mbar_arrive(smem_u32(&sh->plan_ready));
+            APROF(a, 64);
             if (blockIdx.x == 0) aux_write_outputs(q, sh, ax, a);
             Plan pl;
             plan_static(pl, q);
             plan_routed(pl, sh->n_hg, sh->n_lg);
-            const int nb = (dm.d + 1023) >> 10, n_tasks = T * nb;
-            if ((int)blockIdx.x < n_tasks) {   // CTA-uniform
-                ok = aux_wait_ge(q, sh, a, p.sync + SY_P2_DONE, 4 * (pl.endC - pl.endB));
+            // combine units: 64 threads take 256 columns of one token
+            const int nb = (dm.d + 255) >> 8, n_tasks = T * nb;
+            if ((int)blockIdx.x * 4 < n_tasks) {   // CTA-uniform
+                APROF(a, 65);
+                ok = aux_wait_ge(q, sh, a, p.sync + SY_P2_DONE, 4 * ((pl.sh_early ? pl.nCs : 0) + pl.endC - pl.endB));
+                APROF(a, 66);
                 if (ok)
-                    for (int task = blockIdx.x; task < n_tasks; task += gridDim.x) aux_combine(q, ax, a, task / nb, task % nb);
+                    for (int task = blockIdx.x * 4 + (a.atid >> 6); task < n_tasks; task += gridDim.x * 4)
+                        aux_combine(q, ax, task / nb, (task % nb) * 256 + (a.atid & 63) * 4);
+                APROF(a, 67);
             }
         }
     }
@@ -888,7 +1051,7 @@ size_t dtc_smem_bytes(const Dims &dm, int conf_stride, int stages) {
 }
 
 int dtc_stages(const Dims &dm, int conf_stride, size_t max_smem) {
-    for (int s = MAX_STAGES; s >= 4; --s)
+    for (int s = MAX_STAGES; s >= 3; --s)
         if (dtc_smem_bytes(dm, conf_stride, s) <= max_smem) return s;
     return 0;
 }
@@ -900,13 +1063,13 @@ bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem) {
     if (dm.N > 256 || dm.S > 256) return false;
     if ((size_t)dm.T * dm.K > 1024 || (size_t)dm.T * dm.N > 8192) return false;
     if (dm.d % 8 || dm.I % 8 || dm.Is % 8 || dm.r % 8) return false;
-    const int kcIs = (dm.Is + 63) / 64;
+    const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
     if ((kcIs + CHUNKS_PER_SPLIT - 1) / CHUNKS_PER_SPLIT > MAX_SPLIT) return false;
-    return dtc_stages(dm, conf_stride, max_smem) >= 4;
+    return dtc_stages(dm, conf_stride, max_smem) >= 3;
 }
 
 int decode_tc_nsplit(const Dims &dm) {
-    const int kcIs = (dm.Is + 63) / 64;
+    const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
     return (kcIs + CHUNKS_PER_SPLIT - 1) / CHUNKS_PER_SPLIT;
 }
 
@@ -924,8 +1087,14 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
     q.p = p;
     q.part_split = part_split;
     q.stages = dtc_stages(dm, p.conf_stride, (size_t)max_smem_optin);
-    if (q.stages < 4) return -1;
-    const int kcIs = (dm.Is + 63) / 64;
+    if (q.stages < 3) return -1;
+#ifdef SPICE_TUNE
+    if (const char *e = getenv("SPICE_DTC_STAGES")) {
+        const int v = atoi(e);
+        if (v >= 2 && v <= q.stages) q.stages = v;
+    }
+#endif
+    const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
     q.nsplit_sh = decode_tc_nsplit(dm);
     q.cps_sh = (kcIs + q.nsplit_sh - 1) / q.nsplit_sh;
     {
@@ -960,5 +1129,19 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
     }
     return 1;
 }
+
+#ifdef SPICE_PROF
+extern "C" int spice_debug_dtc_prof_read(unsigned long long *host, size_t n_words) {
+    const size_t total = sizeof(unsigned long long) * (size_t)PR_CTAS * PR_ROLES * PR_EVENTS * 2;
+    if (n_words * 8 < total) return -1;
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(host, g_dtc_prof, total) == cudaSuccess ? 0 : -2;
+}
+extern "C" int spice_debug_dtc_prof_clear(void) {
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_dtc_prof) != cudaSuccess) return -1;
+    return cudaMemset(ptr, 0, sizeof(unsigned long long) * (size_t)PR_CTAS * PR_ROLES * PR_EVENTS * 2) == cudaSuccess ? 0 : -2;
+}
+#endif
 
 }  // namespace spice

@@ -77,7 +77,7 @@ int launch_combine(const Dims &dm, const CombineArgs &a, const Tables &tb, cudaS
 
 // ---- fused decode kernel (decode.cu)
 // words of the dependency-counter array
-enum { SY_ABORT = 0, SY_TEAMS_DONE, SY_R1_DONE, SY_ROUTE_DONE, SY_P2_DONE, SY_P1_ALL, SY_GROUP0 = 8 };
+enum { SY_ABORT = 0, SY_TEAMS_DONE, SY_R1_DONE, SY_ROUTE_DONE, SY_P2_DONE, SY_P1_ALL, SY_NEXT_TASK, SY_GROUP0 = 8 };
 
 struct DecodeParams {
     Dims dm;

@@ -17,6 +17,7 @@
 // Every wait is bounded: on expiry the CTA records SPICE_ERR_TIMEOUT, stops, drains its own copies
 // in flight (again bounded), frees its TMEM and returns.  No load uses cluster multicast.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "spice_internal.cuh"
 #include "tc_device.cuh"
@@ -323,8 +324,12 @@ bool tc_encode_map3(CUtensorMap *m, const void *base, uint64_t cols, uint64_t ro
     cuuint64_t strides[2] = {cols * 2, mat_stride_elems * 2};
     cuuint32_t box[3] = {BK, box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
+    CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+#ifdef SPICE_TUNE
+    if (const char *e = getenv("SPICE_PROMO")) promo = (CUtensorMapL2promotion)atoi(e);
+#endif
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
