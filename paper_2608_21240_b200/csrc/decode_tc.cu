@@ -94,7 +94,7 @@ struct Ctl {
 
 // auxiliary team's shared memory (routing scratch and the tables every role reads)
 struct AuxSmem {
-    float *lg, *conf, *gate, *coef, *xch;
+    float *conf, *gate, *coef, *xch;
     int *soe, *idx, *key, *pos, *perm_h, *perm_l, *cnt_hit, *cnt_low, *off_hit, *off_low, *ent;
     unsigned char *cls;
     GroupDesc *gtab;
@@ -110,13 +110,12 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
         return o;
     };
     const size_t n = (size_t)dm.T * dm.K, TN = (size_t)dm.T * dm.N;
-    const size_t o_lg = take(TN * 4), o_conf = take((conf_stride ? TN : (size_t)dm.T) * 4), o_gate = take(n * 4);
+    const size_t o_conf = take((conf_stride ? TN : (size_t)dm.T) * 4), o_gate = take(n * 4);
     const size_t o_coef = take((size_t)dm.T * 4), o_xch = take((size_t)2 * nb * 64 * 4);
     const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_key = take(n * 4), o_pos = take(n * 4);
     const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take(4 * 256 * 4), o_ent = take((size_t)4 * nb * 4);
     const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
     if (s) {
-        s->lg = reinterpret_cast<float *>(base + o_lg);
         s->conf = reinterpret_cast<float *>(base + o_conf);
         s->gate = reinterpret_cast<float *>(base + o_gate);
         s->coef = reinterpret_cast<float *>(base + o_coef);
@@ -187,12 +186,13 @@ __device__ __forceinline__ unsigned long long now_ns() {
 #ifdef SPICE_PROF
 constexpr int PR_CTAS = 148, PR_ROLES = 4, PR_EVENTS = 512;
 __device__ unsigned long long g_dtc_prof[PR_CTAS * PR_ROLES * PR_EVENTS * 2];
+__device__ unsigned long long g_dtc_cal[PR_CTAS * 4];   // (global ns, cycle counter) at the start and end of each CTA
 #define DPROF(role, cnt, tag)                                                                 \
     do {                                                                                      \
         if (blockIdx.x < PR_CTAS && (cnt) < PR_EVENTS) {                                      \
             const size_t o_ = (((size_t)blockIdx.x * PR_ROLES + (role)) * PR_EVENTS + (cnt)) * 2; \
             g_dtc_prof[o_] = (unsigned long long)(tag);                                       \
-            g_dtc_prof[o_ + 1] = now_ns();                                                    \
+            g_dtc_prof[o_ + 1] = (unsigned long long)clock64();                               \
             ++(cnt);                                                                          \
         }                                                                                     \
     } while (0)
@@ -303,7 +303,7 @@ __device__ __forceinline__ bool aux_wait_ge(const DtcParams &q, Ctl *sh, const A
 
 // router logits: unit u = (expert e, token subset s); each warp takes the tokens s*8 + warp (+ 8*r1_sub ...).
 // Same arithmetic order as the stand-alone router (route_device.cuh): logits agree bit for bit.
-__device__ __noinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) {
+__device__ __forceinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) {
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
     const int n_units = dm.N * q.r1_sub;
@@ -326,101 +326,101 @@ __device__ __noinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) {
 // Routing decisions from the logits, entirely in shared memory.  Every CTA computes the same tables
 // (the code is deterministic: counts by atomics, positions by ranking); CTA 0 also writes the outputs.
 // The arithmetic of the gates is that of warp_topk_gates (route_device.cuh).
-__device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
+__device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
     const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
-    // all of this thread's logits are requested before the first one is parked
-#pragma unroll 1
-    for (int i0 = a.atid; i0 < T * N; i0 += AUX_T * 4) {
-        float v[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = (i0 + u * AUX_T < T * N) ? __ldcg(p.logits + i0 + u * AUX_T) : 0.f;
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (i0 + u * AUX_T < T * N) ax.lg[i0 + u * AUX_T] = (v[u] == v[u]) ? v[u] : -INFINITY;   // NaN never wins
-    }
-    aux_sync();
-    APROF(a, 70);
-    // winners by ranking: rank = #{j : l_j > l_e or (l_j == l_e and j < e)}; 16 candidates are read per step
-    // (four 128-bit reads issued together) so the compare chain never waits for shared memory
-#pragma unroll 1
-    for (int i = a.atid; i < T * N; i += AUX_T) {
-        const int t = i / N, e = i - t * N;
-        const float *l = ax.lg + t * N;
-        const float v = l[e];
-        int rank = 0;
-        int j = 0;
-        if ((N & 3) == 0) {
-            const float4 *l4 = reinterpret_cast<const float4 *>(l);
-#pragma unroll 1
-            for (; j + 16 <= N; j += 16) {
-                const float4 q0 = l4[(j >> 2)], q1 = l4[(j >> 2) + 1], q2 = l4[(j >> 2) + 2], q3 = l4[(j >> 2) + 3];
-                const float u[16] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w, q2.x, q2.y, q2.z, q2.w, q3.x, q3.y, q3.z, q3.w};
-#pragma unroll
-                for (int c = 0; c < 16; ++c) rank += (int)(u[c] > v) | ((int)(u[c] == v) & (int)(j + c < e));
-            }
-        }
-#pragma unroll 1
-        for (; j < N; ++j) {
-            const float u = l[j];
-            rank += (int)(u > v) | ((int)(u == v) & (int)(j < e));
-        }
-        if (rank < K) {
-            ax.idx[t * K + rank] = e;
-            ax.gate[t * K + rank] = v;   // the logit for now
-        }
-    }
-    aux_sync();
-    APROF(a, 71);
-    // gates: p_k = exp(l_k - l_0); denominator = sum over the winners in k order, or the full softmax sum
+    // Phase 1, one warp per token, no barrier inside: the token's logits go from L2 straight into registers
+    // (element e = lane + 32 m), the K winners are found by K rounds of two warp reductions on order-preserving
+    // integer keys (largest key, then smallest index among its holders: equal logits go to the smaller expert
+    // index), then gates and classes of the token's K entries follow in lanes 0..K-1.
+    constexpr int NPL = 8;   // elements per lane, N <= 256
 #pragma unroll 1
     for (int t = a.aw; t < T; t += AUX_W) {
-        const float m = ax.gate[t * K];
+        float val[NPL];
+        uint32_t key[NPL];
+#pragma unroll
+        for (int m = 0; m < NPL; ++m) {
+            const int e = a.lane + 32 * m;
+            val[m] = e < N ? __ldcg(p.logits + (size_t)t * N + e) : 0.f;
+        }
+#pragma unroll
+        for (int m = 0; m < NPL; ++m) {
+            const int e = a.lane + 32 * m;
+            float v = val[m];
+            v = (v == v) ? v + 0.0f : -INFINITY;   // NaN never wins; -0 and +0 are one value
+            val[m] = v;
+            const uint32_t bts = __float_as_uint(v);
+            key[m] = e < N ? ((bts & 0x80000000u) ? ~bts : (bts | 0x80000000u)) : 0u;   // 0 is below every real key
+        }
+        int my_idx = 0;
+        float my_val = 0.f;
+        if (key[0] != 1u) APROF(a, 75);
+#pragma unroll 1
+        for (int k = 0; k < K; ++k) {
+            uint32_t bk = 0u;
+            int bi = 0x7fffffff;
+#pragma unroll
+            for (int m = 0; m < NPL; ++m)
+                if (key[m] > bk) {
+                    bk = key[m];
+                    bi = a.lane + 32 * m;
+                }
+            const uint32_t wmax = __reduce_max_sync(0xffffffffu, bk);
+            const int widx = (int)__reduce_min_sync(0xffffffffu, (unsigned)(bk == wmax ? bi : 0x7fffffff));
+#pragma unroll
+            for (int m = 0; m < NPL; ++m)
+                if (a.lane + 32 * m == widx) key[m] = 0u;   // taken
+            if (a.lane == k) {
+                my_idx = widx;
+                my_val = __uint_as_float((wmax & 0x80000000u) ? (wmax ^ 0x80000000u) : ~wmax);
+            }
+        }
+        APROF(a, 76);
+        // gates: p_k = exp(l_k - l_0); denominator = sum over the winners in k order, or the full softmax sum
+        const float mx = __shfl_sync(0xffffffffu, my_val, 0);
         float denom = 0.f;
         if (!p.norm_topk) {
             float sacc = 0.f;
-#pragma unroll 1
-            for (int e = a.lane; e < N; e += 32) sacc += expf(ax.lg[t * N + e] - m);
+#pragma unroll
+            for (int m = 0; m < NPL; ++m)
+                if (a.lane + 32 * m < N) sacc += expf(val[m] - mx);
             denom = warp_sum(sacc);
         }
-        const float pk = (a.lane < K) ? expf(ax.gate[t * K + a.lane] - m) : 0.f;
+        const float pk = (a.lane < K) ? expf(my_val - mx) : 0.f;
         if (p.norm_topk) {
             float sacc = 0.f;
 #pragma unroll 1
             for (int k = 0; k < K; ++k) sacc += __shfl_sync(0xffffffffu, pk, k);
             denom = sacc;
         }
-        __syncwarp();
-        if (a.lane < K) ax.gate[t * K + a.lane] = pk / denom;
-    }
-    aux_sync();
-    APROF(a, 72);
-    // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
-#pragma unroll 1
-    for (int i = a.atid; i < n; i += AUX_T) {
-        const int e = ax.idx[i];
-        const int sl = ax.soe[e];
-        int c, key = -1;
-        if (sl >= S) {
-            atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
-            c = SPICE_MISS_EXACT;
-        } else if (sl >= 0) {
-            c = SPICE_HIT;
-            key = sl;
-            atomicAdd(&ax.cnt_hit[sl], 1);
-        } else {
-            const int t = i / K;
-            const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
-            c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
-            if (c == SPICE_LOWCONF) {
-                key = 1024 + e;
-                atomicAdd(&ax.cnt_low[e], 1);
+        // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
+        if (a.lane < K) {
+            const int i = t * K + a.lane, e = my_idx;
+            const int sl = ax.soe[e];
+            int c, gkey = -1;
+            if (sl >= S) {
+                atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
+                c = SPICE_MISS_EXACT;
+            } else if (sl >= 0) {
+                c = SPICE_HIT;
+                gkey = sl;
+                atomicAdd(&ax.cnt_hit[sl], 1);
+            } else {
+                const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
+                c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
+                if (c == SPICE_LOWCONF) {
+                    gkey = 1024 + e;
+                    atomicAdd(&ax.cnt_low[e], 1);
+                }
             }
+            ax.idx[i] = e;
+            ax.gate[i] = pk / denom;
+            ax.cls[i] = (unsigned char)c;
+            ax.key[i] = gkey;
+            atomicAdd(&sh->s_cnt[c], 1);
         }
-        ax.cls[i] = (unsigned char)c;
-        ax.key[i] = key;
-        atomicAdd(&sh->s_cnt[c], 1);
+        APROF(a, 77);
     }
     aux_sync();
     APROF(a, 73);
@@ -506,7 +506,7 @@ __device__ __noinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSme
 }
 
 // CTA 0: routing results for the caller (top-k, gates, classes, counts, residual-miss list in (t,k) order)
-__device__ __noinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, const AuxSmem &ax, const AuxCtx &a) {
+__device__ __forceinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, const AuxSmem &ax, const AuxCtx &a) {
     const DecodeParams &p = q.p;
     const int K = p.dm.K, n = p.dm.T * K;
 #pragma unroll 1
@@ -640,6 +640,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
+#ifdef SPICE_PROF
+    if (threadIdx.x == 0 && blockIdx.x < PR_CTAS) {
+        g_dtc_cal[blockIdx.x * 4 + 0] = now_ns();
+        g_dtc_cal[blockIdx.x * 4 + 1] = (unsigned long long)clock64();
+    }
+#endif
 
     if (warp == 0) {
         // ---------------- TMA producer: lane 0 drives, lanes 0-5 each issue one of a stage's copies.  A stage holds
@@ -1025,6 +1031,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS));
     }
+#ifdef SPICE_PROF
+    if (threadIdx.x == 0 && blockIdx.x < PR_CTAS) {
+        g_dtc_cal[blockIdx.x * 4 + 2] = now_ns();
+        g_dtc_cal[blockIdx.x * 4 + 3] = (unsigned long long)clock64();
+    }
+#endif
     // the last CTA to finish clears the counters for the next launch (after an abort the host does it)
     if (threadIdx.x == 0) {
         if (sh->abort_flag) atomicMax(p.tb.status, (int)SPICE_ERR_TIMEOUT);
@@ -1136,6 +1148,10 @@ extern "C" int spice_debug_dtc_prof_read(unsigned long long *host, size_t n_word
     if (n_words * 8 < total) return -1;
     cudaDeviceSynchronize();
     return cudaMemcpyFromSymbol(host, g_dtc_prof, total) == cudaSuccess ? 0 : -2;
+}
+extern "C" int spice_debug_dtc_cal_read(unsigned long long *host) {
+    cudaDeviceSynchronize();
+    return cudaMemcpyFromSymbol(host, g_dtc_cal, sizeof(unsigned long long) * PR_CTAS * 4) == cudaSuccess ? 0 : -2;
 }
 extern "C" int spice_debug_dtc_prof_clear(void) {
     void *ptr = nullptr;
