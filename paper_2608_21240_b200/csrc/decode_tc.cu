@@ -96,6 +96,7 @@ struct Ctl {
 struct AuxSmem {
     float *conf, *gate, *coef, *xch;
     int *soe, *idx, *key, *pos, *perm_h, *perm_l, *cnt_hit, *cnt_low, *off_hit, *off_low, *ent;
+    int *ready;   // [1 + S + N] group g's gate/up (or A_e) tiles are all published (set by the watcher warp)
     unsigned char *cls;
     GroupDesc *gtab;
 };
@@ -115,6 +116,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
     const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_key = take(n * 4), o_pos = take(n * 4);
     const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take(4 * 256 * 4), o_ent = take((size_t)4 * nb * 4);
     const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
+    const size_t o_rdy = take((1 + (size_t)dm.S + dm.N) * 4);
     if (s) {
         s->conf = reinterpret_cast<float *>(base + o_conf);
         s->gate = reinterpret_cast<float *>(base + o_gate);
@@ -134,6 +136,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
         s->ent = reinterpret_cast<int *>(base + o_ent);
         s->cls = base + o_cls;
         s->gtab = reinterpret_cast<GroupDesc *>(base + o_gt);
+        s->ready = reinterpret_cast<int *>(base + o_rdy);
     }
     return off;
 }
@@ -154,6 +157,14 @@ __device__ __forceinline__ int ld_relaxed(const int *p) {
 }
 __device__ __forceinline__ void red_release_add(int *p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_cta(const int *p) {
+    int v;
+    asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_cta(int *p, int v) {
+    asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v) : "memory");
 }
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void *src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
@@ -632,6 +643,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         for (int i = 0; i < 4; ++i) sh->s_cnt[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    for (int i = threadIdx.x; i < 1 + dm.S + dm.N; i += DTC_THREADS) ax.ready[i] = 0;
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
@@ -664,7 +676,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             int end = pl.nA;
             bool ok = true;
             // ids: the first one is the CTA's index, every later one is drawn from a global counter.  The draw is
-            // issued a whole task ahead of its use, so its latency hides behind the task's copies.
+            // issued before the task's copies and used after them, so its latency hides behind the copies.
             int id = blockIdx.x;
             auto lead_wait = [&](uint32_t bar, uint32_t parity) {   // lane 0 waits, the outcome is uniform
                 int r = 1;
@@ -672,8 +684,6 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 return __shfl_sync(PM, r, 0) != 0;
             };
             while (ok) {
-                int drawn = 0;
-                if (lane == 0) drawn = (int)gridDim.x + atomicAdd(p.sync + SY_NEXT_TASK, 1);
                 if (id >= end) {
                     if (routed) break;
                     if (lane == 0) DPROF(0, npf, 30);
@@ -761,7 +771,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 if (lane == 0) DPROF(0, npf, 10 + t.kind);
                 if (dep >= 0) {
                     int r = 1;
-                    if (lane == 0) r = wait_ge(p.sync + dep, dep_target, p.sync, p.tb.status, p.spin_limit, abort_flag) ? 1 : 0;
+                    if (lane == 0) {
+                        const int seen = ld_acquire_cta(ax.ready + t.gi);
+                        DPROF(0, npf, 24 + (seen ? 1 : 0));
+                        if (!seen)   // not yet seen by the watcher warp: poll here
+                            r = wait_ge(p.sync + dep, dep_target, p.sync, p.tb.status, p.spin_limit, abort_flag) ? 1 : 0;
+                    }
                     __syncwarp(PM);
                     if (__shfl_sync(PM, r, 0) == 0) { ok = false; break; }
                     if (lane == 0) DPROF(0, npf, 22);
@@ -778,6 +793,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     ++tcount;
                 }
                 if (lane == 0) DPROF(0, npf, 21);
+                // (drawn only now: an acquire or a fence issued while the atomic is in flight would wait for it)
+                int drawn = 0;
+                if (lane == 0) drawn = (int)gridDim.x + atomicAdd(p.sync + SY_NEXT_TASK, 1);
                 // this lane's copy of every stage: lanes 0,1 the (first) weight box of sub-chunk 0,1; lanes 2,3 the
                 // second weight box (up rows); lanes 4,5 the tokens
                 const int sub = lane & 1, what = lane >> 1;
@@ -795,6 +813,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
                     __syncwarp(PM);
                     if (my_on) tma_load_3d(dst + my_off, my_map, kx, my_y, my_z, full);
+#ifdef SPICE_PROF_STAGES
+                    if (lane == 0 && it < 64) DPROF(0, npf, 90);
+#endif
                     if (++s == stages) {
                         s = 0;
                         ring_phase ^= 1;
@@ -854,7 +875,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     for (int c = 0; c < 2; ++c) {
                         const uint64_t da = make_desc(a0 + c * SUB_A), db = make_desc(b0 + c * NB * 128);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | c | k) ? 1u : 0u);
+                        for (int k = 0; k < 4; ++k) {
+#ifdef SPICE_EXP_NOMMA
+                            if (kb == 0 && c == 0 && k == 0)
+#endif
+                            tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | c | k) ? 1u : 0u);
+                        }
                     }
                     tc_commit(smem_u32(&sh->empty[s]));
                     if (++s == stages) {
@@ -964,7 +990,11 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 __syncwarp();
                 if (warp == 2 && lane == 0) DPROF(1, npf, 58);
                 if (lane == 0) {
+#ifdef SPICE_EXP_RELAXED
+                    asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(ctr), "r"(1) : "memory");
+#else
                     red_release_add(ctr, 1);
+#endif
                     mbar_arrive(smem_u32(&sh->tq_empty[slot]));
                 }
             }
@@ -1012,6 +1042,30 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             Plan pl;
             plan_static(pl, q);
             plan_routed(pl, sh->n_hg, sh->n_lg);
+            // Warp 1 watches the per-group counters while the weights stream, so that the producer finds a flag in
+            // shared memory instead of paying a round trip to L2 when it reaches a down tile.  It ends when every
+            // group is complete (or on abort / after its time limit); the producer never depends on it.
+            if (a.aw == 1) {
+                const int n_groups = 1 + pl.n_hg + pl.n_lg;
+                const long long w0 = clock64();
+                bool all = false;
+#pragma unroll 1
+                for (int round = 0; !all; ++round) {
+                    bool mine = true;
+#pragma unroll 1
+                    for (int g = a.lane; g < n_groups; g += 32) {
+                        if (ax.ready[g]) continue;
+                        const int target = 4 * (g == 0 ? pl.tIs : (g <= pl.n_hg ? pl.tI : pl.tz));
+                        if (ld_acquire(p.sync + SY_GROUP0 + g) >= target) st_release_cta(ax.ready + g, 1);
+                        else mine = false;
+                    }
+                    all = __all_sync(0xffffffffu, mine);
+                    if (!all) {
+                        if (*abort_flag || ld_relaxed(p.sync + SY_ABORT) || clock64() - w0 > ROLE_WAIT_CYCLES) break;
+                        __nanosleep(256);
+                    }
+                }
+            }
             // combine units: 64 threads take 256 columns of one token
             const int nb = (dm.d + 255) >> 8, n_tasks = T * nb;
             if ((int)blockIdx.x * 4 < n_tasks) {   // CTA-uniform
