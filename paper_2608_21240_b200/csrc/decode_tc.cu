@@ -660,11 +660,15 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
 #endif
 
     if (warp == 0) {
-        // ---------------- TMA producer: lane 0 drives, lanes 0-5 each issue one of a stage's copies.  A stage holds
-        // two 64-element sub-chunks: waiting for a free stage, arming it and issuing a copy cost a thread a few hundred
-        // cycles whatever the size, so the stage is made large and its copies are issued side by side.
-        constexpr unsigned PM = 0x3Fu;
-        if (lane < 6) {
+        // ---------------- TMA producer: lane 0 drives, lanes 0-3 each issue one of a stage's copies.  A stage holds
+        // two 64-element sub-chunks.  The SM accepts a TMA instruction only every 150 cycles or so, whatever its size
+        // and whichever thread issues it, so the copies are made as large as the tensor maps allow: for the big
+        // matrices ONE box covers both sub-chunks (and both the gate and the up rows) of a stage -- the maps view a
+        // row as [k-block][64] with the k-block as an outer dimension, so the box lands as [k-block][row][64] -- and
+        // one more box brings the token rows.  Operands whose reduction length is the LoRE rank use plain maps, one
+        // box per sub-chunk (lanes 2 and 3).
+        constexpr unsigned PM = 0xFu;
+        if (lane < 4) {
             Plan pl;
             plan_static(pl, q);
             bool routed = false;
@@ -697,7 +701,8 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 // resolve the task: operands, k range, dependency
                 TaskDesc t{};
                 const CUtensorMap *ma, *mb;
-                int a_row0, a_row1 = -1, a_z = 0, b_z = 0, k0 = 0, dep = -1, dep_target = 0;
+                int a_row0, a_z = 0, b_z = 0, k0 = 0, dep = -1, dep_target = 0;
+                bool plain = false;   // operands with reduction length r: plain maps, one box per sub-chunk
                 const int c0 = pl.endB + (pl.sh_early ? 0 : pl.nCs);   // first down tile of a slot
                 const bool sh_down = pl.sh_early ? (id >= pl.tIs && id < pl.nA) : (id >= pl.endB && id < c0);
                 if (id < pl.tIs) {                       // gate/up tile of the shared expert
@@ -707,7 +712,6 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     ma = &maps.m[MAP_SH_GU];
                     mb = &maps.m[MAP_H];
                     a_row0 = t.tile * 64;
-                    a_row1 = dm.Is + t.tile * 64;
                 } else if (sh_down) {                    // down tile of the shared expert, one K range
                     const int l = id - (pl.sh_early ? pl.tIs : pl.endB);
                     t.kind = TASK_DOWN;
@@ -729,7 +733,6 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     ma = &maps.m[MAP_SLOT_GU];
                     mb = &maps.m[MAP_H];
                     a_row0 = t.tile * 64;
-                    a_row1 = dm.I + t.tile * 64;
                     a_z = ax.gtab[t.gi].id;
                 } else if (id < pl.endB) {               // A_e tile of a low-confidence expert
                     const int l = id - pl.nA - pl.nBh;
@@ -762,6 +765,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     t.nk = pl.kcr;
                     ma = &maps.m[MAP_LORE_B];
                     mb = &maps.m[MAP_Z];
+                    plain = true;
                     a_row0 = t.tile * 128;
                     a_z = ax.gtab[t.gi].id;
                     b_z = t.gi - 1 - pl.n_hg;
@@ -796,23 +800,24 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 // (drawn only now: an acquire or a fence issued while the atomic is in flight would wait for it)
                 int drawn = 0;
                 if (lane == 0) drawn = (int)gridDim.x + atomicAdd(p.sync + SY_NEXT_TASK, 1);
-                // this lane's copy of every stage: lanes 0,1 the (first) weight box of sub-chunk 0,1; lanes 2,3 the
-                // second weight box (up rows); lanes 4,5 the tokens
-                const int sub = lane & 1, what = lane >> 1;
-                const CUtensorMap *my_map = what == 2 ? mb : ma;
-                const uint32_t my_off = what == 2 ? (uint32_t)(A_BYTES + sub * NB * 128)
-                                                  : (uint32_t)(sub * SUB_A + (what == 1 ? SUB_A / 2 : 0));
-                const int my_y = what == 0 ? a_row0 : (what == 1 ? a_row1 : 0);
-                const int my_z = what == 2 ? b_z : a_z;
-                const bool my_on = what != 1 || a_row1 >= 0;
+                // this lane's copy of every stage: lane 0 the weights, lane 1 the tokens (sub-chunk 0 only when the
+                // maps are plain); lanes 2, 3 the same for sub-chunk 1 of plain maps
+                const int sub = lane >> 1, is_b = lane & 1;
+                const CUtensorMap *my_map = is_b ? mb : ma;
+                const uint32_t my_off = is_b ? (uint32_t)(A_BYTES + sub * NB * 128) : (uint32_t)(sub * SUB_A);
+                const int my_y = is_b ? 0 : a_row0;
+                const int my_z = is_b ? b_z : a_z;
+                const bool my_on = sub == 0 || plain;
                 for (int kb = 0; kb < t.nk; ++kb, ++it) {
                     if (!lead_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1)) { ok = false; break; }
                     const uint32_t full = smem_u32(&sh->full[s]);
                     const uint32_t dst = smem_u32(ring + (size_t)s * STAGE_BYTES);
-                    const int kx = (k0 + kb) * KSTAGE + sub * 64;
                     if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
                     __syncwarp(PM);
-                    if (my_on) tma_load_3d(dst + my_off, my_map, kx, my_y, my_z, full);
+                    if (my_on) {
+                        if (plain) tma_load_5d(dst + my_off, my_map, (k0 + kb) * KSTAGE + sub * 64, my_y, 0, 0, my_z, full);
+                        else tma_load_5d(dst + my_off, my_map, 0, my_y, 0, (k0 + kb) * 2, my_z, full);
+                    }
 #ifdef SPICE_PROF_STAGES
                     if (lane == 0 && it < 64) DPROF(0, npf, 90);
 #endif
@@ -1106,11 +1111,6 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
 
 // ------------------------------------------------------------------------------------------
 // host side
-bool make_map3(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t mats, uint64_t mat_stride_elems,
-               uint32_t box_rows) {
-    return tc_encode_map3(m, base, cols, rows, mats, mat_stride_elems, box_rows);
-}
-
 size_t dtc_smem_bytes(const Dims &dm, int conf_stride, int stages) {
     const int nb = nb_of(dm.T);
     return 1024 + (size_t)stages * stage_bytes_of(nb) + ((sizeof(Ctl) + 15) & ~size_t(15)) + aux_layout(dm, conf_stride, nb, nullptr, nullptr);
@@ -1128,7 +1128,8 @@ bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem) {
     if (dm.T < 1 || dm.T > 64) return false;
     if (dm.N > 256 || dm.S > 256) return false;
     if ((size_t)dm.T * dm.K > 1024 || (size_t)dm.T * dm.N > 8192) return false;
-    if (dm.d % 8 || dm.I % 8 || dm.Is % 8 || dm.r % 8) return false;
+    // the big operands are viewed as [row][k-block][64]: their reduction lengths must be whole k-blocks
+    if (dm.d % 64 || dm.I % 64 || dm.Is % 64 || dm.r % 8) return false;
     const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
     if ((kcIs + CHUNKS_PER_SPLIT - 1) / CHUNKS_PER_SPLIT > MAX_SPLIT) return false;
     return dtc_stages(dm, conf_stride, max_smem) >= 3;
@@ -1173,16 +1174,31 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
     const uint64_t n = T * dm.K, g_hit = (uint64_t)dm.S < n ? dm.S : n, g_low = (uint64_t)dm.N < n ? dm.N : n;
     DtcMaps maps;
     bool ok = true;
-    ok = ok && make_map3(&maps.m[MAP_H], p.h, d, T, 1, T * d, nb);
-    ok = ok && make_map3(&maps.m[MAP_SLOT_GU], p.w.slot_w_gate_up, d, 2 * I, dm.S, 2 * I * d, 64);
-    ok = ok && make_map3(&maps.m[MAP_SH_GU], p.w.shared_w_gate_up, d, 2 * Is, 1, 2 * Is * d, 64);
-    ok = ok && make_map3(&maps.m[MAP_LORE_A], p.w.lore_A, d, r, dm.N, r * d, 128);
-    ok = ok && make_map3(&maps.m[MAP_SLOT_D], p.w.slot_w_down, I, d, dm.S, d * I, 128);
-    ok = ok && make_map3(&maps.m[MAP_SH_D], p.w.shared_w_down, Is, d, 1, d * Is, 128);
-    ok = ok && make_map3(&maps.m[MAP_LORE_B], p.w.lore_B, r, d, dm.N, d * r, 128);
-    ok = ok && make_map3(&maps.m[MAP_ACT_HIT], p.act_hit16, I, T, g_hit, T * I, nb);
-    ok = ok && make_map3(&maps.m[MAP_ACT_SH], p.act_shared16, Is, T, 1, T * Is, nb);
-    ok = ok && make_map3(&maps.m[MAP_Z], p.z16, r, T, g_low, T * r, nb);
+    // big operands: (64 elements, rows, halves, k-blocks of 64, matrices); the box takes two k-blocks
+    auto big = [&](int which, const void *base, uint64_t rows, uint64_t K, uint64_t halves, uint64_t mats, uint64_t mat_elems,
+                   uint32_t box_rows) {
+        const uint64_t dims[5] = {64, rows, halves, K / 64, mats};
+        const uint64_t strides[4] = {K * 2, rows * K * 2, 128, mat_elems * 2};
+        const uint32_t box[5] = {64, box_rows, (uint32_t)halves, 2, 1};
+        ok = ok && tc_encode_map5(&maps.m[which], base, dims, strides, box);
+    };
+    // operands reduced over the LoRE rank: (k, rows, 1, 1, matrices), one 64-element box per sub-chunk
+    auto plain = [&](int which, const void *base, uint64_t rows, uint64_t K, uint64_t mats, uint32_t box_rows) {
+        const uint64_t dims[5] = {K, rows, 1, 1, mats};
+        const uint64_t strides[4] = {K * 2, rows * K * 2, rows * K * 2, rows * K * 2};
+        const uint32_t box[5] = {64, box_rows, 1, 1, 1};
+        ok = ok && tc_encode_map5(&maps.m[which], base, dims, strides, box);
+    };
+    big(MAP_H, p.h, T, d, 1, 1, T * d, nb);
+    big(MAP_SLOT_GU, p.w.slot_w_gate_up, I, d, 2, dm.S, 2 * I * d, 64);
+    big(MAP_SH_GU, p.w.shared_w_gate_up, Is, d, 2, 1, 2 * Is * d, 64);
+    big(MAP_LORE_A, p.w.lore_A, r, d, 1, dm.N, r * d, 128);
+    big(MAP_SLOT_D, p.w.slot_w_down, d, I, 1, dm.S, d * I, 128);
+    big(MAP_SH_D, p.w.shared_w_down, d, Is, 1, 1, d * Is, 128);
+    plain(MAP_LORE_B, p.w.lore_B, d, r, dm.N, 128);
+    big(MAP_ACT_HIT, p.act_hit16, T, I, 1, g_hit, T * I, nb);
+    big(MAP_ACT_SH, p.act_shared16, T, Is, 1, 1, T * Is, nb);
+    plain(MAP_Z, p.z16, T, r, g_low, nb);
     if (!ok) return -1;
     const size_t smem = dtc_smem_bytes(dm, p.conf_stride, q.stages);
     const void *fn = nb == 16 ? reinterpret_cast<const void *>(decode_tc_kernel<16>)

@@ -6,9 +6,8 @@
 
 namespace spice {
 
-// host: tensor map of a 3-D bf16 tensor [mats, rows, cols], box 1 x box_rows x 64, 128-byte swizzle (tc_gemm.cu)
-bool tc_encode_map3(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t mats, uint64_t mat_stride_elems,
-                    uint32_t box_rows);
+// host: 5-D bf16 tensor map from extents, byte strides of dimensions 1..4 and box; 128-byte swizzle (tc_gemm.cu)
+bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], const uint64_t strides[4], const uint32_t box[5]);
 
 namespace tcdev {
 
@@ -81,10 +80,12 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
     return d;
 }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t mbar) {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(mbar)
-                 : "memory");
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, int c4,
+                                            uint32_t mbar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(mbar)
+        : "memory");
 }
 // orders accesses of this thread through the generic proxy (plain loads / stores) with its accesses through
 // the async proxy (TMA): needed between data written by ordinary stores and a TMA load of the same bytes

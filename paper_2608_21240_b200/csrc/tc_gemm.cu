@@ -17,7 +17,6 @@
 // Every wait is bounded: on expiry the CTA records SPICE_ERR_TIMEOUT, stops, drains its own copies
 // in flight (again bounded), frees its TMEM and returns.  No load uses cluster multicast.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "spice_internal.cuh"
 #include "tc_device.cuh"
@@ -314,23 +313,20 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, ui
 
 }  // namespace
 
-// 3-D bf16 tensor [mats, rows, cols] (cols contiguous, matrices mat_stride_elems apart),
-// box = 1 x box_rows x 64 columns, 128-byte swizzle, zero fill
-bool tc_encode_map3(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t mats, uint64_t mat_stride_elems,
-                    uint32_t box_rows) {
+// 5-D bf16 tensor map with explicit extents, byte strides (dimensions 1..4) and box; 128-byte swizzle, zero fill.
+// The innermost box extent must be 64 elements (one swizzle span).
+bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], const uint64_t strides[4], const uint32_t box[5]) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[3] = {cols, rows, mats};
-    cuuint64_t strides[2] = {cols * 2, mat_stride_elems * 2};
-    cuuint32_t box[3] = {BK, box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
-#ifdef SPICE_TUNE
-    if (const char *e = getenv("SPICE_PROMO")) promo = (CUtensorMapL2promotion)atoi(e);
-#endif
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    cuuint64_t gd[5], gs[4];
+    cuuint32_t bx[5], estr[5] = {1, 1, 1, 1, 1};
+    for (int i = 0; i < 5; ++i) {
+        gd[i] = dims[i];
+        bx[i] = box[i];
+    }
+    for (int i = 0; i < 4; ++i) gs[i] = strides[i];
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), gd, gs, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 namespace {
