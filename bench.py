@@ -176,6 +176,8 @@ def run_ours(args):
     h = bf16_tensor(wl0.h, dev)
     conf = torch.from_numpy(wl0.conf).to(dev)
     layer = B.SpiceLayer(cfg_of(shape), T, device=local)
+    if args.path:
+        layer.set_option(B.OPT_PATH, args.path)
     y = torch.empty(T, shape.d, dtype=torch.bfloat16, device=dev)
     idx = torch.empty(T, shape.top_k, dtype=torch.int32, device=dev)
     gate = torch.empty(T, shape.top_k, dtype=torch.float32, device=dev)
@@ -372,6 +374,8 @@ def main():
     ap.add_argument("--shape", default="dsv2lite")
     ap.add_argument("--tokens", type=int, default=16)
     ap.add_argument("--replicas", type=int, default=8)
+    ap.add_argument("--path", type=int, default=0,
+                    help="kernel path (SPICE_OPT_PATH): 0 auto, 1 general kernels, 2 no fused kernel, 3 mma.sync decode kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()

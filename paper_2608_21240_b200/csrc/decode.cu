@@ -1,6 +1,8 @@
-// Fused decode kernel: the whole MoE layer (Eq. 1 routing; Sec. 4.2 hit / low-confidence /
+// Fused decode kernel on mma.sync: the whole MoE layer (Eq. 1 routing; Sec. 4.2 hit / low-confidence /
 // exact-recovery policy; exact resident experts; shared expert + LoRE surrogate; gate-weighted
-// aggregation of Sec. 2.1) in ONE persistent cooperative launch for small batches (T <= 32).
+// aggregation of Sec. 2.1) in ONE persistent cooperative launch for small batches (T <= 16).
+// It serves the shapes the tcgen05 / TMA decode kernel (decode_tc.cu) does not take (dimensions that are
+// multiples of 8 but not of 64) and can be selected explicitly (SPICE_OPT_PATH = 3).
 //
 // The layer is HBM-bound at these batch sizes: every weight byte is needed once and reused by at
 // most T tokens.  The kernel therefore is a weight streamer.  One CTA per SM holds the tokens in
@@ -37,7 +39,6 @@ namespace {
 constexpr int DT = 512;     // threads per CTA
 constexpr int TEAM = 256;   // threads per team
 constexpr int TW = 8;       // warps per team
-constexpr int NT_MAX = 2;   // n-tiles of 8 tokens
 constexpr int XPAD = 64;    // row padding (bytes) of the token tile in shared memory
 
 __device__ __forceinline__ int ld_acquire(const int *p) {
@@ -810,11 +811,7 @@ __device__ __forceinline__ int team_run(const DecodeParams &p, const Plan &pl, T
     constexpr int MATS = DUAL ? 2 : 1;
     // k-steps in flight per warp.  More than the bandwidth-delay product only deepens the memory queues
     // (every dependent access on the router's critical path then waits behind them): measured optimum.
-#ifdef SPICE_U_P2
-    constexpr int U = (EPI == EPI_PART2) ? SPICE_U_P2 : (DUAL ? UD : 2 * UD);
-#else
     constexpr int U = DUAL ? UD : 2 * UD;
-#endif
     constexpr int MYFL = EPI == EPI_ACT ? FL_ACT : (EPI == EPI_Z ? FL_Z : (EPI == EPI_PART ? FL_PART : FL_PART2));
     const int c = tc.lane & 3;
     const uint4 zero = make_uint4(0, 0, 0, 0);

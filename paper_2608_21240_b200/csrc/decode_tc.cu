@@ -95,7 +95,8 @@ struct Ctl {
 // auxiliary team's shared memory (routing scratch and the tables every role reads)
 struct AuxSmem {
     float *conf, *gate, *coef, *xch;
-    int *soe, *idx, *key, *pos, *perm_h, *perm_l, *cnt_hit, *cnt_low, *off_hit, *off_low, *ent;
+    int *soe, *idx, *key, *pos, *perm_h, *perm_l, *off_hit, *off_low, *ent;
+    uint32_t *mask_hit, *mask_low;   // [256][2] members of a slot's / an expert's group as a bit mask over the tokens
     int *ready;   // [1 + S + N] group g's gate/up (or A_e) tiles are all published (set by the watcher warp)
     unsigned char *cls;
     GroupDesc *gtab;
@@ -114,7 +115,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
     const size_t o_conf = take((conf_stride ? TN : (size_t)dm.T) * 4), o_gate = take(n * 4);
     const size_t o_coef = take((size_t)dm.T * 4), o_xch = take((size_t)2 * nb * 64 * 4);
     const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_key = take(n * 4), o_pos = take(n * 4);
-    const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take(4 * 256 * 4), o_ent = take((size_t)4 * nb * 4);
+    const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take(6 * 256 * 4), o_ent = take((size_t)4 * nb * 4);
     const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
     const size_t o_rdy = take((1 + (size_t)dm.S + dm.N) * 4);
     if (s) {
@@ -129,10 +130,10 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
         s->perm_h = reinterpret_cast<int *>(base + o_ph);
         s->perm_l = reinterpret_cast<int *>(base + o_pl);
         int *hist = reinterpret_cast<int *>(base + o_hist);
-        s->cnt_hit = hist;
-        s->cnt_low = hist + 256;
-        s->off_hit = hist + 512;
-        s->off_low = hist + 768;
+        s->off_hit = hist;
+        s->off_low = hist + 256;
+        s->mask_hit = reinterpret_cast<uint32_t *>(hist + 512);
+        s->mask_low = reinterpret_cast<uint32_t *>(hist + 1024);
         s->ent = reinterpret_cast<int *>(base + o_ent);
         s->cls = base + o_cls;
         s->gtab = reinterpret_cast<GroupDesc *>(base + o_gt);
@@ -341,103 +342,132 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
     const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
-    // Phase 1, one warp per token, no barrier inside: the token's logits go from L2 straight into registers
-    // (element e = lane + 32 m), the K winners are found by K rounds of two warp reductions on order-preserving
-    // integer keys (largest key, then smallest index among its holders: equal logits go to the smaller expert
-    // index), then gates and classes of the token's K entries follow in lanes 0..K-1.
+    // Phase 1, one warp per token (two tokens at a time, interleaved, so that the reductions of one hide the latency
+    // of the other), no barrier inside: the logits go from L2 straight into registers (element e = lane + 32 m),
+    // the K winners are found by K rounds of two warp reductions on order-preserving integer keys (largest key, then
+    // smallest index among its holders: equal logits go to the smaller expert index), then gates and classes of
+    // the token's K entries follow in lanes 0..K-1.  A group's members are kept as a bit mask over the tokens.
     constexpr int NPL = 8;   // elements per lane, N <= 256
+    constexpr int TT = 2;
 #pragma unroll 1
-    for (int t = a.aw; t < T; t += AUX_W) {
-        float val[NPL];
-        uint32_t key[NPL];
+    for (int t0 = a.aw; t0 < T; t0 += AUX_W * TT) {
+        float val[TT][NPL];
+        uint32_t key[TT][NPL];
 #pragma unroll
-        for (int m = 0; m < NPL; ++m) {
-            const int e = a.lane + 32 * m;
-            val[m] = e < N ? __ldcg(p.logits + (size_t)t * N + e) : 0.f;
+        for (int u = 0; u < TT; ++u) {
+            const int t = t0 + u * AUX_W;
+#pragma unroll
+            for (int m = 0; m < NPL; ++m) {
+                const int e = a.lane + 32 * m;
+                val[u][m] = (e < N && t < T) ? __ldcg(p.logits + (size_t)t * N + e) : 0.f;
+            }
         }
 #pragma unroll
-        for (int m = 0; m < NPL; ++m) {
-            const int e = a.lane + 32 * m;
-            float v = val[m];
-            v = (v == v) ? v + 0.0f : -INFINITY;   // NaN never wins; -0 and +0 are one value
-            val[m] = v;
-            const uint32_t bts = __float_as_uint(v);
-            key[m] = e < N ? ((bts & 0x80000000u) ? ~bts : (bts | 0x80000000u)) : 0u;   // 0 is below every real key
+        for (int u = 0; u < TT; ++u)
+#pragma unroll
+            for (int m = 0; m < NPL; ++m) {
+                const int e = a.lane + 32 * m;
+                float v = val[u][m];
+                v = (v == v) ? v + 0.0f : -INFINITY;   // NaN never wins; -0 and +0 are one value
+                val[u][m] = v;
+                const uint32_t bts = __float_as_uint(v);
+                key[u][m] = e < N ? ((bts & 0x80000000u) ? ~bts : (bts | 0x80000000u)) : 0u;   // 0 is below every real key
+            }
+        int my_idx[TT];
+        float my_val[TT];
+#pragma unroll
+        for (int u = 0; u < TT; ++u) {
+            my_idx[u] = 0;
+            my_val[u] = 0.f;
         }
-        int my_idx = 0;
-        float my_val = 0.f;
-        if (key[0] != 1u) APROF(a, 75);
+        if (key[0][0] != 1u) APROF(a, 75);
 #pragma unroll 1
         for (int k = 0; k < K; ++k) {
-            uint32_t bk = 0u;
-            int bi = 0x7fffffff;
+            uint32_t bk[TT], wmax[TT];
+            int bi[TT], widx[TT];
 #pragma unroll
-            for (int m = 0; m < NPL; ++m)
-                if (key[m] > bk) {
-                    bk = key[m];
-                    bi = a.lane + 32 * m;
+            for (int u = 0; u < TT; ++u) {
+                bk[u] = 0u;
+                bi[u] = 0x7fffffff;
+#pragma unroll
+                for (int m = 0; m < NPL; ++m)
+                    if (key[u][m] > bk[u]) {
+                        bk[u] = key[u][m];
+                        bi[u] = a.lane + 32 * m;
+                    }
+            }
+#pragma unroll
+            for (int u = 0; u < TT; ++u) wmax[u] = __reduce_max_sync(0xffffffffu, bk[u]);
+#pragma unroll
+            for (int u = 0; u < TT; ++u)
+                widx[u] = (int)__reduce_min_sync(0xffffffffu, (unsigned)(bk[u] == wmax[u] ? bi[u] : 0x7fffffff));
+#pragma unroll
+            for (int u = 0; u < TT; ++u) {
+#pragma unroll
+                for (int m = 0; m < NPL; ++m)
+                    if (a.lane + 32 * m == widx[u]) key[u][m] = 0u;   // taken
+                if (a.lane == k) {
+                    my_idx[u] = widx[u];
+                    my_val[u] = __uint_as_float((wmax[u] & 0x80000000u) ? (wmax[u] ^ 0x80000000u) : ~wmax[u]);
                 }
-            const uint32_t wmax = __reduce_max_sync(0xffffffffu, bk);
-            const int widx = (int)__reduce_min_sync(0xffffffffu, (unsigned)(bk == wmax ? bi : 0x7fffffff));
-#pragma unroll
-            for (int m = 0; m < NPL; ++m)
-                if (a.lane + 32 * m == widx) key[m] = 0u;   // taken
-            if (a.lane == k) {
-                my_idx = widx;
-                my_val = __uint_as_float((wmax & 0x80000000u) ? (wmax ^ 0x80000000u) : ~wmax);
             }
         }
         APROF(a, 76);
-        // gates: p_k = exp(l_k - l_0); denominator = sum over the winners in k order, or the full softmax sum
-        const float mx = __shfl_sync(0xffffffffu, my_val, 0);
-        float denom = 0.f;
-        if (!p.norm_topk) {
-            float sacc = 0.f;
 #pragma unroll
-            for (int m = 0; m < NPL; ++m)
-                if (a.lane + 32 * m < N) sacc += expf(val[m] - mx);
-            denom = warp_sum(sacc);
-        }
-        const float pk = (a.lane < K) ? expf(my_val - mx) : 0.f;
-        if (p.norm_topk) {
-            float sacc = 0.f;
-#pragma unroll 1
-            for (int k = 0; k < K; ++k) sacc += __shfl_sync(0xffffffffu, pk, k);
-            denom = sacc;
-        }
-        // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
-        if (a.lane < K) {
-            const int i = t * K + a.lane, e = my_idx;
-            const int sl = ax.soe[e];
-            int c, gkey = -1;
-            if (sl >= S) {
-                atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
-                c = SPICE_MISS_EXACT;
-            } else if (sl >= 0) {
-                c = SPICE_HIT;
-                gkey = sl;
-                atomicAdd(&ax.cnt_hit[sl], 1);
-            } else {
-                const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
-                c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
-                if (c == SPICE_LOWCONF) {
-                    gkey = 1024 + e;
-                    atomicAdd(&ax.cnt_low[e], 1);
-                }
+        for (int u = 0; u < TT; ++u) {
+            const int t = t0 + u * AUX_W;
+            if (t >= T) continue;   // warp-uniform
+            // gates: p_k = exp(l_k - l_0); denominator = sum over the winners in k order, or the full softmax sum
+            const float mx = __shfl_sync(0xffffffffu, my_val[u], 0);
+            float denom = 0.f;
+            if (!p.norm_topk) {
+                float sacc = 0.f;
+#pragma unroll
+                for (int m = 0; m < NPL; ++m)
+                    if (a.lane + 32 * m < N) sacc += expf(val[u][m] - mx);
+                denom = warp_sum(sacc);
             }
-            ax.idx[i] = e;
-            ax.gate[i] = pk / denom;
-            ax.cls[i] = (unsigned char)c;
-            ax.key[i] = gkey;
-            atomicAdd(&sh->s_cnt[c], 1);
+            const float pk = (a.lane < K) ? expf(my_val[u] - mx) : 0.f;
+            if (p.norm_topk) {
+                float sacc = 0.f;
+#pragma unroll 1
+                for (int k = 0; k < K; ++k) sacc += __shfl_sync(0xffffffffu, pk, k);
+                denom = sacc;
+            }
+            // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
+            if (a.lane < K) {
+                const int i = t * K + a.lane, e = my_idx[u];
+                const int sl = ax.soe[e];
+                int c, gkey = -1;
+                if (sl >= S) {
+                    atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
+                    c = SPICE_MISS_EXACT;
+                } else if (sl >= 0) {
+                    c = SPICE_HIT;
+                    gkey = sl;
+                    atomicOr(&ax.mask_hit[2 * sl + (t >> 5)], 1u << (t & 31));
+                } else {
+                    const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
+                    c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
+                    if (c == SPICE_LOWCONF) {
+                        gkey = 1024 + e;
+                        atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
+                    }
+                }
+                ax.idx[i] = e;
+                ax.gate[i] = pk / denom;
+                ax.cls[i] = (unsigned char)c;
+                ax.key[i] = gkey;
+                atomicAdd(&sh->s_cnt[c], 1);
+            }
         }
-        APROF(a, 77);
     }
     aux_sync();
     APROF(a, 73);
     // groups: thread i owns slot i and expert i; packed scan of (entries, non-empty flag << 16)
     {
-        const int ch = a.atid < S ? ax.cnt_hit[a.atid] : 0, cl = a.atid < N ? ax.cnt_low[a.atid] : 0;
+        const int ch = a.atid < S ? __popc(ax.mask_hit[2 * a.atid]) + __popc(ax.mask_hit[2 * a.atid + 1]) : 0;
+        const int cl = a.atid < N ? __popc(ax.mask_low[2 * a.atid]) + __popc(ax.mask_low[2 * a.atid + 1]) : 0;
         const int va = ch | ((ch > 0) << 16), vb = cl | ((cl > 0) << 16);
         int ia = va, ib = vb;
 #pragma unroll
@@ -486,23 +516,16 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
     }
     aux_sync();
     APROF(a, 74);
-    // position of every entry inside its group = offset of the group + number of earlier entries of the group
+    // position of every entry inside its group = offset of the group + number of members with a smaller token index
+    // (an expert occurs at most once among a token's K choices, so the members of a group are distinct tokens)
 #pragma unroll 1
     for (int i = a.atid; i < n; i += AUX_T) {
-        const int key = ax.key[i];
+        const int key = ax.key[i], t = i / K;
         int pos = -1;
         if (key >= 0) {
-            int rank = 0, j = 0;
-            const int4 *k4 = reinterpret_cast<const int4 *>(ax.key);
-#pragma unroll 1
-            for (; j + 16 <= i; j += 16) {
-                const int4 q0 = k4[(j >> 2)], q1 = k4[(j >> 2) + 1], q2 = k4[(j >> 2) + 2], q3 = k4[(j >> 2) + 3];
-                rank += (q0.x == key) + (q0.y == key) + (q0.z == key) + (q0.w == key) + (q1.x == key) + (q1.y == key) +
-                        (q1.z == key) + (q1.w == key) + (q2.x == key) + (q2.y == key) + (q2.z == key) + (q2.w == key) +
-                        (q3.x == key) + (q3.y == key) + (q3.z == key) + (q3.w == key);
-            }
-#pragma unroll 1
-            for (; j < i; ++j) rank += ax.key[j] == key;
+            const uint32_t *mk = key < 1024 ? ax.mask_hit + 2 * key : ax.mask_low + 2 * (key - 1024);
+            const uint32_t below = (1u << (t & 31)) - 1u;
+            const int rank = t < 32 ? __popc(mk[0] & below) : __popc(mk[0]) + __popc(mk[1] & below);
             if (key < 1024) {
                 pos = ax.off_hit[key] + rank;
                 ax.perm_h[pos] = i;
@@ -880,12 +903,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     for (int c = 0; c < 2; ++c) {
                         const uint64_t da = make_desc(a0 + c * SUB_A), db = make_desc(b0 + c * NB * 128);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-#ifdef SPICE_EXP_NOMMA
-                            if (kb == 0 && c == 0 && k == 0)
-#endif
-                            tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | c | k) ? 1u : 0u);
-                        }
+                        for (int k = 0; k < 4; ++k) tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | c | k) ? 1u : 0u);
                     }
                     tc_commit(smem_u32(&sh->empty[s]));
                     if (++s == stages) {
@@ -995,11 +1013,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 __syncwarp();
                 if (warp == 2 && lane == 0) DPROF(1, npf, 58);
                 if (lane == 0) {
-#ifdef SPICE_EXP_RELAXED
-                    asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(ctr), "r"(1) : "memory");
-#else
                     red_release_add(ctr, 1);
-#endif
                     mbar_arrive(smem_u32(&sh->tq_empty[slot]));
                 }
             }
@@ -1023,8 +1037,8 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
 #pragma unroll 1
         for (int i = a.atid; i < n_conf; i += AUX_T) cp_async4(smem_u32(ax.conf + i), p.conf + i);
         asm volatile("cp.async.commit_group;" ::: "memory");
-        ax.cnt_hit[a.atid] = 0;
-        ax.cnt_low[a.atid] = 0;
+        ax.mask_hit[2 * a.atid] = ax.mask_hit[2 * a.atid + 1] = 0u;
+        ax.mask_low[2 * a.atid] = ax.mask_low[2 * a.atid + 1] = 0u;
         APROF(a, 61);
         aux_logits(q, a);
         APROF(a, 62);
@@ -1032,14 +1046,6 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         bool ok = aux_wait_ge(q, sh, a, p.sync + SY_R1_DONE, N * q.r1_sub);
         APROF(a, 63);
         if (ok) {
-#ifdef SPICE_ROUTE_TWICE
-            aux_route(q, sh, ax, a);
-            ax.cnt_hit[a.atid] = 0;
-            ax.cnt_low[a.atid] = 0;
-            if (a.atid < 4) sh->s_cnt[a.atid] = 0;
-            aux_sync();
-            APROF(a, 79);
-#endif
             aux_route(q, sh, ax, a);
             if (a.atid == 0) mbar_arrive(smem_u32(&sh->plan_ready));
             APROF(a, 64);

@@ -13,7 +13,7 @@ from tests._gpu import (GATE_ATOL, LOGIT_ATOL, bf16_tensor, cfg_of, check_routin
 
 pytestmark = pytest.mark.gpu
 
-DECODE_CASES = [("tiny", 4), ("dsv2lite", 1), ("dsv2lite", 4), ("dsv2lite", 16),
+DECODE_CASES = [("tiny", 4), ("dsv2lite", 1), ("dsv2lite", 4), ("dsv2lite", 16), ("dsv2lite", 33), ("dsv2lite", 64),
                 ("qwen2_57b", 1), ("qwen2_57b", 8), ("qwen2_57b", 32)]
 
 
@@ -158,6 +158,29 @@ def test_moe_layer_fwd_general_kernels_match_oracle(name, T):
     assert torch.equal(fused.idx, out.idx) and torch.equal(fused.gate, out.gate) and torch.equal(fused.cls, out.cls)
     diff = (fused.y.float() - out.y.float()).abs().max().item()
     assert diff <= 1e-2 * out.y.float().abs().max().item() + 1e-3
+    L.close()
+
+
+@pytest.mark.parametrize("name,T", [("tiny", 4), ("dsv2lite", 1), ("dsv2lite", 16), ("qwen2_57b", 8)])
+def test_mma_sync_decode_kernel_matches_oracle_and_tcgen05_kernel(name, T):
+    """The mma.sync decode kernel (forced) against the oracle, and against the default tcgen05 decode kernel."""
+    wl = _layer_case(name, T, variant=2)
+    s = wl.shape
+    ref = run_oracle(wl, want_full=False)
+    L = B.SpiceLayer(cfg_of(s), T)
+    w = upload(wl)
+    h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+    new = L.moe_layer_fwd(w, h, conf)
+    L.set_option(B.OPT_PATH, 3)
+    n0 = L.launch_count()
+    old = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert L.launch_count() - n0 == 1 and L.device_status() == 0
+    for out in (new, old):
+        check_routing(out, ref, T, s.top_k)
+        err, bound = y_close(out.y.float().cpu().numpy(), ref.y)
+        assert err <= bound, f"max err {err:.3e} > bound {bound:.3e}"
+    assert torch.equal(new.idx, old.idx) and torch.equal(new.gate, old.gate) and torch.equal(new.cls, old.cls)
     L.close()
 
 
