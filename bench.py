@@ -303,6 +303,158 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- 26-layer decode stack (config 5)
+def stack_residency(idx, n_experts, n_slots, tau, rng, hit_rate=0.7):
+    """Residency and confidences of one layer GIVEN its routing (host logic of the input recipe, no method arithmetic):
+    selected experts are made resident in random order until >= hit_rate of the picks hit, the remaining slots hold
+    unselected experts (stale prefetches); a miss is low-confidence with probability 1/2."""
+    picks = idx.ravel()
+    selected = rng.permutation(np.unique(picks))
+    resident, hits = [], 0
+    for e in selected:
+        if hits >= hit_rate * picks.size or len(resident) >= n_slots:
+            break
+        resident.append(int(e))
+        hits += int((picks == e).sum())
+    sel = set(selected.tolist())
+    resident += [int(e) for e in rng.permutation(n_experts) if e not in sel][: n_slots - len(resident)]
+    soe = np.full(n_experts, -1, np.int32)
+    soe[np.array(resident)] = rng.permutation(len(resident)).astype(np.int32)
+    conf = rng.random((idx.shape[0], n_experts)).astype(np.float32)
+    for t in range(idx.shape[0]):
+        for e in idx[t]:
+            if soe[e] < 0:
+                conf[t, e] = np.float32(rng.uniform(0.0, tau * 0.999) if rng.random() < 0.5 else rng.uniform(tau * 1.001, 1.0))
+    return soe, conf
+
+
+def run_stack(args):
+    """--stack: one step = the MoE layers of a 26-layer DeepSeek-V2-Lite-shaped decoder for one decode batch of 8
+    tokens, free running: 26 layer calls back to back on one stream, each with its own weights (13.5 GB in all, so
+    the L2 is cold for every layer), the residual stream updated inside the call (x += y)."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_21240_b200 import binding as B
+    from paper_2608_21240_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()
+    shape = W.SHAPES["dsv2lite_stack"]
+    T, n_layers = 8, 26
+    peaks = load_peaks()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(W.BASE_SEED + 5000 + 1000 * rank)
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([W.BASE_SEED, 5, 777, rank])))
+    layer = B.SpiceLayer(B.cfg_of(shape), T, device=local)
+    if args.path:
+        layer.set_option(B.OPT_PATH, args.path)
+    stream = torch.cuda.current_stream()
+    weights, hs, confs = [], [], []
+    idx = torch.empty(T, shape.top_k, dtype=torch.int32, device=dev)
+    gate = torch.empty(T, shape.top_k, dtype=torch.float32, device=dev)
+    cls = torch.empty(T, shape.top_k, dtype=torch.uint8, device=dev)
+    for l in range(n_layers):
+        w = device_replica(torch, B, shape, gen, dev)
+        h = torch.randn(T, shape.d, generator=gen, device=dev, dtype=torch.float32).to(torch.bfloat16)
+        B.spice_route_topk(layer.ctx, h, w.w_router, T, idx, gate, stream=stream)
+        torch.cuda.synchronize()
+        soe, conf = stack_residency(idx.cpu().numpy(), shape.n_experts, shape.n_slots, shape.tau, rng)
+        w.slot_of_expert.copy_(torch.from_numpy(soe))
+        weights.append(w)
+        hs.append(h)
+        confs.append(torch.from_numpy(conf).to(dev))
+    structs = [w.c_struct() for w in weights]
+    x = torch.zeros(T, shape.d, dtype=torch.bfloat16, device=dev)      # residual stream
+    y = torch.empty(T, shape.d, dtype=torch.bfloat16, device=dev)
+
+    def step():
+        for l in range(n_layers):
+            B.spice_moe_layer_fwd(layer.ctx, structs[l], hs[l], confs[l], T, y, x_resid=x, idx=idx, cls=cls, stream=stream)
+
+    total_bytes, hit_frac = 0, []
+    for l in range(n_layers):
+        B.spice_moe_layer_fwd(layer.ctx, structs[l], hs[l], confs[l], T, y, idx=idx, cls=cls, stream=stream)
+        torch.cuda.synchronize()
+        b, _, _ = algorithmic_bytes(shape, T, idx.cpu().numpy(), cls.cpu().numpy())
+        total_bytes += b
+        hit_frac.append(float((cls.cpu().numpy() == 0).mean()))
+    sampler = ClockSampler(local) if rank == 0 else None
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    l0 = layer.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    w1 = time.time()
+    if world > 1:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    launches = layer.launch_count() - l0
+    # end to end: the residual stream comes from pinned host memory and goes back every step
+    x_host = torch.zeros(T, shape.d, dtype=torch.bfloat16).pin_memory()
+    out_host = torch.empty(T, shape.d, dtype=torch.bfloat16).pin_memory()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_e2e = args.steps
+    f0.record(stream)
+    for _ in range(n_e2e):
+        x.copy_(x_host, non_blocking=True)
+        step()
+        out_host.copy_(x, non_blocking=True)
+        stream.synchronize()
+    f1.record(stream)
+    torch.cuda.synchronize()
+    ms_e2e = f0.elapsed_time(f1)
+    if sampler:
+        sampler.stop()
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev)
+    status = layer.device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status} after the timed region")
+    if rank == 0:
+        achieved = total_bytes * args.steps / (ms * 1e-3) / 1e9
+        out = {
+            "metric": "moe_stack_decode_tokens_per_s", "value": whole_job_throughput(T, args.steps, world, ms), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"MoE layers of a {n_layers}-layer DeepSeek-V2-Lite-shaped decoder, decode batch {T}, "
+                                   f"free running ({shape.n_slots} resident slots per layer, residency chosen given the "
+                                   f"routing: mean hit rate {np.mean(hit_frac):.2f}, misses low-confidence w.p. 1/2)",
+                       "tokens_per_step": T, "layer_calls_per_step": n_layers,
+                       "cold_l2": f"every layer has its own weights ({total_bytes / 1e6:.0f} MB touched per step, "
+                                  f"L2 is 126 MB); no flush in the timed region",
+                       "multi_gpu": "replicas only (no collective on the data path)"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                         "kernel": "all 26 launches of a step (sum of the calls' algorithmic bytes / time per step)",
+                         "algorithmic_bytes_per_step": float(total_bytes), "peak_source": peaks["source"]},
+            "e2e": {"value": whole_job_throughput(T, n_e2e, world, ms_e2e), "unit": UNIT,
+                    "h2d_bytes_per_step": int(x_host.numel() * 2), "d2h_bytes_per_step": int(out_host.numel() * 2),
+                    "ms_per_step": ms_e2e / n_e2e},
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(w0, w1) if sampler else None,
+            "cpu_baseline": None,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 def oracle_call(wl, tokens):
     """One oracle evaluation of the GPU part of the layer for the given tokens."""
@@ -376,12 +528,16 @@ def main():
     ap.add_argument("--replicas", type=int, default=8)
     ap.add_argument("--path", type=int, default=0,
                     help="kernel path (SPICE_OPT_PATH): 0 auto, 1 general kernels, 2 no fused kernel, 3 mma.sync decode kernel")
+    ap.add_argument("--stack", action="store_true",
+                    help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
+    elif args.stack:
+        run_stack(args)
     else:
         run_ours(args)
 

@@ -64,3 +64,17 @@ def test_zipf_router_is_skewed():
     idx, _ = oracle.topk_gates(oracle.router_logits(wl.h, wl.w_router), wl.shape.top_k)
     load = np.bincount(idx.ravel(), minlength=64)
     assert load.max() > 6 * max(1, np.median(load))
+
+
+def test_stack_residency_recipe_reaches_the_hit_rate_and_fills_the_slots():
+    """Input recipe of the 26-layer stack timing (bench.py --stack): host logic only."""
+    import bench
+    rng = np.random.Generator(np.random.PCG64(7))
+    N, S, K, T, tau = 64, 26, 6, 8, 0.6
+    idx = np.stack([rng.permutation(N)[:K] for _ in range(T)]).astype(np.int32)
+    soe, conf = bench.stack_residency(idx, N, S, tau, rng)
+    assert (soe >= 0).sum() == S and sorted(soe[soe >= 0].tolist()) == list(range(S))
+    hits = (soe[idx] >= 0).mean()
+    assert hits >= 0.7 or (soe[np.unique(idx)] >= 0).all()
+    miss_conf = conf[np.arange(T)[:, None], idx][soe[idx] < 0]
+    assert np.all(np.abs(miss_conf - tau) > 1e-4) and conf.shape == (T, N) and conf.dtype == np.float32
