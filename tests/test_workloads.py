@@ -75,6 +75,7 @@ def test_stack_residency_recipe_reaches_the_hit_rate_and_fills_the_slots():
     soe, conf = bench.stack_residency(idx, N, S, tau, rng)
     assert (soe >= 0).sum() == S and sorted(soe[soe >= 0].tolist()) == list(range(S))
     hits = (soe[idx] >= 0).mean()
-    assert hits >= 0.7 or (soe[np.unique(idx)] >= 0).all()
+    # the target rate is reached unless the slots ran out first (then every slot holds a selected expert)
+    assert hits >= 0.7 or (soe[np.unique(idx)] >= 0).sum() == S
     miss_conf = conf[np.arange(T)[:, None], idx][soe[idx] < 0]
     assert np.all(np.abs(miss_conf - tau) > 1e-4) and conf.shape == (T, N) and conf.dtype == np.float32
