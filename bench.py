@@ -28,6 +28,9 @@ if ROOT not in sys.path:
 METRIC = "moe_layer_decode_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised under
+# profiles/ (same workload with 2 weight sets; mean of the two captured launches), keyed by (shape, tokens, path)
+CAPTURED_TRAFFIC = {("dsv2lite", 16, 0): (492.6e6, "profiles/decode_tc_kernel_dsv2lite_T16.md")}
 
 
 def load_peaks():
@@ -222,20 +225,26 @@ def run_ours(args):
     launches = layer.launch_count() - l0
     total_bytes = sum(rep_bytes[i % R] for i in range(args.steps))
 
-    # end to end: inputs start in pinned host memory, the result is read back to the host every step
-    h_host = h.cpu().pin_memory()
-    conf_host = conf.cpu().pin_memory()
-    y_host = torch.empty(T, shape.d, dtype=torch.bfloat16).pin_memory()
-    cnt_host = torch.empty(3, dtype=torch.int32).pin_memory()
-    h_dev, conf_dev = torch.empty_like(h), torch.empty_like(conf)
+    # end to end: inputs start in pinned host memory, the result is read back to the host every step.  The caller
+    # packs what travels together: one pinned block (h, conf) -> one device block, one device block (y, counts) -> host.
+    in_bytes = h.numel() * 2 + conf.numel() * 4
+    in_host = torch.empty(in_bytes, dtype=torch.uint8).pin_memory()
+    in_dev = torch.empty(in_bytes, dtype=torch.uint8, device=dev)
+    in_host[: h.numel() * 2].copy_(h.cpu().view(torch.uint8).reshape(-1))
+    in_host[h.numel() * 2:].copy_(conf.cpu().view(torch.uint8).reshape(-1))
+    h_dev = in_dev[: h.numel() * 2].view(torch.bfloat16).view(T, shape.d)
+    conf_dev = in_dev[h.numel() * 2:].view(torch.float32).view_as(conf)
+    out_bytes = T * shape.d * 2 + 16
+    out_dev = torch.empty(out_bytes, dtype=torch.uint8, device=dev)
+    out_host = torch.empty(out_bytes, dtype=torch.uint8).pin_memory()
+    y_e2e = out_dev[: T * shape.d * 2].view(torch.bfloat16).view(T, shape.d)
+    cnt_e2e = out_dev[T * shape.d * 2:].view(torch.int32)[:3]
 
     def e2e_step(i):
-        h_dev.copy_(h_host, non_blocking=True)
-        conf_dev.copy_(conf_host, non_blocking=True)
-        B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h_dev, conf_dev, T, y, idx=idx, gate=gate, cls=cls,
-                              counts=counts, stream=stream)
-        y_host.copy_(y, non_blocking=True)
-        cnt_host.copy_(counts, non_blocking=True)
+        in_dev.copy_(in_host, non_blocking=True)
+        B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h_dev, conf_dev, T, y_e2e, idx=idx, gate=gate, cls=cls,
+                              counts=cnt_e2e, stream=stream)
+        out_host.copy_(out_dev, non_blocking=True)
         stream.synchronize()     # the caller consumes y before the next step
 
     for i in range(min(args.warmup, 5)):
@@ -281,7 +290,9 @@ def run_ours(args):
                        "distinct_lowconf_experts_mean": float(np.mean(rep_low)),
                        "multi_gpu": "replicas only (no collective on the data path)"},
             "roofline": ({"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                          "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                          "frac": achieved / peaks["hbm_gbs"],
+                          "traffic": CAPTURED_TRAFFIC.get((shape.name, T, args.path), (None, None))[0],
+                          "traffic_source": CAPTURED_TRAFFIC.get((shape.name, T, args.path), (None, None))[1],
                           "kernel": "all launches of spice_moe_layer_fwd (algorithmic bytes of the call / time per call)",
                           "algorithmic_bytes_per_step": total_bytes / args.steps, "peak_source": peaks["source"],
                           "frac_of_nominal_8TBs": achieved / 8000.0} if not prefill else
@@ -291,8 +302,8 @@ def run_ours(args):
                                     "the grouped GEMM kernels alone are in profiles/)",
                           "peak_source": peaks["source"], "frac_of_nominal_2250": tfs / 2250.0}),
             "e2e": {"value": whole_job_throughput(T, n_e2e, world, ms_e2e), "unit": UNIT,
-                    "h2d_bytes_per_step": int(h_host.numel() * 2 + conf_host.numel() * 4),
-                    "d2h_bytes_per_step": int(y_host.numel() * 2 + 12), "ms_per_step": ms_e2e / n_e2e},
+                    "h2d_bytes_per_step": int(in_bytes), "d2h_bytes_per_step": int(out_bytes),
+                    "ms_per_step": ms_e2e / n_e2e},
             "gpu_launches": int(launches),
             "clocks": sampler.summary(w0, w1) if sampler else None,
         }

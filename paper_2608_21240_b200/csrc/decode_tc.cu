@@ -37,7 +37,6 @@
 // the CTA records SPICE_ERR_TIMEOUT, raises the abort flag, drains its copies in flight, frees
 // its TMEM and returns.  No load uses cluster multicast.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "route_device.cuh"
 #include "spice_internal.cuh"
@@ -1161,12 +1160,6 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
     q.part_split = part_split;
     q.stages = dtc_stages(dm, p.conf_stride, (size_t)max_smem_optin);
     if (q.stages < 3) return -1;
-#ifdef SPICE_TUNE
-    if (const char *e = getenv("SPICE_DTC_STAGES")) {
-        const int v = atoi(e);
-        if (v >= 2 && v <= q.stages) q.stages = v;
-    }
-#endif
     const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
     q.nsplit_sh = decode_tc_nsplit(dm);
     q.cps_sh = (kcIs + q.nsplit_sh - 1) / q.nsplit_sh;

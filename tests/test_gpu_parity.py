@@ -253,6 +253,37 @@ def test_moe_layer_fwd_unnormalised_gates_and_cpu_residual_and_resid_stream():
     L.close()
 
 
+@pytest.mark.parametrize("T", [7, 17, 48])
+def test_tcgen05_decode_kernel_all_token_widths_scalar_conf_full_softmax_and_residuals(T):
+    """The tcgen05 decode kernel at 16, 32 and 64 token columns, on a shape with ragged tiles (I = 192: 3 gate/up
+    tiles; I_s = 320; r = 24 on plain maps), one confidence per token, full-softmax gates, CPU residual and residual stream."""
+    s = W.scaled_shape(W.SHAPES["tiny"], d=320, n_experts=12, top_k=3, inter=192, inter_shared=320, lore_rank=24,
+                       n_slots=5)
+    wl = _layer_case(s, T, variant=20 + T)
+    conf1 = np.ascontiguousarray(wl.conf[:, 0])
+    ref = run_oracle(wl, want_full=True, norm_topk=0, conf=conf1)
+    y_cpu = torch.from_numpy((ref.y_full - ref.y).astype(np.float32)).cuda()
+    L = B.SpiceLayer(cfg_of(s, norm_topk=0, conf_per_expert=False), T)
+    w = upload(wl)
+    x0 = torch.randn(T, s.d, device="cuda").bfloat16()
+    x = x0.clone()
+    n0 = L.launch_count()
+    out = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(conf1).cuda(), y_cpu_residual=y_cpu, x_resid=x)
+    torch.cuda.synchronize()
+    assert L.launch_count() - n0 == 1 and L.device_status() == 0
+    check_routing(out, ref, T, s.top_k)
+    err, bound = y_close(out.y.float().cpu().numpy(), ref.y_full)
+    assert err <= bound, f"max err {err:.3e} > bound {bound:.3e}"
+    errx, boundx = y_close(x.float().cpu().numpy(), x0.float().cpu().numpy().astype(np.float64) + ref.y_full)
+    assert errx <= boundx + 2e-2    # bf16 rounding of the O(1) residual stream
+    # the general kernels agree on every routing decision
+    L.set_option(B.OPT_PATH, 1)
+    gen = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(conf1).cuda(), y_cpu_residual=y_cpu)
+    assert L.launch_count() - n0 > 2
+    assert torch.equal(gen.idx, out.idx) and torch.equal(gen.gate, out.gate) and torch.equal(gen.cls, out.cls)
+    L.close()
+
+
 def test_split_exports_compose_to_the_fused_call():
     wl = _layer_case("dsv2lite", 4, variant=2)
     s = wl.shape
