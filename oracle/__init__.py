@@ -96,6 +96,18 @@ def topk_gates(logits, K: int, norm_topk: int = 1):
     return idx, gate
 
 
+def draft_confidence(logits, K: int):
+    """Sec. 4.1: pi_hat = softmax(logits), S_hat = TopK (Eq. 2), C = probability mass of S_hat (Eq. 5).
+    Returns (idx_hat [T,K], pi_hat [T,N], conf [T])."""
+    l = np.ascontiguousarray(logits, dtype=np.float64)
+    T, N = l.shape
+    idx = np.empty((T, K), dtype=np.int32)
+    pi = np.empty((T, N), dtype=np.float64)
+    conf = np.empty(T, dtype=np.float64)
+    _load().oracle_draft_confidence(C.c_int(T), C.c_int(N), C.c_int(K), _p(l), _p(idx), _p(pi), _p(conf))
+    return idx, pi, conf
+
+
 def classify(idx, resident, conf, tau: float, conf_stride: Optional[int] = None):
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     T, K = idx.shape

@@ -108,6 +108,39 @@ void oracle_topk_gates(int T, int N, int K, int norm_topk, const double *logits,
     }
 }
 
+/* Draft-router confidence of Sec. 4.1: pi_hat = softmax(draft logits) over all N experts,
+ * S_hat = TopK(pi_hat, K) (Eq. 2), C(pi_hat) = sum_{i in S_hat} pi_hat_i (Eq. 5).
+ * Written out from the definitions: the full distribution first, then K rounds of arg-max over the
+ * probabilities not yet taken (ties to the smaller index), then the sum in order of selection. */
+void oracle_draft_confidence(int T, int N, int K, const double *logits, int32_t *idx_hat, double *pi_hat, double *conf) {
+    for (int t = 0; t < T; ++t) {
+        const double *l = logits + (size_t)t * N;
+        double *p = pi_hat + (size_t)t * N;
+        int32_t *ix = idx_hat + (size_t)t * K;
+        double m = l[0];
+        for (int e = 1; e < N; ++e)
+            if (l[e] > m) m = l[e];
+        double denom = 0.0;
+        for (int e = 0; e < N; ++e) denom += exp(l[e] - m);
+        for (int e = 0; e < N; ++e) p[e] = exp(l[e] - m) / denom;
+        double c = 0.0;
+        for (int k = 0; k < K; ++k) {
+            int best = -1;
+            for (int e = 0; e < N; ++e) {
+                int taken = 0;
+                for (int q = 0; q < k; ++q)
+                    if (ix[q] == e) taken = 1;
+                if (taken) continue;
+                /* compare the logits: exp is monotone but may round two different logits to one probability */
+                if (best < 0 || l[e] > l[best]) best = e;
+            }
+            ix[k] = best;
+            c += p[best];
+        }
+        conf[t] = c;
+    }
+}
+
 /* Sec. 4.2 runtime policy: resident -> exact (HIT); missing and low confidence -> surrogate
  * (LOWCONF); any other miss -> exact recovery (MISS_EXACT).  counts[c] = entries of class c. */
 void oracle_classify(int T, int N, int K, const int32_t *idx, const uint8_t *resident, const float *conf,

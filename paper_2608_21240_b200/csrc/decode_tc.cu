@@ -33,7 +33,7 @@
 //   D  combine y_t = c_t S(h_t) + sum_k g_k part_{t,k}  (auxiliary teams)          (all C tiles)
 // Dependencies are counters in global memory: red.release by the finishing warp, bounded
 // ld.acquire polls by the waiting one.  Data written by plain stores and later fetched by TMA is
-// ordered with fence.proxy.async on both sides.  Every wait in the kernel is bounded; on expiry
+// ordered by a fence.proxy.async between the reader's acquire and its TMA copies.  Every wait in the kernel is bounded; on expiry
 // the CTA records SPICE_ERR_TIMEOUT, raises the abort flag, drains its copies in flight, frees
 // its TMEM and returns.  No load uses cluster multicast.
 #include <cuda.h>
@@ -745,7 +745,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     mb = &maps.m[MAP_ACT_SH];
                     a_row0 = t.tile * 128;
                     dep = SY_GROUP0;
-                    dep_target = 4 * pl.tIs;
+                    dep_target = 2 * pl.tIs;
                 } else if (id < pl.nA + pl.nBh) {        // gate/up tile of a resident slot
                     const int l = id - pl.nA;
                     t.kind = TASK_ACT;
@@ -778,7 +778,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     a_z = ax.gtab[t.gi].id;
                     b_z = t.gi - 1;
                     dep = SY_GROUP0 + t.gi;
-                    dep_target = 4 * pl.tI;
+                    dep_target = 2 * pl.tI;
                 } else {                                 // B_e tile of a low-confidence expert
                     const int l = id - c0 - pl.nCh;
                     t.kind = TASK_DOWN;
@@ -1008,11 +1008,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 ++n_down;
                 if (lane == 0) mbar_arrive(smem_u32(&sh->tq_empty[slot]));
             } else {
-                fence_proxy_async();   // act / z rows are fetched by TMA in the tasks that depend on this one
+                // Publish: only warps that stored rows signal (gate/up tiles: the two gate-row warps).  The release is
+                // one loaded memory round trip; the proxy fence that the TMA reads of these rows need lies on the
+                // reader's side of the release / acquire pair (in the producer), which keeps it off this path.
                 __syncwarp();
-                if (warp == 2 && lane == 0) DPROF(1, npf, 58);
                 if (lane == 0) {
-                    red_release_add(ctr, 1);
+                    if (t.kind != TASK_ACT || qd < 2) red_release_add(ctr, 1);
                     mbar_arrive(smem_u32(&sh->tq_empty[slot]));
                 }
             }
@@ -1065,14 +1066,14 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
 #pragma unroll 1
                     for (int g = a.lane; g < n_groups; g += 32) {
                         if (ax.ready[g]) continue;
-                        const int target = 4 * (g == 0 ? pl.tIs : (g <= pl.n_hg ? pl.tI : pl.tz));
+                        const int target = g == 0 ? 2 * pl.tIs : (g <= pl.n_hg ? 2 * pl.tI : 4 * pl.tz);
                         if (ld_acquire(p.sync + SY_GROUP0 + g) >= target) st_release_cta(ax.ready + g, 1);
                         else mine = false;
                     }
                     all = __all_sync(0xffffffffu, mine);
                     if (!all) {
                         if (*abort_flag || ld_relaxed(p.sync + SY_ABORT) || clock64() - w0 > ROLE_WAIT_CYCLES) break;
-                        __nanosleep(256);
+                        __nanosleep(100);
                     }
                 }
             }

@@ -318,3 +318,44 @@ def test_p12_y_full_equals_dense_when_nothing_is_substituted(seed):
     assert res.counts[2] == 0 and res.counts[1] > 0
     dense, _, _ = dense_layer(wl)
     assert rel(res.y_full, dense) < 1e-9
+
+
+# ------------------------------------------------------------------ draft-router confidence (Sec. 4.1, Eq. 2 and Eq. 5)
+def test_p13_draft_confidence_hand_example():
+    """Logits ln(1..4): the distribution is (0.1, 0.2, 0.3, 0.4) by inspection, so the top two experts are 3 and 2
+    and the confidence is 0.7; with K = N the mass is 1, with K = 1 it is the largest probability."""
+    logits = np.log(np.array([[1.0, 2.0, 3.0, 4.0]]))
+    idx, pi, conf = oracle.draft_confidence(logits, 2)
+    assert idx.tolist() == [[3, 2]]
+    assert np.allclose(pi, [[0.1, 0.2, 0.3, 0.4]], atol=1e-15)
+    assert abs(conf[0] - 0.7) < 1e-15
+    assert abs(oracle.draft_confidence(logits, 4)[2][0] - 1.0) < 1e-15
+    assert abs(oracle.draft_confidence(logits, 1)[2][0] - 0.4) < 1e-15
+
+
+@pytest.mark.parametrize("N,K", [(8, 2), (64, 6), (64, 8), (10, 10)])
+def test_p13_draft_confidence_invariants(N, K):
+    rng = np.random.default_rng(5 + N + K)
+    logits = rng.standard_normal((7, N)) * 1.3
+    idx, pi, conf = oracle.draft_confidence(logits, K)
+    # a distribution; independent numpy path: sort the softmax, add the K largest
+    assert np.allclose(pi.sum(axis=1), 1.0, atol=1e-14) and (pi >= 0).all()
+    z = np.exp(logits - logits.max(axis=1, keepdims=True))
+    p = z / z.sum(axis=1, keepdims=True)
+    assert np.allclose(conf, np.sort(p, axis=1)[:, ::-1][:, :K].sum(axis=1), atol=1e-14)
+    assert np.array_equal(idx, np.argsort(-logits, axis=1, kind="stable")[:, :K])
+    # shift invariance, bounds, monotone in K, uniform logits give K / N
+    assert np.allclose(oracle.draft_confidence(logits + 3.25, K)[2], conf, atol=1e-14)
+    assert (conf <= 1.0 + 1e-15).all() and (conf >= K / N - 1e-15).all()
+    if K > 1:
+        assert (oracle.draft_confidence(logits, K - 1)[2] < conf).all()
+    assert np.allclose(oracle.draft_confidence(np.full((2, N), 0.37), K)[2], K / N, atol=1e-15)
+    # the selected set and its probabilities are those of the router of Eq. 1 with un-normalised gates
+    idx1, gate1 = oracle.topk_gates(logits, K, norm_topk=0)
+    assert np.array_equal(idx1, idx) and np.allclose(gate1.sum(axis=1), conf, atol=1e-14)
+
+
+def test_p13_draft_confidence_ties_prefer_lower_index():
+    logits = np.array([[0.5, 1.0, 1.0, 0.5, 1.0]])
+    idx, pi, conf = oracle.draft_confidence(logits, 2)
+    assert idx.tolist() == [[1, 2]]
