@@ -466,6 +466,62 @@ def run_stack(args):
         dist.destroy_process_group()
 
 
+# ----------------------------------------------------------------------------- draft-router confidence (Sec. 4.1)
+def run_draft_confidence(args):
+    """--op draft_confidence: one step = spice_draft_confidence over one batch (router copy of one layer)."""
+    import torch
+
+    from paper_2608_21240_b200 import binding as B
+    from paper_2608_21240_b200 import workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    B.lib()
+    shape = W.SHAPES[args.shape]
+    T, R = args.tokens, max(args.replicas, 64)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(W.BASE_SEED + 77)
+    routers = [(torch.randn(shape.n_experts, shape.d, generator=gen, device=dev) * 0.02).to(torch.bfloat16) for _ in range(R)]
+    hs = [torch.randn(T, shape.d, generator=gen, device=dev).to(torch.bfloat16) for _ in range(R)]
+    layer = B.SpiceLayer(B.cfg_of(shape), T, device=dev.index)
+    idx = torch.empty(T, shape.top_k, dtype=torch.int32, device=dev)
+    conf = torch.empty(T, dtype=torch.float32, device=dev)
+    pi = torch.empty(T, shape.n_experts, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def step(i):
+        B.spice_draft_confidence(layer.ctx, hs[i % R], routers[i % R], T, idx, conf, pi, stream=stream)
+
+    for i in range(args.warmup):
+        step(i)
+    flush.fill_(1)        # cold L2 at the start; the rotating inputs (R sets) keep the router rows out of L1
+    torch.cuda.synchronize()
+    l0 = layer.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    nbytes = 2 * shape.n_experts * shape.d + 2 * T * shape.d + 4 * T * (shape.n_experts + shape.top_k + 1)
+    peaks = load_peaks()
+    achieved = nbytes * args.steps / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "draft_confidence_tokens_per_s", "value": T * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"draft-router confidence, {shape.name} router (N={shape.n_experts}, d={shape.d}, K={shape.top_k}), "
+                               f"batch {T} tokens, {R} rotating input sets (warm L2: {R * nbytes / 1e6:.1f} MB in all)"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                     "kernel": "route_topk_kernel + draft_confidence_kernel (latency-bound at decode batches: "
+                               "the call moves well under a megabyte)", "peak_source": peaks["source"]},
+        "gpu_launches": int(layer.launch_count() - l0)}))
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 def oracle_call(wl, tokens):
     """One oracle evaluation of the GPU part of the layer for the given tokens."""
@@ -541,12 +597,16 @@ def main():
                     help="kernel path (SPICE_OPT_PATH): 0 auto, 1 general kernels, 2 no fused kernel, 3 mma.sync decode kernel")
     ap.add_argument("--stack", action="store_true",
                     help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
+    ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence"],
+                    help="what a step is: the MoE layer call (default) or the draft-router confidence call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
+    elif args.op == "draft_confidence":
+        run_draft_confidence(args)
     elif args.stack:
         run_stack(args)
     else:

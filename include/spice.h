@@ -141,6 +141,18 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w /*
                                  int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
                                  float *resid_gate, void *stream);
 
+/* Draft-router confidence (Sec. 4.1): the producer of the `conf` input above.
+ *   pi_hat[t,:] = softmax over all N experts of  h_hat[t,:] . w_draft_router[e,:]      (predicted routing distribution)
+ *   idx_hat[t,0..K-1] = TopK(pi_hat[t,:], K)                                          (Eq. 2; same order and tie rule as Eq. 1)
+ *   conf[t] = sum_{i in idx_hat[t,:]} pi_hat[t,i]                                      (Eq. 5), summed in k order
+ * h_hat [T,d] bf16: hidden states the draft predictor hands to the layer's router copy; w_draft_router [N,d] bf16.
+ * idx_hat [T,K] int32 out; conf [T] fp32 out: the per-token confidence (the conf_stride = 0 layout of
+ * spice_classify_misses / spice_moe_layer_fwd); pi_hat [T,N] fp32 out, optional (NULL: not wanted): the
+ * per-(token, expert) layout (conf_stride = N).  The logits use the arithmetic of spice_route_topk, so idx_hat equals
+ * what spice_route_topk returns for the same inputs, and pi_hat[t, idx_hat[t,k]] equals its gate with norm_topk = 0. */
+spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, const spice_bf16 *w_draft_router,
+                                    int32_t T, int32_t *idx_hat, float *pi_hat, float *conf, void *stream);
+
 /* The resident-expert FFN for callers that cannot allocate (the paper has no counterpart: this is
  * a packaging variant of spice_grouped_expert_ffn, not a step of the method).
  *

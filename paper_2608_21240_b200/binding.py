@@ -55,7 +55,7 @@ def lib() -> C.CDLL:
         for name in ("spice_create", "spice_destroy", "spice_workspace_bytes", "spice_route_topk",
                      "spice_classify_misses", "spice_grouped_expert_ffn", "spice_lore_surrogate",
                      "spice_moe_layer_fwd", "spice_get_device_status", "spice_launch_count", "spice_set_option",
-                     "spice_grouped_expert_ffn_static"):
+                     "spice_grouped_expert_ffn_static", "spice_draft_confidence"):
             getattr(L, name).restype = C.c_int
         L.spice_static_scratch_bytes.restype = C.c_size_t
         _lib = L
@@ -123,6 +123,12 @@ def spice_route_topk(ctx, h, w_router, T, idx, gate, logits=None, stream=None) -
     _check(lib().spice_route_topk(ctx, _ptr(h, torch.bfloat16), _ptr(w_router, torch.bfloat16), C.c_int32(T),
                                   _ptr(idx, torch.int32), _ptr(gate, torch.float32), _ptr(logits, torch.float32),
                                   _stream(stream)), "spice_route_topk")
+
+
+def spice_draft_confidence(ctx, h_hat, w_draft_router, T, idx_hat, conf, pi_hat=None, stream=None) -> None:
+    _check(lib().spice_draft_confidence(ctx, _ptr(h_hat, torch.bfloat16), _ptr(w_draft_router, torch.bfloat16), C.c_int32(T),
+                                        _ptr(idx_hat, torch.int32), _ptr(pi_hat, torch.float32), _ptr(conf, torch.float32),
+                                        _stream(stream)), "spice_draft_confidence")
 
 
 def spice_classify_misses(ctx, idx, gate, slot_of_expert, conf, T, cls, slot, counts, resid_tok=None, resid_k=None,
@@ -243,6 +249,13 @@ class SpiceLayer:
         logits = self._empty((T, N), torch.float32) if want_logits else None
         spice_route_topk(self.ctx, h, w_router, T, idx, gate, logits, stream)
         return (idx, gate, logits) if want_logits else (idx, gate)
+
+    def draft_confidence(self, h_hat, w_draft_router, want_pi=False, stream=None):
+        T, K, N = h_hat.shape[0], self.cfg.top_k, self.cfg.n_experts
+        idx, conf = self._empty((T, K), torch.int32), self._empty((T,), torch.float32)
+        pi = self._empty((T, N), torch.float32) if want_pi else None
+        spice_draft_confidence(self.ctx, h_hat, w_draft_router, T, idx, conf, pi, stream)
+        return (idx, conf, pi) if want_pi else (idx, conf)
 
     def classify_misses(self, idx, gate, slot_of_expert, conf, stream=None):
         T, K = idx.shape

@@ -17,6 +17,7 @@ struct spice_ctx {
     float *ws_gate;
     uint8_t *ws_cls;
     float *y32;        // [Tm, d] fp32 accumulator of the fused call
+    float *draft_logits;            // [Tm, N] logits of spice_draft_confidence when the caller does not want pi_hat
     // fused decode kernel
     float *logits;                  // [Td, N]
     __nv_bfloat16 *act_hit16, *act_shared16, *z16;
@@ -75,6 +76,7 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->ws_gate = cv.take<float>(n);
     c->ws_cls = cv.take<uint8_t>(n);
     c->y32 = cv.take<float>(Tm * g.d);
+    c->draft_logits = cv.take<float>(Tm * g.n_experts);
     // decode kernels: activations of a group are kept for every token of the batch ([group][T][width])
     const size_t Td = Tm < 64 ? Tm : 64, nd = Td * K;
     const size_t g_hit = (size_t)g.n_slots < nd ? g.n_slots : nd, g_low = (size_t)g.n_experts < nd ? g.n_experts : nd;
@@ -259,6 +261,19 @@ spice_status spice_route_topk(spice_ctx *ctx, const spice_bf16 *h, const spice_b
     SPICE_LAUNCH(launch_route_topk(dims_of(ctx, T), ctx->cfg.norm_topk, reinterpret_cast<const __nv_bfloat16 *>(h),
                                    reinterpret_cast<const __nv_bfloat16 *>(w_router), idx, gate, logits,
                                    static_cast<cudaStream_t>(stream)));
+    return SPICE_OK;
+}
+
+spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, const spice_bf16 *w_draft_router, int32_t T,
+                                    int32_t *idx_hat, float *pi_hat, float *conf, void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    if (T == 0) return SPICE_OK;
+    if (!h_hat || !w_draft_router || !idx_hat || !conf || !aligned16(h_hat) || !aligned16(w_draft_router))
+        return SPICE_ERR_INVALID_ARG;
+    SPICE_LAUNCH(launch_draft_confidence(dims_of(ctx, T), reinterpret_cast<const __nv_bfloat16 *>(h_hat),
+                                         reinterpret_cast<const __nv_bfloat16 *>(w_draft_router), idx_hat, ctx->ws_gate,
+                                         ctx->draft_logits, pi_hat, conf, static_cast<cudaStream_t>(stream)));
     return SPICE_OK;
 }
 

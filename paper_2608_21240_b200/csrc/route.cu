@@ -74,6 +74,46 @@ __global__ void route_topk_kernel(const __nv_bfloat16 *__restrict__ h, const __n
     }
 }
 
+// Draft-router confidence (Sec. 4.1, Eq. 5) from the logits, winners and full-softmax gates that
+// route_topk_kernel produced with norm_topk = 0: conf[t] = sum of the K gates in k order; optionally the whole
+// distribution pi_hat = exp(l - l_max) / denom, with the denominator summed exactly as the gates' was
+// (lane-strided partial sums, xor-shuffle tree), so pi_hat[t, idx[t,k]] equals gate[t,k] bit for bit.
+// One warp per token; lp holds the logits on entry and, when pi_out == lp, the distribution on exit.
+__global__ void __launch_bounds__(256) draft_confidence_kernel(const float *lp, const int32_t *__restrict__ idx,
+                                                               const float *__restrict__ gate, int T, int N, int K,
+                                                               float *pi_out, float *__restrict__ conf) {
+    const int lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (t >= T) return;   // warp-uniform
+    if (lane == 0) {
+        float c = 0.f;
+        for (int k = 0; k < K; ++k) c += gate[(size_t)t * K + k];
+        conf[t] = c;
+    }
+    if (!pi_out) return;
+    const float *l = lp + (size_t)t * N;
+    float m = l[idx[(size_t)t * K]];
+    if (!(m == m)) m = -INFINITY;
+    float s = 0.f;
+#pragma unroll 1
+    for (int e = lane; e < N; e += 32) s += expf(l[e] - m);
+    const float denom = warp_sum(s);
+    __syncwarp();   // every lane has read its logits before the row is overwritten in place
+#pragma unroll 1
+    for (int e = lane; e < N; e += 32) pi_out[(size_t)t * N + e] = expf(l[e] - m) / denom;
+}
+
+int launch_draft_confidence(const Dims &dm, const __nv_bfloat16 *h_hat, const __nv_bfloat16 *w_draft, int32_t *idx_hat,
+                            float *gate_ws, float *logits_ws, float *pi_hat, float *conf, cudaStream_t st) {
+    // logits land in pi_hat when the caller wants the distribution (converted in place), else in the workspace
+    float *lp = pi_hat ? pi_hat : logits_ws;
+    int n = launch_route_topk(dm, /*norm_topk=*/0, h_hat, w_draft, idx_hat, gate_ws, lp, st);
+    if (n < 0) return -1;
+    const int wpb = 8;
+    draft_confidence_kernel<<<(dm.T + wpb - 1) / wpb, wpb * 32, 0, st>>>(lp, idx_hat, gate_ws, dm.T, dm.N, dm.K, pi_hat, conf);
+    return cudaGetLastError() == cudaSuccess ? n + 1 : -1;
+}
+
 template <int TPC>
 static int launch_tpc(const Dims &dm, int norm_topk, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router,
                       int32_t *idx, float *gate, float *logits, int threads, cudaStream_t st) {

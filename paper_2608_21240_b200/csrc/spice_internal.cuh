@@ -48,6 +48,10 @@ struct Dims {
 int launch_route_topk(const Dims &dm, int norm_topk, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router,
                       int32_t *idx, float *gate, float *logits, cudaStream_t st);
 
+// draft-router confidence: route with full-softmax gates, then the per-token sum and (optionally) the distribution
+int launch_draft_confidence(const Dims &dm, const __nv_bfloat16 *h_hat, const __nv_bfloat16 *w_draft, int32_t *idx_hat,
+                            float *gate_ws, float *logits_ws, float *pi_hat, float *conf, cudaStream_t st);
+
 int launch_classify(const Dims &dm, int conf_stride, float tau, const int32_t *idx, const float *gate,
                     const int32_t *slot_of_expert, const float *conf, uint8_t *cls, int32_t *slot,
                     int32_t *counts, int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,

@@ -284,6 +284,41 @@ def test_tcgen05_decode_kernel_all_token_widths_scalar_conf_full_softmax_and_res
     L.close()
 
 
+@pytest.mark.parametrize("name,T", [("tiny", 4), ("dsv2lite", 16), ("qwen2_57b", 8), ("dsv2lite", 300)])
+def test_draft_confidence_matches_oracle_and_feeds_the_layer(name, T):
+    """Sec. 4.1, Eq. 2 and Eq. 5: predicted set bit-exact, confidence and distribution within fp32 rounding; the
+    confidences are accepted by the layer call in both layouts."""
+    wl = _layer_case(name, T, variant=31)
+    s = wl.shape
+    logits = oracle.router_logits(wl.h, wl.w_router)
+    ref_idx, ref_pi, ref_conf = oracle.draft_confidence(logits, s.top_k)
+    L = B.SpiceLayer(cfg_of(s), T)
+    h, wr = bf16_tensor(wl.h), bf16_tensor(wl.w_router)
+    idx, conf, pi = L.draft_confidence(h, wr, want_pi=True)
+    idx2, conf2 = L.draft_confidence(h, wr)
+    torch.cuda.synchronize()
+    assert np.array_equal(idx.cpu().numpy(), ref_idx) and torch.equal(idx, idx2) and torch.equal(conf, conf2)
+    assert np.abs(conf.cpu().numpy().astype(np.float64) - ref_conf).max() <= s.top_k * GATE_ATOL
+    assert np.abs(pi.cpu().numpy().astype(np.float64) - ref_pi).max() <= GATE_ATOL
+    # the router of Eq. 1 on the same inputs selects the same experts; its un-normalised gates are pi_hat's entries
+    Lf = B.SpiceLayer(cfg_of(s, norm_topk=0), T)
+    ridx, rgate = Lf.route_topk(h, wr)
+    assert torch.equal(ridx, idx) and torch.equal(rgate, torch.gather(pi, 1, idx.long()))
+    Lf.close()
+    if T <= 64:
+        # per-token confidence and per-(token, expert) probabilities as the `conf` input of the layer
+        w = upload(wl)
+        ref1 = run_oracle(wl, want_full=False, conf=conf.cpu().numpy())    # the same fp32 numbers decide on both sides
+        L1 = B.SpiceLayer(cfg_of(s, conf_per_expert=False), T)
+        out1 = L1.moe_layer_fwd(w, h, conf)
+        assert np.array_equal(out1.cls.cpu().numpy(), ref1.cls)
+        L1.close()
+        out2 = L.moe_layer_fwd(w, h, pi)
+        ref2 = run_oracle(wl, want_full=False, conf=pi.cpu().numpy())
+        assert np.array_equal(out2.cls.cpu().numpy(), ref2.cls)
+    L.close()
+
+
 def test_split_exports_compose_to_the_fused_call():
     wl = _layer_case("dsv2lite", 4, variant=2)
     s = wl.shape
