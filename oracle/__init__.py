@@ -108,6 +108,57 @@ def draft_confidence(logits, K: int):
     return idx, pi, conf
 
 
+def _round_bf16(x: np.ndarray) -> np.ndarray:
+    """Nearest bf16 (ties to even) of fp64 values, returned as fp64: the draft state is kept in bf16 between depths."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
+def prefetch_rollout(x, layers, top_k: int, l_min: int, l_max: int, tau: float):
+    """Algorithm 1 (Sec. 4.1), per token, in the algorithm's own order and notation.
+
+    x [T,d]: current hidden states.  layers[l-1] = dict(w_router, shared=(w_gate, w_up, w_down), lore_A, lore_B) of
+    depth l.  For every depth l = 1..l_max while the token still speculates:
+        pi^(l) = router^(l)(h^(l-1)); S^(l) = TopK(pi^(l), K); enqueue S^(l); C^(l) = sum_{i in S^(l)} pi^(l)_i;
+        if l >= l_min and C^(l) < tau: stop (the current prediction is retained);
+        h^(l) = Attn^(l)(h^(l-1)) + sum_{i in S^(l)} pi^(l)_i E~_i(h^(l-1)),  E~_i = S^(l) + B_i A_i.
+    Readings: Attn^(l) is not specified for a single state and is taken as the identity; the state is held in bf16
+    between depths (the library's activation type).  Returns (idx_hat [l_max,T,K] with -1 past a token's last depth,
+    conf [l_max,T] with 0 there, depth [T] = number of predictions enqueued, h_final [T,d])."""
+    h = _round_bf16(np.asarray(x, dtype=np.float64))
+    T, d = h.shape
+    idx_hat = np.full((l_max, T, top_k), -1, dtype=np.int32)
+    conf = np.zeros((l_max, T), dtype=np.float64)
+    depth = np.zeros(T, dtype=np.int32)
+    active = np.ones(T, dtype=bool)
+    for l in range(1, l_max + 1):
+        L = layers[l - 1]
+        logits = router_logits(h.astype(np.float32), L["w_router"])
+        ix, pi, c = draft_confidence(logits, top_k)
+        new_h = h.copy()
+        for t in range(T):
+            if not active[t]:
+                continue
+            idx_hat[l - 1, t] = ix[t]
+            conf[l - 1, t] = c[t]
+            depth[t] = l
+            if l >= l_min and c[t] < tau:
+                active[t] = False
+                continue
+            if l == l_max:
+                continue        # the loop ends here: no further state is needed
+            ht = h[t].astype(np.float32)
+            s = swiglu_ffn(*L["shared"], ht)
+            acc = h[t].copy()
+            for k in range(top_k):
+                i = int(ix[t, k])
+                acc += pi[t, i] * (s + lore_delta(L["lore_A"][i], L["lore_B"][i], ht))
+            new_h[t] = acc
+        h = _round_bf16(new_h)
+    return idx_hat, conf, depth, h
+
+
 def classify(idx, resident, conf, tau: float, conf_stride: Optional[int] = None):
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     T, K = idx.shape

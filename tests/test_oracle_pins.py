@@ -359,3 +359,81 @@ def test_p13_draft_confidence_ties_prefer_lower_index():
     logits = np.array([[0.5, 1.0, 1.0, 0.5, 1.0]])
     idx, pi, conf = oracle.draft_confidence(logits, 2)
     assert idx.tolist() == [[1, 2]]
+
+
+# ------------------------------------------------------------------ Algorithm 1: speculative prefetch rollout
+def _rollout_layers(rng, L, N, d, Is, r, shared_scale=0.3, lore_scale=0.3, same_router=False):
+    wr = W.bf16_round(rng.standard_normal((N, d)).astype(np.float32))
+    out = []
+    for _ in range(L):
+        out.append(dict(
+            w_router=wr if same_router else W.bf16_round(rng.standard_normal((N, d)).astype(np.float32)),
+            shared=tuple(W.bf16_round((rng.standard_normal(sz) * shared_scale).astype(np.float32)) for sz in ((Is, d), (Is, d), (d, Is))),
+            lore_A=W.bf16_round((rng.standard_normal((N, r, d)) * lore_scale).astype(np.float32)),
+            lore_B=W.bf16_round((rng.standard_normal((N, d, r)) * lore_scale).astype(np.float32))))
+    return out
+
+
+def test_p14_rollout_depth_one_is_the_draft_confidence():
+    rng = np.random.default_rng(14)
+    N, d, K, T = 10, 32, 3, 6
+    layers = _rollout_layers(rng, 1, N, d, 16, 4)
+    x = W.bf16_round(rng.standard_normal((T, d)).astype(np.float32))
+    idx, conf, depth, h = oracle.prefetch_rollout(x, layers, K, 1, 1, 0.5)
+    ix, pi, c = oracle.draft_confidence(oracle.router_logits(x, layers[0]["w_router"]), K)
+    assert np.array_equal(idx[0], ix) and np.array_equal(conf[0], c) and (depth == 1).all() and np.array_equal(h, x)
+
+
+def test_p14_rollout_halting_rule():
+    """tau = 0 never halts (depth = l_max); tau > 1 halts as soon as l >= l_min, keeping the prediction made there;
+    in between, a token stops exactly at the first depth >= l_min whose confidence is below tau."""
+    rng = np.random.default_rng(15)
+    N, d, K, T, L = 12, 32, 2, 9, 5
+    layers = _rollout_layers(rng, L, N, d, 16, 4)
+    x = W.bf16_round(rng.standard_normal((T, d)).astype(np.float32))
+    idx, conf, depth, _ = oracle.prefetch_rollout(x, layers, K, 2, L, 0.0)
+    assert (depth == L).all() and (idx >= 0).all()
+    idx, conf, depth, _ = oracle.prefetch_rollout(x, layers, K, 3, L, 1.5)
+    assert (depth == 3).all() and (idx[:3] >= 0).all() and (idx[3:] == -1).all() and (conf[3:] == 0).all()
+    tau = float(np.median(conf[:3]))
+    idx2, conf2, depth2, _ = oracle.prefetch_rollout(x, layers, K, 2, L, tau)
+    for t in range(T):
+        below = [l for l in range(2, L + 1) if conf2[l - 1, t] < tau and depth2[t] >= l]
+        assert depth2[t] == (below[0] if below else L)
+        assert (idx2[depth2[t]:, t] == -1).all() and (idx2[:depth2[t], t] >= 0).all()
+    assert len(set(depth2.tolist())) > 1      # the threshold actually separates the tokens
+
+
+def test_p14_rollout_state_projection_matches_numpy():
+    """One projection step written out with numpy matmuls: h1 = h0 + C S(h0) + sum_i pi_i B_i A_i h0 (Attn = identity),
+    and its two special cases: zero LoRE (shared expert only) and zero shared expert (low-rank maps only)."""
+    rng = np.random.default_rng(16)
+    N, d, K, T, Is, r = 8, 24, 3, 4, 16, 5
+    x = W.bf16_round(rng.standard_normal((T, d)).astype(np.float32))
+    for shared_scale, lore_scale in ((0.3, 0.3), (0.3, 0.0), (0.0, 0.3)):
+        layers = _rollout_layers(rng, 2, N, d, Is, r, shared_scale, lore_scale)
+        _, _, depth, h1 = oracle.prefetch_rollout(x, layers, K, 2, 2, 0.0)
+        L0 = layers[0]
+        logits = x.astype(np.float64) @ L0["w_router"].astype(np.float64).T
+        p = np.exp(logits - logits.max(axis=1, keepdims=True))
+        p /= p.sum(axis=1, keepdims=True)
+        sel = np.argsort(-logits, axis=1, kind="stable")[:, :K]
+        S = np_ffn(*L0["shared"], x)
+        want = x.astype(np.float64).copy()
+        for t in range(T):
+            want[t] += p[t, sel[t]].sum() * S[t]
+            for i in sel[t]:
+                want[t] += p[t, i] * (L0["lore_B"][i].astype(np.float64) @ (L0["lore_A"][i].astype(np.float64) @ x[t].astype(np.float64)))
+        assert (depth == 2).all()
+        assert np.abs(h1 - want).max() <= 2.0 ** -8 * np.abs(want).max()      # h1 is the bf16 rounding of `want`
+
+
+def test_p14_rollout_fixed_point_when_nothing_is_added():
+    """Zero shared expert and zero LoRE: the state never moves, so with one router for all depths every depth
+    predicts the same set with the same confidence."""
+    rng = np.random.default_rng(17)
+    N, d, K, T, L = 9, 16, 2, 5, 4
+    layers = _rollout_layers(rng, L, N, d, 8, 3, 0.0, 0.0, same_router=True)
+    x = W.bf16_round(rng.standard_normal((T, d)).astype(np.float32))
+    idx, conf, depth, h = oracle.prefetch_rollout(x, layers, K, 1, L, 0.0)
+    assert np.array_equal(h, x) and all(np.array_equal(idx[l], idx[0]) and np.array_equal(conf[l], conf[0]) for l in range(L))
