@@ -522,6 +522,78 @@ def run_draft_confidence(args):
         "gpu_launches": int(layer.launch_count() - l0)}))
 
 
+# ----------------------------------------------------------------------------- Algorithm 1 rollout
+def run_rollout(args):
+    """--op rollout: one step = spice_prefetch_rollout (Algorithm 1) over one decode batch, l_min = 2, l_max = 4."""
+    import torch
+
+    from paper_2608_21240_b200 import binding as B
+    from paper_2608_21240_b200 import workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    B.lib()
+    shape = W.SHAPES[args.shape]
+    T, l_min, l_max = args.tokens, 2, 4
+    R = max(2, min(args.replicas, 8))          # rotating sets of l_max layers
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(W.BASE_SEED + 99)
+
+    def rn(*sz):
+        return (torch.randn(*sz, generator=gen, device=dev, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+
+    s = shape
+    dummy = torch.zeros(8, dtype=torch.bfloat16, device=dev)
+    soe = torch.full((s.n_experts,), -1, dtype=torch.int32, device=dev)
+    sets = [[B.LayerWeights(w_router=rn(s.n_experts, s.d), slot_w_gate_up=dummy, slot_w_down=dummy, slot_of_expert=soe,
+                            shared_w_gate_up=rn(2 * s.inter_shared, s.d), shared_w_down=rn(s.d, s.inter_shared),
+                            lore_A=rn(s.n_experts, s.lore_rank, s.d), lore_B=rn(s.n_experts, s.d, s.lore_rank))
+             for _ in range(l_max)] for _ in range(R)]
+    structs = [[w.c_struct() for w in ws] for ws in sets]
+    x = torch.randn(T, s.d, generator=gen, device=dev).to(torch.bfloat16)
+    layer = B.SpiceLayer(B.cfg_of(shape), T, device=dev.index)
+    idx = torch.empty(l_max, T, s.top_k, dtype=torch.int32, device=dev)
+    conf = torch.empty(l_max, T, dtype=torch.float32, device=dev)
+    depth = torch.empty(T, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    # a threshold that stops about half of the tokens at l_min: the median confidence at that depth
+    B.spice_prefetch_rollout(layer.ctx, structs[0], x, T, l_min, l_max, 0.0, idx, conf, depth, stream=stream)
+    torch.cuda.synchronize()
+    tau = float(conf[l_min - 1].median().item())
+
+    def step(i):
+        B.spice_prefetch_rollout(layer.ctx, structs[i % R], x, T, l_min, l_max, tau, idx, conf, depth, stream=stream)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    l0 = layer.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    mean_depth = float(depth.float().mean().item())
+    nbytes = (l_max - 1) * 2 * (s.n_experts * s.d + 3 * s.d * s.inter_shared) + 2 * s.n_experts * s.d
+    peaks = load_peaks()
+    achieved = nbytes * args.steps / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "prefetch_rollout_tokens_per_s", "value": T * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"Algorithm 1 rollout, {shape.name}-shaped layers (router, shared expert, LoRE factors), batch {T} "
+                               f"tokens, l_min={l_min}, l_max={l_max}, tau={tau:.3f} (median confidence at l_min), mean depth "
+                               f"{mean_depth:.2f}, {R} rotating sets of {l_max} layers"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                     "kernel": "all launches of the call; bytes = routers and shared experts of the depths that project "
+                               "(LoRE factors of the selected experts not counted)", "peak_source": peaks["source"]},
+        "gpu_launches": int(layer.launch_count() - l0)}))
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 def oracle_call(wl, tokens):
     """One oracle evaluation of the GPU part of the layer for the given tokens."""
@@ -597,7 +669,7 @@ def main():
                     help="kernel path (SPICE_OPT_PATH): 0 auto, 1 general kernels, 2 no fused kernel, 3 mma.sync decode kernel")
     ap.add_argument("--stack", action="store_true",
                     help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
-    ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence"],
+    ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout"],
                     help="what a step is: the MoE layer call (default) or the draft-router confidence call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
@@ -607,6 +679,8 @@ def main():
         run_reference(args)
     elif args.op == "draft_confidence":
         run_draft_confidence(args)
+    elif args.op == "rollout":
+        run_rollout(args)
     elif args.stack:
         run_stack(args)
     else:

@@ -153,6 +153,25 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w /*
 spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, const spice_bf16 *w_draft_router,
                                     int32_t T, int32_t *idx_hat, float *pi_hat, float *conf, void *stream);
 
+/* Speculative prefetch rollout (Algorithm 1, Sec. 4.1) for a batch of tokens, all depths on the device.
+ * For depth l = 1 .. l_max, for every token that still speculates, with h^(0) = x_current:
+ *     pi^(l) = softmax(router^(l)(h^(l-1))),  S^(l) = TopK(pi^(l), K) is enqueued,  C^(l) = sum_{i in S^(l)} pi^(l)_i;
+ *     if l >= l_min and C^(l) < tau the token stops here (this prediction is kept, deeper ones are not made);
+ *     h^(l) = h^(l-1) + sum_{i in S^(l)} pi^(l)_i * ( S^(l)(h^(l-1)) + B_i A_i h^(l-1) ).
+ * Readings of the paper: the attention term of the projection, which the paper does not define for a single state, is the
+ * identity; the state is held in bf16 between depths; a NaN confidence does not stop a token.
+ *   w: HOST array of l_max structs, w[l-1] = weights of the layer at depth l; only w_router, shared_w_gate_up,
+ *      shared_w_down, lore_A and lore_B are read (of w[l_max-1] only w_router).
+ *   x_current [T,d] bf16.  1 <= l_min <= l_max <= 64.  tau: the threshold of Algorithm 1 (need not be cfg.tau).
+ *   idx_hat [l_max,T,K] int32 out: predicted sets, -1 past a token's last depth.  conf [l_max,T] fp32 out, 0 there.
+ *   depth [T] int32 out: number of predictions enqueued for the token (>= min(l_min, l_max)).
+ *   h_final [T,d] bf16 out, optional: the draft state after the last projection made for each token.
+ * The prefetch queue of Algorithm 1 is the union over l of idx_hat[l-1, t, :] for l <= depth[t]; issuing the copies is the
+ * host runtime's job.  The call launches about 8 kernels per depth and is bound by their launch latency at decode batches. */
+spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w /* host array */,
+                                    const spice_bf16 *x_current, int32_t T, int32_t l_min, int32_t l_max, float tau,
+                                    int32_t *idx_hat, float *conf, int32_t *depth, spice_bf16 *h_final, void *stream);
+
 /* The resident-expert FFN for callers that cannot allocate (the paper has no counterpart: this is
  * a packaging variant of spice_grouped_expert_ffn, not a step of the method).
  *

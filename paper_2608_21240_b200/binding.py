@@ -55,7 +55,7 @@ def lib() -> C.CDLL:
         for name in ("spice_create", "spice_destroy", "spice_workspace_bytes", "spice_route_topk",
                      "spice_classify_misses", "spice_grouped_expert_ffn", "spice_lore_surrogate",
                      "spice_moe_layer_fwd", "spice_get_device_status", "spice_launch_count", "spice_set_option",
-                     "spice_grouped_expert_ffn_static", "spice_draft_confidence"):
+                     "spice_grouped_expert_ffn_static", "spice_draft_confidence", "spice_prefetch_rollout"):
             getattr(L, name).restype = C.c_int
         L.spice_static_scratch_bytes.restype = C.c_size_t
         _lib = L
@@ -129,6 +129,16 @@ def spice_draft_confidence(ctx, h_hat, w_draft_router, T, idx_hat, conf, pi_hat=
     _check(lib().spice_draft_confidence(ctx, _ptr(h_hat, torch.bfloat16), _ptr(w_draft_router, torch.bfloat16), C.c_int32(T),
                                         _ptr(idx_hat, torch.int32), _ptr(pi_hat, torch.float32), _ptr(conf, torch.float32),
                                         _stream(stream)), "spice_draft_confidence")
+
+
+def spice_prefetch_rollout(ctx, weights, x_current, T, l_min, l_max, tau, idx_hat, conf, depth, h_final=None,
+                           stream=None) -> None:
+    """weights: sequence of l_max LayerWeightsC structs (depth 1 first)."""
+    arr = (LayerWeightsC * l_max)(*weights)
+    _check(lib().spice_prefetch_rollout(ctx, arr, _ptr(x_current, torch.bfloat16), C.c_int32(T), C.c_int32(l_min),
+                                        C.c_int32(l_max), C.c_float(tau), _ptr(idx_hat, torch.int32),
+                                        _ptr(conf, torch.float32), _ptr(depth, torch.int32), _ptr(h_final, torch.bfloat16),
+                                        _stream(stream)), "spice_prefetch_rollout")
 
 
 def spice_classify_misses(ctx, idx, gate, slot_of_expert, conf, T, cls, slot, counts, resid_tok=None, resid_k=None,
@@ -256,6 +266,17 @@ class SpiceLayer:
         pi = self._empty((T, N), torch.float32) if want_pi else None
         spice_draft_confidence(self.ctx, h_hat, w_draft_router, T, idx, conf, pi, stream)
         return (idx, conf, pi) if want_pi else (idx, conf)
+
+    def prefetch_rollout(self, weights, x_current, l_min, l_max, tau, stream=None):
+        """weights: list of l_max LayerWeights (depth 1 first).  Returns (idx_hat, conf, depth, h_final)."""
+        T, K = x_current.shape[0], self.cfg.top_k
+        idx = self._empty((l_max, T, K), torch.int32)
+        conf = self._empty((l_max, T), torch.float32)
+        depth = self._empty((T,), torch.int32)
+        h_final = self._empty((T, self.cfg.d), torch.bfloat16)
+        spice_prefetch_rollout(self.ctx, [w.c_struct() for w in weights], x_current, T, l_min, l_max, tau, idx, conf,
+                               depth, h_final, stream)
+        return idx, conf, depth, h_final
 
     def classify_misses(self, idx, gate, slot_of_expert, conf, stream=None):
         T, K = idx.shape

@@ -18,6 +18,10 @@ struct spice_ctx {
     uint8_t *ws_cls;
     float *y32;        // [Tm, d] fp32 accumulator of the fused call
     float *draft_logits;            // [Tm, N] logits of spice_draft_confidence when the caller does not want pi_hat
+    // speculative prefetch rollout
+    __nv_bfloat16 *roll_h, *roll_y; // [Tm, d] draft state and scratch output
+    float *roll_conf;               // [Tm]
+    int32_t *roll_active;           // [Tm]
     // fused decode kernel
     float *logits;                  // [Td, N]
     __nv_bfloat16 *act_hit16, *act_shared16, *z16;
@@ -77,6 +81,10 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->ws_cls = cv.take<uint8_t>(n);
     c->y32 = cv.take<float>(Tm * g.d);
     c->draft_logits = cv.take<float>(Tm * g.n_experts);
+    c->roll_h = cv.take<__nv_bfloat16>(Tm * g.d);
+    c->roll_y = cv.take<__nv_bfloat16>(Tm * g.d);
+    c->roll_conf = cv.take<float>(Tm);
+    c->roll_active = cv.take<int32_t>(Tm);
     // decode kernels: activations of a group are kept for every token of the batch ([group][T][width])
     const size_t Td = Tm < 64 ? Tm : 64, nd = Td * K;
     const size_t g_hit = (size_t)g.n_slots < nd ? g.n_slots : nd, g_low = (size_t)g.n_experts < nd ? g.n_experts : nd;
@@ -274,6 +282,29 @@ spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, con
     SPICE_LAUNCH(launch_draft_confidence(dims_of(ctx, T), reinterpret_cast<const __nv_bfloat16 *>(h_hat),
                                          reinterpret_cast<const __nv_bfloat16 *>(w_draft_router), idx_hat, ctx->ws_gate,
                                          ctx->draft_logits, pi_hat, conf, static_cast<cudaStream_t>(stream)));
+    return SPICE_OK;
+}
+
+spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *x_current, int32_t T,
+                                    int32_t l_min, int32_t l_max, float tau, int32_t *idx_hat, float *conf, int32_t *depth,
+                                    spice_bf16 *h_final, void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    if (l_max < 1 || l_max > 64 || l_min < 1 || l_min > l_max) return SPICE_ERR_INVALID_ARG;
+    if (T == 0) return SPICE_OK;
+    if (!w || !x_current || !idx_hat || !conf || !depth || !aligned16(x_current)) return SPICE_ERR_INVALID_ARG;
+    for (int l = 0; l < l_max; ++l) {
+        if (!w[l].w_router || !aligned16(w[l].w_router)) return SPICE_ERR_INVALID_ARG;
+        if (l + 1 < l_max && !weights_ok(&w[l], false, true)) return SPICE_ERR_INVALID_ARG;   // the last depth only routes
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Dims dm = dims_of(ctx, T);
+    const size_t bytes = (size_t)T * dm.d * sizeof(__nv_bfloat16);
+    if (cudaMemcpyAsync(ctx->roll_h, x_current, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SPICE_ERR_CUDA;
+    SPICE_LAUNCH(launch_rollout(dm, w, l_min, l_max, tau, ctx->roll_h, ctx->roll_y, ctx->ws_idx, ctx->ws_gate, ctx->ws_cls,
+                                ctx->roll_conf, ctx->draft_logits, ctx->roll_active, ctx->tb, idx_hat, conf, depth, st));
+    if (h_final && cudaMemcpyAsync(h_final, ctx->roll_h, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return SPICE_ERR_CUDA;
     return SPICE_OK;
 }
 

@@ -213,7 +213,12 @@ __global__ void __launch_bounds__(256) combine_kernel(Dims dm, CombineArgs a, Ta
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (a.accumulate) acc = *reinterpret_cast<const float4 *>(a.y32 + (size_t)t * d + j);
     if (a.kind_mask & KIND_SHARED) {
-        const float c = tb.coef_shared[t];
+        float c = tb.coef_shared[t];
+        if (a.shared_coef_low_sum) {   // sum of the LOWCONF gates alone, in k order
+            c = 0.f;
+            for (int k = 0; k < K; ++k)
+                if (a.cls[t * K + k] == SPICE_LOWCONF) c += a.gate[t * K + k];
+        }
         const float4 s = *reinterpret_cast<const float4 *>(tb.part_shared + (size_t)t * d + j);
         acc.x = fmaf(c, s.x, acc.x); acc.y = fmaf(c, s.y, acc.y);
         acc.z = fmaf(c, s.z, acc.z); acc.w = fmaf(c, s.w, acc.w);

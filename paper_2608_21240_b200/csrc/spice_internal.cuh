@@ -76,8 +76,14 @@ struct CombineArgs {
     __nv_bfloat16 *y16;         // bf16 output or NULL
     const float *y_cpu;         // optional fp32 addend
     __nv_bfloat16 *x_resid;     // optional bf16 in/out residual stream
+    int shared_coef_low_sum;    // 1: the shared expert enters with sum of LOWCONF gates (no "1 +"): rollout projection
 };
 int launch_combine(const Dims &dm, const CombineArgs &a, const Tables &tb, cudaStream_t st);
+
+// ---- speculative prefetch rollout, Algorithm 1 (rollout.cu); w: host array of l_max structs
+int launch_rollout(const Dims &dm, const spice_layer_weights *w, int l_min, int l_max, float tau, __nv_bfloat16 *h_state,
+                   __nv_bfloat16 *y_scratch, int32_t *idx_ws, float *gate_ws, uint8_t *cls_ws, float *conf_ws, float *logits_ws,
+                   int32_t *active_ws, const Tables &tb, int32_t *idx_hat, float *conf, int32_t *depth, cudaStream_t st);
 
 // ---- fused decode kernel (decode.cu)
 // words of the dependency-counter array

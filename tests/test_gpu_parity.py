@@ -319,6 +319,56 @@ def test_draft_confidence_matches_oracle_and_feeds_the_layer(name, T):
     L.close()
 
 
+def _rollout_case(shape, T, L, variant, l_min):
+    """Layers of depths 1..L from the seeded generator, a threshold that splits the tokens, and a check (through the
+    oracle) that every routing decision the rollout takes has a margin fp32 summation order cannot cross."""
+    for v in range(variant, variant + 50):
+        wls = [W.make_layer(shape, T, variant=v, layer=l) for l in range(L)]
+        enforce_margins(wls[0])
+        layers = [dict(w_router=wl.w_router, shared=wl.shared(), lore_A=wl.lore()[0], lore_B=wl.lore()[1]) for wl in wls]
+        x = wls[0].h
+        _, conf0, _, _ = oracle.prefetch_rollout(x, layers, shape.top_k, l_min, L, 0.0)
+        cs = np.sort(conf0[l_min - 1:].ravel())
+        tau = float(0.5 * (cs[cs.size // 2 - 1] + cs[cs.size // 2]))      # between two observed confidences
+        ok = np.abs(conf0 - tau).min() > 1e-4
+        for l in range(1, L + 1):
+            _, _, depth, h_prev = oracle.prefetch_rollout(x, layers[:l], shape.top_k, min(l_min, l), l, tau)
+            lg = np.sort(oracle.router_logits(h_prev.astype(np.float32), layers[l - 1]["w_router"]), axis=1)[:, ::-1]
+            gaps = (lg[:, :shape.top_k] - lg[:, 1:shape.top_k + 1]).min(axis=1)
+            ok = ok and bool((gaps[depth == l] >= 1e-3).all())
+        if ok:
+            return wls, layers, x, tau
+    raise AssertionError("no variant with safe margins found")
+
+
+@pytest.mark.parametrize("name,T,L,l_min", [("tiny", 6, 3, 1), ("tiny", 19, 4, 2), ("dsv2lite", 4, 3, 2)])
+def test_prefetch_rollout_matches_oracle(name, T, L, l_min):
+    """Algorithm 1: predicted sets and halting depths bit-exact, confidences within fp32 rounding, the draft state after
+    the last projection within the output tolerance."""
+    s = W.SHAPES[name]
+    wls, layers, x, tau = _rollout_case(s, T, L, 40, l_min)
+    ref_idx, ref_conf, ref_depth, ref_h = oracle.prefetch_rollout(x, layers, s.top_k, l_min, L, tau)
+    assert len(set(ref_depth.tolist())) > 1, "the threshold should stop some tokens early"
+    Lyr = B.SpiceLayer(cfg_of(s), T)
+    ws = [upload(wl) for wl in wls]
+    n0 = Lyr.launch_count()
+    idx, conf, depth, h_final = Lyr.prefetch_rollout(ws, bf16_tensor(x), l_min, L, tau)
+    torch.cuda.synchronize()
+    assert Lyr.device_status() == 0 and Lyr.launch_count() - n0 == 3 * L + 5 * (L - 1)
+    assert np.array_equal(depth.cpu().numpy(), ref_depth)
+    assert np.array_equal(idx.cpu().numpy(), ref_idx)
+    assert np.abs(conf.cpu().numpy().astype(np.float64) - ref_conf).max() <= s.top_k * GATE_ATOL
+    err, bound = y_close(h_final.float().cpu().numpy(), ref_h)
+    assert err <= bound + 2e-2, f"max err {err:.3e}"      # + bf16 rounding of the O(1) state
+    # depth 1 is the draft-confidence call
+    i1, c1 = Lyr.draft_confidence(bf16_tensor(x), ws[0].w_router)
+    assert torch.equal(i1, idx[0]) and torch.equal(c1, conf[0])
+    # argument errors launch nothing
+    with pytest.raises(B.SpiceError):
+        Lyr.prefetch_rollout(ws, bf16_tensor(x), L + 1, L, tau)
+    Lyr.close()
+
+
 def test_split_exports_compose_to_the_fused_call():
     wl = _layer_case("dsv2lite", 4, variant=2)
     s = wl.shape
