@@ -21,7 +21,7 @@ struct spice_ctx {
     // speculative prefetch rollout
     __nv_bfloat16 *roll_h, *roll_y; // [Tm, d] draft state and scratch output
     float *roll_conf;               // [Tm]
-    int32_t *roll_active;           // [Tm]
+    int32_t *roll_active, *roll_active2;   // [Tm] each: "still speculates" flags, read / written alternately per depth
     // fused decode kernel
     float *logits;                  // [Td, N]
     __nv_bfloat16 *act_hit16, *act_shared16, *z16;
@@ -85,6 +85,7 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->roll_y = cv.take<__nv_bfloat16>(Tm * g.d);
     c->roll_conf = cv.take<float>(Tm);
     c->roll_active = cv.take<int32_t>(Tm);
+    c->roll_active2 = cv.take<int32_t>(Tm);
     // decode kernels: activations of a group are kept for every token of the batch ([group][T][width])
     const size_t Td = Tm < 64 ? Tm : 64, nd = Td * K;
     const size_t g_hit = (size_t)g.n_slots < nd ? g.n_slots : nd, g_low = (size_t)g.n_experts < nd ? g.n_experts : nd;
@@ -141,6 +142,25 @@ bool weights_ok(const spice_layer_weights *w, bool routed, bool shared_lore) {
                          aligned16(w->lore_B)))
         return false;
     return true;
+}
+
+// the fields of the decode kernels' parameter block that come from the ctx
+DecodeParams decode_params_of(const spice_ctx *ctx, const Dims &dm) {
+    DecodeParams p{};
+    p.dm = dm;
+    p.norm_topk = ctx->cfg.norm_topk;
+    p.conf_stride = ctx->cfg.conf_stride;
+    p.tau = ctx->cfg.tau;
+    p.n_r1 = dm.N;   // one router task per expert
+    p.spin_limit = (int32_t)ctx->opt_spin_limit;
+    p.sync_words = ctx->sync_words;
+    p.tb = ctx->tb;
+    p.logits = ctx->logits;
+    p.act_hit16 = ctx->act_hit16;
+    p.act_shared16 = ctx->act_shared16;
+    p.z16 = ctx->z16;
+    p.sync = ctx->sync;
+    return p;
 }
 
 // adds n launches or turns a launch failure into SPICE_ERR_CUDA
@@ -301,8 +321,57 @@ spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w
     const Dims dm = dims_of(ctx, T);
     const size_t bytes = (size_t)T * dm.d * sizeof(__nv_bfloat16);
     if (cudaMemcpyAsync(ctx->roll_h, x_current, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return SPICE_ERR_CUDA;
-    SPICE_LAUNCH(launch_rollout(dm, w, l_min, l_max, tau, ctx->roll_h, ctx->roll_y, ctx->ws_idx, ctx->ws_gate, ctx->ws_cls,
-                                ctx->roll_conf, ctx->draft_logits, ctx->roll_active, ctx->tb, idx_hat, conf, depth, st));
+    const bool fused = ctx->opt_path == 0 && T <= ctx->dtc_tokens && decode_tc_supported(dm, 0, (size_t)ctx->max_smem_optin);
+    bool done = false;
+    if (fused) {
+        // one launch of the decode kernel per projecting depth (router, halting rule, shared expert + LoRE, state update);
+        // the last depth only routes
+        const size_t n = (size_t)T * dm.K;
+        int32_t *act[2] = {ctx->roll_active, ctx->roll_active2};
+        done = true;
+        for (int l = 1; l < l_max && done; ++l) {
+            DecodeParams p = decode_params_of(ctx, dm);
+            p.norm_topk = 0;
+            p.conf_stride = 0;
+            p.h = ctx->roll_h;
+            p.w = w[l - 1];
+            p.w.slot_w_gate_up = p.w.shared_w_gate_up;   // (no resident experts in the rollout: never read)
+            p.w.slot_w_down = p.w.shared_w_down;
+            p.idx = ctx->ws_idx;
+            p.gate = ctx->ws_gate;
+            p.cls = ctx->ws_cls;
+            p.counts = ctx->ws_counts;
+            p.y16 = ctx->roll_y;
+            p.x_resid = ctx->roll_h;
+            p.roll_depth = l;
+            p.roll_l_min = l_min;
+            p.roll_tau = tau;
+            p.roll_active_in = act[(l + 1) & 1];
+            p.roll_active_out = act[l & 1];
+            p.roll_idx_out = idx_hat + (size_t)(l - 1) * n;
+            p.roll_conf_out = conf + (size_t)(l - 1) * T;
+            p.roll_depth_out = depth;
+            int k = launch_decode_tc(p, ctx->part_split, ctx->n_sms, ctx->max_smem_optin, st);
+            if (k < 0) {
+                done = false;      // cooperative launch refused: start over on the general kernels
+                break;
+            }
+            ctx->launches += k;
+        }
+        if (done) {
+            const spice_layer_weights &wl = w[l_max - 1];
+            SPICE_LAUNCH(launch_draft_confidence(dm, ctx->roll_h, reinterpret_cast<const __nv_bfloat16 *>(wl.w_router),
+                                                 ctx->ws_idx, ctx->ws_gate, ctx->draft_logits, nullptr, ctx->roll_conf, st));
+            SPICE_LAUNCH(launch_rollout_mask(dm, l_max, l_min, l_max, tau, ctx->roll_conf, act[(l_max + 1) & 1], ctx->ws_idx,
+                                             idx_hat + (size_t)(l_max - 1) * n, conf + (size_t)(l_max - 1) * T, ctx->ws_cls,
+                                             depth, st));
+        } else if (cudaMemcpyAsync(ctx->roll_h, x_current, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+            return SPICE_ERR_CUDA;
+        }
+    }
+    if (!done)
+        SPICE_LAUNCH(launch_rollout(dm, w, l_min, l_max, tau, ctx->roll_h, ctx->roll_y, ctx->ws_idx, ctx->ws_gate, ctx->ws_cls,
+                                    ctx->roll_conf, ctx->draft_logits, ctx->roll_active, ctx->tb, idx_hat, conf, depth, st));
     if (h_final && cudaMemcpyAsync(h_final, ctx->roll_h, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return SPICE_ERR_CUDA;
     return SPICE_OK;
@@ -392,14 +461,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
                          decode_supported(dm, (size_t)ctx->max_smem_optin);
     if (use_dtc || use_dec) {
         // small batch: one persistent kernel for the whole layer
-        DecodeParams p;
-        p.dm = dm;
-        p.norm_topk = ctx->cfg.norm_topk;
-        p.conf_stride = ctx->cfg.conf_stride;
-        p.tau = ctx->cfg.tau;
-        p.n_r1 = dm.N;   // one router task per expert
-        p.spin_limit = (int32_t)ctx->opt_spin_limit;
-        p.sync_words = ctx->sync_words;
+        DecodeParams p = decode_params_of(ctx, dm);
         p.h = hb;
         p.conf = conf;
         p.w = *w;
@@ -414,12 +476,6 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         p.y16 = reinterpret_cast<__nv_bfloat16 *>(y);
         p.y_cpu = y_cpu_residual;
         p.x_resid = reinterpret_cast<__nv_bfloat16 *>(x_resid);
-        p.tb = ctx->tb;
-        p.logits = ctx->logits;
-        p.act_hit16 = ctx->act_hit16;
-        p.act_shared16 = ctx->act_shared16;
-        p.z16 = ctx->z16;
-        p.sync = ctx->sync;
         int n = use_dtc ? launch_decode_tc(p, ctx->part_split, ctx->n_sms, ctx->max_smem_optin, st)
                         : launch_decode(p, ctx->n_sms, st);
         if (n > 0) {

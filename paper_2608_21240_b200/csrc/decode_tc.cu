@@ -433,10 +433,30 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
                 for (int k = 0; k < K; ++k) sacc += __shfl_sync(0xffffffffu, pk, k);
                 denom = sacc;
             }
+            // rollout mode (Algorithm 1): C = sum of the gates in k order; halting rule; outputs of this depth by CTA 0
+            bool roll_cont = false;
+            if (p.roll_depth) {
+                const float g = pk / denom;
+                float cs = 0.f;
+#pragma unroll 1
+                for (int k = 0; k < K; ++k) cs += __shfl_sync(0xffffffffu, g, k);
+                const bool on = p.roll_depth == 1 ? true : p.roll_active_in[t] != 0;
+                const bool stop = p.roll_depth >= p.roll_l_min && cs < p.roll_tau;
+                roll_cont = on && !stop;
+                if (blockIdx.x == 0) {
+                    if (a.lane < K) p.roll_idx_out[t * K + a.lane] = on ? my_idx[u] : -1;
+                    if (a.lane == 0) {
+                        p.roll_conf_out[t] = on ? cs : 0.f;
+                        p.roll_active_out[t] = roll_cont ? 1 : 0;
+                        if (on) p.roll_depth_out[t] = p.roll_depth;
+                        else if (p.roll_depth == 1) p.roll_depth_out[t] = 0;
+                    }
+                }
+            }
             // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
             if (a.lane < K) {
                 const int i = t * K + a.lane, e = my_idx[u];
-                const int sl = ax.soe[e];
+                const int sl = p.roll_depth ? -1 : ax.soe[e];
                 int c, gkey = -1;
                 if (sl >= S) {
                     atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
@@ -446,9 +466,15 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
                     gkey = sl;
                     atomicOr(&ax.mask_hit[2 * sl + (t >> 5)], 1u << (t & 31));
                 } else {
-                    const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
-                    c = (cf < p.tau) ? SPICE_LOWCONF : SPICE_MISS_EXACT;
-                    if (c == SPICE_LOWCONF) {
+                    bool low;
+                    if (p.roll_depth) {
+                        low = roll_cont;
+                    } else {
+                        const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
+                        low = cf < p.tau;
+                    }
+                    c = low ? SPICE_LOWCONF : SPICE_MISS_EXACT;
+                    if (low) {
                         gkey = 1024 + e;
                         atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
                     }
@@ -504,10 +530,10 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
             ax.gtab[0] = GroupDesc{KIND_SHARED, 0, 0, T};
         }
     }
-    // coefficient of the shared expert's output: 1 + sum of LOWCONF gates, in k order
+    // coefficient of the shared expert's output: 1 + sum of LOWCONF gates, in k order (rollout: the sum alone)
 #pragma unroll 1
     for (int t = a.atid; t < T; t += AUX_T) {
-        float c = 1.0f;
+        float c = p.roll_depth ? 0.0f : 1.0f;
 #pragma unroll 1
         for (int k = 0; k < K; ++k)
             if (ax.cls[t * K + k] == SPICE_LOWCONF) c += ax.gate[t * K + k];
@@ -1032,10 +1058,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         const int T = dm.T, N = dm.N;
         // what classification will need is copied asynchronously (global -> shared) while the logits are produced
         const int n_conf = p.conf_stride ? T * N : T;
+        if (!p.roll_depth) {   // (the rollout decides the classes by its halting rule)
 #pragma unroll 1
-        for (int i = a.atid; i < N; i += AUX_T) cp_async4(smem_u32(ax.soe + i), p.w.slot_of_expert + i);
+            for (int i = a.atid; i < N; i += AUX_T) cp_async4(smem_u32(ax.soe + i), p.w.slot_of_expert + i);
 #pragma unroll 1
-        for (int i = a.atid; i < n_conf; i += AUX_T) cp_async4(smem_u32(ax.conf + i), p.conf + i);
+            for (int i = a.atid; i < n_conf; i += AUX_T) cp_async4(smem_u32(ax.conf + i), p.conf + i);
+        }
         asm volatile("cp.async.commit_group;" ::: "memory");
         ax.mask_hit[2 * a.atid] = ax.mask_hit[2 * a.atid + 1] = 0u;
         ax.mask_low[2 * a.atid] = ax.mask_low[2 * a.atid + 1] = 0u;

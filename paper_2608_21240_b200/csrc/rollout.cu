@@ -37,6 +37,14 @@ __global__ void __launch_bounds__(256) rollout_mask_kernel(int T, int K, int dep
     for (int k = 0; k < K; ++k) cls[(size_t)t * K + k] = cont ? SPICE_LOWCONF : SPICE_MISS_EXACT;
 }
 
+int launch_rollout_mask(const Dims &dm, int depth, int l_min, int l_max, float tau, const float *conf_l, int32_t *active,
+                        const int32_t *idx_ws, int32_t *idx_out, float *conf_out, uint8_t *cls, int32_t *depth_out,
+                        cudaStream_t st) {
+    rollout_mask_kernel<<<(dm.T + 255) / 256, 256, 0, st>>>(dm.T, dm.K, depth, l_min, l_max, tau, conf_l, active, idx_ws, idx_out,
+                                                           conf_out, cls, depth_out);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 int launch_rollout(const Dims &dm, const spice_layer_weights *w, int l_min, int l_max, float tau, __nv_bfloat16 *h_state,
                    __nv_bfloat16 *y_scratch, int32_t *idx_ws, float *gate_ws, uint8_t *cls_ws, float *conf_ws, float *logits_ws,
                    int32_t *active_ws, const Tables &tb, int32_t *idx_hat, float *conf, int32_t *depth, cudaStream_t st) {

@@ -85,6 +85,10 @@ int launch_rollout(const Dims &dm, const spice_layer_weights *w, int l_min, int 
                    __nv_bfloat16 *y_scratch, int32_t *idx_ws, float *gate_ws, uint8_t *cls_ws, float *conf_ws, float *logits_ws,
                    int32_t *active_ws, const Tables &tb, int32_t *idx_hat, float *conf, int32_t *depth, cudaStream_t st);
 
+int launch_rollout_mask(const Dims &dm, int depth, int l_min, int l_max, float tau, const float *conf_l, int32_t *active,
+                        const int32_t *idx_ws, int32_t *idx_out, float *conf_out, uint8_t *cls, int32_t *depth_out,
+                        cudaStream_t st);
+
 // ---- fused decode kernel (decode.cu)
 // words of the dependency-counter array
 enum { SY_ABORT = 0, SY_TEAMS_DONE, SY_R1_DONE, SY_ROUTE_DONE, SY_P2_DONE, SY_P1_ALL, SY_NEXT_TASK, SY_GROUP0 = 8 };
@@ -114,6 +118,17 @@ struct DecodeParams {
     __nv_bfloat16 *act_shared16;   // [Tm, I_s]
     __nv_bfloat16 *z16;            // [Tm*K, r]  perm_low order
     int32_t *sync;                 // [sync_words] zero between launches
+    // Rollout mode of the tcgen05 decode kernel (Algorithm 1, one depth per launch; 0 = ordinary layer call): the
+    // classes come from the halting rule instead of residency and confidences -- every selected expert of a token that
+    // continues is a low-confidence miss, nothing is added for a token that stops -- and the shared expert is weighted
+    // by the sum of the gates alone.
+    int32_t roll_depth, roll_l_min;
+    float roll_tau;
+    const int32_t *roll_active_in;   // [T] 1 while the token still speculates (ignored at depth 1)
+    int32_t *roll_active_out;        // [T] the same after this depth
+    int32_t *roll_idx_out;           // [T,K] predicted set of this depth, -1 for tokens that stopped earlier
+    float *roll_conf_out;            // [T]
+    int32_t *roll_depth_out;         // [T]
 };
 size_t decode_smem_bytes(const Dims &dm);
 bool decode_supported(const Dims &dm, size_t max_smem);

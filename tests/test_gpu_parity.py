@@ -321,8 +321,10 @@ def test_draft_confidence_matches_oracle_and_feeds_the_layer(name, T):
 
 def _rollout_case(shape, T, L, variant, l_min):
     """Layers of depths 1..L from the seeded generator, a threshold that splits the tokens, and a check (through the
-    oracle) that every routing decision the rollout takes has a margin fp32 summation order cannot cross."""
-    for v in range(variant, variant + 50):
+    oracle) that every decision the rollout takes has a margin that rounding cannot cross: 1e-3 between logits at depth 1
+    (fp32 summation order), 5e-3 at later depths and 1e-3 between a confidence and the threshold (the draft state is bf16
+    and the GPU also rounds the intermediate activations to bf16, which moves later logits by up to ~1e-3)."""
+    for v in range(variant, variant + 300):
         wls = [W.make_layer(shape, T, variant=v, layer=l) for l in range(L)]
         enforce_margins(wls[0])
         layers = [dict(w_router=wl.w_router, shared=wl.shared(), lore_A=wl.lore()[0], lore_B=wl.lore()[1]) for wl in wls]
@@ -330,18 +332,18 @@ def _rollout_case(shape, T, L, variant, l_min):
         _, conf0, _, _ = oracle.prefetch_rollout(x, layers, shape.top_k, l_min, L, 0.0)
         cs = np.sort(conf0[l_min - 1:].ravel())
         tau = float(0.5 * (cs[cs.size // 2 - 1] + cs[cs.size // 2]))      # between two observed confidences
-        ok = np.abs(conf0 - tau).min() > 1e-4
+        ok = np.abs(conf0 - tau).min() > 1e-3
         for l in range(1, L + 1):
             _, _, depth, h_prev = oracle.prefetch_rollout(x, layers[:l], shape.top_k, min(l_min, l), l, tau)
             lg = np.sort(oracle.router_logits(h_prev.astype(np.float32), layers[l - 1]["w_router"]), axis=1)[:, ::-1]
             gaps = (lg[:, :shape.top_k] - lg[:, 1:shape.top_k + 1]).min(axis=1)
-            ok = ok and bool((gaps[depth == l] >= 1e-3).all())
+            ok = ok and bool((gaps[depth == l] >= (1e-3 if l == 1 else 5e-3)).all())
         if ok:
             return wls, layers, x, tau
     raise AssertionError("no variant with safe margins found")
 
 
-@pytest.mark.parametrize("name,T,L,l_min", [("tiny", 6, 3, 1), ("tiny", 19, 4, 2), ("dsv2lite", 4, 3, 2)])
+@pytest.mark.parametrize("name,T,L,l_min", [("tiny", 6, 3, 1), ("tiny", 9, 4, 2), ("dsv2lite", 4, 3, 2)])
 def test_prefetch_rollout_matches_oracle(name, T, L, l_min):
     """Algorithm 1: predicted sets and halting depths bit-exact, confidences within fp32 rounding, the draft state after
     the last projection within the output tolerance."""
@@ -354,15 +356,28 @@ def test_prefetch_rollout_matches_oracle(name, T, L, l_min):
     n0 = Lyr.launch_count()
     idx, conf, depth, h_final = Lyr.prefetch_rollout(ws, bf16_tensor(x), l_min, L, tau)
     torch.cuda.synchronize()
-    assert Lyr.device_status() == 0 and Lyr.launch_count() - n0 == 3 * L + 5 * (L - 1)
+    # one fused launch per projecting depth + the last depth's router, confidence and halting kernels
+    assert Lyr.device_status() == 0 and Lyr.launch_count() - n0 == (L - 1) + 3
     assert np.array_equal(depth.cpu().numpy(), ref_depth)
     assert np.array_equal(idx.cpu().numpy(), ref_idx)
-    assert np.abs(conf.cpu().numpy().astype(np.float64) - ref_conf).max() <= s.top_k * GATE_ATOL
+    dconf = np.abs(conf.cpu().numpy().astype(np.float64) - ref_conf)
+    assert dconf[0].max() <= s.top_k * GATE_ATOL and dconf.max() <= 1e-3      # later depths inherit the bf16 state's rounding
     err, bound = y_close(h_final.float().cpu().numpy(), ref_h)
     assert err <= bound + 2e-2, f"max err {err:.3e}"      # + bf16 rounding of the O(1) state
     # depth 1 is the draft-confidence call
     i1, c1 = Lyr.draft_confidence(bf16_tensor(x), ws[0].w_router)
     assert torch.equal(i1, idx[0]) and torch.equal(c1, conf[0])
+    # the same rollout on the general-shape kernels
+    Lyr.set_option(B.OPT_PATH, 1)
+    n1 = Lyr.launch_count()
+    gidx, gconf, gdepth, gh = Lyr.prefetch_rollout(ws, bf16_tensor(x), l_min, L, tau)
+    torch.cuda.synchronize()
+    assert Lyr.launch_count() - n1 == 3 * L + 5 * (L - 1)
+    assert torch.equal(gidx, idx) and torch.equal(gdepth, depth)
+    assert (gconf[0] - conf[0]).abs().max().item() <= s.top_k * GATE_ATOL and (gconf - conf).abs().max().item() <= 1e-3
+    err, bound = y_close(gh.float().cpu().numpy(), ref_h)
+    assert err <= bound + 2e-2
+    Lyr.set_option(B.OPT_PATH, 0)
     # argument errors launch nothing
     with pytest.raises(B.SpiceError):
         Lyr.prefetch_rollout(ws, bf16_tensor(x), L + 1, L, tau)
