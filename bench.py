@@ -7,7 +7,11 @@ DeepSeek-V2-Lite-shaped layer.  Successive steps rotate through several independ
 layer weight sets so that the bytes touched between two uses of the same weights are
 several times the L2 capacity (cold-L2 timing without a flush inside the timed region).
 
-Prints ONE JSON line (see README for the keys).
+Prints ONE JSON line: metric, value, unit, timing, `config` (the workload), `roofline` (algorithmic bytes or FLOPs of
+the timed calls over their time, against the measured peak), `e2e` (the same metric with host<->device copies inside
+the timed region), `cpu_baseline` (the CPU oracle on the host cores), `clocks`, `gpu_launches`.
+
+Other modes: --stack (26-layer decode stack), --op draft_confidence, --op rollout, --impl reference (CPU oracle).
 """
 from __future__ import annotations
 
