@@ -87,6 +87,7 @@ struct Ctl {
     int n_hg, n_lg;
     int aux_flag;
     int last_flag;
+    int no_more;   // the producer has issued its last task
     int wsum[2][AUX_W];
     int s_cnt[4];
 };
@@ -687,6 +688,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         sh->abort_flag = 0;
         sh->aux_flag = 0;
         sh->last_flag = 0;
+        sh->no_more = 0;
         sh->n_hg = sh->n_lg = 0;
         for (int i = 0; i < 4; ++i) sh->s_cnt[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -821,19 +823,29 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     dep_target = 4 * pl.tz;
                 }
                 if (lane == 0) DPROF(0, npf, 10 + t.kind);
+                // this lane's copy of every stage: lane 0 the weights, lane 1 the tokens (sub-chunk 0 only when the
+                // maps are plain); lanes 2, 3 the same for sub-chunk 1 of plain maps
+                const int sub = lane >> 1, is_b = lane & 1;
+                const CUtensorMap *my_map = is_b ? mb : ma;
+                const uint32_t my_off = is_b ? (uint32_t)(A_BYTES + sub * NB * 128) : (uint32_t)(sub * SUB_A);
+                const int my_y = is_b ? 0 : a_row0;
+                const int my_z = is_b ? b_z : a_z;
+                const bool my_on = sub == 0 || plain;
+                auto copy = [&](int kb, int stage) {   // this lane's box of k-stage kb into ring stage `stage`
+                    const uint32_t full = smem_u32(&sh->full[stage]);
+                    const uint32_t dst = smem_u32(ring + (size_t)stage * STAGE_BYTES);
+                    if (plain) tma_load_5d(dst + my_off, my_map, (k0 + kb) * KSTAGE + sub * 64, my_y, 0, 0, my_z, full);
+                    else tma_load_5d(dst + my_off, my_map, 0, my_y, 0, (k0 + kb) * 2, my_z, full);
+                };
+                // has the watcher warp already seen the group complete?
+                bool pending = false;
                 if (dep >= 0) {
-                    int r = 1;
+                    int seen = 0;
                     if (lane == 0) {
-                        const int seen = ld_acquire_cta(ax.ready + t.gi);
+                        seen = ld_acquire_cta(ax.ready + t.gi);
                         DPROF(0, npf, 24 + (seen ? 1 : 0));
-                        if (!seen)   // not yet seen by the watcher warp: poll here
-                            r = wait_ge(p.sync + dep, dep_target, p.sync, p.tb.status, p.spin_limit, abort_flag) ? 1 : 0;
                     }
-                    __syncwarp(PM);
-                    if (__shfl_sync(PM, r, 0) == 0) { ok = false; break; }
-                    if (lane == 0) DPROF(0, npf, 22);
-                    fence_proxy_async();
-                    if (lane == 0) DPROF(0, npf, 23);
+                    pending = __shfl_sync(PM, seen, 0) == 0;
                 }
                 {   // hand the task to the MMA and epilogue roles
                     const int slot = tcount % TQ;
@@ -845,27 +857,45 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     ++tcount;
                 }
                 if (lane == 0) DPROF(0, npf, 21);
+                int kb0 = 0;
+                if (pending) {
+                    // The activations are not there yet, but the weights do not depend on them: arm the first stages
+                    // and start their weight copies, wait, then add the token copies to the same stages.
+                    const int pre = min(t.nk, stages);
+                    const int s0 = s;
+                    for (int kb = 0; kb < pre && ok; ++kb, ++it) {
+                        if (!lead_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1)) { ok = false; break; }
+                        if (lane == 0) mbar_expect_tx(smem_u32(&sh->full[s]), STAGE_BYTES);
+                        __syncwarp(PM);
+                        if (my_on && !is_b) copy(kb, s);
+                        if (++s == stages) {
+                            s = 0;
+                            ring_phase ^= 1;
+                        }
+                    }
+                    if (!ok) break;
+                    int r = 1;
+                    if (lane == 0) r = wait_ge(p.sync + dep, dep_target, p.sync, p.tb.status, p.spin_limit, abort_flag) ? 1 : 0;
+                    __syncwarp(PM);
+                    if (__shfl_sync(PM, r, 0) == 0) { ok = false; break; }
+                    if (lane == 0) DPROF(0, npf, 22);
+                    fence_proxy_async();
+                    for (int kb = 0, ss = s0; kb < pre; ++kb) {
+                        if (my_on && is_b) copy(kb, ss);
+                        if (++ss == stages) ss = 0;
+                    }
+                    kb0 = pre;
+                } else if (dep >= 0) {
+                    fence_proxy_async();
+                }
                 // (drawn only now: an acquire or a fence issued while the atomic is in flight would wait for it)
                 int drawn = 0;
                 if (lane == 0) drawn = (int)gridDim.x + atomicAdd(p.sync + SY_NEXT_TASK, 1);
-                // this lane's copy of every stage: lane 0 the weights, lane 1 the tokens (sub-chunk 0 only when the
-                // maps are plain); lanes 2, 3 the same for sub-chunk 1 of plain maps
-                const int sub = lane >> 1, is_b = lane & 1;
-                const CUtensorMap *my_map = is_b ? mb : ma;
-                const uint32_t my_off = is_b ? (uint32_t)(A_BYTES + sub * NB * 128) : (uint32_t)(sub * SUB_A);
-                const int my_y = is_b ? 0 : a_row0;
-                const int my_z = is_b ? b_z : a_z;
-                const bool my_on = sub == 0 || plain;
-                for (int kb = 0; kb < t.nk; ++kb, ++it) {
+                for (int kb = kb0; kb < t.nk; ++kb, ++it) {
                     if (!lead_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1)) { ok = false; break; }
-                    const uint32_t full = smem_u32(&sh->full[s]);
-                    const uint32_t dst = smem_u32(ring + (size_t)s * STAGE_BYTES);
-                    if (lane == 0) mbar_expect_tx(full, STAGE_BYTES);
+                    if (lane == 0) mbar_expect_tx(smem_u32(&sh->full[s]), STAGE_BYTES);
                     __syncwarp(PM);
-                    if (my_on) {
-                        if (plain) tma_load_5d(dst + my_off, my_map, (k0 + kb) * KSTAGE + sub * 64, my_y, 0, 0, my_z, full);
-                        else tma_load_5d(dst + my_off, my_map, 0, my_y, 0, (k0 + kb) * 2, my_z, full);
-                    }
+                    if (my_on) copy(kb, s);
 #ifdef SPICE_PROF_STAGES
                     if (lane == 0 && it < 64) DPROF(0, npf, 90);
 #endif
@@ -875,6 +905,8 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     }
                 }
                 id = __shfl_sync(PM, drawn, 0);
+                // nothing will follow this task: let the epilogue publish its down tiles as it finishes them
+                if (routed && id >= end && lane == 0) st_release_cta(&sh->no_more, 1);
             }
             if (lane == 0) DPROF(0, npf, 40);
             if (ok && lane == 0) {   // tell the other roles that the list is exhausted
@@ -1032,6 +1064,11 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             if (warp == 2 && lane == 0) DPROF(1, npf, 57);
             if (t.kind == TASK_DOWN) {
                 ++n_down;
+                if (ld_acquire_cta(&sh->no_more)) {   // (warp-uniform: one shared word)
+                    __syncwarp();
+                    if (lane == 0) red_release_add(p.sync + SY_P2_DONE, n_down);
+                    n_down = 0;
+                }
                 if (lane == 0) mbar_arrive(smem_u32(&sh->tq_empty[slot]));
             } else {
                 // Publish: only warps that stored rows signal (gate/up tiles: the two gate-row warps).  The release is
