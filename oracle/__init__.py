@@ -108,6 +108,31 @@ def draft_confidence(logits, K: int):
     return idx, pi, conf
 
 
+def lore_calibrate(H, R, rank: int, ridge: float = 0.0):
+    """LoRE calibration of one (layer, expert) pair (Sec. 4.2): the rank-r linear map Delta(h) = B A h that minimises
+        sum_{h in D} || E(h) - S(h) - B A h ||_2^2
+    over the calibration tokens, H [n,d] the hidden states and R [n,d] the residual targets E(h) - S(h).
+    Written out as the closed-form minimiser (reduced-rank regression): the least-squares map W (R ~ H W), the fitted
+    values H W, their r leading right singular vectors V; then B = V and A = (W V)^T.  With ridge > 0 the
+    least-squares step is regularised: W = (H^T H + ridge * tr(H^T H)/d * I)^-1 H^T R.
+    Returns (A [r,d], B [d,r], loss) in fp64; loss is the objective at (A, B)."""
+    H = np.asarray(H, dtype=np.float64)
+    R = np.asarray(R, dtype=np.float64)
+    n, d = H.shape
+    G = H.T @ H
+    if ridge > 0.0:
+        W = np.linalg.solve(G + ridge * np.trace(G) / d * np.eye(d), H.T @ R)
+    else:
+        W = np.linalg.lstsq(H, R, rcond=None)[0]
+    fitted = H @ W
+    _, _, Vt = np.linalg.svd(fitted, full_matrices=False)
+    V = Vt[:rank].T
+    B = V
+    A = (W @ V).T
+    loss = float(((R - (H @ A.T) @ B.T) ** 2).sum())
+    return A, B, loss
+
+
 def _round_bf16(x: np.ndarray) -> np.ndarray:
     """Nearest bf16 (ties to even) of fp64 values, returned as fp64: the draft state is kept in bf16 between depths."""
     u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)

@@ -437,3 +437,53 @@ def test_p14_rollout_fixed_point_when_nothing_is_added():
     x = W.bf16_round(rng.standard_normal((T, d)).astype(np.float32))
     idx, conf, depth, h = oracle.prefetch_rollout(x, layers, K, 1, L, 0.0)
     assert np.array_equal(h, x) and all(np.array_equal(idx[l], idx[0]) and np.array_equal(conf[l], conf[0]) for l in range(L))
+
+
+# ------------------------------------------------------------------ LoRE calibration (Sec. 4.2, the fitting objective)
+def _lore_loss(H, R, A, B):
+    return float(((R - (H @ A.T) @ B.T) ** 2).sum())
+
+
+def test_p15_lore_calibration_is_eckart_young_for_orthonormal_inputs():
+    """H with orthonormal columns and an exactly linear target R = H M^T: the objective is ||M - BA||_F^2, whose minimiser
+    over rank-r maps is the truncated SVD of M (Eckart-Young), with loss = sum of the discarded squared singular values."""
+    rng = np.random.default_rng(21)
+    n, d, r = 40, 12, 4
+    H = np.linalg.qr(rng.standard_normal((n, d)))[0]
+    M = rng.standard_normal((d, d))
+    A, B, loss = oracle.lore_calibrate(H, H @ M.T, r)
+    U, S, Vt = np.linalg.svd(M)
+    assert np.allclose(B @ A, (U[:, :r] * S[:r]) @ Vt[:r], atol=1e-10)
+    assert abs(loss - (S[r:] ** 2).sum()) <= 1e-10 * (S ** 2).sum()
+
+
+def test_p15_lore_calibration_recovers_a_rank_r_residual_exactly_and_improves_with_rank():
+    rng = np.random.default_rng(22)
+    n, d, r = 60, 16, 3
+    H = rng.standard_normal((n, d)) * np.linspace(0.3, 2.0, d)        # anisotropic inputs
+    A0, B0 = rng.standard_normal((r, d)), rng.standard_normal((d, r))
+    R = (H @ A0.T) @ B0.T
+    A, B, loss = oracle.lore_calibrate(H, R, r)
+    assert loss <= 1e-18 * (R ** 2).sum() and np.allclose(B @ A, B0 @ A0, atol=1e-9)
+    # a generic (full-rank, noisy) target: the loss falls with the rank and reaches ordinary least squares at r = d
+    R = rng.standard_normal((n, d)) + H @ rng.standard_normal((d, d))
+    losses = [oracle.lore_calibrate(H, R, k)[2] for k in range(1, d + 1)]
+    assert all(a >= b - 1e-9 for a, b in zip(losses, losses[1:]))
+    ols = float(((R - H @ np.linalg.lstsq(H, R, rcond=None)[0]) ** 2).sum())
+    assert abs(losses[-1] - ols) <= 1e-9 * ols
+
+
+def test_p15_lore_calibration_is_a_minimum():
+    """No rank-r perturbation of the returned factors lowers the objective (first-order optimality, probed at random),
+    and random rank-r maps are worse."""
+    rng = np.random.default_rng(23)
+    n, d, r = 50, 10, 2
+    H = rng.standard_normal((n, d)) * np.linspace(0.5, 1.5, d)
+    R = rng.standard_normal((n, d)) + H @ rng.standard_normal((d, d)) * 0.5
+    A, B, loss = oracle.lore_calibrate(H, R, r)
+    assert abs(loss - _lore_loss(H, R, A, B)) <= 1e-9 * loss
+    for _ in range(200):
+        dA, dB = rng.standard_normal(A.shape), rng.standard_normal(B.shape)
+        for eps in (1e-3, 1e-2, 1e-1):
+            assert _lore_loss(H, R, A + eps * dA, B + eps * dB) >= loss - 1e-9 * loss
+    assert min(_lore_loss(H, R, rng.standard_normal(A.shape), rng.standard_normal(B.shape)) for _ in range(50)) > loss
