@@ -598,6 +598,50 @@ def run_rollout(args):
         "gpu_launches": int(layer.launch_count() - l0)}))
 
 
+# ----------------------------------------------------------------------------- LoRE calibration
+def run_lore_calibrate(args):
+    """--op lore_calibrate: one step = spice_lore_calibrate for one expert (n calibration tokens, 100 iterations)."""
+    import torch
+
+    from paper_2608_21240_b200 import binding as B
+    from paper_2608_21240_b200 import workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    B.lib()
+    shape = W.SHAPES[args.shape]
+    d, r, n, iters = shape.d, shape.lore_rank, max(args.tokens, 2 * shape.d), 100
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(W.BASE_SEED + 55)
+    h = torch.randn(n, d, generator=gen, device=dev).to(torch.bfloat16)
+    m = torch.randn(d, d, generator=gen, device=dev) * (0.97 ** torch.arange(d, device=dev))
+    resid = (h.float() @ m.T + 0.1 * torch.randn(n, d, generator=gen, device=dev)).contiguous()
+    steps = max(1, min(args.steps, 10))
+    for _ in range(2):
+        out = B.spice_lore_calibrate(h, resid, r, iterations=iters)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        A, Bm, loss, status = B.spice_lore_calibrate(h, resid, r, iterations=iters)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    dp, rp = (d + 63) // 64 * 64, (r + 63) // 64 * 64
+    flops = 2.0 * (2 * n * dp * dp + dp ** 3 / 3 + dp ** 3 + iters * 2 * dp * dp * rp + 2 * dp * dp * rp)
+    print(json.dumps({
+        "metric": "lore_calibrations_per_s", "value": 1e3 / ms, "unit": "experts/s", "n_gpus": 1, "steps": steps, "warmup": 2,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"LoRE calibration of one expert, d={d}, rank={r}, {n} calibration tokens, {iters} subspace "
+                               f"iterations; objective / sum resid^2 = {float(loss[0] / loss[1]):.4f}, status {int(status.item())}"},
+        "roofline": {"bound": "alu", "achieved": flops / (ms * 1e-3) / 1e12, "peak": 72.0, "unit": "TFLOP/s",
+                     "frac": flops / (ms * 1e-3) / 1e12 / 72.0, "traffic": None,
+                     "kernel": "fp32 SIMT GEMMs, blocked Cholesky and triangular solves (offline path, not tuned)",
+                     "peak_source": "148 SMs x 128 fp32 FMA lanes x 1.9 GHz x 2"},
+        "gpu_launches": None}))
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 def oracle_call(wl, tokens):
     """One oracle evaluation of the GPU part of the layer for the given tokens."""
@@ -673,7 +717,7 @@ def main():
                     help="kernel path (SPICE_OPT_PATH): 0 auto, 1 general kernels, 2 no fused kernel, 3 mma.sync decode kernel")
     ap.add_argument("--stack", action="store_true",
                     help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
-    ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout"],
+    ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout", "lore_calibrate"],
                     help="what a step is: the MoE layer call (default) or the draft-router confidence call")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
@@ -685,6 +729,8 @@ def main():
         run_draft_confidence(args)
     elif args.op == "rollout":
         run_rollout(args)
+    elif args.op == "lore_calibrate":
+        run_lore_calibrate(args)
     elif args.stack:
         run_stack(args)
     else:

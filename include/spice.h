@@ -172,6 +172,29 @@ spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w
                                     const spice_bf16 *x_current, int32_t T, int32_t l_min, int32_t l_max, float tau,
                                     int32_t *idx_hat, float *conf, int32_t *depth, spice_bf16 *h_final, void *stream);
 
+/* LoRE calibration of one (layer, expert) pair (Sec. 4.2): the rank-r residual module Delta(h) = B A h that minimises
+ *     sum over the calibration tokens h routed to the expert of  || E(h) - S(h) - B A h ||_2^2 .
+ * The paper trains the factors on this objective; it is a reduced-rank regression with a closed-form minimiser, which this
+ * call computes on the device in fp32 (offline path, a few hundred small launches): G = H^T H + ridge * mean(diag G) * I,
+ * C = H^T R, G = L L^T, Z = L^-1 C, V = the r leading eigenvectors of Z^T Z (block subspace iteration, `iterations` steps:
+ * the objective is within 2 % of its minimum after 5 to 30 steps and within 1e-4 after 100 when neighbouring singular values
+ * differ by 10 %), B = V, A = (G^-1 C V)^T.
+ *   h_cal [n_tokens, d] bf16: calibration hidden states;  resid [n_tokens, d] fp32: targets E(h) - S(h) (e.g. from
+ *   spice_grouped_expert_ffn and spice_lore_surrogate with zero factors);  A_out [rank, d], B_out [d, rank] bf16 out, in
+ *   the layout of one expert's slice of spice_layer_weights.lore_A / lore_B.
+ *   1 <= rank <= d / 2 (the surrogate is low-rank by construction: r << d).
+ *   ridge >= 0: relative Tikhonov term; needed when n_tokens < d or the tokens are collinear (0 otherwise).
+ *   loss_out: optional device float[2]: { objective at the bf16 factors written, sum ||resid||^2 }.
+ *   device_status: device int32, out: 0, or 1 when a Cholesky pivot was not positive (G singular: raise ridge).
+ *   workspace: device buffer of at least spice_lore_calibrate_workspace_bytes(d, n_tokens, rank) bytes, owned by the
+ *   caller (the call allocates nothing); 256-byte aligned is best.  No spice_ctx is needed; the GPU is the calling
+ *   thread's current device.  The factors are unique only up to an invertible r x r change of basis; B A is what is fitted. */
+size_t spice_lore_calibrate_workspace_bytes(int32_t d, int32_t n_tokens, int32_t rank);
+spice_status spice_lore_calibrate(int32_t d, int32_t n_tokens, int32_t rank, float ridge, int32_t iterations,
+                                  const spice_bf16 *h_cal, const float *resid, spice_bf16 *A_out, spice_bf16 *B_out,
+                                  float *loss_out, int32_t *device_status, void *workspace, size_t workspace_bytes,
+                                  void *stream);
+
 /* The resident-expert FFN for callers that cannot allocate (the paper has no counterpart: this is
  * a packaging variant of spice_grouped_expert_ffn, not a step of the method).
  *

@@ -58,6 +58,8 @@ def lib() -> C.CDLL:
                      "spice_grouped_expert_ffn_static", "spice_draft_confidence", "spice_prefetch_rollout"):
             getattr(L, name).restype = C.c_int
         L.spice_static_scratch_bytes.restype = C.c_size_t
+        L.spice_lore_calibrate.restype = C.c_int
+        L.spice_lore_calibrate_workspace_bytes.restype = C.c_size_t
         _lib = L
     return _lib
 
@@ -139,6 +141,26 @@ def spice_prefetch_rollout(ctx, weights, x_current, T, l_min, l_max, tau, idx_ha
                                         C.c_int32(l_max), C.c_float(tau), _ptr(idx_hat, torch.int32),
                                         _ptr(conf, torch.float32), _ptr(depth, torch.int32), _ptr(h_final, torch.bfloat16),
                                         _stream(stream)), "spice_prefetch_rollout")
+
+
+def spice_lore_calibrate(h_cal, resid, rank, ridge=0.0, iterations=100, stream=None):
+    """Fit the LoRE factors of one expert on the device.  h_cal [n,d] bf16, resid [n,d] fp32 (device tensors).
+    Returns (A [rank,d] bf16, B [d,rank] bf16, loss tensor [2] = (objective, sum resid^2), status tensor [1])."""
+    n, d = h_cal.shape
+    dev = h_cal.device
+    nbytes = int(lib().spice_lore_calibrate_workspace_bytes(C.c_int32(d), C.c_int32(n), C.c_int32(rank)))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    A = torch.empty(rank, d, dtype=torch.bfloat16, device=dev)
+    Bm = torch.empty(d, rank, dtype=torch.bfloat16, device=dev)
+    loss = torch.empty(2, dtype=torch.float32, device=dev)
+    status = torch.empty(1, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib().spice_lore_calibrate(C.c_int32(d), C.c_int32(n), C.c_int32(rank), C.c_float(ridge), C.c_int32(iterations),
+                                          _ptr(h_cal, torch.bfloat16), _ptr(resid, torch.float32), _ptr(A, torch.bfloat16),
+                                          _ptr(Bm, torch.bfloat16), _ptr(loss, torch.float32), _ptr(status, torch.int32),
+                                          C.c_void_p(ws.data_ptr()), C.c_size_t(nbytes), _stream(stream)),
+               "spice_lore_calibrate")
+    return A, Bm, loss, status
 
 
 def spice_classify_misses(ctx, idx, gate, slot_of_expert, conf, T, cls, slot, counts, resid_tok=None, resid_k=None,

@@ -377,6 +377,25 @@ spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w
     return SPICE_OK;
 }
 
+size_t spice_lore_calibrate_workspace_bytes(int32_t d, int32_t n_tokens, int32_t rank) {
+    if (d < 1 || n_tokens < 1 || rank < 1) return 0;
+    return lore_calibrate_workspace_bytes(d, n_tokens, rank);
+}
+
+spice_status spice_lore_calibrate(int32_t d, int32_t n_tokens, int32_t rank, float ridge, int32_t iterations,
+                                  const spice_bf16 *h_cal, const float *resid, spice_bf16 *A_out, spice_bf16 *B_out,
+                                  float *loss_out, int32_t *device_status, void *workspace, size_t workspace_bytes,
+                                  void *stream) {
+    if (d < 8 || d % 8 || rank < 1 || 2 * rank > d || n_tokens < 1 || iterations < 0 || iterations > 1000 || !(ridge >= 0.f))
+        return SPICE_ERR_INVALID_ARG;
+    if (!h_cal || !resid || !A_out || !B_out || !device_status || !workspace) return SPICE_ERR_INVALID_ARG;
+    if (workspace_bytes < lore_calibrate_workspace_bytes(d, n_tokens, rank)) return SPICE_ERR_WORKSPACE;
+    int n = launch_lore_calibrate(d, n_tokens, rank, ridge, iterations, reinterpret_cast<const __nv_bfloat16 *>(h_cal), resid,
+                                  reinterpret_cast<__nv_bfloat16 *>(A_out), reinterpret_cast<__nv_bfloat16 *>(B_out), loss_out,
+                                  device_status, workspace, static_cast<cudaStream_t>(stream));
+    return n < 0 ? SPICE_ERR_CUDA : SPICE_OK;
+}
+
 spice_status spice_classify_misses(spice_ctx *ctx, const int32_t *idx, const float *gate,
                                    const int32_t *slot_of_expert, const float *conf, int32_t T, uint8_t *cls,
                                    int32_t *slot, int32_t *counts, int32_t *resid_tok, int32_t *resid_k,

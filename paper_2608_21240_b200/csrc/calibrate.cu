@@ -1,0 +1,407 @@
+// LoRE calibration of one (layer, expert) pair (Sec. 4.2 of the paper): fit the rank-r residual module
+//     Delta(h) = B A h,   A: r x d,  B: d x r,
+// that minimises  sum_{h in D} || E(h) - S(h) - B A h ||_2^2  over the calibration tokens routed to the expert.
+// The paper says the parameters are "trained by minimizing" this objective; the objective is a reduced-rank
+// regression and has a closed-form minimiser, which is what is computed here (in fp32, offline path):
+//     G = H^T H (+ ridge),  C = H^T R          H [n,d] hidden states, R [n,d] targets E(h) - S(h)
+//     G = L L^T,  Z = L^-1 C                   (then the fitted values satisfy  Yhat^T Yhat = Z^T Z)
+//     V = r leading eigenvectors of Z^T Z      block subspace iteration, orthonormalised by Cholesky QR (twice)
+//     B = V,   A = ( L^-T Z V )^T = ( W V )^T  with W = G^-1 C the least-squares map
+// Everything is dense fp32 linear algebra on d x d matrices built from tiled SGEMMs, 64 x 64 Cholesky /
+// triangular-solve blocks and a few element-wise kernels, launched in order on one stream; nothing synchronises
+// with the host.  The caller provides the workspace (spice_lore_calibrate_workspace_bytes).
+#include "spice_internal.cuh"
+
+namespace spice {
+
+namespace {
+
+constexpr int TB = 64;    // block size of the factorisations and tile of the SGEMM
+constexpr int BK = 16;
+
+__host__ __device__ inline int pad64(int v) { return (v + 63) / 64 * 64; }
+
+// C[M,N] = alpha * op(A) * op(B) + beta * C, row-major.  TA: A is stored [K,M] (lda); TB_: B is stored [N,K] (ldb).
+template <bool TA, bool TB_>
+__global__ void __launch_bounds__(256) sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int lda,
+                                                    const float *__restrict__ B, int ldb, float beta, float *__restrict__ C,
+                                                    int ldc) {
+    __shared__ float As[BK][TB + 4], Bs[BK][TB + 4];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int m0 = blockIdx.y * TB, n0 = blockIdx.x * TB;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        for (int e = threadIdx.x; e < BK * TB; e += 256) {
+            int kk, mm;
+            if (TA) { kk = e / TB; mm = e % TB; } else { mm = e / BK; kk = e % BK; }
+            const int gm = m0 + mm, gk = k0 + kk;
+            As[kk][mm] = (gm < M && gk < K) ? (TA ? A[(size_t)gk * lda + gm] : A[(size_t)gm * lda + gk]) : 0.f;
+            int kb, nn;
+            if (TB_) { nn = e / BK; kb = e % BK; } else { kb = e / TB; nn = e % TB; }
+            const int gn = n0 + nn, gkb = k0 + kb;
+            Bs[kb][nn] = (gn < N && gkb < K) ? (TB_ ? B[(size_t)gn * ldb + gkb] : B[(size_t)gkb * ldb + gn]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int gm = m0 + ty * 4 + i, gn = n0 + tx * 4 + j;
+            if (gm < M && gn < N) {
+                float *c = C + (size_t)gm * ldc + gn;
+                *c = alpha * acc[i][j] + (beta != 0.f ? beta * *c : 0.f);
+            }
+        }
+}
+
+template <bool TA, bool TB_>
+int gemm(int M, int N, int K, float alpha, const float *A, int lda, const float *B, int ldb, float beta, float *C, int ldc,
+         cudaStream_t st) {
+    if (M <= 0 || N <= 0) return 0;
+    dim3 grid((N + TB - 1) / TB, (M + TB - 1) / TB);
+    sgemm_kernel<TA, TB_><<<grid, 256, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+// bf16 [rows, cols] -> fp32 [rows, ld] with zero columns cols..ld-1
+__global__ void widen_pad_kernel(const __nv_bfloat16 *__restrict__ src, int rows, int cols, float *__restrict__ dst, int ld) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)rows * ld) return;
+    const int r = (int)(i / ld), c = (int)(i % ld);
+    dst[i] = c < cols ? __bfloat162float(src[(size_t)r * cols + c]) : 0.f;
+}
+
+// scal[0] = trace of the leading d x d block / d
+__global__ void mean_diag_kernel(const float *__restrict__ G, int ld, int d, float *scal) {
+    __shared__ float red[256];
+    float s = 0.f;
+    for (int i = threadIdx.x; i < d; i += 256) s += G[(size_t)i * ld + i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) scal[0] = red[0] / (float)d;
+}
+
+// diagonal: G[i,i] += ridge * scal[0] for i < d; padding rows / columns i >= d become the identity
+__global__ void regularise_kernel(float *G, int ld, int d, int dp, float ridge, const float *scal) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)dp * dp) return;
+    const int r = (int)(i / dp), c = (int)(i % dp);
+    float *g = G + (size_t)r * ld + c;
+    if (r >= d || c >= d) *g = (r == c) ? 1.f : 0.f;
+    else if (r == c) *g += ridge * scal[0];
+}
+
+// Cholesky of one 64 x 64 diagonal block in place (lower triangle; the strict upper triangle is zeroed).
+// A pivot that is not positive is replaced by a tiny positive number and flagged.
+__global__ void __launch_bounds__(64) potrf64_kernel(float *A, int ld, int32_t *flag) {
+    __shared__ float a[TB][TB + 1];
+    const int t = threadIdx.x;
+    for (int r = 0; r < TB; ++r) a[r][t] = A[(size_t)r * ld + t];
+    __syncthreads();
+    for (int j = 0; j < TB; ++j) {
+        if (t == j) {
+            float p = a[j][j];
+            if (!(p > 0.f)) {
+                p = 1e-20f;
+                atomicOr(flag, 1);
+            }
+            a[j][j] = sqrtf(p);
+        }
+        __syncthreads();
+        const float piv = a[j][j];
+        if (t > j) a[t][j] /= piv;
+        __syncthreads();
+        // trailing update: row t, columns j+1 .. t
+        if (t > j) {
+            const float ltj = a[t][j];
+            for (int c = j + 1; c <= t; ++c) a[t][c] -= ltj * a[c][j];
+        }
+        __syncthreads();
+    }
+    for (int r = 0; r < TB; ++r) A[(size_t)r * ld + t] = t <= r ? a[r][t] : 0.f;
+}
+
+// X <- X L^-T for a panel of rows (one CTA of 64 threads takes 64 rows): X [rows, 64] (ldx), L 64 x 64 lower (ldl)
+__global__ void __launch_bounds__(64) trsm_right_lt_kernel(float *X, int ldx, int rows, const float *__restrict__ L, int ldl) {
+    __shared__ float l[TB][TB + 1];
+    const int t = threadIdx.x;
+    for (int r = 0; r < TB; ++r) l[r][t] = L[(size_t)r * ldl + t];
+    __syncthreads();
+    const int row = blockIdx.x * TB + t;
+    if (row >= rows) return;
+    float x[TB];
+#pragma unroll
+    for (int c = 0; c < TB; ++c) x[c] = X[(size_t)row * ldx + c];
+    // solve y L^T = x: y_c = (x_c - sum_{q<c} y_q L[c][q]) / L[c][c]
+#pragma unroll 1
+    for (int c = 0; c < TB; ++c) {
+        float s = x[c];
+        for (int qq = 0; qq < c; ++qq) s -= x[qq] * l[c][qq];
+        x[c] = s / l[c][c];
+    }
+#pragma unroll
+    for (int c = 0; c < TB; ++c) X[(size_t)row * ldx + c] = x[c];
+}
+
+// X <- L^-1 X (TRANS = false) or L^-T X (TRANS = true) for a block row X [64, cols] (ldx); one thread per column
+template <bool TRANS>
+__global__ void __launch_bounds__(64) trsm_left_kernel(float *X, int ldx, int cols, const float *__restrict__ L, int ldl) {
+    __shared__ float l[TB][TB + 1];
+    const int t = threadIdx.x;
+    for (int r = 0; r < TB; ++r) l[r][t] = L[(size_t)r * ldl + t];
+    __syncthreads();
+    const int col = blockIdx.x * TB + t;
+    if (col >= cols) return;
+    float x[TB];
+#pragma unroll
+    for (int r = 0; r < TB; ++r) x[r] = X[(size_t)r * ldx + col];
+    if (!TRANS) {
+#pragma unroll 1
+        for (int r = 0; r < TB; ++r) {
+            float s = x[r];
+            for (int qq = 0; qq < r; ++qq) s -= l[r][qq] * x[qq];
+            x[r] = s / l[r][r];
+        }
+    } else {
+#pragma unroll 1
+        for (int r = TB - 1; r >= 0; --r) {
+            float s = x[r];
+            for (int qq = r + 1; qq < TB; ++qq) s -= l[qq][r] * x[qq];
+            x[r] = s / l[r][r];
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < TB; ++r) X[(size_t)r * ldx + col] = x[r];
+}
+
+// deterministic start block for the subspace iteration: a hash of (row, column) mapped to (-1, 1)
+__global__ void init_block_kernel(float *Q, int rows, int ld, int cols) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)rows * ld) return;
+    const int r = (int)(i / ld), c = (int)(i % ld);
+    uint32_t h = (uint32_t)r * 2654435761u ^ ((uint32_t)c + 0x9e3779b9u) * 2246822519u;
+    h ^= h >> 15; h *= 2246822519u; h ^= h >> 13; h *= 3266489917u; h ^= h >> 16;
+    Q[i] = c < cols ? ((float)(h >> 8) * (1.0f / 8388608.0f) - 1.0f) : 0.f;
+}
+
+// S (rp x rp): padding rows / columns >= r become the identity.  In the first pass of the Cholesky QR a small multiple of
+// the largest diagonal entry is added to the diagonal: the columns of a power-iterated block can be dependent to working
+// precision, and the factorisation must not break down on directions that carry no weight (the second pass restores
+// orthonormality of what is left).
+__global__ void fix_gram_kernel(float *S, int rp, int r, float jitter) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rp * rp) return;
+    const int a = i / rp, b = i % rp;
+    if (a >= r || b >= r) {
+        S[i] = (a == b) ? 1.f : 0.f;
+    } else if (a == b && jitter > 0.f) {
+        float mx = 0.f;
+        for (int q = 0; q < r; ++q) mx = fmaxf(mx, S[q * rp + q]);   // (reads diagonal entries other threads may be updating:
+        S[i] += jitter * mx;                                          //  the bound only has to be of the right magnitude)
+    }
+}
+
+__global__ void write_factors_kernel(const float *__restrict__ V, const float *__restrict__ X, int ld, int d, int r,
+                                     __nv_bfloat16 *__restrict__ A, __nv_bfloat16 *__restrict__ B) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)d * r) return;
+    const int j = (int)(i / r), qq = (int)(i % r);
+    B[(size_t)j * r + qq] = __float2bfloat16(V[(size_t)j * ld + qq]);      // B [d, r]
+    A[(size_t)qq * d + j] = __float2bfloat16(X[(size_t)j * ld + qq]);      // A [r, d] = X^T
+}
+
+// out[0] += sum (R - T)^2, out[1] += sum R^2 over a slice
+__global__ void __launch_bounds__(256) loss_kernel(const float *__restrict__ R, int ldr, const float *__restrict__ T, int ldt, int n,
+                                                   int d, float *out) {
+    __shared__ float r0[256], r1[256];
+    float a = 0.f, b = 0.f;
+    const size_t total = (size_t)n * d;
+    for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < total; i += (size_t)gridDim.x * 256) {
+        const int row = (int)(i / d), c = (int)(i % d);
+        const float rv = R[(size_t)row * ldr + c], dv = rv - T[(size_t)row * ldt + c];
+        a += dv * dv;
+        b += rv * rv;
+    }
+    r0[threadIdx.x] = a;
+    r1[threadIdx.x] = b;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) {
+            r0[threadIdx.x] += r0[threadIdx.x + o];
+            r1[threadIdx.x] += r1[threadIdx.x + o];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        atomicAdd(out, r0[0]);
+        atomicAdd(out + 1, r1[0]);
+    }
+}
+
+__global__ void widen_kernel(const __nv_bfloat16 *__restrict__ src, size_t n, float *__restrict__ dst) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = __bfloat162float(src[i]);
+}
+
+#define CK(expr)                 \
+    do {                         \
+        int k_ = (expr);         \
+        if (k_ < 0) return -1;   \
+        launches += k_;          \
+    } while (0)
+#define CKL()                                             \
+    do {                                                  \
+        if (cudaGetLastError() != cudaSuccess) return -1; \
+        ++launches;                                       \
+    } while (0)
+
+// in-place blocked Cholesky of the leading np x np block (np a multiple of 64), lower triangle
+int cholesky(float *G, int ld, int np, int32_t *flag, cudaStream_t st) {
+    int launches = 0;
+    for (int k = 0; k < np; k += TB) {
+        float *diag = G + (size_t)k * ld + k;
+        potrf64_kernel<<<1, 64, 0, st>>>(diag, ld, flag);
+        CKL();
+        const int rem = np - k - TB;
+        if (rem > 0) {
+            float *panel = G + (size_t)(k + TB) * ld + k;
+            trsm_right_lt_kernel<<<rem / TB, 64, 0, st>>>(panel, ld, rem, diag, ld);
+            CKL();
+            CK((gemm<false, true>(rem, rem, TB, -1.f, panel, ld, panel, ld, 1.f, G + (size_t)(k + TB) * ld + (k + TB), ld, st)));
+        }
+    }
+    return launches;
+}
+
+// Y [np, cols] <- Y L^-T with L np x np lower (np a multiple of 64): column blocks left to right
+int solve_right_lt(float *Y, int ldy, int rows, const float *L, int ldl, int np, cudaStream_t st) {
+    int launches = 0;
+    for (int j = 0; j < np; j += TB) {
+        if (j > 0)   // Y_j -= Y_{<j} L[j, <j]^T
+            CK((gemm<false, true>(rows, TB, j, -1.f, Y, ldy, L + (size_t)j * ldl, ldl, 1.f, Y + j, ldy, st)));
+        trsm_right_lt_kernel<<<(rows + TB - 1) / TB, 64, 0, st>>>(Y + j, ldy, rows, L + (size_t)j * ldl + j, ldl);
+        CKL();
+    }
+    return launches;
+}
+
+// Q [dp, rp] <- orthonormal basis of its columns by Cholesky QR, twice
+int orthonormalise(float *Q, int dp, int rp, int r, float *S, int32_t *flag, cudaStream_t st) {
+    int launches = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+        CK((gemm<true, false>(rp, rp, dp, 1.f, Q, rp, Q, rp, 0.f, S, rp, st)));
+        fix_gram_kernel<<<(rp * rp + 255) / 256, 256, 0, st>>>(S, rp, r, pass == 0 ? 1e-6f : 0.f);
+        CKL();
+        CK(cholesky(S, rp, rp, flag, st));
+        CK(solve_right_lt(Q, rp, dp, S, rp, rp, st));
+    }
+    return launches;
+}
+
+}  // namespace
+
+size_t lore_calibrate_workspace_bytes(int d, int n, int r) {
+    const size_t dp = pad64(d), rp = pad64(r);
+    // H32 / T2 [n, dp], G [dp, dp], C [dp, dp], Q, P, Y [dp, rp] each, S [rp, rp], T1 [n, rp], A32 [rp, dp], B32 [dp, rp], scalars
+    size_t f = (size_t)n * dp + 2 * dp * dp + 3 * dp * rp + rp * rp + (size_t)n * rp + 2 * dp * rp + 64;
+    return f * sizeof(float) + 256;
+}
+
+int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __nv_bfloat16 *h_cal, const float *resid,
+                          __nv_bfloat16 *A_out, __nv_bfloat16 *B_out, float *loss_out, int32_t *flag, void *workspace,
+                          cudaStream_t st) {
+    int launches = 0;
+    const int dp = pad64(d), rp = pad64(r);
+    float *w = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(workspace) + 255) & ~uintptr_t(255));
+    float *H32 = w;                      w += (size_t)n * dp;
+    float *G = w;                        w += (size_t)dp * dp;
+    float *C = w;                        w += (size_t)dp * dp;
+    float *Q = w;                        w += (size_t)dp * rp;
+    float *P = w;                        w += (size_t)dp * rp;
+    float *Y = w;                        w += (size_t)dp * rp;
+    float *S = w;                        w += (size_t)rp * rp;
+    float *T1 = w;                       w += (size_t)n * rp;
+    float *A32 = w;                      w += (size_t)rp * dp;
+    float *B32 = w;                      w += (size_t)dp * rp;
+    float *scal = w;
+    int32_t *qr_flag = reinterpret_cast<int32_t *>(scal + 8);   // pivots clamped inside the Cholesky QR are not an error
+    if (cudaMemsetAsync(flag, 0, sizeof(int32_t), st) != cudaSuccess) return -1;
+    widen_pad_kernel<<<(unsigned)(((size_t)n * dp + 255) / 256), 256, 0, st>>>(h_cal, n, d, H32, dp);
+    CKL();
+    // G = H^T H, C = H^T R (columns >= d of C stay zero)
+    CK((gemm<true, false>(dp, dp, n, 1.f, H32, dp, H32, dp, 0.f, G, dp, st)));
+    if (cudaMemsetAsync(C, 0, sizeof(float) * (size_t)dp * dp, st) != cudaSuccess) return -1;
+    CK((gemm<true, false>(dp, d, n, 1.f, H32, dp, resid, d, 0.f, C, dp, st)));
+    mean_diag_kernel<<<1, 256, 0, st>>>(G, dp, d, scal);
+    CKL();
+    regularise_kernel<<<(unsigned)(((size_t)dp * dp + 255) / 256), 256, 0, st>>>(G, dp, d, dp, ridge, scal);
+    CKL();
+    CK(cholesky(G, dp, dp, flag, st));
+    // Z = L^-1 C, block rows top to bottom (in place in C)
+    for (int k = 0; k < dp; k += TB) {
+        trsm_left_kernel<false><<<dp / TB, 64, 0, st>>>(C + (size_t)k * dp, dp, dp, G + (size_t)k * dp + k, dp);
+        CKL();
+        const int rem = dp - k - TB;
+        if (rem > 0)
+            CK((gemm<false, false>(rem, dp, TB, -1.f, G + (size_t)(k + TB) * dp + k, dp, C + (size_t)k * dp, dp, 1.f,
+                                   C + (size_t)(k + TB) * dp, dp, st)));
+    }
+    float *Z = C;
+    // r leading eigenvectors of Z^T Z by block subspace iteration
+    init_block_kernel<<<(unsigned)(((size_t)dp * rp + 255) / 256), 256, 0, st>>>(Q, dp, rp, r);
+    CKL();
+    CK(orthonormalise(Q, dp, rp, r, S, qr_flag, st));
+    for (int it = 0; it < iters; ++it) {
+        CK((gemm<false, false>(dp, rp, dp, 1.f, Z, dp, Q, rp, 0.f, P, rp, st)));     // P = Z Q
+        CK((gemm<true, false>(dp, rp, dp, 1.f, Z, dp, P, rp, 0.f, Y, rp, st)));      // Y = Z^T P
+        if (cudaMemcpyAsync(Q, Y, sizeof(float) * (size_t)dp * rp, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return -1;
+        CK(orthonormalise(Q, dp, rp, r, S, qr_flag, st));
+    }
+    // B = V = Q;  A^T = W V = L^-T (Z V): block rows bottom to top (in place in P)
+    CK((gemm<false, false>(dp, rp, dp, 1.f, Z, dp, Q, rp, 0.f, P, rp, st)));
+    for (int k = dp - TB; k >= 0; k -= TB) {
+        trsm_left_kernel<true><<<rp / TB, 64, 0, st>>>(P + (size_t)k * rp, rp, rp, G + (size_t)k * dp + k, dp);
+        CKL();
+        if (k > 0)   // P_{<k} -= L[k, <k]^T P_k
+            CK((gemm<true, false>(k, rp, TB, -1.f, G + (size_t)k * dp, dp, P + (size_t)k * rp, rp, 1.f, P, rp, st)));
+    }
+    write_factors_kernel<<<(unsigned)(((size_t)d * r + 255) / 256), 256, 0, st>>>(Q, P, rp, d, r, A_out, B_out);
+    CKL();
+    if (loss_out) {
+        // objective at the bf16 factors that were written: T2 = (H A^T) B^T, loss = sum (R - T2)^2
+        widen_kernel<<<(unsigned)(((size_t)r * d + 255) / 256), 256, 0, st>>>(A_out, (size_t)r * d, A32);
+        CKL();
+        widen_kernel<<<(unsigned)(((size_t)d * r + 255) / 256), 256, 0, st>>>(B_out, (size_t)d * r, B32);
+        CKL();
+        CK((gemm<false, true>(n, r, d, 1.f, H32, dp, A32, d, 0.f, T1, rp, st)));      // T1 = H A^T  [n, r]
+        CK((gemm<false, true>(n, d, r, 1.f, T1, rp, B32, r, 0.f, H32, dp, st)));      // T2 = T1 B^T [n, d], over H32 (no longer needed)
+        if (cudaMemsetAsync(loss_out, 0, 2 * sizeof(float), st) != cudaSuccess) return -1;
+        loss_kernel<<<512, 256, 0, st>>>(resid, d, H32, dp, n, d, loss_out);
+        CKL();
+    }
+    return launches;
+}
+
+}  // namespace spice

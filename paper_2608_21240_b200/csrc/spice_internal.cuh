@@ -89,6 +89,12 @@ int launch_rollout_mask(const Dims &dm, int depth, int l_min, int l_max, float t
                         const int32_t *idx_ws, int32_t *idx_out, float *conf_out, uint8_t *cls, int32_t *depth_out,
                         cudaStream_t st);
 
+// ---- LoRE calibration (calibrate.cu): closed-form rank-r fit of the residual E(h) - S(h) over calibration tokens
+size_t lore_calibrate_workspace_bytes(int d, int n, int r);
+int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __nv_bfloat16 *h_cal, const float *resid,
+                          __nv_bfloat16 *A_out, __nv_bfloat16 *B_out, float *loss_out, int32_t *flag, void *workspace,
+                          cudaStream_t st);
+
 // ---- fused decode kernel (decode.cu)
 // words of the dependency-counter array
 enum { SY_ABORT = 0, SY_TEAMS_DONE, SY_R1_DONE, SY_ROUTE_DONE, SY_P2_DONE, SY_P1_ALL, SY_NEXT_TASK, SY_GROUP0 = 8 };
