@@ -17,6 +17,7 @@ struct spice_ctx {
     float *ws_gate;
     uint8_t *ws_cls;
     float *y32;        // [Tm, d] fp32 accumulator of the fused call
+    GroupScratch gsc;               // scratch of the multi-CTA classify / group kernels
     float *draft_logits;            // [Tm, N] logits of spice_draft_confidence when the caller does not want pi_hat
     // speculative prefetch rollout
     __nv_bfloat16 *roll_h, *roll_y; // [Tm, d] draft state and scratch output
@@ -80,6 +81,9 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->ws_gate = cv.take<float>(n);
     c->ws_cls = cv.take<uint8_t>(n);
     c->y32 = cv.take<float>(Tm * g.d);
+    c->gsc.cnt = cv.take<int32_t>(4096);
+    c->gsc.off = cv.take<int32_t>(2048);
+    c->gsc.blk_miss = cv.take<int32_t>(n / 1024 + 2);
     c->draft_logits = cv.take<float>(Tm * g.n_experts);
     c->roll_h = cv.take<__nv_bfloat16>(Tm * g.d);
     c->roll_y = cv.take<__nv_bfloat16>(Tm * g.d);
@@ -410,7 +414,7 @@ spice_status spice_classify_misses(spice_ctx *ctx, const int32_t *idx, const flo
     if (!idx || !gate || !slot_of_expert || !conf || !cls || !slot || !counts) return SPICE_ERR_INVALID_ARG;
     if (!(resid_tok && resid_k && resid_expert && resid_gate)) resid_tok = resid_k = resid_expert = nullptr, resid_gate = nullptr;
     SPICE_LAUNCH(launch_classify(dims_of(ctx, T), ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, slot_of_expert, conf,
-                                 cls, slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
+                                 cls, slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st, &ctx->gsc));
     return SPICE_OK;
 }
 
@@ -425,7 +429,7 @@ spice_status spice_grouped_expert_ffn(spice_ctx *ctx, const spice_layer_weights 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Dims dm = dims_of(ctx, T);
     const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
-    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, slot, ctx->tb, st));
+    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, slot, ctx->tb, st, &ctx->gsc));
     SPICE_LAUNCH(launch_gateup(dm, KIND_HIT, *w, hb, ctx->tb, st));
     SPICE_LAUNCH(launch_down(dm, KIND_HIT, *w, ctx->tb, st));
     CombineArgs ca{KIND_HIT, 1, gate, cls, y, nullptr, nullptr, nullptr};
@@ -445,7 +449,7 @@ spice_status spice_lore_surrogate(spice_ctx *ctx, const spice_layer_weights *w, 
     const Dims dm = dims_of(ctx, T);
     const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
     // no slot array: HIT entries are left out of the grouping
-    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, nullptr, ctx->tb, st));
+    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, nullptr, ctx->tb, st, &ctx->gsc));
     SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED, *w, hb, ctx->tb, st));
     SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
     SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_LOW, *w, ctx->tb, st));
@@ -506,8 +510,8 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     SPICE_LAUNCH(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
                                    gate, nullptr, st));
     SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
-                                 ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st));
-    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st));
+                                 ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st, &ctx->gsc));
+    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st, &ctx->gsc));
     if (ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm)) {
         // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
         // LoRE on the general kernels

@@ -52,13 +52,20 @@ int launch_route_topk(const Dims &dm, int norm_topk, const __nv_bfloat16 *h, con
 int launch_draft_confidence(const Dims &dm, const __nv_bfloat16 *h_hat, const __nv_bfloat16 *w_draft, int32_t *idx_hat,
                             float *gate_ws, float *logits_ws, float *pi_hat, float *conf, cudaStream_t st);
 
+// scratch of the multi-CTA classify / group kernels (large batches); without it the single-CTA kernels run
+struct GroupScratch {
+    int32_t *cnt;        // [4096]: entries per slot [0,1024) and per expert [1024,2048), then the cursors [2048,4096)
+    int32_t *off;        // [2048]: first position of each slot's / expert's group
+    int32_t *blk_miss;   // [ceil(Tm*K / 1024)]: exact-recovery misses per chunk of 1024 entries
+};
+
 int launch_classify(const Dims &dm, int conf_stride, float tau, const int32_t *idx, const float *gate,
                     const int32_t *slot_of_expert, const float *conf, uint8_t *cls, int32_t *slot,
                     int32_t *counts, int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
-                    float *resid_gate, int32_t *status, cudaStream_t st);
+                    float *resid_gate, int32_t *status, cudaStream_t st, const GroupScratch *scratch = nullptr);
 
 int launch_group(const Dims &dm, const int32_t *idx, const float *gate, const uint8_t *cls,
-                 const int32_t *slot, const Tables &tb, cudaStream_t st);
+                 const int32_t *slot, const Tables &tb, cudaStream_t st, const GroupScratch *scratch = nullptr);
 
 // Reference ("v1") expert path: warp-per-row GEMV kernels for any shape.
 int launch_gateup(const Dims &dm, int kind_mask, const spice_layer_weights &w, const __nv_bfloat16 *h,

@@ -497,6 +497,36 @@ def test_config4_prefill_4096_tokens_skewed_loads_sampled_against_oracle():
     L.close()
 
 
+def test_large_batch_with_misses_multi_cta_tables_sampled_against_oracle():
+    """3000 tokens of the small layer with 5 of 8 experts resident: 6000 (token, expert) entries take the multi-CTA
+    classification / grouping kernels, and every class occurs.  Routing, classes, counts and the ORDERED residual-miss list
+    are compared for all tokens (also through the split exports), outputs for a sample."""
+    wl = _layer_case("tiny", 3000, variant=13)
+    s = wl.shape
+    tokens = sorted(np.random.default_rng(5).choice(3000, size=40, replace=False).tolist())
+    ref = run_oracle(wl, tokens=tokens, want_full=False)
+    assert min(ref.counts.tolist()) > 200
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    w = upload(wl)
+    h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+    out = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    check_routing(out, ref, wl.T, s.top_k)
+    err, bound = y_close(out.y.float().cpu().numpy()[np.asarray(tokens)], ref.y)
+    assert err <= bound, (err, bound)
+    idx, gate = L.route_topk(h, w.w_router)
+    cls, slot, counts, resid = L.classify_misses(idx, gate, w.slot_of_expert, conf)
+    assert torch.equal(cls, out.cls) and torch.equal(counts, out.counts)
+    n_miss = int(counts[1].item())
+    assert torch.equal(resid[0][:n_miss], out.resid_tok[:n_miss]) and torch.equal(resid[2][:n_miss], out.resid_expert[:n_miss])
+    # the general kernels on the tables the multi-CTA grouping built
+    L.set_option(B.OPT_PATH, 1)
+    gen = L.moe_layer_fwd(w, h, conf)
+    assert (gen.y.float() - out.y.float()).abs().max().item() <= 2e-2 * out.y.float().abs().max().item() + 2e-3
+    assert L.device_status() == 0
+    L.close()
+
+
 def test_config5_decode_stack_teacher_forced_per_layer():
     """26 layers of DeepSeek-V2-Lite shape, batch 8, slot cache of 26 experts with ~70 % hits.  Each GPU layer
     call gets the oracle chain's input for that layer (bf16-level output error must not be allowed to flip later
