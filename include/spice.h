@@ -15,7 +15,8 @@
  *   - bf16 tensors are passed as spice_bf16* (raw 16-bit patterns), row-major, 16-byte aligned,
  *     weights in [out, in] order.  Expert FFNs are SwiGLU: E(x) = W_d ( silu(W_g x) * (W_u x) ).
  *   - All calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default stream)
- *     and return without synchronising.  The library allocates device memory only in
+ *     and return without synchronising (spice_moe_layer_fwd can therefore be captured into a CUDA
+ *     graph; pointers are baked in at capture time).  The library allocates device memory only in
  *     spice_create; per call it allocates nothing.  A ctx must not be used by two streams at once.
  *   - Errors found on the host return a code and launch nothing.  Conditions found on the device
  *     (expert id out of range, slot index >= n_slots, an expired bounded wait) never trap: the
