@@ -167,11 +167,18 @@ spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, con
  *   idx_hat [l_max,T,K] int32 out: predicted sets, -1 past a token's last depth.  conf [l_max,T] fp32 out, 0 there.
  *   depth [T] int32 out: number of predictions enqueued for the token (>= min(l_min, l_max)).
  *   h_final [T,d] bf16 out, optional: the draft state after the last projection made for each token.
- * The prefetch queue of Algorithm 1 is the union over l of idx_hat[l-1, t, :] for l <= depth[t]; issuing the copies is the
- * host runtime's job.  The call launches about 8 kernels per depth and is bound by their launch latency at decode batches. */
+ *   prefetch_mask [l_max, N] uint8 out, optional: the prefetch intents of Eq. 3 for the batch, kept per depth because
+ *       depth l names experts of the layer l ahead: prefetch_mask[l-1, e] = 1 iff some token enqueues expert e at depth l.
+ * Issuing the copies is the host runtime's job.  The call launches about 8 kernels per depth and is bound by their launch latency at decode batches. */
 spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w /* host array */,
                                     const spice_bf16 *x_current, int32_t T, int32_t l_min, int32_t l_max, float tau,
-                                    int32_t *idx_hat, float *conf, int32_t *depth, spice_bf16 *h_final, void *stream);
+                                    int32_t *idx_hat, float *conf, int32_t *depth, spice_bf16 *h_final,
+                                    uint8_t *prefetch_mask, void *stream);
+
+/* Eq. 4 (host arithmetic, no device work): H_min = ceil(P * M_e / (B_PCIe * T_comp)), the lookahead depth needed to hide the
+ * transfer of n_prefetch experts of expert_bytes each per layer behind t_comp_s seconds of compute per layer over a link of
+ * pcie_bytes_per_s.  Returns -1 on a non-positive bandwidth or compute window. */
+int32_t spice_min_lookahead_depth(int32_t n_prefetch, double expert_bytes, double pcie_bytes_per_s, double t_comp_s);
 
 /* LoRE calibration of one (layer, expert) pair (Sec. 4.2): the rank-r residual module Delta(h) = B A h that minimises
  *     sum over the calibration tokens h routed to the expert of  || E(h) - S(h) - B A h ||_2^2 .

@@ -184,6 +184,25 @@ def prefetch_rollout(x, layers, top_k: int, l_min: int, l_max: int, tau: float):
     return idx_hat, conf, depth, h
 
 
+def prefetch_set(idx_hat, n_experts: int) -> np.ndarray:
+    """Eq. 3: the prefetch intents are the union of the predicted sets.  Experts of different depths belong to different
+    layers, so the union over the batch is kept per depth: mask[l-1, e] = 1 iff some token predicts expert e at depth l."""
+    idx_hat = np.asarray(idx_hat)
+    L = idx_hat.shape[0]
+    mask = np.zeros((L, n_experts), dtype=np.uint8)
+    for l in range(L):
+        for e in idx_hat[l].ravel():
+            if e >= 0:
+                mask[l, int(e)] = 1
+    return mask
+
+
+def min_lookahead_depth(n_prefetch: int, expert_bytes: float, pcie_bytes_per_s: float, t_comp_s: float) -> int:
+    """Eq. 4: H_min = ceil(P * M_e / (B_PCIe * T_comp)), the depth needed to hide P expert transfers per layer."""
+    import math
+    return int(math.ceil(n_prefetch * expert_bytes / (pcie_bytes_per_s * t_comp_s)))
+
+
 def classify(idx, resident, conf, tau: float, conf_stride: Optional[int] = None):
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     T, K = idx.shape

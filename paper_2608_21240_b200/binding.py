@@ -133,14 +133,20 @@ def spice_draft_confidence(ctx, h_hat, w_draft_router, T, idx_hat, conf, pi_hat=
                                         _stream(stream)), "spice_draft_confidence")
 
 
+def spice_min_lookahead_depth(n_prefetch, expert_bytes, pcie_bytes_per_s, t_comp_s) -> int:
+    f = lib().spice_min_lookahead_depth
+    f.restype = C.c_int32
+    return int(f(C.c_int32(n_prefetch), C.c_double(expert_bytes), C.c_double(pcie_bytes_per_s), C.c_double(t_comp_s)))
+
+
 def spice_prefetch_rollout(ctx, weights, x_current, T, l_min, l_max, tau, idx_hat, conf, depth, h_final=None,
-                           stream=None) -> None:
+                           prefetch_mask=None, stream=None) -> None:
     """weights: sequence of l_max LayerWeightsC structs (depth 1 first)."""
     arr = (LayerWeightsC * l_max)(*weights)
     _check(lib().spice_prefetch_rollout(ctx, arr, _ptr(x_current, torch.bfloat16), C.c_int32(T), C.c_int32(l_min),
                                         C.c_int32(l_max), C.c_float(tau), _ptr(idx_hat, torch.int32),
                                         _ptr(conf, torch.float32), _ptr(depth, torch.int32), _ptr(h_final, torch.bfloat16),
-                                        _stream(stream)), "spice_prefetch_rollout")
+                                        _ptr(prefetch_mask, torch.uint8), _stream(stream)), "spice_prefetch_rollout")
 
 
 def spice_lore_calibrate(h_cal, resid, rank, ridge=0.0, iterations=100, stream=None):
@@ -296,8 +302,9 @@ class SpiceLayer:
         conf = self._empty((l_max, T), torch.float32)
         depth = self._empty((T,), torch.int32)
         h_final = self._empty((T, self.cfg.d), torch.bfloat16)
+        self.prefetch_mask = self._empty((l_max, self.cfg.n_experts), torch.uint8)
         spice_prefetch_rollout(self.ctx, [w.c_struct() for w in weights], x_current, T, l_min, l_max, tau, idx, conf,
-                               depth, h_final, stream)
+                               depth, h_final, self.prefetch_mask, stream)
         return idx, conf, depth, h_final
 
     def classify_misses(self, idx, gate, slot_of_expert, conf, stream=None):

@@ -296,6 +296,14 @@ spice_status spice_route_topk(spice_ctx *ctx, const spice_bf16 *h, const spice_b
     return SPICE_OK;
 }
 
+int32_t spice_min_lookahead_depth(int32_t n_prefetch, double expert_bytes, double pcie_bytes_per_s, double t_comp_s) {
+    if (n_prefetch < 0 || !(expert_bytes >= 0.0) || !(pcie_bytes_per_s > 0.0) || !(t_comp_s > 0.0)) return -1;
+    const double x = (double)n_prefetch * expert_bytes / (pcie_bytes_per_s * t_comp_s);
+    if (!(x < 2147483647.0)) return -1;
+    const int32_t f = (int32_t)x;
+    return (double)f < x ? f + 1 : f;
+}
+
 spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, const spice_bf16 *w_draft_router, int32_t T,
                                     int32_t *idx_hat, float *pi_hat, float *conf, void *stream) {
     spice_status s = check_call(ctx, T);
@@ -311,7 +319,7 @@ spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, con
 
 spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *x_current, int32_t T,
                                     int32_t l_min, int32_t l_max, float tau, int32_t *idx_hat, float *conf, int32_t *depth,
-                                    spice_bf16 *h_final, void *stream) {
+                                    spice_bf16 *h_final, uint8_t *prefetch_mask, void *stream) {
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     if (l_max < 1 || l_max > 64 || l_min < 1 || l_min > l_max) return SPICE_ERR_INVALID_ARG;
@@ -378,6 +386,7 @@ spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w
                                     ctx->roll_conf, ctx->draft_logits, ctx->roll_active, ctx->tb, idx_hat, conf, depth, st));
     if (h_final && cudaMemcpyAsync(h_final, ctx->roll_h, bytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return SPICE_ERR_CUDA;
+    if (prefetch_mask) SPICE_LAUNCH(launch_prefetch_set(dm, l_max, idx_hat, prefetch_mask, st));
     return SPICE_OK;
 }
 

@@ -37,6 +37,22 @@ __global__ void __launch_bounds__(256) rollout_mask_kernel(int T, int K, int dep
     for (int k = 0; k < K; ++k) cls[(size_t)t * K + k] = cont ? SPICE_LOWCONF : SPICE_MISS_EXACT;
 }
 
+// Eq. 3: union of the predicted sets over the batch, per depth: mask[l, e] = 1 iff some token predicts expert e at depth l+1
+__global__ void __launch_bounds__(256) prefetch_set_kernel(const int32_t *__restrict__ idx_hat, size_t per_depth, int n_depths, int N,
+                                                           uint8_t *__restrict__ mask) {
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= per_depth * n_depths) return;
+    const int e = idx_hat[i];
+    if (e >= 0 && e < N) mask[(i / per_depth) * N + e] = 1;
+}
+
+int launch_prefetch_set(const Dims &dm, int l_max, const int32_t *idx_hat, uint8_t *mask, cudaStream_t st) {
+    if (cudaMemsetAsync(mask, 0, (size_t)l_max * dm.N, st) != cudaSuccess) return -1;
+    const size_t per_depth = (size_t)dm.T * dm.K, total = per_depth * l_max;
+    prefetch_set_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(idx_hat, per_depth, l_max, dm.N, mask);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 int launch_rollout_mask(const Dims &dm, int depth, int l_min, int l_max, float tau, const float *conf_l, int32_t *active,
                         const int32_t *idx_ws, int32_t *idx_out, float *conf_out, uint8_t *cls, int32_t *depth_out,
                         cudaStream_t st) {

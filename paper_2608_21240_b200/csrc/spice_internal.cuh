@@ -92,6 +92,7 @@ int launch_rollout(const Dims &dm, const spice_layer_weights *w, int l_min, int 
                    __nv_bfloat16 *y_scratch, int32_t *idx_ws, float *gate_ws, uint8_t *cls_ws, float *conf_ws, float *logits_ws,
                    int32_t *active_ws, const Tables &tb, int32_t *idx_hat, float *conf, int32_t *depth, cudaStream_t st);
 
+int launch_prefetch_set(const Dims &dm, int l_max, const int32_t *idx_hat, uint8_t *mask, cudaStream_t st);
 int launch_rollout_mask(const Dims &dm, int depth, int l_min, int l_max, float tau, const float *conf_l, int32_t *active,
                         const int32_t *idx_ws, int32_t *idx_out, float *conf_out, uint8_t *cls, int32_t *depth_out,
                         cudaStream_t st);

@@ -53,3 +53,14 @@ def test_binding_refuses_host_tensors():
     import torch
     with pytest.raises(B.SpiceError):
         B._ptr(torch.zeros(4))
+
+
+def test_min_lookahead_depth_is_eq4_host_arithmetic():
+    """Eq. 4 needs no device: checked against the oracle's ceiling formula on a grid of values, and on bad arguments."""
+    import itertools
+    import oracle
+    from paper_2608_21240_b200 import binding as B
+    for P, Me, Bw, Tc in itertools.product((0, 1, 2, 6), (17.3e6, 55e6), (12e9, 25e9, 50e9), (0.2e-3, 0.5e-3, 1.4e-3, 5e-3)):
+        assert B.spice_min_lookahead_depth(P, Me, Bw, Tc) == oracle.min_lookahead_depth(P, Me, Bw, Tc)
+    assert B.spice_min_lookahead_depth(2, 17.3e6, 25e9, 0.5e-3) == 3
+    assert B.spice_min_lookahead_depth(2, 17.3e6, 0.0, 0.5e-3) == -1 and B.spice_min_lookahead_depth(-1, 1.0, 1.0, 1.0) == -1

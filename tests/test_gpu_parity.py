@@ -364,6 +364,8 @@ def test_prefetch_rollout_matches_oracle(name, T, L, l_min):
     assert dconf[0].max() <= s.top_k * GATE_ATOL and dconf.max() <= 1e-3      # later depths inherit the bf16 state's rounding
     err, bound = y_close(h_final.float().cpu().numpy(), ref_h)
     assert err <= bound + 2e-2, f"max err {err:.3e}"      # + bf16 rounding of the O(1) state
+    # Eq. 3: the per-depth union of the predicted sets
+    assert np.array_equal(Lyr.prefetch_mask.cpu().numpy(), oracle.prefetch_set(ref_idx, s.n_experts))
     # depth 1 is the draft-confidence call
     i1, c1 = Lyr.draft_confidence(bf16_tensor(x), ws[0].w_router)
     assert torch.equal(i1, idx[0]) and torch.equal(c1, conf[0])

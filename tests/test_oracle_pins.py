@@ -487,3 +487,13 @@ def test_p15_lore_calibration_is_a_minimum():
         for eps in (1e-3, 1e-2, 1e-1):
             assert _lore_loss(H, R, A + eps * dA, B + eps * dB) >= loss - 1e-9 * loss
     assert min(_lore_loss(H, R, rng.standard_normal(A.shape), rng.standard_normal(B.shape)) for _ in range(50)) > loss
+
+
+def test_p16_prefetch_set_and_minimum_lookahead_depth():
+    """Eq. 3 on a hand example, and Eq. 4 on the numbers of a worked case: 2 experts of 17.3 MB per layer over a 25 GB/s
+    link need 1.384 ms; with 0.5 ms of compute per layer that is 3 layers of lookahead (2.77 -> 3), with 1.4 ms it is 1."""
+    idx_hat = np.array([[[3, 1], [1, 0]], [[2, 2], [-1, -1]]])        # depth 1: tokens {3,1}, {1,0}; depth 2: {2,2}, stopped
+    assert oracle.prefetch_set(idx_hat, 5).tolist() == [[1, 1, 0, 1, 0], [0, 0, 1, 0, 0]]
+    assert oracle.min_lookahead_depth(2, 17.3e6, 25e9, 0.5e-3) == 3
+    assert oracle.min_lookahead_depth(2, 17.3e6, 25e9, 1.4e-3) == 1
+    assert oracle.min_lookahead_depth(0, 17.3e6, 25e9, 1e-3) == 0
