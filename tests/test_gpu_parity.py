@@ -356,8 +356,8 @@ def test_prefetch_rollout_matches_oracle(name, T, L, l_min):
     n0 = Lyr.launch_count()
     idx, conf, depth, h_final = Lyr.prefetch_rollout(ws, bf16_tensor(x), l_min, L, tau)
     torch.cuda.synchronize()
-    # one fused launch per projecting depth + the last depth's router, confidence and halting kernels
-    assert Lyr.device_status() == 0 and Lyr.launch_count() - n0 == (L - 1) + 3
+    # one fused launch per projecting depth + the last depth's router, confidence and halting kernels + the prefetch set
+    assert Lyr.device_status() == 0 and Lyr.launch_count() - n0 == (L - 1) + 3 + 1
     assert np.array_equal(depth.cpu().numpy(), ref_depth)
     assert np.array_equal(idx.cpu().numpy(), ref_idx)
     dconf = np.abs(conf.cpu().numpy().astype(np.float64) - ref_conf)
@@ -374,7 +374,7 @@ def test_prefetch_rollout_matches_oracle(name, T, L, l_min):
     n1 = Lyr.launch_count()
     gidx, gconf, gdepth, gh = Lyr.prefetch_rollout(ws, bf16_tensor(x), l_min, L, tau)
     torch.cuda.synchronize()
-    assert Lyr.launch_count() - n1 == 3 * L + 5 * (L - 1)
+    assert Lyr.launch_count() - n1 == 3 * L + 5 * (L - 1) + 1
     assert torch.equal(gidx, idx) and torch.equal(gdepth, depth)
     assert (gconf[0] - conf[0]).abs().max().item() <= s.top_k * GATE_ATOL and (gconf - conf).abs().max().item() <= 1e-3
     err, bound = y_close(gh.float().cpu().numpy(), ref_h)
