@@ -1138,7 +1138,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     all = __all_sync(0xffffffffu, mine);
                     if (!all) {
                         if (*abort_flag || ld_relaxed(p.sync + SY_ABORT) || clock64() - w0 > ROLE_WAIT_CYCLES) break;
-                        __nanosleep(100);
+                        __nanosleep(400);
                     }
                 }
             }
