@@ -320,7 +320,9 @@ __device__ __forceinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) 
     const Dims &dm = p.dm;
     const int n_units = dm.N * q.r1_sub;
     int done = 0;
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x, ++done) {
+    // (units are dealt from the last CTA down: the first CTAs start with the shared expert's tiles, and a load issued
+    // behind an SM's own weight stream waits for the bytes already queued)
+    for (int u = gridDim.x - 1 - blockIdx.x; u < n_units; u += gridDim.x, ++done) {
         const int e = u % dm.N, s = u / dm.N;
         const __nv_bfloat16 *row = reinterpret_cast<const __nv_bfloat16 *>(p.w.w_router) + (size_t)e * dm.d;
         for (int t = s * AUX_W + a.aw; t < dm.T; t += AUX_W * q.r1_sub) {
@@ -338,16 +340,17 @@ __device__ __forceinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) 
 // Routing decisions from the logits, entirely in shared memory.  Every CTA computes the same tables
 // (the code is deterministic: counts by atomics, positions by ranking); CTA 0 also writes the outputs.
 // The arithmetic of the gates is that of warp_topk_gates (route_device.cuh).
-__device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
+template <int NPL>
+__device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
-    const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
-    // Phase 1, one warp per token (two tokens at a time, interleaved, so that the reductions of one hide the latency
+    const int T = dm.T, N = dm.N, K = dm.K, S = dm.S;
+    // One warp per token (two tokens at a time, interleaved, so that the reductions of one hide the latency
     // of the other), no barrier inside: the logits go from L2 straight into registers (element e = lane + 32 m),
     // the K winners are found by K rounds of two warp reductions on order-preserving integer keys (largest key, then
     // smallest index among its holders: equal logits go to the smaller expert index), then gates and classes of
     // the token's K entries follow in lanes 0..K-1.  A group's members are kept as a bit mask over the tokens.
-    constexpr int NPL = 8;   // elements per lane, N <= 256
+    // NPL = elements per lane (N <= 32 NPL).
     constexpr int TT = 2;
 #pragma unroll 1
     for (int t0 = a.aw; t0 < T; t0 += AUX_W * TT) {
@@ -488,6 +491,15 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
             }
         }
     }
+}
+
+__device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
+    const DecodeParams &p = q.p;
+    const Dims &dm = p.dm;
+    const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
+    if (N <= 64) aux_route_tokens<2>(q, sh, ax, a);
+    else if (N <= 128) aux_route_tokens<4>(q, sh, ax, a);
+    else aux_route_tokens<8>(q, sh, ax, a);
     aux_sync();
     APROF(a, 73);
     // groups: thread i owns slot i and expert i; packed scan of (entries, non-empty flag << 16)
