@@ -30,6 +30,7 @@ struct spice_ctx {
     int32_t sync_words;
     int32_t decode_tokens;          // largest T of the mma.sync decode kernel (0: path unavailable)
     int32_t dtc_tokens;             // largest T of the tcgen05 decode kernel (0: path unavailable)
+    float *route_logits;            // [Tm, N] router logits of large batches (tensor-core router)
     float *part_split;              // [splits][Td, d] partial shared-expert outputs of the tcgen05 decode kernel
     int n_sms, max_smem_optin;
     TcBuffers tcb;                  // tensor-core path buffers (large batches)
@@ -85,6 +86,7 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->gsc.off = cv.take<int32_t>(2048);
     c->gsc.blk_miss = cv.take<int32_t>(n / 1024 + 2);
     c->draft_logits = cv.take<float>(Tm * g.n_experts);
+    c->route_logits = cv.take<float>(Tm * g.n_experts);
     c->roll_h = cv.take<__nv_bfloat16>(Tm * g.d);
     c->roll_y = cv.take<__nv_bfloat16>(Tm * g.d);
     c->roll_conf = cv.take<float>(Tm);
@@ -516,12 +518,20 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         }
         // cooperative launch refused (e.g. device shared with another context): use the general path
     }
-    SPICE_LAUNCH(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
-                                   gate, nullptr, st));
+    const bool tc_path = ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm);
+    if (tc_path && T >= 256 && tc_router_ok(dm)) {
+        // large batch: the logits are a GEMM of their own (a status word of the GEMM is the tables' one)
+        SPICE_LAUNCH(launch_tc_router_logits(dm, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), ctx->route_logits,
+                                             ctx->tcb, ctx->n_sms, st));
+        SPICE_LAUNCH(launch_topk_from_logits(dm, ctx->cfg.norm_topk, ctx->route_logits, idx, gate, st));
+    } else {
+        SPICE_LAUNCH(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
+                                       gate, nullptr, st));
+    }
     SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
                                  ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st, &ctx->gsc));
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st, &ctx->gsc));
-    if (ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm)) {
+    if (tc_path) {
         // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
         // LoRE on the general kernels
         SPICE_LAUNCH(launch_tc_expert_path(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));

@@ -103,6 +103,32 @@ __global__ void __launch_bounds__(256) draft_confidence_kernel(const float *lp, 
     for (int e = lane; e < N; e += 32) pi_out[(size_t)t * N + e] = expf(l[e] - m) / denom;
 }
 
+// Top-K and gates from logits that another kernel left in global memory ([T, N] fp32): one warp per token, the row
+// is copied to shared memory first.  Used for large batches, whose logits come from the tensor cores.
+__global__ void __launch_bounds__(256) topk_from_logits_kernel(const float *__restrict__ logits, int T, int N, int K, int norm_topk,
+                                                               int32_t *__restrict__ idx, float *__restrict__ gate) {
+    extern __shared__ __align__(16) float smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    float *row = smem + (size_t)warp * N;
+    float *sel_val = smem + (size_t)nwarps * N + warp * 32;
+    int *sel_idx = reinterpret_cast<int *>(smem + (size_t)nwarps * N + nwarps * 32) + warp * 32;
+    const int t = blockIdx.x * nwarps + warp;
+    if (t >= T) return;   // warp-uniform; no block-wide barrier below
+#pragma unroll 1
+    for (int e = lane; e < N; e += 32) row[e] = logits[(size_t)t * N + e];
+    __syncwarp();
+    if (N <= 256) warp_topk_gates(row, N, K, norm_topk, lane, idx + (size_t)t * K, gate + (size_t)t * K, nullptr, sel_idx, sel_val);
+    else warp_topk_gates_rounds(row, N, K, norm_topk, lane, idx + (size_t)t * K, gate + (size_t)t * K, nullptr);
+}
+
+int launch_topk_from_logits(const Dims &dm, int norm_topk, const float *logits, int32_t *idx, float *gate, cudaStream_t st) {
+    const int nwarps = 8;
+    const size_t smem = ((size_t)nwarps * dm.N + 2 * nwarps * 32) * sizeof(float);
+    if (smem > 48 * 1024) return -1;
+    topk_from_logits_kernel<<<(dm.T + nwarps - 1) / nwarps, nwarps * 32, smem, st>>>(logits, dm.T, dm.N, dm.K, norm_topk, idx, gate);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 int launch_draft_confidence(const Dims &dm, const __nv_bfloat16 *h_hat, const __nv_bfloat16 *w_draft, int32_t *idx_hat,
                             float *gate_ws, float *logits_ws, float *pi_hat, float *conf, cudaStream_t st) {
     // logits land in pi_hat when the caller wants the distribution (converted in place), else in the workspace

@@ -13,7 +13,10 @@
 //   warp 1   issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) on the staged tiles; the
 //            accumulator (256 TMEM columns) is double-buffered so the epilogue of tile i overlaps
 //            the main loop of tile i+1; tcgen05.commit releases ring stages / publishes accumulators
-//   warps 2-5 epilogue: tcgen05.ld 32 lanes x 32 columns at a time, SwiGLU or plain, masked stores
+//   warps 2-5 epilogue: tcgen05.ld 32 lanes x 32 columns at a time, SwiGLU or plain; every warp turns its
+//            32 x 32 piece through a private shared-memory buffer so that its global stores are whole
+//            16-byte pieces of consecutive columns (a store then touches 4-8 lines instead of 32)
+// The same kernel (plain mode) computes the router logits of batches of 256 tokens and more.
 // Every wait is bounded: on expiry the CTA records SPICE_ERR_TIMEOUT, stops, drains its own copies
 // in flight (again bounded), frees its TMEM and returns.  No load uses cluster multicast.
 #include <cuda.h>
@@ -31,8 +34,13 @@ constexpr int BM = 128, BK = 64, BN2 = 256;          // CTA tile: 128 rows x 256
 constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN2 * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TC_THREADS = 192;
+constexpr int STG_WARP_BYTES = 32 * 144;             // an epilogue warp's transposition buffer
 
 constexpr uint32_t IDESC = make_idesc(BM, BN2);
+
+// SiLU with the fast reciprocal: the result is rounded to bf16 right after, and under the power cap every
+// instruction the epilogue does not issue is clock for the tensor pipe
+__device__ __forceinline__ float silu_x(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 
 struct TcShared {
     alignas(8) unsigned long long full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
@@ -66,6 +74,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
     // ring first (1024-byte aligned tiles), control block after it
     unsigned char *ring = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     TcShared *sh = reinterpret_cast<TcShared *>(ring + STAGES * STAGE_BYTES);
+    unsigned char *stage_base = ring + STAGES * STAGE_BYTES + 256;   // (TcShared is smaller than 256 bytes)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sh->abort_flag;
 
@@ -163,53 +172,65 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
             const int r = q * 32 + lane;                       // row inside the tile
             const bool row_ok = r < mt.rows;
             const uint32_t t0 = tmem_base + buf * BN2 + ((uint32_t)(q * 32) << 16);
+            // A thread holds one row of the tile, so a warp-wide store of its registers would touch 32 lines with a
+            // few bytes each.  Each warp instead passes 32 columns of its 32 rows through a private piece of shared
+            // memory (row pitch chosen so that the 16-byte accesses do not collide) and writes them out with whole
+            // 16-byte pieces of consecutive columns per lane: a store then covers 8 (bf16) or 4 (fp32) rows' runs.
+            unsigned char *stg = stage_base + (warp - 2) * STG_WARP_BYTES;
             if (MODE == 0) {
                 const int col0 = nt * 128;
-                __nv_bfloat16 *orow = g.out16 + (size_t)(mt.row0 + r) * g.ld;
+                constexpr int PITCH = 80;   // 64 B of bf16 per row + 16
 #pragma unroll 1
                 for (int c = 0; c < 128; c += 32) {
                     uint32_t gv[32], uv[32];
                     tc_ld32(t0 + c, gv);
                     tc_ld32(t0 + 128 + c, uv);
                     tc_wait_ld();
-                    if (row_ok) {
+                    uint32_t pk[16];
 #pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
-                            const int col = col0 + c + j;
-                            const float a0 = silu_f(__uint_as_float(gv[j])) * __uint_as_float(uv[j]);
-                            const float a1 = silu_f(__uint_as_float(gv[j + 1])) * __uint_as_float(uv[j + 1]);
-                            if (col + 1 < g.n_cols) {
-                                __nv_bfloat162 pk = __floats2bfloat162_rn(a0, a1);
-                                *reinterpret_cast<__nv_bfloat162 *>(orow + col) = pk;
-                            } else if (col < g.n_cols) {
-                                orow[col] = __float2bfloat16(a0);
-                            }
-                        }
+                    for (int j = 0; j < 32; j += 2) {
+                        const float a0 = silu_x(__uint_as_float(gv[j])) * __uint_as_float(uv[j]);
+                        const float a1 = silu_x(__uint_as_float(gv[j + 1])) * __uint_as_float(uv[j + 1]);
+                        __nv_bfloat162 b2 = __floats2bfloat162_rn(a0, a1);
+                        pk[j >> 1] = *reinterpret_cast<uint32_t *>(&b2);
                     }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        *reinterpret_cast<uint4 *>(stg + lane * PITCH + k * 16) = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = i * 8 + (lane >> 2), part = lane & 3;
+                        const int col = col0 + c + part * 8;
+                        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * PITCH + part * 16);
+                        if (q * 32 + rr < mt.rows && col < g.n_cols)   // (n_cols is a multiple of 8)
+                            *reinterpret_cast<uint4 *>(g.out16 + (size_t)(mt.row0 + q * 32 + rr) * g.ld + col) = val;
+                    }
+                    __syncwarp();
                 }
             } else {
                 const int col0 = nt * BN2;
-                const int out_r = row_ok ? (g.row_map ? g.row_map[mt.row0 + r] : mt.row0 + r) : 0;
-                float *orow = g.out32 + (size_t)out_r * g.ld;
+                const int out_r = row_ok ? (g.row_map ? g.row_map[mt.row0 + r] : mt.row0 + r) : -1;
+                constexpr int PITCH = 144;   // 128 B of fp32 per row + 16
 #pragma unroll 1
                 for (int c = 0; c < BN2; c += 32) {
                     uint32_t v[32];
                     tc_ld32(t0 + c, v);
                     tc_wait_ld();
-                    if (row_ok) {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            const int col = col0 + c + j;
-                            if (col + 3 < g.n_cols) {
-                                *reinterpret_cast<float4 *>(orow + col) =
-                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                                                __uint_as_float(v[j + 3]));
-                            } else {
-                                for (int e = 0; e < 4; ++e)
-                                    if (col + e < g.n_cols) orow[col + e] = __uint_as_float(v[j + e]);
-                            }
-                        }
+                    for (int k = 0; k < 8; ++k)
+                        *reinterpret_cast<uint4 *>(stg + lane * PITCH + k * 16) = make_uint4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int rr = i * 4 + (lane >> 3), part = lane & 7;
+                        const int col = col0 + c + part * 4;
+                        const int orow = __shfl_sync(0xffffffffu, out_r, rr);
+                        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * PITCH + part * 16);
+                        if (orow >= 0 && col < g.n_cols)   // (n_cols is a multiple of 4)
+                            *reinterpret_cast<uint4 *>(g.out32 + (size_t)orow * g.ld + col) = val;
                     }
+                    __syncwarp();
                 }
             }
             tc_fence_before();
@@ -219,7 +240,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
     }
     tc_fence_before();
     __syncthreads();
-    if (threadIdx.x == 0 && sh->abort_flag) atomicMax(g.status, (int)SPICE_ERR_TIMEOUT);
+    if (threadIdx.x == 0 && sh->abort_flag && g.status) atomicMax(g.status, (int)SPICE_ERR_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
@@ -331,7 +352,8 @@ bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], co
 
 namespace {
 
-constexpr size_t TC_SMEM = STAGES * STAGE_BYTES + sizeof(TcShared) + 1024;
+static_assert(sizeof(TcShared) <= 256, "control block");
+constexpr size_t TC_SMEM = STAGES * STAGE_BYTES + 256 + 4 * STG_WARP_BYTES + 1024;
 
 }  // namespace
 
@@ -349,6 +371,31 @@ bool tc_shape_ok(const Dims &dm) {
     // TMA: row pitches must be multiples of 16 bytes (dims are multiples of 8: yes); nothing else is required,
     // partial tiles are zero-filled on load and masked on store
     return dm.d % 8 == 0 && dm.I % 8 == 0 && dm.Is % 8 == 0;
+}
+
+// Router logits of a large batch (Eq. 1) as one GEMM on the tensor cores: logits[T, N] = h W_r^T, fp32 out.  The
+// router matrix plays the weight operand of "slot" 0 (rows past N are zero-filled by the tensor map).
+bool tc_router_ok(const Dims &dm) { return tc_shape_ok(dm) && dm.N <= BN2 && dm.N % 4 == 0; }
+
+int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router, float *logits,
+                            const TcBuffers &b, int n_sms, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    build_shared_mtiles_kernel<<<1, 32, 0, st>>>(dm.T, b.mtiles_shared, b.n_mtiles_shared);
+    if (!make_map(&ma, h, dm.T, dm.d, BM) || !make_map(&mb, w_router, dm.N, dm.d, 128)) return -1;
+    TcGemmArgs g{};
+    g.mtiles = b.mtiles_shared;
+    g.n_mtiles = b.n_mtiles_shared;
+    g.n_ntiles = 1;
+    g.K = dm.d;
+    g.b_rows_per_slot = 0;
+    g.b_second_off = 0;
+    g.n_cols = dm.N;
+    g.out32 = logits;
+    g.row_map = nullptr;
+    g.ld = dm.N;
+    g.status = nullptr;
+    tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
 // The exact-expert part of a large batch: gather, grouped gate/up + SwiGLU, grouped down, for the hit groups and

@@ -9,6 +9,11 @@ from paper_2608_21240_b200 import workloads as W
 
 Y_RTOL, Y_ATOL = 1e-2, 1e-3      # max|gpu - oracle| <= 1e-2 * max|oracle| + 1e-3
 GATE_ATOL = 2e-6
+# Batches of 256 tokens and more take their router logits from the tensor cores, whose fp32 accumulator truncates
+# after every 16-term step: over d / 16 steps the logit error is bounded by (d / 16) * 2^-23 * max|partial sum|
+# (2.7e-4 for d = 3584 and partial sums up to 10; observed 1.5e-5) and a gate moves by at most a quarter of that.
+GATE_ATOL_TC = 7e-5
+TC_ROUTER_TOKENS = 256
 LOGIT_ATOL = 2e-4
 
 
@@ -22,10 +27,11 @@ def y_close(y_gpu: np.ndarray, y_ref: np.ndarray):
 
 
 def check_routing(out, ref, T, K):
-    """Bit-exact idx / cls / counts / residual list; gates within fp32 rounding."""
+    """Bit-exact idx / cls / counts / residual list; gates within the rounding of the path that produced the logits."""
+    gate_atol = GATE_ATOL_TC if T >= TC_ROUTER_TOKENS else GATE_ATOL
     idx = out.idx.cpu().numpy()
     assert np.array_equal(idx, ref.idx), "top-k indices differ"
-    assert np.abs(out.gate.cpu().numpy().astype(np.float64) - ref.gate).max() <= GATE_ATOL
+    assert np.abs(out.gate.cpu().numpy().astype(np.float64) - ref.gate).max() <= gate_atol
     assert np.array_equal(out.cls.cpu().numpy(), ref.cls), "classification differs"
     counts = out.counts.cpu().numpy()
     assert counts.tolist() == ref.counts.tolist()
@@ -34,4 +40,4 @@ def check_routing(out, ref, T, K):
     assert np.array_equal(out.resid_k.cpu().numpy()[:n], ref.resid_k)
     assert np.array_equal(out.resid_expert.cpu().numpy()[:n], ref.resid_expert)
     if n:
-        assert np.abs(out.resid_gate.cpu().numpy()[:n].astype(np.float64) - ref.resid_gate).max() <= GATE_ATOL
+        assert np.abs(out.resid_gate.cpu().numpy()[:n].astype(np.float64) - ref.resid_gate).max() <= gate_atol
