@@ -6,6 +6,7 @@ resident slots, shared expert + LoRE surrogate, combine) over one decode batch o
 DeepSeek-V2-Lite-shaped layer.  Successive steps rotate through several independent
 layer weight sets so that the bytes touched between two uses of the same weights are
 several times the L2 capacity (cold-L2 timing without a flush inside the timed region).
+The timed steps are submitted as replayed CUDA graphs of captured steps (--launch eager: one call per step).
 
 Prints ONE JSON line: metric, value, unit, timing, `config` (the workload), `roofline` (algorithmic bytes or FLOPs of
 the timed calls over their time, against the measured peak), `e2e` (the same metric with host<->device copies inside
@@ -194,7 +195,7 @@ def run_ours(args):
 
     def step(i):
         B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h, conf, T, y, idx=idx, gate=gate, cls=cls, counts=counts,
-                              stream=stream)
+                              stream=torch.cuda.current_stream())
 
     # algorithmic bytes of every replica's call (from the routing the library itself produced)
     rep_bytes, rep_hit, rep_low, rep_hit_picks = [], [], [], []
@@ -214,19 +215,12 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     l0 = layer.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    w0 = time.time()
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    w1 = time.time()
+    step(0)
+    launches_per_step = layer.launch_count() - l0
+    ms, how, w0, w1 = timed_steps(torch, step, args.steps, args.launch)
     if world > 1:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    launches = layer.launch_count() - l0
+    launches = launches_per_step * args.steps
     total_bytes = sum(rep_bytes[i % R] for i in range(args.steps))
 
     # end to end: inputs start in pinned host memory, the result is read back to the host every step.  The caller
@@ -290,6 +284,7 @@ def run_ours(args):
                                    f"tau={shape.tau}, Beta(2,2) confidences)",
                        "tokens_per_step": T, "cold_l2": f"steps rotate through {R} independent weight sets "
                        f"({sum(rep_bytes) / 1e6:.0f} MB between reuses, L2 is 126 MB); no flush in the timed region",
+                       "launch": how,
                        "distinct_hit_experts_mean": float(np.mean(rep_hit)),
                        "distinct_lowconf_experts_mean": float(np.mean(rep_low)),
                        "multi_gpu": "replicas only (no collective on the data path)"},
@@ -316,6 +311,47 @@ def run_ours(args):
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def timed_steps(torch, step_fn, n_steps, launch):
+    """Times exactly n_steps calls of step_fn(i) (which enqueues step i on torch's current stream) with CUDA events.
+    launch == "graph": the steps are captured into CUDA graphs of up to 256 steps and replayed, the way a decode loop
+    submits a fixed layer call; launch == "eager": one library call per step from Python.  Returns (ms, description)."""
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    how = "one library call per step"
+    plan = None
+    if launch == "graph":
+        try:
+            chunk = min(n_steps, 256)
+            sizes = [chunk] + ([n_steps % chunk] if n_steps % chunk else [])
+            graphs = []
+            for n in sizes:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for i in range(n):
+                        step_fn(i)
+                graphs.append(g)
+            plan = [graphs[0]] * (n_steps // chunk) + (graphs[1:] if n_steps % chunk else [])
+            for g in graphs:
+                g.replay()          # untimed: instantiates and uploads the graph
+            how = f"CUDA graphs of {chunk} captured steps, replayed"
+        except Exception as ex:     # capture refused: time the eager loop and say so
+            plan = None
+            how = f"one library call per step (graph capture failed: {type(ex).__name__})"
+    torch.cuda.synchronize()
+    w0 = time.time()
+    e0.record(stream)
+    if plan is not None:
+        for g in plan:
+            g.replay()
+    else:
+        for i in range(n_steps):
+            step_fn(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    w1 = time.time()
+    return e0.elapsed_time(e1), how, w0, w1
 
 
 # ----------------------------------------------------------------------------- 26-layer decode stack (config 5)
@@ -393,7 +429,8 @@ def run_stack(args):
 
     def step():
         for l in range(n_layers):
-            B.spice_moe_layer_fwd(layer.ctx, structs[l], hs[l], confs[l], T, y, x_resid=x, idx=idx, cls=cls, stream=stream)
+            B.spice_moe_layer_fwd(layer.ctx, structs[l], hs[l], confs[l], T, y, x_resid=x, idx=idx, cls=cls,
+                                  stream=torch.cuda.current_stream())
 
     total_bytes, hit_frac = 0, []
     for l in range(n_layers):
@@ -409,18 +446,12 @@ def run_stack(args):
     if world > 1:
         dist.barrier()
     l0 = layer.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    w0 = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    torch.cuda.synchronize()
-    w1 = time.time()
+    step()
+    launches_per_step = layer.launch_count() - l0
+    ms, how, w0, w1 = timed_steps(torch, lambda i: step(), args.steps, args.launch)
     if world > 1:
         dist.barrier()
-    ms = e0.elapsed_time(e1)
-    launches = layer.launch_count() - l0
+    launches = launches_per_step * args.steps
     # end to end: the residual stream comes from pinned host memory and goes back every step
     x_host = torch.zeros(T, shape.d, dtype=torch.bfloat16).pin_memory()
     out_host = torch.empty(T, shape.d, dtype=torch.bfloat16).pin_memory()
@@ -450,7 +481,7 @@ def run_stack(args):
             "config": {"workload": f"MoE layers of a {n_layers}-layer DeepSeek-V2-Lite-shaped decoder, decode batch {T}, "
                                    f"free running ({shape.n_slots} resident slots per layer, residency chosen given the "
                                    f"routing: mean hit rate {np.mean(hit_frac):.2f}, misses low-confidence w.p. 1/2)",
-                       "tokens_per_step": T, "layer_calls_per_step": n_layers,
+                       "tokens_per_step": T, "layer_calls_per_step": n_layers, "launch": how,
                        "cold_l2": f"every layer has its own weights ({total_bytes / 1e6:.0f} MB touched per step, "
                                   f"L2 is 126 MB); no flush in the timed region",
                        "multi_gpu": "replicas only (no collective on the data path)"},
@@ -719,6 +750,8 @@ def main():
                     help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
     ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout", "lore_calibrate"],
                     help="what a step is: the MoE layer call (default) or the draft-router confidence call")
+    ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
+                    help="how the timed steps are submitted: replayed CUDA graphs of captured steps (default) or one call per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
