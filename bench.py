@@ -328,7 +328,7 @@ def timed_steps(torch, step_fn, n_steps, launch):
             graphs = []
             for n in sizes:
                 g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g):
+                with torch.cuda.graph(g, capture_error_mode="thread_local"):   # other threads (NCCL watchdog) may call CUDA
                     for i in range(n):
                         step_fn(i)
                 graphs.append(g)

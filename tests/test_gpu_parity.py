@@ -115,6 +115,33 @@ def test_classify_threshold_edges_and_scalar_conf():
     L.close()
 
 
+@pytest.mark.parametrize("name,T", [("tiny", 6), ("dsv2lite", 8), ("tiny", 300)])
+def test_a_token_of_nans_stays_in_its_own_row(name, T):
+    """Tokens are independent (Sec. 2.1: every token is routed and combined on its own).  A token whose hidden state
+    is NaN selects the experts 0..K-1 (NaN never wins a comparison, equal logits go to the smaller index) and gets a
+    NaN output; routing, classes and outputs of every OTHER token equal the oracle's for the clean batch.  Covers the
+    fused decode kernel (every group is multiplied with all token columns) and the large-batch path (tensor-core
+    router, grouped GEMMs)."""
+    wl = _layer_case(name, T, variant=31)
+    s = wl.shape
+    ref = run_oracle(wl, want_full=False)
+    bad = 2
+    h = wl.h.copy()
+    h[bad, :] = np.nan
+    L = B.SpiceLayer(cfg_of(s), T)
+    out = L.moe_layer_fwd(upload(wl), bf16_tensor(h), torch.from_numpy(wl.conf).cuda())
+    torch.cuda.synchronize()
+    keep = np.arange(T) != bad
+    idx, cls, y = out.idx.cpu().numpy(), out.cls.cpu().numpy(), out.y.float().cpu().numpy()
+    assert idx[bad].tolist() == list(range(s.top_k))
+    assert np.array_equal(idx[keep], ref.idx[keep]) and np.array_equal(cls[keep], ref.cls[keep])
+    assert np.isnan(y[bad]).all() and np.isfinite(y[keep]).all()
+    err, bound = y_close(y[keep], ref.y[keep])
+    assert err <= bound, (err, bound)
+    assert L.device_status() == 0
+    L.close()
+
+
 def _fwd_and_check(wl, tokens=None, y_cpu=None, general_path=False, **ora):
     s = wl.shape
     ref = run_oracle(wl, tokens=tokens, **ora)
