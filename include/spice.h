@@ -135,7 +135,7 @@ spice_status spice_lore_surrogate(spice_ctx *ctx, const spice_layer_weights *w /
  *   y [T,d] bf16 out.  idx, gate, cls, counts, resid_*: as above; each may be NULL when not wanted.
  * Equals spice_route_topk, spice_classify_misses, y = 0, spice_grouped_expert_ffn,
  * spice_lore_surrogate applied in turn, up to fp32 summation order and the final bf16 rounding.
- * Batches of 256 tokens and more take their router logits from a tensor-core GEMM (fp32 accumulation, truncated after
+ * Batches of more than 64 tokens take their router logits from a tensor-core GEMM (fp32 accumulation, truncated after
  * every 16 terms): the selection rule is the same, the logits differ from spice_route_topk's by up to ~1e-5, so idx
  * agrees with it whenever a token's K-th and (K+1)-th logits are further apart than that; gates agree to 4e-6. */
 spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w /* host struct */,

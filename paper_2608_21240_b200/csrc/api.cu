@@ -106,7 +106,7 @@ void carve(spice_ctx *c, char *base, size_t *total) {
         c->tcb.x_perm = cv.take<__nv_bfloat16>(n * g.d);
         c->tcb.act16 = cv.take<__nv_bfloat16>(n * g.inter);
         c->tcb.act_shared16 = cv.take<__nv_bfloat16>(Tm * g.inter_shared);
-        c->tcb.mtiles = cv.take<MTile>(n / 128 + g.n_slots + 1);
+        c->tcb.mtiles = cv.take<MTile>(n / 128 + (g.n_slots > g.n_experts ? g.n_slots : g.n_experts) + 2);   // hit groups, later LOW groups
         c->tcb.mtiles_shared = cv.take<MTile>(Tm / 128 + 1);
         c->tcb.n_mtiles = cv.take<int32_t>(4);
         c->tcb.n_mtiles_shared = cv.take<int32_t>(4);
@@ -519,7 +519,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         // cooperative launch refused (e.g. device shared with another context): use the general path
     }
     const bool tc_path = ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm);
-    if (tc_path && T >= 256 && tc_router_ok(dm)) {
+    if (tc_path && T > 64 && tc_router_ok(dm)) {
         // large batch: the logits are a GEMM of their own (a status word of the GEMM is the tables' one)
         SPICE_LAUNCH(launch_tc_router_logits(dm, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), ctx->route_logits,
                                              ctx->tcb, ctx->n_sms, st));
@@ -535,8 +535,13 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
         // LoRE on the general kernels
         SPICE_LAUNCH(launch_tc_expert_path(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
-        SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
-        SPICE_LAUNCH(launch_down(dm, KIND_LOW, *w, ctx->tb, st));
+        if (tc_lore_ok(dm)) {
+            SPICE_LAUNCH(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 1, st));
+        } else {
+            SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
+            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 0, st));
+        }
     } else {
         SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED | KIND_HIT, *w, hb, ctx->tb, st));
         SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));

@@ -252,6 +252,49 @@ __global__ void __launch_bounds__(256) combine_kernel(Dims dm, CombineArgs a, Ta
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// LoRE up-projection alone (LOW groups only): part[entry, j] = sum_k B_e[j,k] z[p,k].  The reduction is only r long,
+// so a warp per output row would leave most lanes idle; here a THREAD owns output column j, streams its row of B_e
+// (r bf16) and applies it to LB tokens at a time whose z rows sit in shared memory (all threads read the same word:
+// a broadcast).  Groups are walked with a stride, so a launch that finds no LOW group costs a few small CTAs.
+constexpr int LB = 8;        // tokens per pass
+constexpr int LB_GROUPS = 32;
+
+__global__ void __launch_bounds__(256) lore_b_kernel(Dims dm, spice_layer_weights w, Tables tb, int z_after_hits) {
+    extern __shared__ __align__(16) float zs[];   // [LB][r]
+    const int r = dm.r, d = dm.d;
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    const int first = 1 + tb.hdr[HDR_N_HIT_GROUPS], n_groups = tb.hdr[HDR_N_GROUPS];
+    for (int g = first + blockIdx.y; g < n_groups; g += gridDim.y) {
+        const GroupDesc grp = tb.groups[g];
+        if (grp.kind != KIND_LOW) continue;   // (uniform)
+        const __nv_bfloat16 *row = reinterpret_cast<const __nv_bfloat16 *>(w.lore_B) + ((size_t)grp.id * d + (j < d ? j : 0)) * r;
+        // (z rows are numbered like the low entries, or behind the hit entries when the GEMM path produced them)
+        const float *z = tb.z_low + (size_t)(grp.off + (z_after_hits ? tb.hdr[HDR_N_HIT] : 0)) * r;
+        const int32_t *perm = tb.perm_low + grp.off;
+        for (int p0 = 0; p0 < grp.m; p0 += LB) {
+            const int mt = min(LB, grp.m - p0);
+            __syncthreads();
+            for (int v = threadIdx.x; v < LB * r; v += 256) zs[v] = v < mt * r ? z[(size_t)p0 * r + v] : 0.f;
+            __syncthreads();
+            float acc[LB];
+#pragma unroll
+            for (int m = 0; m < LB; ++m) acc[m] = 0.f;
+            if (j < d) {
+#pragma unroll 2
+                for (int k = 0; k < r; k += 8) {
+                    const uint4 u = *reinterpret_cast<const uint4 *>(row + k);
+#pragma unroll
+                    for (int m = 0; m < LB; ++m) fma8(u, zs + m * r + k, acc[m]);
+                }
+#pragma unroll
+                for (int m = 0; m < LB; ++m)
+                    if (m < mt) tb.part[(size_t)perm[p0 + m] * d + j] = acc[m];
+            }
+        }
+    }
+}
+
 static inline int max_groups(const Dims &dm) {
     const int n = dm.T * dm.K;
     return 1 + min(dm.S, n) + min(dm.N, n);
@@ -275,6 +318,14 @@ int launch_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloa
 int launch_down(const Dims &dm, int kind_mask, const spice_layer_weights &w, const Tables &tb, cudaStream_t st) {
     dim3 grid((dm.d + GW - 1) / GW, kind_mask == KIND_LOW ? min(dm.N, dm.T * dm.K) : max_groups(dm));
     down_kernel<<<grid, GT, 0, st>>>(dm, kind_mask, w, tb);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_lore_b(const Dims &dm, const spice_layer_weights &w, const Tables &tb, int z_after_hits, cudaStream_t st) {
+    const size_t smem = (size_t)LB * dm.r * sizeof(float);
+    if (smem > 48 * 1024) return z_after_hits ? -1 : launch_down(dm, KIND_LOW, w, tb, st);
+    dim3 grid((dm.d + 255) / 256, min(LB_GROUPS, min(dm.N, dm.T * dm.K)));
+    lore_b_kernel<<<grid, 256, smem, st>>>(dm, w, tb, z_after_hits);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

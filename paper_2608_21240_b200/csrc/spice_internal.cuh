@@ -73,6 +73,7 @@ int launch_gateup(const Dims &dm, int kind_mask, const spice_layer_weights &w, c
 int launch_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
                   cudaStream_t st);
 int launch_down(const Dims &dm, int kind_mask, const spice_layer_weights &w, const Tables &tb, cudaStream_t st);
+int launch_lore_b(const Dims &dm, const spice_layer_weights &w, const Tables &tb, int z_after_hits, cudaStream_t st);   // LOW groups only
 
 struct CombineArgs {
     int kind_mask;              // which terms enter
@@ -177,6 +178,10 @@ int launch_tc_expert_path(const Dims &dm, const spice_layer_weights &w, const __
 bool tc_router_ok(const Dims &dm);
 int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router, float *logits,
                             const TcBuffers &b, int n_sms, cudaStream_t st);
+// LoRE of a large batch: z = A_e h through the GEMM kernel (rows n_hit + p of tb.z_low), then lore_b_kernel
+bool tc_lore_ok(const Dims &dm);
+int launch_tc_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb, const TcBuffers &b,
+                     int n_sms, cudaStream_t st);
 int launch_topk_from_logits(const Dims &dm, int norm_topk, const float *logits, int32_t *idx, float *gate, cudaStream_t st);
 
 // ---- small device helpers

@@ -16,7 +16,7 @@
 //   warps 2-5 epilogue: tcgen05.ld 32 lanes x 32 columns at a time, SwiGLU or plain; every warp turns its
 //            32 x 32 piece through a private shared-memory buffer so that its global stores are whole
 //            16-byte pieces of consecutive columns (a store then touches 4-8 lines instead of 32)
-// The same kernel (plain mode) computes the router logits of batches of 256 tokens and more.
+// The same kernel (plain mode) computes the router logits of batches of more than 64 tokens.
 // Every wait is bounded: on expiry the CTA records SPICE_ERR_TIMEOUT, stops, drains its own copies
 // in flight (again bounded), frees its TMEM and returns.  No load uses cluster multicast.
 #include <cuda.h>
@@ -396,6 +396,72 @@ int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_b
     g.status = nullptr;
     tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+// ---- LoRE down-projection z = A_e h of the LOW groups of a large batch, through the same GEMM kernel.
+// The low entries' tokens are gathered behind the hit entries' rows of x_perm (rows n_hit + p, p in perm_low order),
+// lore_A plays the weight operand with the expert index as the "slot" (r rows each), z lands in tb.z_low at the
+// same row numbers (fp32), where lore_b_kernel picks it up.
+__global__ void __launch_bounds__(256) gather_low_rows_kernel(const __nv_bfloat16 *__restrict__ h, const int32_t *__restrict__ perm,
+                                                              const int32_t *__restrict__ hdr, int K, int d,
+                                                              __nv_bfloat16 *__restrict__ out) {
+    const int n_hit = hdr[HDR_N_HIT], n_low = hdr[HDR_N_LOW];
+    const int vec = d >> 3;
+    for (int p = blockIdx.x; p < n_low; p += gridDim.x) {
+        const int t = perm[p] / K;
+        const uint4 *src = reinterpret_cast<const uint4 *>(h + (size_t)t * d);
+        uint4 *dst = reinterpret_cast<uint4 *>(out + (size_t)(n_hit + p) * d);
+        for (int v = threadIdx.x; v < vec; v += blockDim.x) dst[v] = src[v];
+    }
+}
+
+// m-tiles of the LOW groups (they follow the hit groups in the group list); one warp, a group per lane
+__global__ void build_low_mtiles_kernel(const GroupDesc *__restrict__ groups, const int32_t *__restrict__ hdr, MTile *mtiles,
+                                        int32_t *n_mtiles) {
+    if (blockIdx.x != 0 || threadIdx.x >= 32) return;
+    const int lane = threadIdx.x;
+    const int n_hg = hdr[HDR_N_HIT_GROUPS], n_lg = hdr[HDR_N_LOW_GROUPS], n_hit = hdr[HDR_N_HIT];
+    int base = 0;
+    for (int g0 = 0; g0 < n_lg; g0 += 32) {
+        GroupDesc grp{0, 0, 0, 0};
+        if (g0 + lane < n_lg) grp = groups[1 + n_hg + g0 + lane];
+        const int nt = (grp.m + BM - 1) / BM;
+        int inc = nt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += v;
+        }
+        const int first = base + inc - nt;
+        for (int j = 0; j < nt; ++j) mtiles[first + j] = MTile{grp.id, n_hit + grp.off + j * BM, min(BM, grp.m - j * BM), 0};
+        base += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) *n_mtiles = base;
+}
+
+bool tc_lore_ok(const Dims &dm) { return tc_shape_ok(dm) && dm.r <= BN2 && dm.r % 8 == 0; }
+
+int launch_tc_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb, const TcBuffers &b,
+                     int n_sms, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    const size_t cap = (size_t)dm.T * dm.K;
+    build_low_mtiles_kernel<<<1, 32, 0, st>>>(tb.groups, tb.hdr, b.mtiles, b.n_mtiles);
+    gather_low_rows_kernel<<<n_sms * 2, 256, 0, st>>>(h, tb.perm_low, tb.hdr, dm.K, dm.d, b.x_perm);
+    if (!make_map(&ma, b.x_perm, cap, dm.d, BM) || !make_map(&mb, w.lore_A, (uint64_t)dm.N * dm.r, dm.d, 128)) return -1;
+    TcGemmArgs g{};
+    g.mtiles = b.mtiles;
+    g.n_mtiles = b.n_mtiles;
+    g.n_ntiles = 1;
+    g.K = dm.d;
+    g.b_rows_per_slot = dm.r;
+    g.b_second_off = 0;
+    g.n_cols = dm.r;
+    g.out32 = tb.z_low;
+    g.row_map = nullptr;
+    g.ld = dm.r;
+    g.status = tb.status;
+    tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    return cudaGetLastError() == cudaSuccess ? 3 : -1;
 }
 
 // The exact-expert part of a large batch: gather, grouped gate/up + SwiGLU, grouped down, for the hit groups and
