@@ -31,6 +31,8 @@ struct spice_ctx {
     int32_t decode_tokens;          // largest T of the mma.sync decode kernel (0: path unavailable)
     int32_t dtc_tokens;             // largest T of the tcgen05 decode kernel (0: path unavailable)
     float *route_logits;            // [Tm, N] router logits of large batches (tensor-core router)
+    cudaStream_t side;              // large batches: the shared expert runs here beside the routing chain (null: in line)
+    cudaEvent_t ev_fork, ev_join;
     float *part_split;              // [splits][Td, d] partial shared-expert outputs of the tcgen05 decode kernel
     int n_sms, max_smem_optin;
     TcBuffers tcb;                  // tensor-core path buffers (large batches)
@@ -220,6 +222,20 @@ spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg
     c->decode_tokens = (coop && decode_prepare(c->max_smem_optin) == 0) ? (max_tokens < 16 ? max_tokens : 16) : 0;
     c->tcb = TcBuffers{};
     c->tc_ok = tc_available() && tc_prepare() == 0;
+    c->side = nullptr;
+    c->ev_fork = c->ev_join = nullptr;
+    if (c->tc_ok) {
+        if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            if (c->side) cudaStreamDestroy(c->side);
+            if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+            if (c->ev_join) cudaEventDestroy(c->ev_join);
+            c->side = nullptr;
+            c->ev_fork = c->ev_join = nullptr;
+        }
+    }
     c->dtc_tokens = (coop && c->tc_ok && decode_tc_prepare(c->max_smem_optin) == 0) ? (max_tokens < 64 ? max_tokens : 64) : 0;
     carve(c, nullptr, &c->ws_bytes);
     if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
@@ -242,6 +258,11 @@ spice_status spice_destroy(spice_ctx *ctx) {
     if (!ctx) return SPICE_OK;
     cudaSetDevice(ctx->device);
     cudaError_t e = cudaFree(ctx->ws);
+    if (ctx->side) {
+        cudaStreamDestroy(ctx->side);
+        cudaEventDestroy(ctx->ev_fork);
+        cudaEventDestroy(ctx->ev_join);
+    }
     delete ctx;
     return e == cudaSuccess ? SPICE_OK : SPICE_ERR_CUDA;
 }
@@ -519,6 +540,20 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         // cooperative launch refused (e.g. device shared with another context): use the general path
     }
     const bool tc_path = ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm);
+    // The shared expert needs nothing but h: it runs on the context's side stream beside the routing chain (router,
+    // classification, grouping, gather occupy few SMs) and joins before the combine.  Both event edges are ordinary
+    // stream dependencies, so the call can still be captured into a CUDA graph.
+    bool forked = false;
+    if (tc_path) {
+        if (ctx->side && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
+            cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess) {
+            SPICE_LAUNCH(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ctx->side));
+            if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return SPICE_ERR_CUDA;
+            forked = true;
+        } else {
+            cudaGetLastError();
+        }
+    }
     if (tc_path && T > 64 && tc_router_ok(dm)) {
         // large batch: the logits are a GEMM of their own (a status word of the GEMM is the tables' one)
         SPICE_LAUNCH(launch_tc_router_logits(dm, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), ctx->route_logits,
@@ -534,7 +569,8 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     if (tc_path) {
         // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
         // LoRE on the general kernels
-        SPICE_LAUNCH(launch_tc_expert_path(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        SPICE_LAUNCH(launch_tc_routed(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        if (!forked) SPICE_LAUNCH(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
         if (tc_lore_ok(dm)) {
             SPICE_LAUNCH(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
             SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 1, st));
@@ -547,6 +583,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
         SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_HIT | KIND_LOW, *w, ctx->tb, st));
     }
+    if (forked && cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SPICE_ERR_CUDA;
     CombineArgs ca{KIND_SHARED | KIND_HIT | KIND_LOW, 0, gate, cls, nullptr, reinterpret_cast<__nv_bfloat16 *>(y),
                    y_cpu_residual, reinterpret_cast<__nv_bfloat16 *>(x_resid)};
     SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));

@@ -172,8 +172,10 @@ struct TcBuffers {
 bool tc_available();
 int tc_prepare();
 bool tc_shape_ok(const Dims &dm);
-int launch_tc_expert_path(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
-                          const TcBuffers &b, int n_sms, cudaStream_t st);
+int launch_tc_routed(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
+                     const TcBuffers &b, int n_sms, cudaStream_t st);
+int launch_tc_shared(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
+                     const TcBuffers &b, int n_sms, cudaStream_t st);
 // router logits of a large batch as a GEMM, then Top-K from the stored logits (route.cu)
 bool tc_router_ok(const Dims &dm);
 int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router, float *logits,

@@ -380,11 +380,13 @@ bool tc_router_ok(const Dims &dm) { return tc_shape_ok(dm) && dm.N <= BN2 && dm.
 int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router, float *logits,
                             const TcBuffers &b, int n_sms, cudaStream_t st) {
     CUtensorMap ma, mb;
-    build_shared_mtiles_kernel<<<1, 32, 0, st>>>(dm.T, b.mtiles_shared, b.n_mtiles_shared);
+    // (the tile list of the routed experts is free until the grouping has run; the shared expert's list may be in
+    // use on the side stream)
+    build_shared_mtiles_kernel<<<1, 32, 0, st>>>(dm.T, b.mtiles, b.n_mtiles);
     if (!make_map(&ma, h, dm.T, dm.d, BM) || !make_map(&mb, w_router, dm.N, dm.d, 128)) return -1;
     TcGemmArgs g{};
-    g.mtiles = b.mtiles_shared;
-    g.n_mtiles = b.n_mtiles_shared;
+    g.mtiles = b.mtiles;
+    g.n_mtiles = b.n_mtiles;
     g.n_ntiles = 1;
     g.K = dm.d;
     g.b_rows_per_slot = 0;
@@ -464,11 +466,11 @@ int launch_tc_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bf
     return cudaGetLastError() == cudaSuccess ? 3 : -1;
 }
 
-// The exact-expert part of a large batch: gather, grouped gate/up + SwiGLU, grouped down, for the hit groups and
-// for the shared expert.  Results land in tb.part (by entry id) and tb.part_shared (by token) as fp32, exactly
-// where the general kernels put them, so the LoRE path and the combine kernel are shared with the general path.
-int launch_tc_expert_path(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
-                          const TcBuffers &b, int n_sms, cudaStream_t st) {
+// The exact-expert part of a large batch: gather, grouped gate/up + SwiGLU, grouped down for the hit groups.
+// Results land in tb.part (by entry id) (the shared expert's in tb.part_shared, by token) as fp32, exactly where the
+// general kernels put them, so the combine kernel is shared with the general path.
+int launch_tc_routed(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
+                     const TcBuffers &b, int n_sms, cudaStream_t st) {
     CUtensorMap ma, mb;
     int launches = 0;
     const size_t cap = (size_t)dm.T * dm.K;
@@ -503,7 +505,17 @@ int launch_tc_expert_path(const Dims &dm, const spice_layer_weights &w, const __
     g.ld = dm.d;
     tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
     ++launches;
-    // ---- shared expert: one group of all T tokens, A is h itself
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+// The shared expert S of a large batch: one group of all T tokens, A is h itself.  It depends on nothing but h, so
+// the caller may run it on a second stream beside the routing chain.
+int launch_tc_shared(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
+                     const TcBuffers &b, int n_sms, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    int launches = 0;
+    TcGemmArgs g{};
+    g.status = tb.status;
     build_shared_mtiles_kernel<<<1, 32, 0, st>>>(dm.T, b.mtiles_shared, b.n_mtiles_shared);
     ++launches;
     if (!make_map(&ma, h, dm.T, dm.d, BM) || !make_map(&mb, w.shared_w_gate_up, (uint64_t)2 * dm.Is, dm.d, 128)) return -1;
