@@ -32,7 +32,7 @@ struct spice_ctx {
     int32_t dtc_tokens;             // largest T of the tcgen05 decode kernel (0: path unavailable)
     float *route_logits;            // [Tm, N] router logits of large batches (tensor-core router)
     cudaStream_t side;              // large batches: the shared expert runs here beside the routing chain (null: in line)
-    cudaEvent_t ev_fork, ev_join;
+    cudaEvent_t ev_fork, ev_join, ev_grouped;
     float *part_split;              // [splits][Td, d] partial shared-expert outputs of the tcgen05 decode kernel
     int n_sms, max_smem_optin;
     TcBuffers tcb;                  // tensor-core path buffers (large batches)
@@ -110,8 +110,10 @@ void carve(spice_ctx *c, char *base, size_t *total) {
         c->tcb.act_shared16 = cv.take<__nv_bfloat16>(Tm * g.inter_shared);
         c->tcb.mtiles = cv.take<MTile>(n / 128 + (g.n_slots > g.n_experts ? g.n_slots : g.n_experts) + 2);   // hit groups, later LOW groups
         c->tcb.mtiles_shared = cv.take<MTile>(Tm / 128 + 1);
+        c->tcb.mtiles_low = cv.take<MTile>(n / 128 + g.n_experts + 2);
         c->tcb.n_mtiles = cv.take<int32_t>(4);
         c->tcb.n_mtiles_shared = cv.take<int32_t>(4);
+        c->tcb.n_mtiles_low = cv.take<int32_t>(4);
     }
     *total = (cv.off + 255) & ~size_t(255);
 }
@@ -223,17 +225,19 @@ spice_status spice_create(spice_ctx **out, int32_t device, const spice_layer_cfg
     c->tcb = TcBuffers{};
     c->tc_ok = tc_available() && tc_prepare() == 0;
     c->side = nullptr;
-    c->ev_fork = c->ev_join = nullptr;
+    c->ev_fork = c->ev_join = c->ev_grouped = nullptr;
     if (c->tc_ok) {
         if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+            cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_grouped, cudaEventDisableTiming) != cudaSuccess) {
             cudaGetLastError();
             if (c->side) cudaStreamDestroy(c->side);
             if (c->ev_fork) cudaEventDestroy(c->ev_fork);
             if (c->ev_join) cudaEventDestroy(c->ev_join);
+            if (c->ev_grouped) cudaEventDestroy(c->ev_grouped);
             c->side = nullptr;
-            c->ev_fork = c->ev_join = nullptr;
+            c->ev_fork = c->ev_join = c->ev_grouped = nullptr;
         }
     }
     c->dtc_tokens = (coop && c->tc_ok && decode_tc_prepare(c->max_smem_optin) == 0) ? (max_tokens < 64 ? max_tokens : 64) : 0;
@@ -262,6 +266,7 @@ spice_status spice_destroy(spice_ctx *ctx) {
         cudaStreamDestroy(ctx->side);
         cudaEventDestroy(ctx->ev_fork);
         cudaEventDestroy(ctx->ev_join);
+        cudaEventDestroy(ctx->ev_grouped);
     }
     delete ctx;
     return e == cudaSuccess ? SPICE_OK : SPICE_ERR_CUDA;
@@ -548,7 +553,6 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         if (ctx->side && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
             cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess) {
             SPICE_LAUNCH(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ctx->side));
-            if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return SPICE_ERR_CUDA;
             forked = true;
         } else {
             cudaGetLastError();
@@ -569,15 +573,23 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     if (tc_path) {
         // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
         // LoRE on the general kernels
+        // the LoRE groups need the grouping, not the routed experts: on the side stream they run beside the routed GEMMs
+        cudaStream_t ls = st;
+        if (forked) {
+            if (cudaEventRecord(ctx->ev_grouped, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_grouped, 0) != cudaSuccess)
+                return SPICE_ERR_CUDA;
+            ls = ctx->side;
+        }
         SPICE_LAUNCH(launch_tc_routed(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
         if (!forked) SPICE_LAUNCH(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
         if (tc_lore_ok(dm)) {
-            SPICE_LAUNCH(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
-            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 1, st));
+            SPICE_LAUNCH(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ls));
+            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 1, ls));
         } else {
-            SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
-            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 0, st));
+            SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, ls));
+            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 0, ls));
         }
+        if (forked && cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return SPICE_ERR_CUDA;   // (after whatever ran there)
     } else {
         SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED | KIND_HIT, *w, hb, ctx->tb, st));
         SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));

@@ -166,8 +166,8 @@ struct TcBuffers {
     __nv_bfloat16 *x_perm;        // [Tm*K, d]   tokens gathered in perm_hit order
     __nv_bfloat16 *act16;         // [Tm*K, I]   silu(gate)*up of HIT entries
     __nv_bfloat16 *act_shared16;  // [Tm, I_s]
-    MTile *mtiles, *mtiles_shared;
-    int32_t *n_mtiles, *n_mtiles_shared;
+    MTile *mtiles, *mtiles_shared, *mtiles_low;   // tile lists: routed (also the router's), shared expert, LOW groups
+    int32_t *n_mtiles, *n_mtiles_shared, *n_mtiles_low;
 };
 bool tc_available();
 int tc_prepare();

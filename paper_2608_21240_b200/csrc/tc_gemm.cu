@@ -443,10 +443,14 @@ __global__ void build_low_mtiles_kernel(const GroupDesc *__restrict__ groups, co
 
 bool tc_lore_ok(const Dims &dm) { return tc_shape_ok(dm) && dm.r <= BN2 && dm.r % 8 == 0; }
 
-int launch_tc_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb, const TcBuffers &b,
+int launch_tc_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb, const TcBuffers &b0,
                      int n_sms, cudaStream_t st) {
     CUtensorMap ma, mb;
     const size_t cap = (size_t)dm.T * dm.K;
+    // (a tile list of its own: on the side stream the routed GEMMs may be reading theirs at the same time)
+    TcBuffers b = b0;
+    b.mtiles = b0.mtiles_low;
+    b.n_mtiles = b0.n_mtiles_low;
     build_low_mtiles_kernel<<<1, 32, 0, st>>>(tb.groups, tb.hdr, b.mtiles, b.n_mtiles);
     gather_low_rows_kernel<<<n_sms * 2, 256, 0, st>>>(h, tb.perm_low, tb.hdr, dm.K, dm.d, b.x_perm);
     if (!make_map(&ma, b.x_perm, cap, dm.d, BM) || !make_map(&mb, w.lore_A, (uint64_t)dm.N * dm.r, dm.d, 128)) return -1;
