@@ -467,8 +467,12 @@ spice_status spice_grouped_expert_ffn(spice_ctx *ctx, const spice_layer_weights 
     const Dims dm = dims_of(ctx, T);
     const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, slot, ctx->tb, st, &ctx->gsc));
-    SPICE_LAUNCH(launch_gateup(dm, KIND_HIT, *w, hb, ctx->tb, st));
-    SPICE_LAUNCH(launch_down(dm, KIND_HIT, *w, ctx->tb, st));
+    if (T > 64 && ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm)) {
+        SPICE_LAUNCH(launch_tc_routed(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));   // grouped GEMM on the tensor cores
+    } else {
+        SPICE_LAUNCH(launch_gateup(dm, KIND_HIT, *w, hb, ctx->tb, st));
+        SPICE_LAUNCH(launch_down(dm, KIND_HIT, *w, ctx->tb, st));
+    }
     CombineArgs ca{KIND_HIT, 1, gate, cls, y, nullptr, nullptr, nullptr};
     SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));
     return SPICE_OK;
@@ -487,9 +491,15 @@ spice_status spice_lore_surrogate(spice_ctx *ctx, const spice_layer_weights *w, 
     const __nv_bfloat16 *hb = reinterpret_cast<const __nv_bfloat16 *>(h);
     // no slot array: HIT entries are left out of the grouping
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, nullptr, ctx->tb, st, &ctx->gsc));
-    SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED, *w, hb, ctx->tb, st));
-    SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
-    SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_LOW, *w, ctx->tb, st));
+    if (T > 64 && ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm) && tc_lore_ok(dm)) {
+        SPICE_LAUNCH(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        SPICE_LAUNCH(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 1, st));
+    } else {
+        SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED, *w, hb, ctx->tb, st));
+        SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
+        SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_LOW, *w, ctx->tb, st));
+    }
     CombineArgs ca{KIND_SHARED | KIND_LOW, 1, gate, cls, y, nullptr, nullptr, nullptr};
     SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));
     return SPICE_OK;
