@@ -470,11 +470,13 @@ def test_batch_independence_and_repeatability():
     L.close()
 
 
-def test_layer_calls_replay_from_a_cuda_graph():
-    """Three layer calls (fused decode kernel, residual stream updated in place) captured into one CUDA graph and replayed:
-    same bits as the eager calls.  The calls make no host synchronisation and take every pointer at call time."""
-    s = W.SHAPES["dsv2lite"]
-    T = 8
+@pytest.mark.parametrize("name,T", [("dsv2lite", 8), ("tiny", 150)])
+def test_layer_calls_replay_from_a_cuda_graph(name, T):
+    """Three layer calls (residual stream updated in place) captured into one CUDA graph and replayed: same bits as the
+    eager calls.  The calls make no host synchronisation and take every pointer at call time.  Batch 8: the fused decode
+    kernel.  Batch 150: the large-batch path, whose shared expert and LoRE groups run on the context's side stream
+    (the fork and the join are captured as edges of the graph)."""
+    s = W.SHAPES[name]
     wls = [W.make_layer(s, T, variant=200 + i) for i in range(3)]
     ws = [upload(wl) for wl in wls]
     structs = [w.c_struct() for w in ws]
