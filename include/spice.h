@@ -18,6 +18,9 @@
  *     and return without synchronising (spice_moe_layer_fwd can therefore be captured into a CUDA
  *     graph; pointers are baked in at capture time).  The library allocates device memory only in
  *     spice_create; per call it allocates nothing.  A ctx must not be used by two streams at once.
+ *     For batches above 64 tokens spice_moe_layer_fwd runs the shared expert and the LoRE groups on a
+ *     stream the ctx owns, forked from and joined back to `stream` by events inside the call: the
+ *     caller sees stream order, and a capture of `stream` takes the fork in as edges of the graph.
  *   - Errors found on the host return a code and launch nothing.  Conditions found on the device
  *     (expert id out of range, slot index >= n_slots, an expired bounded wait) never trap: the
  *     entry is treated as an exact-recovery miss or skipped, a status word is set, and
