@@ -6,7 +6,8 @@ resident slots, shared expert + LoRE surrogate, combine) over one decode batch o
 DeepSeek-V2-Lite-shaped layer.  Successive steps rotate through several independent
 layer weight sets so that the bytes touched between two uses of the same weights are
 several times the L2 capacity (cold-L2 timing without a flush inside the timed region).
-The timed steps are submitted as replayed CUDA graphs of captured steps (--launch eager: one call per step).
+Decode steps are submitted as replayed CUDA graphs of captured steps (--launch eager: one call per step); batches above
+64 tokens, a dozen kernels on two streams per step, as one library call per step.
 
 Prints ONE JSON line: metric, value, unit, timing, `config` (the workload), `roofline` (algorithmic bytes or FLOPs of
 the timed calls over their time, against the measured peak), `e2e` (the same metric with host<->device copies inside
@@ -217,7 +218,8 @@ def run_ours(args):
     l0 = layer.launch_count()
     step(0)
     launches_per_step = layer.launch_count() - l0
-    ms, how, w0, w1 = timed_steps(torch, step, args.steps, args.launch)
+    launch = args.launch if args.launch != "auto" else ("eager" if prefill else "graph")
+    ms, how, w0, w1 = timed_steps(torch, step, args.steps, launch)
     if world > 1:
         dist.barrier()
     launches = launches_per_step * args.steps
@@ -448,7 +450,7 @@ def run_stack(args):
     l0 = layer.launch_count()
     step()
     launches_per_step = layer.launch_count() - l0
-    ms, how, w0, w1 = timed_steps(torch, lambda i: step(), args.steps, args.launch)
+    ms, how, w0, w1 = timed_steps(torch, lambda i: step(), args.steps, "eager" if args.launch == "eager" else "graph")
     if world > 1:
         dist.barrier()
     launches = launches_per_step * args.steps
@@ -750,8 +752,10 @@ def main():
                     help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
     ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout", "lore_calibrate"],
                     help="what a step is: the MoE layer call (default) or the draft-router confidence call")
-    ap.add_argument("--launch", default="graph", choices=["graph", "eager"],
-                    help="how the timed steps are submitted: replayed CUDA graphs of captured steps (default) or one call per step")
+    ap.add_argument("--launch", default="auto", choices=["auto", "graph", "eager"],
+                    help="how the timed steps are submitted: replayed CUDA graphs of captured steps, or one library call per "
+                         "step; auto = graphs for decode batches (one kernel per step, launch-bound), calls for batches "
+                         "above 64 tokens (a dozen kernels on two streams per step)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
