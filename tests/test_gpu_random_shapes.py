@@ -44,3 +44,46 @@ def test_fused_and_general_paths_agree_on_random_shapes(seed):
         assert (ya - yb).abs().max().item() <= 2e-2 * yb.abs().max().item() + 2e-3, tag
         L.close()
     assert fused_seen >= 6      # most of these shapes are taken by a fused kernel
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_large_batch_and_general_paths_agree_on_random_shapes(seed):
+    """The same for batches above 64 tokens: tensor-core path (router logits, grouped GEMMs, shared expert and LoRE
+    groups on the side stream, lore_b_kernel) against the general-shape kernels.  The draws include expert counts that
+    are not multiples of 4 (fp32 router instead of the GEMM), LoRE ranks above 256 (general LoRE kernels inside the
+    tensor-core path), empty residencies (no hit group) and every expert resident (no LoRE group).  Top-k sets are
+    compared only where the two routers' logits cannot disagree: tokens whose K-th and (K+1)-th logits are closer than
+    1e-4 are left out (the inputs of these shapes are not margin-enforced)."""
+    rng = np.random.default_rng(2000 + seed)
+    base = W.SHAPES["tiny"]
+    for it in range(8):
+        d = int(rng.choice([64, 128, 320, 512, 1024]))
+        N = int(rng.choice([6, 17, 32, 64, 100]))
+        K = int(rng.integers(1, min(N, 8) + 1))
+        s = W.scaled_shape(base, d=d, n_experts=N, top_k=K, inter=int(rng.choice([64, 192, 448])),
+                           inter_shared=int(rng.choice([64, 256, 576])), lore_rank=int(rng.choice([8, 24, 64, 72, 264])),
+                           n_slots=int(rng.integers(1, N + 1)), norm_topk=int(rng.integers(0, 2)))
+        T = int(rng.integers(65, 700))
+        n_res = int(rng.choice([0, s.n_slots, int(rng.integers(0, s.n_slots + 1))]))
+        wl = W.make_layer(s, T, variant=7000 + 100 * seed + it, n_resident=n_res)
+        w = B.upload(wl)
+        L = B.SpiceLayer(B.cfg_of(s), T)
+        h, conf = B.bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+        a = L.moe_layer_fwd(w, h, conf)
+        torch.cuda.synchronize()
+        assert L.device_status() == 0
+        L.set_option(B.OPT_PATH, 1)
+        b = L.moe_layer_fwd(w, h, conf)
+        torch.cuda.synchronize()
+        tag = f"shape {s.d},{s.n_experts},{s.top_k},{s.inter},{s.inter_shared},{s.lore_rank},{s.n_slots} T={T} res={n_res}"
+        logits = torch.from_numpy(wl.h.astype(np.float64) @ wl.w_router.astype(np.float64).T)
+        top = torch.sort(logits, dim=1, descending=True).values
+        clear = ((top[:, K - 1] - top[:, K]).abs() > 1e-4) if K < N else torch.ones(T, dtype=torch.bool)
+        clear = clear.cuda()
+        assert int(clear.sum()) >= 0.95 * T, tag
+        assert torch.equal(a.idx[clear], b.idx[clear]) and torch.equal(a.cls[clear], b.cls[clear]), tag
+        assert (a.gate[clear] - b.gate[clear]).abs().max().item() <= 7e-5, tag
+        ya, yb = a.y.float()[clear], b.y.float()[clear]
+        assert bool(torch.isfinite(a.y.float()).all()), tag
+        assert (ya - yb).abs().max().item() <= 2e-2 * yb.abs().max().item() + 2e-3, tag
+        L.close()
