@@ -581,8 +581,8 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
                                  ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st, &ctx->gsc));
     SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st, &ctx->gsc));
     if (tc_path) {
-        // batches the decode kernel does not take: exact experts and shared expert on the tensor cores,
-        // LoRE on the general kernels
+        // batches the decode kernel does not take: exact experts, shared expert and LoRE down-projection on the
+        // tensor cores (grouped GEMM kernel), LoRE up-projection on lore_b_kernel
         // the LoRE groups need the grouping, not the routed experts: on the side stream they run beside the routed GEMMs
         cudaStream_t ls = st;
         if (forked) {
