@@ -173,12 +173,13 @@ def run_ours(args):
     # replica 0 comes from the numpy generator (the CPU baseline needs the same numbers);
     # the others are drawn on the device with the same distributions
     prefill = T > 64   # large batch: the grouped GEMM is tensor-bound; use the skewed (Zipf) router of config 4
-    wl0 = W.make_layer(shape, T, variant=100 + rank, zipf=prefill)
+    zipf = prefill if args.router == "auto" else args.router == "zipf"
+    wl0 = W.make_layer(shape, T, variant=100 + rank, zipf=zipf)
     upload, bf16_tensor, cfg_of = B.upload, B.bf16_tensor, B.cfg_of
     gen = torch.Generator(device=dev)
     gen.manual_seed(W.BASE_SEED + 1000 * rank)
     reps = [upload(wl0, dev)] + [device_replica(torch, B, shape, gen, dev) for _ in range(R - 1)]
-    if prefill:
+    if zipf:
         for r in reps[1:]:
             r.w_router.copy_(reps[0].w_router)   # same popularity skew in every weight set
     structs = [r.c_struct() for r in reps]
@@ -775,6 +776,9 @@ def main():
                     help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
     ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout", "lore_calibrate"],
                     help="what a step is: the MoE layer call (default) or the draft-router confidence call")
+    ap.add_argument("--router", default="auto", choices=["auto", "uniform", "zipf"],
+                    help="router of the synthetic layer: i.i.d. weights (uniform loads) or the Zipf-skewed one of config 4; "
+                         "auto = uniform for decode batches, zipf above 64 tokens")
     ap.add_argument("--launch", default="auto", choices=["auto", "graph", "eager"],
                     help="how the timed steps are submitted: replayed CUDA graphs of captured steps, or one library call per "
                          "step; auto = graphs for decode batches (one kernel per step, launch-bound), calls for batches "
