@@ -7,7 +7,8 @@
 //     G = L L^T,  Z = L^-1 C                   (then the fitted values satisfy  Yhat^T Yhat = Z^T Z)
 //     V = r leading eigenvectors of Z^T Z      block subspace iteration, orthonormalised by Cholesky QR (twice)
 //     B = V,   A = ( L^-T Z V )^T = ( W V )^T  with W = G^-1 C the least-squares map
-// Everything is dense fp32 linear algebra on d x d matrices built from tiled SGEMMs, 64 x 64 Cholesky /
+// Everything is dense fp32 linear algebra on d x d matrices built from tiled SGEMMs (split over the reduction,
+// with the slices summed in a fixed order, where a product has too few output tiles to fill the GPU), 64 x 64 Cholesky /
 // triangular-solve blocks and a few element-wise kernels, launched in order on one stream; nothing synchronises
 // with the host.  The caller provides the workspace (spice_lore_calibrate_workspace_bytes).
 #include "spice_internal.cuh"
@@ -25,7 +26,7 @@ __host__ __device__ inline int pad64(int v) { return (v + 63) / 64 * 64; }
 template <bool TA, bool TB_>
 __global__ void __launch_bounds__(256) sgemm_kernel(int M, int N, int K, float alpha, const float *__restrict__ A, int lda,
                                                     const float *__restrict__ B, int ldb, float beta, float *__restrict__ C,
-                                                    int ldc) {
+                                                    int ldc, int kchunk, float *__restrict__ part) {
     __shared__ float As[BK][TB + 4], Bs[BK][TB + 4];
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int m0 = blockIdx.y * TB, n0 = blockIdx.x * TB;
@@ -34,7 +35,11 @@ __global__ void __launch_bounds__(256) sgemm_kernel(int M, int N, int K, float a
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-    for (int k0 = 0; k0 < K; k0 += BK) {
+    // blockIdx.z takes the reduction range [z kchunk, (z+1) kchunk): products with few output tiles are split over
+    // the reduction so that they fill the machine; the slices are summed in z order by splitk_reduce_kernel
+    const int kb = blockIdx.z * kchunk;
+    K = min(K, kb + kchunk);
+    for (int k0 = kb; k0 < K; k0 += BK) {
         for (int e = threadIdx.x; e < BK * TB; e += 256) {
             int kk, mm;
             if (TA) { kk = e / TB; mm = e % TB; } else { mm = e / BK; kk = e % BK; }
@@ -66,19 +71,51 @@ __global__ void __launch_bounds__(256) sgemm_kernel(int M, int N, int K, float a
         for (int j = 0; j < 4; ++j) {
             const int gm = m0 + ty * 4 + i, gn = n0 + tx * 4 + j;
             if (gm < M && gn < N) {
-                float *c = C + (size_t)gm * ldc + gn;
-                *c = alpha * acc[i][j] + (beta != 0.f ? beta * *c : 0.f);
+                if (part) {
+                    part[((size_t)blockIdx.z * M + gm) * N + gn] = acc[i][j];
+                } else {
+                    float *c = C + (size_t)gm * ldc + gn;
+                    *c = alpha * acc[i][j] + (beta != 0.f ? beta * *c : 0.f);
+                }
             }
         }
 }
+
+// C = alpha * (sum over the nz slices of part, in slice order) + beta * C
+__global__ void splitk_reduce_kernel(int M, int N, int nz, float alpha, const float *__restrict__ part, float beta,
+                                     float *__restrict__ C, int ldc) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)M * N) return;
+    float s = 0.f;
+    for (int z = 0; z < nz; ++z) s += part[(size_t)z * M * N + i];
+    float *c = C + (i / N) * (size_t)ldc + (i % N);
+    *c = alpha * s + (beta != 0.f ? beta * *c : 0.f);
+}
+
+// scratch for the split products (set by launch_lore_calibrate for the duration of a call)
+thread_local float *t_splitk_ws = nullptr;
+thread_local size_t t_splitk_floats = 0;
 
 template <bool TA, bool TB_>
 int gemm(int M, int N, int K, float alpha, const float *A, int lda, const float *B, int ldb, float beta, float *C, int ldc,
          cudaStream_t st) {
     if (M <= 0 || N <= 0) return 0;
     dim3 grid((N + TB - 1) / TB, (M + TB - 1) / TB);
-    sgemm_kernel<TA, TB_><<<grid, 256, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    const int tiles = (int)(grid.x * grid.y);
+    int nz = 1;
+    if (t_splitk_ws && tiles < 74 && K >= 512) {
+        nz = min(min(148 / tiles, K / 256), 32);
+        while (nz > 1 && (size_t)nz * M * N > t_splitk_floats) --nz;
+    }
+    if (nz <= 1) {
+        sgemm_kernel<TA, TB_><<<grid, 256, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, K, nullptr);
+        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    }
+    const int kchunk = ((K + nz - 1) / nz + BK - 1) / BK * BK;
+    grid.z = (K + kchunk - 1) / kchunk;
+    sgemm_kernel<TA, TB_><<<grid, 256, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, kchunk, t_splitk_ws);
+    splitk_reduce_kernel<<<(unsigned)(((size_t)M * N + 255) / 256), 256, 0, st>>>(M, N, (int)grid.z, alpha, t_splitk_ws, beta, C, ldc);
+    return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
 // bf16 [rows, cols] -> fp32 [rows, ld] with zero columns cols..ld-1
@@ -326,6 +363,7 @@ size_t lore_calibrate_workspace_bytes(int d, int n, int r) {
     const size_t dp = pad64(d), rp = pad64(r);
     // H32 / T2 [n, dp], G [dp, dp], C [dp, dp], Q, P, Y [dp, rp] each, S [rp, rp], T1 [n, rp], A32 [rp, dp], B32 [dp, rp], scalars
     size_t f = (size_t)n * dp + 2 * dp * dp + 3 * dp * rp + rp * rp + (size_t)n * rp + 2 * dp * rp + 64;
+    f += 8 * dp * rp;   // slices of the products that are split over their reduction
     return f * sizeof(float) + 256;
 }
 
@@ -345,7 +383,9 @@ int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __n
     float *T1 = w;                       w += (size_t)n * rp;
     float *A32 = w;                      w += (size_t)rp * dp;
     float *B32 = w;                      w += (size_t)dp * rp;
-    float *scal = w;
+    float *scal = w;                     w += 64;
+    t_splitk_ws = w;
+    t_splitk_floats = (size_t)8 * dp * rp;
     int32_t *qr_flag = reinterpret_cast<int32_t *>(scal + 8);   // pivots clamped inside the Cholesky QR are not an error
     if (cudaMemsetAsync(flag, 0, sizeof(int32_t), st) != cudaSuccess) return -1;
     widen_pad_kernel<<<(unsigned)(((size_t)n * dp + 255) / 256), 256, 0, st>>>(h_cal, n, d, H32, dp);
@@ -401,6 +441,7 @@ int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __n
         loss_kernel<<<512, 256, 0, st>>>(resid, d, H32, dp, n, d, loss_out);
         CKL();
     }
+    t_splitk_ws = nullptr;
     return launches;
 }
 
