@@ -152,13 +152,15 @@ __global__ void regularise_kernel(float *G, int ld, int d, int dp, float ridge, 
 
 // Cholesky of one 64 x 64 diagonal block in place (lower triangle; the strict upper triangle is zeroed).
 // A pivot that is not positive is replaced by a tiny positive number and flagged.
-__global__ void __launch_bounds__(64) potrf64_kernel(float *A, int ld, int32_t *flag) {
+__global__ void __launch_bounds__(256) potrf64_kernel(float *A, int ld, int32_t *flag) {
     __shared__ float a[TB][TB + 1];
-    const int t = threadIdx.x;
-    for (int r = 0; r < TB; ++r) a[r][t] = A[(size_t)r * ld + t];
+    // 256 threads: thread (t, part) owns row t and the columns c = part (mod 4) of the trailing update
+    const int t = threadIdx.x & 63, part = threadIdx.x >> 6;
+#pragma unroll 4
+    for (int r = part; r < TB; r += 4) a[r][t] = A[(size_t)r * ld + t];
     __syncthreads();
     for (int j = 0; j < TB; ++j) {
-        if (t == j) {
+        if (threadIdx.x == j) {
             float p = a[j][j];
             if (!(p > 0.f)) {
                 p = 1e-20f;
@@ -168,22 +170,24 @@ __global__ void __launch_bounds__(64) potrf64_kernel(float *A, int ld, int32_t *
         }
         __syncthreads();
         const float piv = a[j][j];
-        if (t > j) a[t][j] /= piv;
+        if (part == 0 && t > j) a[t][j] /= piv;
         __syncthreads();
         // trailing update: row t, columns j+1 .. t
         if (t > j) {
             const float ltj = a[t][j];
-            for (int c = j + 1; c <= t; ++c) a[t][c] -= ltj * a[c][j];
+            for (int c = j + 1 + ((part - (j + 1)) & 3); c <= t; c += 4) a[t][c] -= ltj * a[c][j];
         }
         __syncthreads();
     }
-    for (int r = 0; r < TB; ++r) A[(size_t)r * ld + t] = t <= r ? a[r][t] : 0.f;
+#pragma unroll 4
+    for (int r = part; r < TB; r += 4) A[(size_t)r * ld + t] = t <= r ? a[r][t] : 0.f;
 }
 
 // X <- X L^-T for a panel of rows (one CTA of 64 threads takes 64 rows): X [rows, 64] (ldx), L 64 x 64 lower (ldl)
 __global__ void __launch_bounds__(64) trsm_right_lt_kernel(float *X, int ldx, int rows, const float *__restrict__ L, int ldl) {
     __shared__ float l[TB][TB + 1];
     const int t = threadIdx.x;
+#pragma unroll 8
     for (int r = 0; r < TB; ++r) l[r][t] = L[(size_t)r * ldl + t];
     __syncthreads();
     const int row = blockIdx.x * TB + t;
@@ -191,10 +195,11 @@ __global__ void __launch_bounds__(64) trsm_right_lt_kernel(float *X, int ldx, in
     float x[TB];
 #pragma unroll
     for (int c = 0; c < TB; ++c) x[c] = X[(size_t)row * ldx + c];
-    // solve y L^T = x: y_c = (x_c - sum_{q<c} y_q L[c][q]) / L[c][c]
-#pragma unroll 1
+    // solve y L^T = x: y_c = (x_c - sum_{q<c} y_q L[c][q]) / L[c][c]   (fully unrolled: x stays in registers)
+#pragma unroll
     for (int c = 0; c < TB; ++c) {
         float s = x[c];
+#pragma unroll
         for (int qq = 0; qq < c; ++qq) s -= x[qq] * l[c][qq];
         x[c] = s / l[c][c];
     }
@@ -319,7 +324,7 @@ int cholesky(float *G, int ld, int np, int32_t *flag, cudaStream_t st) {
     int launches = 0;
     for (int k = 0; k < np; k += TB) {
         float *diag = G + (size_t)k * ld + k;
-        potrf64_kernel<<<1, 64, 0, st>>>(diag, ld, flag);
+        potrf64_kernel<<<1, 256, 0, st>>>(diag, ld, flag);
         CKL();
         const int rem = np - k - TB;
         if (rem > 0) {
