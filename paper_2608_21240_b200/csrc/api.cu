@@ -577,9 +577,8 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         SPICE_LAUNCH(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
                                        gate, nullptr, st));
     }
-    SPICE_LAUNCH(launch_classify(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
-                                 ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb.status, st, &ctx->gsc));
-    SPICE_LAUNCH(launch_group(dm, idx, gate, cls, ctx->ws_slot, ctx->tb, st, &ctx->gsc));
+    SPICE_LAUNCH(launch_classify_group(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
+                                       ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb, st, &ctx->gsc));
     if (tc_path) {
         // batches the decode kernel does not take: exact experts, shared expert and LoRE down-projection on the
         // tensor cores (grouped GEMM kernel), LoRE up-projection on lore_b_kernel

@@ -38,14 +38,14 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_tot /* [33]
     return warp_tot[warp] + inc - v;
 }
 
-__global__ void __launch_bounds__(CT) classify_kernel(int T, int N, int K, int S, int conf_stride, float tau,
-                                                      const int32_t *__restrict__ idx, const float *__restrict__ gate,
-                                                      const int32_t *__restrict__ slot_of_expert,
-                                                      const float *__restrict__ conf, uint8_t *__restrict__ cls,
-                                                      int32_t *__restrict__ slot, int32_t *__restrict__ counts,
-                                                      int32_t *__restrict__ resid_tok, int32_t *__restrict__ resid_k,
-                                                      int32_t *__restrict__ resid_expert,
-                                                      float *__restrict__ resid_gate, int32_t *__restrict__ status) {
+// (cls and slot carry no __restrict__: the fused kernel below reads them back after a barrier)
+__device__ __forceinline__ void classify_body(int T, int N, int K, int S, int conf_stride, float tau,
+                                              const int32_t *__restrict__ idx, const float *__restrict__ gate,
+                                              const int32_t *__restrict__ slot_of_expert, const float *__restrict__ conf,
+                                              uint8_t *cls, int32_t *slot, int32_t *__restrict__ counts,
+                                              int32_t *__restrict__ resid_tok, int32_t *__restrict__ resid_k,
+                                              int32_t *__restrict__ resid_expert, float *__restrict__ resid_gate,
+                                              int32_t *__restrict__ status) {
     __shared__ int warp_tot[33];
     __shared__ int s_cnt[3];
     if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0;
@@ -94,6 +94,18 @@ __global__ void __launch_bounds__(CT) classify_kernel(int T, int N, int K, int S
     if (threadIdx.x < 3) counts[threadIdx.x] = s_cnt[threadIdx.x];
 }
 
+__global__ void __launch_bounds__(CT) classify_kernel(int T, int N, int K, int S, int conf_stride, float tau,
+                                                      const int32_t *__restrict__ idx, const float *__restrict__ gate,
+                                                      const int32_t *__restrict__ slot_of_expert,
+                                                      const float *__restrict__ conf, uint8_t *__restrict__ cls,
+                                                      int32_t *__restrict__ slot, int32_t *__restrict__ counts,
+                                                      int32_t *__restrict__ resid_tok, int32_t *__restrict__ resid_k,
+                                                      int32_t *__restrict__ resid_expert,
+                                                      float *__restrict__ resid_gate, int32_t *__restrict__ status) {
+    classify_body(T, N, K, S, conf_stride, tau, idx, gate, slot_of_expert, conf, cls, slot, counts, resid_tok, resid_k,
+                  resid_expert, resid_gate, status);
+}
+
 // Builds, from cls / slot / idx / gate:
 //   groups[0] = shared expert (m = T); then one group per slot with >= 1 HIT entry (slot order);
 //   then one group per expert with >= 1 LOWCONF entry (expert order);
@@ -102,9 +114,8 @@ __global__ void __launch_bounds__(CT) classify_kernel(int T, int N, int K, int S
 // Positions inside a group are handed out by warp-aggregated shared-memory atomics; the order of
 // entries inside a group is therefore not fixed, which no result depends on (every entry's row is
 // computed independently and the combine step gathers by entry id).
-__global__ void __launch_bounds__(CT) group_kernel(int T, int N, int K, int S, const int32_t *__restrict__ idx,
-                                                   const float *__restrict__ gate, const uint8_t *__restrict__ cls,
-                                                   const int32_t *__restrict__ slot, Tables tb) {
+__device__ __forceinline__ void group_body(int T, int N, int K, int S, const int32_t *__restrict__ idx,
+                                           const float *__restrict__ gate, const uint8_t *cls, const int32_t *slot, Tables tb) {
     __shared__ int warp_tot[33];
     __shared__ int cnt_hit[1024], cnt_low[1024];   // later reused as cursors
     __shared__ int off_hit[1024], off_low[1024];
@@ -188,6 +199,27 @@ __global__ void __launch_bounds__(CT) group_kernel(int T, int N, int K, int S, c
             if (cls[t * K + k] == SPICE_LOWCONF) c += gate[t * K + k];
         tb.coef_shared[t] = c;
     }
+}
+
+__global__ void __launch_bounds__(CT) group_kernel(int T, int N, int K, int S, const int32_t *__restrict__ idx,
+                                                   const float *__restrict__ gate, const uint8_t *__restrict__ cls,
+                                                   const int32_t *__restrict__ slot, Tables tb) {
+    group_body(T, N, K, S, idx, gate, cls, slot, tb);
+}
+
+// Both steps in one launch for batches whose tables one CTA builds: classification, a barrier (the classes and slots
+// it wrote are read back by the same CTA), grouping.
+__global__ void __launch_bounds__(CT) classify_group_kernel(int T, int N, int K, int S, int conf_stride, float tau,
+                                                            const int32_t *__restrict__ idx, const float *__restrict__ gate,
+                                                            const int32_t *__restrict__ slot_of_expert,
+                                                            const float *__restrict__ conf, uint8_t *cls, int32_t *slot,
+                                                            int32_t *__restrict__ counts, int32_t *__restrict__ resid_tok,
+                                                            int32_t *__restrict__ resid_k, int32_t *__restrict__ resid_expert,
+                                                            float *__restrict__ resid_gate, int32_t *__restrict__ status, Tables tb) {
+    classify_body(T, N, K, S, conf_stride, tau, idx, gate, slot_of_expert, conf, cls, slot, counts, resid_tok, resid_k,
+                  resid_expert, resid_gate, status);
+    __syncthreads();
+    group_body(T, N, K, S, idx, gate, cls, slot, tb);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -363,6 +395,22 @@ int launch_classify(const Dims &dm, int conf_stride, float tau, const int32_t *i
     }
     classify_kernel<<<1, CT, 0, st>>>(dm.T, dm.N, dm.K, dm.S, conf_stride, tau, idx, gate, slot_of_expert, conf, cls,
                                       slot, counts, resid_tok, resid_k, resid_expert, resid_gate, status);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_classify_group(const Dims &dm, int conf_stride, float tau, const int32_t *idx, const float *gate,
+                          const int32_t *slot_of_expert, const float *conf, uint8_t *cls, int32_t *slot, int32_t *counts,
+                          int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert, float *resid_gate, const Tables &tb,
+                          cudaStream_t st, const GroupScratch *scratch) {
+    if (dm.T * dm.K > MC_ENTRIES) {
+        const int a = launch_classify(dm, conf_stride, tau, idx, gate, slot_of_expert, conf, cls, slot, counts, resid_tok, resid_k,
+                                      resid_expert, resid_gate, tb.status, st, scratch);
+        if (a < 0) return -1;
+        const int b = launch_group(dm, idx, gate, cls, slot, tb, st, scratch);
+        return b < 0 ? -1 : a + b;
+    }
+    classify_group_kernel<<<1, CT, 0, st>>>(dm.T, dm.N, dm.K, dm.S, conf_stride, tau, idx, gate, slot_of_expert, conf, cls, slot,
+                                            counts, resid_tok, resid_k, resid_expert, resid_gate, tb.status, tb);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -67,6 +67,12 @@ int launch_classify(const Dims &dm, int conf_stride, float tau, const int32_t *i
 int launch_group(const Dims &dm, const int32_t *idx, const float *gate, const uint8_t *cls,
                  const int32_t *slot, const Tables &tb, cudaStream_t st, const GroupScratch *scratch = nullptr);
 
+// classification and grouping of one call: one launch while a single CTA builds the tables, else the launches above
+int launch_classify_group(const Dims &dm, int conf_stride, float tau, const int32_t *idx, const float *gate,
+                          const int32_t *slot_of_expert, const float *conf, uint8_t *cls, int32_t *slot, int32_t *counts,
+                          int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert, float *resid_gate, const Tables &tb,
+                          cudaStream_t st, const GroupScratch *scratch = nullptr);
+
 // Reference ("v1") expert path: warp-per-row GEMV kernels for any shape.
 int launch_gateup(const Dims &dm, int kind_mask, const spice_layer_weights &w, const __nv_bfloat16 *h,
                   const Tables &tb, cudaStream_t st);
