@@ -134,10 +134,16 @@ def lore_calibrate(H, R, rank: int, ridge: float = 0.0):
 
 
 def _round_bf16(x: np.ndarray) -> np.ndarray:
-    """Nearest bf16 (ties to even) of fp64 values, returned as fp64: the draft state is kept in bf16 between depths."""
-    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
-    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
-    return r.view(np.float32).astype(np.float64)
+    """Nearest bf16 (ties to even) of fp64 values, returned as fp64: the draft state is kept in bf16 between depths.
+    A bf16 keeps 8 significant bits, so 45 of the 52 fraction bits of the fp64 pattern are dropped in ONE rounding
+    (no detour over fp32, which would round twice).  Meant for finite values of normal bf16 magnitude (2^-126 .. 3.4e38);
+    zeros keep their sign."""
+    u = np.ascontiguousarray(x, dtype=np.float64).view(np.uint64)
+    drop = np.uint64(45)
+    half_minus_one = np.uint64((1 << 44) - 1)
+    keep_mask = np.uint64(0xFFFFFFFFFFFFFFFF ^ ((1 << 45) - 1))
+    r = (u + half_minus_one + ((u >> drop) & np.uint64(1))) & keep_mask
+    return r.view(np.float64)
 
 
 def prefetch_rollout(x, layers, top_k: int, l_min: int, l_max: int, tau: float):

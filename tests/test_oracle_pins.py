@@ -439,6 +439,44 @@ def test_p14_rollout_fixed_point_when_nothing_is_added():
     assert np.array_equal(h, x) and all(np.array_equal(idx[l], idx[0]) and np.array_equal(conf[l], conf[0]) for l in range(L))
 
 
+def test_p14_rollout_state_rounding_is_nearest_even_bf16():
+    """The bf16 rounding of the draft state between depths, pinned on hand-written values (a bf16 keeps 8 significant
+    bits: the spacing in [1, 2) is 2^-7, so 1 + 2^-8 lies exactly between 1 and 1 + 2^-7).  Truncation fails the
+    round-up rows, round-half-up fails the first tie, round-half-down the second; a detour over fp32 fails the last two
+    rows, which sit within 2^-30 of a tie (fp32 would first round them ONTO the tie)."""
+    f = oracle._round_bf16
+    u = 2.0 ** -7                      # one bf16 step in [1, 2)
+    rows = [
+        (1.0, 1.0),                            # representable
+        (-3.140625, -3.140625),                # representable, negative (-(3 + 9/64): 8 significant bits)
+        (1.0 + 0.5 * u, 1.0),                  # tie, even mantissa below   -> down
+        (1.0 + 1.5 * u, 1.0 + 2 * u),          # tie, even mantissa above   -> up
+        (-(1.0 + 1.5 * u), -(1.0 + 2 * u)),    # the same tie, negative: magnitude rounds, sign kept
+        (1.0 + 0.5 * u + 2.0 ** -20, 1.0 + u),       # just above a tie -> up
+        (1.0 + 0.5 * u - 2.0 ** -20, 1.0),           # just below a tie -> down
+        (1.0 + 0.75 * u, 1.0 + u),             # above half -> up (truncation would give 1)
+        (1.0 + 0.25 * u, 1.0),                 # below half -> down
+        (255.5, 256.0),                        # tie at the top of a binade (255 = 11111111b is odd) carries into the exponent
+        (2.0 ** -100 * (1.0 + 0.75 * u), 2.0 ** -100 * (1.0 + u)),   # the same away from 1
+        (1.0 + 0.5 * u + 2.0 ** -30, 1.0 + u),       # above the tie by less than an fp32 ulp (2^-23): still up
+        (1.0 + 1.5 * u - 2.0 ** -30, 1.0 + u),       # below the tie by less than an fp32 ulp: still down
+    ]
+    x = np.array([a for a, _ in rows], dtype=np.float64)
+    want = np.array([b for _, b in rows], dtype=np.float64)
+    got = f(x)
+    assert got.dtype == np.float64 and np.array_equal(got, want), list(zip(x.tolist(), got.tolist(), want.tolist()))
+    assert np.array_equal(f(got), got)                       # idempotent
+    assert np.signbit(f(np.array([-0.0]))[0]) and f(np.array([0.0]))[0] == 0.0
+    # every result has at most 8 significant bits: scaled to [128, 256) it is an integer
+    rng = np.random.default_rng(141)
+    r = f(rng.standard_normal(1000) * 10.0 ** rng.integers(-3, 4, 1000))
+    m, _ = np.frexp(r)
+    assert np.array_equal(m * 256.0, np.round(m * 256.0))
+    # and it agrees with the generator's fp32 -> bf16 rounding wherever the input is an fp32 value
+    x32 = (rng.standard_normal(1000) * 3.0).astype(np.float32)
+    assert np.array_equal(f(x32.astype(np.float64)), W.bf16_round(x32).astype(np.float64))
+
+
 # ------------------------------------------------------------------ LoRE calibration (Sec. 4.2, the fitting objective)
 def _lore_loss(H, R, A, B):
     return float(((R - (H @ A.T) @ B.T) ** 2).sum())
