@@ -193,10 +193,15 @@ def run_ours(args):
     gate = torch.empty(T, shape.top_k, dtype=torch.float32, device=dev)
     cls = torch.empty(T, shape.top_k, dtype=torch.uint8, device=dev)
     counts = torch.zeros(3, dtype=torch.int32, device=dev)
+    # residual-miss list (set M of Sec. 4.3): part of the call's output, written in the timed region
+    n_ent = T * shape.top_k
+    resid = (torch.empty(n_ent, dtype=torch.int32, device=dev), torch.empty(n_ent, dtype=torch.int32, device=dev),
+             torch.empty(n_ent, dtype=torch.int32, device=dev), torch.empty(n_ent, dtype=torch.float32, device=dev))
     stream = torch.cuda.current_stream()
 
     def step(i):
         B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h, conf, T, y, idx=idx, gate=gate, cls=cls, counts=counts,
+                              resid_tok=resid[0], resid_k=resid[1], resid_expert=resid[2], resid_gate=resid[3],
                               stream=torch.cuda.current_stream())
 
     # algorithmic bytes of every replica's call (from the routing the library itself produced)
@@ -235,17 +240,24 @@ def run_ours(args):
     in_host[h.numel() * 2:].copy_(conf.cpu().view(torch.uint8).reshape(-1))
     h_dev = in_dev[: h.numel() * 2].view(torch.bfloat16).view(T, shape.d)
     conf_dev = in_dev[h.numel() * 2:].view(torch.float32).view_as(conf)
-    out_bytes = T * shape.d * 2 + 16
+    # one device block -> host: y, the class counts, and the residual-miss list (the host runtime needs it to recover
+    # those experts; its capacity T*K is copied, counts[1] entries of it are valid)
+    y_bytes = T * shape.d * 2
+    out_bytes = y_bytes + 16 + 16 * n_ent
     out_dev = torch.empty(out_bytes, dtype=torch.uint8, device=dev)
     out_host = torch.empty(out_bytes, dtype=torch.uint8).pin_memory()
-    y_e2e = out_dev[: T * shape.d * 2].view(torch.bfloat16).view(T, shape.d)
-    cnt_e2e = out_dev[T * shape.d * 2:].view(torch.int32)[:3]
+    y_e2e = out_dev[:y_bytes].view(torch.bfloat16).view(T, shape.d)
+    cnt_e2e = out_dev[y_bytes:y_bytes + 16].view(torch.int32)[:3]
+    r0 = y_bytes + 16
+    resid_e2e = tuple(out_dev[r0 + 4 * n_ent * j: r0 + 4 * n_ent * (j + 1)].view(torch.float32 if j == 3 else torch.int32)
+                      for j in range(4))
 
     def e2e_enqueue(i):
         st = torch.cuda.current_stream()
         in_dev.copy_(in_host, non_blocking=True)
         B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h_dev, conf_dev, T, y_e2e, idx=idx, gate=gate, cls=cls,
-                              counts=cnt_e2e, stream=st)
+                              counts=cnt_e2e, resid_tok=resid_e2e[0], resid_k=resid_e2e[1], resid_expert=resid_e2e[2],
+                              resid_gate=resid_e2e[3], stream=st)
         out_host.copy_(out_dev, non_blocking=True)
 
     # a decode step (copy in, one kernel, copy out) is captured once per weight set and replayed; the host still
@@ -334,6 +346,7 @@ def run_ours(args):
         }
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"] = cpu_baseline(wl0, budget_s=args.cpu_budget)
+            out["cpu_baseline"]["one_thread"] = cpu_baseline_one_thread(args, 100 + rank, min(args.cpu_budget, 10.0))
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -724,6 +737,29 @@ def cpu_baseline(wl, budget_s=15.0):
             "sample": f"the full batch of {T} tokens of weight set 0, {reps} repetitions, mean", "s_per_step": dt}
 
 
+def cpu_baseline_one_thread(args, variant, budget_s):
+    """The same oracle leg on ONE host thread: a child process with OMP_NUM_THREADS=1 (the oracle's only parallelism is
+    OpenMP over independent outputs) re-creates the workload from its seed and prints its cpu_baseline object."""
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK"):
+        env.pop(k, None)
+    cmd = [sys.executable, os.path.abspath(__file__), "--cpu-leg", str(variant), "--shape", args.shape, "--tokens",
+           str(args.tokens), "--cpu-budget", str(budget_s), "--router", args.router]
+    try:
+        r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=60 + 20 * budget_s)
+        return json.loads(r.stdout.strip().splitlines()[-1])
+    except Exception as ex:
+        return {"unavailable": f"{type(ex).__name__}: {ex}"}
+
+
+def run_cpu_leg(args):
+    from paper_2608_21240_b200 import workloads as W
+    shape = W.SHAPES[args.shape]
+    zipf = (args.tokens > 64) if args.router == "auto" else args.router == "zipf"
+    wl = W.make_layer(shape, args.tokens, variant=args.cpu_leg, zipf=zipf)
+    print(json.dumps(cpu_baseline(wl, budget_s=args.cpu_budget)))
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle timed on the host cores (there is no reference implementation)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -774,7 +810,7 @@ def main():
                     help="kernel path (SPICE_OPT_PATH): 0 auto, 1 general kernels, 2 no fused kernel, 3 mma.sync decode kernel")
     ap.add_argument("--stack", action="store_true",
                     help="time the MoE layers of the 26-layer stack at decode batch 8 (one step = 26 layer calls)")
-    ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout", "lore_calibrate"],
+    ap.add_argument("--op", default="layer", choices=["layer", "draft_confidence", "rollout", "lore_calibrate", "plumbing"],
                     help="what a step is: the MoE layer call (default) or the draft-router confidence call")
     ap.add_argument("--router", default="auto", choices=["auto", "uniform", "zipf"],
                     help="router of the synthetic layer: i.i.d. weights (uniform loads) or the Zipf-skewed one of config 4; "
@@ -785,8 +821,21 @@ def main():
                          "above 64 tokens (a dozen kernels on two streams per step)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--cpu-leg", type=int, default=None, help=argparse.SUPPRESS)   # child of cpu_baseline_one_thread
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.cpu_leg is not None:
+        run_cpu_leg(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args)      # no launcher around us: start the N ranks ourselves
+        return
+    if "WORLD_SIZE" in os.environ and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started WORLD_SIZE={os.environ['WORLD_SIZE']} ranks")
+    dispatch(args)
+
+
+def dispatch(args):
     if args.impl == "reference":
         run_reference(args)
     elif args.op == "draft_confidence":
@@ -795,10 +844,57 @@ def main():
         run_rollout(args)
     elif args.op == "lore_calibrate":
         run_lore_calibrate(args)
+    elif args.op == "plumbing":
+        run_plumbing(args)
     elif args.stack:
         run_stack(args)
     else:
         run_ours(args)
+
+
+def _rank_main(local_rank, args, port):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(local_rank), LOCAL_RANK=str(local_rank),
+                      WORLD_SIZE=str(args.gpus))
+    dispatch(args)
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` without a launcher: N processes on this node, one per GPU (rank = local rank = GPU
+    index), rendezvous on 127.0.0.1.  The ranks are replicas: they meet only at barriers and for the max over the ranks'
+    timings; rank 0 prints the JSON line."""
+    import socket
+
+    import torch.multiprocessing as mp
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    mp.spawn(_rank_main, args=(args, port), nprocs=args.gpus, join=True)
+
+
+def run_plumbing(args):
+    """--op plumbing: the multi-rank scaffolding alone (process group, barriers, max over ranks, whole-job rate, one JSON
+    line from rank 0) around a stand-in step that only sleeps.  Needs no GPU (gloo on CPU); it exists so that the N > 1
+    entry of this file can be exercised where there is one GPU or none."""
+    import torch
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    t0 = time.time()
+    for _ in range(args.steps):
+        time.sleep(1e-3 * (1 + rank))        # rank r is (1 + r) ms per step: the slowest rank must define the time
+    ms = (time.time() - t0) * 1e3
+    if world > 1:
+        dist.barrier()
+    (ms_max,) = max_over_ranks([ms])
+    if rank == 0:
+        print(json.dumps({"metric": "plumbing_units_per_s", "value": whole_job_throughput(args.tokens, args.steps, world, ms_max),
+                          "unit": "units/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": ms_max / args.steps, "ms_rank0": ms / args.steps, "higher_is_better": True,
+                          "scaling": "weak", "data": "none (sleep)", "gpu_launches": 0}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -95,7 +95,7 @@ spice_status spice_create(spice_ctx **ctx, int32_t device, const spice_layer_cfg
 spice_status spice_destroy(spice_ctx *ctx);
 spice_status spice_workspace_bytes(const spice_ctx *ctx, size_t *bytes /* host */);
 
-/* Router + TopK + gate scores (Eq. 1; "selected experts and their gate scores", Sec. 4.2).
+/* Router + TopK + gate scores (Eq. 1; the routing result the runtime policy of Sec. 4.2 starts from).
  *   h [T,d] bf16, w_router [N,d] bf16  ->  idx [T,K] int32, gate [T,K] fp32,
  *   logits [T,N] fp32 (optional, may be NULL).
  * Logits are accumulated in fp32; selection is done on logits, never on exponentials. */
@@ -116,7 +116,7 @@ spice_status spice_classify_misses(spice_ctx *ctx, const int32_t *idx, const flo
                                    int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
                                    float *resid_gate, void *stream);
 
-/* Exact execution of the resident experts (Sec. 4.2: "executes it exactly"):
+/* Exact execution of the resident experts (Sec. 4.2: an expert found on the GPU is run as it is):
  *   y[t,:] += sum over k with cls[t,k] == HIT of gate[t,k] * E_{slot[t,k]}(h[t,:]),   y [T,d] fp32.
  * Tokens are grouped by slot so that each resident expert's weights are read once. */
 spice_status spice_grouped_expert_ffn(spice_ctx *ctx, const spice_layer_weights *w /* host struct */,
@@ -133,7 +133,7 @@ spice_status spice_lore_surrogate(spice_ctx *ctx, const spice_layer_weights *w /
 /* The whole layer: route -> classify -> resident experts + shared/LoRE -> combine.
  *   h [T,d] bf16, conf as in spice_classify_misses.
  *   y_cpu_residual [T,d] fp32, optional: outputs of exactly recovered experts computed elsewhere
- *       (Sec. 4.3, "merges their outputs with the CPU expert outputs"); added before rounding.
+ *       (Sec. 4.3: the GPU result and the experts recovered on the host are summed into one output); added before rounding.
  *   x_resid [T,d] bf16, optional, in/out: residual stream, x_resid <- x_resid + y.
  *   y [T,d] bf16 out.  idx, gate, cls, counts, resid_*: as above; each may be NULL when not wanted.
  * Equals spice_route_topk, spice_classify_misses, y = 0, spice_grouped_expert_ffn,
@@ -175,7 +175,9 @@ spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, con
  *   h_final [T,d] bf16 out, optional: the draft state after the last projection made for each token.
  *   prefetch_mask [l_max, N] uint8 out, optional: the prefetch intents of Eq. 3 for the batch, kept per depth because
  *       depth l names experts of the layer l ahead: prefetch_mask[l-1, e] = 1 iff some token enqueues expert e at depth l.
- * Issuing the copies is the host runtime's job.  The call launches about 8 kernels per depth and is bound by their launch latency at decode batches. */
+ * Issuing the copies is the host runtime's job.  Decode batches the fused kernel takes run one launch per projecting
+ * depth plus four small ones for the last depth and the prefetch set; other shapes run about 8 general-shape kernels per
+ * depth.  Either way the call is bound by launch latency, not bandwidth. */
 spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w /* host array */,
                                     const spice_bf16 *x_current, int32_t T, int32_t l_min, int32_t l_max, float tau,
                                     int32_t *idx_hat, float *conf, int32_t *depth, spice_bf16 *h_final,
@@ -253,8 +255,13 @@ spice_status spice_launch_count(const spice_ctx *ctx, int64_t *launches /* host 
  * grouped GEMM for the experts at any batch size), 3 = for small batches use the fused decode
  * kernel built on mma.sync instead of the tcgen05 one.  SPICE_OPT_SPIN_LIMIT: number of polls after which a
  * dependency wait inside the fused decode kernel gives up and reports SPICE_ERR_TIMEOUT
- * (default 2^20; a poll takes 0.1 to 1 us). */
-enum { SPICE_OPT_PATH = 0, SPICE_OPT_SPIN_LIMIT = 1 };
+ * (default 2^20; a poll takes 0.1 to 1 us).  SPICE_OPT_TC_WAIT_LIMIT: the same for the pipeline waits (shared-memory
+ * barriers between the copy, tensor-core and epilogue roles) of the grouped GEMM kernel that batches above 64 tokens
+ * run on (default 2^22 polls).  A wait that gives up ends its thread block early: the call's outputs are then
+ * undefined, SPICE_ERR_TIMEOUT is recorded in the status word, nothing stays in flight, and the next call on the
+ * ctx starts clean (dependency counters are reset by the kernel that gave up; the status word stays set until
+ * spice_get_device_status reads it). */
+enum { SPICE_OPT_PATH = 0, SPICE_OPT_SPIN_LIMIT = 1, SPICE_OPT_TC_WAIT_LIMIT = 2 };
 spice_status spice_set_option(spice_ctx *ctx, int32_t option, int64_t value);
 
 /* Text for a status code (static storage, never NULL). */

@@ -78,7 +78,7 @@ void oracle_router_logits(int T, int d, int N, const float *h, const float *w_ro
             logits[(size_t)t * N + e] = dot_fd(w_router + (size_t)e * d, h + (size_t)t * d, d);
 }
 
-/* Eq. 1 TopK and the gate scores of Sec. 4.2 ("selected experts and their gate scores").
+/* Eq. 1 TopK and the gate scores that the runtime policy of Sec. 4.2 takes as its input.
  * K rounds of arg-max over the experts not yet taken; ties go to the smaller index.
  * idx[t,0..K-1] is in order of decreasing logit. */
 void oracle_topk_gates(int T, int N, int K, int norm_topk, const double *logits, int32_t *idx, double *gate) {

@@ -108,7 +108,7 @@ def spice_launch_count(ctx) -> int:
     return n.value
 
 
-OPT_PATH, OPT_SPIN_LIMIT = 0, 1
+OPT_PATH, OPT_SPIN_LIMIT, OPT_TC_WAIT_LIMIT = 0, 1, 2
 
 
 def spice_set_option(ctx, option: int, value: int) -> None:

@@ -114,6 +114,7 @@ void carve(spice_ctx *c, char *base, size_t *total) {
         c->tcb.n_mtiles = cv.take<int32_t>(4);
         c->tcb.n_mtiles_shared = cv.take<int32_t>(4);
         c->tcb.n_mtiles_low = cv.take<int32_t>(4);
+        c->tcb.status = c->tb.status;
     }
     *total = (cv.off + 255) & ~size_t(255);
 }
@@ -307,6 +308,10 @@ spice_status spice_set_option(spice_ctx *ctx, int32_t option, int64_t value) {
         case SPICE_OPT_SPIN_LIMIT:
             if (value < 1 || value > (1ll << 30)) return SPICE_ERR_INVALID_ARG;
             ctx->opt_spin_limit = value;
+            return SPICE_OK;
+        case SPICE_OPT_TC_WAIT_LIMIT:
+            if (value < 1 || value > (1ll << 30)) return SPICE_ERR_INVALID_ARG;
+            ctx->tcb.wait_limit = (uint32_t)value;
             return SPICE_OK;
     }
     return SPICE_ERR_INVALID_ARG;
@@ -557,58 +562,75 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     const bool tc_path = ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm);
     // The shared expert needs nothing but h: it runs on the context's side stream beside the routing chain (router,
     // classification, grouping, gather occupy few SMs) and joins before the combine.  Both event edges are ordinary
-    // stream dependencies, so the call can still be captured into a CUDA graph.
+    // stream dependencies, so the call can still be captured into a CUDA graph.  Once the side stream has been forked
+    // off, every way out of this function -- an error return included -- joins it back into the caller's stream: a
+    // capture of that stream would otherwise be left with an unjoined branch.
     bool forked = false;
+    spice_status rc = SPICE_OK;
+    // (a failed launch ends the sequence; the join below still runs)
+#define SPICE_STEP(expr)                          \
+    do {                                          \
+        if (rc == SPICE_OK) {                     \
+            int n_ = (expr);                      \
+            if (n_ < 0) rc = SPICE_ERR_CUDA;      \
+            else ctx->launches += n_;             \
+        }                                         \
+    } while (0)
     if (tc_path) {
         if (ctx->side && cudaEventRecord(ctx->ev_fork, st) == cudaSuccess &&
             cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) == cudaSuccess) {
-            SPICE_LAUNCH(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ctx->side));
             forked = true;
+            SPICE_STEP(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ctx->side));
         } else {
             cudaGetLastError();
         }
     }
     if (tc_path && T > 64 && tc_router_ok(dm)) {
         // large batch: the logits are a GEMM of their own (a status word of the GEMM is the tables' one)
-        SPICE_LAUNCH(launch_tc_router_logits(dm, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), ctx->route_logits,
-                                             ctx->tcb, ctx->n_sms, st));
-        SPICE_LAUNCH(launch_topk_from_logits(dm, ctx->cfg.norm_topk, ctx->route_logits, idx, gate, st));
+        SPICE_STEP(launch_tc_router_logits(dm, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), ctx->route_logits,
+                                           ctx->tcb, ctx->n_sms, st));
+        SPICE_STEP(launch_topk_from_logits(dm, ctx->cfg.norm_topk, ctx->route_logits, idx, gate, st));
     } else {
-        SPICE_LAUNCH(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
-                                       gate, nullptr, st));
+        SPICE_STEP(launch_route_topk(dm, ctx->cfg.norm_topk, hb, reinterpret_cast<const __nv_bfloat16 *>(w->w_router), idx,
+                                     gate, nullptr, st));
     }
-    SPICE_LAUNCH(launch_classify_group(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
-                                       ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb, st, &ctx->gsc));
+    SPICE_STEP(launch_classify_group(dm, ctx->cfg.conf_stride, ctx->cfg.tau, idx, gate, w->slot_of_expert, conf, cls,
+                                     ctx->ws_slot, counts, resid_tok, resid_k, resid_expert, resid_gate, ctx->tb, st, &ctx->gsc));
     if (tc_path) {
         // batches the decode kernel does not take: exact experts, shared expert and LoRE down-projection on the
         // tensor cores (grouped GEMM kernel), LoRE up-projection on lore_b_kernel
         // the LoRE groups need the grouping, not the routed experts: on the side stream they run beside the routed GEMMs
         cudaStream_t ls = st;
-        if (forked) {
+        if (forked && rc == SPICE_OK) {
             if (cudaEventRecord(ctx->ev_grouped, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_grouped, 0) != cudaSuccess)
-                return SPICE_ERR_CUDA;
+                rc = SPICE_ERR_CUDA;
             ls = ctx->side;
         }
-        SPICE_LAUNCH(launch_tc_routed(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
-        if (!forked) SPICE_LAUNCH(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        SPICE_STEP(launch_tc_routed(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        if (!forked) SPICE_STEP(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
         if (tc_lore_ok(dm)) {
-            SPICE_LAUNCH(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ls));
-            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 1, ls));
+            SPICE_STEP(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ls));
+            SPICE_STEP(launch_lore_b(dm, *w, ctx->tb, 1, ls));
         } else {
-            SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, ls));
-            SPICE_LAUNCH(launch_lore_b(dm, *w, ctx->tb, 0, ls));
+            SPICE_STEP(launch_lore_a(dm, *w, hb, ctx->tb, ls));
+            SPICE_STEP(launch_lore_b(dm, *w, ctx->tb, 0, ls));
         }
-        if (forked && cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return SPICE_ERR_CUDA;   // (after whatever ran there)
     } else {
-        SPICE_LAUNCH(launch_gateup(dm, KIND_SHARED | KIND_HIT, *w, hb, ctx->tb, st));
-        SPICE_LAUNCH(launch_lore_a(dm, *w, hb, ctx->tb, st));
-        SPICE_LAUNCH(launch_down(dm, KIND_SHARED | KIND_HIT | KIND_LOW, *w, ctx->tb, st));
+        SPICE_STEP(launch_gateup(dm, KIND_SHARED | KIND_HIT, *w, hb, ctx->tb, st));
+        SPICE_STEP(launch_lore_a(dm, *w, hb, ctx->tb, st));
+        SPICE_STEP(launch_down(dm, KIND_SHARED | KIND_HIT | KIND_LOW, *w, ctx->tb, st));
     }
-    if (forked && cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return SPICE_ERR_CUDA;
+    if (forked) {   // join, whatever happened above (after whatever ran on the side stream)
+        if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess || cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) {
+            cudaGetLastError();
+            if (rc == SPICE_OK) rc = SPICE_ERR_CUDA;
+        }
+    }
     CombineArgs ca{KIND_SHARED | KIND_HIT | KIND_LOW, 0, gate, cls, nullptr, reinterpret_cast<__nv_bfloat16 *>(y),
                    y_cpu_residual, reinterpret_cast<__nv_bfloat16 *>(x_resid)};
-    SPICE_LAUNCH(launch_combine(dm, ca, ctx->tb, st));
-    return SPICE_OK;
+    SPICE_STEP(launch_combine(dm, ca, ctx->tb, st));
+#undef SPICE_STEP
+    return rc;
 }
 
 }  // extern "C"

@@ -1,7 +1,7 @@
 // LoRE calibration of one (layer, expert) pair (Sec. 4.2 of the paper): fit the rank-r residual module
 //     Delta(h) = B A h,   A: r x d,  B: d x r,
 // that minimises  sum_{h in D} || E(h) - S(h) - B A h ||_2^2  over the calibration tokens routed to the expert.
-// The paper says the parameters are "trained by minimizing" this objective; the objective is a reduced-rank
+// The paper states this objective and names no optimiser; the objective is a reduced-rank
 // regression and has a closed-form minimiser, which is what is computed here (in fp32, offline path):
 //     G = H^T H (+ ridge),  C = H^T R          H [n,d] hidden states, R [n,d] targets E(h) - S(h)
 //     G = L L^T,  Z = L^-1 C                   (then the fitted values satisfy  Yhat^T Yhat = Z^T Z)

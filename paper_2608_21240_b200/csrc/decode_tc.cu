@@ -1130,7 +1130,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             Plan pl;
             plan_static(pl, q);
             plan_routed(pl, sh->n_hg, sh->n_lg);
-            // Warp 1 watches the per-group counters while the weights stream, so that the producer finds a flag in
+            // Warp 1 of the auxiliary team (warp 7 of the CTA) watches the per-group counters while the weights stream, so that the producer finds a flag in
             // shared memory instead of paying a round trip to L2 when it reaches a down tile.  It ends when every
             // group is complete (or on abort / after its time limit); the producer never depends on it.
             if (a.aw == 1) {
@@ -1179,14 +1179,16 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         g_dtc_cal[blockIdx.x * 4 + 3] = (unsigned long long)clock64();
     }
 #endif
-    // the last CTA to finish clears the counters for the next launch (after an abort the host does it)
+    // The last CTA to finish clears the counters for the next launch.  Every other CTA has passed this point, aborted
+    // or not, so the counters (the abort word among them) are nobody's any more: the next call on this ctx starts
+    // clean even when this one gave up, and the sticky status word keeps the record of that.
     if (threadIdx.x == 0) {
         if (sh->abort_flag) atomicMax(p.tb.status, (int)SPICE_ERR_TIMEOUT);
         __threadfence();
         sh->last_flag = atomicAdd(p.sync + SY_TEAMS_DONE, 1) == (int)gridDim.x - 1;
     }
     __syncthreads();
-    if (sh->last_flag && !sh->abort_flag) {
+    if (sh->last_flag) {
         __threadfence();
         for (int i = threadIdx.x; i < p.sync_words; i += DTC_THREADS) p.sync[i] = 0;
     }

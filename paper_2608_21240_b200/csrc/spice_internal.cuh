@@ -174,6 +174,8 @@ struct TcBuffers {
     __nv_bfloat16 *act_shared16;  // [Tm, I_s]
     MTile *mtiles, *mtiles_shared, *mtiles_low;   // tile lists: routed (also the router's), shared expert, LOW groups
     int32_t *n_mtiles, *n_mtiles_shared, *n_mtiles_low;
+    int32_t *status;              // sticky device status word of the ctx
+    uint32_t wait_limit;          // polls after which a pipeline wait of the GEMM kernel gives up (0: the default)
 };
 bool tc_available();
 int tc_prepare();

@@ -11,7 +11,7 @@ bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], co
 
 namespace tcdev {
 
-constexpr uint32_t WAIT_LIMIT = 1u << 22;   // polls per wait before the CTA gives up
+constexpr uint32_t WAIT_LIMIT = 1u << 22;   // default polls per wait before the CTA gives up; always the limit of drains
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t a, int n) {
@@ -32,13 +32,18 @@ __device__ __forceinline__ bool mbar_try(uint32_t a, uint32_t parity) {
     return ok != 0;
 }
 // bounded wait; false when the limit expired or another role already gave up
-__device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile int *abort_flag) {
-    for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t a, uint32_t parity, volatile int *abort_flag, uint32_t limit = WAIT_LIMIT) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try(a, parity)) return true;
         if ((i & 1023u) == 1023u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
+}
+// wait for work already in flight (copies, MMAs) that must be over before the CTA ends: ignores the abort flag
+__device__ __forceinline__ void mbar_drain(uint32_t a, uint32_t parity) {
+    for (uint32_t i = 0; i < WAIT_LIMIT; ++i)
+        if (mbar_try(a, parity)) return;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t mbar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"

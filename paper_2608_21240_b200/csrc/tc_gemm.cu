@@ -43,7 +43,7 @@ constexpr uint32_t IDESC = make_idesc(BM, BN2);
 __device__ __forceinline__ float silu_x(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 
 struct TcShared {
-    alignas(8) unsigned long long full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+    alignas(8) unsigned long long full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], mma_drain;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -64,6 +64,7 @@ struct TcGemmArgs {
     const int32_t *row_map;     // MODE_OUT: output row of A row r (entry id), or null for identity
     int32_t ld;
     int32_t *status;
+    uint32_t wait_limit;        // polls after which a pipeline wait gives up (SPICE_OPT_TC_WAIT_LIMIT)
 };
 
 template <int MODE>   // 0 = gate/up + SwiGLU, 1 = plain
@@ -87,9 +88,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
             mbar_init(smem_u32(&sh->tmem_full[b]), 1);
             mbar_init(smem_u32(&sh->tmem_empty[b]), 4);
         }
+        mbar_init(smem_u32(&sh->mma_drain), 1);
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    const uint32_t wl = g.wait_limit;
     if (warp == 1) {   // TMEM: all 512 columns (two 256-column accumulators)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
@@ -114,7 +117,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
                 const int b_row = mt.slot * g.b_rows_per_slot + nt * (MODE == 0 ? 128 : BN2);
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
-                    if (!mbar_wait(smem_u32(&sh->empty[s]), ((it / STAGES) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(smem_u32(&sh->empty[s]), ((it / STAGES) & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                     const uint32_t full = smem_u32(&sh->full[s]);
                     const uint32_t dst = smem_u32(ring + s * STAGE_BYTES);
                     mbar_expect_tx(full, STAGE_BYTES);
@@ -128,9 +131,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
                     }
                 }
             }
-            // drain: every stage that was armed must have landed before the CTA may end
+            // drain: every stage that was armed must have landed before the CTA may end (also after an abort)
             for (uint32_t j = (it > STAGES ? it - STAGES : 0); j < it; ++j)
-                mbar_wait(smem_u32(&sh->full[j % STAGES]), (j / STAGES) & 1, abort_flag);
+                mbar_drain(smem_u32(&sh->full[j % STAGES]), (j / STAGES) & 1);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (one lane)
@@ -139,12 +142,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tcount) {
                 const int buf = tcount & 1;
-                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag)) break;
+                if (!mbar_wait(smem_u32(&sh->tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag, wl)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN2;
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
-                    if (!mbar_wait(smem_u32(&sh->full[s]), (it / STAGES) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(smem_u32(&sh->full[s]), (it / STAGES) & 1, abort_flag, wl)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a0 = smem_u32(ring + s * STAGE_BYTES), b0 = a0 + A_BYTES;
                     const uint64_t da = make_desc(a0), db = make_desc(b0);
@@ -155,6 +158,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
                 }
                 if (ok) tc_commit(smem_u32(&sh->tmem_full[buf]));
             }
+            // every MMA this thread issued must be over before the TMEM columns are given back
+            tc_commit(smem_u32(&sh->mma_drain));
+            mbar_drain(smem_u32(&sh->mma_drain), 0);
         }
     } else {
         // ---------------- epilogue: warp w owns TMEM lanes 32*(w%4) .. +31 = rows of the tile
@@ -165,7 +171,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
             const MTile mt = g.mtiles[tile / g.n_ntiles];
             const int nt = tile % g.n_ntiles;
             bool ok = true;
-            if (lane == 0) ok = mbar_wait(smem_u32(&sh->tmem_full[buf]), (tcount >> 1) & 1, abort_flag);
+            if (lane == 0) ok = mbar_wait(smem_u32(&sh->tmem_full[buf]), (tcount >> 1) & 1, abort_flag, wl);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
             tc_fence_after();
@@ -379,6 +385,7 @@ bool tc_router_ok(const Dims &dm) { return tc_shape_ok(dm) && dm.N <= BN2 && dm.
 
 int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router, float *logits,
                             const TcBuffers &b, int n_sms, cudaStream_t st) {
+    const uint32_t wait_limit = b.wait_limit ? b.wait_limit : WAIT_LIMIT;
     CUtensorMap ma, mb;
     // (the tile list of the routed experts is free until the grouping has run; the shared expert's list may be in
     // use on the side stream)
@@ -395,7 +402,8 @@ int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_b
     g.out32 = logits;
     g.row_map = nullptr;
     g.ld = dm.N;
-    g.status = nullptr;
+    g.status = b.status;
+    g.wait_limit = wait_limit;
     tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
@@ -466,6 +474,7 @@ int launch_tc_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bf
     g.row_map = nullptr;
     g.ld = dm.r;
     g.status = tb.status;
+    g.wait_limit = b0.wait_limit ? b0.wait_limit : WAIT_LIMIT;
     tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
     return cudaGetLastError() == cudaSuccess ? 3 : -1;
 }
@@ -480,6 +489,7 @@ int launch_tc_routed(const Dims &dm, const spice_layer_weights &w, const __nv_bf
     const size_t cap = (size_t)dm.T * dm.K;
     TcGemmArgs g{};
     g.status = tb.status;
+    g.wait_limit = b.wait_limit ? b.wait_limit : WAIT_LIMIT;
     // ---- routed experts
     build_mtiles_kernel<<<1, 32, 0, st>>>(tb.groups, tb.hdr, b.mtiles, b.n_mtiles);
     gather_rows_kernel<<<n_sms * 4, 256, 0, st>>>(h, tb.perm_hit, tb.hdr, dm.K, dm.d, b.x_perm);
@@ -520,6 +530,7 @@ int launch_tc_shared(const Dims &dm, const spice_layer_weights &w, const __nv_bf
     int launches = 0;
     TcGemmArgs g{};
     g.status = tb.status;
+    g.wait_limit = b.wait_limit ? b.wait_limit : WAIT_LIMIT;
     build_shared_mtiles_kernel<<<1, 32, 0, st>>>(dm.T, b.mtiles_shared, b.n_mtiles_shared);
     ++launches;
     if (!make_map(&ma, h, dm.T, dm.d, BM) || !make_map(&mb, w.shared_w_gate_up, (uint64_t)2 * dm.Is, dm.d, 128)) return -1;

@@ -9,7 +9,7 @@ import oracle
 from paper_2608_21240_b200 import binding as B
 from paper_2608_21240_b200 import workloads as W
 from tests._cases import enforce_margins, run_oracle
-from tests._gpu import (GATE_ATOL, LOGIT_ATOL, bf16_tensor, cfg_of, check_routing, upload, y_close)
+from tests._gpu import (GATE_ATOL, LOGIT_ATOL, Y_ATOL, Y_RTOL, bf16_tensor, cfg_of, check_routing, upload, y_close)
 
 pytestmark = pytest.mark.gpu
 
@@ -238,6 +238,40 @@ def test_expired_dependency_wait_reports_timeout_and_recovers():
     torch.cuda.synchronize()
     assert L.device_status() == 0
     assert torch.equal(again.y, good.y) and torch.equal(again.idx, good.idx)
+    # the kernel that gave up resets the dependency counters itself: a call that follows WITHOUT a status read in
+    # between is complete and correct, and the status word still tells that an earlier call timed out
+    L.set_option(B.OPT_SPIN_LIMIT, 1)
+    L.moe_layer_fwd(w, h, conf)
+    L.set_option(B.OPT_SPIN_LIMIT, 1 << 20)
+    third = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert torch.equal(third.y, good.y) and torch.equal(third.cls, good.cls)
+    assert L.device_status() == 6 and L.device_status() == 0
+    L.close()
+
+
+def test_expired_pipeline_wait_of_the_large_batch_gemm_reports_timeout_and_recovers():
+    """The same for the grouped GEMM kernel of batches above 64 tokens: with a limit of one poll a role's wait on its
+    shared-memory barrier (e.g. the tensor-core warp's wait for the first tile copy) runs out, the thread block records
+    SPICE_ERR_TIMEOUT, lets its copies and MMAs in flight finish, frees its TMEM and returns; nothing hangs, and the
+    next call with the default limit gives the first call's bits."""
+    wl = _layer_case("tiny", 200, variant=12)
+    s = wl.shape
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    w = upload(wl)
+    h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+    good = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    L.set_option(B.OPT_TC_WAIT_LIMIT, 1)
+    L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert L.device_status() == 6               # SPICE_ERR_TIMEOUT
+    L.set_option(B.OPT_TC_WAIT_LIMIT, 1 << 22)
+    again = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    assert torch.equal(again.y, good.y) and torch.equal(again.idx, good.idx) and torch.equal(again.cls, good.cls)
     L.close()
 
 
@@ -439,7 +473,7 @@ def test_split_exports_compose_to_the_fused_call(name, T):
     ref = run_oracle(wl, want_full=False)
     err, bound = y_close(y.cpu().numpy(), ref.y)
     assert err <= bound
-    assert (y.bfloat16().float() - fused.y.float()).abs().max().item() <= 2e-2 * fused.y.float().abs().max().item()
+    assert (y.bfloat16().float() - fused.y.float()).abs().max().item() <= Y_RTOL * fused.y.float().abs().max().item() + Y_ATOL
     # the routed part alone: oracle with the shared/LoRE part removed = hits only
     hits_only = np.zeros_like(ref.y)
     for t in range(wl.T):
@@ -467,6 +501,38 @@ def test_batch_independence_and_repeatability():
         assert torch.equal(one.idx[0], a.idx[t]) and torch.equal(one.cls[0], a.cls[t])
         diff = (one.y[0].float() - a.y[t].float()).abs().max().item()
         assert diff <= 1e-2 * a.y[t].float().abs().max().item() + 1e-3
+    L.close()
+
+
+@pytest.mark.parametrize("T", [1, 4, 16, 64])
+def test_repeated_calls_over_rotating_weight_sets_are_bit_identical(T):
+    """240 back-to-back layer calls that rotate through 4 independent weight sets (2.6 GB, so every call streams its
+    weights from HBM with a cold L2, as in a decode loop): every output of every later pass equals the first pass bit
+    for bit.  Inside the fused decode kernel the activations of a group are written by ordinary stores of one CTA and
+    fetched by TMA copies of others, ordered by a release / acquire pair on the group's counter and a proxy fence on the
+    reader's side; a gap in that ordering would show here as a rare stale tile."""
+    s = W.SHAPES["dsv2lite"]
+    sets = [W.make_layer(s, T, variant=300 + i) for i in range(4)]
+    ws = [upload(wl) for wl in sets]
+    structs = [w.c_struct() for w in ws]
+    L = B.SpiceLayer(cfg_of(s), T)
+    h, conf = bf16_tensor(sets[0].h), torch.from_numpy(sets[0].conf).cuda()
+    n_pass = 60
+    ys = torch.empty(n_pass, 4, T, s.d, dtype=torch.bfloat16, device="cuda")
+    idx = torch.empty(n_pass, 4, T, s.top_k, dtype=torch.int32, device="cuda")
+    cls = torch.empty(n_pass, 4, T, s.top_k, dtype=torch.uint8, device="cuda")
+    st = torch.cuda.current_stream()
+    n0 = L.launch_count()
+    for p in range(n_pass):
+        for i in range(4):
+            B.spice_moe_layer_fwd(L.ctx, structs[i], h, conf, T, ys[p, i], idx=idx[p, i], cls=cls[p, i], stream=st)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0 and L.launch_count() - n0 == 4 * n_pass     # one fused kernel per call
+    assert bool(torch.isfinite(ys[0].float()).all()) and int((cls[0] == 0).sum()) > 0
+    assert not torch.equal(ys[0, 0], ys[0, 1])                                   # the sets really differ
+    same = (ys == ys[0:1]).flatten(1).all(dim=1)
+    assert bool(same.all()), f"passes that differ from the first: {torch.nonzero(~same).flatten().tolist()[:10]}"
+    assert bool((idx == idx[0:1]).all()) and bool((cls == cls[0:1]).all())
     L.close()
 
 
@@ -548,26 +614,66 @@ def test_corrupt_slot_table_sets_status_without_faulting():
     L.close()
 
 
+def _config4_sample(idx, n_experts, n_random=64, seed=4):
+    """Tokens for the oracle at 4096 tokens, chosen from the ORACLE's routing so that every expert's row range is looked
+    at from both ends: per expert its first and its last token (the first and the last 128-row tile of its group hold
+    them whenever the group is laid out in token order), one token out of every 128 of its list (a group of m tokens
+    spans ceil(m / 128) tiles), every token of an expert that has at most four, plus random tokens."""
+    rng = np.random.default_rng(seed)
+    T = idx.shape[0]
+    pick = set(rng.choice(T, size=n_random, replace=False).tolist())
+    for e in range(n_experts):
+        toks = np.nonzero((idx == e).any(axis=1))[0]
+        if toks.size == 0:
+            continue
+        pick.update(toks[::128].tolist())
+        pick.update((int(toks[0]), int(toks[-1])))
+        if toks.size <= 4:
+            pick.update(toks.tolist())
+    return sorted(pick)
+
+
 def test_config4_prefill_4096_tokens_skewed_loads_sampled_against_oracle():
     """DeepSeek-V2-Lite-shaped layer, 4096 tokens, Zipf-skewed router, every expert resident.
-    Routing / classification are compared for all tokens, outputs for a sample the oracle can afford."""
+    Routing / classification are compared for all tokens.  Outputs: against the oracle on a sample that touches both
+    ends and every 128th row of every expert's group, and -- because the grouping of such batches places rows by
+    atomics, so that no host-side choice can name the tile a token lands in -- ALL 4096 tokens of the tensor-core path
+    against the general-shape kernels (GPU against GPU at the output tolerance), which therefore covers every 128-row
+    tile of every group, the last partial tile of the hottest expert and the smallest group included."""
     wl = _layer_case("dsv2lite_prefill", 4096, zipf=True)
     s = wl.shape
-    tokens = sorted(np.random.default_rng(4).choice(4096, size=24, replace=False).tolist())
+    pre = run_oracle(wl, skip_ffn=True)
+    tokens = _config4_sample(pre.idx, s.n_experts)
+    assert 150 <= len(tokens) <= 400
     ref = run_oracle(wl, tokens=tokens, want_full=False)
     load = np.bincount(ref.idx.ravel(), minlength=s.n_experts)
     assert load.max() > 8 * max(1, load.min())            # loads really are imbalanced
+    assert load.max() > 3000 and load.min() < 128          # a group of dozens of tiles and one smaller than a tile
     assert ref.counts.tolist() == [4096 * s.top_k, 0, 0]
     L = B.SpiceLayer(cfg_of(s), wl.T)
     w = upload(wl)
-    out = L.moe_layer_fwd(w, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
+    h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+    n0 = L.launch_count()
+    out = L.moe_layer_fwd(w, h, conf)
     torch.cuda.synchronize()
+    n_tc = L.launch_count() - n0
     check_routing(out, ref, wl.T, s.top_k)
     y = out.y.float().cpu().numpy()
     assert np.isfinite(y).all()
     err, bound = y_close(y[np.asarray(tokens)], ref.y)
     assert err <= bound, (err, bound)
     assert L.device_status() == 0
+    # every token, every tile: the same call on the general-shape kernels
+    L.set_option(B.OPT_PATH, 1)
+    gen = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0 and L.launch_count() - n0 - n_tc > 0
+    assert torch.equal(gen.idx, out.idx) and torch.equal(gen.cls, out.cls)
+    yg = gen.y.float().cpu().numpy()
+    errg, boundg = y_close(yg[np.asarray(tokens)], ref.y)
+    assert errg <= boundg, (errg, boundg)
+    diff = np.abs(yg - y).max(axis=1)
+    assert diff.max() <= Y_RTOL * np.abs(yg).max() + Y_ATOL, (int(diff.argmax()), float(diff.max()))
     L.close()
 
 
@@ -596,7 +702,7 @@ def test_large_batch_with_misses_multi_cta_tables_sampled_against_oracle():
     # the general kernels on the tables the multi-CTA grouping built
     L.set_option(B.OPT_PATH, 1)
     gen = L.moe_layer_fwd(w, h, conf)
-    assert (gen.y.float() - out.y.float()).abs().max().item() <= 2e-2 * out.y.float().abs().max().item() + 2e-3
+    assert (gen.y.float() - out.y.float()).abs().max().item() <= Y_RTOL * out.y.float().abs().max().item() + Y_ATOL
     assert L.device_status() == 0
     L.close()
 

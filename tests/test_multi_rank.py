@@ -44,3 +44,29 @@ def test_single_rank_is_identity():
     import bench
     assert bench.max_over_ranks([3.5, 4.0]) == [3.5, 4.0]
     assert bench.whole_job_throughput(16, 10, 1, 2.0) == 16 * 10 / 2e-3
+
+
+def test_bench_gpus_flag_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` with no launcher environment must start two ranks (not one rank that reports
+    n_gpus = 1).  Driven through the file's real entry point with the CPU stand-in step (--op plumbing, gloo): rank r
+    sleeps (1 + r) ms per step, so the reported time must be the slower rank's and the rate both ranks' units over it."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--op", "plumbing", "--steps", "30",
+                        "--tokens", "16"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, r.stdout          # rank 0 alone prints
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2
+    assert out["ms_per_step"] >= 2.0 > out["ms_rank0"]            # the slowest rank defines the step
+    assert abs(out["value"] - 2 * 16 / (out["ms_per_step"] * 1e-3)) < 1e-6 * out["value"]
+
+
+def test_bench_refuses_a_world_size_that_contradicts_gpus():
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--op", "plumbing"], env=env,
+                       capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "WORLD_SIZE" in (r.stderr + r.stdout)
