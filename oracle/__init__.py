@@ -209,6 +209,69 @@ def min_lookahead_depth(n_prefetch: int, expert_bytes: float, pcie_bytes_per_s: 
     return int(math.ceil(n_prefetch * expert_bytes / (pcie_bytes_per_s * t_comp_s)))
 
 
+# ---------------------------------------------------------------------------------------------------------------
+# Second weight precision (the paper reports every result at BF16 and at one quantised precision, Sec. 5.1 / Table 1,
+# and names that format without defining it).  Reading taken here: weights of the routed and shared experts stored as
+# 8-bit floats in the E4M3 layout (1 sign, 4 exponent bits with bias 7, 3 fraction bits; no infinities; S.1111.111 is
+# NaN; largest finite value 448; subnormals m/8 * 2^-6) with ONE power-of-two scale per output row:
+#     s_r = 2^ceil(log2(max_j |W_rj| / 448))   (1 for an all-zero row),   q_rj = nearest E4M3 value of W_rj / s_r,
+# ties to the even code, magnitudes above 448 saturate.  The layer on such weights is BY DEFINITION the layer of
+# `layer()` above evaluated on the dequantised values s_r * q_rj (exact in fp32, since s_r is a power of two and q has
+# four significant bits); router and LoRE factors keep their precision, so no routing decision depends on the format.
+
+
+def _e4m3_finite_values() -> np.ndarray:
+    """The 127 non-negative finite E4M3 values in code order (code = exponent field * 8 + fraction), as fp64."""
+    vals = []
+    for code in range(127):                      # code 127 = 1111.111 is NaN
+        e, m = code >> 3, code & 7
+        vals.append(m / 8.0 * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7))
+    return np.array(vals, dtype=np.float64)
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """Value (fp64) of E4M3 bytes; 0x7F / 0xFF decode to NaN."""
+    c = np.asarray(codes, dtype=np.uint8)
+    mag = np.concatenate([_e4m3_finite_values(), [np.nan]])[c & 0x7F]
+    return np.where(c & 0x80, -mag, mag)
+
+
+def e4m3_encode(x) -> np.ndarray:
+    """Nearest finite E4M3 value of every element of x (fp64 arithmetic), as bytes.  Written as the definition: among
+    the two neighbouring representable magnitudes the nearer one wins, an exact tie goes to the one whose code is even
+    (round-half-to-even), magnitudes beyond 448 give 448.  The sign is kept (also for zero); NaN gives 0x7F."""
+    x = np.asarray(x, dtype=np.float64)
+    table = _e4m3_finite_values()
+    a = np.minimum(np.abs(x), table[-1])
+    hi = np.searchsorted(table, a, side="left")          # first code whose value is >= a
+    hi = np.minimum(hi, 126)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = a - table[lo], table[hi] - a
+    take_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(take_hi, hi, lo).astype(np.uint8)
+    code = np.where(np.isnan(x), np.uint8(0x7F), code)
+    return (code | np.where(np.signbit(x) & ~np.isnan(x), np.uint8(0x80), np.uint8(0))).astype(np.uint8)
+
+
+def quantize_e4m3_rows(W):
+    """Per-row power-of-two scale and E4M3 codes of a weight matrix [..., rows, cols] (see the reading above).
+    Returns (codes uint8 of W's shape, scale fp32 of W's shape without the last axis)."""
+    W = np.asarray(W, dtype=np.float64)
+    amax = np.abs(W).max(axis=-1)
+    m, e = np.frexp(amax / 448.0)                        # amax / 448 = m * 2^e, m in [0.5, 1)
+    exp = np.where(m == 0.5, e - 1, e)                   # ceil(log2(.)) without a logarithm
+    scale = np.where(amax > 0, np.ldexp(1.0, exp), 1.0)
+    return e4m3_encode(W / scale[..., None]), scale.astype(np.float32)
+
+
+def dequantize_e4m3_rows(codes, scale) -> np.ndarray:
+    """s_r * q_rj as fp32 (exact for power-of-two scales)."""
+    v = e4m3_decode(codes) * np.asarray(scale, dtype=np.float64)[..., None]
+    out = v.astype(np.float32)
+    assert np.array_equal(out.astype(np.float64), v, equal_nan=True), "scale is not a power of two (or out of range)"
+    return out
+
+
 def classify(idx, resident, conf, tau: float, conf_stride: Optional[int] = None):
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     T, K = idx.shape

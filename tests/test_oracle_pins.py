@@ -535,3 +535,107 @@ def test_p16_prefetch_set_and_minimum_lookahead_depth():
     assert oracle.min_lookahead_depth(2, 17.3e6, 25e9, 0.5e-3) == 3
     assert oracle.min_lookahead_depth(2, 17.3e6, 25e9, 1.4e-3) == 1
     assert oracle.min_lookahead_depth(0, 17.3e6, 25e9, 1e-3) == 0
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# P17: the 8-bit weight format (E4M3 codes, one power-of-two scale per output row) that stands in for the paper's
+# second, quantised weight precision (Sec. 5.1, Table 1).  The format's constants below are written by hand from its
+# definition (1-4-3 bits, bias 7, no infinities, largest finite value 448, subnormal step 2^-9).
+def test_p17_e4m3_code_values_by_hand():
+    hand = {0x00: 0.0, 0x01: 2.0 ** -9, 0x07: 7 * 2.0 ** -9, 0x08: 2.0 ** -6, 0x0F: 1.875 * 2.0 ** -6, 0x30: 0.5, 0x38: 1.0,
+            0x39: 1.125, 0x3F: 1.875, 0x40: 2.0, 0x44: 3.0, 0x78: 256.0, 0x7E: 448.0, 0xB8: -1.0, 0xFE: -448.0, 0x81: -2.0 ** -9}
+    codes = np.array(sorted(hand), dtype=np.uint8)
+    assert oracle.e4m3_decode(codes).tolist() == [hand[int(c)] for c in codes]
+    assert np.isnan(oracle.e4m3_decode(np.array([0x7F, 0xFF], np.uint8))).all()
+    assert np.signbit(oracle.e4m3_decode(np.array([0x80], np.uint8))[0])               # -0
+    # strictly increasing in the code, and every finite code survives decode -> encode
+    allc = np.arange(256, dtype=np.uint8)
+    fin = allc[(allc & 0x7F) != 0x7F]
+    v = oracle.e4m3_decode(fin)
+    assert (np.diff(v[:127]) > 0).all() and np.array_equal(oracle.e4m3_encode(v), fin)
+
+
+def test_p17_e4m3_rounding_is_nearest_even_and_saturates():
+    enc = lambda *xs: oracle.e4m3_encode(np.array(xs, dtype=np.float64)).tolist()
+    # halfway between 1.0 (0x38) and 1.125 (0x39): the even code 0x38; between 1.125 and 1.25 (0x3A): the even code 0x3A
+    assert enc(1.0625, 1.1875, -1.0625, -1.1875) == [0x38, 0x3A, 0xB8, 0xBA]
+    assert enc(1.0625 + 1e-9, 1.0625 - 1e-9, 1.1875 - 1e-9) == [0x39, 0x38, 0x39]
+    # across a binade: 1.875 (0x3F) | 2.0 (0x40): halfway 1.9375 -> even code 0x40
+    assert enc(1.9375, 1.93, 1.94) == [0x40, 0x3F, 0x40]
+    # subnormals: half the smallest step ties to zero, one and a half steps tie to code 2
+    assert enc(2.0 ** -10, 3 * 2.0 ** -10, 2.0 ** -10 + 1e-12, 2.0 ** -11) == [0x00, 0x02, 0x01, 0x00]
+    # the last normal step of the subnormal range: 7/8 * 2^-6 (0x07) | 2^-6 (0x08)
+    assert enc(7.5 * 2.0 ** -9) == [0x08]
+    # saturation instead of NaN / infinity; NaN stays NaN
+    assert enc(448.0, 449.0, 480.0, 1e30, -1e30, np.inf) == [0x7E, 0x7E, 0x7E, 0x7E, 0xFE, 0x7E]
+    assert enc(np.nan) == [0x7F] and enc(-0.0) == [0x80]
+
+
+def test_p17_e4m3_encode_agrees_with_the_library_cast():
+    """An independent implementation of the same rounding: torch's float8_e4m3fn cast (CPU).  It does not saturate, so
+    the comparison is made where no saturation occurs (|x| <= 448)."""
+    import torch
+    rng = np.random.default_rng(171)
+    x = np.concatenate([rng.standard_normal(200000) * rng.choice([1e-3, 0.02, 1.0, 50.0, 150.0], 200000),
+                        np.linspace(-448.0, 448.0, 20001), oracle.e4m3_decode(np.arange(0, 127, dtype=np.uint8)),
+                        0.5 * (oracle.e4m3_decode(np.arange(0, 126, dtype=np.uint8)) + oracle.e4m3_decode(np.arange(1, 127, dtype=np.uint8)))])
+    x = x[np.abs(x) <= 448.0]
+    ours = oracle.e4m3_encode(x)
+    lib = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(ours, lib)
+
+
+def test_p17_row_scales_and_round_trip():
+    rng = np.random.default_rng(172)
+    Wm = (rng.standard_normal((40, 256)) * 0.02 * rng.choice([1e-3, 1.0, 30.0], (40, 1))).astype(np.float32)
+    Wm[3] = 0.0                               # an all-zero row
+    Wm[4, :] = 0.0
+    Wm[4, 7] = 448.0 * 2.0 ** -5              # row maximum exactly 448 * 2^k: the scale is 2^k, the code 0x7E
+    q, s = oracle.quantize_e4m3_rows(Wm)
+    assert q.shape == Wm.shape and q.dtype == np.uint8 and s.shape == (40,) and s.dtype == np.float32
+    m, _ = np.frexp(s.astype(np.float64))
+    assert (m == 0.5).all()                                              # powers of two
+    assert s[3] == 1.0 and (q[3] & 0x7F).max() == 0 and s[4] == np.float32(2.0 ** -5) and q[4, 7] == 0x7E
+    scaled_max = np.abs(Wm.astype(np.float64)).max(axis=1) / s
+    nz = scaled_max > 0
+    assert (scaled_max[nz] > 224.0).all() and (scaled_max[nz] <= 448.0).all()    # the largest element lands in the top binade
+    back = oracle.dequantize_e4m3_rows(q, s)
+    assert back.dtype == np.float32
+    err = np.abs(back.astype(np.float64) - Wm)
+    # nearest value: half a step of 4 significant bits where the scaled value is normal, half a subnormal step below
+    bound = np.maximum(2.0 ** -4 * np.abs(Wm), 2.0 ** -10 * s[:, None])
+    assert (err <= bound).all() and err.max() > 0
+    # dequantised weights are a fixed point of quantise -> dequantise (the codes may move by one exponent step where a
+    # row's maximum rounded down to 224 * s, which the scale rule then reads as 448 * s/2; the VALUES do not move)
+    q2, s2 = oracle.quantize_e4m3_rows(back)
+    assert np.array_equal(oracle.dequantize_e4m3_rows(q2, s2), back)
+    assert ((s2 == s) | (s2 == s / 2)).all() and (s2 == s).sum() >= 30
+    # and they are bf16 values (four significant bits times a power of two), so the GPU's bf16 kernels can take them as they are
+    assert np.array_equal(W.bf16_round(back), back)
+    # batched shapes quantise row by row
+    q3, s3 = oracle.quantize_e4m3_rows(Wm.reshape(4, 10, 256))
+    assert np.array_equal(q3.reshape(40, 256), q) and np.array_equal(s3.reshape(40), s)
+
+
+def test_p17_layer_on_quantised_weights_is_the_layer_on_their_dequantised_values():
+    """The layer at the second precision is defined through the same equations on s_r * q_rj; with weights that are
+    already representable (scale 1) it IS the bf16 layer, and in general it stays close to it: the per-weight relative
+    error of at most 2^-4 averages out over the d-term dot products."""
+    wl = W.make_layer("tiny", 4, variant=17)
+    s = wl.shape
+
+    def deq(w):
+        return oracle.dequantize_e4m3_rows(*oracle.quantize_e4m3_rows(w))
+
+    kw = dict(h=wl.h, w_router=wl.w_router, lore_A=wl.lore()[0], lore_B=wl.lore()[1], resident=wl.resident, conf=wl.conf,
+              top_k=s.top_k, tau=s.tau)
+    base = oracle.layer(experts=[wl.expert(e) for e in range(s.n_experts)], shared=wl.shared(), **kw)
+    q8 = oracle.layer(experts=[tuple(deq(w) for w in wl.expert(e)) for e in range(s.n_experts)],
+                      shared=tuple(deq(w) for w in wl.shared()), **kw)
+    assert np.array_equal(q8.idx, base.idx) and np.array_equal(q8.cls, base.cls) and np.array_equal(q8.gate, base.gate)
+    rel = np.abs(q8.y - base.y).max() / np.abs(base.y).max()
+    assert 1e-4 < rel < 0.1, rel
+    # representable weights: quantisation is the identity, so the two layers coincide bit for bit
+    rep = [tuple(deq(w) for w in wl.expert(e)) for e in range(s.n_experts)]
+    again = oracle.layer(experts=[tuple(deq(w) for w in ws) for ws in rep], shared=tuple(deq(deq(w)) for w in wl.shared()), **kw)
+    assert np.array_equal(again.y, q8.y)
