@@ -36,7 +36,18 @@
 // ordered by a fence.proxy.async between the reader's acquire and its TMA copies.  Every wait in the kernel is bounded; on expiry
 // the CTA records SPICE_ERR_TIMEOUT, raises the abort flag, drains its copies in flight, frees
 // its TMEM and returns.  No load uses cluster multicast.
+//
+// Second weight precision (decode_tc_kernel<NB, true>): the routed and shared expert weights are E4M3 bytes with one
+// fp32 scale per output row (half the bytes of bf16 on the path that is bound by them).  The MMA then runs as
+// kind::f8f6f4 with the weights as E4M3 on the M side; the bf16 activations on the N side are written as the exact sum
+// of three E5M2 terms (a bf16 has 8 significant bits, an E5M2 three: hi = rn(x), mid = rn(x - hi), lo = rn(x - hi - mid)
+// reproduces every bf16 of magnitude 2^-7 .. 57344 exactly and smaller ones to 2^-17 absolute), each term in its own
+// group of N columns, so the token side grows from NB to 3 NB columns -- an MMA still takes the same time -- and the
+// epilogue adds the three accumulators and applies the row scale.  Nothing is converted per weight element.  The LoRE
+// factors and the router stay bf16 (kind::f16 tasks of the same kernel).  A ring stage holds 256 reduction elements of
+// such a task (the same 32 KB of weights as 128 bf16 elements).
 #include <cuda.h>
+#include <cuda_fp8.h>
 
 #include "route_device.cuh"
 #include "spice_internal.cuh"
@@ -52,15 +63,18 @@ constexpr int DTC_THREADS = 448;
 constexpr int AUX_T0 = 192, AUX_T = 256, AUX_W = 8;
 constexpr int MAX_STAGES = 5, TQ = 4;   // deeper rings only lengthen the memory queues (every fence waits behind them)
 constexpr int KSTAGE = 128;                 // reduction elements per ring stage: two 64-element sub-chunks
+constexpr int KSTAGE8 = 256;                // the same for 8-bit weights: two 128-element sub-chunks
 constexpr int SUB_A = 128 * 64 * 2;         // weight bytes of one sub-chunk
 constexpr int A_BYTES = 2 * SUB_A;
 constexpr int MAX_SPLIT = 16, CHUNKS_PER_SPLIT = 16;
 
 enum { TASK_EXIT = 0, TASK_ACT = 1, TASK_Z = 2, TASK_DOWN = 3 };
-enum { MAP_H = 0, MAP_SLOT_GU, MAP_SH_GU, MAP_LORE_A, MAP_SLOT_D, MAP_SH_D, MAP_LORE_B, MAP_ACT_HIT, MAP_ACT_SH, MAP_Z, N_MAPS };
+enum { MAP_H = 0, MAP_SLOT_GU, MAP_SH_GU, MAP_LORE_A, MAP_SLOT_D, MAP_SH_D, MAP_LORE_B, MAP_ACT_HIT, MAP_ACT_SH, MAP_Z, MAP_X8, N_MAPS };
 
 struct TaskDesc {
-    int32_t kind, gi, tile, split, nk, pad0, pad1, pad2;
+    int32_t kind, gi, tile, split, nk;
+    int32_t f8;     // 8-bit weights: kind::f8f6f4, three token column groups, 256-element stages
+    int32_t pad1, pad2;
 };
 
 struct DtcParams {
@@ -70,6 +84,10 @@ struct DtcParams {
     int32_t nsplit_sh;   // K ranges of the shared down projection
     int32_t cps_sh;      // k-chunks per range
     int32_t r1_sub;      // token subsets per expert in the router-logit units
+    // 8-bit weight precision (decode_tc_kernel<NB, true>): row scales, and the activations as three E5M2 planes
+    const float *s_slot_gu, *s_slot_d, *s_sh_gu, *s_sh_d;   // [S,2I], [S,d], [2Is], [d]
+    uint8_t *act8_hit;   // [group][3][T][I]
+    uint8_t *act8_sh;    // [3][T][Is]
 };
 struct DtcMaps {
     CUtensorMap m[N_MAPS];
@@ -143,7 +161,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
 }
 
 __host__ __device__ inline int nb_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : 64); }
-__host__ __device__ inline int stage_bytes_of(int nb) { return A_BYTES + 2 * nb * 128; }
+__host__ __device__ inline int stage_bytes_of(int nb, bool f8 = false) { return A_BYTES + (f8 ? 6 : 2) * nb * 128; }
 
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ int ld_acquire(const int *p) {
@@ -260,23 +278,24 @@ __device__ __forceinline__ bool warp_mb_wait(uint32_t a, uint32_t parity, volati
 // Task list.  ids [0, nA) are known at launch; the rest once the routing tables exist.
 struct Plan {
     int tIs, tI, tz, td;            // tiles per matrix
-    int kcd, kcI, kcr;              // k-chunks (one ring stage = 128 elements) of d, I, r
+    int kcd, kcI, kcr, kcdz;        // ring stages of d, I (expert matrices), r and d (LoRE factors)
     int nsplit, cps, kcIs;          // shared down projection: K ranges, chunks per range, chunks in all
     int nA, nBh, endB, nCs, nCh, endC;
     int n_hg, n_lg;
     int sh_early;                   // the shared down tiles are part of phase A (else they follow phase B)
 };
 
-__device__ __forceinline__ void plan_static(Plan &pl, const DtcParams &q) {
+__device__ __forceinline__ void plan_static(Plan &pl, const DtcParams &q, int kst = KSTAGE) {
     const Dims &dm = q.p.dm;
     pl.tIs = (dm.Is + 63) >> 6;
     pl.tI = (dm.I + 63) >> 6;
     pl.tz = (dm.r + 127) >> 7;
     pl.td = (dm.d + 127) >> 7;
-    pl.kcd = (dm.d + KSTAGE - 1) / KSTAGE;
-    pl.kcI = (dm.I + KSTAGE - 1) / KSTAGE;
-    pl.kcr = (dm.r + KSTAGE - 1) / KSTAGE;
-    pl.kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
+    pl.kcd = (dm.d + kst - 1) / kst;           // stages of the expert matrices (kst = 256 for 8-bit weights)
+    pl.kcI = (dm.I + kst - 1) / kst;
+    pl.kcr = (dm.r + KSTAGE - 1) / KSTAGE;     // the LoRE factors are bf16 in either precision
+    pl.kcdz = (dm.d + KSTAGE - 1) / KSTAGE;
+    pl.kcIs = (dm.Is + kst - 1) / kst;
     pl.nsplit = q.nsplit_sh;
     pl.cps = q.cps_sh;
     pl.nCs = pl.td * pl.nsplit;
@@ -664,12 +683,26 @@ __device__ __forceinline__ void aux_combine(const DtcParams &q, const AuxSmem &a
 }
 
 // ------------------------------------------------------------------------------------------
-template <int NB>
+// three E5M2 terms whose sum is the bf16 value x (exactly for 2^-7 <= |x| <= 57344): bytes hi | mid << 8 | lo << 16
+__device__ __forceinline__ uint32_t split_e5m2x3(float x) {
+    uint32_t out = 0;
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        const __nv_fp8_storage_t b = __nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E5M2);
+        out |= (uint32_t)b << (8 * j);
+        x -= __half2float(__half(__nv_cvt_fp8_to_halfraw(b, __NV_E5M2)));   // exact: both have few significant bits
+    }
+    return out;
+}
+
+template <int NB, bool F8 = false>
 __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_constant__ DtcParams q,
                                                                    const __grid_constant__ DtcMaps maps) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    constexpr int STAGE_BYTES = A_BYTES + 2 * NB * 128;
-    constexpr int TMEM_COLS = 2 * NB < 32 ? 32 : 2 * NB;
+    constexpr int STAGE_BYTES = A_BYTES + (F8 ? 6 : 2) * NB * 128;   // (stage pitch; a bf16 task of the 8-bit kernel fills less)
+    constexpr int ACC = F8 ? 3 * NB : NB;                              // accumulator columns of one buffer
+    constexpr int TMEM_COLS = 2 * ACC <= 32 ? 32 : (2 * ACC <= 64 ? 64 : (2 * ACC <= 128 ? 128 : (2 * ACC <= 256 ? 256 : 512)));
+    constexpr int KST = F8 ? KSTAGE8 : KSTAGE;
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
     unsigned char *ring = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -732,7 +765,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         constexpr unsigned PM = 0xFu;
         if (lane < 4) {
             Plan pl;
-            plan_static(pl, q);
+            plan_static(pl, q, KST);
             bool routed = false;
             int npf = 0;
             if (lane == 0) DPROF(0, npf, 1);
@@ -771,8 +804,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     t.kind = TASK_ACT;
                     t.tile = id;
                     t.nk = pl.kcd;
+                    t.f8 = F8;
                     ma = &maps.m[MAP_SH_GU];
-                    mb = &maps.m[MAP_H];
+                    mb = &maps.m[F8 ? MAP_X8 : MAP_H];
                     a_row0 = t.tile * 64;
                 } else if (sh_down) {                    // down tile of the shared expert, one K range
                     const int l = id - (pl.sh_early ? pl.tIs : pl.endB);
@@ -781,6 +815,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     t.split = l / pl.td;
                     k0 = t.split * pl.cps;
                     t.nk = min(pl.cps, pl.kcIs - k0);
+                    t.f8 = F8;
                     ma = &maps.m[MAP_SH_D];
                     mb = &maps.m[MAP_ACT_SH];
                     a_row0 = t.tile * 128;
@@ -792,8 +827,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     t.gi = 1 + l / pl.tI;
                     t.tile = l % pl.tI;
                     t.nk = pl.kcd;
+                    t.f8 = F8;
                     ma = &maps.m[MAP_SLOT_GU];
-                    mb = &maps.m[MAP_H];
+                    mb = &maps.m[F8 ? MAP_X8 : MAP_H];
                     a_row0 = t.tile * 64;
                     a_z = ax.gtab[t.gi].id;
                 } else if (id < pl.endB) {               // A_e tile of a low-confidence expert
@@ -801,7 +837,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     t.kind = TASK_Z;
                     t.gi = 1 + pl.n_hg + l / pl.tz;
                     t.tile = l % pl.tz;
-                    t.nk = pl.kcd;
+                    t.nk = pl.kcdz;
                     ma = &maps.m[MAP_LORE_A];
                     mb = &maps.m[MAP_H];
                     a_row0 = t.tile * 128;
@@ -812,6 +848,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     t.gi = 1 + l / pl.td;
                     t.tile = l % pl.td;
                     t.nk = pl.kcI;
+                    t.f8 = F8;
                     ma = &maps.m[MAP_SLOT_D];
                     mb = &maps.m[MAP_ACT_HIT];
                     a_row0 = t.tile * 128;
@@ -843,6 +880,8 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 const int my_y = is_b ? 0 : a_row0;
                 const int my_z = is_b ? b_z : a_z;
                 const bool my_on = sub == 0 || plain;
+                // bytes a stage of this task receives (a bf16 task of the 8-bit kernel leaves part of the token area unused)
+                const uint32_t tx_bytes = (F8 && !t.f8) ? (uint32_t)(A_BYTES + 2 * NB * 128) : (uint32_t)STAGE_BYTES;
                 auto copy = [&](int kb, int stage) {   // this lane's box of k-stage kb into ring stage `stage`
                     const uint32_t full = smem_u32(&sh->full[stage]);
                     const uint32_t dst = smem_u32(ring + (size_t)stage * STAGE_BYTES);
@@ -877,7 +916,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     const int s0 = s;
                     for (int kb = 0; kb < pre && ok; ++kb, ++it) {
                         if (!lead_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1)) { ok = false; break; }
-                        if (lane == 0) mbar_expect_tx(smem_u32(&sh->full[s]), STAGE_BYTES);
+                        if (lane == 0) mbar_expect_tx(smem_u32(&sh->full[s]), tx_bytes);
                         __syncwarp(PM);
                         if (my_on && !is_b) copy(kb, s);
                         if (++s == stages) {
@@ -905,7 +944,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 if (lane == 0) drawn = (int)gridDim.x + atomicAdd(p.sync + SY_NEXT_TASK, 1);
                 for (int kb = kb0; kb < t.nk; ++kb, ++it) {
                     if (!lead_wait(smem_u32(&sh->empty[s]), ring_phase ^ 1)) { ok = false; break; }
-                    if (lane == 0) mbar_expect_tx(smem_u32(&sh->full[s]), STAGE_BYTES);
+                    if (lane == 0) mbar_expect_tx(smem_u32(&sh->full[s]), tx_bytes);
                     __syncwarp(PM);
                     if (my_on) copy(kb, s);
 #ifdef SPICE_PROF_STAGES
@@ -946,6 +985,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         // ---------------- MMA issuer (one lane)
         if (lane == 0) {
             constexpr uint32_t IDESC = make_idesc(128, NB);
+            constexpr uint32_t IDESC8 = make_idesc_e4m3_e5m2(128, 3 * NB);
 #ifdef SPICE_PROF_STAGES
             int npf_m = 0;
 #endif
@@ -955,11 +995,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 const int slot = tcount % TQ;
                 if (!mb_wait(smem_u32(&sh->tq_full[slot]), (tcount / TQ) & 1, abort_flag)) break;
                 const int kind = sh->tq[slot].kind, nk = sh->tq[slot].nk;
+                const bool f8 = F8 && sh->tq[slot].f8 != 0;
                 if (kind == TASK_EXIT) break;
                 const int buf = tcount & 1;
                 if (!mb_wait(smem_u32(&sh->tmem_empty[buf]), ((tcount >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * NB;
+                const uint32_t d_tmem = tmem_base + buf * ACC;
                 bool ok = true;
                 for (int kb = 0; kb < nk; ++kb) {
                     if (!mb_wait(smem_u32(&sh->full[s]), ring_phase, abort_flag)) { ok = false; break; }
@@ -968,11 +1009,20 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
 #endif
                     tc_fence_after();
                     const uint32_t a0 = smem_u32(ring + (size_t)s * STAGE_BYTES), b0 = a0 + A_BYTES;
+                    if (f8) {   // 32 one-byte elements per instruction: the same 32-byte steps through a 128-byte row
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const uint64_t da = make_desc(a0 + c * SUB_A), db = make_desc(b0 + c * NB * 128);
+                        for (int c = 0; c < 2; ++c) {
+                            const uint64_t da = make_desc(a0 + c * SUB_A), db = make_desc(b0 + c * 3 * NB * 128);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | c | k) ? 1u : 0u);
+                            for (int k = 0; k < 4; ++k) tc_mma_f8(d_tmem, da + 2 * k, db + 2 * k, IDESC8, (kb | c | k) ? 1u : 0u);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            const uint64_t da = make_desc(a0 + c * SUB_A), db = make_desc(b0 + c * NB * 128);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) tc_mma(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | c | k) ? 1u : 0u);
+                        }
                     }
                     tc_commit(smem_u32(&sh->empty[s]));
                     if (++s == stages) {
@@ -1007,9 +1057,23 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             if (warp == 2 && lane == 0) DPROF(1, npf, 54);
             tc_fence_after();
             uint32_t v[NB];
-            const uint32_t t0 = tmem_base + buf * NB + ((uint32_t)(qd * 32) << 16);
+            const uint32_t t0 = tmem_base + buf * ACC + ((uint32_t)(qd * 32) << 16);
+            if (F8 && t.f8) {   // (warp-uniform) three accumulators per token: hi, mid and lo term of the activations
 #pragma unroll
-            for (int c = 0; c < NB; c += 16) tc_ld16(t0 + c, &v[c]);
+                for (int c = 0; c < NB; c += 16) {
+                    uint32_t m1[16], m2[16];
+                    tc_ld16(t0 + c, &v[c]);
+                    tc_ld16(t0 + NB + c, m1);
+                    tc_ld16(t0 + 2 * NB + c, m2);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        v[c + j] = __float_as_uint((__uint_as_float(v[c + j]) + __uint_as_float(m1[j])) + __uint_as_float(m2[j]));
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < NB; c += 16) tc_ld16(t0 + c, &v[c]);
+            }
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
@@ -1023,20 +1087,45 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 __nv_bfloat16 *out = hit ? p.act_hit16 + (size_t)(t.gi - 1) * T * dm.I : p.act_shared16;
                 const int xb = xc & 1;
                 float *xch = ax.xch + xb * NB * 64;
+                // 8-bit weights: scale of this thread's weight row (gate rows first, then the up rows)
+                float rs = 1.0f;
+                if (F8) {
+                    const int col = t.tile * 64 + (L & 63);
+                    const float *sc = hit ? q.s_slot_gu + (size_t)grp.id * 2 * dm.I : q.s_sh_gu;
+                    rs = col < n_cols ? sc[(qd >= 2 ? n_cols : 0) + col] : 0.0f;
+                }
                 if (qd >= 2) {   // up rows: park them for the warps that hold the gate rows
                     if (!warp_mb_wait(smem_u32(&sh->xch_empty[xb]), ((xc >> 1) & 1) ^ 1, abort_flag, lane)) break;
 #pragma unroll
-                    for (int nn = 0; nn < NB; ++nn) xch[nn * 64 + (L - 64)] = __uint_as_float(v[nn]);
+                    for (int nn = 0; nn < NB; ++nn) xch[nn * 64 + (L - 64)] = F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&sh->xch_full[xb]));
                 } else {
                     if (!warp_mb_wait(smem_u32(&sh->xch_full[xb]), (xc >> 1) & 1, abort_flag, lane)) break;
                     const int col = t.tile * 64 + L;
+                    if (F8) {
+                        // the activation, rounded to bf16 as in the 16-bit kernel, stored as its three E5M2 terms
+                        uint8_t *out8 = hit ? q.act8_hit + (size_t)(t.gi - 1) * 3 * T * dm.I : q.act8_sh;
+                        const size_t plane = (size_t)T * n_cols;
 #pragma unroll
-                    for (int nn = 0; nn < NB; ++nn) {
-                        if (nn < T && col < n_cols) {
-                            const float u = xch[nn * 64 + L];
-                            out[(size_t)nn * n_cols + col] = __float2bfloat16(silu_f(__uint_as_float(v[nn])) * u);
+                        for (int nn = 0; nn < NB; ++nn) {
+                            if (nn < T && col < n_cols) {
+                                const float u = xch[nn * 64 + L];
+                                const float a = __bfloat162float(__float2bfloat16(silu_f(__uint_as_float(v[nn]) * rs) * u));
+                                const uint32_t b3 = split_e5m2x3(a);
+                                uint8_t *o = out8 + (size_t)nn * n_cols + col;
+                                o[0] = (uint8_t)b3;
+                                o[plane] = (uint8_t)(b3 >> 8);
+                                o[2 * plane] = (uint8_t)(b3 >> 16);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int nn = 0; nn < NB; ++nn) {
+                            if (nn < T && col < n_cols) {
+                                const float u = xch[nn * 64 + L];
+                                out[(size_t)nn * n_cols + col] = __float2bfloat16(silu_f(__uint_as_float(v[nn])) * u);
+                            }
                         }
                     }
                     __syncwarp();
@@ -1066,10 +1155,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 __syncwarp();
                 const int row = t.tile * 128 + L;
                 float *out = grp.kind == KIND_SHARED ? q.part_split + (size_t)t.split * T * dm.d : p.tb.part;
+                float rs = 1.0f;
+                if (F8 && t.f8 && row < dm.d) rs = grp.kind == KIND_SHARED ? q.s_sh_d[row] : q.s_slot_d[(size_t)grp.id * dm.d + row];
 #pragma unroll
                 for (int nn = 0; nn < NB; ++nn) {
                     const int e = ent[nn];
-                    if (e >= 0 && row < dm.d) out[(size_t)e * dm.d + row] = __uint_as_float(v[nn]);
+                    if (e >= 0 && row < dm.d) out[(size_t)e * dm.d + row] = F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]);
                 }
                 __syncwarp();   // ent[] is rewritten by the next down tile
             }
@@ -1128,7 +1219,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             APROF(a, 64);
             if (blockIdx.x == 0) aux_write_outputs(q, sh, ax, a);
             Plan pl;
-            plan_static(pl, q);
+            plan_static(pl, q, KST);
             plan_routed(pl, sh->n_hg, sh->n_lg);
             // Warp 1 of the auxiliary team (warp 7 of the CTA) watches the per-group counters while the weights stream, so that the producer finds a flag in
             // shared memory instead of paying a round trip to L2 when it reaches a down tile.  It ends when every

@@ -41,8 +41,11 @@ def test_lore_calibration_reaches_the_oracle_objective(d, n, r, ridge):
     assert got >= loss_ref * (1 - 1e-6) - 1e-9 * total or ridge > 0
     assert got <= loss_ref * 1.01 + 2e-4 * total, (got, loss_ref, total)
     # the fitted map itself (unique when the singular values are distinct): B A against the oracle's
+    # The returned factors are bf16: each entry of B A carries at most 2^-8 * sum_k |B_ik| |A_kj| of rounding
+    # (2^-9 per factor), measured 2.6e-3 .. 3.8e-3 of max|B A| on these cases -- inside the output tolerance.
     diff = np.abs(Bm @ A - B_ref @ A_ref).max()
-    assert diff <= 2e-2 * np.abs(B_ref @ A_ref).max() + 1e-3
+    assert diff <= 1e-2 * np.abs(B_ref @ A_ref).max() + 1e-3
+    assert diff <= 2.0 ** -8 * (np.abs(B_ref) @ np.abs(A_ref)).max() + 1e-3 * np.abs(B_ref @ A_ref).max()
 
 
 def test_lore_calibration_recovers_an_exactly_low_rank_residual():
@@ -54,7 +57,7 @@ def test_lore_calibration_recovers_an_exactly_low_rank_residual():
     A, Bm, loss_dev, status = _fit(H, R, r)
     total = float((R ** 2).sum())
     assert status == 0 and _objective(H, R, A, Bm) <= 1e-4 * total       # bf16 rounding of the factors: ~2^-16 relative
-    assert np.abs(Bm @ A - B0 @ A0).max() <= 2e-2 * np.abs(B0 @ A0).max()
+    assert np.abs(Bm @ A - B0 @ A0).max() <= 1e-2 * np.abs(B0 @ A0).max() + 1e-3
 
 
 def test_lore_calibration_flags_a_singular_gram_matrix_and_checks_arguments():
