@@ -36,7 +36,7 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised under
 # profiles/ (same workload with 2 weight sets; mean of the two captured launches), keyed by (shape, tokens, path)
-CAPTURED_TRAFFIC = {("dsv2lite", 16, 0): (492.6e6, "profiles/decode_tc_kernel_dsv2lite_T16.md")}
+CAPTURED_TRAFFIC = {("dsv2lite", 16, 0, "bf16"): (492.6e6, "profiles/decode_tc_kernel_dsv2lite_T16.md")}
 
 
 def load_peaks():
@@ -117,13 +117,18 @@ def whole_job_throughput(units_per_rank_per_step, steps, world, ms_max):
 
 
 # ----------------------------------------------------------------------------- workload
-def algorithmic_bytes(shape, T, idx, cls):
-    """Bytes the method must move for one layer call (bf16 weights read once per distinct expert)."""
+def algorithmic_bytes(shape, T, idx, cls, fp8=False):
+    """Bytes the method must move for one layer call (weights read once per distinct expert: bf16, or for fp8 one byte
+    per expert weight plus a 4-byte scale per weight row; router and LoRE factors are bf16 in both)."""
     s = shape
     hit = {int(e) for e, c in zip(idx.ravel(), cls.ravel()) if c == 0}
     low = {int(e) for e, c in zip(idx.ravel(), cls.ravel()) if c == 2}
-    w = 2 * (s.n_experts * s.d + 3 * s.d * s.inter_shared + len(hit) * 3 * s.d * s.inter
-             + len(low) * 2 * s.lore_rank * s.d)
+    expert_w = 3 * s.d * s.inter_shared + len(hit) * 3 * s.d * s.inter
+    if fp8:
+        expert_w = expert_w + 4 * ((2 * s.inter_shared + s.d) + len(hit) * (2 * s.inter + s.d))
+    else:
+        expert_w = 2 * expert_w
+    w = 2 * (s.n_experts * s.d + len(low) * 2 * s.lore_rank * s.d) + expert_w
     act = 2 * T * s.d + 2 * T * s.d + 4 * T * s.top_k
     return w + act, len(hit), len(low)
 
@@ -182,7 +187,12 @@ def run_ours(args):
     if zipf:
         for r in reps[1:]:
             r.w_router.copy_(reps[0].w_router)   # same popularity skew in every weight set
+    fp8 = args.dtype == "fp8"
+    if fp8:
+        reps = [B.quantize_layer(r) for r in reps]      # the bf16 sets are released once quantised
+        torch.cuda.synchronize()
     structs = [r.c_struct() for r in reps]
+    layer_call = B.spice_moe_layer_fwd_fp8 if fp8 else B.spice_moe_layer_fwd
     h = bf16_tensor(wl0.h, dev)
     conf = torch.from_numpy(wl0.conf).to(dev)
     layer = B.SpiceLayer(cfg_of(shape), T, device=local)
@@ -200,7 +210,7 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     def step(i):
-        B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h, conf, T, y, idx=idx, gate=gate, cls=cls, counts=counts,
+        layer_call(layer.ctx, structs[i % R], h, conf, T, y, idx=idx, gate=gate, cls=cls, counts=counts,
                               resid_tok=resid[0], resid_k=resid[1], resid_expert=resid[2], resid_gate=resid[3],
                               stream=torch.cuda.current_stream())
 
@@ -209,7 +219,7 @@ def run_ours(args):
     for i in range(R):
         step(i)
         torch.cuda.synchronize()
-        b, nh, nl = algorithmic_bytes(shape, T, idx.cpu().numpy(), cls.cpu().numpy())
+        b, nh, nl = algorithmic_bytes(shape, T, idx.cpu().numpy(), cls.cpu().numpy(), fp8)
         rep_bytes.append(b)
         rep_hit.append(nh)
         rep_low.append(nl)
@@ -255,7 +265,7 @@ def run_ours(args):
     def e2e_enqueue(i):
         st = torch.cuda.current_stream()
         in_dev.copy_(in_host, non_blocking=True)
-        B.spice_moe_layer_fwd(layer.ctx, structs[i % R], h_dev, conf_dev, T, y_e2e, idx=idx, gate=gate, cls=cls,
+        layer_call(layer.ctx, structs[i % R], h_dev, conf_dev, T, y_e2e, idx=idx, gate=gate, cls=cls,
                               counts=cnt_e2e, resid_tok=resid_e2e[0], resid_k=resid_e2e[1], resid_expert=resid_e2e[2],
                               resid_gate=resid_e2e[3], stream=st)
         out_host.copy_(out_dev, non_blocking=True)
@@ -313,11 +323,13 @@ def run_ours(args):
         out = {
             "metric": METRIC, "value": tok_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": "fp8_e4m3_weights_bf16_activations" if fp8 else "bf16", "data": "synthetic",
             "config": {"workload": f"{shape.name} decode layer, batch {T} tokens "
                                    f"(d={shape.d}, N={shape.n_experts}, K={shape.top_k}, I={shape.inter}, "
                                    f"I_s={shape.inter_shared}, r={shape.lore_rank}, {shape.n_slots} resident slots, "
                                    f"tau={shape.tau}, Beta(2,2) confidences)",
+                       "weights": ("expert and shared-expert matrices as E4M3 bytes with one power-of-two scale per row "
+                                   "(quantised on the device from the bf16 sets); router and LoRE factors bf16") if fp8 else "bf16",
                        "tokens_per_step": T, "cold_l2": f"steps rotate through {R} independent weight sets "
                        f"({sum(rep_bytes) / 1e6:.0f} MB between reuses, L2 is 126 MB); no flush in the timed region",
                        "launch": how,
@@ -326,8 +338,8 @@ def run_ours(args):
                        "multi_gpu": "replicas only (no collective on the data path)"},
             "roofline": ({"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                           "frac": achieved / peaks["hbm_gbs"],
-                          "traffic": CAPTURED_TRAFFIC.get((shape.name, T, args.path), (None, None))[0],
-                          "traffic_source": CAPTURED_TRAFFIC.get((shape.name, T, args.path), (None, None))[1],
+                          "traffic": CAPTURED_TRAFFIC.get((shape.name, T, args.path, args.dtype), (None, None))[0],
+                          "traffic_source": CAPTURED_TRAFFIC.get((shape.name, T, args.path, args.dtype), (None, None))[1],
                           "kernel": "all launches of spice_moe_layer_fwd (algorithmic bytes of the call / time per call)",
                           "algorithmic_bytes_per_step": total_bytes / args.steps, "peak_source": peaks["source"],
                           "frac_of_nominal_8TBs": achieved / 8000.0} if not prefill else
@@ -819,6 +831,9 @@ def main():
                     help="how the timed steps are submitted: replayed CUDA graphs of captured steps, or one library call per "
                          "step; auto = graphs for decode batches (one kernel per step, launch-bound), calls for batches "
                          "above 64 tokens (a dozen kernels on two streams per step)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp8"],
+                    help="weight precision of the expert matrices: bf16, or fp8 = E4M3 bytes with a scale per row "
+                         "(spice_moe_layer_fwd_fp8; decode batches up to 32 tokens)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--cpu-leg", type=int, default=None, help=argparse.SUPPRESS)   # child of cpu_baseline_one_thread

@@ -211,6 +211,51 @@ spice_status spice_lore_calibrate(int32_t d, int32_t n_tokens, int32_t rank, flo
                                   float *loss_out, int32_t *device_status, void *workspace, size_t workspace_bytes,
                                   void *stream);
 
+/* ---- Second weight precision: 8-bit expert weights (the paper reports every result at BF16 and at one quantised
+ * precision, Sec. 5.1 and Table 1, and names that format without defining it).  Reading taken by this library: the
+ * matrices of the routed experts and of the shared expert are stored as E4M3 bytes (1 sign, 4 exponent bits with bias 7,
+ * 3 fraction bits; no infinities, S.1111.111 is NaN, largest value 448) with ONE fp32 scale per output row; the weight
+ * the layer computes with is scale[row] * value(code).  Router and LoRE factors keep bf16, so routing and classification
+ * do not depend on the precision.  Activations stay bf16 (inputs, the intermediate silu(g)*u, outputs): the layer at this
+ * precision is, by definition, spice_moe_layer_fwd on the dequantised weights.  Half the weight bytes cross HBM. */
+typedef struct {
+    const spice_bf16 *w_router;         /* [N, d] bf16                                       */
+    const uint8_t *slot_q_gate_up;      /* [S, 2I, d] E4M3: I gate rows, then I up rows      */
+    const float *slot_s_gate_up;        /* [S, 2I] row scales                                */
+    const uint8_t *slot_q_down;         /* [S, d, I] E4M3                                    */
+    const float *slot_s_down;           /* [S, d]                                            */
+    const int32_t *slot_of_expert;      /* [N]; slot index, or -1 when not resident          */
+    const uint8_t *shared_q_gate_up;    /* [2 I_s, d] E4M3                                   */
+    const float *shared_s_gate_up;      /* [2 I_s]                                           */
+    const uint8_t *shared_q_down;       /* [d, I_s] E4M3                                     */
+    const float *shared_s_down;         /* [d]                                               */
+    const spice_bf16 *lore_A;           /* [N, r, d] bf16                                    */
+    const spice_bf16 *lore_B;           /* [N, d, r] bf16                                    */
+} spice_layer_weights_fp8;
+
+/* Quantiser of that format: for each of `rows` rows of the bf16 matrix w [rows, cols] (cols a multiple of 8)
+ *     scale[r] = 2^ceil(log2(max_j |w[r,j]| / 448))   (1 for an all-zero row),
+ *     q[r,j]   = the E4M3 value nearest to w[r,j] / scale[r], ties to the even code, magnitudes above 448 saturate.
+ * w, q [rows, cols] uint8 and scale [rows] fp32 are device pointers owned by the caller (q, scale: out; 16-byte aligned
+ * w and q).  No ctx: the GPU is the calling thread's current device.  Any positive finite scales are accepted by the
+ * layer call; the powers of two written here make the dequantised weights exact in fp32 (and in bf16). */
+spice_status spice_quantize_e4m3_rows(const spice_bf16 *w, int64_t rows, int32_t cols, uint8_t *q, float *scale,
+                                      void *stream);
+
+/* spice_moe_layer_fwd at the 8-bit weight precision; every other argument, every output and every rule (top-k order,
+ * classes, residual list, optional residual inputs) as there.  Covers decode batches: T <= 32, and d, inter and
+ * inter_shared multiples of 128 (SPICE_ERR_UNSUPPORTED_SHAPE otherwise; there is no second kernel path behind it, and
+ * SPICE_ERR_CUDA is returned when the device refuses the cooperative launch).  Two launches: the input activations are
+ * first written as the sum of three E5M2 terms (exact for bf16 magnitudes from 2^-7 to 57344; smaller ones to 2^-17
+ * absolute, larger ones saturate), the same is done with the intermediate activations inside the layer kernel, and the
+ * tensor cores multiply E4M3 weights with those terms (kind::f8f6f4), fp32 accumulation, row scale in the epilogue. */
+spice_status spice_moe_layer_fwd_fp8(spice_ctx *ctx, const spice_layer_weights_fp8 *w /* host struct */,
+                                     const spice_bf16 *h, const float *conf, int32_t T,
+                                     const float *y_cpu_residual, spice_bf16 *x_resid, spice_bf16 *y,
+                                     int32_t *idx, float *gate, uint8_t *cls, int32_t *counts,
+                                     int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
+                                     float *resid_gate, void *stream);
+
 /* The resident-expert FFN for callers that cannot allocate (the paper has no counterpart: this is
  * a packaging variant of spice_grouped_expert_ffn, not a step of the method).
  *

@@ -39,6 +39,14 @@ class LayerWeightsC(C.Structure):
                 ("lore_A", C.c_void_p), ("lore_B", C.c_void_p)]
 
 
+class LayerWeightsFp8C(C.Structure):
+    """Mirror of spice_layer_weights_fp8 (device pointers)."""
+    _fields_ = [("w_router", C.c_void_p), ("slot_q_gate_up", C.c_void_p), ("slot_s_gate_up", C.c_void_p),
+                ("slot_q_down", C.c_void_p), ("slot_s_down", C.c_void_p), ("slot_of_expert", C.c_void_p),
+                ("shared_q_gate_up", C.c_void_p), ("shared_s_gate_up", C.c_void_p), ("shared_q_down", C.c_void_p),
+                ("shared_s_down", C.c_void_p), ("lore_A", C.c_void_p), ("lore_B", C.c_void_p)]
+
+
 _lib = None
 
 
@@ -55,7 +63,8 @@ def lib() -> C.CDLL:
         for name in ("spice_create", "spice_destroy", "spice_workspace_bytes", "spice_route_topk",
                      "spice_classify_misses", "spice_grouped_expert_ffn", "spice_lore_surrogate",
                      "spice_moe_layer_fwd", "spice_get_device_status", "spice_launch_count", "spice_set_option",
-                     "spice_grouped_expert_ffn_static", "spice_draft_confidence", "spice_prefetch_rollout"):
+                     "spice_grouped_expert_ffn_static", "spice_draft_confidence", "spice_prefetch_rollout",
+                     "spice_quantize_e4m3_rows", "spice_moe_layer_fwd_fp8"):
             getattr(L, name).restype = C.c_int
         L.spice_static_scratch_bytes.restype = C.c_size_t
         L.spice_lore_calibrate.restype = C.c_int
@@ -220,6 +229,28 @@ def spice_moe_layer_fwd(ctx, weights: LayerWeightsC, h, conf, T, y, y_cpu_residu
                                      _stream(stream)), "spice_moe_layer_fwd")
 
 
+def spice_quantize_e4m3_rows(w, q, scale, stream=None) -> None:
+    """w [..., cols] bf16 -> q (uint8, same shape) and scale (fp32, shape without the last axis): E4M3 codes with one
+    power-of-two scale per row."""
+    cols = w.shape[-1]
+    rows = w.numel() // cols
+    with torch.cuda.device(w.device):
+        _check(lib().spice_quantize_e4m3_rows(_ptr(w, torch.bfloat16), C.c_int64(rows), C.c_int32(cols), _ptr(q, torch.uint8),
+                                              _ptr(scale, torch.float32), _stream(stream)), "spice_quantize_e4m3_rows")
+
+
+def spice_moe_layer_fwd_fp8(ctx, weights: "LayerWeightsFp8C", h, conf, T, y, y_cpu_residual=None, x_resid=None, idx=None,
+                            gate=None, cls=None, counts=None, resid_tok=None, resid_k=None, resid_expert=None,
+                            resid_gate=None, stream=None) -> None:
+    _check(lib().spice_moe_layer_fwd_fp8(ctx, C.byref(weights), _ptr(h, torch.bfloat16), _ptr(conf, torch.float32),
+                                         C.c_int32(T), _ptr(y_cpu_residual, torch.float32),
+                                         _ptr(x_resid, torch.bfloat16), _ptr(y, torch.bfloat16), _ptr(idx, torch.int32),
+                                         _ptr(gate, torch.float32), _ptr(cls, torch.uint8), _ptr(counts, torch.int32),
+                                         _ptr(resid_tok, torch.int32), _ptr(resid_k, torch.int32),
+                                         _ptr(resid_expert, torch.int32), _ptr(resid_gate, torch.float32),
+                                         _stream(stream)), "spice_moe_layer_fwd_fp8")
+
+
 # ------------------------------------------------------------------ convenience wrappers
 @dataclass
 class LayerWeights:
@@ -238,6 +269,45 @@ class LayerWeights:
                              _ptr(self.slot_w_down, torch.bfloat16), _ptr(self.slot_of_expert, torch.int32),
                              _ptr(self.shared_w_gate_up, torch.bfloat16), _ptr(self.shared_w_down, torch.bfloat16),
                              _ptr(self.lore_A, torch.bfloat16), _ptr(self.lore_B, torch.bfloat16))
+
+
+@dataclass
+class LayerWeightsFp8:
+    """Device tensors of one layer at the 8-bit weight precision; see spice_layer_weights_fp8."""
+    w_router: torch.Tensor          # [N,d] bf16
+    slot_q_gate_up: torch.Tensor    # [S,2I,d] uint8 (E4M3)
+    slot_s_gate_up: torch.Tensor    # [S,2I] fp32
+    slot_q_down: torch.Tensor       # [S,d,I] uint8
+    slot_s_down: torch.Tensor       # [S,d] fp32
+    slot_of_expert: torch.Tensor    # [N] int32
+    shared_q_gate_up: torch.Tensor  # [2Is,d] uint8
+    shared_s_gate_up: torch.Tensor  # [2Is] fp32
+    shared_q_down: torch.Tensor     # [d,Is] uint8
+    shared_s_down: torch.Tensor     # [d] fp32
+    lore_A: torch.Tensor            # [N,r,d] bf16
+    lore_B: torch.Tensor            # [N,d,r] bf16
+
+    def c_struct(self) -> LayerWeightsFp8C:
+        u8, f32, bf = torch.uint8, torch.float32, torch.bfloat16
+        return LayerWeightsFp8C(_ptr(self.w_router, bf), _ptr(self.slot_q_gate_up, u8), _ptr(self.slot_s_gate_up, f32),
+                                _ptr(self.slot_q_down, u8), _ptr(self.slot_s_down, f32), _ptr(self.slot_of_expert, torch.int32),
+                                _ptr(self.shared_q_gate_up, u8), _ptr(self.shared_s_gate_up, f32),
+                                _ptr(self.shared_q_down, u8), _ptr(self.shared_s_down, f32), _ptr(self.lore_A, bf),
+                                _ptr(self.lore_B, bf))
+
+
+def quantize_layer(w: "LayerWeights") -> LayerWeightsFp8:
+    """The 8-bit form of a bf16 weight set: four calls of spice_quantize_e4m3_rows (allocation of the outputs only)."""
+    def qz(t):
+        q = torch.empty(t.shape, dtype=torch.uint8, device=t.device)
+        s = torch.empty(t.shape[:-1], dtype=torch.float32, device=t.device)
+        spice_quantize_e4m3_rows(t, q, s)
+        return q, s
+    sgu, ssgu = qz(w.slot_w_gate_up)
+    sd, ssd = qz(w.slot_w_down)
+    hgu, shgu = qz(w.shared_w_gate_up)
+    hd, shd = qz(w.shared_w_down)
+    return LayerWeightsFp8(w.w_router, sgu, ssgu, sd, ssd, w.slot_of_expert, hgu, shgu, hd, shd, w.lore_A, w.lore_B)
 
 
 @dataclass
@@ -335,6 +405,18 @@ class SpiceLayer:
                          self._empty((n,), torch.float32))
         spice_moe_layer_fwd(self.ctx, w.c_struct(), h, conf, T, o.y, y_cpu_residual, x_resid, o.idx, o.gate, o.cls,
                             o.counts, o.resid_tok, o.resid_k, o.resid_expert, o.resid_gate, stream)
+        return o
+
+    def moe_layer_fwd_fp8(self, w: LayerWeightsFp8, h, conf, y_cpu_residual=None, x_resid=None, stream=None) -> LayerOutputs:
+        T, K, d = h.shape[0], self.cfg.top_k, self.cfg.d
+        n = max(T * K, 1)
+        o = LayerOutputs(self._empty((T, d), torch.bfloat16), self._empty((T, K), torch.int32),
+                         self._empty((T, K), torch.float32), self._empty((T, K), torch.uint8),
+                         torch.zeros(3, dtype=torch.int32, device=self.dev), self._empty((n,), torch.int32),
+                         self._empty((n,), torch.int32), self._empty((n,), torch.int32),
+                         self._empty((n,), torch.float32))
+        spice_moe_layer_fwd_fp8(self.ctx, w.c_struct(), h, conf, T, o.y, y_cpu_residual, x_resid, o.idx, o.gate, o.cls,
+                                o.counts, o.resid_tok, o.resid_k, o.resid_expert, o.resid_gate, stream)
         return o
 
     def set_option(self, option: int, value: int) -> None:

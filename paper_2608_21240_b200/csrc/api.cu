@@ -34,6 +34,7 @@ struct spice_ctx {
     cudaStream_t side;              // large batches: the shared expert runs here beside the routing chain (null: in line)
     cudaEvent_t ev_fork, ev_join, ev_grouped;
     float *part_split;              // [splits][Td, d] partial shared-expert outputs of the tcgen05 decode kernel
+    uint8_t *x8_h, *act8_hit, *act8_sh;   // 8-bit weight precision: activations as three E5M2 planes
     int n_sms, max_smem_optin;
     TcBuffers tcb;                  // tensor-core path buffers (large batches)
     bool tc_ok;
@@ -102,6 +103,12 @@ void carve(spice_ctx *c, char *base, size_t *total) {
     c->act_shared16 = cv.take<__nv_bfloat16>(Td * g.inter_shared);
     c->z16 = cv.take<__nv_bfloat16>((g_low * Td > nd ? g_low * Td : nd) * g.lore_rank);
     c->part_split = cv.take<float>((size_t)decode_tc_nsplit(dims_of_cfg(g, 1)) * Td * g.d);
+    {   // 8-bit weight precision (decode batches of at most 32 tokens)
+        const size_t T8 = Tm < 32 ? Tm : 32, n8 = T8 * K, g8 = (size_t)g.n_slots < n8 ? g.n_slots : n8;
+        c->x8_h = cv.take<uint8_t>(3 * T8 * g.d);
+        c->act8_hit = cv.take<uint8_t>(g8 * 3 * T8 * g.inter);
+        c->act8_sh = cv.take<uint8_t>(3 * T8 * g.inter_shared);
+    }
     c->sync_words = SY_GROUP0 + 1 + g.n_slots + g.n_experts;
     c->sync = cv.take<int32_t>(c->sync_words);
     {   // buffers of the tensor-core path
@@ -182,11 +189,16 @@ DecodeParams decode_params_of(const spice_ctx *ctx, const Dims &dm) {
         ctx->launches += n_;                     \
     } while (0)
 
+spice_status layer_general_path(spice_ctx *ctx, const spice_layer_weights *w, const __nv_bfloat16 *hb, const float *conf, int32_t T,
+                                const float *y_cpu_residual, spice_bf16 *x_resid, spice_bf16 *y, int32_t *idx, float *gate,
+                                uint8_t *cls, int32_t *counts, int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
+                                float *resid_gate, cudaStream_t st);
+
 }  // namespace
 
 extern "C" {
 
-int32_t spice_version(void) { return 100; }
+int32_t spice_version(void) { return 200; }
 
 const char *spice_status_string(spice_status s) {
     switch (s) {
@@ -559,6 +571,80 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
         }
         // cooperative launch refused (e.g. device shared with another context): use the general path
     }
+    return layer_general_path(ctx, w, hb, conf, T, y_cpu_residual, x_resid, y, idx, gate, cls, counts, resid_tok, resid_k,
+                              resid_expert, resid_gate, st);
+}
+
+spice_status spice_quantize_e4m3_rows(const spice_bf16 *w, int64_t rows, int32_t cols, uint8_t *q, float *scale, void *stream) {
+    if (rows < 0 || cols < 8 || cols % 8) return SPICE_ERR_INVALID_ARG;
+    if (rows == 0) return SPICE_OK;
+    if (!w || !q || !scale || !aligned16(w) || !aligned16(q)) return SPICE_ERR_INVALID_ARG;
+    return launch_quantize_e4m3_rows(reinterpret_cast<const __nv_bfloat16 *>(w), (size_t)rows, cols, q, scale,
+                                     static_cast<cudaStream_t>(stream)) < 0 ? SPICE_ERR_CUDA : SPICE_OK;
+}
+
+spice_status spice_moe_layer_fwd_fp8(spice_ctx *ctx, const spice_layer_weights_fp8 *w, const spice_bf16 *h, const float *conf,
+                                     int32_t T, const float *y_cpu_residual, spice_bf16 *x_resid, spice_bf16 *y, int32_t *idx,
+                                     float *gate, uint8_t *cls, int32_t *counts, int32_t *resid_tok, int32_t *resid_k,
+                                     int32_t *resid_expert, float *resid_gate, void *stream) {
+    spice_status s = check_call(ctx, T);
+    if (s != SPICE_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!counts) counts = ctx->ws_counts;
+    if (T == 0) return cudaMemsetAsync(counts, 0, 3 * sizeof(int32_t), st) == cudaSuccess ? SPICE_OK : SPICE_ERR_CUDA;
+    if (!w || !w->w_router || !w->slot_of_expert || !w->slot_q_gate_up || !w->slot_s_gate_up || !w->slot_q_down || !w->slot_s_down ||
+        !w->shared_q_gate_up || !w->shared_s_gate_up || !w->shared_q_down || !w->shared_s_down || !w->lore_A || !w->lore_B)
+        return SPICE_ERR_INVALID_ARG;
+    if (!aligned16(w->w_router) || !aligned16(w->slot_q_gate_up) || !aligned16(w->slot_q_down) || !aligned16(w->shared_q_gate_up) ||
+        !aligned16(w->shared_q_down) || !aligned16(w->lore_A) || !aligned16(w->lore_B))
+        return SPICE_ERR_INVALID_ARG;
+    if (!h || !conf || !y || !aligned16(h) || !aligned16(y)) return SPICE_ERR_INVALID_ARG;
+    if ((y_cpu_residual && !aligned16(y_cpu_residual)) || (x_resid && !aligned16(x_resid))) return SPICE_ERR_INVALID_ARG;
+    const Dims dm = dims_of(ctx, T);
+    if (T > 32 || T > ctx->dtc_tokens || !decode_tc_supported(dm, ctx->cfg.conf_stride, (size_t)ctx->max_smem_optin, true))
+        return SPICE_ERR_UNSUPPORTED_SHAPE;
+    if (!idx) idx = ctx->ws_idx;
+    if (!gate) gate = ctx->ws_gate;
+    if (!cls) cls = ctx->ws_cls;
+    if (!(resid_tok && resid_k && resid_expert && resid_gate)) resid_tok = resid_k = resid_expert = nullptr, resid_gate = nullptr;
+    DecodeParams p = decode_params_of(ctx, dm);
+    p.h = reinterpret_cast<const __nv_bfloat16 *>(h);
+    p.conf = conf;
+    p.w = spice_layer_weights{};
+    p.w.w_router = w->w_router;
+    p.w.slot_of_expert = w->slot_of_expert;
+    p.w.lore_A = w->lore_A;
+    p.w.lore_B = w->lore_B;
+    p.idx = idx;
+    p.gate = gate;
+    p.cls = cls;
+    p.counts = counts;
+    p.resid_tok = resid_tok;
+    p.resid_k = resid_k;
+    p.resid_expert = resid_expert;
+    p.resid_gate = resid_gate;
+    p.y16 = reinterpret_cast<__nv_bfloat16 *>(y);
+    p.y_cpu = y_cpu_residual;
+    p.x_resid = reinterpret_cast<__nv_bfloat16 *>(x_resid);
+    Fp8Layer f8{w->slot_q_gate_up, w->slot_q_down, w->shared_q_gate_up, w->shared_q_down,
+                w->slot_s_gate_up, w->slot_s_down, w->shared_s_gate_up, w->shared_s_down,
+                ctx->x8_h, ctx->act8_hit, ctx->act8_sh};
+    const int n = launch_decode_tc(p, ctx->part_split, ctx->n_sms, ctx->max_smem_optin, st, &f8);
+    if (n < 0) return SPICE_ERR_CUDA;
+    ctx->launches += n;
+    return SPICE_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+// the layer on the kernels for batches and shapes the fused decode kernels do not take
+spice_status layer_general_path(spice_ctx *ctx, const spice_layer_weights *w, const __nv_bfloat16 *hb, const float *conf, int32_t T,
+                                const float *y_cpu_residual, spice_bf16 *x_resid, spice_bf16 *y, int32_t *idx, float *gate,
+                                uint8_t *cls, int32_t *counts, int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert,
+                                float *resid_gate, cudaStream_t st) {
+    const Dims dm = dims_of(ctx, T);
     const bool tc_path = ctx->opt_path != 1 && ctx->opt_path != 3 && ctx->tc_ok && tc_shape_ok(dm);
     // The shared expert needs nothing but h: it runs on the context's side stream beside the routing chain (router,
     // classification, grouping, gather occupy few SMs) and joins before the combine.  Both event edges are ordinary
@@ -633,4 +719,4 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
     return rc;
 }
 
-}  // extern "C"
+}  // namespace

@@ -700,7 +700,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                                                                    const __grid_constant__ DtcMaps maps) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     constexpr int STAGE_BYTES = A_BYTES + (F8 ? 6 : 2) * NB * 128;   // (stage pitch; a bf16 task of the 8-bit kernel fills less)
-    constexpr int ACC = F8 ? 3 * NB : NB;                              // accumulator columns of one buffer
+    constexpr int ACC = F8 ? 4 * NB : NB;                              // TMEM columns between the two accumulator buffers (8-bit: 3 NB used)
     constexpr int TMEM_COLS = 2 * ACC <= 32 ? 32 : (2 * ACC <= 64 ? 64 : (2 * ACC <= 128 ? 128 : (2 * ACC <= 256 ? 256 : 512)));
     constexpr int KST = F8 ? KSTAGE8 : KSTAGE;
     const DecodeParams &p = q.p;
@@ -1287,53 +1287,69 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
 
 // ------------------------------------------------------------------------------------------
 // host side
-size_t dtc_smem_bytes(const Dims &dm, int conf_stride, int stages) {
+size_t dtc_smem_bytes(const Dims &dm, int conf_stride, int stages, bool f8) {
     const int nb = nb_of(dm.T);
-    return 1024 + (size_t)stages * stage_bytes_of(nb) + ((sizeof(Ctl) + 15) & ~size_t(15)) + aux_layout(dm, conf_stride, nb, nullptr, nullptr);
+    return 1024 + (size_t)stages * stage_bytes_of(nb, f8) + ((sizeof(Ctl) + 15) & ~size_t(15)) + aux_layout(dm, conf_stride, nb, nullptr, nullptr);
 }
 
-int dtc_stages(const Dims &dm, int conf_stride, size_t max_smem) {
+int dtc_stages(const Dims &dm, int conf_stride, size_t max_smem, bool f8) {
     for (int s = MAX_STAGES; s >= 3; --s)
-        if (dtc_smem_bytes(dm, conf_stride, s) <= max_smem) return s;
+        if (dtc_smem_bytes(dm, conf_stride, s, f8) <= max_smem) return s;
     return 0;
 }
 
 }  // namespace
 
-bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem) {
-    if (dm.T < 1 || dm.T > 64) return false;
+bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem, bool f8) {
+    if (dm.T < 1 || dm.T > (f8 ? 32 : 64)) return false;
+    // 8-bit weights are viewed as [row][k-block][128 bytes]
+    if (f8 && (dm.d % 128 || dm.I % 128 || dm.Is % 128)) return false;
     if (dm.N > 256 || dm.S > 256) return false;
     if ((size_t)dm.T * dm.K > 1024 || (size_t)dm.T * dm.N > 8192) return false;
     // the big operands are viewed as [row][k-block][64]: their reduction lengths must be whole k-blocks
     if (dm.d % 64 || dm.I % 64 || dm.Is % 64 || dm.r % 8) return false;
-    const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
-    if ((kcIs + CHUNKS_PER_SPLIT - 1) / CHUNKS_PER_SPLIT > MAX_SPLIT) return false;
-    return dtc_stages(dm, conf_stride, max_smem) >= 3;
+    if (decode_tc_nsplit(dm, f8) > MAX_SPLIT) return false;
+    return dtc_stages(dm, conf_stride, max_smem, f8) >= 3;
 }
 
-int decode_tc_nsplit(const Dims &dm) {
-    const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
+int decode_tc_nsplit(const Dims &dm, bool f8) {
+    const int kst = f8 ? KSTAGE8 : KSTAGE;
+    const int kcIs = (dm.Is + kst - 1) / kst;
     return (kcIs + CHUNKS_PER_SPLIT - 1) / CHUNKS_PER_SPLIT;
 }
 
 int decode_tc_prepare(int max_smem_optin) {
-    const void *fns[3] = {reinterpret_cast<const void *>(decode_tc_kernel<16>), reinterpret_cast<const void *>(decode_tc_kernel<32>),
-                          reinterpret_cast<const void *>(decode_tc_kernel<64>)};
+    const void *fns[5] = {reinterpret_cast<const void *>(decode_tc_kernel<16>), reinterpret_cast<const void *>(decode_tc_kernel<32>),
+                          reinterpret_cast<const void *>(decode_tc_kernel<64>), reinterpret_cast<const void *>(decode_tc_kernel<16, true>),
+                          reinterpret_cast<const void *>(decode_tc_kernel<32, true>)};
     for (const void *fn : fns)
         if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem_optin) != cudaSuccess) return -1;
     return 0;
 }
 
-int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int max_smem_optin, cudaStream_t st) {
+int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int max_smem_optin, cudaStream_t st, const Fp8Layer *f8) {
     const Dims &dm = p.dm;
-    DtcParams q;
+    DtcParams q{};
     q.p = p;
     q.part_split = part_split;
-    q.stages = dtc_stages(dm, p.conf_stride, (size_t)max_smem_optin);
+    q.stages = dtc_stages(dm, p.conf_stride, (size_t)max_smem_optin, f8 != nullptr);
     if (q.stages < 3) return -1;
-    const int kcIs = (dm.Is + KSTAGE - 1) / KSTAGE;
-    q.nsplit_sh = decode_tc_nsplit(dm);
+    const int kst = f8 ? KSTAGE8 : KSTAGE;
+    const int kcIs = (dm.Is + kst - 1) / kst;
+    q.nsplit_sh = decode_tc_nsplit(dm, f8 != nullptr);
     q.cps_sh = (kcIs + q.nsplit_sh - 1) / q.nsplit_sh;
+    int launches = 1;
+    if (f8) {
+        q.s_slot_gu = f8->s_slot_gu;
+        q.s_slot_d = f8->s_slot_d;
+        q.s_sh_gu = f8->s_sh_gu;
+        q.s_sh_d = f8->s_sh_d;
+        q.act8_hit = f8->act8_hit;
+        q.act8_sh = f8->act8_sh;
+        // the token operand of the gate/up tiles: h as three E5M2 planes (one small launch ahead of the layer kernel)
+        if (launch_split_e5m2x3(p.h, (size_t)dm.T * dm.d, f8->x8_h, st) < 0) return -1;
+        ++launches;
+    }
     {
         const int per = (dm.T + AUX_W - 1) / AUX_W, fit = n_ctas / dm.N;
         q.r1_sub = per < 1 ? 1 : per;
@@ -1359,27 +1375,57 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
         const uint32_t box[5] = {64, box_rows, 1, 1, 1};
         ok = ok && tc_encode_map5(&maps.m[which], base, dims, strides, box);
     };
+    // 8-bit weights: (128 bytes, rows, halves, k-blocks of 128, matrices); the box takes two k-blocks
+    auto big8 = [&](int which, const void *base, uint64_t rows, uint64_t K, uint64_t halves, uint64_t mats, uint64_t mat_bytes,
+                    uint32_t box_rows) {
+        const uint64_t dims[5] = {128, rows, halves, K / 128, mats};
+        const uint64_t strides[4] = {K, rows * K, 128, mat_bytes};
+        const uint32_t box[5] = {128, box_rows, (uint32_t)halves, 2, 1};
+        ok = ok && tc_encode_map5(&maps.m[which], base, dims, strides, box, 1);
+    };
+    // activations as three E5M2 planes [group][3][T][K]: (128 bytes, tokens, terms, k-blocks, groups); the box takes all
+    // three terms of nb tokens and two k-blocks and lands as [k-block][term][token][128]
+    auto x8 = [&](int which, const void *base, uint64_t K, uint64_t groups) {
+        const uint64_t dims[5] = {128, T, 3, K / 128, groups};
+        const uint64_t strides[4] = {K, T * K, 128, 3 * T * K};
+        const uint32_t box[5] = {128, (uint32_t)nb, 3, 2, 1};
+        ok = ok && tc_encode_map5(&maps.m[which], base, dims, strides, box, 1);
+    };
     big(MAP_H, p.h, T, d, 1, 1, T * d, nb);
-    big(MAP_SLOT_GU, p.w.slot_w_gate_up, I, d, 2, dm.S, 2 * I * d, 64);
-    big(MAP_SH_GU, p.w.shared_w_gate_up, Is, d, 2, 1, 2 * Is * d, 64);
     big(MAP_LORE_A, p.w.lore_A, r, d, 1, dm.N, r * d, 128);
-    big(MAP_SLOT_D, p.w.slot_w_down, d, I, 1, dm.S, d * I, 128);
-    big(MAP_SH_D, p.w.shared_w_down, d, Is, 1, 1, d * Is, 128);
     plain(MAP_LORE_B, p.w.lore_B, d, r, dm.N, 128);
-    big(MAP_ACT_HIT, p.act_hit16, T, I, 1, g_hit, T * I, nb);
-    big(MAP_ACT_SH, p.act_shared16, T, Is, 1, 1, T * Is, nb);
     plain(MAP_Z, p.z16, T, r, g_low, nb);
+    if (f8) {
+        big8(MAP_SLOT_GU, f8->q_slot_gu, I, d, 2, dm.S, 2 * I * d, 64);
+        big8(MAP_SH_GU, f8->q_sh_gu, Is, d, 2, 1, 2 * Is * d, 64);
+        big8(MAP_SLOT_D, f8->q_slot_d, d, I, 1, dm.S, d * I, 128);
+        big8(MAP_SH_D, f8->q_sh_d, d, Is, 1, 1, d * Is, 128);
+        x8(MAP_X8, f8->x8_h, d, 1);
+        x8(MAP_ACT_HIT, f8->act8_hit, I, g_hit);
+        x8(MAP_ACT_SH, f8->act8_sh, Is, 1);
+    } else {
+        big(MAP_SLOT_GU, p.w.slot_w_gate_up, I, d, 2, dm.S, 2 * I * d, 64);
+        big(MAP_SH_GU, p.w.shared_w_gate_up, Is, d, 2, 1, 2 * Is * d, 64);
+        big(MAP_SLOT_D, p.w.slot_w_down, d, I, 1, dm.S, d * I, 128);
+        big(MAP_SH_D, p.w.shared_w_down, d, Is, 1, 1, d * Is, 128);
+        big(MAP_ACT_HIT, p.act_hit16, T, I, 1, g_hit, T * I, nb);
+        big(MAP_ACT_SH, p.act_shared16, T, Is, 1, 1, T * Is, nb);
+        maps.m[MAP_X8] = maps.m[MAP_H];   // (never used)
+    }
     if (!ok) return -1;
-    const size_t smem = dtc_smem_bytes(dm, p.conf_stride, q.stages);
-    const void *fn = nb == 16 ? reinterpret_cast<const void *>(decode_tc_kernel<16>)
-                              : (nb == 32 ? reinterpret_cast<const void *>(decode_tc_kernel<32>)
-                                          : reinterpret_cast<const void *>(decode_tc_kernel<64>));
+    const size_t smem = dtc_smem_bytes(dm, p.conf_stride, q.stages, f8 != nullptr);
+    const void *fn;
+    if (f8)
+        fn = nb == 16 ? reinterpret_cast<const void *>(decode_tc_kernel<16, true>) : reinterpret_cast<const void *>(decode_tc_kernel<32, true>);
+    else
+        fn = nb == 16 ? reinterpret_cast<const void *>(decode_tc_kernel<16>)
+                      : (nb == 32 ? reinterpret_cast<const void *>(decode_tc_kernel<32>) : reinterpret_cast<const void *>(decode_tc_kernel<64>));
     void *args[] = {&q, &maps};
     if (cudaLaunchCooperativeKernel(fn, dim3(n_ctas), dim3(DTC_THREADS), args, smem, st) != cudaSuccess) {
         cudaGetLastError();
         return -1;
     }
-    return 1;
+    return launches;
 }
 
 #ifdef SPICE_PROF

@@ -157,10 +157,26 @@ int decode_prepare(int max_smem_optin);
 int launch_decode(const DecodeParams &p, int n_ctas, cudaStream_t st);
 
 // ---- fused decode kernel on tcgen05 / TMA (decode_tc.cu); shares DecodeParams and the counter words
-bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem);
-int decode_tc_nsplit(const Dims &dm);   // K ranges of the shared expert's down projection (rows of part_split)
+// The layer at the 8-bit weight precision: E4M3 codes and fp32 row scales of the expert matrices (layouts of
+// spice_layer_weights_fp8), and the ctx buffers that hold activations as three E5M2 planes.
+struct Fp8Layer {
+    const uint8_t *q_slot_gu, *q_slot_d, *q_sh_gu, *q_sh_d;
+    const float *s_slot_gu, *s_slot_d, *s_sh_gu, *s_sh_d;
+    uint8_t *x8_h;       // [3][T][d]
+    uint8_t *act8_hit;   // [group][3][T][I]
+    uint8_t *act8_sh;    // [3][T][Is]
+};
+bool decode_tc_supported(const Dims &dm, int conf_stride, size_t max_smem, bool f8 = false);
+int decode_tc_nsplit(const Dims &dm, bool f8 = false);   // K ranges of the shared expert's down projection (rows of part_split)
 int decode_tc_prepare(int max_smem_optin);
-int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int max_smem_optin, cudaStream_t st);
+int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int max_smem_optin, cudaStream_t st,
+                     const Fp8Layer *f8 = nullptr);
+
+// ---- 8-bit formats (fp8.cu)
+// per-row power-of-two scale and E4M3 codes of a bf16 matrix [rows, cols]
+int launch_quantize_e4m3_rows(const __nv_bfloat16 *w, size_t rows, int cols, uint8_t *q, float *scale, cudaStream_t st);
+// x[n] bf16 -> three E5M2 planes out[3][n] whose sum is x
+int launch_split_e5m2x3(const __nv_bfloat16 *x, size_t n, uint8_t *out, cudaStream_t st);
 
 // ---- tensor-core path for large batches (tc_gemm.cu)
 // One m-tile of the grouped problem: rows [row0, row0+rows) of the gathered activation buffer, all of

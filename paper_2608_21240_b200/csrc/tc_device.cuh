@@ -6,8 +6,10 @@
 
 namespace spice {
 
-// host: 5-D bf16 tensor map from extents, byte strides of dimensions 1..4 and box; 128-byte swizzle (tc_gemm.cu)
-bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], const uint64_t strides[4], const uint32_t box[5]);
+// host: 5-D tensor map (bf16 elements, or bytes when elem_bytes == 1) from extents, byte strides of dimensions 1..4 and
+// box; 128-byte swizzle (tc_gemm.cu)
+bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], const uint64_t strides[4], const uint32_t box[5],
+                    int elem_bytes = 2);
 
 namespace tcdev {
 
@@ -62,6 +64,14 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0)
         : "memory");
 }
+// the same for 8-bit floating-point operands (kind::f8f6f4; the element types are fields of the instruction descriptor)
+__device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0)
+        : "memory");
+}
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,"
@@ -105,6 +115,12 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t *v) {
 // instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N accumulator
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// instruction descriptor of kind::f8f6f4: A = E4M3 (format code 0), B = E5M2 (format code 1), fp32 accumulator,
+// both operands K-major, M x N accumulator
+__host__ __device__ constexpr uint32_t make_idesc_e4m3_e5m2(int M, int N) {
+    return (1u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 }  // namespace tcdev

@@ -340,9 +340,10 @@ bool make_map(CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, ui
 
 }  // namespace
 
-// 5-D bf16 tensor map with explicit extents, byte strides (dimensions 1..4) and box; 128-byte swizzle, zero fill.
-// The innermost box extent must be 64 elements (one swizzle span).
-bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], const uint64_t strides[4], const uint32_t box[5]) {
+// 5-D tensor map (bf16, or bytes) with explicit extents, byte strides (dimensions 1..4) and box; 128-byte swizzle, zero
+// fill.  The innermost box extent must be one swizzle span: 64 bf16 elements or 128 bytes.
+bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], const uint64_t strides[4], const uint32_t box[5],
+                    int elem_bytes) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t gd[5], gs[4];
@@ -352,7 +353,8 @@ bool tc_encode_map5(CUtensorMap *m, const void *base, const uint64_t dims[5], co
         bx[i] = box[i];
     }
     for (int i = 0; i < 4; ++i) gs[i] = strides[i];
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), gd, gs, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return fn(m, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), gd,
+              gs, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
