@@ -107,7 +107,6 @@ struct Ctl {
     int last_flag;
     int no_more;   // the producer has issued its last task
     int wsum[2][AUX_W];
-    int s_cnt[4];
 };
 
 // auxiliary team's shared memory (routing scratch and the tables every role reads)
@@ -506,7 +505,6 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                 ax.gate[i] = pk / denom;
                 ax.cls[i] = (unsigned char)c;
                 ax.key[i] = gkey;
-                atomicAdd(&sh->s_cnt[c], 1);
             }
         }
     }
@@ -607,12 +605,14 @@ __device__ __forceinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, c
         p.cls[i] = ax.cls[i];
     }
     if (a.aw == 0) {
-        int base = 0;
+        int base = 0, n_hit = 0, n_low = 0;
 #pragma unroll 1
         for (int i0 = 0; i0 < n; i0 += 32) {
             const int i = i0 + a.lane;
             const bool miss = i < n && ax.cls[i] == SPICE_MISS_EXACT;
             const unsigned m = __ballot_sync(0xffffffffu, miss);
+            n_hit += __popc(__ballot_sync(0xffffffffu, i < n && ax.cls[i] == SPICE_HIT));
+            n_low += __popc(__ballot_sync(0xffffffffu, i < n && ax.cls[i] == SPICE_LOWCONF));
             if (miss && p.resid_tok) {
                 const int o = base + __popc(m & ((1u << a.lane) - 1u));
                 p.resid_tok[o] = i / K;
@@ -622,7 +622,7 @@ __device__ __forceinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, c
             }
             base += __popc(m);
         }
-        if (a.lane < 3) p.counts[a.lane] = sh->s_cnt[a.lane];
+        if (a.lane < 3) p.counts[a.lane] = a.lane == SPICE_HIT ? n_hit : (a.lane == SPICE_MISS_EXACT ? base : n_low);
     }
 }
 
@@ -735,10 +735,15 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         sh->last_flag = 0;
         sh->no_more = 0;
         sh->n_hg = sh->n_lg = 0;
-        for (int i = 0; i < 4; ++i) sh->s_cnt[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = threadIdx.x; i < 1 + dm.S + dm.N; i += DTC_THREADS) ax.ready[i] = 0;
+    {   // the router matrix is needed first and by few warps: every thread of the grid asks for one of its lines now
+        const size_t n_lines = ((size_t)dm.N * dm.d * 2 + 127) >> 7;
+        const size_t g = (size_t)blockIdx.x * DTC_THREADS + threadIdx.x, n_thr = (size_t)gridDim.x * DTC_THREADS;
+        for (size_t l = g; l < n_lines; l += n_thr)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.w.w_router) + (l << 7)));
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
@@ -777,6 +782,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             // ids: the first one is the CTA's index, every later one is drawn from a global counter.  The draw is
             // issued before the task's copies and used after them, so its latency hides behind the copies.
             int id = blockIdx.x;
+            const uint64_t w_policy = l2_policy_evict_first();
             auto lead_wait = [&](uint32_t bar, uint32_t parity) {   // lane 0 waits, the outcome is uniform
                 int r = 1;
                 if (lane == 0) r = mb_wait(bar, parity, abort_flag) ? 1 : 0;
@@ -885,8 +891,15 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 auto copy = [&](int kb, int stage) {   // this lane's box of k-stage kb into ring stage `stage`
                     const uint32_t full = smem_u32(&sh->full[stage]);
                     const uint32_t dst = smem_u32(ring + (size_t)stage * STAGE_BYTES);
-                    if (plain) tma_load_5d(dst + my_off, my_map, (k0 + kb) * KSTAGE + sub * 64, my_y, 0, 0, my_z, full);
-                    else tma_load_5d(dst + my_off, my_map, 0, my_y, 0, (k0 + kb) * 2, my_z, full);
+                    // (weights are read once per call: evict-first, so that they do not displace the kernel's code, the
+                    // router matrix and the activations from L2; the token operands keep the default policy)
+                    if (plain) {
+                        if (is_b) tma_load_5d(dst + my_off, my_map, (k0 + kb) * KSTAGE + sub * 64, my_y, 0, 0, my_z, full);
+                        else tma_load_5d_hint(dst + my_off, my_map, (k0 + kb) * KSTAGE + sub * 64, my_y, 0, 0, my_z, full, w_policy);
+                    } else {
+                        if (is_b) tma_load_5d(dst + my_off, my_map, 0, my_y, 0, (k0 + kb) * 2, my_z, full);
+                        else tma_load_5d_hint(dst + my_off, my_map, 0, my_y, 0, (k0 + kb) * 2, my_z, full, w_policy);
+                    }
                 };
                 // has the watcher warp already seen the group complete?
                 bool pending = false;

@@ -102,6 +102,20 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(mbar)
         : "memory");
 }
+// the same with an L2 eviction policy for the lines it brings in (createpolicy below)
+__device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, int c3, int c4,
+                                                 uint32_t mbar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(mbar), "l"(policy)
+        : "memory");
+}
+// L2 policy "evict first": data that is read exactly once (streamed weights) should not push out what is reused
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 // orders accesses of this thread through the generic proxy (plain loads / stores) with its accesses through
 // the async proxy (TMA): needed between data written by ordinary stores and a TMA load of the same bytes
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
