@@ -15,7 +15,7 @@ from typing import Optional
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libspice.so")
+LIB_PATH = os.environ.get("SPICE_LIB") or os.path.join(_PKG, "libspice.so")   # SPICE_LIB: an instrumented or older build
 
 SPICE_OK = 0
 HIT, MISS_EXACT, LOWCONF = 0, 1, 2

@@ -692,7 +692,7 @@ spice_status layer_general_path(spice_ctx *ctx, const spice_layer_weights *w, co
                 rc = SPICE_ERR_CUDA;
             ls = ctx->side;
         }
-        SPICE_STEP(launch_tc_routed(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
+        SPICE_STEP(launch_tc_routed(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st, gate));
         if (!forked) SPICE_STEP(launch_tc_shared(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, st));
         if (tc_lore_ok(dm)) {
             SPICE_STEP(launch_tc_lore_a(dm, *w, hb, ctx->tb, ctx->tcb, ctx->n_sms, ls));
@@ -714,6 +714,7 @@ spice_status layer_general_path(spice_ctx *ctx, const spice_layer_weights *w, co
     }
     CombineArgs ca{KIND_SHARED | KIND_HIT | KIND_LOW, 0, gate, cls, nullptr, reinterpret_cast<__nv_bfloat16 *>(y),
                    y_cpu_residual, reinterpret_cast<__nv_bfloat16 *>(x_resid)};
+    ca.hit_rows_gated16 = tc_path ? 1 : 0;
     SPICE_STEP(launch_combine(dm, ca, ctx->tb, st));
 #undef SPICE_STEP
     return rc;

@@ -228,6 +228,12 @@ __global__ void __launch_bounds__(256) combine_kernel(Dims dm, CombineArgs a, Ta
         const int c = a.cls[i];
         const bool use = (c == SPICE_HIT && (a.kind_mask & KIND_HIT)) || (c == SPICE_LOWCONF && (a.kind_mask & KIND_LOW));
         if (!use || tb.pos_of_entry[i] < 0) continue;
+        if (a.hit_rows_gated16 && c == SPICE_HIT) {   // gate applied by the producer, bf16 row in the fp32 row's first half
+            const uint2 u = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(tb.part + (size_t)i * d) + j);
+            acc.x += bf_lo(u.x); acc.y += bf_hi(u.x);
+            acc.z += bf_lo(u.y); acc.w += bf_hi(u.y);
+            continue;
+        }
         const float g = a.gate[i];
         const float4 s = *reinterpret_cast<const float4 *>(tb.part + (size_t)i * d + j);
         acc.x = fmaf(g, s.x, acc.x); acc.y = fmaf(g, s.y, acc.y);

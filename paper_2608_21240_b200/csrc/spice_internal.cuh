@@ -91,6 +91,7 @@ struct CombineArgs {
     const float *y_cpu;         // optional fp32 addend
     __nv_bfloat16 *x_resid;     // optional bf16 in/out residual stream
     int shared_coef_low_sum;    // 1: the shared expert enters with sum of LOWCONF gates (no "1 +"): rollout projection
+    int hit_rows_gated16;       // 1: rows of HIT entries in tb.part are bf16 and already multiplied by their gate
 };
 int launch_combine(const Dims &dm, const CombineArgs &a, const Tables &tb, cudaStream_t st);
 
@@ -196,8 +197,10 @@ struct TcBuffers {
 bool tc_available();
 int tc_prepare();
 bool tc_shape_ok(const Dims &dm);
+// gate16 != NULL: the down projection writes gate[entry] * row as bf16 into the first half of the entry's row of tb.part
+// (CombineArgs::hit_rows_gated16 tells the combine); NULL: plain fp32 rows
 int launch_tc_routed(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
-                     const TcBuffers &b, int n_sms, cudaStream_t st);
+                     const TcBuffers &b, int n_sms, cudaStream_t st, const float *gate16 = nullptr);
 int launch_tc_shared(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
                      const TcBuffers &b, int n_sms, cudaStream_t st);
 // router logits of a large batch as a GEMM, then Top-K from the stored logits (route.cu)

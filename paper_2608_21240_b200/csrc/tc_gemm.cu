@@ -5,6 +5,8 @@
 //
 //   MODE_ACT : act[row, i]        = silu(X W_g^T)[row,i] * (X W_u^T)[row,i]      (bf16 out)
 //   MODE_OUT : out[orow(row), j]  = (act W_d^T)[row, j]                          (fp32 out)
+//   MODE_GATED: out[orow(row), j] = gate[orow(row)] * (act W_d^T)[row, j]        (bf16 out: the routed down projection
+//              of large batches, whose 6 rows per token the combine then only adds; half the bytes of fp32 rows)
 //
 // C[M,N] = A[M,K] B[N,K]^T with both operands K-major.  A rows are tokens (gathered so that every
 // group is a contiguous row range), B rows are weight rows.  One persistent CTA per SM:
@@ -62,12 +64,13 @@ struct TcGemmArgs {
     __nv_bfloat16 *out16;       // MODE_ACT: [rows, ld]
     float *out32;               // MODE_OUT: [orows, ld]
     const int32_t *row_map;     // MODE_OUT: output row of A row r (entry id), or null for identity
+    const float *row_scale;     // MODE_GATED: factor of output row orow (the entry's gate)
     int32_t ld;
     int32_t *status;
     uint32_t wait_limit;        // polls after which a pipeline wait gives up (SPICE_OPT_TC_WAIT_LIMIT)
 };
 
-template <int MODE>   // 0 = gate/up + SwiGLU, 1 = plain
+template <int MODE>   // 0 = gate/up + SwiGLU, 1 = plain fp32, 2 = plain, scaled per output row, bf16
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                         const __grid_constant__ CUtensorMap map_b,
                                                                         const TcGemmArgs g) {
@@ -211,6 +214,37 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
                         const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * PITCH + part * 16);
                         if (q * 32 + rr < mt.rows && col < g.n_cols)   // (n_cols is a multiple of 8)
                             *reinterpret_cast<uint4 *>(g.out16 + (size_t)(mt.row0 + q * 32 + rr) * g.ld + col) = val;
+                    }
+                    __syncwarp();
+                }
+            } else if (MODE == 2) {
+                const int col0 = nt * BN2;
+                const int out_r = row_ok ? (g.row_map ? g.row_map[mt.row0 + r] : mt.row0 + r) : -1;
+                const float sc = out_r >= 0 ? g.row_scale[out_r] : 0.f;
+                constexpr int PITCH = 80;   // 64 B of bf16 per row + 16
+#pragma unroll 1
+                for (int c = 0; c < BN2; c += 32) {
+                    uint32_t v[32];
+                    tc_ld32(t0 + c, v);
+                    tc_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        __nv_bfloat162 b2 = __floats2bfloat162_rn(sc * __uint_as_float(v[j]), sc * __uint_as_float(v[j + 1]));
+                        pk[j >> 1] = *reinterpret_cast<uint32_t *>(&b2);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        *reinterpret_cast<uint4 *>(stg + lane * PITCH + k * 16) = make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = i * 8 + (lane >> 2), part = lane & 3;
+                        const int col = col0 + c + part * 8;
+                        const int orow = __shfl_sync(0xffffffffu, out_r, rr);
+                        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * PITCH + part * 16);
+                        if (orow >= 0 && col < g.n_cols)   // (n_cols is a multiple of 8)
+                            *reinterpret_cast<uint4 *>(g.out16 + (size_t)orow * g.ld + col) = val;
                     }
                     __syncwarp();
                 }
@@ -372,6 +406,8 @@ int tc_prepare() {
         return -1;
     if (cudaFuncSetAttribute(tc_grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM) != cudaSuccess)
         return -1;
+    if (cudaFuncSetAttribute(tc_grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM) != cudaSuccess)
+        return -1;
     return 0;
 }
 
@@ -485,7 +521,7 @@ int launch_tc_lore_a(const Dims &dm, const spice_layer_weights &w, const __nv_bf
 // Results land in tb.part (by entry id) (the shared expert's in tb.part_shared, by token) as fp32, exactly where the
 // general kernels put them, so the combine kernel is shared with the general path.
 int launch_tc_routed(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
-                     const TcBuffers &b, int n_sms, cudaStream_t st) {
+                     const TcBuffers &b, int n_sms, cudaStream_t st, const float *gate16) {
     CUtensorMap ma, mb;
     int launches = 0;
     const size_t cap = (size_t)dm.T * dm.K;
@@ -515,11 +551,21 @@ int launch_tc_routed(const Dims &dm, const spice_layer_weights &w, const __nv_bf
     g.b_rows_per_slot = dm.d;
     g.b_second_off = 0;
     g.n_cols = dm.d;
-    g.out16 = nullptr;
-    g.out32 = tb.part;
     g.row_map = tb.perm_hit;
-    g.ld = dm.d;
-    tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    if (gate16) {
+        // gated bf16 rows, each in the first half of the entry's fp32 row of tb.part (so rows of other entries, which the
+        // LoRE kernels may be writing as fp32 at the same time on another stream, are not touched)
+        g.out16 = reinterpret_cast<__nv_bfloat16 *>(tb.part);
+        g.out32 = nullptr;
+        g.row_scale = gate16;
+        g.ld = 2 * dm.d;
+        tc_grouped_gemm_kernel<2><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    } else {
+        g.out16 = nullptr;
+        g.out32 = tb.part;
+        g.ld = dm.d;
+        tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    }
     ++launches;
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
