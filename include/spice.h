@@ -245,10 +245,10 @@ spice_status spice_quantize_e4m3_rows(const spice_bf16 *w, int64_t rows, int32_t
 /* spice_moe_layer_fwd at the 8-bit weight precision; every other argument, every output and every rule (top-k order,
  * classes, residual list, optional residual inputs) as there.  Covers decode batches: T <= 32, and d, inter and
  * inter_shared multiples of 128 (SPICE_ERR_UNSUPPORTED_SHAPE otherwise; there is no second kernel path behind it, and
- * SPICE_ERR_CUDA is returned when the device refuses the cooperative launch).  Two launches: the input activations are
- * first written as the sum of three E5M2 terms (exact for bf16 magnitudes from 2^-7 to 57344; smaller ones to 2^-17
- * absolute, larger ones saturate), the same is done with the intermediate activations inside the layer kernel, and the
- * tensor cores multiply E4M3 weights with those terms (kind::f8f6f4), fp32 accumulation, row scale in the epilogue. */
+ * SPICE_ERR_CUDA is returned when the device refuses the cooperative launch).  One launch: inside the kernel the input
+ * activations and later the intermediate ones are written as the sum of three E5M2 terms (exact for bf16 magnitudes from
+ * 2^-7 to 57344; smaller ones to 2^-17 absolute, larger ones saturate), and the tensor cores multiply E4M3 weights with
+ * those terms (kind::f8f6f4), fp32 accumulation, row scale in the epilogue. */
 spice_status spice_moe_layer_fwd_fp8(spice_ctx *ctx, const spice_layer_weights_fp8 *w /* host struct */,
                                      const spice_bf16 *h, const float *conf, int32_t T,
                                      const float *y_cpu_residual, spice_bf16 *x_resid, spice_bf16 *y,

@@ -88,6 +88,7 @@ struct DtcParams {
     const float *s_slot_gu, *s_slot_d, *s_sh_gu, *s_sh_d;   // [S,2I], [S,d], [2Is], [d]
     uint8_t *act8_hit;   // [group][3][T][I]
     uint8_t *act8_sh;    // [3][T][Is]
+    uint8_t *x8_h;       // [3][T][d]: the input activations, written by the auxiliary teams at the start of the kernel
 };
 struct DtcMaps {
     CUtensorMap m[N_MAPS];
@@ -352,6 +353,33 @@ __device__ __forceinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) 
     if (done) {   // CTA-uniform
         aux_sync();
         if (a.atid == 0) red_release_add(p.sync + SY_R1_DONE, done);
+    }
+}
+
+// three E5M2 terms whose sum is the bf16 value x (exactly for 2^-7 <= |x| <= 57344): bytes hi | mid << 8 | lo << 16
+__device__ __forceinline__ uint32_t split_e5m2x3(float x) {
+    uint32_t out = 0;
+#pragma unroll
+    for (int j = 0; j < 3; ++j) {
+        const __nv_fp8_storage_t b = __nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E5M2);
+        out |= (uint32_t)b << (8 * j);
+        x -= __half2float(__half(__nv_cvt_fp8_to_halfraw(b, __NV_E5M2)));   // exact: both have few significant bits
+    }
+    return out;
+}
+
+// 8-bit weights: number of CTAs that write the three-term copy of h (= the target of SY_H8_DONE)
+__device__ __forceinline__ int h8_ctas(const DtcParams &q) {
+    const int n_units = q.p.dm.N * q.r1_sub, free_ctas = (int)gridDim.x - n_units;
+    return free_ctas >= 8 ? free_ctas : (int)gridDim.x;
+}
+__device__ __forceinline__ void aux_split_h(const DtcParams &q, const AuxCtx &a, int n, int part, int parts) {
+#pragma unroll 1
+    for (int i = part * AUX_T + a.atid; i < n; i += parts * AUX_T) {
+        const uint32_t b3 = split_e5m2x3(__bfloat162float(q.p.h[i]));
+        q.x8_h[i] = (uint8_t)b3;
+        q.x8_h[(size_t)n + i] = (uint8_t)(b3 >> 8);
+        q.x8_h[2 * (size_t)n + i] = (uint8_t)(b3 >> 16);
     }
 }
 
@@ -683,18 +711,6 @@ __device__ __forceinline__ void aux_combine(const DtcParams &q, const AuxSmem &a
 }
 
 // ------------------------------------------------------------------------------------------
-// three E5M2 terms whose sum is the bf16 value x (exactly for 2^-7 <= |x| <= 57344): bytes hi | mid << 8 | lo << 16
-__device__ __forceinline__ uint32_t split_e5m2x3(float x) {
-    uint32_t out = 0;
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-        const __nv_fp8_storage_t b = __nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E5M2);
-        out |= (uint32_t)b << (8 * j);
-        x -= __half2float(__half(__nv_cvt_fp8_to_halfraw(b, __NV_E5M2)));   // exact: both have few significant bits
-    }
-    return out;
-}
-
 template <int NB, bool F8 = false>
 __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_constant__ DtcParams q,
                                                                    const __grid_constant__ DtcMaps maps) {
@@ -782,6 +798,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             // ids: the first one is the CTA's index, every later one is drawn from a global counter.  The draw is
             // issued before the task's copies and used after them, so its latency hides behind the copies.
             int id = blockIdx.x;
+            bool h8_ok = false;   // (8-bit weights) the three-term copy of h is complete
             const uint64_t w_policy = l2_policy_evict_first();
             auto lead_wait = [&](uint32_t bar, uint32_t parity) {   // lane 0 waits, the outcome is uniform
                 int r = 1;
@@ -901,8 +918,15 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                         else tma_load_5d_hint(dst + my_off, my_map, 0, my_y, 0, (k0 + kb) * 2, my_z, full, w_policy);
                     }
                 };
-                // has the watcher warp already seen the group complete?
+                // 8-bit weights: the first gate/up task of the CTA waits for the three-term copy of h, which the auxiliary
+                // teams of all CTAs write at the start of the kernel (its weights are copied meanwhile, like a down tile's)
                 bool pending = false;
+                if (F8 && t.kind == TASK_ACT && !h8_ok) {
+                    dep = SY_H8_DONE;
+                    dep_target = h8_ctas(q);
+                    pending = true;
+                } else
+                // has the watcher warp already seen the group complete?
                 if (dep >= 0) {
                     int seen = 0;
                     if (lane == 0) {
@@ -943,6 +967,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     __syncwarp(PM);
                     if (__shfl_sync(PM, r, 0) == 0) { ok = false; break; }
                     if (lane == 0) DPROF(0, npf, 22);
+                    if (F8 && dep == SY_H8_DONE) h8_ok = true;
                     fence_proxy_async();
                     for (int kb = 0, ss = s0; kb < pre; ++kb) {
                         if (my_on && is_b) copy(kb, ss);
@@ -1221,7 +1246,27 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         ax.mask_hit[2 * a.atid] = ax.mask_hit[2 * a.atid + 1] = 0u;
         ax.mask_low[2 * a.atid] = ax.mask_low[2 * a.atid + 1] = 0u;
         APROF(a, 61);
-        aux_logits(q, a);
+        if (F8) {
+            // h as the sum of three E5M2 terms, written before anything else by the CTAs that hold no router-logit unit
+            // (the first h8_ctas ones; all CTAs when fewer than 8 are free, then after their logits), a slice each;
+            // published with one counter that the producers poll
+            const int n = T * dm.d, nc = h8_ctas(q);
+            if (nc < (int)gridDim.x) {
+                if ((int)blockIdx.x < nc) {   // (CTA-uniform)
+                    aux_split_h(q, a, n, blockIdx.x, nc);
+                    aux_sync();
+                    if (a.atid == 0) red_release_add(p.sync + SY_H8_DONE, 1);
+                }
+                aux_logits(q, a);
+            } else {
+                aux_logits(q, a);
+                aux_split_h(q, a, n, blockIdx.x, nc);
+                aux_sync();
+                if (a.atid == 0) red_release_add(p.sync + SY_H8_DONE, 1);
+            }
+        } else {
+            aux_logits(q, a);
+        }
         APROF(a, 62);
         asm volatile("cp.async.wait_group 0;" ::: "memory");   // (made visible to the team by the barriers of the wait below)
         bool ok = aux_wait_ge(q, sh, a, p.sync + SY_R1_DONE, N * q.r1_sub);
@@ -1359,9 +1404,7 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
         q.s_sh_d = f8->s_sh_d;
         q.act8_hit = f8->act8_hit;
         q.act8_sh = f8->act8_sh;
-        // the token operand of the gate/up tiles: h as three E5M2 planes (one small launch ahead of the layer kernel)
-        if (launch_split_e5m2x3(p.h, (size_t)dm.T * dm.d, f8->x8_h, st) < 0) return -1;
-        ++launches;
+        q.x8_h = f8->x8_h;
     }
     {
         const int per = (dm.T + AUX_W - 1) / AUX_W, fit = n_ctas / dm.N;

@@ -1,4 +1,4 @@
-// The 8-bit weight format of the layer's second precision and the activation format its kernels use.
+// The 8-bit weight format of the layer's second precision.
 //
 // The paper reports every result at BF16 and at one quantised weight precision (Sec. 5.1, Table 1) without defining the
 // latter.  Here: E4M3 codes (1-4-3 bits, bias 7, no infinities, largest value 448) with one power-of-two scale per
@@ -59,34 +59,12 @@ __global__ void __launch_bounds__(256) quantize_e4m3_rows_kernel(const __nv_bflo
     }
 }
 
-// x = hi + mid + lo with three E5M2 values: hi = rn(x), mid = rn(x - hi), lo = rn(x - hi - mid).  A bf16 has 8
-// significant bits, an E5M2 three, so the sum is exact for 2^-7 <= |x| <= 57344 (2^-17 absolute below; larger values
-// saturate).
-__global__ void __launch_bounds__(256) split_e5m2x3_kernel(const __nv_bfloat16 *__restrict__ x, size_t n, uint8_t *__restrict__ out) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        float v = __bfloat162float(x[i]);
-#pragma unroll
-        for (int j = 0; j < 3; ++j) {
-            const __nv_fp8_storage_t b = __nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E5M2);
-            out[(size_t)j * n + i] = b;
-            v -= __half2float(__half(__nv_cvt_fp8_to_halfraw(b, __NV_E5M2)));
-        }
-    }
-}
-
 }  // namespace
 
 int launch_quantize_e4m3_rows(const __nv_bfloat16 *w, size_t rows, int cols, uint8_t *q, float *scale, cudaStream_t st) {
     if (rows == 0) return 0;
     const size_t blocks = (rows + 7) / 8;
     quantize_e4m3_rows_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), 256, 0, st>>>(w, rows, cols, q, scale);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
-}
-
-int launch_split_e5m2x3(const __nv_bfloat16 *x, size_t n, uint8_t *out, cudaStream_t st) {
-    if (n == 0) return 0;
-    const size_t blocks = (n + 255) / 256;
-    split_e5m2x3_kernel<<<(unsigned)(blocks < 1184 ? blocks : 1184), 256, 0, st>>>(x, n, out);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -113,7 +113,7 @@ int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __n
 
 // ---- fused decode kernel (decode.cu)
 // words of the dependency-counter array
-enum { SY_ABORT = 0, SY_TEAMS_DONE, SY_R1_DONE, SY_ROUTE_DONE, SY_P2_DONE, SY_P1_ALL, SY_NEXT_TASK, SY_GROUP0 = 8 };
+enum { SY_ABORT = 0, SY_TEAMS_DONE, SY_R1_DONE, SY_ROUTE_DONE, SY_P2_DONE, SY_P1_ALL, SY_NEXT_TASK, SY_H8_DONE, SY_GROUP0 = 8 };
 
 struct DecodeParams {
     Dims dm;
@@ -176,8 +176,7 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
 // ---- 8-bit formats (fp8.cu)
 // per-row power-of-two scale and E4M3 codes of a bf16 matrix [rows, cols]
 int launch_quantize_e4m3_rows(const __nv_bfloat16 *w, size_t rows, int cols, uint8_t *q, float *scale, cudaStream_t st);
-// x[n] bf16 -> three E5M2 planes out[3][n] whose sum is x
-int launch_split_e5m2x3(const __nv_bfloat16 *x, size_t n, uint8_t *out, cudaStream_t st);
+
 
 // ---- tensor-core path for large batches (tc_gemm.cu)
 // One m-tile of the grouped problem: rows [row0, row0+rows) of the gathered activation buffer, all of
