@@ -81,8 +81,10 @@ def _check(code: int, what: str) -> None:
 def _ptr(t: Optional[torch.Tensor], dtype=None) -> C.c_void_p:
     if t is None:
         return C.c_void_p(0)
-    if not t.is_cuda or not t.is_contiguous():
-        raise SpiceError("tensors passed to libspice must be contiguous CUDA tensors")
+    # (pinned host memory is device-accessible under unified addressing: a caller may let the kernels write small
+    # results straight into it instead of copying them back)
+    if not (t.is_cuda or t.is_pinned()) or not t.is_contiguous():
+        raise SpiceError("tensors passed to libspice must be contiguous CUDA tensors (or pinned host tensors)")
     if dtype is not None and t.dtype != dtype:
         raise SpiceError(f"expected dtype {dtype}, got {t.dtype}")
     return C.c_void_p(t.data_ptr())

@@ -1,6 +1,8 @@
 // C ABI of libspice: argument checking, workspace ownership and kernel dispatch.
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "spice_internal.cuh"
 
 using namespace spice;
@@ -44,6 +46,15 @@ struct spice_ctx {
 };
 
 namespace {
+
+// NVTX range around the host side of an entry point (named after it): a profiler's timeline shows which call enqueued
+// which kernels; without a profiler attached the calls return at once.
+struct Range {
+    explicit Range(const char *name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+    Range(const Range &) = delete;
+    Range &operator=(const Range &) = delete;
+};
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -331,6 +342,7 @@ spice_status spice_set_option(spice_ctx *ctx, int32_t option, int64_t value) {
 
 spice_status spice_route_topk(spice_ctx *ctx, const spice_bf16 *h, const spice_bf16 *w_router, int32_t T,
                               int32_t *idx, float *gate, float *logits, void *stream) {
+    Range range_("spice_route_topk");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     if (T == 0) return SPICE_OK;
@@ -351,6 +363,7 @@ int32_t spice_min_lookahead_depth(int32_t n_prefetch, double expert_bytes, doubl
 
 spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, const spice_bf16 *w_draft_router, int32_t T,
                                     int32_t *idx_hat, float *pi_hat, float *conf, void *stream) {
+    Range range_("spice_draft_confidence");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     if (T == 0) return SPICE_OK;
@@ -365,6 +378,7 @@ spice_status spice_draft_confidence(spice_ctx *ctx, const spice_bf16 *h_hat, con
 spice_status spice_prefetch_rollout(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *x_current, int32_t T,
                                     int32_t l_min, int32_t l_max, float tau, int32_t *idx_hat, float *conf, int32_t *depth,
                                     spice_bf16 *h_final, uint8_t *prefetch_mask, void *stream) {
+    Range range_("spice_prefetch_rollout");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     if (l_max < 1 || l_max > 64 || l_min < 1 || l_min > l_max) return SPICE_ERR_INVALID_ARG;
@@ -444,6 +458,7 @@ spice_status spice_lore_calibrate(int32_t d, int32_t n_tokens, int32_t rank, flo
                                   const spice_bf16 *h_cal, const float *resid, spice_bf16 *A_out, spice_bf16 *B_out,
                                   float *loss_out, int32_t *device_status, void *workspace, size_t workspace_bytes,
                                   void *stream) {
+    Range range_("spice_lore_calibrate");
     if (d < 8 || d % 8 || rank < 1 || 2 * rank > d || n_tokens < 1 || iterations < 0 || iterations > 1000 || !(ridge >= 0.f))
         return SPICE_ERR_INVALID_ARG;
     if (!h_cal || !resid || !A_out || !B_out || !device_status || !workspace) return SPICE_ERR_INVALID_ARG;
@@ -458,6 +473,7 @@ spice_status spice_classify_misses(spice_ctx *ctx, const int32_t *idx, const flo
                                    const int32_t *slot_of_expert, const float *conf, int32_t T, uint8_t *cls,
                                    int32_t *slot, int32_t *counts, int32_t *resid_tok, int32_t *resid_k,
                                    int32_t *resid_expert, float *resid_gate, void *stream) {
+    Range range_("spice_classify_misses");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -475,6 +491,7 @@ spice_status spice_classify_misses(spice_ctx *ctx, const int32_t *idx, const flo
 spice_status spice_grouped_expert_ffn(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *h,
                                       const int32_t *idx, const float *gate, const uint8_t *cls,
                                       const int32_t *slot, int32_t T, float *y, void *stream) {
+    Range range_("spice_grouped_expert_ffn");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     if (T == 0) return SPICE_OK;
@@ -498,6 +515,7 @@ spice_status spice_grouped_expert_ffn(spice_ctx *ctx, const spice_layer_weights 
 spice_status spice_lore_surrogate(spice_ctx *ctx, const spice_layer_weights *w, const spice_bf16 *h,
                                   const int32_t *idx, const float *gate, const uint8_t *cls, int32_t T, float *y,
                                   void *stream) {
+    Range range_("spice_lore_surrogate");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     if (T == 0) return SPICE_OK;
@@ -527,6 +545,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
                                  spice_bf16 *y, int32_t *idx, float *gate, uint8_t *cls, int32_t *counts,
                                  int32_t *resid_tok, int32_t *resid_k, int32_t *resid_expert, float *resid_gate,
                                  void *stream) {
+    Range range_("spice_moe_layer_fwd");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -576,6 +595,7 @@ spice_status spice_moe_layer_fwd(spice_ctx *ctx, const spice_layer_weights *w, c
 }
 
 spice_status spice_quantize_e4m3_rows(const spice_bf16 *w, int64_t rows, int32_t cols, uint8_t *q, float *scale, void *stream) {
+    Range range_("spice_quantize_e4m3_rows");
     if (rows < 0 || cols < 8 || cols % 8) return SPICE_ERR_INVALID_ARG;
     if (rows == 0) return SPICE_OK;
     if (!w || !q || !scale || !aligned16(w) || !aligned16(q)) return SPICE_ERR_INVALID_ARG;
@@ -587,6 +607,7 @@ spice_status spice_moe_layer_fwd_fp8(spice_ctx *ctx, const spice_layer_weights_f
                                      int32_t T, const float *y_cpu_residual, spice_bf16 *x_resid, spice_bf16 *y, int32_t *idx,
                                      float *gate, uint8_t *cls, int32_t *counts, int32_t *resid_tok, int32_t *resid_k,
                                      int32_t *resid_expert, float *resid_gate, void *stream) {
+    Range range_("spice_moe_layer_fwd_fp8");
     spice_status s = check_call(ctx, T);
     if (s != SPICE_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
