@@ -7,7 +7,11 @@
 //     G = L L^T,  Z = L^-1 C                   (then the fitted values satisfy  Yhat^T Yhat = Z^T Z)
 //     V = r leading eigenvectors of Z^T Z      block subspace iteration, orthonormalised by Cholesky QR (twice)
 //     B = V,   A = ( L^-T Z V )^T = ( W V )^T  with W = G^-1 C the least-squares map
-// Everything is dense fp32 linear algebra on d x d matrices built from tiled SGEMMs (split over the reduction,
+// The two Gram products, 2 n d^2 multiply-adds each and a third of the work, run on the tensor cores: H is bf16, so
+// H^T H is a bf16 x bf16 product with fp32 accumulation and nothing is lost; the fp32 targets are written as the sum of
+// three bf16 terms (24 significant bits), so H^T R is three such products added in a fixed order.  The operands are
+// transposed copies (reduction index contiguous) and the kernel is the plain mode of the grouped GEMM of large batches.
+// Everything else is dense fp32 linear algebra on d x d matrices built from tiled SGEMMs (split over the reduction,
 // with the slices summed in a fixed order, where a product has too few output tiles to fill the GPU), 64 x 64 Cholesky /
 // triangular-solve blocks and a few element-wise kernels, launched in order on one stream; nothing synchronises
 // with the host.  The caller provides the workspace (spice_lore_calibrate_workspace_bytes).
@@ -116,6 +120,58 @@ int gemm(int M, int N, int K, float alpha, const float *A, int lda, const float 
     sgemm_kernel<TA, TB_><<<grid, 256, 0, st>>>(M, N, K, alpha, A, lda, B, ldb, beta, C, ldc, kchunk, t_splitk_ws);
     splitk_reduce_kernel<<<(unsigned)(((size_t)M * N + 255) / 256), 256, 0, st>>>(M, N, (int)grid.z, alpha, t_splitk_ws, beta, C, ldc);
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+// dst[c, r] = src[r, c] for a bf16 matrix [rows, cols]; dst is [cols_pad, ld] with zeros outside (32 x 32 tiles)
+__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16 *__restrict__ src, int rows, int cols,
+                                                             __nv_bfloat16 *__restrict__ dst, int cols_pad, int ld) {
+    __shared__ __nv_bfloat16 t[32][33];
+    const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8) {
+        const int r = r0 + i, c = c0 + tx;
+        t[i][tx] = (r < rows && c < cols) ? src[(size_t)r * cols + c] : __float2bfloat16(0.f);
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+        const int c = c0 + i, r = r0 + tx;
+        if (c < cols_pad && r < ld) dst[(size_t)c * ld + r] = t[tx][i];
+    }
+}
+
+// the same for an fp32 matrix, written as three bf16 planes whose sum is the value to 24 bits: x1 = bf16(x),
+// x2 = bf16(x - x1), x3 = bf16(x - x1 - x2); plane p at dst + p * cols_pad * ld
+__global__ void __launch_bounds__(256) transpose_split3_kernel(const float *__restrict__ src, int rows, int cols,
+                                                               __nv_bfloat16 *__restrict__ dst, int cols_pad, int ld) {
+    __shared__ float t[32][33];
+    const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8) {
+        const int r = r0 + i, c = c0 + tx;
+        t[i][tx] = (r < rows && c < cols) ? src[(size_t)r * cols + c] : 0.f;
+    }
+    __syncthreads();
+    const size_t plane = (size_t)cols_pad * ld;
+    for (int i = ty; i < 32; i += 8) {
+        const int c = c0 + i, r = r0 + tx;
+        if (c < cols_pad && r < ld) {
+            float x = t[tx][i];
+            const __nv_bfloat16 x1 = __float2bfloat16(x);
+            x -= __bfloat162float(x1);
+            const __nv_bfloat16 x2 = __float2bfloat16(x);
+            x -= __bfloat162float(x2);
+            const size_t o = (size_t)c * ld + r;
+            dst[o] = x1;
+            dst[plane + o] = x2;
+            dst[2 * plane + o] = __float2bfloat16(x);
+        }
+    }
+}
+
+// c = (a + b) + c3, element-wise over a [rows, ld] matrix
+__global__ void sum3_kernel(float *__restrict__ a, const float *__restrict__ b, const float *__restrict__ c3, size_t n) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) a[i] = (a[i] + b[i]) + c3[i];
 }
 
 // bf16 [rows, cols] -> fp32 [rows, ld] with zero columns cols..ld-1
@@ -362,6 +418,13 @@ int orthonormalise(float *Q, int dp, int rp, int r, float *S, int32_t *flag, cud
     return launches;
 }
 
+// tensor-core Gram products: transposed bf16 copies of H (1 plane) and R (3 planes), [dp, n8] each, two more [dp, dp] fp32
+// outputs, and the GEMM's tile list
+size_t gram_tc_bytes(size_t dp, size_t n) {
+    const size_t n8 = (n + 7) / 8 * 8;
+    return 4 * dp * n8 * sizeof(__nv_bfloat16) + 2 * dp * dp * sizeof(float) + (dp / 128 + 2) * sizeof(MTile) + 1024;
+}
+
 }  // namespace
 
 size_t lore_calibrate_workspace_bytes(int d, int n, int r) {
@@ -369,8 +432,9 @@ size_t lore_calibrate_workspace_bytes(int d, int n, int r) {
     // H32 / T2 [n, dp], G [dp, dp], C [dp, dp], Q, P, Y [dp, rp] each, S [rp, rp], T1 [n, rp], A32 [rp, dp], B32 [dp, rp], scalars
     size_t f = (size_t)n * dp + 2 * dp * dp + 3 * dp * rp + rp * rp + (size_t)n * rp + 2 * dp * rp + 64;
     f += 8 * dp * rp;   // slices of the products that are split over their reduction
-    return f * sizeof(float) + 256;
+    return f * sizeof(float) + 256 + gram_tc_bytes(dp, (size_t)n);
 }
+
 
 int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __nv_bfloat16 *h_cal, const float *resid,
                           __nv_bfloat16 *A_out, __nv_bfloat16 *B_out, float *loss_out, int32_t *flag, void *workspace,
@@ -389,16 +453,43 @@ int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __n
     float *A32 = w;                      w += (size_t)rp * dp;
     float *B32 = w;                      w += (size_t)dp * rp;
     float *scal = w;                     w += 64;
-    t_splitk_ws = w;
+    t_splitk_ws = w;                     w += (size_t)8 * dp * rp;
     t_splitk_floats = (size_t)8 * dp * rp;
+    // buffers of the tensor-core Gram products
+    const size_t n8 = ((size_t)n + 7) / 8 * 8;
+    float *C2 = w;                       w += (size_t)dp * dp;
+    float *C3 = w;                       w += (size_t)dp * dp;
+    __nv_bfloat16 *Ht16 = reinterpret_cast<__nv_bfloat16 *>((reinterpret_cast<uintptr_t>(w) + 255) & ~uintptr_t(255));
+    __nv_bfloat16 *Rt16 = Ht16 + (size_t)dp * n8;                 // three planes
+    MTile *mt = reinterpret_cast<MTile *>((reinterpret_cast<uintptr_t>(Rt16 + 3 * (size_t)dp * n8) + 255) & ~uintptr_t(255));
+    int32_t *n_mt = reinterpret_cast<int32_t *>(mt + dp / 128 + 1);
     int32_t *qr_flag = reinterpret_cast<int32_t *>(scal + 8);   // pivots clamped inside the Cholesky QR are not an error
     if (cudaMemsetAsync(flag, 0, sizeof(int32_t), st) != cudaSuccess) return -1;
     widen_pad_kernel<<<(unsigned)(((size_t)n * dp + 255) / 256), 256, 0, st>>>(h_cal, n, d, H32, dp);
     CKL();
     // G = H^T H, C = H^T R (columns >= d of C stay zero)
-    CK((gemm<true, false>(dp, dp, n, 1.f, H32, dp, H32, dp, 0.f, G, dp, st)));
-    if (cudaMemsetAsync(C, 0, sizeof(float) * (size_t)dp * dp, st) != cudaSuccess) return -1;
-    CK((gemm<true, false>(dp, d, n, 1.f, H32, dp, resid, d, 0.f, C, dp, st)));
+    int n_sms = 0, dev = 0;
+    const bool tc = tc_available() && tc_prepare() == 0 && cudaGetDevice(&dev) == cudaSuccess &&
+                    cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n_sms > 0;
+    if (tc) {
+        // on the tensor cores: transposed copies (the token index becomes the contiguous reduction index), H as it is
+        // (bf16), R as three bf16 planes; padded rows and columns are zero
+        dim3 tg((unsigned)((n8 + 31) / 32), (unsigned)((dp + 31) / 32));
+        transpose_bf16_kernel<<<tg, 256, 0, st>>>(h_cal, n, d, Ht16, dp, (int)n8);
+        CKL();
+        transpose_split3_kernel<<<tg, 256, 0, st>>>(resid, n, d, Rt16, dp, (int)n8);
+        CKL();
+        CK(launch_tc_plain(Ht16, dp, Ht16, dp, n, (int)n8, G, dp, mt, n_mt, n_sms, st));
+        float *outs[3] = {C, C2, C3};
+        for (int pl = 0; pl < 3; ++pl)
+            CK(launch_tc_plain(Ht16, dp, Rt16 + (size_t)pl * dp * n8, dp, n, (int)n8, outs[pl], dp, mt, n_mt, n_sms, st));
+        sum3_kernel<<<(unsigned)(((size_t)dp * dp + 255) / 256), 256, 0, st>>>(C, C2, C3, (size_t)dp * dp);
+        CKL();
+    } else {
+        CK((gemm<true, false>(dp, dp, n, 1.f, H32, dp, H32, dp, 0.f, G, dp, st)));
+        if (cudaMemsetAsync(C, 0, sizeof(float) * (size_t)dp * dp, st) != cudaSuccess) return -1;
+        CK((gemm<true, false>(dp, d, n, 1.f, H32, dp, resid, d, 0.f, C, dp, st)));
+    }
     mean_diag_kernel<<<1, 256, 0, st>>>(G, dp, d, scal);
     CKL();
     regularise_kernel<<<(unsigned)(((size_t)dp * dp + 255) / 256), 256, 0, st>>>(G, dp, d, dp, ridge, scal);

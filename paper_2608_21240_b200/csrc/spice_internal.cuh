@@ -202,6 +202,9 @@ int launch_tc_routed(const Dims &dm, const spice_layer_weights &w, const __nv_bf
                      const TcBuffers &b, int n_sms, cudaStream_t st, const float *gate16 = nullptr);
 int launch_tc_shared(const Dims &dm, const spice_layer_weights &w, const __nv_bfloat16 *h, const Tables &tb,
                      const TcBuffers &b, int n_sms, cudaStream_t st);
+// out[M,N] fp32 (ld) = A[M,K] B[N,K]^T on the tensor cores; bf16 operands with row pitch ldk (multiple of 8, zero padded)
+int launch_tc_plain(const __nv_bfloat16 *A, int M, const __nv_bfloat16 *B, int N, int K, int ldk, float *out, int ld, MTile *mtiles,
+                    int32_t *n_mtiles, int n_sms, cudaStream_t st);
 // router logits of a large batch as a GEMM, then Top-K from the stored logits (route.cu)
 bool tc_router_ok(const Dims &dm);
 int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router, float *logits,

@@ -446,6 +446,31 @@ int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_b
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
+// A plain product on the tensor cores: out[M, N] (fp32, leading dimension ld) = A[M, K] B[N, K]^T, both operands bf16,
+// K-major with row pitch ldk elements (a multiple of 8).  mtiles: room for ceil(M / 128) entries, n_mtiles: one int.
+int launch_tc_plain(const __nv_bfloat16 *A, int M, const __nv_bfloat16 *B, int N, int K, int ldk, float *out, int ld, MTile *mtiles,
+                    int32_t *n_mtiles, int n_sms, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    build_shared_mtiles_kernel<<<1, 32, 0, st>>>(M, mtiles, n_mtiles);
+    // (make_map takes the row pitch as the column count; columns past K are zero by construction of the callers' buffers)
+    if (!make_map(&ma, A, M, ldk, BM) || !make_map(&mb, B, N, ldk, 128)) return -1;
+    TcGemmArgs g{};
+    g.mtiles = mtiles;
+    g.n_mtiles = n_mtiles;
+    g.n_ntiles = (N + BN2 - 1) / BN2;
+    g.K = K;
+    g.b_rows_per_slot = 0;
+    g.b_second_off = 0;
+    g.n_cols = N;
+    g.out32 = out;
+    g.row_map = nullptr;
+    g.ld = ld;
+    g.status = nullptr;
+    g.wait_limit = WAIT_LIMIT;
+    tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
 // ---- LoRE down-projection z = A_e h of the LOW groups of a large batch, through the same GEMM kernel.
 // The low entries' tokens are gathered behind the hit entries' rows of x_perm (rows n_hit + p, p in perm_low order),
 // lore_A plays the weight operand with the expert index as the "slot" (r rows each), z lands in tb.z_low at the

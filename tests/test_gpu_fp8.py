@@ -158,3 +158,85 @@ def test_fp8_layer_refuses_what_it_does_not_cover():
     with pytest.raises(B.SpiceError, match="unsupported"):
         L.moe_layer_fwd_fp8(w8, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
     L.close()
+
+
+def test_fp8_layer_repeats_bit_identically_over_rotating_weight_sets_and_from_a_graph():
+    """120 back-to-back calls over 4 quantised weight sets (cold L2 for every call), then the same calls replayed from a
+    CUDA graph: every pass gives the first pass's bits.  Inside the kernel the three-term copy of h and of the
+    intermediate activations is written by ordinary stores and fetched by TMA copies of other thread blocks, ordered by
+    counters; a gap in that ordering would show here as a rare stale tile."""
+    s = W.SHAPES["dsv2lite"]
+    T = 4
+    sets = [W.make_layer(s, T, variant=400 + i) for i in range(4)]
+    w8 = [B.quantize_layer(upload(wl)) for wl in sets]
+    torch.cuda.synchronize()
+    structs = [w.c_struct() for w in w8]
+    L = B.SpiceLayer(cfg_of(s), T)
+    h, conf = bf16_tensor(sets[0].h), torch.from_numpy(sets[0].conf).cuda()
+    n_pass = 30
+    ys = torch.empty(n_pass, 4, T, s.d, dtype=torch.bfloat16, device="cuda")
+    st = torch.cuda.current_stream()
+    for p in range(n_pass):
+        for i in range(4):
+            B.spice_moe_layer_fwd_fp8(L.ctx, structs[i], h, conf, T, ys[p, i], stream=st)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0 and bool(torch.isfinite(ys[0].float()).all()) and not torch.equal(ys[0, 0], ys[0, 1])
+    same = (ys == ys[0:1]).flatten(1).all(dim=1)
+    assert bool(same.all()), f"passes that differ from the first: {torch.nonzero(~same).flatten().tolist()[:10]}"
+    yg = torch.empty(4, T, s.d, dtype=torch.bfloat16, device="cuda")
+    g = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=side):
+        for i in range(4):
+            B.spice_moe_layer_fwd_fp8(L.ctx, structs[i], h, conf, T, yg[i], stream=torch.cuda.current_stream())
+    for _ in range(3):
+        yg.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(yg, ys[0])
+    assert L.device_status() == 0
+    L.close()
+
+
+def test_fp8_layer_keeps_a_token_of_nans_in_its_own_row():
+    """Tokens are independent (Sec. 2.1).  The three E5M2 terms of a NaN are NaN, and every group is multiplied with all
+    token columns, so this checks that a NaN column of the 8-bit MMA stays a column."""
+    wl = W.make_layer("dsv2lite", 8, variant=61)
+    enforce_margins(wl)
+    s = wl.shape
+    ref = run_oracle(_Dequantised(wl), want_full=False)
+    bad = 5
+    h = wl.h.copy()
+    h[bad, :] = np.nan
+    L = B.SpiceLayer(cfg_of(s), wl.T)
+    out = L.moe_layer_fwd_fp8(B.quantize_layer(upload(wl)), bf16_tensor(h), torch.from_numpy(wl.conf).cuda())
+    torch.cuda.synchronize()
+    keep = np.arange(wl.T) != bad
+    idx, cls, y = out.idx.cpu().numpy(), out.cls.cpu().numpy(), out.y.float().cpu().numpy()
+    assert idx[bad].tolist() == list(range(s.top_k))
+    assert np.array_equal(idx[keep], ref.idx[keep]) and np.array_equal(cls[keep], ref.cls[keep])
+    assert np.isnan(y[bad]).all() and np.isfinite(y[keep]).all()
+    err, bound = y_close(y[keep], ref.y[keep])
+    assert err <= bound, (err, bound)
+    assert L.device_status() == 0
+    L.close()
+
+
+def test_fp8_layer_activation_range():
+    """Activations far from 1: the three-term form is exact from 2^-7 to 57344 and holds smaller values to 2^-17, so a
+    batch scaled by 2^-6 or by 2^7 (intermediate activations up to ~3e4) still matches the oracle (the layer is not scale-invariant: SwiGLU is not
+    homogeneous, so the oracle is re-run on the scaled inputs)."""
+    s = W.scaled_shape(W.SHAPES["tiny"], d=256, n_experts=8, top_k=2, inter=256, inter_shared=256, lore_rank=16, n_slots=5)
+    for scale in (2.0 ** -6, 2.0 ** 7):
+        wl = W.make_layer(s, 6, variant=90)
+        wl.h = W.bf16_round((wl.h * scale).astype(np.float32))
+        enforce_margins(wl, 1e-3 * min(scale, 1.0))
+        ref = run_oracle(_Dequantised(wl), want_full=False)
+        L = B.SpiceLayer(cfg_of(s), wl.T)
+        out = L.moe_layer_fwd_fp8(B.quantize_layer(upload(wl)), bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
+        torch.cuda.synchronize()
+        assert np.array_equal(out.idx.cpu().numpy(), ref.idx) and np.array_equal(out.cls.cpu().numpy(), ref.cls)
+        err, bound = y_close(out.y.float().cpu().numpy(), ref.y)
+        assert err <= bound, (scale, err, bound)
+        L.close()
