@@ -321,6 +321,89 @@ __global__ void fix_gram_kernel(float *S, int rp, int r, float jitter) {
     }
 }
 
+// ---- one Cholesky-QR pass of a block of 64 columns in three launches (the general path below takes six)
+// (1) Gram matrix of one 64-row slab of Q [rows, 64]: part[b] = Q_b^T Q_b
+__global__ void __launch_bounds__(256) qr_gram_slab_kernel(const float *__restrict__ Q, int rows, float *__restrict__ part) {
+    __shared__ float q[TB][TB + 1];
+    const int r0 = blockIdx.x * TB;
+    for (int e = threadIdx.x; e < TB * TB; e += 256) {
+        const int k = e / TB, c = e % TB;
+        q[k][c] = r0 + k < rows ? Q[(size_t)(r0 + k) * TB + c] : 0.f;
+    }
+    __syncthreads();
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < TB; ++k) {
+        float a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = q[k][ty * 4 + i];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) b[j] = q[k][tx * 4 + j];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    float *out = part + (size_t)blockIdx.x * TB * TB;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out[(ty * 4 + i) * TB + tx * 4 + j] = acc[i][j];
+}
+
+// (2) S = sum of the slabs' Gram matrices in slab order; rows / columns >= r become the identity; in the first pass a
+// small multiple of the largest diagonal entry is added to the diagonal (see fix_gram_kernel); Cholesky in place in shared
+// memory; L (lower, strict upper triangle zero) to global memory.  One CTA.
+__global__ void __launch_bounds__(256) qr_factor_kernel(const float *__restrict__ part, int n_slabs, int r, float jitter,
+                                                        float *__restrict__ L, int32_t *flag) {
+    __shared__ float a[TB][TB + 1];
+    __shared__ float s_max;
+    for (int e = threadIdx.x; e < TB * TB; e += 256) {
+        float s = 0.f;
+        for (int b = 0; b < n_slabs; ++b) s += part[(size_t)b * TB * TB + e];
+        const int i = e / TB, j = e % TB;
+        a[i][j] = (i >= r || j >= r) ? (i == j ? 1.f : 0.f) : s;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float mx = 0.f;
+        for (int i = 0; i < r; ++i) mx = fmaxf(mx, a[i][i]);
+        s_max = mx;
+    }
+    __syncthreads();
+    if (jitter > 0.f && (int)threadIdx.x < r) a[threadIdx.x][threadIdx.x] += jitter * s_max;
+    __syncthreads();
+    const int t = threadIdx.x & 63, pt = threadIdx.x >> 6;
+    for (int j = 0; j < TB; ++j) {
+        if (threadIdx.x == j) {
+            float p = a[j][j];
+            if (!(p > 0.f)) {
+                p = 1e-20f;
+                atomicOr(flag, 1);
+            }
+            a[j][j] = sqrtf(p);
+        }
+        __syncthreads();
+        const float piv = a[j][j];
+        if (pt == 0 && t > j) a[t][j] /= piv;
+        __syncthreads();
+        if (t > j) {
+            const float ltj = a[t][j];
+            for (int c = j + 1 + ((pt - (j + 1)) & 3); c <= t; c += 4) a[t][c] -= ltj * a[c][j];
+        }
+        __syncthreads();
+    }
+    for (int e = threadIdx.x; e < TB * TB; e += 256) {
+        const int i = e / TB, j = e % TB;
+        L[e] = j <= i ? a[i][j] : 0.f;
+    }
+}
+
 __global__ void write_factors_kernel(const float *__restrict__ V, const float *__restrict__ X, int ld, int d, int r,
                                      __nv_bfloat16 *__restrict__ A, __nv_bfloat16 *__restrict__ B) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -408,6 +491,18 @@ int solve_right_lt(float *Y, int ldy, int rows, const float *L, int ldl, int np,
 // Q [dp, rp] <- orthonormal basis of its columns by Cholesky QR, twice
 int orthonormalise(float *Q, int dp, int rp, int r, float *S, int32_t *flag, cudaStream_t st) {
     int launches = 0;
+    if (rp == TB && t_splitk_ws && (size_t)(dp / TB) * TB * TB <= t_splitk_floats) {
+        // a block of 64 columns: slab Gram matrices, one CTA that sums and factorises them, the triangular solve
+        for (int pass = 0; pass < 2; ++pass) {
+            qr_gram_slab_kernel<<<dp / TB, 256, 0, st>>>(Q, dp, t_splitk_ws);
+            CKL();
+            qr_factor_kernel<<<1, 256, 0, st>>>(t_splitk_ws, dp / TB, r, pass == 0 ? 1e-6f : 0.f, S, flag);
+            CKL();
+            trsm_right_lt_kernel<<<dp / TB, 64, 0, st>>>(Q, rp, dp, S, rp);
+            CKL();
+        }
+        return launches;
+    }
     for (int pass = 0; pass < 2; ++pass) {
         CK((gemm<true, false>(rp, rp, dp, 1.f, Q, rp, Q, rp, 0.f, S, rp, st)));
         fix_gram_kernel<<<(rp * rp + 255) / 256, 256, 0, st>>>(S, rp, r, pass == 0 ? 1e-6f : 0.f);
