@@ -168,6 +168,57 @@ __global__ void __launch_bounds__(256) transpose_split3_kernel(const float *__re
     }
 }
 
+// Operands of the subspace iteration's two products on the tensor cores.  An fp32 value is written as x1 + x2 with
+// x1 = bf16(x), x2 = bf16(x - x1) (16 significant bits), and a product Z Q as Z1 Q1 + Z1 Q2 + Z2 Q1 (the dropped term
+// Z2 Q2 is 2^-16 of the result): ONE product with the three pairs laid side by side along the reduction index,
+// [Z1 | Z1 | Z2] [Q1 | Q2 | Q1]^T, so that the accumulator in tensor memory adds them.
+// dst [n, 3 n] from the fp32 matrix src [n, n] (ld): row i = (row i of src, or column i when TRANS) as [x1 | x1 | x2]
+template <bool TRANS>
+__global__ void __launch_bounds__(256) split2_cat_matrix_kernel(const float *__restrict__ src, int n, int ld, __nv_bfloat16 *__restrict__ dst) {
+    __shared__ float t[32][33];
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;   // tile of dst rows r0.., reduction index c0..
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8) {
+        // want v(r, c) = TRANS ? src[c][r] : src[r][c]; read coalesced along the contiguous index of src
+        const int a = TRANS ? c0 + i : r0 + i, b = TRANS ? r0 + tx : c0 + tx;
+        t[i][tx] = (a < n && b < n) ? src[(size_t)a * ld + b] : 0.f;
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+        const int r = r0 + i, c = c0 + tx;
+        if (r < n && c < n) {
+            const float x = TRANS ? t[tx][i] : t[i][tx];
+            const __nv_bfloat16 x1 = __float2bfloat16(x), x2 = __float2bfloat16(x - __bfloat162float(x1));
+            __nv_bfloat16 *row = dst + (size_t)r * 3 * n;
+            row[c] = x1;
+            row[n + c] = x1;
+            row[2 * n + c] = x2;
+        }
+    }
+}
+// dst [cols, 3 n] from the fp32 block src [n, cols] (ld = cols): row j = column j of src as [x1 | x2 | x1]
+__global__ void __launch_bounds__(256) split2_cat_block_kernel(const float *__restrict__ src, int n, int cols, __nv_bfloat16 *__restrict__ dst) {
+    __shared__ float t[32][33];
+    const int k0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8) {
+        const int k = k0 + i, j = j0 + tx;
+        t[i][tx] = (k < n && j < cols) ? src[(size_t)k * cols + j] : 0.f;
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+        const int j = j0 + i, k = k0 + tx;
+        if (j < cols && k < n) {
+            const float x = t[tx][i];
+            const __nv_bfloat16 x1 = __float2bfloat16(x), x2 = __float2bfloat16(x - __bfloat162float(x1));
+            __nv_bfloat16 *row = dst + (size_t)j * 3 * n;
+            row[k] = x1;
+            row[n + k] = x2;
+            row[2 * n + k] = x1;
+        }
+    }
+}
+
 // c = (a + b) + c3, element-wise over a [rows, ld] matrix
 __global__ void sum3_kernel(float *__restrict__ a, const float *__restrict__ b, const float *__restrict__ c3, size_t n) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -519,6 +570,13 @@ size_t gram_tc_bytes(size_t dp, size_t n) {
     const size_t n8 = (n + 7) / 8 * 8;
     return 4 * dp * n8 * sizeof(__nv_bfloat16) + 2 * dp * dp * sizeof(float) + (dp / 128 + 2) * sizeof(MTile) + 1024;
 }
+// tensor-core products of the subspace iteration (blocks of 64 columns): [Z1|Z1|Z2] and its transposed twin, the block's
+// operand, the partial results of the ranges of the reduction, the tile list
+constexpr int IT_SPLIT = 8;
+size_t iter_tc_bytes(size_t dp) {
+    return 2 * dp * 3 * dp * sizeof(__nv_bfloat16) + TB * 3 * dp * sizeof(__nv_bfloat16) + IT_SPLIT * dp * TB * sizeof(float) +
+           (IT_SPLIT * (dp / 128 + 1) + 2) * sizeof(MTile) + 1024;
+}
 
 }  // namespace
 
@@ -527,7 +585,7 @@ size_t lore_calibrate_workspace_bytes(int d, int n, int r) {
     // H32 / T2 [n, dp], G [dp, dp], C [dp, dp], Q, P, Y [dp, rp] each, S [rp, rp], T1 [n, rp], A32 [rp, dp], B32 [dp, rp], scalars
     size_t f = (size_t)n * dp + 2 * dp * dp + 3 * dp * rp + rp * rp + (size_t)n * rp + 2 * dp * rp + 64;
     f += 8 * dp * rp;   // slices of the products that are split over their reduction
-    return f * sizeof(float) + 256 + gram_tc_bytes(dp, (size_t)n);
+    return f * sizeof(float) + 256 + gram_tc_bytes(dp, (size_t)n) + iter_tc_bytes(dp);
 }
 
 
@@ -558,6 +616,13 @@ int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __n
     __nv_bfloat16 *Rt16 = Ht16 + (size_t)dp * n8;                 // three planes
     MTile *mt = reinterpret_cast<MTile *>((reinterpret_cast<uintptr_t>(Rt16 + 3 * (size_t)dp * n8) + 255) & ~uintptr_t(255));
     int32_t *n_mt = reinterpret_cast<int32_t *>(mt + dp / 128 + 1);
+    // buffers of the tensor-core products of the subspace iteration
+    __nv_bfloat16 *Zcat = reinterpret_cast<__nv_bfloat16 *>((reinterpret_cast<uintptr_t>(n_mt + 4) + 255) & ~uintptr_t(255));
+    __nv_bfloat16 *Ztcat = Zcat + (size_t)dp * 3 * dp;
+    __nv_bfloat16 *Bcat = Ztcat + (size_t)dp * 3 * dp;
+    float *it_part = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(Bcat + (size_t)TB * 3 * dp) + 255) & ~uintptr_t(255));
+    MTile *it_mt = reinterpret_cast<MTile *>(it_part + (size_t)IT_SPLIT * dp * TB);
+    int32_t *it_n_mt = reinterpret_cast<int32_t *>(it_mt + IT_SPLIT * (dp / 128 + 1));
     int32_t *qr_flag = reinterpret_cast<int32_t *>(scal + 8);   // pivots clamped inside the Cholesky QR are not an error
     if (cudaMemsetAsync(flag, 0, sizeof(int32_t), st) != cudaSuccess) return -1;
     widen_pad_kernel<<<(unsigned)(((size_t)n * dp + 255) / 256), 256, 0, st>>>(h_cal, n, d, H32, dp);
@@ -604,10 +669,37 @@ int launch_lore_calibrate(int d, int n, int r, float ridge, int iters, const __n
     init_block_kernel<<<(unsigned)(((size_t)dp * rp + 255) / 256), 256, 0, st>>>(Q, dp, rp, r);
     CKL();
     CK(orthonormalise(Q, dp, rp, r, S, qr_flag, st));
+    const bool tc_iter = tc && rp == TB && iters > 0;
+    const int k_split = ((3 * dp + IT_SPLIT - 1) / IT_SPLIT + 63) / 64 * 64;
+    if (tc_iter) {
+        dim3 mg((unsigned)((dp + 31) / 32), (unsigned)((dp + 31) / 32));
+        split2_cat_matrix_kernel<false><<<mg, 256, 0, st>>>(Z, dp, dp, Zcat);
+        CKL();
+        split2_cat_matrix_kernel<true><<<mg, 256, 0, st>>>(Z, dp, dp, Ztcat);
+        CKL();
+        CK(launch_tc_splitk_tiles(dp, IT_SPLIT, it_mt, it_n_mt, st));
+    }
     for (int it = 0; it < iters; ++it) {
-        CK((gemm<false, false>(dp, rp, dp, 1.f, Z, dp, Q, rp, 0.f, P, rp, st)));     // P = Z Q
-        CK((gemm<true, false>(dp, rp, dp, 1.f, Z, dp, P, rp, 0.f, Y, rp, st)));      // Y = Z^T P
-        if (cudaMemcpyAsync(Q, Y, sizeof(float) * (size_t)dp * rp, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return -1;
+        if (tc_iter) {
+            // P = Z Q and Q <- Z^T P on the tensor cores (two-term operands, see split2_cat_matrix_kernel), each cut into
+            // IT_SPLIT ranges of the reduction whose partial results are added in range order
+            dim3 bg((unsigned)((dp + 31) / 32), (unsigned)((rp + 31) / 32));
+            const unsigned rb = (unsigned)(((size_t)dp * rp + 255) / 256);
+            split2_cat_block_kernel<<<bg, 256, 0, st>>>(Q, dp, rp, Bcat);
+            CKL();
+            CK(launch_tc_plain_splitk(Zcat, dp, Bcat, rp, k_split, 3 * dp, it_part, rp, it_mt, it_n_mt, n_sms, st));
+            splitk_reduce_kernel<<<rb, 256, 0, st>>>(dp, rp, IT_SPLIT, 1.f, it_part, 0.f, P, rp);
+            CKL();
+            split2_cat_block_kernel<<<bg, 256, 0, st>>>(P, dp, rp, Bcat);
+            CKL();
+            CK(launch_tc_plain_splitk(Ztcat, dp, Bcat, rp, k_split, 3 * dp, it_part, rp, it_mt, it_n_mt, n_sms, st));
+            splitk_reduce_kernel<<<rb, 256, 0, st>>>(dp, rp, IT_SPLIT, 1.f, it_part, 0.f, Q, rp);
+            CKL();
+        } else {
+            CK((gemm<false, false>(dp, rp, dp, 1.f, Z, dp, Q, rp, 0.f, P, rp, st)));     // P = Z Q
+            CK((gemm<true, false>(dp, rp, dp, 1.f, Z, dp, P, rp, 0.f, Y, rp, st)));      // Y = Z^T P
+            if (cudaMemcpyAsync(Q, Y, sizeof(float) * (size_t)dp * rp, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return -1;
+        }
         CK(orthonormalise(Q, dp, rp, r, S, qr_flag, st));
     }
     // B = V = Q;  A^T = W V = L^-T (Z V): block rows bottom to top (in place in P)

@@ -205,6 +205,10 @@ int launch_tc_shared(const Dims &dm, const spice_layer_weights &w, const __nv_bf
 // out[M,N] fp32 (ld) = A[M,K] B[N,K]^T on the tensor cores; bf16 operands with row pitch ldk (multiple of 8, zero padded)
 int launch_tc_plain(const __nv_bfloat16 *A, int M, const __nv_bfloat16 *B, int N, int K, int ldk, float *out, int ld, MTile *mtiles,
                     int32_t *n_mtiles, int n_sms, cudaStream_t st);
+// the same cut into n_split ranges of k_split reduction elements; partial results at out + s * M * ld (tile list built once)
+int launch_tc_splitk_tiles(int M, int n_split, MTile *mtiles, int32_t *n_mtiles, cudaStream_t st);
+int launch_tc_plain_splitk(const __nv_bfloat16 *A, int M, const __nv_bfloat16 *B, int N, int k_split, int ldk, float *out, int ld,
+                           const MTile *mtiles, const int32_t *n_mtiles, int n_sms, cudaStream_t st);
 // router logits of a large batch as a GEMM, then Top-K from the stored logits (route.cu)
 bool tc_router_ok(const Dims &dm);
 int launch_tc_router_logits(const Dims &dm, const __nv_bfloat16 *h, const __nv_bfloat16 *w_router, float *logits,

@@ -65,6 +65,7 @@ struct TcGemmArgs {
     float *out32;               // MODE_OUT: [orows, ld]
     const int32_t *row_map;     // MODE_OUT: output row of A row r (entry id), or null for identity
     const float *row_scale;     // MODE_GATED: factor of output row orow (the entry's gate)
+    int32_t split_rows;         // plain fp32 mode, product split over its reduction: rows of one partial result (MTile::pad = range)
     int32_t ld;
     int32_t *status;
     uint32_t wait_limit;        // polls after which a pipeline wait gives up (SPICE_OPT_TC_WAIT_LIMIT)
@@ -118,19 +119,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
                 const MTile mt = g.mtiles[tile / g.n_ntiles];
                 const int nt = tile % g.n_ntiles;
                 const int b_row = mt.slot * g.b_rows_per_slot + nt * (MODE == 0 ? 128 : BN2);
+                const int k_off = mt.pad * g.K;   // a tile of a product that is split over its reduction takes range `pad`
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(smem_u32(&sh->empty[s]), ((it / STAGES) & 1) ^ 1, abort_flag, wl)) { ok = false; break; }
                     const uint32_t full = smem_u32(&sh->full[s]);
                     const uint32_t dst = smem_u32(ring + s * STAGE_BYTES);
                     mbar_expect_tx(full, STAGE_BYTES);
-                    tma_load_2d(dst, &map_a, kb * BK, mt.row0, full);
+                    tma_load_2d(dst, &map_a, k_off + kb * BK, mt.row0, full);
                     if (MODE == 0) {
-                        tma_load_2d(dst + A_BYTES, &map_b, kb * BK, b_row, full);                              // gate rows
-                        tma_load_2d(dst + A_BYTES + B_BYTES / 2, &map_b, kb * BK, b_row + g.b_second_off, full);  // up rows
+                        tma_load_2d(dst + A_BYTES, &map_b, k_off + kb * BK, b_row, full);                              // gate rows
+                        tma_load_2d(dst + A_BYTES + B_BYTES / 2, &map_b, k_off + kb * BK, b_row + g.b_second_off, full);  // up rows
                     } else {
-                        tma_load_2d(dst + A_BYTES, &map_b, kb * BK, b_row, full);
-                        tma_load_2d(dst + A_BYTES + B_BYTES / 2, &map_b, kb * BK, b_row + 128, full);
+                        tma_load_2d(dst + A_BYTES, &map_b, k_off + kb * BK, b_row, full);
+                        tma_load_2d(dst + A_BYTES + B_BYTES / 2, &map_b, k_off + kb * BK, b_row + 128, full);
                     }
                 }
             }
@@ -250,7 +252,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_grouped_gemm_kernel(const __
                 }
             } else {
                 const int col0 = nt * BN2;
-                const int out_r = row_ok ? (g.row_map ? g.row_map[mt.row0 + r] : mt.row0 + r) : -1;
+                const int out_r = row_ok ? (g.row_map ? g.row_map[mt.row0 + r] : mt.row0 + r + mt.pad * g.split_rows) : -1;
                 constexpr int PITCH = 144;   // 128 B of fp32 per row + 16
 #pragma unroll 1
                 for (int c = 0; c < BN2; c += 32) {
@@ -469,6 +471,40 @@ int launch_tc_plain(const __nv_bfloat16 *A, int M, const __nv_bfloat16 *B, int N
     g.wait_limit = WAIT_LIMIT;
     tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+// tile list of a product split over its reduction: for every range s, the m-tiles of all M rows
+__global__ void build_splitk_mtiles_kernel(int M, int n_split, MTile *mtiles, int32_t *n_mtiles) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    int n = 0;
+    for (int s = 0; s < n_split; ++s)
+        for (int r = 0; r < M; r += BM) mtiles[n++] = MTile{0, r, min(BM, M - r), s};
+    *n_mtiles = n;
+}
+
+// The same product cut into n_split ranges of k_split reduction elements (a multiple of 64): range s writes its partial
+// result to out + s * M * ld (the caller adds them, in range order).  For products with few output tiles: M / 128 tiles
+// would leave most SMs idle.  mtiles: room for n_split * ceil(M / 128) entries, built by launch_tc_splitk_tiles.
+int launch_tc_splitk_tiles(int M, int n_split, MTile *mtiles, int32_t *n_mtiles, cudaStream_t st) {
+    build_splitk_mtiles_kernel<<<1, 32, 0, st>>>(M, n_split, mtiles, n_mtiles);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+int launch_tc_plain_splitk(const __nv_bfloat16 *A, int M, const __nv_bfloat16 *B, int N, int k_split, int ldk, float *out, int ld,
+                           const MTile *mtiles, const int32_t *n_mtiles, int n_sms, cudaStream_t st) {
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, M, ldk, BM) || !make_map(&mb, B, N, ldk, 128)) return -1;
+    TcGemmArgs g{};
+    g.mtiles = mtiles;
+    g.n_mtiles = n_mtiles;
+    g.n_ntiles = (N + BN2 - 1) / BN2;
+    g.K = k_split;
+    g.n_cols = N;
+    g.out32 = out;
+    g.ld = ld;
+    g.split_rows = M;
+    g.wait_limit = WAIT_LIMIT;
+    tc_grouped_gemm_kernel<1><<<n_sms, TC_THREADS, TC_SMEM, st>>>(ma, mb, g);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 // ---- LoRE down-projection z = A_e h of the LOW groups of a large batch, through the same GEMM kernel.
