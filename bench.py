@@ -739,7 +739,8 @@ def run_lore_calibrate(args):
                                f"iterations; objective / sum resid^2 = {float(loss[0] / loss[1]):.4f}, status {int(status.item())}"},
         "roofline": {"bound": "alu", "achieved": flops / (ms * 1e-3) / 1e12, "peak": 72.0, "unit": "TFLOP/s",
                      "frac": flops / (ms * 1e-3) / 1e12 / 72.0, "traffic": None,
-                     "kernel": "fp32 SIMT GEMMs, blocked Cholesky and triangular solves (offline path, not tuned)",
+                     "kernel": "Gram and subspace-iteration products on the tensor cores, blocked Cholesky / triangular solves in "
+                               "fp32 SIMT; a chain of ~1400 small dependent launches (offline path)",
                      "peak_source": "148 SMs x 128 fp32 FMA lanes x 1.9 GHz x 2"},
         "gpu_launches": None}))
 
