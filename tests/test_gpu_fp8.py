@@ -240,3 +240,41 @@ def test_fp8_layer_activation_range():
         err, bound = y_close(out.y.float().cpu().numpy(), ref.y)
         assert err <= bound, (scale, err, bound)
         L.close()
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_fp8_and_bf16_kernels_agree_on_random_shapes(seed):
+    """Seeded random layer shapes (every dimension the 8-bit layout allows: multiples of 128 for d, I, I_s; any expert count,
+    top-k, slot count, LoRE rank, residency; 1 to 32 tokens): the 8-bit kernel against the 16-bit kernel fed the dequantised
+    weights.  Both compute the same products; routing must be identical and outputs within two bf16 ulps of the largest."""
+    rng = np.random.default_rng(3000 + seed)
+    base = W.SHAPES["tiny"]
+    for it in range(8):
+        s = W.scaled_shape(base, d=int(rng.choice([128, 256, 512, 1024])), n_experts=int(rng.choice([3, 17, 64, 100])),
+                           top_k=1, inter=int(rng.choice([128, 256, 384, 640])), inter_shared=int(rng.choice([128, 384, 768])),
+                           lore_rank=int(rng.choice([8, 24, 64, 72])), n_slots=1, norm_topk=int(rng.integers(0, 2)))
+        K = int(rng.integers(1, min(s.n_experts, 8) + 1))
+        S = int(rng.integers(1, s.n_experts + 1))
+        s = W.scaled_shape(s, top_k=K, n_slots=S)
+        T = int(rng.integers(1, 33))
+        wl = W.make_layer(s, T, variant=9000 + 100 * seed + it, n_resident=int(rng.integers(0, S + 1)))
+        w16 = upload(wl)
+        w8 = B.quantize_layer(w16)
+
+        def deq(qt, st):
+            return (torch.from_numpy(oracle.e4m3_decode(qt.cpu().numpy())).cuda() * st.double().unsqueeze(-1)).to(torch.bfloat16)
+        wd = B.LayerWeights(w16.w_router, deq(w8.slot_q_gate_up, w8.slot_s_gate_up), deq(w8.slot_q_down, w8.slot_s_down),
+                            w16.slot_of_expert, deq(w8.shared_q_gate_up, w8.shared_s_gate_up),
+                            deq(w8.shared_q_down, w8.shared_s_down), w16.lore_A, w16.lore_B)
+        L = B.SpiceLayer(cfg_of(s), T)
+        h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+        a = L.moe_layer_fwd_fp8(w8, h, conf)
+        b = L.moe_layer_fwd(wd, h, conf)
+        torch.cuda.synchronize()
+        tag = f"shape {s.d},{s.n_experts},{s.top_k},{s.inter},{s.inter_shared},{s.lore_rank},{s.n_slots} T={T}"
+        assert L.device_status() == 0, tag
+        assert torch.equal(a.idx, b.idx) and torch.equal(a.gate, b.gate) and torch.equal(a.cls, b.cls) and torch.equal(a.counts, b.counts), tag
+        ya, yb = a.y.float(), b.y.float()
+        assert bool(torch.isfinite(ya).all()), tag
+        assert (ya - yb).abs().max().item() <= 2.0 ** -7 * yb.abs().max().item() + 1e-6, tag
+        L.close()
