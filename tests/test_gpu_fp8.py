@@ -70,7 +70,7 @@ def test_quantiser_matches_the_oracle_bit_for_bit():
     assert torch.equal(q3.view(300, 512), q) and torch.equal(s3.view(300), s)
 
 
-FP8_CASES = [("dsv2lite", 1), ("dsv2lite", 4), ("dsv2lite", 16), ("dsv2lite", 27), ("qwen2_57b", 1), ("qwen2_57b", 8), ("qwen2_57b", 32)]
+FP8_CASES = [("dsv2lite", 1), ("dsv2lite", 4), ("dsv2lite", 16), ("dsv2lite", 27), ("qwen2_57b", 1), ("qwen2_57b", 8), ("qwen2_57b", 19)]
 
 
 @pytest.mark.parametrize("name,T", FP8_CASES)
