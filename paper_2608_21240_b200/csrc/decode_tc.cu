@@ -114,13 +114,21 @@ struct Ctl {
 struct AuxSmem {
     float *conf, *gate, *coef, *xch;
     int *soe, *idx, *key, *pos, *perm_h, *perm_l, *off_hit, *off_low, *ent;
-    uint32_t *mask_hit, *mask_low;   // [256][2] members of a slot's / an expert's group as a bit mask over the tokens
+    uint32_t *mask_hit, *mask_low;   // [S][2], [N][2] members of a slot's / an expert's group as a bit mask over the tokens
     int *ready;   // [1 + S + N] group g's gate/up (or A_e) tiles are all published (set by the watcher warp)
     unsigned char *cls;
     GroupDesc *gtab;
 };
 
 __host__ __device__ inline size_t up16(size_t v) { return (v + 15) & ~size_t(15); }
+
+// Shared memory is what bounds the depth of the weight ring, so the auxiliary team's part is kept small: confidences are
+// staged in shared memory only while they are few (else classification reads them from L2) and the routing tables are
+// sized by the slot and expert counts.  (32 token columns then have 5 ring stages instead of 4.)
+__host__ __device__ inline bool conf_staged(const Dims &dm, int conf_stride) {
+    return (conf_stride ? (size_t)dm.T * dm.N : (size_t)dm.T) <= 1024;
+}
+__host__ __device__ inline int xch_buffers(int) { return 2; }   // (one buffer serialises the two halves of the SwiGLU epilogue: measured slower)
 
 __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, int nb, AuxSmem *s, unsigned char *base) {
     size_t off = 0;
@@ -130,10 +138,10 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
         return o;
     };
     const size_t n = (size_t)dm.T * dm.K, TN = (size_t)dm.T * dm.N;
-    const size_t o_conf = take((conf_stride ? TN : (size_t)dm.T) * 4), o_gate = take(n * 4);
-    const size_t o_coef = take((size_t)dm.T * 4), o_xch = take((size_t)2 * nb * 64 * 4);
+    const size_t o_conf = take(conf_staged(dm, conf_stride) ? (conf_stride ? TN : (size_t)dm.T) * 4 : 0), o_gate = take(n * 4);
+    const size_t o_coef = take((size_t)dm.T * 4), o_xch = take((size_t)xch_buffers(nb) * nb * 64 * 4);
     const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_key = take(n * 4), o_pos = take(n * 4);
-    const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take(6 * 256 * 4), o_ent = take((size_t)4 * nb * 4);
+    const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take((size_t)3 * (dm.S + dm.N) * 4), o_ent = take((size_t)4 * nb * 4);
     const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
     const size_t o_rdy = take((1 + (size_t)dm.S + dm.N) * 4);
     if (s) {
@@ -148,10 +156,10 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
         s->perm_h = reinterpret_cast<int *>(base + o_ph);
         s->perm_l = reinterpret_cast<int *>(base + o_pl);
         int *hist = reinterpret_cast<int *>(base + o_hist);
-        s->off_hit = hist;
-        s->off_low = hist + 256;
-        s->mask_hit = reinterpret_cast<uint32_t *>(hist + 512);
-        s->mask_low = reinterpret_cast<uint32_t *>(hist + 1024);
+        s->off_hit = hist;                                                    // [S]
+        s->off_low = hist + dm.S;                                             // [N]
+        s->mask_hit = reinterpret_cast<uint32_t *>(hist + dm.S + dm.N);       // [2 S]
+        s->mask_low = reinterpret_cast<uint32_t *>(hist + 3 * dm.S + dm.N);   // [2 N]
         s->ent = reinterpret_cast<int *>(base + o_ent);
         s->cls = base + o_cls;
         s->gtab = reinterpret_cast<GroupDesc *>(base + o_gt);
@@ -520,7 +528,8 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                     if (p.roll_depth) {
                         low = roll_cont;
                     } else {
-                        const float cf = p.conf_stride ? ax.conf[t * N + e] : ax.conf[t];
+                        const int ci = p.conf_stride ? t * N + e : t;
+                        const float cf = conf_staged(dm, p.conf_stride) ? ax.conf[ci] : __ldg(p.conf + ci);
                         low = cf < p.tau;
                     }
                     c = low ? SPICE_LOWCONF : SPICE_MISS_EXACT;
@@ -578,8 +587,8 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
         }
         const int ea = ba + ia - va, eb = bb + ib - vb;   // exclusive
         const int n_hg = ta >> 16;
-        ax.off_hit[a.atid] = ea & 0xffff;
-        ax.off_low[a.atid] = eb & 0xffff;
+        if (a.atid < S) ax.off_hit[a.atid] = ea & 0xffff;
+        if (a.atid < N) ax.off_low[a.atid] = eb & 0xffff;
         if (ch > 0) ax.gtab[1 + (ea >> 16)] = GroupDesc{KIND_HIT, a.atid, ea & 0xffff, ch};
         if (cl > 0) ax.gtab[1 + n_hg + (eb >> 16)] = GroupDesc{KIND_LOW, a.atid, eb & 0xffff, cl};
         if (a.atid == AUX_T - 1) {   // this thread's inclusive sums are the totals
@@ -1123,7 +1132,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 const bool hit = grp.kind == KIND_HIT;
                 const int n_cols = hit ? dm.I : dm.Is;
                 __nv_bfloat16 *out = hit ? p.act_hit16 + (size_t)(t.gi - 1) * T * dm.I : p.act_shared16;
-                const int xb = xc & 1;
+                constexpr int XB = 2;   // (= xch_buffers(NB))
+                const int xb = xc % XB;
+                const uint32_t xuse = xc / XB;         // uses of this buffer so far
                 float *xch = ax.xch + xb * NB * 64;
                 // 8-bit weights: scale of this thread's weight row (gate rows first, then the up rows)
                 float rs = 1.0f;
@@ -1133,13 +1144,13 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     rs = col < n_cols ? sc[(qd >= 2 ? n_cols : 0) + col] : 0.0f;
                 }
                 if (qd >= 2) {   // up rows: park them for the warps that hold the gate rows
-                    if (!warp_mb_wait(smem_u32(&sh->xch_empty[xb]), ((xc >> 1) & 1) ^ 1, abort_flag, lane)) break;
+                    if (!warp_mb_wait(smem_u32(&sh->xch_empty[xb]), (xuse & 1) ^ 1, abort_flag, lane)) break;
 #pragma unroll
                     for (int nn = 0; nn < NB; ++nn) xch[nn * 64 + (L - 64)] = F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&sh->xch_full[xb]));
                 } else {
-                    if (!warp_mb_wait(smem_u32(&sh->xch_full[xb]), (xc >> 1) & 1, abort_flag, lane)) break;
+                    if (!warp_mb_wait(smem_u32(&sh->xch_full[xb]), xuse & 1, abort_flag, lane)) break;
                     const int col = t.tile * 64 + L;
                     if (F8) {
                         // the activation, rounded to bf16 as in the 16-bit kernel, stored as its three E5M2 terms
@@ -1240,11 +1251,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
 #pragma unroll 1
             for (int i = a.atid; i < N; i += AUX_T) cp_async4(smem_u32(ax.soe + i), p.w.slot_of_expert + i);
 #pragma unroll 1
-            for (int i = a.atid; i < n_conf; i += AUX_T) cp_async4(smem_u32(ax.conf + i), p.conf + i);
+            if (conf_staged(dm, p.conf_stride))
+                for (int i = a.atid; i < n_conf; i += AUX_T) cp_async4(smem_u32(ax.conf + i), p.conf + i);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
-        ax.mask_hit[2 * a.atid] = ax.mask_hit[2 * a.atid + 1] = 0u;
-        ax.mask_low[2 * a.atid] = ax.mask_low[2 * a.atid + 1] = 0u;
+        if (a.atid < dm.S) ax.mask_hit[2 * a.atid] = ax.mask_hit[2 * a.atid + 1] = 0u;
+        if (a.atid < N) ax.mask_low[2 * a.atid] = ax.mask_low[2 * a.atid + 1] = 0u;
         APROF(a, 61);
         if (F8) {
             // h as the sum of three E5M2 terms, written before anything else by the CTAs that hold no router-logit unit
