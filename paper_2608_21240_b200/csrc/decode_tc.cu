@@ -124,11 +124,14 @@ __host__ __device__ inline size_t up16(size_t v) { return (v + 15) & ~size_t(15)
 
 // Shared memory is what bounds the depth of the weight ring, so the auxiliary team's part is kept small: confidences are
 // staged in shared memory only while they are few (else classification reads them from L2) and the routing tables are
-// sized by the slot and expert counts.  (32 token columns then have 5 ring stages instead of 4.)
+// sized by the slot and expert counts, and the exchange area of the SwiGLU epilogue covers 32 token columns at a time.
+// (32 token columns then have 5 ring stages instead of 4, 64 columns 4 instead of 3.)
 __host__ __device__ inline bool conf_staged(const Dims &dm, int conf_stride) {
     return (conf_stride ? (size_t)dm.T * dm.N : (size_t)dm.T) <= 1024;
 }
-__host__ __device__ inline int xch_buffers(int) { return 2; }   // (one buffer serialises the two halves of the SwiGLU epilogue: measured slower)
+// the SwiGLU epilogue's exchange area: two buffers of min(nb, 32) token columns x 64 rows (one buffer would serialise the
+// epilogue's two halves: measured slower)
+__host__ __device__ inline size_t xch_floats(int nb) { return (size_t)2 * (nb > 32 ? 32 : nb) * 64; }
 
 __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, int nb, AuxSmem *s, unsigned char *base) {
     size_t off = 0;
@@ -139,7 +142,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
     };
     const size_t n = (size_t)dm.T * dm.K, TN = (size_t)dm.T * dm.N;
     const size_t o_conf = take(conf_staged(dm, conf_stride) ? (conf_stride ? TN : (size_t)dm.T) * 4 : 0), o_gate = take(n * 4);
-    const size_t o_coef = take((size_t)dm.T * 4), o_xch = take((size_t)xch_buffers(nb) * nb * 64 * 4);
+    const size_t o_coef = take((size_t)dm.T * 4), o_xch = take(xch_floats(nb) * 4);
     const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_key = take(n * 4), o_pos = take(n * 4);
     const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take((size_t)3 * (dm.S + dm.N) * 4), o_ent = take((size_t)4 * nb * 4);
     const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
@@ -1132,10 +1135,10 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 const bool hit = grp.kind == KIND_HIT;
                 const int n_cols = hit ? dm.I : dm.Is;
                 __nv_bfloat16 *out = hit ? p.act_hit16 + (size_t)(t.gi - 1) * T * dm.I : p.act_shared16;
-                constexpr int XB = 2;   // (= xch_buffers(NB))
-                const int xb = xc % XB;
-                const uint32_t xuse = xc / XB;         // uses of this buffer so far
-                float *xch = ax.xch + xb * NB * 64;
+                // The up rows reach the warps that hold the gate rows through a double-buffered exchange area of
+                // XW token columns; a tile of 64 columns goes through it in two rounds (the buffers alternate, so the
+                // rounds pipeline like consecutive tiles do), which keeps the area small enough for a deeper weight ring.
+                constexpr int XW = NB > 32 ? 32 : NB, XR = NB / XW;
                 // 8-bit weights: scale of this thread's weight row (gate rows first, then the up rows)
                 float rs = 1.0f;
                 if (F8) {
@@ -1143,44 +1146,54 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     const float *sc = hit ? q.s_slot_gu + (size_t)grp.id * 2 * dm.I : q.s_sh_gu;
                     rs = col < n_cols ? sc[(qd >= 2 ? n_cols : 0) + col] : 0.0f;
                 }
-                if (qd >= 2) {   // up rows: park them for the warps that hold the gate rows
-                    if (!warp_mb_wait(smem_u32(&sh->xch_empty[xb]), (xuse & 1) ^ 1, abort_flag, lane)) break;
+                bool dead = false;
 #pragma unroll
-                    for (int nn = 0; nn < NB; ++nn) xch[nn * 64 + (L - 64)] = F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh->xch_full[xb]));
-                } else {
-                    if (!warp_mb_wait(smem_u32(&sh->xch_full[xb]), xuse & 1, abort_flag, lane)) break;
-                    const int col = t.tile * 64 + L;
-                    if (F8) {
-                        // the activation, rounded to bf16 as in the 16-bit kernel, stored as its three E5M2 terms
-                        uint8_t *out8 = hit ? q.act8_hit + (size_t)(t.gi - 1) * 3 * T * dm.I : q.act8_sh;
-                        const size_t plane = (size_t)T * n_cols;
+                for (int xr = 0; xr < XR; ++xr, ++xc) {
+                    const int xb = xc & 1;
+                    const uint32_t xuse = xc >> 1;   // uses of this buffer so far
+                    float *xch = ax.xch + xb * XW * 64;
+                    if (qd >= 2) {   // up rows: park them for the warps that hold the gate rows
+                        if (!warp_mb_wait(smem_u32(&sh->xch_empty[xb]), (xuse & 1) ^ 1, abort_flag, lane)) { dead = true; break; }
 #pragma unroll
-                        for (int nn = 0; nn < NB; ++nn) {
-                            if (nn < T && col < n_cols) {
-                                const float u = xch[nn * 64 + L];
-                                const float a = __bfloat162float(__float2bfloat16(silu_f(__uint_as_float(v[nn]) * rs) * u));
-                                const uint32_t b3 = split_e5m2x3(a);
-                                uint8_t *o = out8 + (size_t)nn * n_cols + col;
-                                o[0] = (uint8_t)b3;
-                                o[plane] = (uint8_t)(b3 >> 8);
-                                o[2 * plane] = (uint8_t)(b3 >> 16);
-                            }
-                        }
+                        for (int nn = 0; nn < XW; ++nn)
+                            xch[nn * 64 + (L - 64)] = F8 ? __uint_as_float(v[xr * XW + nn]) * rs : __uint_as_float(v[xr * XW + nn]);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sh->xch_full[xb]));
                     } else {
+                        if (!warp_mb_wait(smem_u32(&sh->xch_full[xb]), xuse & 1, abort_flag, lane)) { dead = true; break; }
+                        const int col = t.tile * 64 + L;
+                        if (F8) {
+                            // the activation, rounded to bf16 as in the 16-bit kernel, stored as its three E5M2 terms
+                            uint8_t *out8 = hit ? q.act8_hit + (size_t)(t.gi - 1) * 3 * T * dm.I : q.act8_sh;
+                            const size_t plane = (size_t)T * n_cols;
 #pragma unroll
-                        for (int nn = 0; nn < NB; ++nn) {
-                            if (nn < T && col < n_cols) {
-                                const float u = xch[nn * 64 + L];
-                                out[(size_t)nn * n_cols + col] = __float2bfloat16(silu_f(__uint_as_float(v[nn])) * u);
+                            for (int nn = 0; nn < XW; ++nn) {
+                                const int tk = xr * XW + nn;
+                                if (tk < T && col < n_cols) {
+                                    const float u = xch[nn * 64 + L];
+                                    const float a = __bfloat162float(__float2bfloat16(silu_f(__uint_as_float(v[tk]) * rs) * u));
+                                    const uint32_t b3 = split_e5m2x3(a);
+                                    uint8_t *o = out8 + (size_t)tk * n_cols + col;
+                                    o[0] = (uint8_t)b3;
+                                    o[plane] = (uint8_t)(b3 >> 8);
+                                    o[2 * plane] = (uint8_t)(b3 >> 16);
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int nn = 0; nn < XW; ++nn) {
+                                const int tk = xr * XW + nn;
+                                if (tk < T && col < n_cols) {
+                                    const float u = xch[nn * 64 + L];
+                                    out[(size_t)tk * n_cols + col] = __float2bfloat16(silu_f(__uint_as_float(v[tk])) * u);
+                                }
                             }
                         }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sh->xch_empty[xb]));
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh->xch_empty[xb]));
                 }
-                ++xc;
+                if (dead) break;
             } else if (t.kind == TASK_Z) {
                 const int row = t.tile * 128 + L;
                 __nv_bfloat16 *out = p.z16 + (size_t)(t.gi - 1 - sh->n_hg) * T * dm.r;
