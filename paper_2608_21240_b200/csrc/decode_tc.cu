@@ -113,7 +113,7 @@ struct Ctl {
 // auxiliary team's shared memory (routing scratch and the tables every role reads)
 struct AuxSmem {
     float *conf, *gate, *coef, *xch;
-    int *soe, *idx, *key, *pos, *perm_h, *perm_l, *off_hit, *off_low, *ent;
+    int *soe, *idx, *pos, *perm_h, *perm_l, *off_hit, *off_low, *ent;
     uint32_t *mask_hit, *mask_low;   // [S][2], [N][2] members of a slot's / an expert's group as a bit mask over the tokens
     int *ready;   // [1 + S + N] group g's gate/up (or A_e) tiles are all published (set by the watcher warp)
     unsigned char *cls;
@@ -143,7 +143,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
     const size_t n = (size_t)dm.T * dm.K, TN = (size_t)dm.T * dm.N;
     const size_t o_conf = take(conf_staged(dm, conf_stride) ? (conf_stride ? TN : (size_t)dm.T) * 4 : 0), o_gate = take(n * 4);
     const size_t o_coef = take((size_t)dm.T * 4), o_xch = take(xch_floats(nb) * 4);
-    const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_key = take(n * 4), o_pos = take(n * 4);
+    const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_pos = take(n * 4);
     const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take((size_t)3 * (dm.S + dm.N) * 4), o_ent = take((size_t)4 * nb * 4);
     const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
     const size_t o_rdy = take((1 + (size_t)dm.S + dm.N) * 4);
@@ -154,7 +154,6 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
         s->xch = reinterpret_cast<float *>(base + o_xch);
         s->soe = reinterpret_cast<int *>(base + o_soe);
         s->idx = reinterpret_cast<int *>(base + o_idx);
-        s->key = reinterpret_cast<int *>(base + o_key);
         s->pos = reinterpret_cast<int *>(base + o_pos);
         s->perm_h = reinterpret_cast<int *>(base + o_ph);
         s->perm_l = reinterpret_cast<int *>(base + o_pl);
@@ -514,17 +513,16 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                     }
                 }
             }
-            // classification (Sec. 4.2 policy); key = grouping key: slot (HIT), 1024 + e (LOWCONF), -1
+            // classification (Sec. 4.2 policy)
             if (a.lane < K) {
                 const int i = t * K + a.lane, e = my_idx[u];
                 const int sl = p.roll_depth ? -1 : ax.soe[e];
-                int c, gkey = -1;
+                int c;
                 if (sl >= S) {
                     atomicMax(p.tb.status, (int)SPICE_ERR_BAD_TABLE);
                     c = SPICE_MISS_EXACT;
                 } else if (sl >= 0) {
                     c = SPICE_HIT;
-                    gkey = sl;
                     atomicOr(&ax.mask_hit[2 * sl + (t >> 5)], 1u << (t & 31));
                 } else {
                     bool low;
@@ -536,15 +534,11 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                         low = cf < p.tau;
                     }
                     c = low ? SPICE_LOWCONF : SPICE_MISS_EXACT;
-                    if (low) {
-                        gkey = 1024 + e;
-                        atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
-                    }
+                    if (low) atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
                 }
                 ax.idx[i] = e;
                 ax.gate[i] = pk / denom;
                 ax.cls[i] = (unsigned char)c;
-                ax.key[i] = gkey;
             }
         }
     }
@@ -615,7 +609,9 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
     // (an expert occurs at most once among a token's K choices, so the members of a group are distinct tokens)
 #pragma unroll 1
     for (int i = a.atid; i < n; i += AUX_T) {
-        const int key = ax.key[i], t = i / K;
+        // grouping key of the entry: its slot (HIT), 1024 + its expert (LOWCONF), -1 (listed for exact recovery)
+        const int e_i = ax.idx[i], c_i = ax.cls[i];
+        const int key = c_i == SPICE_HIT ? ax.soe[e_i] : (c_i == SPICE_LOWCONF ? 1024 + e_i : -1), t = i / K;
         int pos = -1;
         if (key >= 0) {
             const uint32_t *mk = key < 1024 ? ax.mask_hit + 2 * key : ax.mask_low + 2 * (key - 1024);
