@@ -84,6 +84,8 @@ struct DtcParams {
     int32_t nsplit_sh;   // K ranges of the shared down projection
     int32_t cps_sh;      // k-chunks per range
     int32_t r1_sub;      // token subsets per expert in the router-logit units
+    int32_t n_spec;      // slots 0 .. n_spec-1 are groups 1 .. n_spec whether or not a token is routed to them: their gate/up
+                         // tiles are known at launch and stream while the routing is being computed
     // 8-bit weight precision (decode_tc_kernel<NB, true>): row scales, and the activations as three E5M2 planes
     const float *s_slot_gu, *s_slot_d, *s_sh_gu, *s_sh_d;   // [S,2I], [S,d], [2Is], [d]
     uint8_t *act8_hit;   // [group][3][T][I]
@@ -113,7 +115,7 @@ struct Ctl {
 // auxiliary team's shared memory (routing scratch and the tables every role reads)
 struct AuxSmem {
     float *conf, *gate, *coef, *xch;
-    int *soe, *idx, *pos, *perm_h, *perm_l, *off_hit, *off_low, *ent;
+    int *soe, *idx, *pos, *perm_h, *perm_l, *off_hit, *off_low;
     uint32_t *mask_hit, *mask_low;   // [S][2], [N][2] members of a slot's / an expert's group as a bit mask over the tokens
     int *ready;   // [1 + S + N] group g's gate/up (or A_e) tiles are all published (set by the watcher warp)
     unsigned char *cls;
@@ -144,7 +146,7 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
     const size_t o_conf = take(conf_staged(dm, conf_stride) ? (conf_stride ? TN : (size_t)dm.T) * 4 : 0), o_gate = take(n * 4);
     const size_t o_coef = take((size_t)dm.T * 4), o_xch = take(xch_floats(nb) * 4);
     const size_t o_soe = take((size_t)dm.N * 4), o_idx = take(n * 4), o_pos = take(n * 4);
-    const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take((size_t)3 * (dm.S + dm.N) * 4), o_ent = take((size_t)4 * nb * 4);
+    const size_t o_ph = take(n * 4), o_pl = take(n * 4), o_hist = take((size_t)3 * (dm.S + dm.N) * 4);
     const size_t o_cls = take(n), o_gt = take((1 + (size_t)dm.S + dm.N) * sizeof(GroupDesc));
     const size_t o_rdy = take((1 + (size_t)dm.S + dm.N) * 4);
     if (s) {
@@ -162,7 +164,6 @@ __host__ __device__ inline size_t aux_layout(const Dims &dm, int conf_stride, in
         s->off_low = hist + dm.S;                                             // [N]
         s->mask_hit = reinterpret_cast<uint32_t *>(hist + dm.S + dm.N);       // [2 S]
         s->mask_low = reinterpret_cast<uint32_t *>(hist + 3 * dm.S + dm.N);   // [2 N]
-        s->ent = reinterpret_cast<int *>(base + o_ent);
         s->cls = base + o_cls;
         s->gtab = reinterpret_cast<GroupDesc *>(base + o_gt);
         s->ready = reinterpret_cast<int *>(base + o_rdy);
@@ -284,6 +285,12 @@ __device__ __forceinline__ bool warp_mb_wait(uint32_t a, uint32_t parity, volati
     return ok;
 }
 
+// a down tile's value of one member column: row `row` of the entry that is the rank-th of the group's list
+__device__ __noinline__ void store_member_row(float *out, const int *perm, int rank, int d, int row, float val) {
+    const int e = perm[rank];
+    if (row < d) out[(size_t)e * d + row] = val;
+}
+
 // ------------------------------------------------------------------------------------------
 // Task list.  ids [0, nA) are known at launch; the rest once the routing tables exist.
 struct Plan {
@@ -313,8 +320,11 @@ __device__ __forceinline__ void plan_static(Plan &pl, const DtcParams &q, int ks
     // gate/up tiles, so they go first only when the CTAs that take them would have nothing else to do.
     pl.sh_early = (pl.tIs + pl.nCs <= (int)gridDim.x) ? 1 : 0;
     pl.nA = pl.tIs + (pl.sh_early ? pl.nCs : 0);
-    pl.n_hg = pl.n_lg = pl.nBh = pl.nCh = 0;
-    pl.endB = pl.endC = pl.nA;
+    // gate/up tiles of the slots that are groups regardless of the routing (the leading hit groups, in slot order)
+    pl.n_hg = q.n_spec;
+    pl.nBh = q.n_spec * pl.tI;
+    pl.n_lg = pl.nCh = 0;
+    pl.endB = pl.endC = pl.nA + pl.nBh;
 }
 __device__ __forceinline__ void plan_routed(Plan &pl, int n_hg, int n_lg) {
     pl.n_hg = n_hg;
@@ -342,6 +352,33 @@ __device__ __forceinline__ bool aux_wait_ge(const DtcParams &q, Ctl *sh, const A
     return ok;
 }
 
+// G router logits of one expert row: tokens t, t + step, ... (those past the batch are computed on the last token's row and
+// dropped).  Per dot: slices k = lane*8 + 256 i reduced by slice_dot and added in increasing i, then the xor-shuffle tree.
+template <int G>
+__device__ __forceinline__ void logits_group(const DecodeParams &p, const __nv_bfloat16 *__restrict__ row, int t, int step, int e,
+                                             int lane) {
+    const Dims &dm = p.dm;
+    const __nv_bfloat16 *x[G];
+    float acc[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const int tg = min(t + g * step, dm.T - 1);
+        x[g] = p.h + (size_t)tg * dm.d;
+        acc[g] = 0.f;
+    }
+#pragma unroll 4
+    for (int k = lane * 8; k < dm.d; k += 256) {
+        const uint4 u = *reinterpret_cast<const uint4 *>(row + k);
+#pragma unroll
+        for (int g = 0; g < G; ++g) acc[g] += slice_dot(u, *reinterpret_cast<const uint4 *>(x[g] + k));
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        const float tot = warp_sum(acc[g]);
+        if (lane == 0 && t + g * step < dm.T) p.logits[(size_t)(t + g * step) * dm.N + e] = tot;
+    }
+}
+
 // router logits: unit u = (expert e, token subset s); each warp takes the tokens s*8 + warp (+ 8*r1_sub ...).
 // Same arithmetic order as the stand-alone router (route_device.cuh): logits agree bit for bit.
 __device__ __forceinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) {
@@ -354,11 +391,13 @@ __device__ __forceinline__ void aux_logits(const DtcParams &q, const AuxCtx &a) 
     for (int u = gridDim.x - 1 - blockIdx.x; u < n_units; u += gridDim.x, ++done) {
         const int e = u % dm.N, s = u / dm.N;
         const __nv_bfloat16 *row = reinterpret_cast<const __nv_bfloat16 *>(p.w.w_router) + (size_t)e * dm.d;
-        for (int t = s * AUX_W + a.aw; t < dm.T; t += AUX_W * q.r1_sub) {
-            const float sdot = lane_dot_bf16(row, p.h + (size_t)t * dm.d, dm.d, a.lane);
-            const float tot = warp_sum(sdot);
-            if (a.lane == 0) p.logits[(size_t)t * dm.N + e] = tot;
-        }
+        // the warp's tokens four (or two) at a time: the router row is loaded once for them and their loads are all in
+        // flight together; each dot keeps the summation order of lane_dot_bf16
+        const int step = AUX_W * q.r1_sub;
+        int t = s * AUX_W + a.aw;
+        for (; t + 2 * step < dm.T; t += 4 * step) logits_group<4>(p, row, t, step, e, a.lane);
+        for (; t + step < dm.T; t += 2 * step) logits_group<2>(p, row, t, step, e, a.lane);
+        for (; t < dm.T; t += step) logits_group<1>(p, row, t, step, e, a.lane);
     }
     if (done) {   // CTA-uniform
         aux_sync();
@@ -396,7 +435,11 @@ __device__ __forceinline__ void aux_split_h(const DtcParams &q, const AuxCtx &a,
 // Routing decisions from the logits, entirely in shared memory.  Every CTA computes the same tables
 // (the code is deterministic: counts by atomics, positions by ranking); CTA 0 also writes the outputs.
 // The arithmetic of the gates is that of warp_topk_gates (route_device.cuh).
-template <int NPL>
+// DIST: the batch is spread over the grid instead (CTA c takes tokens 8c .. 8c+7, a warp one token), the warp writes its
+// token's entries to the caller's idx / gate / cls arrays and every CTA collects all of them afterwards (aux_route): per
+// CTA the work no longer grows with the batch.  The token's confidences then travel with its logits (same indexing, one
+// coalesced load) and the winner's value is handed to lane k by a shuffle, so classification waits for no load of its own.
+template <int NPL, bool DIST>
 __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
@@ -407,10 +450,11 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
     // smallest index among its holders: equal logits go to the smaller expert index), then gates and classes of
     // the token's K entries follow in lanes 0..K-1.  A group's members are kept as a bit mask over the tokens.
     // NPL = elements per lane (N <= 32 NPL).
-    constexpr int TT = 2;
+    constexpr int TT = DIST ? 1 : 2;
+    const int t_first = DIST ? (int)blockIdx.x * AUX_W + a.aw : a.aw, t_pass = DIST ? (int)gridDim.x * AUX_W : AUX_W * TT;
 #pragma unroll 1
-    for (int t0 = a.aw; t0 < T; t0 += AUX_W * TT) {
-        float val[TT][NPL];
+    for (int t0 = t_first; t0 < T; t0 += t_pass) {
+        float val[TT][NPL], cf[TT][NPL];
         uint32_t key[TT][NPL];
 #pragma unroll
         for (int u = 0; u < TT; ++u) {
@@ -419,6 +463,7 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
             for (int m = 0; m < NPL; ++m) {
                 const int e = a.lane + 32 * m;
                 val[u][m] = (e < N && t < T) ? __ldcg(p.logits + (size_t)t * N + e) : 0.f;
+                if (DIST) cf[u][m] = (e < N && t < T && !p.roll_depth) ? __ldg(p.conf + (p.conf_stride ? (size_t)t * N + e : (size_t)t)) : 0.f;
             }
         }
 #pragma unroll
@@ -433,11 +478,12 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                 key[u][m] = e < N ? ((bts & 0x80000000u) ? ~bts : (bts | 0x80000000u)) : 0u;   // 0 is below every real key
             }
         int my_idx[TT];
-        float my_val[TT];
+        float my_val[TT], my_cf[TT];
 #pragma unroll
         for (int u = 0; u < TT; ++u) {
             my_idx[u] = 0;
             my_val[u] = 0.f;
+            my_cf[u] = 0.f;
         }
         if (key[0][0] != 1u) APROF(a, 75);
 #pragma unroll 1
@@ -462,12 +508,17 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                 widx[u] = (int)__reduce_min_sync(0xffffffffu, (unsigned)(bk[u] == wmax[u] ? bi[u] : 0x7fffffff));
 #pragma unroll
             for (int u = 0; u < TT; ++u) {
+                float wc = 0.f;   // DIST: the winner's confidence, from the lane that holds it
 #pragma unroll
-                for (int m = 0; m < NPL; ++m)
+                for (int m = 0; m < NPL; ++m) {
                     if (a.lane + 32 * m == widx[u]) key[u][m] = 0u;   // taken
+                    if (DIST && (widx[u] >> 5) == m) wc = cf[u][m];
+                }
+                if (DIST) wc = __shfl_sync(0xffffffffu, wc, widx[u] & 31);
                 if (a.lane == k) {
                     my_idx[u] = widx[u];
                     my_val[u] = __uint_as_float((wmax[u] & 0x80000000u) ? (wmax[u] ^ 0x80000000u) : ~wmax[u]);
+                    if (DIST) my_cf[u] = wc;
                 }
             }
         }
@@ -523,41 +574,76 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                     c = SPICE_MISS_EXACT;
                 } else if (sl >= 0) {
                     c = SPICE_HIT;
-                    atomicOr(&ax.mask_hit[2 * sl + (t >> 5)], 1u << (t & 31));
+                    if (!DIST) atomicOr(&ax.mask_hit[2 * sl + (t >> 5)], 1u << (t & 31));
                 } else {
                     bool low;
                     if (p.roll_depth) {
                         low = roll_cont;
                     } else {
                         const int ci = p.conf_stride ? t * N + e : t;
-                        const float cf = conf_staged(dm, p.conf_stride) ? ax.conf[ci] : __ldg(p.conf + ci);
-                        low = cf < p.tau;
+                        const float cfv = DIST ? my_cf[u] : (conf_staged(dm, p.conf_stride) ? ax.conf[ci] : __ldg(p.conf + ci));
+                        low = cfv < p.tau;
                     }
                     c = low ? SPICE_LOWCONF : SPICE_MISS_EXACT;
-                    if (low) atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
+                    if (low && !DIST) atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
                 }
-                ax.idx[i] = e;
-                ax.gate[i] = pk / denom;
-                ax.cls[i] = (unsigned char)c;
+                if (DIST) {
+                    p.idx[i] = e;
+                    p.gate[i] = pk / denom;
+                    p.cls[i] = (unsigned char)c;
+                } else {
+                    ax.idx[i] = e;
+                    ax.gate[i] = pk / denom;
+                    ax.cls[i] = (unsigned char)c;
+                }
             }
         }
     }
 }
 
-__device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
+// the routing of a batch is spread over the grid once a CTA would need more than two passes of its 8 warps (the extra
+// grid-wide hop costs about as much as one pass)
+__device__ __forceinline__ bool route_dist(const DecodeParams &p) { return p.dm.T > 4 * AUX_W && !p.roll_depth; }
+
+__device__ __forceinline__ bool aux_route(const DtcParams &q, Ctl *sh, const AuxSmem &ax, AuxCtx &a) {
     const DecodeParams &p = q.p;
     const Dims &dm = p.dm;
     const int T = dm.T, N = dm.N, K = dm.K, S = dm.S, n = T * K;
-    if (N <= 64) aux_route_tokens<2>(q, sh, ax, a);
-    else if (N <= 128) aux_route_tokens<4>(q, sh, ax, a);
-    else aux_route_tokens<8>(q, sh, ax, a);
+    if (route_dist(p)) {
+        if (N <= 64) aux_route_tokens<2, true>(q, sh, ax, a);
+        else if (N <= 128) aux_route_tokens<4, true>(q, sh, ax, a);
+        else aux_route_tokens<8, true>(q, sh, ax, a);
+        aux_sync();
+        if (a.atid == 0) {
+            int mine = 0;
+            for (int t = (int)blockIdx.x * AUX_W; t < T; t += (int)gridDim.x * AUX_W) mine += min(AUX_W, T - t);
+            if (mine) red_release_add(p.sync + SY_ROUTE_DONE, mine);
+        }
+        if (!aux_wait_ge(q, sh, a, p.sync + SY_ROUTE_DONE, T)) return false;
+        // every CTA collects all entries and rebuilds the groups' member masks
+#pragma unroll 1
+        for (int i = a.atid; i < n; i += AUX_T) {
+            const int e = __ldcg(p.idx + i), t = i / K;
+            const int c = __ldcg(p.cls + i);
+            ax.idx[i] = e;
+            ax.gate[i] = __ldcg(p.gate + i);
+            ax.cls[i] = (unsigned char)c;
+            if (c == SPICE_HIT) atomicOr(&ax.mask_hit[2 * ax.soe[e] + (t >> 5)], 1u << (t & 31));
+            else if (c == SPICE_LOWCONF) atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
+        }
+    } else {
+        if (N <= 64) aux_route_tokens<2, false>(q, sh, ax, a);
+        else if (N <= 128) aux_route_tokens<4, false>(q, sh, ax, a);
+        else aux_route_tokens<8, false>(q, sh, ax, a);
+    }
     aux_sync();
     APROF(a, 73);
     // groups: thread i owns slot i and expert i; packed scan of (entries, non-empty flag << 16)
     {
         const int ch = a.atid < S ? __popc(ax.mask_hit[2 * a.atid]) + __popc(ax.mask_hit[2 * a.atid + 1]) : 0;
         const int cl = a.atid < N ? __popc(ax.mask_low[2 * a.atid]) + __popc(ax.mask_low[2 * a.atid + 1]) : 0;
-        const int va = ch | ((ch > 0) << 16), vb = cl | ((cl > 0) << 16);
+        const bool fh = ch > 0 || a.atid < q.n_spec;   // a group (possibly without members)
+        const int va = ch | (fh << 16), vb = cl | ((cl > 0) << 16);
         int ia = va, ib = vb;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -586,7 +672,7 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
         const int n_hg = ta >> 16;
         if (a.atid < S) ax.off_hit[a.atid] = ea & 0xffff;
         if (a.atid < N) ax.off_low[a.atid] = eb & 0xffff;
-        if (ch > 0) ax.gtab[1 + (ea >> 16)] = GroupDesc{KIND_HIT, a.atid, ea & 0xffff, ch};
+        if (fh) ax.gtab[1 + (ea >> 16)] = GroupDesc{KIND_HIT, a.atid, ea & 0xffff, ch};
         if (cl > 0) ax.gtab[1 + n_hg + (eb >> 16)] = GroupDesc{KIND_LOW, a.atid, eb & 0xffff, cl};
         if (a.atid == AUX_T - 1) {   // this thread's inclusive sums are the totals
             sh->n_hg = n_hg;
@@ -628,17 +714,20 @@ __device__ __forceinline__ void aux_route(const DtcParams &q, Ctl *sh, const Aux
         ax.pos[i] = pos;
     }
     aux_sync();
+    return true;
 }
 
 // CTA 0: routing results for the caller (top-k, gates, classes, counts, residual-miss list in (t,k) order)
 __device__ __forceinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, const AuxSmem &ax, const AuxCtx &a) {
     const DecodeParams &p = q.p;
     const int K = p.dm.K, n = p.dm.T * K;
+    if (!route_dist(p)) {   // (else their owners wrote them)
 #pragma unroll 1
-    for (int i = a.atid; i < n; i += AUX_T) {
-        p.idx[i] = ax.idx[i];
-        p.gate[i] = ax.gate[i];
-        p.cls[i] = ax.cls[i];
+        for (int i = a.atid; i < n; i += AUX_T) {
+            p.idx[i] = ax.idx[i];
+            p.gate[i] = ax.gate[i];
+            p.cls[i] = ax.cls[i];
+        }
     }
     if (a.aw == 0) {
         int base = 0, n_hit = 0, n_low = 0;
@@ -767,6 +856,11 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         const size_t g = (size_t)blockIdx.x * DTC_THREADS + threadIdx.x, n_thr = (size_t)gridDim.x * DTC_THREADS;
         for (size_t l = g; l < n_lines; l += n_thr)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.w.w_router) + (l << 7)));
+        // so are the confidences where classification reads them from global memory
+        const size_t c_lines = (!p.roll_depth && (route_dist(p) || !conf_staged(dm, p.conf_stride)))
+                                   ? ((p.conf_stride ? (size_t)dm.T * dm.N : (size_t)dm.T) * 4 + 127) >> 7 : 0;
+        for (size_t l = n_thr - 1 - g; l < c_lines; l += n_thr)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.conf) + (l << 7)));
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS));
@@ -801,7 +895,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             uint32_t it = 0, tcount = 0;
             int s = 0;
             uint32_t ring_phase = 0;   // parity of the current pass over the ring
-            int end = pl.nA;
+            int end = pl.endB;   // (what is known at launch: the shared expert's tiles and the gate/up tiles of the first n_spec slots)
             bool ok = true;
             // ids: the first one is the CTA's index, every later one is drawn from a global counter.  The draw is
             // issued before the task's copies and used after them, so its latency hides behind the copies.
@@ -862,7 +956,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     ma = &maps.m[MAP_SLOT_GU];
                     mb = &maps.m[F8 ? MAP_X8 : MAP_H];
                     a_row0 = t.tile * 64;
-                    a_z = ax.gtab[t.gi].id;
+                    a_z = t.gi <= q.n_spec ? t.gi - 1 : ax.gtab[t.gi].id;   // (the group table may not exist yet)
                 } else if (id < pl.endB) {               // A_e tile of a low-confidence expert
                     const int l = id - pl.nA - pl.nBh;
                     t.kind = TASK_Z;
@@ -887,6 +981,10 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     b_z = t.gi - 1;
                     dep = SY_GROUP0 + t.gi;
                     dep_target = 2 * pl.tI;
+                    if (ax.gtab[t.gi].m == 0) {   // a slot that is a group without a token: nothing to multiply, the roles only count the tile
+                        t.nk = 0;
+                        dep = -1;
+                    }
                 } else {                                 // B_e tile of a low-confidence expert
                     const int l = id - c0 - pl.nCh;
                     t.kind = TASK_DOWN;
@@ -1125,7 +1223,9 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[buf]));   // accumulator is in registers now
             if (warp == 2 && lane == 0) DPROF(1, npf, 56);
-            const GroupDesc grp = t.gi == 0 ? GroupDesc{KIND_SHARED, 0, 0, T} : ax.gtab[t.gi];
+            // (a gate/up tile of one of the first n_spec slots may be finished before the group table exists)
+            const GroupDesc grp = t.gi == 0 ? GroupDesc{KIND_SHARED, 0, 0, T}
+                                            : (t.kind == TASK_ACT && t.gi <= q.n_spec ? GroupDesc{KIND_HIT, t.gi - 1, 0, 0} : ax.gtab[t.gi]);
             int *ctr = p.sync + SY_GROUP0 + t.gi;
             if (t.kind == TASK_ACT) {
                 const bool hit = grp.kind == KIND_HIT;
@@ -1197,30 +1297,41 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 for (int nn = 0; nn < NB; ++nn)
                     if (nn < T && row < dm.r) out[(size_t)nn * dm.r + row] = __float2bfloat16(__uint_as_float(v[nn]));
             } else {
-                // down tile: column n belongs to entry ent[n] (the token's (t,k) entry routed to this group) or to nobody
-                int *ent = ax.ent + qd * NB;
-                for (int nn = lane; nn < NB; nn += 32) ent[nn] = -1;
-                __syncwarp();
+                // down tile: token column n belongs to the group's entry of token n, if it has one.  The members are a bit
+                // mask over the tokens (warp-uniform tests with constant shifts, no table in shared memory), and the entry of
+                // member n is the rank(n)-th of the group's list, which is ordered by token.
+                uint32_t m0, m1 = 0u;
+                const int *perm = ax.perm_h;
                 if (grp.kind == KIND_SHARED) {
-                    for (int nn = lane; nn < T; nn += 32) ent[nn] = nn;
+                    m0 = T >= 32 ? 0xffffffffu : (1u << T) - 1u;
+                    if (NB > 32) m1 = T >= 64 ? 0xffffffffu : (T > 32 ? (1u << (T - 32)) - 1u : 0u);
                 } else {
-                    const int *perm = grp.kind == KIND_HIT ? ax.perm_h : ax.perm_l;
-                    for (int qq = lane; qq < grp.m; qq += 32) {
-                        const int i = perm[grp.off + qq];
-                        ent[i / dm.K] = i;
-                    }
+                    const uint32_t *mk = grp.kind == KIND_HIT ? ax.mask_hit + 2 * grp.id : ax.mask_low + 2 * grp.id;
+                    m0 = mk[0];
+                    if (NB > 32) m1 = mk[1];
+                    if (grp.kind != KIND_HIT) perm = ax.perm_l;
                 }
-                __syncwarp();
+                const int n0 = __popc(m0);
                 const int row = t.tile * 128 + L;
                 float *out = grp.kind == KIND_SHARED ? q.part_split + (size_t)t.split * T * dm.d : p.tb.part;
                 float rs = 1.0f;
                 if (F8 && t.f8 && row < dm.d) rs = grp.kind == KIND_SHARED ? q.s_sh_d[row] : q.s_slot_d[(size_t)grp.id * dm.d + row];
+                if (grp.kind == KIND_SHARED) {
 #pragma unroll
-                for (int nn = 0; nn < NB; ++nn) {
-                    const int e = ent[nn];
-                    if (e >= 0 && row < dm.d) out[(size_t)e * dm.d + row] = F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]);
+                    for (int nn = 0; nn < NB; ++nn)
+                        if (nn < T && row < dm.d) out[(size_t)nn * dm.d + row] = F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]);
+                } else {
+                    // (few columns are members: the store is a call, so that a column that is not costs a test and a
+                    // skipped branch instead of the predicated instructions of an inlined body)
+                    perm += grp.off;
+#pragma unroll
+                    for (int nn = 0; nn < NB; ++nn) {
+                        const uint32_t w = nn < 32 ? m0 : m1;
+                        if ((w >> (nn & 31)) & 1u)   // (warp-uniform)
+                            store_member_row(out, perm, nn < 32 ? __popc(m0 & ((1u << (nn & 31)) - 1u)) : n0 + __popc(m1 & ((1u << (nn & 31)) - 1u)),
+                                             dm.d, row, F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]));
+                    }
                 }
-                __syncwarp();   // ent[] is rewritten by the next down tile
             }
             if (warp == 2 && lane == 0) DPROF(1, npf, 57);
             if (t.kind == TASK_DOWN) {
@@ -1259,9 +1370,10 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         if (!p.roll_depth) {   // (the rollout decides the classes by its halting rule)
 #pragma unroll 1
             for (int i = a.atid; i < N; i += AUX_T) cp_async4(smem_u32(ax.soe + i), p.w.slot_of_expert + i);
+            if (conf_staged(dm, p.conf_stride)) {
 #pragma unroll 1
-            if (conf_staged(dm, p.conf_stride))
                 for (int i = a.atid; i < n_conf; i += AUX_T) cp_async4(smem_u32(ax.conf + i), p.conf + i);
+            }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
         if (a.atid < dm.S) ax.mask_hit[2 * a.atid] = ax.mask_hit[2 * a.atid + 1] = 0u;
@@ -1292,8 +1404,8 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         asm volatile("cp.async.wait_group 0;" ::: "memory");   // (made visible to the team by the barriers of the wait below)
         bool ok = aux_wait_ge(q, sh, a, p.sync + SY_R1_DONE, N * q.r1_sub);
         APROF(a, 63);
+        if (ok) ok = aux_route(q, sh, ax, a);
         if (ok) {
-            aux_route(q, sh, ax, a);
             if (a.atid == 0) mbar_arrive(smem_u32(&sh->plan_ready));
             APROF(a, 64);
             if (blockIdx.x == 0) aux_write_outputs(q, sh, ax, a);
@@ -1431,6 +1543,22 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
         const int per = (dm.T + AUX_W - 1) / AUX_W, fit = n_ctas / dm.N;
         q.r1_sub = per < 1 ? 1 : per;
         if (q.r1_sub > fit) q.r1_sub = fit < 1 ? 1 : fit;
+    }
+    {
+        // Slots whose gate/up tiles stream before the routing is known (Sec. 4.2 leaves the order of the expert work open).
+        // The routing tables exist 10 to 20 us into the kernel; until then only the shared expert's tiles are known, which
+        // for a small shared expert leaves most SMs without work.  Once the batch brings about 2.25 tokens per expert or
+        // more, nine slots in ten are used by some token, so the first n_spec slots are made groups unconditionally and their
+        // gate/up tiles join the launch-time part of the list: enough of them to fill about 20 us of the stream beside the
+        // shared expert.  A slot that no token chose costs its gate/up bytes (at most n_spec of S slots' worth).
+        q.n_spec = 0;
+        const double wb = f8 ? 1.0 : 2.0;
+        const double shared_bytes = 3.0 * dm.Is * dm.d * wb, slot_gu_bytes = 2.0 * dm.I * dm.d * wb;
+        const double window_bytes = f8 ? 72e6 : 128e6;   // (the 8-bit kernel streams fewer bytes per microsecond)
+        if (!p.roll_depth && 4ll * dm.T * dm.K >= 9ll * dm.N && (long long)dm.T * dm.K >= dm.S && window_bytes > shared_bytes) {
+            const int ns = (int)((window_bytes - shared_bytes) / slot_gu_bytes + 0.5);
+            q.n_spec = ns > dm.S ? dm.S : ns;
+        }
     }
     const int nb = nb_of(dm.T);
     const uint64_t T = dm.T, d = dm.d, I = dm.I, Is = dm.Is, r = dm.r;

@@ -278,3 +278,32 @@ def test_fp8_and_bf16_kernels_agree_on_random_shapes(seed):
         assert bool(torch.isfinite(ya).all()), tag
         assert (ya - yb).abs().max().item() <= 2.0 ** -7 * yb.abs().max().item() + 1e-6, tag
         L.close()
+
+
+@pytest.mark.parametrize("T", [27, 32])
+def test_fp8_slots_streamed_before_the_routing_is_known_but_chosen_by_no_token(T):
+    """The 8-bit kernel also streams the gate/up tiles of the first slots before the routing tables exist; with experts that
+    no token chose in those slots the outputs still match the oracle on the dequantised weights."""
+    wl = W.make_layer("dsv2lite", T, variant=61)
+    enforce_margins(wl)
+    s = wl.shape
+    idx, _ = oracle.topk_gates(oracle.router_logits(wl.h, wl.w_router), s.top_k, s.norm_topk)
+    used = np.zeros(s.n_experts, dtype=bool)
+    used[np.unique(idx)] = True
+    cold = [e for e in range(s.n_experts) if not used[e]][:3]
+    assert cold, "the batch uses every expert: pick another variant"
+    hot = [e for e in range(s.n_experts) if used[e]][: s.n_slots - len(cold)]
+    soe = np.full(s.n_experts, -1, dtype=np.int32)
+    for sl, e in enumerate(cold + hot):
+        soe[e] = sl
+    wl.set_residency(soe)
+    ref = run_oracle(_Dequantised(wl), want_full=False)
+    L = B.SpiceLayer(cfg_of(s), T)
+    w8 = B.quantize_layer(upload(wl))
+    out = L.moe_layer_fwd_fp8(w8, bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda())
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    check_routing(out, ref, T, s.top_k)
+    err, bound = y_close(out.y.float().cpu().numpy(), ref.y)
+    assert err <= bound, f"max err {err:.3e} > bound {bound:.3e}"
+    L.close()

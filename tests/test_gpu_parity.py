@@ -173,6 +173,42 @@ def test_moe_layer_fwd_matches_oracle(name, T):
     L.close()
 
 
+def _residency_with_unused_first_slots(wl, n_first):
+    """Residency in which the first slots hold experts that no token of the batch routes to (as many as there are, at
+    most n_first), the remaining slots experts that are used.  From the oracle's own routing."""
+    s = wl.shape
+    idx, _ = oracle.topk_gates(oracle.router_logits(wl.h, wl.w_router), s.top_k, s.norm_topk)
+    used = np.zeros(s.n_experts, dtype=bool)
+    used[np.unique(idx)] = True
+    cold = [e for e in range(s.n_experts) if not used[e]][:n_first]
+    hot = [e for e in range(s.n_experts) if used[e]][: s.n_slots - len(cold)]
+    soe = np.full(s.n_experts, -1, dtype=np.int32)
+    for sl, e in enumerate(cold + hot):
+        soe[e] = sl
+    wl.set_residency(soe)
+    return len(cold)
+
+
+@pytest.mark.parametrize("name,T,zipf", [("dsv2lite", 24, False), ("dsv2lite", 32, False), ("dsv2lite", 40, True),
+                                         ("dsv2lite", 64, True)])
+def test_slots_streamed_before_the_routing_is_known_but_chosen_by_no_token(name, T, zipf):
+    """From about 2.25 tokens per expert on, the decode kernel streams the gate/up tiles of the first slots before the
+    routing tables exist.  Here the first slots hold experts that no token chose: their tiles are computed and dropped,
+    their down tiles are empty, and every output still matches the oracle."""
+    wl = _layer_case(name, T, variant=9, zipf=zipf)   # (a skewed router leaves experts unused at the larger batches)
+    n_cold = _residency_with_unused_first_slots(wl, 3)
+    assert n_cold >= 1, "the batch uses every expert: pick another variant"
+    L, w, out, ref = _fwd_and_check(wl, want_full=False)
+    assert ref.counts[0] > 0
+    # the same call twice more: bit-identical (the empty groups leave no state behind)
+    h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+    for _ in range(2):
+        again = L.moe_layer_fwd(w, h, conf)
+        assert torch.equal(again.y, out.y) and torch.equal(again.cls, out.cls)
+    assert L.device_status() == 0
+    L.close()
+
+
 @pytest.mark.parametrize("name,T", [("tiny", 4), ("dsv2lite", 4), ("dsv2lite", 16)])
 def test_moe_layer_fwd_general_kernels_match_oracle(name, T):
     """The any-shape kernels (forced) against the oracle, and against the fused decode kernel."""
