@@ -48,6 +48,7 @@
 // such a task (the same 32 KB of weights as 128 bf16 elements).
 #include <cuda.h>
 #include <cuda_fp8.h>
+#include <cmath>
 
 #include "route_device.cuh"
 #include "spice_internal.cuh"
@@ -297,7 +298,7 @@ struct Plan {
     int tIs, tI, tz, td;            // tiles per matrix
     int kcd, kcI, kcr, kcdz;        // ring stages of d, I (expert matrices), r and d (LoRE factors)
     int nsplit, cps, kcIs;          // shared down projection: K ranges, chunks per range, chunks in all
-    int nA, nBh, endB, nCs, nCh, endC;
+    int nA, nSp, n_spec, nBh, endB, nCs, nCh, endC;
     int n_hg, n_lg;
     int sh_early;                   // the shared down tiles are part of phase A (else they follow phase B)
 };
@@ -319,17 +320,19 @@ __device__ __forceinline__ void plan_static(Plan &pl, const DtcParams &q, int ks
     // Before the routing is known only the shared expert can be worked on.  Its down tiles wait for ALL its
     // gate/up tiles, so they go first only when the CTAs that take them would have nothing else to do.
     pl.sh_early = (pl.tIs + pl.nCs <= (int)gridDim.x) ? 1 : 0;
-    pl.nA = pl.tIs + (pl.sh_early ? pl.nCs : 0);
-    // gate/up tiles of the slots that are groups regardless of the routing (the leading hit groups, in slot order)
+    // Known at launch, in this order: the shared expert's gate/up tiles, its early down tiles, the gate/up tiles of the
+    // slots that are groups regardless of the routing (the leading hit groups, in slot order).
+    pl.n_spec = q.n_spec;
+    pl.nSp = q.n_spec * pl.tI;
+    pl.nA = pl.tIs + (pl.sh_early ? pl.nCs : 0) + pl.nSp;
     pl.n_hg = q.n_spec;
-    pl.nBh = q.n_spec * pl.tI;
-    pl.n_lg = pl.nCh = 0;
-    pl.endB = pl.endC = pl.nA + pl.nBh;
+    pl.n_lg = pl.nBh = pl.nCh = 0;
+    pl.endB = pl.endC = pl.nA;
 }
 __device__ __forceinline__ void plan_routed(Plan &pl, int n_hg, int n_lg) {
     pl.n_hg = n_hg;
     pl.n_lg = n_lg;
-    pl.nBh = n_hg * pl.tI;
+    pl.nBh = (n_hg - pl.n_spec) * pl.tI;   // (the first n_spec groups' tiles are part of nA)
     pl.endB = pl.nA + pl.nBh + n_lg * pl.tz;
     pl.nCh = n_hg * pl.td;
     pl.endC = pl.endB + (pl.sh_early ? 0 : pl.nCs) + pl.nCh + n_lg * pl.td;
@@ -895,7 +898,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             uint32_t it = 0, tcount = 0;
             int s = 0;
             uint32_t ring_phase = 0;   // parity of the current pass over the ring
-            int end = pl.endB;   // (what is known at launch: the shared expert's tiles and the gate/up tiles of the first n_spec slots)
+            int end = pl.nA;   // (what is known at launch: the shared expert's tiles and the gate/up tiles of the first n_spec slots)
             bool ok = true;
             // ids: the first one is the CTA's index, every later one is drawn from a global counter.  The draw is
             // issued before the task's copies and used after them, so its latency hides behind the copies.
@@ -924,7 +927,8 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                 int a_row0, a_z = 0, b_z = 0, k0 = 0, dep = -1, dep_target = 0;
                 bool plain = false;   // operands with reduction length r: plain maps, one box per sub-chunk
                 const int c0 = pl.endB + (pl.sh_early ? 0 : pl.nCs);   // first down tile of a slot
-                const bool sh_down = pl.sh_early ? (id >= pl.tIs && id < pl.nA) : (id >= pl.endB && id < c0);
+                const int sp0 = pl.tIs + (pl.sh_early ? pl.nCs : 0);   // first gate/up tile of the slots that are groups regardless
+                const bool sh_down = pl.sh_early ? (id >= pl.tIs && id < sp0) : (id >= pl.endB && id < c0);
                 if (id < pl.tIs) {                       // gate/up tile of the shared expert
                     t.kind = TASK_ACT;
                     t.tile = id;
@@ -946,8 +950,8 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     a_row0 = t.tile * 128;
                     dep = SY_GROUP0;
                     dep_target = 2 * pl.tIs;
-                } else if (id < pl.nA + pl.nBh) {        // gate/up tile of a resident slot
-                    const int l = id - pl.nA;
+                } else if (id < pl.nA + pl.nBh) {        // gate/up tile of a resident slot (the others of the launch-time range are taken above)
+                    const int l = id < pl.nA ? id - sp0 : pl.nSp + id - pl.nA;
                     t.kind = TASK_ACT;
                     t.gi = 1 + l / pl.tI;
                     t.tile = l % pl.tI;
@@ -1546,16 +1550,18 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
     }
     {
         // Slots whose gate/up tiles stream before the routing is known (Sec. 4.2 leaves the order of the expert work open).
-        // The routing tables exist 10 to 20 us into the kernel; until then only the shared expert's tiles are known, which
-        // for a small shared expert leaves most SMs without work.  Once the batch brings about 2.25 tokens per expert or
-        // more, nine slots in ten are used by some token, so the first n_spec slots are made groups unconditionally and their
-        // gate/up tiles join the launch-time part of the list: enough of them to fill about 20 us of the stream beside the
-        // shared expert.  A slot that no token chose costs its gate/up bytes (at most n_spec of S slots' worth).
+        // The routing tables exist 8 to 20 us into the kernel; until then only the shared expert's tiles are known, which
+        // for a small shared expert leaves most SMs without work.  When a slot is left unused by the batch with probability
+        // 0.25 or less under uniform routing ((1 - K/N)^T: 15 tokens or more for 6 of 64 experts), the first n_spec slots are made
+        // groups unconditionally and their gate/up tiles join the launch-time part of the list: enough of them to fill
+        // about 20 us of the stream beside the shared expert.  A slot that no token chose costs its gate/up bytes (at most
+        // n_spec of S slots' worth, part of it in time that would have been idle).
         q.n_spec = 0;
         const double wb = f8 ? 1.0 : 2.0;
         const double shared_bytes = 3.0 * dm.Is * dm.d * wb, slot_gu_bytes = 2.0 * dm.I * dm.d * wb;
         const double window_bytes = f8 ? 72e6 : 128e6;   // (the 8-bit kernel streams fewer bytes per microsecond)
-        if (!p.roll_depth && 4ll * dm.T * dm.K >= 9ll * dm.N && (long long)dm.T * dm.K >= dm.S && window_bytes > shared_bytes) {
+        const double p_unused = pow(1.0 - (double)dm.K / dm.N, (double)dm.T);
+        if (!p.roll_depth && p_unused <= 0.25 && (long long)dm.T * dm.K >= dm.S && window_bytes > shared_bytes) {
             const int ns = (int)((window_bytes - shared_bytes) / slot_gu_bytes + 0.5);
             q.n_spec = ns > dm.S ? dm.S : ns;
         }

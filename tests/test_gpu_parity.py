@@ -189,11 +189,11 @@ def _residency_with_unused_first_slots(wl, n_first):
     return len(cold)
 
 
-@pytest.mark.parametrize("name,T,zipf", [("dsv2lite", 24, False), ("dsv2lite", 32, False), ("dsv2lite", 40, True),
-                                         ("dsv2lite", 64, True)])
+@pytest.mark.parametrize("name,T,zipf", [("dsv2lite", 16, False), ("dsv2lite", 24, False), ("dsv2lite", 32, False),
+                                         ("dsv2lite", 40, True), ("dsv2lite", 64, True)])
 def test_slots_streamed_before_the_routing_is_known_but_chosen_by_no_token(name, T, zipf):
-    """From about 2.25 tokens per expert on, the decode kernel streams the gate/up tiles of the first slots before the
-    routing tables exist.  Here the first slots hold experts that no token chose: their tiles are computed and dropped,
+    """Once a slot is unlikely to go unused (16 tokens on this shape), the decode kernel streams the gate/up tiles of the
+    first slots before the routing tables exist.  Here the first slots hold experts that no token chose: their tiles are computed and dropped,
     their down tiles are empty, and every output still matches the oracle."""
     wl = _layer_case(name, T, variant=9, zipf=zipf)   # (a skewed router leaves experts unused at the larger batches)
     n_cold = _residency_with_unused_first_slots(wl, 3)
