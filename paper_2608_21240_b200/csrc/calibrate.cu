@@ -414,11 +414,28 @@ __global__ void __launch_bounds__(256) qr_factor_kernel(const float *__restrict_
                                                         float *__restrict__ L, int32_t *flag) {
     __shared__ float a[TB][TB + 1];
     __shared__ float s_max;
-    for (int e = threadIdx.x; e < TB * TB; e += 256) {
-        float s = 0.f;
-        for (int b = 0; b < n_slabs; ++b) s += part[(size_t)b * TB * TB + e];
-        const int i = e / TB, j = e % TB;
-        a[i][j] = (i >= r || j >= r) ? (i == j ? 1.f : 0.f) : s;
+    // (four consecutive elements per thread and step, sixteen slabs' loads in flight; the sum stays in slab order)
+    for (int e = threadIdx.x * 4; e < TB * TB; e += 256 * 4) {
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int b0 = 0; b0 < n_slabs; b0 += 16) {
+            float4 v[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u)
+                v[u] = b0 + u < n_slabs ? __ldcg(reinterpret_cast<const float4 *>(part + (size_t)(b0 + u) * TB * TB + e))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                s.x += v[u].x;
+                s.y += v[u].y;
+                s.z += v[u].z;
+                s.w += v[u].w;
+            }
+        }
+        const int i = e / TB, j = e % TB;   // (j is a multiple of 4: the four elements share row i)
+        a[i][j] = (i >= r || j >= r) ? (i == j ? 1.f : 0.f) : s.x;
+        a[i][j + 1] = (i >= r || j + 1 >= r) ? (i == j + 1 ? 1.f : 0.f) : s.y;
+        a[i][j + 2] = (i >= r || j + 2 >= r) ? (i == j + 2 ? 1.f : 0.f) : s.z;
+        a[i][j + 3] = (i >= r || j + 3 >= r) ? (i == j + 3 ? 1.f : 0.f) : s.w;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -429,26 +446,38 @@ __global__ void __launch_bounds__(256) qr_factor_kernel(const float *__restrict_
     __syncthreads();
     if (jitter > 0.f && (int)threadIdx.x < r) a[threadIdx.x][threadIdx.x] += jitter * s_max;
     __syncthreads();
-    const int t = threadIdx.x & 63, pt = threadIdx.x >> 6;
-    for (int j = 0; j < TB; ++j) {
-        if (threadIdx.x == j) {
-            float p = a[j][j];
+    // Right-looking Cholesky by the first 64 threads, thread t holding row t of the lower triangle in registers.  Step j:
+    // every thread publishes its entry of column j, one barrier (the column buffers alternate, so a fast thread's next
+    // column cannot overwrite what a slow one still reads), then each thread scales by the same 1 / sqrt(pivot) -- its own
+    // entry and the entries of the rows above it -- and updates its row.  One barrier of two warps per step instead of three
+    // CTA-wide ones.
+    __shared__ float col[2][TB];
+    if (threadIdx.x < TB) {
+        const int t = threadIdx.x;
+        float row[TB];
+#pragma unroll
+        for (int c = 0; c < TB; ++c) row[c] = a[t][c];
+#pragma unroll
+        for (int j = 0; j < TB; ++j) {
+            float *cb = col[j & 1];
+            if (t >= j) cb[t] = row[j];
+            asm volatile("bar.sync 2, 64;" ::: "memory");
+            float p = cb[j];
             if (!(p > 0.f)) {
                 p = 1e-20f;
-                atomicOr(flag, 1);
+                if (t == j) atomicOr(flag, 1);
             }
-            a[j][j] = sqrtf(p);
+            const float inv = 1.0f / sqrtf(p);
+            if (t >= j) row[j] *= inv;   // (row j's own entry becomes sqrt(pivot) up to rounding)
+            const float ltj = row[j];
+#pragma unroll
+            for (int c = j + 1; c < TB; ++c)
+                if (c <= t) row[c] -= ltj * (cb[c] * inv);
         }
-        __syncthreads();
-        const float piv = a[j][j];
-        if (pt == 0 && t > j) a[t][j] /= piv;
-        __syncthreads();
-        if (t > j) {
-            const float ltj = a[t][j];
-            for (int c = j + 1 + ((pt - (j + 1)) & 3); c <= t; c += 4) a[t][c] -= ltj * a[c][j];
-        }
-        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < TB; ++c) a[t][c] = row[c];
     }
+    __syncthreads();
     for (int e = threadIdx.x; e < TB * TB; e += 256) {
         const int i = e / TB, j = e % TB;
         L[e] = j <= i ? a[i][j] : 0.f;
