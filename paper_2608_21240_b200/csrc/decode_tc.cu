@@ -286,10 +286,18 @@ __device__ __forceinline__ bool warp_mb_wait(uint32_t a, uint32_t parity, volati
     return ok;
 }
 
-// a down tile's value of one member column: row `row` of the entry that is the rank-th of the group's list
-__device__ __noinline__ void store_member_row(float *out, const int *perm, int rank, int d, int row, float val) {
-    const int e = perm[rank];
-    if (row < d) out[(size_t)e * d + row] = val;
+// v[nn] for a register array and an index known only at run time (the same in every lane): a tree of selects on the bits of nn
+template <int N>
+__device__ __forceinline__ uint32_t pick_column(const uint32_t (&v)[N], int nn) {
+    uint32_t s[N / 2];
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) s[i] = (nn & 1) ? v[2 * i + 1] : v[2 * i];
+#pragma unroll
+    for (int w = N / 4, bit = 2; w >= 1; w >>= 1, bit <<= 1) {
+#pragma unroll
+        for (int i = 0; i < w; ++i) s[i] = (nn & bit) ? s[2 * i + 1] : s[2 * i];
+    }
+    return s[0];
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1315,7 +1323,6 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     if (NB > 32) m1 = mk[1];
                     if (grp.kind != KIND_HIT) perm = ax.perm_l;
                 }
-                const int n0 = __popc(m0);
                 const int row = t.tile * 128 + L;
                 float *out = grp.kind == KIND_SHARED ? q.part_split + (size_t)t.split * T * dm.d : p.tb.part;
                 float rs = 1.0f;
@@ -1325,15 +1332,20 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     for (int nn = 0; nn < NB; ++nn)
                         if (nn < T && row < dm.d) out[(size_t)nn * dm.d + row] = F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]);
                 } else {
-                    // (few columns are members: the store is a call, so that a column that is not costs a test and a
-                    // skipped branch instead of the predicated instructions of an inlined body)
+                    // Few columns are members: a short loop over the set bits of the mask, the column's value picked out
+                    // of the accumulator registers by a tree of selects on the bits of its index.  (Sixty-four unrolled
+                    // tests with their stores were straight-line code of some 20 KB that every tile had to fetch again: 2 us
+                    // per tile, which bounded the tiny B_e tiles at the end of the list.)
                     perm += grp.off;
-#pragma unroll
-                    for (int nn = 0; nn < NB; ++nn) {
-                        const uint32_t w = nn < 32 ? m0 : m1;
-                        if ((w >> (nn & 31)) & 1u)   // (warp-uniform)
-                            store_member_row(out, perm, nn < 32 ? __popc(m0 & ((1u << (nn & 31)) - 1u)) : n0 + __popc(m1 & ((1u << (nn & 31)) - 1u)),
-                                             dm.d, row, F8 ? __uint_as_float(v[nn]) * rs : __uint_as_float(v[nn]));
+                    unsigned long long mm = (unsigned long long)m0 | ((unsigned long long)m1 << 32);
+                    int j = 0;
+#pragma unroll 1
+                    while (mm) {
+                        const int nn = __ffsll((long long)mm) - 1;
+                        mm &= mm - 1ull;
+                        const int e = perm[j++];
+                        const float val = __uint_as_float(pick_column<NB>(v, nn));
+                        if (row < dm.d) out[(size_t)e * dm.d + row] = F8 ? val * rs : val;
                     }
                 }
             }
