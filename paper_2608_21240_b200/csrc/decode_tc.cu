@@ -1563,18 +1563,21 @@ int launch_decode_tc(const DecodeParams &p, float *part_split, int n_ctas, int m
     {
         // Slots whose gate/up tiles stream before the routing is known (Sec. 4.2 leaves the order of the expert work open).
         // The routing tables exist 8 to 20 us into the kernel; until then only the shared expert's tiles are known, which
-        // for a small shared expert leaves most SMs without work.  When a slot is left unused by the batch with probability
-        // 0.25 or less under uniform routing ((1 - K/N)^T: 15 tokens or more for 6 of 64 experts), the first n_spec slots are made
-        // groups unconditionally and their gate/up tiles join the launch-time part of the list: enough of them to fill
-        // about 20 us of the stream beside the shared expert.  A slot that no token chose costs its gate/up bytes (at most
-        // n_spec of S slots' worth, part of it in time that would have been idle).
+        // for a small shared expert leaves most SMs without work.  The first n_spec slots are therefore made groups
+        // unconditionally and their gate/up tiles join the launch-time part of the list.  Their number: what fills about
+        // 20 us of the stream beside the shared expert, scaled down by how likely a slot is to go unused.  Measured per
+        // slot (DeepSeek-V2-Lite shape, 16 tokens, uniform and Zipf-skewed routers): a slot that is used shortens the call
+        // by 0.56 us, one that is not lengthens it by 0.91 us (its gate/up bytes, part of them in time that was idle), so
+        // streaming ahead pays while a slot goes unused with probability below 0.38.  Under uniform routing that
+        // probability is (1 - K/N)^T; real routers are more skewed, so the count shrinks linearly from the full window at
+        // probability 0 to nothing at 0.38 (16 tokens, 6 of 64 experts: 0.21, 4 of 8 slots; 32 tokens: 0.04, 7 slots).
         q.n_spec = 0;
         const double wb = f8 ? 1.0 : 2.0;
         const double shared_bytes = 3.0 * dm.Is * dm.d * wb, slot_gu_bytes = 2.0 * dm.I * dm.d * wb;
         const double window_bytes = f8 ? 72e6 : 128e6;   // (the 8-bit kernel streams fewer bytes per microsecond)
-        const double p_unused = pow(1.0 - (double)dm.K / dm.N, (double)dm.T);
-        if (!p.roll_depth && p_unused <= 0.25 && (long long)dm.T * dm.K >= dm.S && window_bytes > shared_bytes) {
-            const int ns = (int)((window_bytes - shared_bytes) / slot_gu_bytes + 0.5);
+        const double p_unused = pow(1.0 - (double)dm.K / dm.N, (double)dm.T), p_even = 0.38;
+        if (!p.roll_depth && p_unused < p_even && (long long)dm.T * dm.K >= dm.S && window_bytes > shared_bytes) {
+            const int ns = (int)((window_bytes - shared_bytes) / slot_gu_bytes * (1.0 - p_unused / p_even) + 0.5);
             q.n_spec = ns > dm.S ? dm.S : ns;
         }
     }
