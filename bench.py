@@ -36,8 +36,8 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu captures summarised under
 # profiles/ (same workload with 2 weight sets; mean of the two captured launches), keyed by (shape, tokens, path)
-CAPTURED_TRAFFIC = {("dsv2lite", 16, 0, "bf16"): (507.2e6, "profiles/decode_tc_kernel_dsv2lite_T16.md"),
-                    ("dsv2lite", 16, 0, "fp8"): (262.2e6, "profiles/decode_tc_kernel_fp8.md")}
+CAPTURED_TRAFFIC = {("dsv2lite", 16, 0, "bf16"): (502.9e6, "profiles/decode_tc_kernel_dsv2lite_T16.md"),
+                    ("dsv2lite", 16, 0, "fp8"): (259.1e6, "profiles/decode_tc_kernel_fp8.md")}
 
 
 def load_peaks():
