@@ -256,9 +256,11 @@ def test_moe_layer_fwd_ragged_token_counts_and_dims(T):
     L.close()
 
 
-def test_expired_dependency_wait_reports_timeout_and_recovers():
-    """A wait that cannot be satisfied within its poll limit ends the kernel with a status, not a hang."""
-    wl = _layer_case("dsv2lite", 16, variant=11)
+@pytest.mark.parametrize("T", [16, 48])
+def test_expired_dependency_wait_reports_timeout_and_recovers(T):
+    """A wait that cannot be satisfied within its poll limit ends the kernel with a status, not a hang.  (48 tokens: the
+    routing is spread over the grid and slots stream ahead of it, so the wait runs out with tiles in flight.)"""
+    wl = _layer_case("dsv2lite", T, variant=11)
     s = wl.shape
     L = B.SpiceLayer(cfg_of(s), wl.T)
     w = upload(wl)
