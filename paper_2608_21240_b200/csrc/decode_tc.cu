@@ -102,7 +102,7 @@ struct Ctl {
     unsigned long long tmem_full[2], tmem_empty[2];
     unsigned long long tq_full[TQ], tq_empty[TQ];
     unsigned long long xch_full[2], xch_empty[2];
-    unsigned long long plan_ready, mma_drain;
+    unsigned long long plan_ready, mma_drain, logits_done;
     TaskDesc tq[TQ];
     uint32_t tmem_base;
     int abort_flag;
@@ -853,6 +853,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             mbar_init(smem_u32(&sh->tq_empty[s]), 5);
         }
         mbar_init(smem_u32(&sh->plan_ready), 1);
+        mbar_init(smem_u32(&sh->logits_done), 1);
         mbar_init(smem_u32(&sh->mma_drain), 1);
         sh->abort_flag = 0;
         sh->aux_flag = 0;
@@ -911,6 +912,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
             // ids: the first one is the CTA's index, every later one is drawn from a global counter.  The draw is
             // issued before the task's copies and used after them, so its latency hides behind the copies.
             int id = blockIdx.x;
+            bool logits_seen = false;   // this CTA's router-logit units are done (only asked before the routing is known)
             bool h8_ok = false;   // (8-bit weights) the three-term copy of h is complete
             const uint64_t w_policy = l2_policy_evict_first();
             auto lead_wait = [&](uint32_t bar, uint32_t parity) {   // lane 0 waits, the outcome is uniform
@@ -1011,6 +1013,12 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
                     b_z = t.gi - 1 - pl.n_hg;
                     dep = SY_GROUP0 + t.gi;
                     dep_target = 4 * pl.tz;
+                }
+                // A gate/up tile streamed ahead of the routing must not delay the routing itself: the loads of the CTA's
+                // router-logit units would queue behind the tile's copies, so the tile waits for them.
+                if (!routed && t.kind == TASK_ACT && t.gi > 0 && (int)gridDim.x - 1 - (int)blockIdx.x < p.dm.N * q.r1_sub && !logits_seen) {
+                    if (!lead_wait(smem_u32(&sh->logits_done), 0)) { ok = false; break; }
+                    logits_seen = true;
                 }
                 if (lane == 0) DPROF(0, npf, 10 + t.kind);
                 // this lane's copy of every stage: lane 0 the weights, lane 1 the tokens (sub-chunk 0 only when the
@@ -1416,6 +1424,7 @@ __global__ void __launch_bounds__(DTC_THREADS, 1) decode_tc_kernel(const __grid_
         } else {
             aux_logits(q, a);
         }
+        if (a.atid == 0) mbar_arrive(smem_u32(&sh->logits_done));   // (after the barrier inside aux_logits, if it had units)
         APROF(a, 62);
         asm volatile("cp.async.wait_group 0;" ::: "memory");   // (made visible to the team by the barriers of the wait below)
         bool ok = aux_wait_ge(q, sh, a, p.sync + SY_R1_DONE, N * q.r1_sub);
