@@ -22,12 +22,16 @@
 //               paired through shared memory) or plain; stores; release of the task's counter
 //   warps 6-13  auxiliary team: router logits (its share), then the routing decisions computed
 //               REDUNDANTLY by every CTA from the logits (top-k, gates, classification, grouping):
-//               the tables land in shared memory without a second grid-wide hop; finally the combine
+//               the tables land in shared memory without a second grid-wide hop (batches of more than
+//               32 tokens: each token is routed by one warp of the grid and every CTA collects the
+//               entries after one more counter); finally the combine
 //
 // Tasks (a CTA starts with the id of its index and draws every further id from a global counter; a task
 // depends only on tasks with smaller ids, and every CTA issues its tasks in increasing order):
 //   A  gate/up tile of the shared expert: 64 gate + 64 up rows, K = d              (no dependency)
 //      down tile of the shared expert: 128 rows, one K range                       (the A gate/up tiles)
+//      gate/up tiles of the first n_spec slots, streamed before the routing is known when a slot is
+//      unlikely to go unused (see launch_decode_tc); such a slot is a group even without a token
 //   B  gate/up tile of a resident slot; A_e tile of a low-confidence expert        (routing)
 //   C  down tile, 128 rows, of a slot; B_e tile                                    (that group's B tiles)
 //   D  combine y_t = c_t S(h_t) + sum_k g_k part_{t,k}  (auxiliary teams)          (all C tiles)
