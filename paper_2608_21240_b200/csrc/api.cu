@@ -189,6 +189,9 @@ DecodeParams decode_params_of(const spice_ctx *ctx, const Dims &dm) {
     p.act_shared16 = ctx->act_shared16;
     p.z16 = ctx->z16;
     p.sync = ctx->sync;
+    p.x_idx = ctx->ws_idx;
+    p.x_gate = ctx->ws_gate;
+    p.x_cls = ctx->ws_cls;
     return p;
 }
 

@@ -451,7 +451,7 @@ __device__ __forceinline__ void aux_split_h(const DtcParams &q, const AuxCtx &a,
 // (the code is deterministic: counts by atomics, positions by ranking); CTA 0 also writes the outputs.
 // The arithmetic of the gates is that of warp_topk_gates (route_device.cuh).
 // DIST: the batch is spread over the grid instead (CTA c takes tokens 8c .. 8c+7, a warp one token), the warp writes its
-// token's entries to the caller's idx / gate / cls arrays and every CTA collects all of them afterwards (aux_route): per
+// token's entries to the context's exchange arrays and every CTA collects all of them afterwards (aux_route): per
 // CTA the work no longer grows with the batch.  The token's confidences then travel with its logits (same indexing, one
 // coalesced load) and the winner's value is handed to lane k by a shuffle, so classification waits for no load of its own.
 template <int NPL, bool DIST>
@@ -603,9 +603,9 @@ __device__ __forceinline__ void aux_route_tokens(const DtcParams &q, Ctl *sh, co
                     if (low && !DIST) atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
                 }
                 if (DIST) {
-                    p.idx[i] = e;
-                    p.gate[i] = pk / denom;
-                    p.cls[i] = (unsigned char)c;
+                    p.x_idx[i] = e;
+                    p.x_gate[i] = pk / denom;
+                    p.x_cls[i] = (unsigned char)c;
                 } else {
                     ax.idx[i] = e;
                     ax.gate[i] = pk / denom;
@@ -638,10 +638,10 @@ __device__ __forceinline__ bool aux_route(const DtcParams &q, Ctl *sh, const Aux
         // every CTA collects all entries and rebuilds the groups' member masks
 #pragma unroll 1
         for (int i = a.atid; i < n; i += AUX_T) {
-            const int e = __ldcg(p.idx + i), t = i / K;
-            const int c = __ldcg(p.cls + i);
+            const int e = __ldcg(p.x_idx + i), t = i / K;
+            const int c = __ldcg(p.x_cls + i);
             ax.idx[i] = e;
-            ax.gate[i] = __ldcg(p.gate + i);
+            ax.gate[i] = __ldcg(p.x_gate + i);
             ax.cls[i] = (unsigned char)c;
             if (c == SPICE_HIT) atomicOr(&ax.mask_hit[2 * ax.soe[e] + (t >> 5)], 1u << (t & 31));
             else if (c == SPICE_LOWCONF) atomicOr(&ax.mask_low[2 * e + (t >> 5)], 1u << (t & 31));
@@ -736,13 +736,15 @@ __device__ __forceinline__ bool aux_route(const DtcParams &q, Ctl *sh, const Aux
 __device__ __forceinline__ void aux_write_outputs(const DtcParams &q, Ctl *sh, const AuxSmem &ax, const AuxCtx &a) {
     const DecodeParams &p = q.p;
     const int K = p.dm.K, n = p.dm.T * K;
-    if (!route_dist(p)) {   // (else their owners wrote them)
+    // (a spread routing was exchanged through the context's arrays: an output that IS such an array is written already,
+    // and other CTAs may still be reading it)
+    const bool dist = route_dist(p);
+    const bool w_idx = !dist || p.idx != p.x_idx, w_gate = !dist || p.gate != p.x_gate, w_cls = !dist || p.cls != p.x_cls;
 #pragma unroll 1
-        for (int i = a.atid; i < n; i += AUX_T) {
-            p.idx[i] = ax.idx[i];
-            p.gate[i] = ax.gate[i];
-            p.cls[i] = ax.cls[i];
-        }
+    for (int i = a.atid; i < n; i += AUX_T) {
+        if (w_idx) p.idx[i] = ax.idx[i];
+        if (w_gate) p.gate[i] = ax.gate[i];
+        if (w_cls) p.cls[i] = ax.cls[i];
     }
     if (a.aw == 0) {
         int base = 0, n_hit = 0, n_low = 0;

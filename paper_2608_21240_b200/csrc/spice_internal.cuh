@@ -131,6 +131,11 @@ struct DecodeParams {
     int32_t *counts;
     int32_t *resid_tok, *resid_k, *resid_expert;
     float *resid_gate;
+    // the context's own [Tm*K] arrays: where the tcgen05 decode kernel exchanges the routing of a batch that it spreads
+    // over the grid (the caller's idx / gate / cls may be mapped host memory and are only ever written)
+    int32_t *x_idx;
+    float *x_gate;
+    uint8_t *x_cls;
     __nv_bfloat16 *y16;
     const float *y_cpu;
     __nv_bfloat16 *x_resid;

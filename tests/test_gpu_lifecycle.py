@@ -76,3 +76,32 @@ def test_calls_on_another_stream_give_the_same_bits():
         assert torch.equal(a.y, b.y) and torch.equal(a.idx, b.idx) and torch.equal(a.counts, b.counts)
         assert L.device_status() == 0
         L.close()
+
+
+def test_spread_routing_with_outputs_in_pinned_host_memory_or_not_wanted():
+    """At more than 32 tokens the decode kernel exchanges the routing between thread blocks through the context's own arrays;
+    the caller's idx / gate / cls are only written: they may live in pinned host memory, and y does not depend on whether
+    they were asked for."""
+    s = W.SHAPES["dsv2lite"]
+    T = 48
+    wl = W.make_layer(s, T, variant=520)
+    w = upload(wl)
+    L = B.SpiceLayer(cfg_of(s), T)
+    h, conf = bf16_tensor(wl.h), torch.from_numpy(wl.conf).cuda()
+    ref = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    n = T * s.top_k
+    idx = torch.empty(n, dtype=torch.int32).pin_memory()
+    gate = torch.empty(n, dtype=torch.float32).pin_memory()
+    cls = torch.empty(n, dtype=torch.uint8).pin_memory()
+    y = torch.empty(T, s.d, dtype=torch.bfloat16, device="cuda")
+    B.spice_moe_layer_fwd(L.ctx, w.c_struct(), h, conf, T, y, idx=idx, gate=gate, cls=cls)
+    torch.cuda.synchronize()
+    assert torch.equal(y, ref.y)
+    assert torch.equal(idx.view(T, -1), ref.idx.cpu().view(T, -1)) and torch.equal(gate.view(T, -1), ref.gate.cpu().view(T, -1))
+    assert torch.equal(cls.view(T, -1), ref.cls.cpu().view(T, -1))
+    y2 = torch.empty_like(y)
+    B.spice_moe_layer_fwd(L.ctx, w.c_struct(), h, conf, T, y2)
+    torch.cuda.synchronize()
+    assert torch.equal(y2, ref.y) and L.device_status() == 0
+    L.close()
