@@ -205,6 +205,12 @@ def test_slots_streamed_before_the_routing_is_known_but_chosen_by_no_token(name,
     for _ in range(2):
         again = L.moe_layer_fwd(w, h, conf)
         assert torch.equal(again.y, out.y) and torch.equal(again.cls, out.cls)
+    # whatever the unused slots hold never reaches an output: NaN weights in them change nothing
+    w.slot_w_gate_up[:n_cold] = float("nan")
+    w.slot_w_down[:n_cold] = float("nan")
+    poisoned = L.moe_layer_fwd(w, h, conf)
+    torch.cuda.synchronize()
+    assert torch.equal(poisoned.y, out.y) and bool(torch.isfinite(poisoned.y.float()).all())
     assert L.device_status() == 0
     L.close()
 
